@@ -1,0 +1,219 @@
+/*
+ * aquakv.h -- C ABI of the B200 (sm_100a) AQUA-KV per-token KV-cache codec.
+ *
+ * The operations are those of the paper "Cache Me If You Must: Adaptive Key-Value Quantization
+ * for Large Language Models": Algorithm 2 (encode), Algorithm 3 (decode) and the attention read
+ * of Algorithm 4 (lines 5-9), with the backbone quantizer Q of Section 2 ("Vector Quantization")
+ * and Section 4.1 ("Alternative quantizers"): group-wise vector quantization after a randomized
+ * Hadamard transform, p = 2 values per code, n in {16, 64, 256} grid points, one fp16 scale per
+ * group.
+ *
+ * Conventions shared by every entry point
+ *   - Every data pointer is a DEVICE pointer owned by the caller unless its name ends in _host.
+ *     The library allocates nothing per call; it uses only the caller's workspace.
+ *   - 16-bit tensors (K, V, reconstructions, adapter matrices, queries, attention output) are
+ *     fp16 or bf16 as chosen in aquakv_params.dtype; all of them share that type.
+ *   - Token-major layout: row t holds the d_kv = n_kv_heads * head_dim values of token t,
+ *     consecutive in memory; rows are `ld` ELEMENTS apart (ld >= d_kv, ld % 8 == 0).  Base
+ *     pointers of 16-bit tensors and of the workspace are 16-byte aligned.
+ *   - Adapter (predictor) matrices are row-major [out_features][in_features] like a linear
+ *     layer's weight: pred[c] = sum_r x[r] * W[c][r] (+ bias[c]).  Wk is [d_kv][d_kv]; Wv is
+ *     [d_kv][2*d_kv] and its input is the concatenation [Vhat_prev ; Khat] (columns 0..d_kv-1
+ *     act on Vhat_prev, columns d_kv..2*d_kv-1 on the freshly reconstructed Khat).  Biases are
+ *     optional fp32 [d_kv] (NULL = none).  Wk == NULL (then Wv, Khat_prev, Vhat_prev must be NULL
+ *     too) selects the predictor-free path of layer 0 (Algorithm 2 lines 1-3).
+ *   - Compressed cache, per tensor (keys and values are separate arrays), per token t:
+ *       codes[t]  : d_kv/2 * log2(n) / 8 bytes; the code of value pair j (values 2j, 2j+1 of the
+ *                   rotated row) occupies bits [j*log2(n), (j+1)*log2(n)) of the row's bit
+ *                   stream, least significant bit first (n = 16: two codes per byte, low nibble
+ *                   = even pair; n = 64: four codes per three bytes; n = 256: one byte each);
+ *       scales[t] : d_kv/scale_group IEEE fp16 bit patterns, the group's root-mean-square
+ *                   residual rounded to nearest even.
+ *     Bits per value = log2(n)/2 + 16/scale_group (2.02 at n = 16, group 1024).
+ *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream).  They never synchronise, print, abort or throw.  Every function
+ *     returning int returns AQUAKV_OK or a negative AQUAKV_ERR_* code; argument errors are
+ *     detected on the host before anything is launched.  n_tokens == 0 is AQUAKV_OK, no launch.
+ *   - Non-finite inputs are memory-safe; the resulting codes/scales are unspecified.
+ *   - A context may be used from one host thread at a time, on the device that was current
+ *     when it was created.
+ */
+#ifndef AQUAKV_H_
+#define AQUAKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AQUAKV_F16 0
+#define AQUAKV_BF16 1
+
+#define AQUAKV_OK 0
+#define AQUAKV_ERR_INVALID_ARG (-1) /* NULL where data is required, negative size, aliasing */
+#define AQUAKV_ERR_UNSUPPORTED (-2) /* a parameter combination the kernels do not cover      */
+#define AQUAKV_ERR_ALIGNMENT (-3)   /* pointer not 16-byte aligned or ld not a multiple of 8 */
+#define AQUAKV_ERR_WORKSPACE (-4)   /* workspace NULL or smaller than aquakv_workspace_bytes */
+#define AQUAKV_ERR_CUDA (-5)        /* a CUDA runtime/driver call failed                     */
+#define AQUAKV_ERR_TIMEOUT (-6)     /* a bounded device-side wait expired (see poll_status)  */
+
+#define AQUAKV_OP_ENCODE 0
+#define AQUAKV_OP_DECODE 1
+#define AQUAKV_OP_DECODE_ATTN 2
+
+/* Parameters of the quantizer Q (Section 4.1: group size, p, n) and of the tensors. */
+typedef struct aquakv_params {
+  int32_t d_kv;        /* values per token row; supported: 256, 512, 1024                       */
+  int32_t had_block;   /* h: Hadamard block, power of two, 64 <= h <= d_kv, divides d_kv        */
+  int32_t scale_group; /* g: values per fp16 scale; multiple of h that divides d_kv             */
+  int32_t grid_dim;    /* p: values per code; must be 2                                         */
+  int32_t grid_size;   /* n: 16, 64 or 256 grid points (2, 3, 4 bits per value)                 */
+  int32_t dtype;       /* AQUAKV_F16 or AQUAKV_BF16                                             */
+} aquakv_params;
+
+typedef struct aquakv_ctx aquakv_ctx; /* opaque; owns the device copies of grid, signs, status */
+
+/* Bytes of one token's codes for these parameters (d_kv/2 * log2(n) / 8), or a negative error. */
+int aquakv_code_bytes(const aquakv_params* params);
+
+/*
+ * Creates a context on the current device.  grid_host: n x 2 floats, the fixed grid of Section 2
+ * ("a lattice optimized for normally distributed vectors"), index = code.  signs_k_host /
+ * signs_v_host: d_kv values in {+1,-1}, the random diagonal of the randomized Hadamard transform
+ * for keys and for values.  All three are copied; the caller may free them after the call.
+ * This is the only entry point that allocates device memory (a few KB) and it synchronises the
+ * device once.  Errors: INVALID_ARG (NULL, sign not +-1, non-finite grid), UNSUPPORTED, CUDA.
+ */
+int aquakv_create(const aquakv_params* params, const float* grid_host, const int8_t* signs_k_host,
+                  const int8_t* signs_v_host, aquakv_ctx** out);
+
+/* Frees the context's device tables.  NULL is accepted.  Pending work must have completed. */
+int aquakv_destroy(aquakv_ctx* ctx);
+
+/*
+ * Workspace the caller must provide to the given operation for n_tokens tokens (bytes, 16-byte
+ * aligned base).  It is bounded: large calls are processed in token chunks sized so that the
+ * intermediate prediction stays resident in the B200's L2 cache.  Returns 0 for n_tokens <= 0,
+ * for an unknown op and for AQUAKV_OP_DECODE_ATTN (use aquakv_decode_attn_workspace_bytes).
+ */
+size_t aquakv_workspace_bytes(const aquakv_ctx* ctx, int64_t n_tokens, int op);
+
+/*
+ * Workspace of aquakv_decode_attn for this problem shape (its split-KV partials depend on the
+ * batch and head counts, which aquakv_workspace_bytes does not see).  0 on invalid arguments.
+ */
+size_t aquakv_decode_attn_workspace_bytes(const aquakv_ctx* ctx, int32_t batch, int64_t ctx_len,
+                                          int32_t n_q_heads, int32_t head_dim);
+
+/*
+ * The predictor alone (Section 3.2: f_key, f_value are linear regressors; Algorithm 2 lines 5
+ * and 8):  P[t][c] = sum_r x_t[r] * W[c][r] + bias[c]  with x_t = in0[t] (in1 == NULL, W is
+ * [d_kv][d_kv]) or the concatenation [in0[t] ; in1[t]] (W is [d_kv][2*d_kv]).  P is fp32
+ * [n_tokens, ldP] (ldP % 4 == 0, 16-byte aligned); accumulation is fp32 on the tensor cores.
+ * Needs no workspace.
+ */
+int aquakv_predict(aquakv_ctx* ctx, int64_t n_tokens, const void* in0, const void* in1,
+                   int64_t ld_in, const void* W, const float* bias, float* P, int64_t ldP,
+                   void* cuda_stream);
+
+#define AQUAKV_ROLE_KEY 0
+#define AQUAKV_ROLE_VALUE 1
+
+/*
+ * One phase of Algorithm 2 on its own (lines 5-7 for keys; lines 8-9 plus the reconstruction for
+ * values), for callers that supply the predictor inputs themselves (e.g. teacher-forced checks):
+ *   pred = [in0 ; in1] W^T + bias;  codes,scales = Q(X - pred);  hat = round16(Q^-1(..) + pred).
+ * role selects the Hadamard signs (AQUAKV_ROLE_KEY / AQUAKV_ROLE_VALUE).  in1 == NULL: single
+ * input, W is [d_kv][d_kv]; otherwise W is [d_kv][2*d_kv].  W == NULL (then in0, in1, bias NULL):
+ * no predictor.  hat may be NULL.  Workspace as for AQUAKV_OP_ENCODE (needed only with W).
+ */
+int aquakv_encode_phase(aquakv_ctx* ctx, int role, int64_t n_tokens, const void* X, int64_t ld_x,
+                        const void* in0, const void* in1, int64_t ld_in, const void* W,
+                        const float* bias, uint8_t* codes, uint16_t* scales, void* hat,
+                        int64_t ld_hat, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * One phase of Algorithm 3 on its own (line 5 for keys, line 7 for values):
+ *   hat = round16(Q^-1(codes, scales) + [in0 ; in1] W^T + bias).  Arguments as above.
+ */
+int aquakv_decode_phase(aquakv_ctx* ctx, int role, int64_t n_tokens, const uint8_t* codes,
+                        const uint16_t* scales, const void* in0, const void* in1, int64_t ld_in,
+                        const void* W, const float* bias, void* hat, int64_t ld_hat,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Algorithm 2 (encode) for one layer and n_tokens tokens:
+ *   K_pred = Khat_prev Wk^T + bk;  Kcodes,Kscales = Q(K - K_pred);  Khat = Q^-1(..) + K_pred;
+ *   V_pred = [Vhat_prev ; Khat] Wv^T + bv;  Vcodes,Vscales = Q(V - V_pred);  Vhat = Q^-1(..) + V_pred.
+ * The reconstructions Khat/Vhat (rounded once to the 16-bit type) are what Algorithm 4 line 14
+ * obtains by decoding the fresh codes again; here they are by-products.  Khat, Vhat may be NULL
+ * (not written; Khat is then kept in the workspace for the value predictor).  Outputs must not
+ * alias inputs.  K,V: [n_tokens, ld_kv]; *_prev: [n_tokens, ld_prev]; Khat,Vhat: [n_tokens, ld_hat].
+ */
+int aquakv_encode(aquakv_ctx* ctx, int64_t n_tokens,
+                  const void* K, const void* V, int64_t ld_kv,
+                  const void* Khat_prev, const void* Vhat_prev, int64_t ld_prev,
+                  const void* Wk, const void* Wv, const float* bk, const float* bv,
+                  uint8_t* Kcodes, uint16_t* Kscales, uint8_t* Vcodes, uint16_t* Vscales,
+                  void* Khat, void* Vhat, int64_t ld_hat,
+                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Algorithm 3 (decode) for one layer:
+ *   Khat = Q^-1(Kcodes,Kscales) + Khat_prev Wk^T + bk;
+ *   Vhat = Q^-1(Vcodes,Vscales) + [Vhat_prev ; Khat] Wv^T + bv,
+ * each rounded once to the 16-bit type.  On the same device, with the same arguments, Khat/Vhat
+ * are bit-identical to those aquakv_encode produced (Algorithm 2 line 7 and Algorithm 3 line 5
+ * are the same expression).  Khat and Vhat are required.
+ */
+int aquakv_decode(aquakv_ctx* ctx, int64_t n_tokens,
+                  const uint8_t* Kcodes, const uint16_t* Kscales,
+                  const uint8_t* Vcodes, const uint16_t* Vscales,
+                  const void* Khat_prev, const void* Vhat_prev, int64_t ld_prev,
+                  const void* Wk, const void* Wv, const float* bk, const float* bv,
+                  void* Khat, void* Vhat, int64_t ld_hat,
+                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Algorithm 3 fused with the attention read of Algorithm 4 (lines 5-9) for single-token queries:
+ * decodes `batch` sequences of `ctx_len` cached tokens each (token index = b*ctx_len + t,
+ * n_tokens = batch*ctx_len) and computes, per sequence b and query head qh,
+ *   out[b][qh] = softmax_t(softmax_scale * q[b][qh] . Khat[b,t][kvh]) . Vhat[b,t][kvh],
+ * kvh = qh / (n_q_heads / n_kv_heads) (grouped-query attention), accumulating in fp32.
+ * n_kv_heads * head_dim must equal d_kv; head_dim must be 64 or 128; n_q_heads a multiple of
+ * n_kv_heads with n_q_heads/n_kv_heads <= 8.  q, out: [batch][n_q_heads][head_dim] 16-bit,
+ * contiguous.  lse: optional fp32 [batch][n_q_heads] log-sum-exp of the scaled scores (NULL =
+ * not written).  Khat, Vhat: optional outputs [n_tokens, ld_hat] for the next layer's decode
+ * (NULL = the reconstruction lives only in the workspace, chunk by chunk).
+ */
+int aquakv_decode_attn(aquakv_ctx* ctx, int32_t batch, int64_t ctx_len,
+                       int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, float softmax_scale,
+                       const void* q,
+                       const uint8_t* Kcodes, const uint16_t* Kscales,
+                       const uint8_t* Vcodes, const uint16_t* Vscales,
+                       const void* Khat_prev, const void* Vhat_prev, int64_t ld_prev,
+                       const void* Wk, const void* Wv, const float* bk, const float* bv,
+                       void* out, float* lse,
+                       void* Khat, void* Vhat, int64_t ld_hat,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Synchronises `cuda_stream` and returns the context's device status word: AQUAKV_OK, or
+ * AQUAKV_ERR_TIMEOUT if a bounded wait inside a kernel (on a TMA or tensor-core completion
+ * barrier) expired since the last poll, in which case that call's outputs are invalid.  The word
+ * is cleared by the poll.  AQUAKV_ERR_CUDA if the stream reports an error.
+ */
+int aquakv_poll_status(aquakv_ctx* ctx, void* cuda_stream);
+
+/* Number of kernels this context has launched since creation (for benchmarks' bookkeeping). */
+int64_t aquakv_launch_count(const aquakv_ctx* ctx);
+
+/* Static, human-readable name of a status code. */
+const char* aquakv_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AQUAKV_H_ */

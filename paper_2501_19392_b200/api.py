@@ -1,0 +1,257 @@
+"""Thin Python binding of libaquakv.so (the C ABI in include/aquakv.h).
+
+Argument marshalling only: torch supplies device memory and the current stream; every step of
+encode / decode / decode-attention runs in the library's CUDA kernels.  There is no CPU or
+PyTorch fallback: importing this module without the built library raises, and every call
+raises `AquaKVError` on a non-zero status.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+F16 = 0
+BF16 = 1
+OP_ENCODE = 0
+OP_DECODE = 1
+OP_DECODE_ATTN = 2
+ROLE_KEY = 0
+ROLE_VALUE = 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libaquakv.so")
+
+SYMBOLS = [
+    "aquakv_code_bytes", "aquakv_create", "aquakv_destroy", "aquakv_workspace_bytes",
+    "aquakv_decode_attn_workspace_bytes", "aquakv_predict", "aquakv_encode", "aquakv_decode",
+    "aquakv_decode_attn", "aquakv_encode_phase", "aquakv_decode_phase", "aquakv_poll_status", "aquakv_launch_count", "aquakv_status_string",
+]
+
+
+class AquaKVError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %d (%s)" % (where, status, status_string(status)))
+
+
+class Params(ctypes.Structure):
+    _fields_ = [("d_kv", ctypes.c_int32), ("had_block", ctypes.c_int32),
+                ("scale_group", ctypes.c_int32), ("grid_dim", ctypes.c_int32),
+                ("grid_size", ctypes.c_int32), ("dtype", ctypes.c_int32)]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError("libaquakv.so is not built (run `python -m paper_2501_19392_b200.build` "
+                          "or __graft_entry__.build()); there is no fallback path")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, f32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_size_t
+    L.aquakv_code_bytes.restype = ctypes.c_int
+    L.aquakv_code_bytes.argtypes = [ctypes.POINTER(Params)]
+    L.aquakv_create.restype = ctypes.c_int
+    L.aquakv_create.argtypes = [ctypes.POINTER(Params), vp, vp, vp, ctypes.POINTER(vp)]
+    L.aquakv_destroy.restype = ctypes.c_int
+    L.aquakv_destroy.argtypes = [vp]
+    L.aquakv_workspace_bytes.restype = sz
+    L.aquakv_workspace_bytes.argtypes = [vp, i64, ctypes.c_int]
+    L.aquakv_decode_attn_workspace_bytes.restype = sz
+    L.aquakv_decode_attn_workspace_bytes.argtypes = [vp, i32, i64, i32, i32]
+    L.aquakv_predict.restype = ctypes.c_int
+    L.aquakv_predict.argtypes = [vp, i64, vp, vp, i64, vp, vp, vp, i64, vp]
+    L.aquakv_encode.restype = ctypes.c_int
+    L.aquakv_encode.argtypes = [vp, i64, vp, vp, i64, vp, vp, i64, vp, vp, vp, vp,
+                                vp, vp, vp, vp, vp, vp, i64, vp, sz, vp]
+    L.aquakv_decode.restype = ctypes.c_int
+    L.aquakv_decode.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp,
+                                vp, vp, i64, vp, sz, vp]
+    L.aquakv_decode_attn.restype = ctypes.c_int
+    L.aquakv_decode_attn.argtypes = [vp, i32, i64, i32, i32, i32, f32, vp, vp, vp, vp, vp,
+                                     vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, sz, vp]
+    L.aquakv_encode_phase.restype = ctypes.c_int
+    L.aquakv_encode_phase.argtypes = [vp, ctypes.c_int, i64, vp, i64, vp, vp, i64, vp, vp, vp, vp, vp, i64,
+                                      vp, sz, vp]
+    L.aquakv_decode_phase.restype = ctypes.c_int
+    L.aquakv_decode_phase.argtypes = [vp, ctypes.c_int, i64, vp, vp, vp, vp, i64, vp, vp, vp, i64, vp, sz, vp]
+    L.aquakv_poll_status.restype = ctypes.c_int
+    L.aquakv_poll_status.argtypes = [vp, vp]
+    L.aquakv_launch_count.restype = i64
+    L.aquakv_launch_count.argtypes = [vp]
+    L.aquakv_status_string.restype = ctypes.c_char_p
+    L.aquakv_status_string.argtypes = [ctypes.c_int]
+    return L
+
+
+lib = _load()
+
+
+def status_string(status: int) -> str:
+    return lib.aquakv_status_string(int(status)).decode()
+
+
+def code_bytes(d_kv: int, grid_size: int, had_block: int = 64, scale_group: int = 64, dtype: int = BF16) -> int:
+    p = Params(d_kv, had_block, scale_group, 2, grid_size, dtype)
+    return int(lib.aquakv_code_bytes(ctypes.byref(p)))
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, torch.Tensor):
+        return t.data_ptr()
+    return int(t)
+
+
+def _ld(t: Optional[torch.Tensor], default: int) -> int:
+    return default if t is None else int(t.stride(0))
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+class Codec:
+    """One aquakv_ctx.  Tensors are torch CUDA tensors: 16-bit rows [T, d_kv] (stride(1) == 1),
+    codes uint8 [T, code_bytes], scales float16 [T, d_kv/scale_group] (both contiguous)."""
+
+    def __init__(self, d_kv: int, had_block: int, scale_group: int, grid: np.ndarray, dtype: int,
+                 signs_k: np.ndarray, signs_v: np.ndarray):
+        self.params = Params(d_kv, had_block, scale_group, 2, int(np.asarray(grid).shape[0]), dtype)
+        g = np.ascontiguousarray(grid, dtype=np.float32)
+        sk = np.ascontiguousarray(signs_k, dtype=np.int8)
+        sv = np.ascontiguousarray(signs_v, dtype=np.int8)
+        h = ctypes.c_void_p()
+        rc = lib.aquakv_create(ctypes.byref(self.params), g.ctypes.data, sk.ctypes.data, sv.ctypes.data,
+                               ctypes.byref(h))
+        if rc:
+            raise AquaKVError(rc, "aquakv_create")
+        self.h = h
+        self.d = d_kv
+        self.dtype = dtype
+        self.torch_dtype = torch.float16 if dtype == F16 else torch.bfloat16
+        self.code_bytes = int(lib.aquakv_code_bytes(ctypes.byref(self.params)))
+        self.n_groups = d_kv // scale_group
+        self._ws = None
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib.aquakv_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- workspace ----------------------------------------------------------------------------
+    def workspace_bytes(self, n_tokens: int, op: int) -> int:
+        return int(lib.aquakv_workspace_bytes(self.h, n_tokens, op))
+
+    def decode_attn_workspace_bytes(self, batch: int, ctx_len: int, n_q_heads: int, head_dim: int) -> int:
+        return int(lib.aquakv_decode_attn_workspace_bytes(self.h, batch, ctx_len, n_q_heads, head_dim))
+
+    def _workspace(self, nbytes: int, device) -> torch.Tensor:
+        if self._ws is None or self._ws.numel() < nbytes or self._ws.device != device:
+            self._ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
+        return self._ws
+
+    # -- entry points -----------------------------------------------------------------------------
+    def predict(self, in0, in1, W, bias=None, out=None):
+        T = in0.shape[0]
+        if out is None:
+            out = torch.empty((T, self.d), dtype=torch.float32, device=in0.device)
+        rc = lib.aquakv_predict(self.h, T, _ptr(in0), _ptr(in1), _ld(in0, self.d), _ptr(W), _ptr(bias),
+                                _ptr(out), _ld(out, self.d), _stream())
+        if rc:
+            raise AquaKVError(rc, "aquakv_predict")
+        return out
+
+    def encode(self, K, V, Khat_prev=None, Vhat_prev=None, Wk=None, Wv=None, bk=None, bv=None,
+               Kcodes=None, Kscales=None, Vcodes=None, Vscales=None, Khat=None, Vhat=None,
+               want_hat: bool = True, workspace=None):
+        T, dev = K.shape[0], K.device
+        if Kcodes is None:
+            Kcodes = torch.empty((T, self.code_bytes), dtype=torch.uint8, device=dev)
+            Vcodes = torch.empty((T, self.code_bytes), dtype=torch.uint8, device=dev)
+            Kscales = torch.empty((T, self.n_groups), dtype=torch.float16, device=dev)
+            Vscales = torch.empty((T, self.n_groups), dtype=torch.float16, device=dev)
+        if want_hat and Khat is None:
+            Khat = torch.empty((T, self.d), dtype=self.torch_dtype, device=dev)
+            Vhat = torch.empty((T, self.d), dtype=self.torch_dtype, device=dev)
+        ws = workspace if workspace is not None else self._workspace(self.workspace_bytes(T, OP_ENCODE), dev)
+        rc = lib.aquakv_encode(self.h, T, _ptr(K), _ptr(V), _ld(K, self.d), _ptr(Khat_prev), _ptr(Vhat_prev),
+                               _ld(Khat_prev, self.d), _ptr(Wk), _ptr(Wv), _ptr(bk), _ptr(bv),
+                               _ptr(Kcodes), _ptr(Kscales), _ptr(Vcodes), _ptr(Vscales),
+                               _ptr(Khat), _ptr(Vhat), _ld(Khat, self.d), _ptr(ws), ws.numel(), _stream())
+        if rc:
+            raise AquaKVError(rc, "aquakv_encode")
+        return Kcodes, Kscales, Vcodes, Vscales, Khat, Vhat
+
+    def decode(self, Kcodes, Kscales, Vcodes, Vscales, Khat_prev=None, Vhat_prev=None, Wk=None, Wv=None,
+               bk=None, bv=None, Khat=None, Vhat=None, workspace=None):
+        T, dev = Kcodes.shape[0], Kcodes.device
+        if Khat is None:
+            Khat = torch.empty((T, self.d), dtype=self.torch_dtype, device=dev)
+            Vhat = torch.empty((T, self.d), dtype=self.torch_dtype, device=dev)
+        ws = workspace if workspace is not None else self._workspace(self.workspace_bytes(T, OP_DECODE), dev)
+        rc = lib.aquakv_decode(self.h, T, _ptr(Kcodes), _ptr(Kscales), _ptr(Vcodes), _ptr(Vscales),
+                               _ptr(Khat_prev), _ptr(Vhat_prev), _ld(Khat_prev, self.d), _ptr(Wk), _ptr(Wv),
+                               _ptr(bk), _ptr(bv), _ptr(Khat), _ptr(Vhat), _ld(Khat, self.d),
+                               _ptr(ws), ws.numel(), _stream())
+        if rc:
+            raise AquaKVError(rc, "aquakv_decode")
+        return Khat, Vhat
+
+    def decode_attn(self, q, Kcodes, Kscales, Vcodes, Vscales, ctx_len: int, n_kv_heads: int,
+                    softmax_scale: float, Khat_prev=None, Vhat_prev=None, Wk=None, Wv=None, bk=None, bv=None,
+                    out=None, lse=None, Khat=None, Vhat=None, want_lse: bool = False, workspace=None):
+        batch, n_q_heads, head_dim = q.shape
+        dev = q.device
+        if out is None:
+            out = torch.empty_like(q)
+        if want_lse and lse is None:
+            lse = torch.empty((batch, n_q_heads), dtype=torch.float32, device=dev)
+        ws = workspace if workspace is not None else self._workspace(
+            self.decode_attn_workspace_bytes(batch, ctx_len, n_q_heads, head_dim), dev)
+        rc = lib.aquakv_decode_attn(self.h, batch, ctx_len, n_q_heads, n_kv_heads, head_dim, softmax_scale,
+                                    _ptr(q), _ptr(Kcodes), _ptr(Kscales), _ptr(Vcodes), _ptr(Vscales),
+                                    _ptr(Khat_prev), _ptr(Vhat_prev), _ld(Khat_prev, self.d), _ptr(Wk), _ptr(Wv),
+                                    _ptr(bk), _ptr(bv), _ptr(out), _ptr(lse), _ptr(Khat), _ptr(Vhat),
+                                    _ld(Khat, self.d), _ptr(ws), ws.numel(), _stream())
+        if rc:
+            raise AquaKVError(rc, "aquakv_decode_attn")
+        return out, lse
+
+    def encode_phase(self, role: int, X, in0=None, in1=None, W=None, bias=None, want_hat: bool = True):
+        T, dev = X.shape[0], X.device
+        codes = torch.empty((T, self.code_bytes), dtype=torch.uint8, device=dev)
+        scales = torch.empty((T, self.n_groups), dtype=torch.float16, device=dev)
+        hat = torch.empty((T, self.d), dtype=self.torch_dtype, device=dev) if want_hat else None
+        ws = self._workspace(self.workspace_bytes(T, OP_ENCODE), dev)
+        rc = lib.aquakv_encode_phase(self.h, role, T, _ptr(X), _ld(X, self.d), _ptr(in0), _ptr(in1),
+                                     _ld(in0, self.d), _ptr(W), _ptr(bias), _ptr(codes), _ptr(scales),
+                                     _ptr(hat), _ld(hat, self.d), _ptr(ws), ws.numel(), _stream())
+        if rc:
+            raise AquaKVError(rc, "aquakv_encode_phase")
+        return codes, scales, hat
+
+    def decode_phase(self, role: int, codes, scales, in0=None, in1=None, W=None, bias=None):
+        T, dev = codes.shape[0], codes.device
+        hat = torch.empty((T, self.d), dtype=self.torch_dtype, device=dev)
+        ws = self._workspace(self.workspace_bytes(T, OP_DECODE), dev)
+        rc = lib.aquakv_decode_phase(self.h, role, T, _ptr(codes), _ptr(scales), _ptr(in0), _ptr(in1),
+                                     _ld(in0, self.d), _ptr(W), _ptr(bias), _ptr(hat), _ld(hat, self.d),
+                                     _ptr(ws), ws.numel(), _stream())
+        if rc:
+            raise AquaKVError(rc, "aquakv_decode_phase")
+        return hat
+
+    def poll_status(self) -> int:
+        return int(lib.aquakv_poll_status(self.h, _stream()))
+
+    def launch_count(self) -> int:
+        return int(lib.aquakv_launch_count(self.h))

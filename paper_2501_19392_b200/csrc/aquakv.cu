@@ -1,0 +1,794 @@
+// Host side of the AQUA-KV codec library: the C ABI declared in include/aquakv.h, argument
+// validation, workspace carving, tensor-map construction and kernel launches.  Every step of
+// Algorithm 2 / Algorithm 3 / the attention read of Algorithm 4 runs in the kernels of
+// gemm_pred.cuh, codec.cuh and attn.cuh; nothing is computed on the host and there is no
+// fallback path.
+//
+// Large calls are cut into token chunks sized so that one chunk's fp32 prediction (and, for the
+// fused attention, its decoded keys/values) stays resident in the 126 MB L2 between the kernel
+// that writes it and the kernel that reads it.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <new>
+
+#include "aquakv.h"
+#include "attn.cuh"
+#include "codec.cuh"
+#include "gemm_pred.cuh"
+
+using namespace aquakv;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct aquakv_ctx {
+  aquakv_params p;
+  int log_h, log_g, bits, code_bytes, n_groups;
+  bool bf16;
+  int device;
+  int sm_count;
+  int chunk_tokens;        // tokens per L2-resident chunk
+  int attn_block_tokens;   // tokens per split-KV block
+  float4* d_grid4;
+  uint32_t* d_signmask[2]; // [0] keys, [1] values
+  int* d_status;
+  GridConst<16> gc16;
+  GridConst<64> gc64;
+  EncodeTiledFn encode_tiled;
+  int64_t launches;
+};
+
+namespace {
+
+constexpr int kRoleK = 0, kRoleV = 1;
+
+inline int ilog2(int v) {
+  int b = 0;
+  while ((1 << b) < v) ++b;
+  return b;
+}
+inline bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t round_up(size_t v, size_t m) { return (v + m - 1) / m * m; }
+
+int check_params(const aquakv_params* p) {
+  if (p == nullptr) return AQUAKV_ERR_INVALID_ARG;
+  if (p->d_kv <= 0 || p->had_block <= 0 || p->scale_group <= 0 || p->grid_size <= 0)
+    return AQUAKV_ERR_INVALID_ARG;
+  if (p->dtype != AQUAKV_F16 && p->dtype != AQUAKV_BF16) return AQUAKV_ERR_INVALID_ARG;
+  if (p->grid_dim != 2) return AQUAKV_ERR_UNSUPPORTED;
+  if (p->d_kv != 256 && p->d_kv != 512 && p->d_kv != 1024) return AQUAKV_ERR_UNSUPPORTED;
+  if (p->grid_size != 16 && p->grid_size != 64 && p->grid_size != 256) return AQUAKV_ERR_UNSUPPORTED;
+  if (!is_pow2(p->had_block) || p->had_block < 64 || p->had_block > p->d_kv)
+    return AQUAKV_ERR_UNSUPPORTED;
+  if (!is_pow2(p->scale_group) || p->scale_group < p->had_block || p->scale_group > p->d_kv)
+    return AQUAKV_ERR_UNSUPPORTED;
+  return AQUAKV_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// launches
+// ---------------------------------------------------------------------------------------------
+int make_tmap(const aquakv_ctx* c, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
+              uint64_t ld_elems, uint32_t box_rows) {
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {ld_elems * 2};
+  const cuuint32_t box[2] = {uint32_t(kBK), box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = c->encode_tiled(
+      m, c->bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2,
+      const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? AQUAKV_OK : AQUAKV_ERR_CUDA;
+}
+
+// P[M, d] = [in0 ; in1] W^T + bias for M rows starting at the given pointers.
+int launch_predict(aquakv_ctx* c, cudaStream_t st, int M, const void* in0, const void* in1,
+                   int64_t ld_in0, int64_t ld_in1, const void* W, const float* bias, float* P,
+                   int64_t ldP) {
+  const int d = c->p.d_kv;
+  const int n_in = in1 != nullptr ? 2 : 1;
+  CUtensorMap tA0, tA1, tB;
+  int rc = make_tmap(c, &tA0, in0, uint64_t(M), uint64_t(d), uint64_t(ld_in0), kBM);
+  if (rc) return rc;
+  if (in1 != nullptr) {
+    rc = make_tmap(c, &tA1, in1, uint64_t(M), uint64_t(d), uint64_t(ld_in1), kBM);
+    if (rc) return rc;
+  } else {
+    tA1 = tA0;
+  }
+  rc = make_tmap(c, &tB, W, uint64_t(d), uint64_t(n_in) * d, uint64_t(n_in) * d, kBN);
+  if (rc) return rc;
+  GemmArgs g;
+  g.M = M;
+  g.N = d;
+  g.nk0 = d / kBK;
+  g.nk1 = in1 != nullptr ? d / kBK : 0;
+  g.P = P;
+  g.ldP = ldP;
+  g.bias = bias;
+  g.status = c->d_status;
+  const int tiles = ((M + kBM - 1) / kBM) * (d / kBN);
+  const int grid = tiles < c->sm_count ? tiles : c->sm_count;
+  if (c->bf16) {
+    gemm_pred_kernel<true><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(tA0, tA1, tB, g);
+  } else {
+    gemm_pred_kernel<false><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(tA0, tA1, tB, g);
+  }
+  ++c->launches;
+  return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
+}
+
+template <int D, int NPTS, bool BF>
+void launch_encode_rows_t(aquakv_ctx* c, cudaStream_t st, const CodecArgs& a, int grid) {
+  if constexpr (NPTS == 16) {
+    encode_rows_kernel<D, 16, BF><<<grid, kCodecThreads, 0, st>>>(c->gc16, a);
+  } else if constexpr (NPTS == 64) {
+    encode_rows_kernel<D, 64, BF><<<grid, kCodecThreads, 0, st>>>(c->gc64, a);
+  } else {
+    GridConst<1> dummy = {};
+    encode_rows_kernel<D, 256, BF><<<grid, kCodecThreads, 0, st>>>(dummy, a);
+  }
+}
+
+template <int D, int NPTS, bool BF>
+void launch_decode_rows_t(aquakv_ctx*, cudaStream_t st, const CodecArgs& a, int grid) {
+  decode_rows_kernel<D, NPTS, BF><<<grid, kCodecThreads, 0, st>>>(a);
+}
+
+#define AQ_DISPATCH_DNB(FN, ...)                                                     \
+  do {                                                                               \
+    const int d_ = c->p.d_kv, n_ = c->p.grid_size;                                   \
+    const bool b_ = c->bf16;                                                         \
+    if (d_ == 256 && n_ == 16 && b_) FN<256, 16, true>(__VA_ARGS__);                 \
+    else if (d_ == 256 && n_ == 16) FN<256, 16, false>(__VA_ARGS__);                 \
+    else if (d_ == 256 && n_ == 64 && b_) FN<256, 64, true>(__VA_ARGS__);            \
+    else if (d_ == 256 && n_ == 64) FN<256, 64, false>(__VA_ARGS__);                 \
+    else if (d_ == 256 && b_) FN<256, 256, true>(__VA_ARGS__);                       \
+    else if (d_ == 256) FN<256, 256, false>(__VA_ARGS__);                            \
+    else if (d_ == 512 && n_ == 16 && b_) FN<512, 16, true>(__VA_ARGS__);            \
+    else if (d_ == 512 && n_ == 16) FN<512, 16, false>(__VA_ARGS__);                 \
+    else if (d_ == 512 && n_ == 64 && b_) FN<512, 64, true>(__VA_ARGS__);            \
+    else if (d_ == 512 && n_ == 64) FN<512, 64, false>(__VA_ARGS__);                 \
+    else if (d_ == 512 && b_) FN<512, 256, true>(__VA_ARGS__);                       \
+    else if (d_ == 512) FN<512, 256, false>(__VA_ARGS__);                            \
+    else if (n_ == 16 && b_) FN<1024, 16, true>(__VA_ARGS__);                        \
+    else if (n_ == 16) FN<1024, 16, false>(__VA_ARGS__);                             \
+    else if (n_ == 64 && b_) FN<1024, 64, true>(__VA_ARGS__);                        \
+    else if (n_ == 64) FN<1024, 64, false>(__VA_ARGS__);                             \
+    else if (b_) FN<1024, 256, true>(__VA_ARGS__);                                   \
+    else FN<1024, 256, false>(__VA_ARGS__);                                          \
+  } while (0)
+
+int codec_grid(const aquakv_ctx* c, int rows) {
+  const int blocks = (rows + kCodecWarps - 1) / kCodecWarps;
+  const int cap = c->sm_count * 8;
+  return blocks < cap ? blocks : cap;
+}
+
+CodecArgs codec_args(const aquakv_ctx* c, int role, int rows) {
+  CodecArgs a;
+  std::memset(&a, 0, sizeof(a));
+  a.signmask = c->d_signmask[role];
+  a.grid4 = c->d_grid4;
+  a.T = rows;
+  a.log_h = c->log_h;
+  a.log_g = c->log_g;
+  return a;
+}
+
+// One phase of Algorithm 2 on `rows` rows: codes/scales = Q(X - P), hat = round16(P + Q^-1(..)).
+int launch_encode_rows(aquakv_ctx* c, cudaStream_t st, int role, int rows, const void* X,
+                       int64_t ldX, const float* P, int64_t ldP, uint8_t* codes, uint16_t* scales,
+                       void* hat, int64_t ldHat) {
+  CodecArgs a = codec_args(c, role, rows);
+  a.X = static_cast<const uint16_t*>(X);
+  a.ldX = ldX;
+  a.P = P;
+  a.ldP = ldP;
+  a.codes = codes;
+  a.scales = scales;
+  a.hat = static_cast<uint16_t*>(hat);
+  a.ldHat = ldHat;
+  const int grid = codec_grid(c, rows);
+  AQ_DISPATCH_DNB(launch_encode_rows_t, c, st, a, grid);
+  ++c->launches;
+  return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
+}
+
+// One phase of Algorithm 3 on `rows` rows: hat = round16(P + Q^-1(codes, scales)).
+int launch_decode_rows(aquakv_ctx* c, cudaStream_t st, int role, int rows, const uint8_t* codes,
+                       const uint16_t* scales, const float* P, int64_t ldP, void* hat,
+                       int64_t ldHat) {
+  CodecArgs a = codec_args(c, role, rows);
+  a.P = P;
+  a.ldP = ldP;
+  a.codes = const_cast<uint8_t*>(codes);
+  a.scales = const_cast<uint16_t*>(scales);
+  a.hat = static_cast<uint16_t*>(hat);
+  a.ldHat = ldHat;
+  const int grid = codec_grid(c, rows);
+  AQ_DISPATCH_DNB(launch_decode_rows_t, c, st, a, grid);
+  ++c->launches;
+  return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
+}
+
+template <int HD, int GQ, bool BF>
+void launch_attn_partial_t(cudaStream_t st, const AttnArgs& a, dim3 grid) {
+  attn_partial_kernel<HD, GQ, BF><<<grid, kAttnThreads, 0, st>>>(a);
+}
+
+int attn_gq(int rep, int* passes) {
+  switch (rep) {
+    case 1: case 2: case 3: case 4: *passes = 1; return rep;
+    case 6: *passes = 2; return 3;
+    case 8: *passes = 2; return 4;
+    default: *passes = 0; return 0;
+  }
+}
+
+int launch_attn_partial(aquakv_ctx* c, cudaStream_t st, const AttnArgs& a, int head_dim,
+                        int n_blocks) {
+  int passes = 0;
+  const int gq = attn_gq(a.n_q_heads / a.n_kv_heads, &passes);
+  const dim3 grid(n_blocks, a.n_kv_heads, passes);
+#define AQ_ATTN(HD, GQ)                                                   \
+  if (head_dim == HD && gq == GQ) {                                       \
+    if (c->bf16) launch_attn_partial_t<HD, GQ, true>(st, a, grid);        \
+    else launch_attn_partial_t<HD, GQ, false>(st, a, grid);               \
+  }
+  AQ_ATTN(64, 1) AQ_ATTN(64, 2) AQ_ATTN(64, 3) AQ_ATTN(64, 4)
+  AQ_ATTN(128, 1) AQ_ATTN(128, 2) AQ_ATTN(128, 3) AQ_ATTN(128, 4)
+#undef AQ_ATTN
+  ++c->launches;
+  return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
+}
+
+int launch_attn_combine(aquakv_ctx* c, cudaStream_t st, const AttnCombineArgs& a, int head_dim,
+                        int batch) {
+  const int grid = batch * a.n_q_heads;
+  if (head_dim == 64) {
+    if (c->bf16) attn_combine_kernel<64, true><<<grid, 64, 0, st>>>(a);
+    else attn_combine_kernel<64, false><<<grid, 64, 0, st>>>(a);
+  } else {
+    if (c->bf16) attn_combine_kernel<128, true><<<grid, 128, 0, st>>>(a);
+    else attn_combine_kernel<128, false><<<grid, 128, 0, st>>>(a);
+  }
+  ++c->launches;
+  return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------------
+// argument checks shared by the entry points
+// ---------------------------------------------------------------------------------------------
+int check_adapters(const void* Khat_prev, const void* Vhat_prev, int64_t ld_prev, const void* Wk,
+                   const void* Wv, const float* bk, const float* bv, int d, bool* has_pred) {
+  const int n_set = (Khat_prev != nullptr) + (Vhat_prev != nullptr) + (Wk != nullptr) + (Wv != nullptr);
+  if (n_set != 0 && n_set != 4) return AQUAKV_ERR_INVALID_ARG;
+  *has_pred = n_set == 4;
+  if (!*has_pred) {
+    if (bk != nullptr || bv != nullptr) return AQUAKV_ERR_INVALID_ARG;
+    return AQUAKV_OK;
+  }
+  if (ld_prev < d) return AQUAKV_ERR_INVALID_ARG;
+  if (ld_prev % 8) return AQUAKV_ERR_ALIGNMENT;
+  if (!aligned16(Khat_prev) || !aligned16(Vhat_prev) || !aligned16(Wk) || !aligned16(Wv))
+    return AQUAKV_ERR_ALIGNMENT;
+  if ((bk != nullptr && !aligned16(bk)) || (bv != nullptr && !aligned16(bv)))
+    return AQUAKV_ERR_ALIGNMENT;
+  return AQUAKV_OK;
+}
+
+int check_rows(const void* p, int64_t ld, int d, bool required) {
+  if (p == nullptr) return required ? AQUAKV_ERR_INVALID_ARG : AQUAKV_OK;
+  if (ld < d) return AQUAKV_ERR_INVALID_ARG;
+  if (ld % 8 || !aligned16(p)) return AQUAKV_ERR_ALIGNMENT;
+  return AQUAKV_OK;
+}
+
+struct EncodeWs {
+  size_t p_off, khat_off, total;
+  int chunk;
+};
+
+EncodeWs encode_ws(const aquakv_ctx* c, int64_t T) {
+  EncodeWs w;
+  const int64_t t128 = int64_t(round_up(size_t(T), 128));
+  w.chunk = int(t128 < c->chunk_tokens ? t128 : c->chunk_tokens);
+  w.p_off = 0;
+  w.khat_off = round_up(size_t(w.chunk) * c->p.d_kv * sizeof(float), 256);
+  w.total = w.khat_off + round_up(size_t(w.chunk) * c->p.d_kv * 2, 256);
+  return w;
+}
+
+struct AttnWs {
+  size_t p_off, khat_off, vhat_off, ml_off, o_off, total;
+  int chunk_blocks;     // split-KV blocks per chunk
+  int n_splits;
+};
+
+AttnWs attn_ws(const aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_heads,
+               int32_t head_dim) {
+  AttnWs w;
+  const int tb = c->attn_block_tokens;
+  w.n_splits = int((ctx_len + tb - 1) / tb);
+  int cb = c->chunk_tokens / tb;
+  if (cb < 1) cb = 1;
+  const int64_t total_blocks = int64_t(batch) * w.n_splits;
+  if (cb > total_blocks) cb = int(total_blocks);
+  w.chunk_blocks = cb;
+  const size_t chunk_rows = size_t(cb) * tb;
+  const size_t d = size_t(c->p.d_kv);
+  w.p_off = 0;
+  w.khat_off = round_up(chunk_rows * d * sizeof(float), 256);
+  w.vhat_off = w.khat_off + round_up(chunk_rows * d * 2, 256);
+  w.ml_off = w.vhat_off + round_up(chunk_rows * d * 2, 256);
+  w.o_off = w.ml_off + round_up(size_t(total_blocks) * n_q_heads * 2 * sizeof(float), 256);
+  w.total = w.o_off + round_up(size_t(total_blocks) * n_q_heads * head_dim * sizeof(float), 256);
+  return w;
+}
+
+}  // namespace
+
+// =============================================================================================
+// C ABI
+// =============================================================================================
+extern "C" {
+
+int aquakv_code_bytes(const aquakv_params* params) {
+  const int rc = check_params(params);
+  if (rc) return rc;
+  return params->d_kv / 2 * ilog2(params->grid_size) / 8;
+}
+
+const char* aquakv_status_string(int status) {
+  switch (status) {
+    case AQUAKV_OK: return "ok";
+    case AQUAKV_ERR_INVALID_ARG: return "invalid argument";
+    case AQUAKV_ERR_UNSUPPORTED: return "unsupported parameter combination";
+    case AQUAKV_ERR_ALIGNMENT: return "misaligned pointer or leading dimension";
+    case AQUAKV_ERR_WORKSPACE: return "workspace missing or too small";
+    case AQUAKV_ERR_CUDA: return "CUDA call failed";
+    case AQUAKV_ERR_TIMEOUT: return "bounded device-side wait expired";
+    default: return "unknown status";
+  }
+}
+
+int aquakv_create(const aquakv_params* params, const float* grid_host, const int8_t* signs_k_host,
+                  const int8_t* signs_v_host, aquakv_ctx** out) {
+  if (out == nullptr) return AQUAKV_ERR_INVALID_ARG;
+  *out = nullptr;
+  int rc = check_params(params);
+  if (rc) return rc;
+  if (grid_host == nullptr || signs_k_host == nullptr || signs_v_host == nullptr)
+    return AQUAKV_ERR_INVALID_ARG;
+  const int d = params->d_kv, n = params->grid_size;
+  for (int i = 0; i < 2 * n; ++i)
+    if (!std::isfinite(grid_host[i])) return AQUAKV_ERR_INVALID_ARG;
+  for (int i = 0; i < d; ++i) {
+    if (signs_k_host[i] != 1 && signs_k_host[i] != -1) return AQUAKV_ERR_INVALID_ARG;
+    if (signs_v_host[i] != 1 && signs_v_host[i] != -1) return AQUAKV_ERR_INVALID_ARG;
+  }
+  aquakv_ctx* c = new (std::nothrow) aquakv_ctx();
+  if (c == nullptr) return AQUAKV_ERR_CUDA;
+  std::memset(c, 0, sizeof(*c));
+  c->p = *params;
+  c->log_h = ilog2(params->had_block);
+  c->log_g = ilog2(params->scale_group);
+  c->bits = ilog2(n);
+  c->code_bytes = d / 2 * c->bits / 8;
+  c->n_groups = d / params->scale_group;
+  c->bf16 = params->dtype == AQUAKV_BF16;
+  c->attn_block_tokens = 256;
+
+  float4 g4[256];
+  for (int i = 0; i < n; ++i) {
+    const float gx = grid_host[2 * i], gy = grid_host[2 * i + 1];
+    const float hn = 0.5f * (gx * gx + gy * gy);
+    g4[i] = make_float4(gx, gy, hn, 0.0f);
+    if (n == 16) { c->gc16.nx[i] = -gx; c->gc16.ny[i] = -gy; c->gc16.hn[i] = hn; }
+    if (n == 64) { c->gc64.nx[i] = -gx; c->gc64.ny[i] = -gy; c->gc64.hn[i] = hn; }
+  }
+  uint32_t masks[2][32];
+  std::memset(masks, 0, sizeof(masks));
+  for (int role = 0; role < 2; ++role) {
+    const int8_t* s = role == kRoleK ? signs_k_host : signs_v_host;
+    for (int e = 0; e < d; ++e)
+      if (s[e] < 0) masks[role][(e >> 3) & 31] |= 1u << (((e >> 8) << 3) | (e & 7));
+  }
+
+  bool ok = cudaGetDevice(&c->device) == cudaSuccess;
+  ok = ok && cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device) == cudaSuccess;
+  if (ok) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    ok = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) == cudaSuccess &&
+         q == cudaDriverEntryPointSuccess && fn != nullptr;
+    c->encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  ok = ok && cudaMalloc(&c->d_grid4, sizeof(float4) * 256) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_signmask[0], sizeof(uint32_t) * 32) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_signmask[1], sizeof(uint32_t) * 32) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_status, sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMemcpy(c->d_grid4, g4, sizeof(float4) * n, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(c->d_signmask[0], masks[0], sizeof(masks[0]), cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(c->d_signmask[1], masks[1], sizeof(masks[1]), cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemset(c->d_status, 0, sizeof(int)) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(gemm_pred_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  int(kGemmSmemBytes)) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(gemm_pred_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  int(kGemmSmemBytes)) == cudaSuccess;
+  ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+  if (!ok) {
+    (void)cudaGetLastError();
+    aquakv_destroy(c);
+    return AQUAKV_ERR_CUDA;
+  }
+  // Two full waves of 128x256 GEMM tiles per chunk: 2 * SMs * 128 * 256 fp32 = 38.8 MB of
+  // prediction, well inside L2 next to the chunk's 16-bit rows.
+  c->chunk_tokens = 2 * c->sm_count * kBM / (d / kBN);
+  *out = c;
+  return AQUAKV_OK;
+}
+
+int aquakv_destroy(aquakv_ctx* c) {
+  if (c == nullptr) return AQUAKV_OK;
+  bool ok = true;
+  if (c->d_grid4) ok = cudaFree(c->d_grid4) == cudaSuccess && ok;
+  if (c->d_signmask[0]) ok = cudaFree(c->d_signmask[0]) == cudaSuccess && ok;
+  if (c->d_signmask[1]) ok = cudaFree(c->d_signmask[1]) == cudaSuccess && ok;
+  if (c->d_status) ok = cudaFree(c->d_status) == cudaSuccess && ok;
+  delete c;
+  return ok ? AQUAKV_OK : AQUAKV_ERR_CUDA;
+}
+
+size_t aquakv_workspace_bytes(const aquakv_ctx* c, int64_t n_tokens, int op) {
+  if (c == nullptr || n_tokens <= 0) return 0;
+  if (op == AQUAKV_OP_ENCODE || op == AQUAKV_OP_DECODE) return encode_ws(c, n_tokens).total;
+  return 0;
+}
+
+size_t aquakv_decode_attn_workspace_bytes(const aquakv_ctx* c, int32_t batch, int64_t ctx_len,
+                                          int32_t n_q_heads, int32_t head_dim) {
+  if (c == nullptr || batch <= 0 || ctx_len <= 0 || n_q_heads <= 0 || head_dim <= 0) return 0;
+  return attn_ws(c, batch, ctx_len, n_q_heads, head_dim).total;
+}
+
+int64_t aquakv_launch_count(const aquakv_ctx* c) { return c ? c->launches : 0; }
+
+int aquakv_poll_status(aquakv_ctx* c, void* cuda_stream) {
+  if (c == nullptr) return AQUAKV_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess) return AQUAKV_ERR_CUDA;
+  int h = 0;
+  if (cudaMemcpy(&h, c->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return AQUAKV_ERR_CUDA;
+  if (h != 0 && cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess) return AQUAKV_ERR_CUDA;
+  return h;
+}
+
+int aquakv_predict(aquakv_ctx* c, int64_t n_tokens, const void* in0, const void* in1, int64_t ld_in,
+                   const void* W, const float* bias, float* P, int64_t ldP, void* cuda_stream) {
+  if (c == nullptr || n_tokens < 0) return AQUAKV_ERR_INVALID_ARG;
+  if (n_tokens == 0) return AQUAKV_OK;
+  const int d = c->p.d_kv;
+  if (in0 == nullptr || W == nullptr || P == nullptr || ld_in < d || ldP < d)
+    return AQUAKV_ERR_INVALID_ARG;
+  if (ld_in % 8 || ldP % 4 || !aligned16(in0) || !aligned16(in1) || !aligned16(W) || !aligned16(P) ||
+      (bias != nullptr && !aligned16(bias)))
+    return AQUAKV_ERR_ALIGNMENT;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t step = int64_t(1) << 20;   // rows per launch (keeps per-launch row counts in int)
+  for (int64_t t0 = 0; t0 < n_tokens; t0 += step) {
+    const int rows = int(n_tokens - t0 < step ? n_tokens - t0 : step);
+    const uint16_t* a0 = static_cast<const uint16_t*>(in0) + t0 * ld_in;
+    const uint16_t* a1 = in1 ? static_cast<const uint16_t*>(in1) + t0 * ld_in : nullptr;
+    const int rc = launch_predict(c, st, rows, a0, a1, ld_in, ld_in, W, bias, P + t0 * ldP, ldP);
+    if (rc) return rc;
+  }
+  return AQUAKV_OK;
+}
+
+int aquakv_encode_phase(aquakv_ctx* c, int role, int64_t n_tokens, const void* X, int64_t ld_x,
+                        const void* in0, const void* in1, int64_t ld_in, const void* W,
+                        const float* bias, uint8_t* codes, uint16_t* scales, void* hat,
+                        int64_t ld_hat, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (c == nullptr || n_tokens < 0 || (role != kRoleK && role != kRoleV)) return AQUAKV_ERR_INVALID_ARG;
+  if (n_tokens == 0) return AQUAKV_OK;
+  const int d = c->p.d_kv;
+  int rc;
+  if ((rc = check_rows(X, ld_x, d, true))) return rc;
+  if ((rc = check_rows(hat, ld_hat, d, false))) return rc;
+  if (codes == nullptr || scales == nullptr) return AQUAKV_ERR_INVALID_ARG;
+  const bool has_pred = W != nullptr;
+  if (has_pred) {
+    if ((rc = check_rows(in0, ld_in, d, true))) return rc;
+    if ((rc = check_rows(in1, ld_in, d, false))) return rc;
+    if (!aligned16(W) || (bias != nullptr && !aligned16(bias))) return AQUAKV_ERR_ALIGNMENT;
+  } else if (in0 != nullptr || in1 != nullptr || bias != nullptr) {
+    return AQUAKV_ERR_INVALID_ARG;
+  }
+  if (hat != nullptr && (hat == X || hat == in0 || hat == in1)) return AQUAKV_ERR_INVALID_ARG;
+  const EncodeWs ws = encode_ws(c, n_tokens);
+  if (has_pred) {
+    if (workspace == nullptr || workspace_bytes < ws.total) return AQUAKV_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  float* P = has_pred ? reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + ws.p_off) : nullptr;
+  const int cb = c->code_bytes, ng = c->n_groups;
+  const uint16_t* Xp = static_cast<const uint16_t*>(X);
+  const uint16_t* a0 = static_cast<const uint16_t*>(in0);
+  const uint16_t* a1 = static_cast<const uint16_t*>(in1);
+  for (int64_t t0 = 0; t0 < n_tokens; t0 += ws.chunk) {
+    const int rows = int(n_tokens - t0 < ws.chunk ? n_tokens - t0 : ws.chunk);
+    if (has_pred) {
+      rc = launch_predict(c, st, rows, a0 + t0 * ld_in, a1 ? a1 + t0 * ld_in : nullptr, ld_in, ld_in,
+                          W, bias, P, d);
+      if (rc) return rc;
+    }
+    rc = launch_encode_rows(c, st, role, rows, Xp + t0 * ld_x, ld_x, P, d, codes + t0 * cb,
+                            scales + t0 * ng,
+                            hat != nullptr ? static_cast<uint16_t*>(hat) + t0 * ld_hat : nullptr, ld_hat);
+    if (rc) return rc;
+  }
+  return AQUAKV_OK;
+}
+
+int aquakv_decode_phase(aquakv_ctx* c, int role, int64_t n_tokens, const uint8_t* codes,
+                        const uint16_t* scales, const void* in0, const void* in1, int64_t ld_in,
+                        const void* W, const float* bias, void* hat, int64_t ld_hat,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (c == nullptr || n_tokens < 0 || (role != kRoleK && role != kRoleV)) return AQUAKV_ERR_INVALID_ARG;
+  if (n_tokens == 0) return AQUAKV_OK;
+  const int d = c->p.d_kv;
+  int rc;
+  if ((rc = check_rows(hat, ld_hat, d, true))) return rc;
+  if (codes == nullptr || scales == nullptr) return AQUAKV_ERR_INVALID_ARG;
+  const bool has_pred = W != nullptr;
+  if (has_pred) {
+    if ((rc = check_rows(in0, ld_in, d, true))) return rc;
+    if ((rc = check_rows(in1, ld_in, d, false))) return rc;
+    if (!aligned16(W) || (bias != nullptr && !aligned16(bias))) return AQUAKV_ERR_ALIGNMENT;
+  } else if (in0 != nullptr || in1 != nullptr || bias != nullptr) {
+    return AQUAKV_ERR_INVALID_ARG;
+  }
+  if (hat == in0 || hat == in1) return AQUAKV_ERR_INVALID_ARG;
+  const EncodeWs ws = encode_ws(c, n_tokens);
+  if (has_pred) {
+    if (workspace == nullptr || workspace_bytes < ws.total) return AQUAKV_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  float* P = has_pred ? reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + ws.p_off) : nullptr;
+  const int cb = c->code_bytes, ng = c->n_groups;
+  const uint16_t* a0 = static_cast<const uint16_t*>(in0);
+  const uint16_t* a1 = static_cast<const uint16_t*>(in1);
+  for (int64_t t0 = 0; t0 < n_tokens; t0 += ws.chunk) {
+    const int rows = int(n_tokens - t0 < ws.chunk ? n_tokens - t0 : ws.chunk);
+    if (has_pred) {
+      rc = launch_predict(c, st, rows, a0 + t0 * ld_in, a1 ? a1 + t0 * ld_in : nullptr, ld_in, ld_in,
+                          W, bias, P, d);
+      if (rc) return rc;
+    }
+    rc = launch_decode_rows(c, st, role, rows, codes + t0 * cb, scales + t0 * ng, P, d,
+                            static_cast<uint16_t*>(hat) + t0 * ld_hat, ld_hat);
+    if (rc) return rc;
+  }
+  return AQUAKV_OK;
+}
+
+int aquakv_encode(aquakv_ctx* c, int64_t n_tokens, const void* K, const void* V, int64_t ld_kv,
+                  const void* Khat_prev, const void* Vhat_prev, int64_t ld_prev, const void* Wk,
+                  const void* Wv, const float* bk, const float* bv, uint8_t* Kcodes,
+                  uint16_t* Kscales, uint8_t* Vcodes, uint16_t* Vscales, void* Khat, void* Vhat,
+                  int64_t ld_hat, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (c == nullptr || n_tokens < 0) return AQUAKV_ERR_INVALID_ARG;
+  if (n_tokens == 0) return AQUAKV_OK;
+  const int d = c->p.d_kv;
+  int rc;
+  if ((rc = check_rows(K, ld_kv, d, true))) return rc;
+  if ((rc = check_rows(V, ld_kv, d, true))) return rc;
+  if ((rc = check_rows(Khat, ld_hat, d, false))) return rc;
+  if ((rc = check_rows(Vhat, ld_hat, d, false))) return rc;
+  if (Kcodes == nullptr || Kscales == nullptr || Vcodes == nullptr || Vscales == nullptr)
+    return AQUAKV_ERR_INVALID_ARG;
+  bool has_pred = false;
+  if ((rc = check_adapters(Khat_prev, Vhat_prev, ld_prev, Wk, Wv, bk, bv, d, &has_pred))) return rc;
+  if ((Khat != nullptr && (Khat == Khat_prev || Khat == K || Khat == Vhat_prev)) ||
+      (Vhat != nullptr && (Vhat == Vhat_prev || Vhat == V || Vhat == Khat_prev || Vhat == Khat)))
+    return AQUAKV_ERR_INVALID_ARG;
+  const EncodeWs ws = encode_ws(c, n_tokens);
+  if (has_pred || Khat == nullptr) {
+    if (workspace == nullptr || workspace_bytes < ws.total) return AQUAKV_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  uint8_t* wsb = static_cast<uint8_t*>(workspace);
+  float* P = has_pred ? reinterpret_cast<float*>(wsb + ws.p_off) : nullptr;
+  const int cb = c->code_bytes, ng = c->n_groups;
+  const uint16_t* Kp = static_cast<const uint16_t*>(K);
+  const uint16_t* Vp = static_cast<const uint16_t*>(V);
+  const uint16_t* Kpv = static_cast<const uint16_t*>(Khat_prev);
+  const uint16_t* Vpv = static_cast<const uint16_t*>(Vhat_prev);
+  for (int64_t t0 = 0; t0 < n_tokens; t0 += ws.chunk) {
+    const int rows = int(n_tokens - t0 < ws.chunk ? n_tokens - t0 : ws.chunk);
+    // keys: Algorithm 2 lines 5-7
+    uint16_t* khat_c = Khat != nullptr ? static_cast<uint16_t*>(Khat) + t0 * ld_hat
+                                       : reinterpret_cast<uint16_t*>(wsb + ws.khat_off);
+    const int64_t ld_khat_c = Khat != nullptr ? ld_hat : d;
+    if (has_pred) {
+      rc = launch_predict(c, st, rows, Kpv + t0 * ld_prev, nullptr, ld_prev, 0, Wk, bk, P, d);
+      if (rc) return rc;
+    }
+    rc = launch_encode_rows(c, st, kRoleK, rows, Kp + t0 * ld_kv, ld_kv, P, d, Kcodes + t0 * cb,
+                            Kscales + t0 * ng, (has_pred || Khat != nullptr) ? khat_c : nullptr,
+                            ld_khat_c);
+    if (rc) return rc;
+    // values: Algorithm 2 lines 8-9 (the value predictor reads the rounded Khat)
+    if (has_pred) {
+      rc = launch_predict(c, st, rows, Vpv + t0 * ld_prev, khat_c, ld_prev, ld_khat_c, Wv, bv, P, d);
+      if (rc) return rc;
+    }
+    rc = launch_encode_rows(c, st, kRoleV, rows, Vp + t0 * ld_kv, ld_kv, P, d, Vcodes + t0 * cb,
+                            Vscales + t0 * ng,
+                            Vhat != nullptr ? static_cast<uint16_t*>(Vhat) + t0 * ld_hat : nullptr,
+                            ld_hat);
+    if (rc) return rc;
+  }
+  return AQUAKV_OK;
+}
+
+int aquakv_decode(aquakv_ctx* c, int64_t n_tokens, const uint8_t* Kcodes, const uint16_t* Kscales,
+                  const uint8_t* Vcodes, const uint16_t* Vscales, const void* Khat_prev,
+                  const void* Vhat_prev, int64_t ld_prev, const void* Wk, const void* Wv,
+                  const float* bk, const float* bv, void* Khat, void* Vhat, int64_t ld_hat,
+                  void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (c == nullptr || n_tokens < 0) return AQUAKV_ERR_INVALID_ARG;
+  if (n_tokens == 0) return AQUAKV_OK;
+  const int d = c->p.d_kv;
+  int rc;
+  if ((rc = check_rows(Khat, ld_hat, d, true))) return rc;
+  if ((rc = check_rows(Vhat, ld_hat, d, true))) return rc;
+  if (Kcodes == nullptr || Kscales == nullptr || Vcodes == nullptr || Vscales == nullptr)
+    return AQUAKV_ERR_INVALID_ARG;
+  bool has_pred = false;
+  if ((rc = check_adapters(Khat_prev, Vhat_prev, ld_prev, Wk, Wv, bk, bv, d, &has_pred))) return rc;
+  if (Khat == Khat_prev || Khat == Vhat_prev || Vhat == Vhat_prev || Vhat == Khat_prev || Vhat == Khat)
+    return AQUAKV_ERR_INVALID_ARG;
+  const EncodeWs ws = encode_ws(c, n_tokens);
+  if (has_pred) {
+    if (workspace == nullptr || workspace_bytes < ws.total) return AQUAKV_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  float* P = has_pred ? reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + ws.p_off) : nullptr;
+  const int cb = c->code_bytes, ng = c->n_groups;
+  const uint16_t* Kpv = static_cast<const uint16_t*>(Khat_prev);
+  const uint16_t* Vpv = static_cast<const uint16_t*>(Vhat_prev);
+  uint16_t* Kh = static_cast<uint16_t*>(Khat);
+  uint16_t* Vh = static_cast<uint16_t*>(Vhat);
+  for (int64_t t0 = 0; t0 < n_tokens; t0 += ws.chunk) {
+    const int rows = int(n_tokens - t0 < ws.chunk ? n_tokens - t0 : ws.chunk);
+    if (has_pred) {
+      rc = launch_predict(c, st, rows, Kpv + t0 * ld_prev, nullptr, ld_prev, 0, Wk, bk, P, d);
+      if (rc) return rc;
+    }
+    rc = launch_decode_rows(c, st, kRoleK, rows, Kcodes + t0 * cb, Kscales + t0 * ng, P, d,
+                            Kh + t0 * ld_hat, ld_hat);
+    if (rc) return rc;
+    if (has_pred) {
+      rc = launch_predict(c, st, rows, Vpv + t0 * ld_prev, Kh + t0 * ld_hat, ld_prev, ld_hat, Wv, bv, P, d);
+      if (rc) return rc;
+    }
+    rc = launch_decode_rows(c, st, kRoleV, rows, Vcodes + t0 * cb, Vscales + t0 * ng, P, d,
+                            Vh + t0 * ld_hat, ld_hat);
+    if (rc) return rc;
+  }
+  return AQUAKV_OK;
+}
+
+int aquakv_decode_attn(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_heads,
+                       int32_t n_kv_heads, int32_t head_dim, float softmax_scale, const void* q,
+                       const uint8_t* Kcodes, const uint16_t* Kscales, const uint8_t* Vcodes,
+                       const uint16_t* Vscales, const void* Khat_prev, const void* Vhat_prev,
+                       int64_t ld_prev, const void* Wk, const void* Wv, const float* bk,
+                       const float* bv, void* out, float* lse, void* Khat, void* Vhat,
+                       int64_t ld_hat, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (c == nullptr || batch < 0 || ctx_len < 0) return AQUAKV_ERR_INVALID_ARG;
+  if (batch == 0 || ctx_len == 0) return AQUAKV_OK;
+  const int d = c->p.d_kv;
+  if (n_q_heads <= 0 || n_kv_heads <= 0 || head_dim <= 0) return AQUAKV_ERR_INVALID_ARG;
+  if (n_kv_heads * head_dim != d || n_q_heads % n_kv_heads) return AQUAKV_ERR_INVALID_ARG;
+  int passes = 0;
+  if ((head_dim != 64 && head_dim != 128) || attn_gq(n_q_heads / n_kv_heads, &passes) == 0)
+    return AQUAKV_ERR_UNSUPPORTED;
+  if (ctx_len > (int64_t(1) << 30)) return AQUAKV_ERR_UNSUPPORTED;
+  if (q == nullptr || out == nullptr || Kcodes == nullptr || Kscales == nullptr ||
+      Vcodes == nullptr || Vscales == nullptr)
+    return AQUAKV_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out)) return AQUAKV_ERR_ALIGNMENT;
+  if (!(softmax_scale == softmax_scale)) return AQUAKV_ERR_INVALID_ARG;
+  int rc;
+  if ((Khat == nullptr) != (Vhat == nullptr)) return AQUAKV_ERR_INVALID_ARG;
+  if ((rc = check_rows(Khat, ld_hat, d, false))) return rc;
+  if ((rc = check_rows(Vhat, ld_hat, d, false))) return rc;
+  bool has_pred = false;
+  if ((rc = check_adapters(Khat_prev, Vhat_prev, ld_prev, Wk, Wv, bk, bv, d, &has_pred))) return rc;
+  if (Khat != nullptr && (Khat == Khat_prev || Khat == Vhat_prev || Vhat == Vhat_prev ||
+                          Vhat == Khat_prev || Vhat == Khat))
+    return AQUAKV_ERR_INVALID_ARG;
+  const AttnWs ws = attn_ws(c, batch, ctx_len, n_q_heads, head_dim);
+  if (workspace == nullptr || workspace_bytes < ws.total) return AQUAKV_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
+
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  uint8_t* wsb = static_cast<uint8_t*>(workspace);
+  float* P = has_pred ? reinterpret_cast<float*>(wsb + ws.p_off) : nullptr;
+  float* part_ml = reinterpret_cast<float*>(wsb + ws.ml_off);
+  float* part_o = reinterpret_cast<float*>(wsb + ws.o_off);
+  const int cb = c->code_bytes, ng = c->n_groups, tb = c->attn_block_tokens;
+  const uint16_t* Kpv = static_cast<const uint16_t*>(Khat_prev);
+  const uint16_t* Vpv = static_cast<const uint16_t*>(Vhat_prev);
+  const int64_t total_blocks = int64_t(batch) * ws.n_splits;
+  auto block_token = [&](int64_t gb) -> int64_t {   // first global token of global block gb
+    if (gb >= total_blocks) return int64_t(batch) * ctx_len;
+    return (gb / ws.n_splits) * ctx_len + (gb % ws.n_splits) * int64_t(tb);
+  };
+  for (int64_t gb0 = 0; gb0 < total_blocks; gb0 += ws.chunk_blocks) {
+    const int64_t gb1 = gb0 + ws.chunk_blocks < total_blocks ? gb0 + ws.chunk_blocks : total_blocks;
+    const int64_t t0 = block_token(gb0), t1 = block_token(gb1);
+    const int rows = int(t1 - t0);
+    uint16_t* kh = Khat != nullptr ? static_cast<uint16_t*>(Khat) + t0 * ld_hat
+                                   : reinterpret_cast<uint16_t*>(wsb + ws.khat_off);
+    uint16_t* vh = Vhat != nullptr ? static_cast<uint16_t*>(Vhat) + t0 * ld_hat
+                                   : reinterpret_cast<uint16_t*>(wsb + ws.vhat_off);
+    const int64_t ldh = Khat != nullptr ? ld_hat : d;
+    if (has_pred) {
+      rc = launch_predict(c, st, rows, Kpv + t0 * ld_prev, nullptr, ld_prev, 0, Wk, bk, P, d);
+      if (rc) return rc;
+    }
+    rc = launch_decode_rows(c, st, kRoleK, rows, Kcodes + t0 * cb, Kscales + t0 * ng, P, d, kh, ldh);
+    if (rc) return rc;
+    if (has_pred) {
+      rc = launch_predict(c, st, rows, Vpv + t0 * ld_prev, kh, ld_prev, ldh, Wv, bv, P, d);
+      if (rc) return rc;
+    }
+    rc = launch_decode_rows(c, st, kRoleV, rows, Vcodes + t0 * cb, Vscales + t0 * ng, P, d, vh, ldh);
+    if (rc) return rc;
+    AttnArgs a;
+    a.q = static_cast<const uint16_t*>(q);
+    a.Kh = kh;
+    a.Vh = vh;
+    a.ld = ldh;
+    a.tok_base = t0;
+    a.blk_begin = gb0;
+    a.ctx = int(ctx_len);
+    a.n_q_heads = n_q_heads;
+    a.n_kv_heads = n_kv_heads;
+    a.n_splits = ws.n_splits;
+    a.block_tokens = tb;
+    a.scale_log2 = softmax_scale * 1.4426950408889634f;
+    a.part_ml = part_ml;
+    a.part_o = part_o;
+    rc = launch_attn_partial(c, st, a, head_dim, int(gb1 - gb0));
+    if (rc) return rc;
+  }
+  AttnCombineArgs ca;
+  ca.part_ml = part_ml;
+  ca.part_o = part_o;
+  ca.out = static_cast<uint16_t*>(out);
+  ca.lse = lse;
+  ca.n_q_heads = n_q_heads;
+  ca.n_splits = ws.n_splits;
+  return launch_attn_combine(c, st, ca, head_dim, batch);
+}
+
+}  // extern "C"

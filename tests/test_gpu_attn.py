@@ -1,0 +1,81 @@
+"""Parity of the fused decode + single-query attention entry point against the oracle's
+dequantize-then-attend (Algorithm 3 followed by Algorithm 4 lines 5-9)."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2501_19392_b200 import synth
+from parity import check_recon, gpu_bits
+from util import bits_to_f64
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+CASES = [
+    # batch, ctx, n_q, n_kv, head_dim, dtype, adapters
+    (2, 300, 32, 8, 128, synth.BF16, True),     # Llama-3.1-8B head layout, ragged split blocks
+    (3, 700, 24, 8, 128, synth.BF16, True),     # 3 query heads per KV head
+    (1, 1, 32, 8, 128, synth.BF16, False),      # single cached token
+    (2, 257, 64, 8, 128, synth.F16, True),      # 8 query heads per KV head (two passes)
+    (2, 130, 32, 8, 64, synth.F16, True),       # head_dim 64 (d_kv = 512)
+    (1, 2100, 8, 8, 128, synth.BF16, False),    # MHA-style, several chunks of blocks
+]
+
+
+@pytest.mark.parametrize("batch,ctx,n_q,n_kv,hd,dtype,adapters", CASES)
+def test_decode_attn_matches_dequantize_then_attend(batch, ctx, n_q, n_kv, hd, dtype, adapters):
+    from paper_2501_19392_b200 import api
+    d = n_kv * hd
+    T = batch * ctx
+    shape = dataclasses.replace(synth.CONFIGS[5], n_kv_heads=n_kv, head_dim=hd, n_q_heads=n_q,
+                                n_tokens=T, n_layers=2, dtype=dtype, had_block=d, scale_group=d, batch=batch)
+    grid = synth.lloyd_grid(16, seed=7, n_samples=1 << 14, iters=25)
+    sk, sv = synth.hadamard_signs(d, 11), synth.hadamard_signs(d, 12)
+    codec = api.Codec(d, d, d, grid, dtype, sk, sv)
+    ora = oracle.Oracle(d, d, d, grid, dtype, sk, sv)
+    cache = synth.random_cache(shape, seed=5001, n_layers=1)
+    q = synth.random_16bit((batch, n_q, hd), dtype, seed=5002)
+    if adapters:
+        ad = synth.random_adapters(shape, seed=5003)
+        prevK = synth.random_16bit((T, d), dtype, seed=5004)
+        prevV = synth.random_16bit((T, d), dtype, seed=5005)
+        Wk, Wv = ad.Wk[1], ad.Wv[1]
+    else:
+        prevK = prevV = Wk = Wv = None
+    b = lambda t: None if t is None else synth.to_bits(t)
+    kd, vd = ora.decode_layer(cache.Kcodes[0].numpy(), b(cache.Kscales[0]), cache.Vcodes[0].numpy(),
+                              b(cache.Vscales[0]), b(prevK), b(prevV), b(Wk), b(Wv))
+    scale = 1.0 / np.sqrt(hd)
+    ref, ref_lse = oracle.attention(dtype, batch, ctx, n_q, n_kv, hd, scale, b(q), kd["hat"], vd["hat"])
+
+    g = lambda t: None if t is None else t.to(DEV)
+    args = (g(q), g(cache.Kcodes[0]), g(cache.Kscales[0]), g(cache.Vcodes[0]), g(cache.Vscales[0]),
+            ctx, n_kv, scale, g(prevK), g(prevV), g(Wk), g(Wv))
+    Kh = torch.empty((T, d), dtype=codec.torch_dtype, device=DEV)
+    Vh = torch.empty((T, d), dtype=codec.torch_dtype, device=DEV)
+    out, lse = codec.decode_attn(*args, Khat=Kh, Vhat=Vh, want_lse=True)
+    assert codec.poll_status() == 0
+    # (1) the decoded cache the kernel attended over, against the oracle's decode (Algorithm 3)
+    check_recon(gpu_bits(Kh), kd["hat_exact"], kd["hat"], dtype)
+    same = (gpu_bits(Kh) == kd["hat"]).all(axis=1)   # rows whose value predictor saw the oracle's K_hat
+    if same.any():
+        check_recon(gpu_bits(Vh)[same], vd["hat_exact"][same], vd["hat"][same], dtype)
+    # (2) the attention arithmetic, teacher-forced: the oracle attends over the SAME decoded rows
+    #     (one-ulp flips in K_hat/V_hat are legitimate and would otherwise leak into this check).
+    #     Bar: 2e-3 of the head's largest output, or a one-ulp flip of the 16-bit output format.
+    ref2, ref2_lse = oracle.attention(dtype, batch, ctx, n_q, n_kv, hd, scale, b(q), gpu_bits(Kh), gpu_bits(Vh))
+    o = out.to(torch.float64).cpu().numpy()
+    ref2_bits = synth.to_bits(torch.from_numpy(ref2).to(codec.torch_dtype)).astype(np.int64)
+    adjacent = np.abs(gpu_bits(out).astype(np.int64) - ref2_bits) <= 1
+    denom = np.abs(ref2).max(axis=-1, keepdims=True)
+    assert np.all((np.abs(o - ref2) <= 2e-3 * denom) | adjacent)
+    assert np.abs(lse.cpu().numpy() - ref2_lse).max() <= 1e-4
+    # (3) end to end against the oracle's own dequantize-then-attend: the flips add a little
+    assert np.abs(o - ref).max() <= 1e-2 * np.abs(ref).max()
+    assert np.abs(lse.cpu().numpy() - ref_lse).max() <= 2e-3
+    # (4) without the optional K_hat/V_hat outputs the result is bit-identical
+    out_b, lse_b = codec.decode_attn(*args, want_lse=True)
+    assert torch.equal(out_b, out) and torch.equal(lse_b, lse)

@@ -1,0 +1,128 @@
+"""Parity of the CUDA library (through its C ABI) against the CPU oracle, element by element, on
+seeded inputs small enough for the oracle but spanning several 128-row GEMM tiles, several
+8-row codec blocks and ragged tails."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2501_19392_b200 import synth
+from parity import check_codes, check_recon, gpu_bits, scale_rows_ok
+from util import bits_to_f64
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda"
+
+
+def make(d, h, g, n, dtype):
+    from paper_2501_19392_b200 import api
+    grid = synth.lloyd_grid(n, seed=7, n_samples=1 << 14, iters=25)
+    sk, sv = synth.hadamard_signs(d, 11), synth.hadamard_signs(d, 12)
+    return api.Codec(d, h, g, grid, dtype, sk, sv), oracle.Oracle(d, h, g, grid, dtype, sk, sv)
+
+
+def chain(cfg, T, L, seed=0, **kw):
+    shape = dataclasses.replace(synth.CONFIGS[cfg], n_tokens=T, n_layers=L, **kw)
+    kv = synth.kv_chain(shape, seed=1000 * cfg + seed)
+    ad = synth.random_adapters(shape, seed=1000 * cfg + 500 + seed, bias=False)
+    return shape, kv, ad
+
+
+LAYER0_CASES = [
+    (512, 64, 64, 16, synth.F16), (1024, 1024, 1024, 16, synth.BF16), (1024, 1024, 1024, 64, synth.BF16),
+    (1024, 1024, 1024, 256, synth.BF16), (1024, 256, 512, 16, synth.F16), (512, 512, 512, 64, synth.BF16),
+    (256, 256, 256, 16, synth.BF16), (256, 64, 128, 256, synth.F16), (512, 128, 512, 16, synth.BF16),
+]
+
+
+@pytest.mark.parametrize("d,h,g,n,dtype", LAYER0_CASES)
+@pytest.mark.parametrize("T", [1, 37, 300])
+def test_layer0_encode_and_decode_match_oracle(d, h, g, n, dtype, T):
+    codec, ora = make(d, h, g, n, dtype)
+    bits = int(np.log2(n))
+    X = synth.random_16bit((T, d), dtype, seed=d + n + T, std=1.7)
+    Xv = synth.random_16bit((T, d), dtype, seed=d + n + T + 1, std=0.02)
+    ok_, ov_ = ora.encode_layer(synth.to_bits(X), synth.to_bits(Xv))
+    Kc, Ks, Vc, Vs, Kh, Vh = codec.encode(X.to(DEV), Xv.to(DEV))
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    for o, c, s, hhat in ((ok_, Kc, Ks, Kh), (ov_, Vc, Vs, Vh)):
+        rows_ok, n_bad = scale_rows_ok(gpu_bits(s.view(torch.float16)), o["scales"], o["scales_exact"])
+        assert n_bad <= max(1, T // 50)
+        check_codes(c.cpu().numpy(), o, bits, rows_ok)
+    # decode of the ORACLE's codes against the oracle's reconstruction
+    Kh2, Vh2 = codec.decode(torch.from_numpy(ok_["codes"]).to(DEV),
+                            torch.from_numpy(ok_["scales"]).view(torch.float16).to(DEV),
+                            torch.from_numpy(ov_["codes"]).to(DEV),
+                            torch.from_numpy(ov_["scales"]).view(torch.float16).to(DEV))
+    check_recon(gpu_bits(Kh2), ok_["hat_exact"], ok_["hat"], dtype)
+    check_recon(gpu_bits(Vh2), ov_["hat_exact"], ov_["hat"], dtype)
+    # the library's decode of its OWN codes reproduces its encoder's reconstruction bit for bit
+    Kh3, Vh3 = codec.decode(Kc, Ks, Vc, Vs)
+    assert torch.equal(Kh3, Kh) and torch.equal(Vh3, Vh)
+
+
+@pytest.mark.parametrize("cfg,T", [(1, 300), (2, 300), (2, 129), (1, 5)])
+def test_predictor_matches_oracle(cfg, T):
+    shape, kv, ad = chain(cfg, T, 2)
+    codec, ora = make(shape.d_kv, shape.had_block, shape.scale_group, shape.grid_size, shape.dtype)
+    K0, V0 = kv.K[0], kv.V[0]
+    for ins, W in (([K0], ad.Wk[1]), ([V0, K0], ad.Wv[1])):
+        P = codec.predict(ins[0].to(DEV), ins[1].to(DEV) if len(ins) > 1 else None, W.to(DEV))
+        ref = ora.predict([synth.to_bits(t) for t in ins], synth.to_bits(W))
+        err = np.abs(P.cpu().numpy().astype(np.float64) - ref)
+        assert err.max() <= 2e-5 * np.sqrt((ref ** 2).mean()) + 1e-6, err.max()
+    assert codec.poll_status() == 0
+
+
+@pytest.mark.parametrize("cfg,T,n", [(1, 300, 16), (2, 300, 16), (2, 131, 64), (3, 64, 16), (3, 64, 64)])
+def test_encode_with_adapters_teacher_forced(cfg, T, n):
+    shape, kv, ad = chain(cfg, T, 3, grid_size=n)
+    codec, ora = make(shape.d_kv, shape.had_block, shape.scale_group, n, shape.dtype)
+    bits = shape.code_bits
+    prevK = prevV = None            # the oracle's reconstructions feed both sides (teacher forcing)
+    for l in range(shape.n_layers):
+        K, V = kv.K[l], kv.V[l]
+        Wk, Wv = (ad.Wk[l], ad.Wv[l]) if l else (None, None)
+        ok_, ov_ = ora.encode_layer(synth.to_bits(K), synth.to_bits(V), prevK, prevV,
+                                    synth.to_bits(Wk) if l else None, synth.to_bits(Wv) if l else None)
+        dev = lambda a: None if a is None else (a.to(DEV) if isinstance(a, torch.Tensor)
+                                                 else synth.from_bits(a, shape.dtype, DEV))
+        Kc, Ks, Vc, Vs, Kh, Vh = codec.encode(dev(K), dev(V), dev(prevK), dev(prevV), dev(Wk), dev(Wv))
+        assert codec.poll_status() == 0
+        rows_ok, _ = scale_rows_ok(gpu_bits(Ks.view(torch.float16)), ok_["scales"], ok_["scales_exact"])
+        check_codes(Kc.cpu().numpy(), ok_, bits, rows_ok)
+        # reconstruction: rows whose codes agree (a near-tie flip legitimately moves its whole Hadamard block)
+        same_codes = rows_ok & (Kc.cpu().numpy() == ok_["codes"]).all(axis=1)
+        assert same_codes.mean() > 0.9
+        check_recon(gpu_bits(Kh), ok_["hat_exact"], ok_["hat"], shape.dtype, same_codes)
+        # values, teacher-forced inside the layer too: the value phase is given the ORACLE's K_hat
+        from paper_2501_19392_b200 import api
+        okh = dev(ok_["hat"])
+        if l:
+            Vc2, Vs2, Vh2 = codec.encode_phase(api.ROLE_VALUE, dev(V), dev(prevV), okh, dev(Wv))
+        else:
+            Vc2, Vs2, Vh2 = codec.encode_phase(api.ROLE_VALUE, dev(V))
+        rows_ok_v, _ = scale_rows_ok(gpu_bits(Vs2.view(torch.float16)), ov_["scales"], ov_["scales_exact"])
+        check_codes(Vc2.cpu().numpy(), ov_, bits, rows_ok_v)
+        same_codes_v = rows_ok_v & (Vc2.cpu().numpy() == ov_["codes"]).all(axis=1)
+        assert same_codes_v.mean() > 0.9
+        check_recon(gpu_bits(Vh2), ov_["hat_exact"], ov_["hat"], shape.dtype, same_codes_v)
+        # the one-call encode agrees with its own phases wherever its K_hat equals the oracle's
+        same_k = (gpu_bits(Kh) == ok_["hat"]).all(axis=1)
+        if same_k.any():
+            assert np.array_equal(Vc.cpu().numpy()[same_k], Vc2.cpu().numpy()[same_k])
+            assert np.array_equal(gpu_bits(Vh)[same_k], gpu_bits(Vh2)[same_k])
+        # decode on the oracle's codes
+        oc = lambda o: (torch.from_numpy(o["codes"]).to(DEV), torch.from_numpy(o["scales"]).view(torch.float16).to(DEV))
+        Khd = codec.decode_phase(api.ROLE_KEY, *oc(ok_), dev(prevK) if l else None, None, dev(Wk))
+        check_recon(gpu_bits(Khd), ok_["hat_exact"], ok_["hat"], shape.dtype)
+        Vhd = codec.decode_phase(api.ROLE_VALUE, *oc(ov_), dev(prevV) if l else None, okh if l else None, dev(Wv))
+        check_recon(gpu_bits(Vhd), ov_["hat_exact"], ov_["hat"], shape.dtype)
+        # self-consistency: decode(own codes) == encoder's reconstruction, bit for bit
+        Kh3, Vh3 = codec.decode(Kc, Ks, Vc, Vs, dev(prevK), dev(prevV), dev(Wk), dev(Wv))
+        assert torch.equal(Kh3, Kh) and torch.equal(Vh3, Vh)
+        prevK, prevV = ok_["hat"], ov_["hat"]
