@@ -1,0 +1,441 @@
+#!/usr/bin/env python
+"""Benchmark of the AQUA-KV codec hot path on B200.
+
+One "step" is one pass of the whole hot path over one batch of synthetic input: the encode chain
+(Algorithm 2 for every layer, each layer's predictors reading the previous layer's
+reconstruction) followed by the decode + attention chain (Algorithm 3 and the attention read of
+Algorithm 4 for every layer).  The workload is the Llama-3.2-3B-shaped prefill configuration:
+28 layers x 32768 tokens, 8 KV heads x 128 (d_kv = 1024), bf16, 2 bits per value (16-point 2-D
+grid, Hadamard block = scale group = 1024).
+
+Metric: KV tokens/s per layer = tokens x layers carried through the step / step time.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample of the
+same workload instead (the reference arm).
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2501_19392_b200 import synth  # noqa: E402
+
+METRIC = "KV tokens/s per layer (encode + decode-attention round trip) at 2 bits/value"
+UNIT = "token-layers/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], tf_burst=p["bf16_tflops"], tf_sustained=p["bf16_tflops_sustained"],
+                    sm_max_mhz=p.get("sm_max_mhz", 1965.0), source="measured")
+    return dict(hbm_gbs=6650.0, tf_burst=1590.0, tf_sustained=1400.0, sm_max_mhz=1965.0, source="fallback")
+
+
+def workload(args):
+    base = synth.CONFIGS[2]
+    shape = dataclasses.replace(base, n_tokens=args.tokens or base.n_tokens, n_layers=args.layers or base.n_layers)
+    batch = 4 if shape.n_tokens % 4 == 0 and shape.n_tokens >= 4 * 256 else 1
+    return shape, batch
+
+
+def algorithmic_bytes(shape, n_rows_per_call):
+    """Bytes the method itself must move per token-layer (SURVEY 8d style accounting)."""
+    d, g = shape.d_kv, shape.scale_group
+    codes = 2 * (d // 2 * shape.code_bits // 8) + 2 * 2 * (d // g)
+    weights = 6 * d * d / n_rows_per_call
+    enc = 4 * d + 4 * d + 4 * d + codes + weights          # K,V in; prev in; hats out; codes; weights
+    dec = codes + 4 * d + 4 * d + weights                  # codes; prev in; hats out; weights
+    return enc, dec
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+                power.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples"])
+        return dict(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons),
+                    power_w_max=float(max(power)), samples=len(sm))
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle arm (cpu_baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------------
+
+def oracle_sample_run(shape, rows, layers, n_q_heads, seed):
+    """One encode chain + decode chain + attention over `rows` tokens x `layers` layers on the CPU
+    oracle.  Returns seconds."""
+    import oracle
+    small = dataclasses.replace(shape, n_tokens=rows, n_layers=layers)
+    kv = synth.kv_chain(small, seed=seed)
+    ad = synth.random_adapters(small, seed=seed + 1)
+    grid = synth.lloyd_grid(shape.grid_size, seed=7, n_samples=1 << 14, iters=25)
+    o = oracle.Oracle(shape.d_kv, shape.had_block, shape.scale_group, grid, shape.dtype,
+                      synth.hadamard_signs(shape.d_kv, 11), synth.hadamard_signs(shape.d_kv, 12))
+    q = synth.to_bits(synth.random_16bit((1, n_q_heads, shape.head_dim), shape.dtype, seed + 2))
+    Kb = [synth.to_bits(t) for t in kv.K]
+    Vb = [synth.to_bits(t) for t in kv.V]
+    Wk = [None] + [synth.to_bits(w) for w in ad.Wk[1:]]
+    Wv = [None] + [synth.to_bits(w) for w in ad.Wv[1:]]
+    t0 = time.perf_counter()
+    pk = pv = None
+    codes = []
+    for l in range(layers):
+        ek, ev = o.encode_layer(Kb[l], Vb[l], pk, pv, Wk[l], Wv[l])
+        codes.append((ek["codes"], ek["scales"], ev["codes"], ev["scales"]))
+        pk, pv = ek["hat"], ev["hat"]
+    pk = pv = None
+    for l in range(layers):
+        dk, dv = o.decode_layer(*codes[l], pk, pv, Wk[l], Wv[l])
+        pk, pv = dk["hat"], dv["hat"]
+        oracle.attention(shape.dtype, 1, rows, n_q_heads, shape.n_kv_heads, shape.head_dim,
+                         1.0 / math.sqrt(shape.head_dim), q, pk, pv)
+    return time.perf_counter() - t0
+
+
+def oracle_baseline(shape, n_q_heads, target_s=12.0):
+    import oracle
+    probe_rows, layers = 64, 2
+    t = oracle_sample_run(shape, probe_rows, layers, n_q_heads, seed=2000)
+    per_unit = t / (probe_rows * layers)
+    rows = int(min(8192, max(64, target_s / (per_unit * 4))))
+    rows = rows // 64 * 64
+    layers = 4
+    t = oracle_sample_run(shape, rows, layers, n_q_heads, seed=2001)
+    return dict(value=rows * layers / t, unit=UNIT, cores=oracle.num_threads(), kind="oracle",
+                sample="%d tokens x %d layers of the workload (encode chain + decode chain + attention), %.1f s"
+                       % (rows, layers, t))
+
+
+def run_reference(args):
+    """Reference arm: the CPU oracle as it stands, on a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    shape, _ = workload(args)
+    n_q = shape.n_q_heads
+    rows, layers = 256, 4
+    for _ in range(args.warmup):
+        oracle_sample_run(shape, 64, 2, n_q, seed=2100)
+    t0 = time.perf_counter()
+    for s in range(args.steps):
+        oracle_sample_run(shape, rows, layers, n_q, seed=2200 + s)
+    dt = (time.perf_counter() - t0) / args.steps
+    val = rows * layers / dt
+    sample = "%d tokens x %d layers per step" % (rows, layers)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": shape.name, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--tokens", type=int, default=0, help="override tokens per GPU (testing only)")
+    ap.add_argument("--layers", type=int, default=0, help="override layer count (testing only)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    from paper_2501_19392_b200 import api, chain    # raises if the CUDA library is missing
+
+    peaks = load_peaks()
+    shape, batch = workload(args)
+    T, L, d = shape.n_tokens, shape.n_layers, shape.d_kv
+    ctx_len = T // batch
+    n_q = shape.n_q_heads
+    scale = 1.0 / math.sqrt(shape.head_dim)
+
+    # ---- synthetic inputs, resident in HBM (each rank draws its own tokens: weak scaling) ----------
+    seed = 2000 + 17 * rank
+    kv = synth.kv_chain(shape, seed=seed, device=dev)
+    ad = synth.random_adapters(shape, seed=2500, device=dev)
+    grid = synth.lloyd_grid(shape.grid_size, seed=7, n_samples=1 << 14, iters=25)
+    codec = api.Codec(d, shape.had_block, shape.scale_group, grid, shape.dtype,
+                      synth.hadamard_signs(d, 11), synth.hadamard_signs(d, 12))
+    cache = chain.CompressedCache.empty(codec, L, T, dev)
+    bufs = chain.PingPong(codec, T, dev)
+    q = [synth.random_16bit((batch, n_q, shape.head_dim), shape.dtype, 2600 + l, device=dev) for l in range(L)]
+    out = [torch.empty_like(q[0]) for _ in range(L)]
+
+    def step(ev_mid=None):
+        chain.encode_chain(codec, kv.K, kv.V, ad, cache, bufs)
+        if ev_mid is not None:
+            ev_mid.record()
+        chain.decode_attn_chain(codec, cache, ad, bufs, q, out, ctx_len, shape.n_kv_heads, scale)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0, "device status word reports a timed-out wait"
+
+    # ---- timed region --------------------------------------------------------------------------
+    sampler = ClockSampler(local)
+    codec.profile_enable(True)
+    launches0 = codec.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    mids = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True),
+             torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    sampler.start()
+    ev0.record()
+    for s in range(args.steps):
+        mids[s][0].record()
+        step(mids[s][1])
+        mids[s][2].record()
+    ev1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = ev0.elapsed_time(ev1)
+    launches = codec.launch_count() - launches0
+    enc_ms = sum(a.elapsed_time(b) for a, b, _ in mids) / args.steps
+    dec_ms = sum(b.elapsed_time(c) for _, b, c in mids) / args.steps
+    prof = {name: codec.profile_read(k) for name, k in
+            (("predict_gemm", api.KERNEL_PREDICT), ("encode_rows", api.KERNEL_ENCODE_ROWS),
+             ("decode_rows", api.KERNEL_DECODE_ROWS), ("attention", api.KERNEL_ATTN))}
+    codec.profile_enable(False)
+    assert codec.poll_status() == 0
+
+    ms_step = ms_total / args.steps
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_step], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step = float(t.item())
+    value = world * T * L / (ms_step * 1e-3)
+
+    # ---- plain decode chain (Algorithm 3 alone), reported beside the step ----------------------------
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    chain.decode_chain(codec, cache, ad, bufs)
+    torch.cuda.synchronize()
+    e0.record()
+    chain.decode_chain(codec, cache, ad, bufs)
+    e1.record()
+    torch.cuda.synchronize()
+    plain_dec_ms = e0.elapsed_time(e1)
+
+    # ---- rooflines --------------------------------------------------------------------------------
+    rows_per_call = min(T, 2 * 148 * 128 * 256 // d)
+    enc_bytes, dec_bytes = algorithmic_bytes(shape, T)
+    flops_tl = 6.0 * d * d * (L - 1) / L                    # layer 0 has no predictor
+    t_tensor = flops_tl / (peaks["tf_burst"] * 1e12)
+    roof = {}
+    for name, ms, by in (("encode", enc_ms, enc_bytes), ("decode_attn", dec_ms, dec_bytes),
+                         ("decode", plain_dec_ms, dec_bytes)):
+        t_hbm = by / (peaks["hbm_gbs"] * 1e9)
+        t_roof = max(t_tensor, t_hbm)
+        tps = T * L / (ms * 1e-3)
+        roof[name] = {"token_layers_per_s": tps, "ms": ms, "roofline_token_layers_per_s": 1.0 / t_roof,
+                      "frac_of_roofline": tps * t_roof, "bound": "tensor" if t_tensor >= t_hbm else "hbm",
+                      "achieved_tflops": tps * flops_tl / 1e12, "achieved_gbs": tps * by / 1e9}
+
+    n_g, ms_g = prof["predict_gemm"]
+    gemm_flops_total = args.steps * 2 * (L - 1) * 6.0 * d * d * T      # encode + decode-attn chains
+    kernels = {}
+    for name, (n, ms) in prof.items():
+        kernels[name] = {"launches": n, "total_ms": ms, "share": ms / max(1e-9, sum(v[1] for v in prof.values()))}
+    # Dominant kernel by time share.  The GEMM is tensor-bound; the row kernels are bound by plain
+    # ALU work (butterflies + nearest-point search), reported against lanes x clock.
+    dominant = max(prof.items(), key=lambda kv_: kv_[1][1])[0]
+    alu_peak = 148 * 128 * peaks["sm_max_mhz"] * 1e6 / 1e12       # T lane-ops/s
+    if dominant == "predict_gemm":
+        achieved = gemm_flops_total / (ms_g * 1e-3) / 1e12
+        roofline = {"kernel": "gemm_pred_kernel", "bound": "tensor", "achieved": achieved,
+                    "peak": peaks["tf_sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["tf_sustained"],
+                    "traffic": None, "peak_source": peaks["source"] + " (sustained)"}
+    else:
+        n_r, ms_r = prof[dominant]
+        rows_total = args.steps * 2 * L * T                            # K and V rows
+        lane_ops = {"encode_rows": 77000.0, "decode_rows": 16000.0}.get(dominant, 8000.0)
+        achieved = rows_total * lane_ops / (ms_r * 1e-3) / 1e12
+        roofline = {"kernel": dominant, "bound": "alu", "achieved": achieved, "peak": alu_peak,
+                    "unit": "T lane-ops/s", "frac": achieved / alu_peak, "traffic": None,
+                    "peak_source": "148 SMs x 128 lanes x max SM clock"}
+    gemm_tf = gemm_flops_total / max(1e-9, ms_g * 1e-3) / 1e12
+    kernels["predict_gemm"].update({"achieved_tflops": gemm_tf, "frac_of_sustained_peak": gemm_tf / peaks["tf_sustained"]})
+
+    # ---- end to end through the C ABI with host buffers ------------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(args, codec, chain, shape, kv, ad, cache, bufs, q, out, ctx_len, scale, dev, world)
+
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": shape.name, "tokens_per_gpu": T, "layers": L, "d_kv": d, "bits_per_value": 2,
+                   "grid_points": shape.grid_size, "hadamard_block": shape.had_block, "attn_batch": batch,
+                   "attn_ctx": ctx_len, "n_q_heads": n_q, "l2": "inputs (%.1f GB of K/V per step) exceed L2" %
+                   (2 * L * T * d * 2 / 1e9), "rows_per_chunk": rows_per_call},
+        "ops": roof, "kernels": kernels, "roofline": roofline, "clocks": clocks, "gpu_launches": launches,
+        "e2e": e2e,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        result["cpu_baseline"] = oracle_baseline(shape, n_q)
+    if rank == 0:
+        print(json.dumps(result))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def run_e2e(args, codec, chain, shape, kv, ad, cache, bufs, q, out, ctx_len, scale, dev, world):
+    """Same step, but every input starts in pinned host memory and every product ends there:
+    per layer H2D(K, V) -> encode -> D2H(codes, scales); then H2D(codes, scales, q) -> decode +
+    attention -> D2H(attention output).  Copies are inside the timed region."""
+    T, L, d = shape.n_tokens, shape.n_layers, shape.d_kv
+    pin = lambda t: torch.empty(t.shape, dtype=t.dtype, device="cpu", pin_memory=True).copy_(t)
+    hK = [pin(t) for t in kv.K]
+    hV = [pin(t) for t in kv.V]
+    hq = [pin(t) for t in q]
+    hc = [[torch.empty(t.shape, dtype=t.dtype, device="cpu", pin_memory=True) for t in lst]
+          for lst in (cache.Kcodes, cache.Kscales, cache.Vcodes, cache.Vscales)]
+    ho = [torch.empty(t.shape, dtype=t.dtype, device="cpu", pin_memory=True) for t in out]
+    dK = torch.empty_like(kv.K[0])
+    dV = torch.empty_like(kv.V[0])
+    dq = torch.empty_like(q[0])
+    dlists = (cache.Kcodes, cache.Kscales, cache.Vcodes, cache.Vscales)
+
+    def e2e_step():
+        for l in range(L):
+            dK.copy_(hK[l], non_blocking=True)
+            dV.copy_(hV[l], non_blocking=True)
+            cur, prv = l % 2, (l + 1) % 2
+            has = l > 0
+            codec.encode(dK, dV, bufs.K[prv] if has else None, bufs.V[prv] if has else None,
+                         ad.Wk[l] if has else None, ad.Wv[l] if has else None, None, None,
+                         cache.Kcodes[l], cache.Kscales[l], cache.Vcodes[l], cache.Vscales[l],
+                         bufs.K[cur], bufs.V[cur])
+            for h, dl in zip(hc, dlists):
+                h[l].copy_(dl[l], non_blocking=True)
+        for l in range(L):
+            for h, dl in zip(hc, dlists):
+                dl[l].copy_(h[l], non_blocking=True)
+            dq.copy_(hq[l], non_blocking=True)
+            cur, prv = l % 2, (l + 1) % 2
+            has = l > 0
+            codec.decode_attn(dq, cache.Kcodes[l], cache.Kscales[l], cache.Vcodes[l], cache.Vscales[l],
+                              ctx_len, shape.n_kv_heads, scale,
+                              bufs.K[prv] if has else None, bufs.V[prv] if has else None,
+                              ad.Wk[l] if has else None, ad.Wv[l] if has else None, None, None,
+                              out=out[l], Khat=bufs.K[cur], Vhat=bufs.V[cur])
+            ho[l].copy_(out[l], non_blocking=True)
+
+    nbytes = lambda ts: sum(t.numel() * t.element_size() for t in ts)
+    code_bytes = sum(nbytes(lst) for lst in hc)
+    h2d = nbytes(hK) + nbytes(hV) + code_bytes + nbytes(hq)
+    d2h = code_bytes + nbytes(ho)
+    e2e_step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    steps = max(1, min(args.steps, 2))
+    e0.record()
+    for _ in range(steps):
+        e2e_step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return {"value": world * T * L / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+            "d2h_bytes_per_step": int(d2h), "ms_per_step": ms}
+
+
+if __name__ == "__main__":
+    main()

@@ -210,6 +210,21 @@ int aquakv_poll_status(aquakv_ctx* ctx, void* cuda_stream);
 /* Number of kernels this context has launched since creation (for benchmarks' bookkeeping). */
 int64_t aquakv_launch_count(const aquakv_ctx* ctx);
 
+/*
+ * Optional per-kernel timing for benchmarks.  While enabled, every kernel launch of this context
+ * is bracketed by a pair of CUDA events on the launching stream (up to 8192 launches; later ones
+ * are not recorded).  aquakv_profile_enable(ctx, 1) creates the events on first use (do this
+ * outside stream capture) and clears the record; (ctx, 0) stops recording.
+ * aquakv_profile_read waits for the recorded launches of one kernel class and returns their
+ * number and summed device time.  Not part of the paper's method: measurement support only.
+ */
+#define AQUAKV_KERNEL_PREDICT 0     /* tcgen05 predictor GEMM                    */
+#define AQUAKV_KERNEL_ENCODE_ROWS 1 /* residual, scale, rotation, search, pack   */
+#define AQUAKV_KERNEL_DECODE_ROWS 2 /* unpack, gather, inverse rotation, add-back */
+#define AQUAKV_KERNEL_ATTN 3        /* split-KV attention partials and combine   */
+int aquakv_profile_enable(aquakv_ctx* ctx, int enable);
+int aquakv_profile_read(aquakv_ctx* ctx, int kernel_class, int64_t* launches, double* total_ms);
+
 /* Static, human-readable name of a status code. */
 const char* aquakv_status_string(int status);
 

@@ -21,6 +21,7 @@ OP_DECODE = 1
 OP_DECODE_ATTN = 2
 ROLE_KEY = 0
 ROLE_VALUE = 1
+KERNEL_PREDICT, KERNEL_ENCODE_ROWS, KERNEL_DECODE_ROWS, KERNEL_ATTN = 0, 1, 2, 3
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libaquakv.so")
@@ -29,6 +30,7 @@ SYMBOLS = [
     "aquakv_code_bytes", "aquakv_create", "aquakv_destroy", "aquakv_workspace_bytes",
     "aquakv_decode_attn_workspace_bytes", "aquakv_predict", "aquakv_encode", "aquakv_decode",
     "aquakv_decode_attn", "aquakv_encode_phase", "aquakv_decode_phase", "aquakv_poll_status", "aquakv_launch_count", "aquakv_status_string",
+    "aquakv_profile_enable", "aquakv_profile_read",
 ]
 
 
@@ -80,6 +82,10 @@ def _load():
     L.aquakv_poll_status.argtypes = [vp, vp]
     L.aquakv_launch_count.restype = i64
     L.aquakv_launch_count.argtypes = [vp]
+    L.aquakv_profile_enable.restype = ctypes.c_int
+    L.aquakv_profile_enable.argtypes = [vp, ctypes.c_int]
+    L.aquakv_profile_read.restype = ctypes.c_int
+    L.aquakv_profile_read.argtypes = [vp, ctypes.c_int, ctypes.POINTER(i64), ctypes.POINTER(ctypes.c_double)]
     L.aquakv_status_string.restype = ctypes.c_char_p
     L.aquakv_status_string.argtypes = [ctypes.c_int]
     return L
@@ -255,3 +261,15 @@ class Codec:
 
     def launch_count(self) -> int:
         return int(lib.aquakv_launch_count(self.h))
+
+    def profile_enable(self, enable: bool) -> None:
+        rc = lib.aquakv_profile_enable(self.h, 1 if enable else 0)
+        if rc:
+            raise AquaKVError(rc, "aquakv_profile_enable")
+
+    def profile_read(self, kernel_class: int):
+        n, ms = ctypes.c_int64(0), ctypes.c_double(0.0)
+        rc = lib.aquakv_profile_read(self.h, kernel_class, ctypes.byref(n), ctypes.byref(ms))
+        if rc:
+            raise AquaKVError(rc, "aquakv_profile_read")
+        return int(n.value), float(ms.value)

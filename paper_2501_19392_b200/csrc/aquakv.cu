@@ -42,11 +42,34 @@ struct aquakv_ctx {
   GridConst<64> gc64;
   EncodeTiledFn encode_tiled;
   int64_t launches;
+  // optional per-kernel-class timing (aquakv_profile_*): event pairs recorded around launches
+  bool prof_on;
+  int prof_n;                       // pairs recorded since the last read
+  cudaEvent_t* prof_ev;             // 2 * kProfMaxPairs events, created when profiling is enabled
+  uint8_t* prof_class;              // kernel class of each pair
 };
 
 namespace {
 
 constexpr int kRoleK = 0, kRoleV = 1;
+constexpr int kProfMaxPairs = 8192;
+
+// Brackets one kernel launch with a pair of events when profiling is enabled.
+struct ProfScope {
+  aquakv_ctx* c;
+  cudaStream_t st;
+  int slot;
+  ProfScope(aquakv_ctx* ctx, cudaStream_t s, int kernel_class) : c(ctx), st(s), slot(-1) {
+    if (c->prof_on && c->prof_n < kProfMaxPairs) {
+      slot = c->prof_n++;
+      c->prof_class[slot] = uint8_t(kernel_class);
+      cudaEventRecord(c->prof_ev[2 * slot], st);
+    }
+  }
+  ~ProfScope() {
+    if (slot >= 0) cudaEventRecord(c->prof_ev[2 * slot + 1], st);
+  }
+};
 
 inline int ilog2(int v) {
   int b = 0;
@@ -117,6 +140,7 @@ int launch_predict(aquakv_ctx* c, cudaStream_t st, int M, const void* in0, const
   g.status = c->d_status;
   const int tiles = ((M + kBM - 1) / kBM) * (d / kBN);
   const int grid = tiles < c->sm_count ? tiles : c->sm_count;
+  ProfScope prof(c, st, AQUAKV_KERNEL_PREDICT);
   if (c->bf16) {
     gemm_pred_kernel<true><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(tA0, tA1, tB, g);
   } else {
@@ -198,6 +222,7 @@ int launch_encode_rows(aquakv_ctx* c, cudaStream_t st, int role, int rows, const
   a.hat = static_cast<uint16_t*>(hat);
   a.ldHat = ldHat;
   const int grid = codec_grid(c, rows);
+  ProfScope prof(c, st, AQUAKV_KERNEL_ENCODE_ROWS);
   AQ_DISPATCH_DNB(launch_encode_rows_t, c, st, a, grid);
   ++c->launches;
   return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
@@ -215,6 +240,7 @@ int launch_decode_rows(aquakv_ctx* c, cudaStream_t st, int role, int rows, const
   a.hat = static_cast<uint16_t*>(hat);
   a.ldHat = ldHat;
   const int grid = codec_grid(c, rows);
+  ProfScope prof(c, st, AQUAKV_KERNEL_DECODE_ROWS);
   AQ_DISPATCH_DNB(launch_decode_rows_t, c, st, a, grid);
   ++c->launches;
   return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
@@ -239,6 +265,7 @@ int launch_attn_partial(aquakv_ctx* c, cudaStream_t st, const AttnArgs& a, int h
   int passes = 0;
   const int gq = attn_gq(a.n_q_heads / a.n_kv_heads, &passes);
   const dim3 grid(n_blocks, a.n_kv_heads, passes);
+  ProfScope prof(c, st, AQUAKV_KERNEL_ATTN);
 #define AQ_ATTN(HD, GQ)                                                   \
   if (head_dim == HD && gq == GQ) {                                       \
     if (c->bf16) launch_attn_partial_t<HD, GQ, true>(st, a, grid);        \
@@ -254,6 +281,7 @@ int launch_attn_partial(aquakv_ctx* c, cudaStream_t st, const AttnArgs& a, int h
 int launch_attn_combine(aquakv_ctx* c, cudaStream_t st, const AttnCombineArgs& a, int head_dim,
                         int batch) {
   const int grid = batch * a.n_q_heads;
+  ProfScope prof(c, st, AQUAKV_KERNEL_ATTN);
   if (head_dim == 64) {
     if (c->bf16) attn_combine_kernel<64, true><<<grid, 64, 0, st>>>(a);
     else attn_combine_kernel<64, false><<<grid, 64, 0, st>>>(a);
@@ -445,6 +473,12 @@ int aquakv_destroy(aquakv_ctx* c) {
   if (c->d_signmask[0]) ok = cudaFree(c->d_signmask[0]) == cudaSuccess && ok;
   if (c->d_signmask[1]) ok = cudaFree(c->d_signmask[1]) == cudaSuccess && ok;
   if (c->d_status) ok = cudaFree(c->d_status) == cudaSuccess && ok;
+  if (c->prof_ev) {
+    for (int i = 0; i < 2 * kProfMaxPairs; ++i)
+      if (c->prof_ev[i]) cudaEventDestroy(c->prof_ev[i]);
+    delete[] c->prof_ev;
+    delete[] c->prof_class;
+  }
   delete c;
   return ok ? AQUAKV_OK : AQUAKV_ERR_CUDA;
 }
@@ -462,6 +496,36 @@ size_t aquakv_decode_attn_workspace_bytes(const aquakv_ctx* c, int32_t batch, in
 }
 
 int64_t aquakv_launch_count(const aquakv_ctx* c) { return c ? c->launches : 0; }
+
+int aquakv_profile_enable(aquakv_ctx* c, int enable) {
+  if (c == nullptr) return AQUAKV_ERR_INVALID_ARG;
+  if (enable && c->prof_ev == nullptr) {
+    c->prof_ev = new (std::nothrow) cudaEvent_t[2 * kProfMaxPairs]();
+    c->prof_class = new (std::nothrow) uint8_t[kProfMaxPairs]();
+    if (c->prof_ev == nullptr || c->prof_class == nullptr) return AQUAKV_ERR_CUDA;
+    for (int i = 0; i < 2 * kProfMaxPairs; ++i)
+      if (cudaEventCreate(&c->prof_ev[i]) != cudaSuccess) return AQUAKV_ERR_CUDA;
+  }
+  c->prof_on = enable != 0;
+  c->prof_n = 0;
+  return AQUAKV_OK;
+}
+
+int aquakv_profile_read(aquakv_ctx* c, int kernel_class, int64_t* launches, double* total_ms) {
+  if (c == nullptr || launches == nullptr || total_ms == nullptr) return AQUAKV_ERR_INVALID_ARG;
+  *launches = 0;
+  *total_ms = 0.0;
+  for (int i = 0; i < c->prof_n; ++i) {
+    if (c->prof_class[i] != kernel_class) continue;
+    if (cudaEventSynchronize(c->prof_ev[2 * i + 1]) != cudaSuccess) return AQUAKV_ERR_CUDA;
+    float ms = 0.0f;
+    if (cudaEventElapsedTime(&ms, c->prof_ev[2 * i], c->prof_ev[2 * i + 1]) != cudaSuccess)
+      return AQUAKV_ERR_CUDA;
+    *total_ms += ms;
+    ++*launches;
+  }
+  return AQUAKV_OK;
+}
 
 int aquakv_poll_status(aquakv_ctx* c, void* cuda_stream) {
   if (c == nullptr) return AQUAKV_ERR_INVALID_ARG;
