@@ -58,6 +58,7 @@ extern "C" {
 #define AQUAKV_ERR_WORKSPACE (-4)   /* workspace NULL or smaller than aquakv_workspace_bytes */
 #define AQUAKV_ERR_CUDA (-5)        /* a CUDA runtime/driver call failed                     */
 #define AQUAKV_ERR_TIMEOUT (-6)     /* a bounded device-side wait expired (see poll_status)  */
+#define AQUAKV_ERR_TOO_LARGE (-7)   /* more tokens than the fixed scratch of a *_noalloc call  */
 
 #define AQUAKV_OP_ENCODE 0
 #define AQUAKV_OP_DECODE 1
@@ -175,6 +176,39 @@ int aquakv_decode(aquakv_ctx* ctx, int64_t n_tokens,
                   const void* Wk, const void* Wv, const float* bk, const float* bv,
                   void* Khat, void* Vhat, int64_t ld_hat,
                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * aquakv_decode for callers that cannot allocate device memory and therefore have no workspace to
+ * hand over.  (The paper has no counterpart: this is a packaging variant of aquakv_decode, same
+ * arithmetic, same kernels.)  Who needs it: a decode step running inside a region where
+ * cudaMalloc is off limits -- a plugin that is given device buffers for its inputs and outputs only,
+ * an inference server whose memory pool is frozen after start-up, a real-time loop that must not
+ * take the allocator's locks or its implicit device synchronisation.
+ *
+ * The fp32 prediction that aquakv_decode keeps in the caller's workspace lives here in a fixed
+ * array inside the library image: AQUAKV_NOALLOC_MAX_TOKENS * 1024 * 4 bytes = 4 MiB of device
+ * memory, reserved on every GPU that loads the library for as long as the process lives.  The
+ * call itself performs no cudaMalloc / cudaFree and calls no routine that allocates.
+ *
+ *   - n_tokens > AQUAKV_NOALLOC_MAX_TOKENS returns AQUAKV_ERR_TOO_LARGE and launches nothing;
+ *     split larger batches into several calls on the same stream.
+ *   - The first call on a device looks up the array's device address (once per device, with that
+ *     device current, which must be the context's device).  Make that first call during start-up,
+ *     before any stream capture; later calls only launch kernels.
+ *   - Every call on a device uses the same array.  Calls issued to one stream are ordered and
+ *     safe; calls that can overlap on the GPU (different streams, different contexts or threads)
+ *     race on it and produce garbage.  The array keeps whatever the last call left there; nothing
+ *     in it needs to start at zero because each call overwrites every row it later reads.
+ *   - All other arguments, results (bit-identical to aquakv_decode) and errors are those of
+ *     aquakv_decode.
+ */
+#define AQUAKV_NOALLOC_MAX_TOKENS 1024
+int aquakv_decode_noalloc(aquakv_ctx* ctx, int64_t n_tokens,
+                          const uint8_t* Kcodes, const uint16_t* Kscales,
+                          const uint8_t* Vcodes, const uint16_t* Vscales,
+                          const void* Khat_prev, const void* Vhat_prev, int64_t ld_prev,
+                          const void* Wk, const void* Wv, const float* bk, const float* bv,
+                          void* Khat, void* Vhat, int64_t ld_hat, void* cuda_stream);
 
 /*
  * Algorithm 3 fused with the attention read of Algorithm 4 (lines 5-9) for single-token queries:

@@ -21,6 +21,7 @@ OP_DECODE = 1
 OP_DECODE_ATTN = 2
 ROLE_KEY = 0
 ROLE_VALUE = 1
+NOALLOC_MAX_TOKENS = 1024
 KERNEL_PREDICT, KERNEL_ENCODE_ROWS, KERNEL_DECODE_ROWS, KERNEL_ATTN = 0, 1, 2, 3
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -29,7 +30,7 @@ LIB_PATH = os.path.join(_HERE, "libaquakv.so")
 SYMBOLS = [
     "aquakv_code_bytes", "aquakv_create", "aquakv_destroy", "aquakv_workspace_bytes",
     "aquakv_decode_attn_workspace_bytes", "aquakv_predict", "aquakv_encode", "aquakv_decode",
-    "aquakv_decode_attn", "aquakv_encode_phase", "aquakv_decode_phase", "aquakv_poll_status", "aquakv_launch_count", "aquakv_status_string",
+    "aquakv_decode_attn", "aquakv_decode_noalloc", "aquakv_encode_phase", "aquakv_decode_phase", "aquakv_poll_status", "aquakv_launch_count", "aquakv_status_string",
     "aquakv_profile_enable", "aquakv_profile_read",
 ]
 
@@ -70,6 +71,9 @@ def _load():
     L.aquakv_decode.restype = ctypes.c_int
     L.aquakv_decode.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp,
                                 vp, vp, i64, vp, sz, vp]
+    L.aquakv_decode_noalloc.restype = ctypes.c_int
+    L.aquakv_decode_noalloc.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp,
+                                        vp, vp, i64, vp]
     L.aquakv_decode_attn.restype = ctypes.c_int
     L.aquakv_decode_attn.argtypes = [vp, i32, i64, i32, i32, i32, f32, vp, vp, vp, vp, vp,
                                      vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, sz, vp]
@@ -210,6 +214,23 @@ class Codec:
                                _ptr(ws), ws.numel(), _stream())
         if rc:
             raise AquaKVError(rc, "aquakv_decode")
+        return Khat, Vhat
+
+    def decode_noalloc(self, Kcodes, Kscales, Vcodes, Vscales, Khat_prev=None, Vhat_prev=None, Wk=None,
+                       Wv=None, bk=None, bv=None, Khat=None, Vhat=None):
+        """aquakv_decode_noalloc: decode without a workspace, for callers that may not allocate
+        device memory; at most NOALLOC_MAX_TOKENS tokens per call.  Khat/Vhat should be passed in by
+        such callers (this wrapper creates them with torch only when they are omitted)."""
+        T, dev = Kcodes.shape[0], Kcodes.device
+        if Khat is None:
+            Khat = torch.empty((T, self.d), dtype=self.torch_dtype, device=dev)
+            Vhat = torch.empty((T, self.d), dtype=self.torch_dtype, device=dev)
+        rc = lib.aquakv_decode_noalloc(self.h, T, _ptr(Kcodes), _ptr(Kscales), _ptr(Vcodes), _ptr(Vscales),
+                                       _ptr(Khat_prev), _ptr(Vhat_prev), _ld(Khat_prev, self.d), _ptr(Wk),
+                                       _ptr(Wv), _ptr(bk), _ptr(bv), _ptr(Khat), _ptr(Vhat),
+                                       _ld(Khat, self.d), _stream())
+        if rc:
+            raise AquaKVError(rc, "aquakv_decode_noalloc")
         return Khat, Vhat
 
     def decode_attn(self, q, Kcodes, Kscales, Vcodes, Vscales, ctx_len: int, n_kv_heads: int,

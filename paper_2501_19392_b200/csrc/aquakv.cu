@@ -13,6 +13,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "aquakv.h"
@@ -385,6 +386,7 @@ const char* aquakv_status_string(int status) {
     case AQUAKV_ERR_WORKSPACE: return "workspace missing or too small";
     case AQUAKV_ERR_CUDA: return "CUDA call failed";
     case AQUAKV_ERR_TIMEOUT: return "bounded device-side wait expired";
+    case AQUAKV_ERR_TOO_LARGE: return "more tokens than the fixed scratch of the no-allocation call holds";
     default: return "unknown status";
   }
 }
@@ -757,6 +759,71 @@ int aquakv_decode(aquakv_ctx* c, int64_t n_tokens, const uint8_t* Kcodes, const 
     if (rc) return rc;
   }
   return AQUAKV_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// aquakv_decode without a caller workspace: the prediction goes through a fixed array that is part
+// of the library image.  In host code the symbol below is only a handle; the device address the
+// kernels need comes from cudaGetSymbolAddress, looked up once per device.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char
+    g_noalloc_scratch[size_t(AQUAKV_NOALLOC_MAX_TOKENS) * 1024 * sizeof(float)];
+
+namespace {
+constexpr int kNoallocMaxDevices = 64;
+std::mutex g_noalloc_mu;
+float* g_noalloc_ptr[kNoallocMaxDevices] = {};
+
+// Device address of the scratch array on `device`, which must be the current device.
+int noalloc_scratch(int device, float** out) {
+  if (device < 0 || device >= kNoallocMaxDevices) return AQUAKV_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_noalloc_mu);
+  if (g_noalloc_ptr[device] == nullptr) {
+    int cur = -1;
+    if (cudaGetDevice(&cur) != cudaSuccess) return AQUAKV_ERR_CUDA;
+    if (cur != device) return AQUAKV_ERR_INVALID_ARG;
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) {
+      (void)cudaGetLastError();
+      return AQUAKV_ERR_CUDA;
+    }
+    g_noalloc_ptr[device] = static_cast<float*>(p);
+  }
+  *out = g_noalloc_ptr[device];
+  return AQUAKV_OK;
+}
+}  // namespace
+
+int aquakv_decode_noalloc(aquakv_ctx* c, int64_t n_tokens, const uint8_t* Kcodes,
+                          const uint16_t* Kscales, const uint8_t* Vcodes, const uint16_t* Vscales,
+                          const void* Khat_prev, const void* Vhat_prev, int64_t ld_prev,
+                          const void* Wk, const void* Wv, const float* bk, const float* bv,
+                          void* Khat, void* Vhat, int64_t ld_hat, void* cuda_stream) {
+  if (c == nullptr || n_tokens < 0) return AQUAKV_ERR_INVALID_ARG;
+  if (n_tokens > AQUAKV_NOALLOC_MAX_TOKENS) return AQUAKV_ERR_TOO_LARGE;
+  if (n_tokens == 0) return AQUAKV_OK;
+  const int d = c->p.d_kv;   // <= 1024, so n_tokens * d floats fit the array
+  int rc;
+  if ((rc = check_rows(Khat, ld_hat, d, true))) return rc;
+  if ((rc = check_rows(Vhat, ld_hat, d, true))) return rc;
+  if (Kcodes == nullptr || Kscales == nullptr || Vcodes == nullptr || Vscales == nullptr)
+    return AQUAKV_ERR_INVALID_ARG;
+  bool has_pred = false;
+  if ((rc = check_adapters(Khat_prev, Vhat_prev, ld_prev, Wk, Wv, bk, bv, d, &has_pred))) return rc;
+  if (Khat == Khat_prev || Khat == Vhat_prev || Vhat == Vhat_prev || Vhat == Khat_prev || Vhat == Khat)
+    return AQUAKV_ERR_INVALID_ARG;
+  float* P = nullptr;
+  if (has_pred && (rc = noalloc_scratch(c->device, &P))) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int rows = int(n_tokens);
+  const uint16_t* Kpv = static_cast<const uint16_t*>(Khat_prev);
+  const uint16_t* Vpv = static_cast<const uint16_t*>(Vhat_prev);
+  uint16_t* Kh = static_cast<uint16_t*>(Khat);
+  uint16_t* Vh = static_cast<uint16_t*>(Vhat);
+  if (has_pred && (rc = launch_predict(c, st, rows, Kpv, nullptr, ld_prev, 0, Wk, bk, P, d))) return rc;
+  if ((rc = launch_decode_rows(c, st, kRoleK, rows, Kcodes, Kscales, P, d, Kh, ld_hat))) return rc;
+  if (has_pred && (rc = launch_predict(c, st, rows, Vpv, Kh, ld_prev, ld_hat, Wv, bv, P, d))) return rc;
+  return launch_decode_rows(c, st, kRoleV, rows, Vcodes, Vscales, P, d, Vh, ld_hat);
 }
 
 int aquakv_decode_attn(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_heads,
