@@ -90,6 +90,19 @@ int aquakv_code_bytes(const aquakv_params* params);
 int aquakv_create(const aquakv_params* params, const float* grid_host, const int8_t* signs_k_host,
                   const int8_t* signs_v_host, aquakv_ctx** out);
 
+/*
+ * The host-built cell table that prunes the nearest-point search of Q (Section 2: each pair of
+ * rotated values goes to the nearest grid point).  The square [-half_extent, half_extent)^2 is cut
+ * into cells_per_side^2 cells; entry [iy*cells_per_side + ix] holds, in bytes 0..3, the ascending
+ * indices of every grid point that is nearest somewhere in that cell (short lists repeat the last
+ * index; at most three distinct ones for grid_size 16, four otherwise), and the value 1 means
+ * "more than that: search all points".  The kernels use the same
+ * table, so a host test can check that it never excludes the true nearest point.  HOST memory
+ * only, no GPU needed.  table == NULL: only report the dimensions.
+ */
+int aquakv_search_table_host(const float* grid_host, int32_t grid_size, int32_t* cells_per_side,
+                             float* half_extent, uint32_t* table, size_t table_capacity);
+
 /* Frees the context's device tables.  NULL is accepted.  Pending work must have completed. */
 int aquakv_destroy(aquakv_ctx* ctx);
 
@@ -256,6 +269,7 @@ int64_t aquakv_launch_count(const aquakv_ctx* ctx);
 #define AQUAKV_KERNEL_ENCODE_ROWS 1 /* residual, scale, rotation, search, pack   */
 #define AQUAKV_KERNEL_DECODE_ROWS 2 /* unpack, gather, inverse rotation, add-back */
 #define AQUAKV_KERNEL_ATTN 3        /* split-KV attention partials and combine   */
+#define AQUAKV_KERNEL_LAYER 4       /* fused layer kernel: predictor GEMMs + row work */
 int aquakv_profile_enable(aquakv_ctx* ctx, int enable);
 int aquakv_profile_read(aquakv_ctx* ctx, int kernel_class, int64_t* launches, double* total_ms);
 

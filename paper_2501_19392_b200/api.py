@@ -28,7 +28,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libaquakv.so")
 
 SYMBOLS = [
-    "aquakv_code_bytes", "aquakv_create", "aquakv_destroy", "aquakv_workspace_bytes",
+    "aquakv_code_bytes", "aquakv_search_table_host", "aquakv_create", "aquakv_destroy", "aquakv_workspace_bytes",
     "aquakv_decode_attn_workspace_bytes", "aquakv_predict", "aquakv_encode", "aquakv_decode",
     "aquakv_decode_attn", "aquakv_decode_noalloc", "aquakv_encode_phase", "aquakv_decode_phase", "aquakv_poll_status", "aquakv_launch_count", "aquakv_status_string",
     "aquakv_profile_enable", "aquakv_profile_read",
@@ -55,6 +55,8 @@ def _load():
     vp, i32, i64, f32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_size_t
     L.aquakv_code_bytes.restype = ctypes.c_int
     L.aquakv_code_bytes.argtypes = [ctypes.POINTER(Params)]
+    L.aquakv_search_table_host.restype = ctypes.c_int
+    L.aquakv_search_table_host.argtypes = [vp, i32, ctypes.POINTER(i32), ctypes.POINTER(f32), vp, sz]
     L.aquakv_create.restype = ctypes.c_int
     L.aquakv_create.argtypes = [ctypes.POINTER(Params), vp, vp, vp, ctypes.POINTER(vp)]
     L.aquakv_destroy.restype = ctypes.c_int
@@ -105,6 +107,21 @@ def status_string(status: int) -> str:
 def code_bytes(d_kv: int, grid_size: int, had_block: int = 64, scale_group: int = 64, dtype: int = BF16) -> int:
     p = Params(d_kv, had_block, scale_group, 2, grid_size, dtype)
     return int(lib.aquakv_code_bytes(ctypes.byref(p)))
+
+
+def search_table(grid: np.ndarray):
+    """(cells_per_side, half_extent, table uint32 [cells, cells]) of aquakv_search_table_host."""
+    g = np.ascontiguousarray(grid, dtype=np.float32)
+    cells, half = ctypes.c_int32(0), ctypes.c_float(0.0)
+    rc = lib.aquakv_search_table_host(g.ctypes.data, g.shape[0], ctypes.byref(cells), ctypes.byref(half), None, 0)
+    if rc:
+        raise AquaKVError(rc, "aquakv_search_table_host")
+    table = np.zeros((cells.value, cells.value), dtype=np.uint32)
+    rc = lib.aquakv_search_table_host(g.ctypes.data, g.shape[0], ctypes.byref(cells), ctypes.byref(half),
+                                      table.ctypes.data, table.size)
+    if rc:
+        raise AquaKVError(rc, "aquakv_search_table_host")
+    return int(cells.value), float(half.value), table
 
 
 def _ptr(t) -> Optional[int]:

@@ -15,11 +15,14 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <vector>
 
 #include "aquakv.h"
 #include "attn.cuh"
 #include "codec.cuh"
 #include "gemm_pred.cuh"
+#include "layer_kernel.cuh"
+#include "search_table.h"
 
 using namespace aquakv;
 
@@ -39,8 +42,8 @@ struct aquakv_ctx {
   float4* d_grid4;
   uint32_t* d_signmask[2]; // [0] keys, [1] values
   int* d_status;
-  GridConst<16> gc16;
-  GridConst<64> gc64;
+  uint32_t* d_search_table;
+  SearchTableSpec search_spec;
   EncodeTiledFn encode_tiled;
   int64_t launches;
   // optional per-kernel-class timing (aquakv_profile_*): event pairs recorded around launches
@@ -152,15 +155,8 @@ int launch_predict(aquakv_ctx* c, cudaStream_t st, int M, const void* in0, const
 }
 
 template <int D, int NPTS, bool BF>
-void launch_encode_rows_t(aquakv_ctx* c, cudaStream_t st, const CodecArgs& a, int grid) {
-  if constexpr (NPTS == 16) {
-    encode_rows_kernel<D, 16, BF><<<grid, kCodecThreads, 0, st>>>(c->gc16, a);
-  } else if constexpr (NPTS == 64) {
-    encode_rows_kernel<D, 64, BF><<<grid, kCodecThreads, 0, st>>>(c->gc64, a);
-  } else {
-    GridConst<1> dummy = {};
-    encode_rows_kernel<D, 256, BF><<<grid, kCodecThreads, 0, st>>>(dummy, a);
-  }
+void launch_encode_rows_t(aquakv_ctx*, cudaStream_t st, const CodecArgs& a, int grid) {
+  encode_rows_kernel<D, NPTS, BF><<<grid, kCodecThreads, 0, st>>>(a);
 }
 
 template <int D, int NPTS, bool BF>
@@ -203,6 +199,8 @@ CodecArgs codec_args(const aquakv_ctx* c, int role, int rows) {
   std::memset(&a, 0, sizeof(a));
   a.signmask = c->d_signmask[role];
   a.grid4 = c->d_grid4;
+  a.search.table = c->d_search_table;
+  a.search.inv_w = c->search_spec.inv_w;
   a.T = rows;
   a.log_h = c->log_h;
   a.log_g = c->log_g;
@@ -364,6 +362,126 @@ AttnWs attn_ws(const aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_
   return w;
 }
 
+// ---------------------------------------------------------------------------------------------
+// fused layer kernel (predictor GEMMs + row work in one persistent launch)
+// ---------------------------------------------------------------------------------------------
+constexpr int kLayerRing = 3;       // prediction buffers
+constexpr int kKhatRing = 3;        // waves of reconstructed keys kept when the caller wants none
+
+struct LayerWs {
+  size_t p_off, khat_off, flags_off, flags_bytes, total;
+  int mw, n_waves, n_mblocks;
+};
+
+LayerWs layer_ws(const aquakv_ctx* c, int64_t T) {
+  LayerWs w;
+  const int d = c->p.d_kv, ntn = d / kBN;
+  w.n_mblocks = int((T + kBM - 1) / kBM);
+  int mw = c->sm_count / ntn;
+  if (mw < 1) mw = 1;
+  if (mw > w.n_mblocks) mw = w.n_mblocks;
+  w.mw = mw;
+  w.n_waves = (w.n_mblocks + mw - 1) / mw;
+  w.p_off = 0;
+  w.khat_off = round_up(size_t(kLayerRing) * mw * kBM * d * sizeof(float), 256);
+  w.flags_off = w.khat_off + round_up(size_t(kKhatRing) * mw * kBM * d * 2, 256);
+  w.flags_bytes = size_t(2) * 2 * w.n_waves * mw * sizeof(int);
+  w.total = w.flags_off + round_up(w.flags_bytes, 256);
+  return w;
+}
+
+template <bool ENC, int D, int NPTS, bool BF>
+int launch_layer_t(cudaStream_t st, int grid, const CUtensorMap* tm, const LayerArgs& a) {
+  static bool attr_set = false;   // per instantiation; contexts are used from one thread at a time
+  constexpr size_t smem = layer_smem_bytes<NPTS>();
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(layer_kernel<ENC, D, NPTS, BF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             int(smem)) != cudaSuccess)
+      return AQUAKV_ERR_CUDA;
+    attr_set = true;
+  }
+  layer_kernel<ENC, D, NPTS, BF><<<grid, kLayerThreads, smem, st>>>(tm[0], tm[1], tm[2], tm[3], tm[4], a);
+  return AQUAKV_OK;
+}
+template <int D, int NPTS, bool BF>
+void launch_layer_enc_t(int* rc, cudaStream_t st, int grid, const CUtensorMap* tm, const LayerArgs& a) {
+  *rc = launch_layer_t<true, D, NPTS, BF>(st, grid, tm, a);
+}
+template <int D, int NPTS, bool BF>
+void launch_layer_dec_t(int* rc, cudaStream_t st, int grid, const CUtensorMap* tm, const LayerArgs& a) {
+  *rc = launch_layer_t<false, D, NPTS, BF>(st, grid, tm, a);
+}
+
+// Algorithm 2 (encode = true) or Algorithm 3 for one layer with predictors, all tokens, one launch.
+int launch_layer(aquakv_ctx* c, cudaStream_t st, bool encode, int64_t T, const void* K, const void* V,
+                 int64_t ld_kv, const void* Khat_prev, const void* Vhat_prev, int64_t ld_prev,
+                 const void* Wk, const void* Wv, const float* bk, const float* bv, uint8_t* Kcodes,
+                 uint16_t* Kscales, uint8_t* Vcodes, uint16_t* Vscales, void* Khat, void* Vhat,
+                 int64_t ld_hat, void* workspace) {
+  const int d = c->p.d_kv;
+  const LayerWs ws = layer_ws(c, T);
+  uint8_t* wsb = static_cast<uint8_t*>(workspace);
+  LayerArgs a;
+  std::memset(&a, 0, sizeof(a));
+  a.T = int(T);
+  a.n_mblocks = ws.n_mblocks;
+  a.mw = ws.mw;
+  a.n_waves = ws.n_waves;
+  a.nb = kLayerRing;
+  a.bk = bk;
+  a.bv = bv;
+  a.P = reinterpret_cast<float*>(wsb + ws.p_off);
+  a.gemm_done = reinterpret_cast<int*>(wsb + ws.flags_off);
+  a.rows_done = a.gemm_done + size_t(2) * ws.n_waves * ws.mw;
+  a.K = static_cast<const uint16_t*>(K);
+  a.V = static_cast<const uint16_t*>(V);
+  a.ldX = ld_kv;
+  a.Kcodes = Kcodes;
+  a.Kscales = Kscales;
+  a.Vcodes = Vcodes;
+  a.Vscales = Vscales;
+  if (Khat != nullptr) {
+    a.khat_ring = 0;
+    a.Khat = static_cast<uint16_t*>(Khat);
+    a.ldKhat = ld_hat;
+  } else {
+    a.khat_ring = kKhatRing;
+    a.Khat = reinterpret_cast<uint16_t*>(wsb + ws.khat_off);
+    a.ldKhat = d;
+  }
+  a.Vhat = static_cast<uint16_t*>(Vhat);
+  a.ldVhat = ld_hat;
+  a.signmask_k = c->d_signmask[kRoleK];
+  a.signmask_v = c->d_signmask[kRoleV];
+  const CodecArgs ca = codec_args(c, kRoleK, 0);
+  a.grid4 = ca.grid4;
+  a.search = ca.search;
+  a.log_h = c->log_h;
+  a.log_g = c->log_g;
+  a.status = c->d_status;
+
+  CUtensorMap tm[5];
+  int rc = make_tmap(c, &tm[0], Khat_prev, uint64_t(T), uint64_t(d), uint64_t(ld_prev), kBM);
+  if (rc) return rc;
+  if ((rc = make_tmap(c, &tm[1], Vhat_prev, uint64_t(T), uint64_t(d), uint64_t(ld_prev), kBM))) return rc;
+  const uint64_t khat_rows = a.khat_ring ? uint64_t(kKhatRing) * ws.mw * kBM : uint64_t(T);
+  if ((rc = make_tmap(c, &tm[2], a.Khat, khat_rows, uint64_t(d), uint64_t(a.ldKhat), kBM))) return rc;
+  if ((rc = make_tmap(c, &tm[3], Wk, uint64_t(d), uint64_t(d), uint64_t(d), kBN))) return rc;
+  if ((rc = make_tmap(c, &tm[4], Wv, uint64_t(d), uint64_t(2) * d, uint64_t(2) * d, kBN))) return rc;
+
+  if (cudaMemsetAsync(a.gemm_done, 0, ws.flags_bytes, st) != cudaSuccess) return AQUAKV_ERR_CUDA;
+  const int grid = ws.mw * (d / kBN);
+  ProfScope prof(c, st, AQUAKV_KERNEL_LAYER);
+  if (encode) {
+    AQ_DISPATCH_DNB(launch_layer_enc_t, &rc, st, grid, tm, a);
+  } else {
+    AQ_DISPATCH_DNB(launch_layer_dec_t, &rc, st, grid, tm, a);
+  }
+  if (rc) return rc;
+  ++c->launches;
+  return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
+}
+
 }  // namespace
 
 // =============================================================================================
@@ -389,6 +507,22 @@ const char* aquakv_status_string(int status) {
     case AQUAKV_ERR_TOO_LARGE: return "more tokens than the fixed scratch of the no-allocation call holds";
     default: return "unknown status";
   }
+}
+
+int aquakv_search_table_host(const float* grid_host, int32_t grid_size, int32_t* cells_per_side,
+                             float* half_extent, uint32_t* table, size_t table_capacity) {
+  if (grid_host == nullptr || cells_per_side == nullptr || half_extent == nullptr)
+    return AQUAKV_ERR_INVALID_ARG;
+  if (grid_size != 16 && grid_size != 64 && grid_size != 256) return AQUAKV_ERR_UNSUPPORTED;
+  for (int i = 0; i < 2 * grid_size; ++i)
+    if (!std::isfinite(grid_host[i])) return AQUAKV_ERR_INVALID_ARG;
+  const SearchTableSpec spec = search_table_spec(grid_host, grid_size);
+  *cells_per_side = spec.cells;
+  *half_extent = spec.half;
+  if (table == nullptr) return AQUAKV_OK;
+  if (table_capacity < size_t(spec.cells) * spec.cells) return AQUAKV_ERR_INVALID_ARG;
+  build_search_table(grid_host, grid_size, spec, table);
+  return AQUAKV_OK;
 }
 
 int aquakv_create(const aquakv_params* params, const float* grid_host, const int8_t* signs_k_host,
@@ -421,11 +555,11 @@ int aquakv_create(const aquakv_params* params, const float* grid_host, const int
   float4 g4[256];
   for (int i = 0; i < n; ++i) {
     const float gx = grid_host[2 * i], gy = grid_host[2 * i + 1];
-    const float hn = 0.5f * (gx * gx + gy * gy);
-    g4[i] = make_float4(gx, gy, hn, 0.0f);
-    if (n == 16) { c->gc16.nx[i] = -gx; c->gc16.ny[i] = -gy; c->gc16.hn[i] = hn; }
-    if (n == 64) { c->gc64.nx[i] = -gx; c->gc64.ny[i] = -gy; c->gc64.hn[i] = hn; }
+    g4[i] = make_float4(gx, gy, 0.0f, 0.0f);
   }
+  c->search_spec = search_table_spec(grid_host, n);
+  std::vector<uint32_t> table(size_t(c->search_spec.cells) * c->search_spec.cells);
+  build_search_table(grid_host, n, c->search_spec, table.data());
   uint32_t masks[2][32];
   std::memset(masks, 0, sizeof(masks));
   for (int role = 0; role < 2; ++role) {
@@ -447,6 +581,9 @@ int aquakv_create(const aquakv_params* params, const float* grid_host, const int
   ok = ok && cudaMalloc(&c->d_signmask[0], sizeof(uint32_t) * 32) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_signmask[1], sizeof(uint32_t) * 32) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_status, sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_search_table, table.size() * sizeof(uint32_t)) == cudaSuccess;
+  ok = ok && cudaMemcpy(c->d_search_table, table.data(), table.size() * sizeof(uint32_t),
+                        cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(c->d_grid4, g4, sizeof(float4) * n, cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(c->d_signmask[0], masks[0], sizeof(masks[0]), cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(c->d_signmask[1], masks[1], sizeof(masks[1]), cudaMemcpyHostToDevice) == cudaSuccess;
@@ -475,6 +612,7 @@ int aquakv_destroy(aquakv_ctx* c) {
   if (c->d_signmask[0]) ok = cudaFree(c->d_signmask[0]) == cudaSuccess && ok;
   if (c->d_signmask[1]) ok = cudaFree(c->d_signmask[1]) == cudaSuccess && ok;
   if (c->d_status) ok = cudaFree(c->d_status) == cudaSuccess && ok;
+  if (c->d_search_table) ok = cudaFree(c->d_search_table) == cudaSuccess && ok;
   if (c->prof_ev) {
     for (int i = 0; i < 2 * kProfMaxPairs; ++i)
       if (c->prof_ev[i]) cudaEventDestroy(c->prof_ev[i]);
@@ -487,7 +625,10 @@ int aquakv_destroy(aquakv_ctx* c) {
 
 size_t aquakv_workspace_bytes(const aquakv_ctx* c, int64_t n_tokens, int op) {
   if (c == nullptr || n_tokens <= 0) return 0;
-  if (op == AQUAKV_OP_ENCODE || op == AQUAKV_OP_DECODE) return encode_ws(c, n_tokens).total;
+  if (op == AQUAKV_OP_ENCODE || op == AQUAKV_OP_DECODE) {
+    const size_t phase_bytes = encode_ws(c, n_tokens).total, layer_bytes = layer_ws(c, n_tokens).total;
+    return phase_bytes > layer_bytes ? phase_bytes : layer_bytes;
+  }
   return 0;
 }
 
@@ -672,9 +813,14 @@ int aquakv_encode(aquakv_ctx* c, int64_t n_tokens, const void* K, const void* V,
       (Vhat != nullptr && (Vhat == Vhat_prev || Vhat == V || Vhat == Khat_prev || Vhat == Khat)))
     return AQUAKV_ERR_INVALID_ARG;
   const EncodeWs ws = encode_ws(c, n_tokens);
-  if (has_pred || Khat == nullptr) {
-    if (workspace == nullptr || workspace_bytes < ws.total) return AQUAKV_ERR_WORKSPACE;
+  if (has_pred) {
+    if (workspace == nullptr || workspace_bytes < aquakv_workspace_bytes(c, n_tokens, AQUAKV_OP_ENCODE))
+      return AQUAKV_ERR_WORKSPACE;
     if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
+    if (n_tokens > (int64_t(1) << 30)) return AQUAKV_ERR_UNSUPPORTED;
+    return launch_layer(c, static_cast<cudaStream_t>(cuda_stream), true, n_tokens, K, V, ld_kv, Khat_prev,
+                        Vhat_prev, ld_prev, Wk, Wv, bk, bv, Kcodes, Kscales, Vcodes, Vscales, Khat, Vhat,
+                        ld_hat, workspace);
   }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   uint8_t* wsb = static_cast<uint8_t*>(workspace);
@@ -731,8 +877,14 @@ int aquakv_decode(aquakv_ctx* c, int64_t n_tokens, const uint8_t* Kcodes, const 
     return AQUAKV_ERR_INVALID_ARG;
   const EncodeWs ws = encode_ws(c, n_tokens);
   if (has_pred) {
-    if (workspace == nullptr || workspace_bytes < ws.total) return AQUAKV_ERR_WORKSPACE;
+    if (workspace == nullptr || workspace_bytes < aquakv_workspace_bytes(c, n_tokens, AQUAKV_OP_DECODE))
+      return AQUAKV_ERR_WORKSPACE;
     if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
+    if (n_tokens > (int64_t(1) << 30)) return AQUAKV_ERR_UNSUPPORTED;
+    return launch_layer(c, static_cast<cudaStream_t>(cuda_stream), false, n_tokens, nullptr, nullptr, 0,
+                        Khat_prev, Vhat_prev, ld_prev, Wk, Wv, bk, bv, const_cast<uint8_t*>(Kcodes),
+                        const_cast<uint16_t*>(Kscales), const_cast<uint8_t*>(Vcodes),
+                        const_cast<uint16_t*>(Vscales), Khat, Vhat, ld_hat, workspace);
   }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   float* P = has_pred ? reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + ws.p_off) : nullptr;

@@ -17,15 +17,38 @@ namespace aquakv {
 constexpr int kCodecWarps = 8;
 constexpr int kCodecThreads = kCodecWarps * 32;
 
-// Grid in kernel-parameter (constant) space for the unrolled nearest-point search:
-// score_i(y) = hn[i] + nx[i]*y0 + ny[i]*y1 with nx = -g_x, ny = -g_y, hn = |g|^2 / 2, whose
-// argmin over i is the nearest grid point.
-template <int N>
-struct GridConst {
-  float nx[N];
-  float ny[N];
-  float hn[N];
+// Nearest-point search.  dist_i(y) = (y0 - g_i.x)^2 + (y1 - g_i.y)^2; the lowest index wins ties.
+// A cell table built on the host (search_table.h) lists, for the cell that holds y, every point
+// that can win there, so only three (n = 16) or four distances are evaluated; cells with more candidates and
+// values outside the table's square fall back to the exhaustive loop.  Both paths evaluate the same
+// fp32 expression, so the result is the exhaustive arg-min bit for bit.  The table (64 x 64
+// entries) and the grid live in shared memory: the row kernels are bound by the load/store and
+// shuffle pipe, and shared-memory gathers of 4 and 8 bytes cost far fewer cycles there than
+// global gathers or 16-byte records.
+constexpr int kSearchCells = 64;          // cells per side of the table (see search_table.h)
+constexpr int kSearchLogCells = 6;
+constexpr uint32_t kCellBruteDev = 1u;    // the one non-ascending entry: search all points
+
+struct SearchDev {
+  const uint32_t* table;   // global copy [64*64] of the candidate lists
+  float inv_w;             // cells / (2 * half extent)
 };
+
+// Shared-memory tables of the row routines.
+template <int NPTS>
+struct RowSmem {
+  uint32_t table[kSearchCells * kSearchCells];
+  float2 grid[NPTS];
+};
+
+template <int NPTS>
+__device__ __forceinline__ void row_smem_fill(RowSmem<NPTS>* rs, const uint32_t* table, const float4* grid4) {
+  for (int i = threadIdx.x; i < kSearchCells * kSearchCells; i += blockDim.x) rs->table[i] = table[i];
+  for (int i = threadIdx.x; i < NPTS; i += blockDim.x) {
+    const float4 g = grid4[i];
+    rs->grid[i] = make_float2(g.x, g.y);
+  }
+}
 
 struct CodecArgs {
   const uint16_t* X;        // encode: target rows (16-bit)              [T, ldX]
@@ -34,7 +57,8 @@ struct CodecArgs {
   long long ldP;
   const uint32_t* signmask; // [32]: bit (c*8+i) of entry `lane` set <=> sign of element
                             //       c*256 + lane*8 + i is -1
-  const float4* grid4;      // [n]: (g_x, g_y, |g|^2/2, 0)
+  const float4* grid4;      // [n]: (g_x, g_y, 0, 0)
+  SearchDev search;
   uint8_t* codes;           // [T, code_bytes]
   uint16_t* scales;         // [T, D/G] fp16 bits
   uint16_t* hat;            // reconstruction rows (16-bit) or nullptr    [T, ldHat]
@@ -167,122 +191,278 @@ __device__ __forceinline__ void group_sums(const float (&v)[NC * 8], float (&ss)
   }
 }
 
+// Cell-table entry of one value pair (marked exhaustive outside the square).
+__device__ __forceinline__ uint32_t search_entry(float y0, float y1, float inv_w,
+                                                 const uint32_t* __restrict__ table_s) {
+  const int ix = __float2int_rd(fmaf(y0, inv_w, 0.5f * kSearchCells));
+  const int iy = __float2int_rd(fmaf(y1, inv_w, 0.5f * kSearchCells));
+  const bool inside = static_cast<unsigned>(ix | iy) < unsigned(kSearchCells);
+  const uint32_t e = table_s[inside ? ((iy << kSearchLogCells) + ix) : 0];
+  return inside ? e : kCellBruteDev;
+}
+
+__device__ __forceinline__ float pair_dist(float y0, float y1, float2 g) {
+  const float dx = __fsub_rn(y0, g.x), dy = __fsub_rn(y1, g.y);
+  return fmaf(dy, dy, __fmul_rn(dx, dx));
+}
+
+// Arg-min over the ascending candidates of a table entry (three for n = 16, else four).
+template <int NPTS>
+__device__ __forceinline__ int nearest_of_candidates(float y0, float y1, uint32_t e,
+                                                     const float2* __restrict__ grid_s) {
+  const int c0 = e & 0xffu, c1 = (e >> 8) & 0xffu, c2 = (e >> 16) & 0xffu;
+  const float t0 = pair_dist(y0, y1, grid_s[c0]);
+  const float t1 = pair_dist(y0, y1, grid_s[c1]);
+  const float t2 = pair_dist(y0, y1, grid_s[c2]);
+  int idx = c0;
+  float best = t0;
+  if (t1 < best) { best = t1; idx = c1; }
+  if (t2 < best) { best = t2; idx = c2; }
+  if constexpr (NPTS > 16) {
+    const int c3 = e >> 24;
+    const float t3 = pair_dist(y0, y1, grid_s[c3]);
+    if (t3 < best) { idx = c3; }
+  }
+  return idx;
+}
+
+template <int NPTS>
+__device__ __noinline__ int nearest_exhaustive(float y0, float y1, const float2* __restrict__ grid_s) {
+  float best = 3.0e38f;
+  int idx = 0;
+  for (int i = 0; i < NPTS; ++i) {
+    const float t = pair_dist(y0, y1, grid_s[i]);
+    if (t < best) { best = t; idx = i; }             // strict: lowest index wins ties
+  }
+  return idx;
+}
+
+// Per-warp constants of the row routines.
+struct RowCtx {
+  uint32_t signmask;       // this lane's entry of CodecArgs::signmask
+  float inv_w;             // SearchDev::inv_w
+  int log_h, log_g;
+  int lane;
+};
+
+// One token row of Q and of the reconstruction (Algorithm 2 lines 6-7 / 9):
+//   codes, scales = Q(x - pred);  hat = round16(pred + Q^-1(codes, scales)).
+// pred_row == nullptr: no predictor.  hat_row == nullptr: reconstruction not wanted.  The prediction
+// is read twice (for the residual and again for the reconstruction) instead of being held in 32
+// registers across the rotation and the search; both reads bypass L1 (ld.global.cg) because the
+// prediction may have been written by another SM of the same kernel just before.
 template <int D, int NPTS, bool kBf16>
-__global__ void __launch_bounds__(kCodecThreads)
-encode_rows_kernel(const __grid_constant__ GridConst<(NPTS <= 64 ? NPTS : 1)> gc, const CodecArgs a) {
+__device__ __forceinline__ void encode_row(const RowCtx& rc, const RowSmem<NPTS>* __restrict__ rsm,
+                                           const uint16_t* __restrict__ x_row,
+                                           const float* __restrict__ pred_row,
+                                           uint8_t* __restrict__ codes_row,
+                                           uint16_t* __restrict__ scales_row,
+                                           uint16_t* __restrict__ hat_row) {
   constexpr int NC = D / 256, NV = NC * 8;
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
-  constexpr int CODE_BYTES = D / 2 * BITS / 8;
-  __shared__ float4 grid_s[NPTS];
-  for (int i = threadIdx.x; i < NPTS; i += blockDim.x) grid_s[i] = a.grid4[i];
-  __syncthreads();
-
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t signmask = a.signmask[lane];
-  const int n_groups = D >> a.log_g;
-  const float inv_g = exp2f(-static_cast<float>(a.log_g));
-  const float rs = exp2f(-0.5f * static_cast<float>(a.log_h));
-
-  for (long long row = (long long)blockIdx.x * kCodecWarps + warp; row < a.T;
-       row += (long long)gridDim.x * kCodecWarps) {
-    float v[NV], p[NV];
-    // ---- residual r = x - pred (Algorithm 2 line 6 / 9) -------------------------------------
+  const int lane = rc.lane;
+  const float inv_g = exp2f(-static_cast<float>(rc.log_g));
+  const float rs = exp2f(-0.5f * static_cast<float>(rc.log_h));
+  float v[NV];
+  // ---- residual r = x - pred -------------------------------------------------------------------
+  {
+    uint4 raw[NC];
 #pragma unroll
-    for (int c = 0; c < NC; ++c) {
-      const int e0 = c * 256 + lane * 8;
-      const uint4 raw = *reinterpret_cast<const uint4*>(a.X + row * a.ldX + e0);
-      const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-      if (a.P != nullptr) {
-        const float4 p0 = *reinterpret_cast<const float4*>(a.P + row * a.ldP + e0);
-        const float4 p1 = *reinterpret_cast<const float4*>(a.P + row * a.ldP + e0 + 4);
-        p[c * 8 + 0] = p0.x; p[c * 8 + 1] = p0.y; p[c * 8 + 2] = p0.z; p[c * 8 + 3] = p0.w;
-        p[c * 8 + 4] = p1.x; p[c * 8 + 5] = p1.y; p[c * 8 + 6] = p1.z; p[c * 8 + 7] = p1.w;
-      } else {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) p[c * 8 + i] = 0.0f;
-      }
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        v[c * 8 + 2 * i] = __fsub_rn(load16<kBf16>(uint16_t(w[i] & 0xffffu)), p[c * 8 + 2 * i]);
-        v[c * 8 + 2 * i + 1] = __fsub_rn(load16<kBf16>(uint16_t(w[i] >> 16)), p[c * 8 + 2 * i + 1]);
-      }
-    }
-    // ---- group scale: root mean square, stored as fp16; normalise with the rounded value ----
-    float ss[NC], sf[NC];
-    group_sums<NC>(v, ss, a.log_g);
-#pragma unroll
-    for (int c = 0; c < NC; ++c) {
-      const float s = fminf(sqrtf(ss[c] * inv_g), 65504.0f);
-      const __half s16 = __float2half_rn(s);
-      sf[c] = __half2float(s16);
-      // one lane per group writes the scale
-      if (a.log_g >= 8) {
-        const int cpg = 1 << (a.log_g - 8);
-        if (lane == 0 && (c % cpg) == 0) a.scales[row * n_groups + c / cpg] = __half_as_ushort(s16);
-      } else {
-        const int lpg = 1 << (a.log_g - 3);   // lanes per group
-        if ((lane % lpg) == 0)
-          a.scales[row * n_groups + c * (256 >> a.log_g) + lane / lpg] = __half_as_ushort(s16);
-      }
-      const float inv = sf[c] > 0.0f ? 1.0f / sf[c] : 0.0f;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) v[c * 8 + i] = apply_sign(v[c * 8 + i] * inv, signmask, c * 8 + i);
-    }
-    // ---- rotate -------------------------------------------------------------------------------
-    fwht_regs_and_lanes<NV>(v, a.log_h, lane);
-    // ---- nearest grid point per pair, pack, gather the chosen points --------------------------
-#pragma unroll
-    for (int c = 0; c < NC; ++c) {
-      uint32_t word = 0;
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const float y0 = v[c * 8 + 2 * k] * rs, y1 = v[c * 8 + 2 * k + 1] * rs;
-        int idx = 0;
-        if constexpr (NPTS <= 64) {
-          float best = fmaf(gc.ny[0], y1, fmaf(gc.nx[0], y0, gc.hn[0]));
-#pragma unroll
-          for (int i = 1; i < NPTS; ++i) {
-            const float t = fmaf(gc.ny[i], y1, fmaf(gc.nx[i], y0, gc.hn[i]));
-            if (t < best) { best = t; idx = i; }     // strict: lowest index wins ties
-          }
-        } else {
-          float best = 3.0e38f;
-          for (int i = 0; i < NPTS; ++i) {
-            const float4 g = grid_s[i];
-            const float t = fmaf(-g.y, y1, fmaf(-g.x, y0, g.z));
-            if (t < best) { best = t; idx = i; }
-          }
-        }
-        word |= uint32_t(idx) << (k * BITS);
-        const float4 g = grid_s[idx];
-        v[c * 8 + 2 * k] = g.x;
-        v[c * 8 + 2 * k + 1] = g.y;
-      }
-      store_code_word<BITS>(a.codes + row * CODE_BYTES, c, lane, word);
-    }
-    // ---- reconstruction (Algorithm 2 line 7): hat = round16(pred + Q^-1(codes)) ---------------
-    if (a.hat != nullptr) {
-      rotate_back_and_scale<NV>(v, sf, signmask, a.log_h, lane);
+    for (int c = 0; c < NC; ++c)
+      raw[c] = *reinterpret_cast<const uint4*>(x_row + c * 256 + lane * 8);
+    if (pred_row != nullptr) {
+      float4 pq[NC][2];
 #pragma unroll
       for (int c = 0; c < NC; ++c) {
-        uint32_t o[4];
+        pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + c * 256 + lane * 8));
+        pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + c * 256 + lane * 8 + 4));
+      }
+#pragma unroll
+      for (int c = 0; c < NC; ++c) {
+        const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
+        const float pp[8] = {pq[c][0].x, pq[c][0].y, pq[c][0].z, pq[c][0].w,
+                             pq[c][1].x, pq[c][1].y, pq[c][1].z, pq[c][1].w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const uint32_t lo = store16<kBf16>(__fadd_rn(p[c * 8 + 2 * i], v[c * 8 + 2 * i]));
-          const uint32_t hi = store16<kBf16>(__fadd_rn(p[c * 8 + 2 * i + 1], v[c * 8 + 2 * i + 1]));
-          o[i] = lo | (hi << 16);
+          v[c * 8 + 2 * i] = __fsub_rn(load16<kBf16>(uint16_t(w[i] & 0xffffu)), pp[2 * i]);
+          v[c * 8 + 2 * i + 1] = __fsub_rn(load16<kBf16>(uint16_t(w[i] >> 16)), pp[2 * i + 1]);
         }
-        *reinterpret_cast<uint4*>(a.hat + row * a.ldHat + c * 256 + lane * 8) =
-            make_uint4(o[0], o[1], o[2], o[3]);
       }
+    } else {
+#pragma unroll
+      for (int c = 0; c < NC; ++c) {
+        const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          v[c * 8 + 2 * i] = load16<kBf16>(uint16_t(w[i] & 0xffffu));
+          v[c * 8 + 2 * i + 1] = load16<kBf16>(uint16_t(w[i] >> 16));
+        }
+      }
+    }
+  }
+  // ---- group scale: root mean square, stored as fp16; normalise with the rounded value --------
+  float ss[NC], sf[NC], inv[NC];
+  group_sums<NC>(v, ss, rc.log_g);
+#pragma unroll
+  for (int c = 0; c < NC; ++c) {
+    const float s = fminf(sqrtf(ss[c] * inv_g), 65504.0f);
+    const __half s16 = __float2half_rn(s);
+    sf[c] = __half2float(s16);
+    if (rc.log_g >= 8) {                 // one lane per group writes the scale
+      const int cpg = 1 << (rc.log_g - 8);
+      if (lane == 0 && (c % cpg) == 0) scales_row[c / cpg] = __half_as_ushort(s16);
+    } else {
+      const int lpg = 1 << (rc.log_g - 3);   // lanes per group
+      if ((lane % lpg) == 0) scales_row[c * (256 >> rc.log_g) + lane / lpg] = __half_as_ushort(s16);
+    }
+    // the rotation is linear: the division by the scale is applied after it, merged with 1/sqrt(h)
+    inv[c] = (sf[c] > 0.0f ? 1.0f / sf[c] : 0.0f) * rs;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[c * 8 + i] = apply_sign(v[c * 8 + i], rc.signmask, c * 8 + i);
+  }
+  // ---- rotate ------------------------------------------------------------------------------------
+  fwht_regs_and_lanes<NV>(v, rc.log_h, lane);
+#pragma unroll
+  for (int c = 0; c < NC; ++c)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[c * 8 + i] *= inv[c];
+  // ---- nearest grid point per pair: all table entries first, then the candidates ----------------
+  uint32_t entry[NV / 2];
+  uint32_t any_brute = 0;
+#pragma unroll
+  for (int j = 0; j < NV / 2; ++j) {
+    entry[j] = search_entry(v[2 * j], v[2 * j + 1], rc.inv_w, rsm->table);
+    any_brute |= uint32_t(entry[j] == kCellBruteDev);
+  }
+  const bool slow = __any_sync(0xffffffffu, any_brute != 0);
+#pragma unroll
+  for (int c = 0; c < NC; ++c) {
+    uint32_t word = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int j = c * 4 + k;
+      int idx;
+      if (!slow) {
+        idx = nearest_of_candidates<NPTS>(v[2 * j], v[2 * j + 1], entry[j], rsm->grid);
+      } else {
+        idx = entry[j] == kCellBruteDev
+                  ? nearest_exhaustive<NPTS>(v[2 * j], v[2 * j + 1], rsm->grid)
+                  : nearest_of_candidates<NPTS>(v[2 * j], v[2 * j + 1], entry[j], rsm->grid);
+      }
+      word |= uint32_t(idx) << (k * BITS);
+      const float2 g = rsm->grid[idx];
+      v[2 * j] = g.x;
+      v[2 * j + 1] = g.y;
+    }
+    store_code_word<BITS>(codes_row, c, lane, word);
+  }
+  // ---- reconstruction: hat = round16(pred + Q^-1(codes)) ---------------------------------------
+  if (hat_row != nullptr) {
+    float4 pq[NC][2];
+    if (pred_row != nullptr) {
+#pragma unroll
+      for (int c = 0; c < NC; ++c) {
+        pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + c * 256 + lane * 8));
+        pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + c * 256 + lane * 8 + 4));
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < NC; ++c) pq[c][0] = pq[c][1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    }
+    rotate_back_and_scale<NV>(v, sf, rc.signmask, rc.log_h, lane);
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+      const float pp[8] = {pq[c][0].x, pq[c][0].y, pq[c][0].z, pq[c][0].w,
+                           pq[c][1].x, pq[c][1].y, pq[c][1].z, pq[c][1].w};
+      uint32_t o[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t lo = store16<kBf16>(__fadd_rn(pp[2 * i], v[c * 8 + 2 * i]));
+        const uint32_t hi = store16<kBf16>(__fadd_rn(pp[2 * i + 1], v[c * 8 + 2 * i + 1]));
+        o[i] = lo | (hi << 16);
+      }
+      *reinterpret_cast<uint4*>(hat_row + c * 256 + lane * 8) = make_uint4(o[0], o[1], o[2], o[3]);
     }
   }
 }
 
-// Algorithm 3 line 5 / 7 given the prediction: hat = round16(pred + Q^-1(codes, scales)).
+template <int D, int NPTS, bool kBf16>
+__global__ void __launch_bounds__(kCodecThreads, 2) encode_rows_kernel(const CodecArgs a) {
+  constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
+  constexpr int CODE_BYTES = D / 2 * BITS / 8;
+  __shared__ RowSmem<NPTS> rsm;
+  row_smem_fill<NPTS>(&rsm, a.search.table, a.grid4);
+  __syncthreads();
+  RowCtx rc;
+  rc.lane = threadIdx.x & 31;
+  rc.signmask = a.signmask[rc.lane];
+  rc.inv_w = a.search.inv_w;
+  rc.log_h = a.log_h;
+  rc.log_g = a.log_g;
+  const int warp = threadIdx.x >> 5;
+  const int n_groups = D >> a.log_g;
+  for (long long row = (long long)blockIdx.x * kCodecWarps + warp; row < a.T;
+       row += (long long)gridDim.x * kCodecWarps) {
+    encode_row<D, NPTS, kBf16>(rc, &rsm, a.X + row * a.ldX,
+                               a.P != nullptr ? a.P + row * a.ldP : nullptr,
+                               a.codes + row * CODE_BYTES, a.scales + row * n_groups,
+                               a.hat != nullptr ? a.hat + row * a.ldHat : nullptr);
+  }
+}
+
+// One token row of Algorithm 3 line 5 / 7 given the prediction:
+//   hat = round16(pred + Q^-1(codes, scales)).  pred_row == nullptr: no predictor.
+template <int D, int NPTS, bool kBf16, typename GridT>
+__device__ __forceinline__ void decode_row(const RowCtx& rc, const GridT* __restrict__ grid_s,
+                                           const uint8_t* __restrict__ codes_row,
+                                           const uint16_t* __restrict__ scales_row,
+                                           const float* __restrict__ pred_row,
+                                           uint16_t* __restrict__ hat_row) {
+  constexpr int NC = D / 256, NV = NC * 8;
+  constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
+  const int lane = rc.lane;
+  float w[NV], sf[NC];
+  float4 pq[NC][2];
+  if (pred_row != nullptr) {
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+      pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + c * 256 + lane * 8));
+      pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + c * 256 + lane * 8 + 4));
+    }
+  } else {
+#pragma unroll
+    for (int c = 0; c < NC; ++c) pq[c][0] = pq[c][1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+  }
+#pragma unroll
+  for (int c = 0; c < NC; ++c) {
+    const uint32_t word = load_code_word<BITS>(codes_row, c, lane);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const GridT g = grid_s[(word >> (k * BITS)) & (NPTS - 1)];
+      w[c * 8 + 2 * k] = g.x;
+      w[c * 8 + 2 * k + 1] = g.y;
+    }
+    const int e0 = c * 256 + lane * 8;
+    sf[c] = __half2float(__ushort_as_half(scales_row[e0 >> rc.log_g]));
+  }
+  rotate_back_and_scale<NV>(w, sf, rc.signmask, rc.log_h, lane);
+#pragma unroll
+  for (int c = 0; c < NC; ++c) {
+    const float pp[8] = {pq[c][0].x, pq[c][0].y, pq[c][0].z, pq[c][0].w,
+                         pq[c][1].x, pq[c][1].y, pq[c][1].z, pq[c][1].w};
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t lo = store16<kBf16>(__fadd_rn(pp[2 * i], w[c * 8 + 2 * i]));
+      const uint32_t hi = store16<kBf16>(__fadd_rn(pp[2 * i + 1], w[c * 8 + 2 * i + 1]));
+      o[i] = lo | (hi << 16);
+    }
+    *reinterpret_cast<uint4*>(hat_row + c * 256 + lane * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
 template <int D, int NPTS, bool kBf16>
 __global__ void __launch_bounds__(kCodecThreads) decode_rows_kernel(const CodecArgs a) {
-  constexpr int NC = D / 256, NV = NC * 8;
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
   constexpr int CODE_BYTES = D / 2 * BITS / 8;
   __shared__ float2 grid_s[NPTS];
@@ -291,49 +471,18 @@ __global__ void __launch_bounds__(kCodecThreads) decode_rows_kernel(const CodecA
     grid_s[i] = make_float2(g.x, g.y);
   }
   __syncthreads();
-
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t signmask = a.signmask[lane];
+  RowCtx rc;
+  rc.lane = threadIdx.x & 31;
+  rc.signmask = a.signmask[rc.lane];
+  rc.inv_w = a.search.inv_w;
+  rc.log_h = a.log_h;
+  rc.log_g = a.log_g;
+  const int warp = threadIdx.x >> 5;
   const int n_groups = D >> a.log_g;
-
   for (long long row = (long long)blockIdx.x * kCodecWarps + warp; row < a.T;
        row += (long long)gridDim.x * kCodecWarps) {
-    float w[NV], sf[NC];
-#pragma unroll
-    for (int c = 0; c < NC; ++c) {
-      const uint32_t word = load_code_word<BITS>(a.codes + row * CODE_BYTES, c, lane);
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const float2 g = grid_s[(word >> (k * BITS)) & (NPTS - 1)];
-        w[c * 8 + 2 * k] = g.x;
-        w[c * 8 + 2 * k + 1] = g.y;
-      }
-      const int e0 = c * 256 + lane * 8;
-      sf[c] = __half2float(__ushort_as_half(a.scales[row * n_groups + (e0 >> a.log_g)]));
-    }
-    rotate_back_and_scale<NV>(w, sf, signmask, a.log_h, lane);
-#pragma unroll
-    for (int c = 0; c < NC; ++c) {
-      const int e0 = c * 256 + lane * 8;
-      float p[8];
-      if (a.P != nullptr) {
-        const float4 p0 = *reinterpret_cast<const float4*>(a.P + row * a.ldP + e0);
-        const float4 p1 = *reinterpret_cast<const float4*>(a.P + row * a.ldP + e0 + 4);
-        p[0] = p0.x; p[1] = p0.y; p[2] = p0.z; p[3] = p0.w;
-        p[4] = p1.x; p[5] = p1.y; p[6] = p1.z; p[7] = p1.w;
-      } else {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) p[i] = 0.0f;
-      }
-      uint32_t o[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint32_t lo = store16<kBf16>(__fadd_rn(p[2 * i], w[c * 8 + 2 * i]));
-        const uint32_t hi = store16<kBf16>(__fadd_rn(p[2 * i + 1], w[c * 8 + 2 * i + 1]));
-        o[i] = lo | (hi << 16);
-      }
-      *reinterpret_cast<uint4*>(a.hat + row * a.ldHat + e0) = make_uint4(o[0], o[1], o[2], o[3]);
-    }
+    decode_row<D, NPTS, kBf16>(rc, grid_s, a.codes + row * CODE_BYTES, a.scales + row * n_groups,
+                               a.P != nullptr ? a.P + row * a.ldP : nullptr, a.hat + row * a.ldHat);
   }
 }
 

@@ -1,0 +1,386 @@
+// One persistent kernel per layer call for Algorithm 2 (encode) and Algorithm 3 (decode) with
+// predictors: the predictor GEMMs (Algorithm 2 lines 5 and 8 / Algorithm 3 lines 5 and 7) run on
+// the tensor cores while, on the same SMs, other warps run the row work of the quantizer
+// (Section 2 "Vector Quantization") and of the reconstruction on tokens whose prediction is
+// already complete.  The fp32 prediction is handed from the GEMM warps to the row warps through a
+// small ring of buffers that stays resident in L2; completion is tracked with counters in global
+// memory.
+//
+// Work layout.  A token block is 128 tokens; a GEMM tile is one token block x 256 output features,
+// so NTN = d_kv/256 CTAs share a token block.  CTA c owns token-block slot ml = c / NTN and feature
+// tile n = c % NTN in every "wave" of gridDim.x / NTN token blocks.  For each wave a CTA computes
+// its key-phase tile and its value-phase tile, and runs the row work of 128/NTN rows of its token
+// block for both phases.  Jobs are ordered  K0, K1, V0, K2, V1, ..., so that the value-phase GEMM of
+// a wave (which reads the reconstructed keys of that wave) is issued one job after its key rows.
+//
+// Dependencies (all counted per job j and token-block slot ml, targets NTN):
+//   gemm_done[j][ml]  -- feature tiles of job j written to the ring        (row warps wait)
+//   rows_done[j][ml]  -- row slices of job j finished                       (the value-phase TMA
+//                        producer waits for the key rows of its wave; the GEMM epilogue waits for
+//                        job j - ring size before it overwrites that ring slot)
+// Every job waits only on jobs with a smaller index (or the same index of the other role), so the
+// schedule cannot dead-lock as long as all CTAs are resident, which the launch guarantees by using at
+// most one CTA per SM.  Every wait is bounded; on expiry the CTA records AQUAKV_ERR_TIMEOUT and
+// all its roles leave their loops.
+//
+// Warp roles: warp 0 = TMA producer, warp 1 = tensor-memory owner + MMA issuer, warps 2..5 =
+// GEMM epilogue (tensor memory -> fp32 rows in the ring), warps 6.. = row warps.
+#pragma once
+
+#include "codec.cuh"
+#include "common.cuh"
+#include "gemm_pred.cuh"
+
+namespace aquakv {
+
+constexpr int kRowWarps = 8;
+constexpr int kLayerThreads = 32 * (6 + kRowWarps);
+constexpr int kLayerStages = 4;
+
+struct LayerSmemTail {
+  uint64_t full[kLayerStages];
+  uint64_t empty[kLayerStages];
+  uint64_t acc_full[kAccStages];
+  uint64_t acc_empty[kAccStages];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+template <int NPTS>
+constexpr size_t layer_smem_bytes() {
+  return 1024 + size_t(kLayerStages) * kStageBytes + sizeof(LayerSmemTail) + 16 + sizeof(RowSmem<NPTS>);
+}
+
+struct LayerArgs {
+  int T;                  // tokens
+  int n_mblocks;          // ceil(T / 128)
+  int mw;                 // token blocks per wave (gridDim.x / NTN)
+  int n_waves;
+  int nb;                 // prediction buffers in the ring
+  const float* bk;        // optional biases [d_kv]
+  const float* bv;
+  float* P;               // ring: [nb][mw * 128][d_kv] fp32
+  int* gemm_done;         // [2 * n_waves][mw], zero at launch
+  int* rows_done;         // [2 * n_waves][mw], zero at launch
+  int khat_ring;          // 0: K^ rows are indexed by token; r > 0: ring of r waves (rows of mw*128)
+  // encode inputs
+  const uint16_t* K;
+  const uint16_t* V;
+  long long ldX;
+  // compressed cache (written by encode, read by decode)
+  uint8_t* Kcodes;
+  uint16_t* Kscales;
+  uint8_t* Vcodes;
+  uint16_t* Vscales;
+  // reconstructions
+  uint16_t* Khat;         // output rows (khat_ring == 0) or the ring
+  long long ldKhat;
+  uint16_t* Vhat;         // output rows or nullptr (encode only)
+  long long ldVhat;
+  const uint32_t* signmask_k;
+  const uint32_t* signmask_v;
+  const float4* grid4;
+  SearchDev search;
+  int log_h, log_g;
+  int* status;
+};
+
+__device__ __forceinline__ void layer_job(int j, int n_waves, int& phase, int& wave) {
+  if (j == 0) { phase = 0; wave = 0; }
+  else if (j == 2 * n_waves - 1) { phase = 1; wave = n_waves - 1; }
+  else if (j & 1) { phase = 0; wave = (j + 1) >> 1; }
+  else { phase = 1; wave = (j >> 1) - 1; }
+}
+__device__ __forceinline__ int layer_key_job(int wave) { return wave == 0 ? 0 : 2 * wave - 1; }
+
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// Spins until *ctr >= target.  Returns false after kWaitLimitNs or if the CTA already aborted.
+__device__ __forceinline__ bool counter_wait_bounded(const int* ctr, int target, volatile int* abort_flag,
+                                                     int* status) {
+  if (ld_acquire(ctr) >= target) return true;
+  const unsigned long long t0 = global_timer_ns();
+  uint32_t spins = 0;
+  while (ld_acquire(ctr) < target) {
+    __nanosleep(64);
+    if ((++spins & 0x3Fu) == 0) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicExch(status, kStatusTimeout);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void named_barrier(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_all() {
+  asm volatile("fence.proxy.async;" ::: "memory");
+}
+
+template <bool kEncode, int D, int NPTS, bool kBf16>
+__global__ void __launch_bounds__(kLayerThreads, 1)
+layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant__ CUtensorMap tmVprev,
+             const __grid_constant__ CUtensorMap tmKhat, const __grid_constant__ CUtensorMap tmWk,
+             const __grid_constant__ CUtensorMap tmWv, const LayerArgs a) {
+  constexpr int NTN = D / kBN;             // feature tiles per token block = CTAs per token block
+  constexpr int RJ = kBM / NTN;            // rows of a token block whose row work this CTA does
+  constexpr int NKD = D / kBK;             // k-blocks per d_kv input features
+  constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
+  constexpr int CODE_BYTES = D / 2 * BITS / 8;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                             ~uintptr_t(1023));
+  LayerSmemTail* tail = reinterpret_cast<LayerSmemTail*>(smem + size_t(kLayerStages) * kStageBytes);
+  RowSmem<NPTS>* rsm = reinterpret_cast<RowSmem<NPTS>*>(
+      (reinterpret_cast<uintptr_t>(tail) + sizeof(LayerSmemTail) + 15) & ~uintptr_t(15));
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int ml = blockIdx.x / NTN;
+  const int n_blk = blockIdx.x % NTN;
+  const int n_jobs = 2 * a.n_waves;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kLayerStages; ++s) {
+      mbar_init(&tail->full[s], 1);
+      mbar_init(&tail->empty[s], 1);
+    }
+    for (int s = 0; s < kAccStages; ++s) {
+      mbar_init(&tail->acc_full[s], 1);
+      mbar_init(&tail->acc_empty[s], 4);
+    }
+    tail->abort_flag = 0;
+    mbar_fence_init();
+  }
+  row_smem_fill<NPTS>(rsm, a.search.table, a.grid4);
+  if (warp == 1) {
+    tmem_alloc(&tail->tmem_base, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = tail->tmem_base;
+  volatile int* abort_flag = &tail->abort_flag;
+
+  if (warp == 0) {
+    // ------------------------------- TMA producer --------------------------------------------
+    if (lane == 0) {
+      tma_prefetch_desc(&tmKprev);
+      tma_prefetch_desc(&tmVprev);
+      tma_prefetch_desc(&tmKhat);
+      tma_prefetch_desc(&tmWk);
+      tma_prefetch_desc(&tmWv);
+      int stage = 0;
+      uint32_t phase_bit = 0;
+      bool ok = true;
+      int issued = 0;
+      for (int j = 0; ok && j < n_jobs; ++j) {
+        int ph, wave;
+        layer_job(j, a.n_waves, ph, wave);
+        const int m = wave * a.mw + ml;
+        if (m >= a.n_mblocks) continue;
+        const int nk = ph == 0 ? NKD : 2 * NKD;
+        const int khat_row = a.khat_ring ? ((wave % a.khat_ring) * a.mw + ml) * kBM : m * kBM;
+        for (int kb = 0; kb < nk; ++kb) {
+          if (ph == 1 && kb == NKD) {
+            // the remaining k-blocks read this wave's reconstructed keys, written by row warps
+            if (!counter_wait_bounded(a.rows_done + layer_key_job(wave) * a.mw + ml, NTN, abort_flag,
+                                      a.status)) {
+              ok = false;
+              break;
+            }
+            fence_proxy_async_all();
+          }
+          if (!mbar_wait_bounded(&tail->empty[stage], phase_bit ^ 1u, abort_flag, a.status)) {
+            ok = false;
+            break;
+          }
+          uint8_t* a_dst = smem + size_t(stage) * kStageBytes;
+          uint8_t* b_dst = a_dst + kABytes;
+          mbar_arrive_expect_tx(&tail->full[stage], kStageBytes);
+          if (ph == 0) {
+            tma_load_2d(a_dst, &tmKprev, &tail->full[stage], kb * kBK, m * kBM);
+            tma_load_2d(b_dst, &tmWk, &tail->full[stage], kb * kBK, n_blk * kBN);
+          } else {
+            if (kb < NKD) {
+              tma_load_2d(a_dst, &tmVprev, &tail->full[stage], kb * kBK, m * kBM);
+            } else {
+              tma_load_2d(a_dst, &tmKhat, &tail->full[stage], (kb - NKD) * kBK, khat_row);
+            }
+            tma_load_2d(b_dst, &tmWv, &tail->full[stage], kb * kBK, n_blk * kBN);
+          }
+          ++issued;
+          if (++stage == kLayerStages) { stage = 0; phase_bit ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // let this CTA's copies in flight land before its shared memory is released
+        int s = stage;
+        uint32_t pb = phase_bit;
+        const int pending = issued < kLayerStages ? issued : kLayerStages;
+        for (int i = 0; i < pending; ++i) {
+          if (s == 0) { s = kLayerStages; pb ^= 1u; }
+          --s;
+          const unsigned long long t0 = global_timer_ns();
+          while (!mbar_try_wait(&tail->full[s], pb) && global_timer_ns() - t0 < kWaitLimitNs) {
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer ----------------------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_f16(kBM, kBN, kBf16);
+      int stage = 0;
+      uint32_t phase_bit = 0;
+      bool ok = true;
+      int it = 0;
+      for (int j = 0; ok && j < n_jobs; ++j) {
+        int ph, wave;
+        layer_job(j, a.n_waves, ph, wave);
+        if (wave * a.mw + ml >= a.n_mblocks) continue;
+        const int nk = ph == 0 ? NKD : 2 * NKD;
+        const int acc = it & 1;
+        const uint32_t acc_phase = (it >> 1) & 1u;
+        ++it;
+        if (!mbar_wait_bounded(&tail->acc_empty[acc], acc_phase ^ 1u, abort_flag, a.status)) break;
+        tc_fence_after_sync();
+        const uint32_t tmem_d = tmem_base + uint32_t(acc * kBN);
+        for (int kb = 0; kb < nk; ++kb) {
+          if (!mbar_wait_bounded(&tail->full[stage], phase_bit, abort_flag, a.status)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after_sync();
+          const uint32_t a_addr = smem_u32(smem + size_t(stage) * kStageBytes);
+          const uint32_t b_addr = a_addr + kABytes;
+#pragma unroll
+          for (int k = 0; k < kBK / kUmmaK; ++k) {
+            const uint64_t da = umma_smem_desc_k128(a_addr + k * kUmmaK * 2);
+            const uint64_t db = umma_smem_desc_k128(b_addr + k * kUmmaK * 2);
+            umma_f16(tmem_d, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit(&tail->empty[stage]);
+          if (++stage == kLayerStages) { stage = 0; phase_bit ^= 1u; }
+        }
+        if (ok) umma_commit(&tail->acc_full[acc]);
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------- GEMM epilogue (4 warps) ---------------------------------
+    const int quarter = warp & 3;   // tensor-memory lanes [32*quarter, 32*quarter+32)
+    int it = 0;
+    for (int j = 0; j < n_jobs; ++j) {
+      int ph, wave;
+      layer_job(j, a.n_waves, ph, wave);
+      const int m = wave * a.mw + ml;
+      if (m >= a.n_mblocks) continue;
+      const int acc = it & 1;
+      const uint32_t acc_phase = (it >> 1) & 1u;
+      ++it;
+      bool ok = true;
+      // the ring slot of this job was last used by job j - nb: its row work must be over
+      if (j >= a.nb) {
+        if (lane == 0) ok = counter_wait_bounded(a.rows_done + (j - a.nb) * a.mw + ml, NTN, abort_flag, a.status);
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+      }
+      if (ok) ok = mbar_wait_bounded(&tail->acc_full[acc], acc_phase, abort_flag, a.status);
+      if (ok) {
+        tc_fence_after_sync();
+        const int r = quarter * 32 + lane;
+        const bool valid = m * kBM + r < a.T;
+        const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * kBN);
+        float* out = a.P + (size_t(j % a.nb) * a.mw * kBM + size_t(ml) * kBM + r) * D + n_blk * kBN;
+        const float* bias = ph == 0 ? a.bk : a.bv;
+#pragma unroll 1
+        for (int c = 0; c < kBN / 32; ++c) {
+          float v[32];
+          tmem_ld_32x32b_x32(taddr + uint32_t(c * 32), v);
+          if (valid) {
+            if (bias != nullptr) {
+              const float* b = bias + n_blk * kBN + c * 32;
+#pragma unroll
+              for (int i = 0; i < 32; ++i) v[i] = __fadd_rn(v[i], __ldg(b + i));
+            }
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              __stcg(reinterpret_cast<float4*>(out + c * 32 + i), make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]));
+          }
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tail->acc_empty[acc]);
+      }
+      __threadfence();
+      named_barrier(1, 128);
+      if (*abort_flag) break;
+      if (warp == 2 && lane == 0) atomicAdd(a.gemm_done + j * a.mw + ml, 1);
+    }
+  } else {
+    // ------------------------------- row warps ------------------------------------------------
+    const int rw = warp - 6;
+    RowCtx rck, rcv;
+    rck.lane = rcv.lane = lane;
+    rck.signmask = a.signmask_k[lane];
+    rcv.signmask = a.signmask_v[lane];
+    rck.inv_w = rcv.inv_w = a.search.inv_w;
+    rck.log_h = rcv.log_h = a.log_h;
+    rck.log_g = rcv.log_g = a.log_g;
+    const int n_groups = D >> a.log_g;
+    for (int j = 0; j < n_jobs; ++j) {
+      int ph, wave;
+      layer_job(j, a.n_waves, ph, wave);
+      const int m = wave * a.mw + ml;
+      if (m >= a.n_mblocks) continue;
+      bool ok = true;
+      if (lane == 0) ok = counter_wait_bounded(a.gemm_done + j * a.mw + ml, NTN, abort_flag, a.status);
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (ok) {
+        const float* pbuf = a.P + (size_t(j % a.nb) * a.mw * kBM + size_t(ml) * kBM) * D;
+        const size_t khat_base = a.khat_ring ? size_t((wave % a.khat_ring) * a.mw + ml) * kBM
+                                             : size_t(m) * kBM;
+        for (int r = n_blk * RJ + rw; r < (n_blk + 1) * RJ; r += kRowWarps) {
+          const long long g = (long long)m * kBM + r;
+          if (g >= a.T) break;
+          const float* pred_row = pbuf + size_t(r) * D;
+          uint16_t* hat_row;
+          if (ph == 0) hat_row = a.Khat + (khat_base + r) * a.ldKhat;
+          else hat_row = a.Vhat != nullptr ? a.Vhat + g * a.ldVhat : nullptr;
+          uint8_t* codes_row = (ph == 0 ? a.Kcodes : a.Vcodes) + g * CODE_BYTES;
+          uint16_t* scales_row = (ph == 0 ? a.Kscales : a.Vscales) + g * n_groups;
+          if constexpr (kEncode) {
+            const uint16_t* x_row = (ph == 0 ? a.K : a.V) + g * a.ldX;
+            encode_row<D, NPTS, kBf16>(ph == 0 ? rck : rcv, rsm, x_row, pred_row, codes_row, scales_row,
+                                       hat_row);
+          } else {
+            decode_row<D, NPTS, kBf16>(ph == 0 ? rck : rcv, rsm->grid, codes_row, scales_row, pred_row, hat_row);
+          }
+        }
+      }
+      __threadfence();
+      fence_proxy_async_all();
+      named_barrier(2, kRowWarps * 32);
+      if (*abort_flag) break;
+      if (rw == 0 && lane == 0) atomicAdd(a.rows_done + j * a.mw + ml, 1);
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace aquakv

@@ -1,0 +1,116 @@
+// Host-side construction of the cell table that prunes the nearest-grid-point search of the
+// backbone quantizer (Section 2 "Vector Quantization": every pair of rotated values is rounded to
+// the nearest of n fixed 2-D points; Section 4.1: n in {16, 64, 256}).
+//
+// The square [-B, B)^2 is cut into C x C cells.  For each cell the table lists every grid point
+// whose Voronoi region meets the (slightly inflated) cell, so the exact arg-min over ALL points
+// equals the arg-min over the listed ones for any y inside the cell.  Cells that need more
+// candidates than the kernel evaluates (three for n = 16, four for larger grids), and values
+// outside the square, are searched exhaustively by the kernel; the table therefore never changes a
+// result, it only skips points that cannot win.
+//
+// Entry layout (uint32): bytes 0..3 = candidate indices in ascending order (short lists repeat
+// their last index); the single descending pattern 0x00000001 marks a cell that must be searched
+// exhaustively.
+#pragma once
+
+#include <cmath>
+#include <cstdint>
+#include <vector>
+
+namespace aquakv {
+
+constexpr uint32_t kCellBrute = 1u;   // bytes (1, 0, 0, 0): not ascending, so never a candidate list
+
+struct SearchTableSpec {
+  int cells;        // C, cells per side (power of two)
+  int log_cells;
+  float half;       // B
+  float inv_w;      // C / (2B), the value the kernel multiplies by
+  int max_cand;     // candidates the kernel evaluates per pair
+};
+
+inline SearchTableSpec search_table_spec(const float* grid, int n) {
+  float m = 0.0f;
+  for (int i = 0; i < 2 * n; ++i) m = std::fmax(m, std::fabs(grid[i]));
+  SearchTableSpec s;
+  s.max_cand = n <= 16 ? 3 : 4;
+  s.cells = 64;          // kSearchCells of codec.cuh: the kernels keep the table in shared memory
+  s.log_cells = 6;
+  s.half = std::ceil((m + 2.0f) * 4.0f) / 4.0f;
+  s.inv_w = float(s.cells) / (2.0f * s.half);
+  return s;
+}
+
+namespace detail {
+struct Pt { double x, y; };
+
+// Keeps the part of the convex polygon with a.x*x + a.y*y <= b (Sutherland-Hodgman).
+inline void clip(std::vector<Pt>& poly, double ax, double ay, double b) {
+  std::vector<Pt> out;
+  const size_t m = poly.size();
+  for (size_t i = 0; i < m; ++i) {
+    const Pt p = poly[i], q = poly[(i + 1) % m];
+    const double fp = ax * p.x + ay * p.y - b, fq = ax * q.x + ay * q.y - b;
+    if (fp <= 0.0) out.push_back(p);
+    if ((fp < 0.0 && fq > 0.0) || (fp > 0.0 && fq < 0.0)) {
+      const double t = fp / (fp - fq);
+      out.push_back(Pt{p.x + t * (q.x - p.x), p.y + t * (q.y - p.y)});
+    }
+  }
+  poly.swap(out);
+}
+}  // namespace detail
+
+// Fills table[cells*cells] (row = y cell, column = x cell).
+inline void build_search_table(const float* grid, int n, const SearchTableSpec& s, uint32_t* table) {
+  const int C = s.cells;
+  const double w = 1.0 / double(s.inv_w);
+  const double eps = 1e-3 * w + 1e-5;        // covers fp32 rounding of the cell index and scores
+  const double tol = 1e-9;
+  std::vector<double> dist(n);
+  std::vector<int> pre, cand;
+  std::vector<detail::Pt> poly;
+  for (int iy = 0; iy < C; ++iy) {
+    for (int ix = 0; ix < C; ++ix) {
+      const double x0 = (ix - C / 2) * w - eps, x1 = (ix + 1 - C / 2) * w + eps;
+      const double y0 = (iy - C / 2) * w - eps, y1 = (iy + 1 - C / 2) * w + eps;
+      const double cx = 0.5 * (x0 + x1), cy = 0.5 * (y0 + y1);
+      const double r = 0.5 * std::sqrt((x1 - x0) * (x1 - x0) + (y1 - y0) * (y1 - y0));
+      double dmin = 1e300;
+      for (int j = 0; j < n; ++j) {
+        const double dx = cx - grid[2 * j], dy = cy - grid[2 * j + 1];
+        dist[j] = std::sqrt(dx * dx + dy * dy);
+        dmin = std::fmin(dmin, dist[j]);
+      }
+      // a point farther than dmin + 2r from the centre loses everywhere in the cell
+      pre.clear();
+      for (int j = 0; j < n; ++j)
+        if (dist[j] <= dmin + 2.0 * r + 1e-9) pre.push_back(j);
+      cand.clear();
+      for (int i : pre) {
+        poly.assign({{x0, y0}, {x1, y0}, {x1, y1}, {x0, y1}});
+        const double gix = grid[2 * i], giy = grid[2 * i + 1];
+        for (int k : pre) {
+          if (k == i || poly.empty()) continue;
+          const double gkx = grid[2 * k], gky = grid[2 * k + 1];
+          // |y - g_i|^2 <= |y - g_k|^2   <=>   2 y.(g_k - g_i) <= |g_k|^2 - |g_i|^2
+          detail::clip(poly, 2.0 * (gkx - gix), 2.0 * (gky - giy),
+                       gkx * gkx + gky * gky - gix * gix - giy * giy + tol);
+        }
+        if (!poly.empty()) cand.push_back(i);
+      }
+      uint32_t e;
+      if (cand.empty() || int(cand.size()) > s.max_cand) {
+        e = kCellBrute;
+      } else {
+        e = 0;
+        for (int k = 0; k < 4; ++k)
+          e |= uint32_t(cand[k < int(cand.size()) ? k : int(cand.size()) - 1]) << (8 * k);
+      }
+      table[size_t(iy) * C + ix] = e;
+    }
+  }
+}
+
+}  // namespace aquakv

@@ -126,3 +126,59 @@ def test_encode_with_adapters_teacher_forced(cfg, T, n):
         Kh3, Vh3 = codec.decode(Kc, Ks, Vc, Vs, dev(prevK), dev(prevV), dev(Wk), dev(Wv))
         assert torch.equal(Kh3, Kh) and torch.equal(Vh3, Vh)
         prevK, prevV = ok_["hat"], ov_["hat"]
+
+
+def _sample_rows(T, seed):
+    rng = np.random.default_rng(seed)
+    edges = [0, 1, 31, 32, 127, 128, 129, 4735, 4736, 4737, 9471, 9472, T - 129, T - 128, T - 2, T - 1]
+    rows = sorted({r for r in edges if 0 <= r < T} | set(rng.integers(0, T, 160).tolist()))
+    return np.array(rows, dtype=np.int64)
+
+
+@pytest.mark.parametrize("T,n", [(32768, 16), (9549, 16), (4737, 64)])
+def test_full_size_layer_on_sampled_rows(T, n):
+    """One layer of the benchmark's launch configuration (all tokens in one call: several waves of
+    token blocks through the fused layer kernel, ragged last block) against the oracle on sampled
+    rows; rows are independent, so the oracle's result for a row does not depend on the others."""
+    shape, kv, ad = chain(2, T, 2, grid_size=n)
+    d, dtype, bits = shape.d_kv, shape.dtype, shape.code_bits
+    codec, ora = make(d, shape.had_block, shape.scale_group, n, dtype)
+    prevK, prevV = kv.K[0], kv.V[0]          # any 16-bit rows serve as the previous layer's reconstruction
+    K, V, Wk, Wv = kv.K[1], kv.V[1], ad.Wk[1], ad.Wv[1]
+    g = lambda t: t.to(DEV)
+    Kc, Ks, Vc, Vs, Kh, Vh = codec.encode(g(K), g(V), g(prevK), g(prevV), g(Wk), g(Wv))
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    rows = _sample_rows(T, seed=T + n)
+    b = synth.to_bits
+    sel = lambda t: b(t)[rows]
+    ok_ = ora.encode_phase(sel(K), [sel(prevK)], b(Wk), None, "k")
+    rows_ok, n_bad = scale_rows_ok(gpu_bits(Ks.view(torch.float16))[rows], ok_["scales"], ok_["scales_exact"])
+    assert n_bad <= 2
+    check_codes(Kc.cpu().numpy()[rows], ok_, bits, rows_ok)
+    same = rows_ok & (Kc.cpu().numpy()[rows] == ok_["codes"]).all(axis=1)
+    assert same.mean() > 0.9
+    check_recon(gpu_bits(Kh)[rows], ok_["hat_exact"], ok_["hat"], dtype, same)
+    # values: the oracle is given the library's reconstructed keys of those rows (teacher forcing)
+    ov_ = ora.encode_phase(sel(V), [sel(prevV), gpu_bits(Kh)[rows]], b(Wv), None, "v")
+    rows_ok_v, n_bad = scale_rows_ok(gpu_bits(Vs.view(torch.float16))[rows], ov_["scales"], ov_["scales_exact"])
+    assert n_bad <= 2
+    check_codes(Vc.cpu().numpy()[rows], ov_, bits, rows_ok_v)
+    same_v = rows_ok_v & (Vc.cpu().numpy()[rows] == ov_["codes"]).all(axis=1)
+    assert same_v.mean() > 0.9
+    check_recon(gpu_bits(Vh)[rows], ov_["hat_exact"], ov_["hat"], dtype, same_v)
+    # decode of the library's own codes reproduces the encoder's reconstruction bit for bit, all rows
+    Kh2, Vh2 = codec.decode(Kc, Ks, Vc, Vs, g(prevK), g(prevV), g(Wk), g(Wv))
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    assert torch.equal(Kh2, Kh) and torch.equal(Vh2, Vh)
+    # the single-phase entry points (separate GEMM and row kernels) agree with the fused kernel, all rows
+    from paper_2501_19392_b200 import api
+    Kc3, Ks3, Kh3 = codec.encode_phase(api.ROLE_KEY, g(K), g(prevK), None, g(Wk))
+    assert torch.equal(Kc3, Kc) and torch.equal(Ks3, Ks) and torch.equal(Kh3, Kh)
+    Vc3, Vs3, Vh3 = codec.encode_phase(api.ROLE_VALUE, g(V), g(prevV), Kh, g(Wv))
+    assert torch.equal(Vc3, Vc) and torch.equal(Vs3, Vs) and torch.equal(Vh3, Vh)
+    # encode without the optional reconstructions (keys kept in the workspace ring) gives the same codes
+    Kc4, Ks4, Vc4, Vs4, _, _ = codec.encode(g(K), g(V), g(prevK), g(prevV), g(Wk), g(Wv), want_hat=False)
+    torch.cuda.synchronize()
+    assert torch.equal(Kc4, Kc) and torch.equal(Vc4, Vc) and torch.equal(Ks4, Ks) and torch.equal(Vs4, Vs)
