@@ -189,7 +189,8 @@ void launch_decode_rows_t(aquakv_ctx*, cudaStream_t st, const CodecArgs& a, int 
   } while (0)
 
 int codec_grid(const aquakv_ctx* c, int rows) {
-  const int blocks = (rows + kCodecWarps - 1) / kCodecWarps;
+  const int rows_per_block = kCodecWarps / (c->p.d_kv >= 512 ? 2 : 1);   // two-warp teams above 256
+  const int blocks = (rows + rows_per_block - 1) / rows_per_block;
   const int cap = c->sm_count * 8;
   return blocks < cap ? blocks : cap;
 }
@@ -393,7 +394,7 @@ LayerWs layer_ws(const aquakv_ctx* c, int64_t T) {
 template <bool ENC, int D, int NPTS, bool BF>
 int launch_layer_t(cudaStream_t st, int grid, const CUtensorMap* tm, const LayerArgs& a) {
   static bool attr_set = false;   // per instantiation; contexts are used from one thread at a time
-  constexpr size_t smem = layer_smem_bytes<NPTS>();
+  constexpr size_t smem = layer_smem_bytes<D, NPTS>();
   if (!attr_set) {
     if (cudaFuncSetAttribute(layer_kernel<ENC, D, NPTS, BF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              int(smem)) != cudaSuccess)

@@ -3,11 +3,15 @@
 // 2-D grid, packed codes) and of the residual / add-back steps of Algorithm 2 (lines 6-7, 9) and
 // Algorithm 3 (lines 5, 7).
 //
-// One warp owns one token row.  Element e of the row lives in lane (e/8)%32, register
-// (e/256)*8 + e%8, so every global access is a 16-byte (16-bit data) or 2x16-byte (fp32) vector
-// per lane and a warp touches whole 128-byte lines.  The Hadamard butterflies over index bits
-// 0-2 and 8-9 are register-local, bits 3-7 are warp shuffles.  The value pair (2j, 2j+1) that
-// shares one code always sits in one lane.
+// A team of one warp (d_kv = 256) or two warps (d_kv = 512, 1024) owns one token row; each warp
+// holds one or two 256-element chunks.  Element e of the row lives in warp (e/256)/chunks-per-warp,
+// lane (e/8)%32, register ((e/256)%chunks-per-warp)*8 + e%8, so every global access is a 16-byte
+// (16-bit data) or 2x16-byte (fp32) vector per lane and a warp touches whole 128-byte lines.  The
+// Hadamard butterflies over index bits 0-2 are register-local, bits 3-7 are warp shuffles, the
+// next bit (two-chunk warps) is register-local again and the top bit crosses the two warps through
+// shared memory.  Splitting a row over two warps halves the registers per thread, which is what
+// lets enough warps be resident to hide the latencies of this shuffle- and load-heavy code.  The
+// value pair (2j, 2j+1) that shares one code always sits in one lane.
 #pragma once
 
 #include "common.cuh"
@@ -120,20 +124,6 @@ __device__ __forceinline__ float apply_sign(float x, uint32_t mask, int i) {
   return __uint_as_float(__float_as_uint(x) ^ ((mask << (31 - i)) & 0x80000000u));
 }
 
-// Q^-1 without the prediction: grid points of this lane's codes -> inverse rotation -> scale.
-// `w` enters holding the gathered grid coordinates and leaves holding xhat.  The exact operation
-// order (multiply by 1/sqrt(h), then by the scale, sign flip) is shared by encode and decode so
-// that both produce bit-identical reconstructions.
-template <int NV>
-__device__ __forceinline__ void rotate_back_and_scale(float (&w)[NV], const float (&sf)[NV / 8],
-                                                      uint32_t signmask, int log_h, int lane) {
-  fwht_regs_and_lanes<NV>(w, log_h, lane);
-  const float rs = exp2f(-0.5f * static_cast<float>(log_h));   // exact for even log_h
-#pragma unroll
-  for (int i = 0; i < NV; ++i)
-    w[i] = apply_sign(__fmul_rn(__fmul_rn(w[i], rs), sf[i >> 3]), signmask, i);
-}
-
 template <int BITS>
 __device__ __forceinline__ uint32_t load_code_word(const uint8_t* row_codes, int chunk, int lane) {
   const int idx = chunk * 32 + lane;   // 8 values = 4 codes = 4*BITS bits per (chunk, lane)
@@ -159,35 +149,6 @@ __device__ __forceinline__ void store_code_word(uint8_t* row_codes, int chunk, i
     p[0] = static_cast<uint8_t>(w);
     p[1] = static_cast<uint8_t>(w >> 8);
     p[2] = static_cast<uint8_t>(w >> 16);
-  }
-}
-
-// Sum of squares of each scale group, delivered to every lane for each of its register chunks.
-template <int NC>
-__device__ __forceinline__ void group_sums(const float (&v)[NC * 8], float (&ss)[NC], int log_g) {
-#pragma unroll
-  for (int c = 0; c < NC; ++c) {
-    float s = 0.0f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) s = fmaf(v[c * 8 + i], v[c * 8 + i], s);
-#pragma unroll
-    for (int b = 3; b < 8; ++b)
-      if (b < log_g) s += __shfl_xor_sync(0xffffffffu, s, 1 << (b - 3));
-    ss[c] = s;
-  }
-  if (log_g > 8) {
-    const int cpg = 1 << (log_g - 8);   // register chunks per group
-    float tot[NC];
-#pragma unroll
-    for (int c = 0; c < NC; ++c) {
-      float s = 0.0f;
-#pragma unroll
-      for (int c2 = 0; c2 < NC; ++c2)
-        if ((c2 / cpg) == (c / cpg)) s += ss[c2];
-      tot[c] = s;
-    }
-#pragma unroll
-    for (int c = 0; c < NC; ++c) ss[c] = tot[c];
   }
 }
 
@@ -237,95 +198,212 @@ __device__ __noinline__ int nearest_exhaustive(float y0, float y1, const float2*
   return idx;
 }
 
+// Geometry of a row team.
+template <int D>
+struct RowTeam {
+  static constexpr int NC = D / 256;                 // 256-element chunks per row
+  static constexpr int TEAM = NC >= 2 ? 2 : 1;       // warps per row
+  static constexpr int CPM = NC / TEAM;              // chunks per warp
+  static constexpr int NV = CPM * 8;                 // values per lane
+  static constexpr int CROSS_BIT = 8 + (CPM == 2 ? 1 : 0);   // index bit that separates the warps
+};
+
+// Exchange buffer of one team (only used when TEAM == 2).
+template <int D>
+struct TeamSmem {
+  float4 x[2][RowTeam<D>::CPM * 2][32];   // [member][16-byte piece][lane]
+  float ss[2][2];                         // [member][chunk] sums of squares
+};
+
 // Per-warp constants of the row routines.
 struct RowCtx {
   uint32_t signmask;       // this lane's entry of CodecArgs::signmask
   float inv_w;             // SearchDev::inv_w
   int log_h, log_g;
   int lane;
+  int member;              // 0 or 1: which half of the row this warp holds
+  int barrier;             // named barrier shared by the two warps of the team
 };
 
-// One token row of Q and of the reconstruction (Algorithm 2 lines 6-7 / 9):
+__device__ __forceinline__ void team_barrier(int id) {
+  asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory");
+}
+
+// Publishes this warp's values (and optionally its chunk sums) and reads the partner's.
+template <int D, bool kWithSums>
+__device__ __forceinline__ void team_exchange(const RowCtx& rc, TeamSmem<D>* ts,
+                                              const float (&v)[RowTeam<D>::NV], float (&o)[RowTeam<D>::NV],
+                                              const float (&ss)[RowTeam<D>::CPM],
+                                              float (&oss)[RowTeam<D>::CPM]) {
+  constexpr int NV = RowTeam<D>::NV, CPM = RowTeam<D>::CPM;
+  team_barrier(rc.barrier);                // the partner has finished reading the previous exchange
+#pragma unroll
+  for (int q = 0; q < NV / 4; ++q)
+    ts->x[rc.member][q][rc.lane] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+  if (kWithSums && rc.lane == 0) {
+#pragma unroll
+    for (int c = 0; c < CPM; ++c) ts->ss[rc.member][c] = ss[c];
+  }
+  team_barrier(rc.barrier);
+#pragma unroll
+  for (int q = 0; q < NV / 4; ++q) {
+    const float4 t = ts->x[rc.member ^ 1][q][rc.lane];
+    o[4 * q] = t.x; o[4 * q + 1] = t.y; o[4 * q + 2] = t.z; o[4 * q + 3] = t.w;
+  }
+  if (kWithSums) {
+#pragma unroll
+    for (int c = 0; c < CPM; ++c) oss[c] = ts->ss[rc.member ^ 1][c];
+  }
+}
+
+// Butterfly over the index bit that separates the two warps: the lower half keeps a + b, the upper
+// half a - b (a = lower half's value, b = upper half's).
+template <int NV>
+__device__ __forceinline__ void cross_butterfly(float (&v)[NV], const float (&o)[NV], int member) {
+#pragma unroll
+  for (int i = 0; i < NV; ++i) v[i] = member == 0 ? __fadd_rn(v[i], o[i]) : __fsub_rn(o[i], v[i]);
+}
+
+// Q^-1 without the prediction for this warp's part of the row: `w` enters holding the gathered grid
+// coordinates and leaves holding xhat.  The operation order (rotation stages by ascending index bit,
+// multiply by 1/sqrt(h), then by the scale, sign flip) is shared by encode and decode so that both
+// produce bit-identical reconstructions.
+template <int D>
+__device__ __forceinline__ void team_rotate_back_and_scale(const RowCtx& rc, TeamSmem<D>* ts,
+                                                           float (&w)[RowTeam<D>::NV],
+                                                           const float (&sf)[RowTeam<D>::CPM]) {
+  using RT = RowTeam<D>;
+  fwht_regs_and_lanes<RT::NV>(w, rc.log_h, rc.lane);
+  if constexpr (RT::TEAM == 2) {
+    if (RT::CROSS_BIT < rc.log_h) {
+      float o[RT::NV], dummy_a[RT::CPM] = {}, dummy_b[RT::CPM];
+      team_exchange<D, false>(rc, ts, w, o, dummy_a, dummy_b);
+      cross_butterfly<RT::NV>(w, o, rc.member);
+    }
+  }
+  const float rs = exp2f(-0.5f * static_cast<float>(rc.log_h));   // exact for even log_h
+#pragma unroll
+  for (int i = 0; i < RT::NV; ++i)
+    w[i] = apply_sign(__fmul_rn(__fmul_rn(w[i], rs), sf[i >> 3]), rc.signmask,
+                      rc.member * RT::NV + i);
+}
+
+// This warp's part of one token row of Q and of the reconstruction (Algorithm 2 lines 6-7 / 9):
 //   codes, scales = Q(x - pred);  hat = round16(pred + Q^-1(codes, scales)).
-// pred_row == nullptr: no predictor.  hat_row == nullptr: reconstruction not wanted.  The prediction
-// is read twice (for the residual and again for the reconstruction) instead of being held in 32
-// registers across the rotation and the search; both reads bypass L1 (ld.global.cg) because the
-// prediction may have been written by another SM of the same kernel just before.
+// All row pointers address the start of the row.  pred_row == nullptr: no predictor.
+// hat_row == nullptr: reconstruction not wanted.  The prediction is read twice (for the residual and
+// again for the reconstruction) instead of being held in registers across the rotation and the
+// search; both reads bypass L1 (ld.global.cg) because the prediction may have been written by
+// another SM of the same kernel just before.  Both warps of a team must call this together.
 template <int D, int NPTS, bool kBf16>
 __device__ __forceinline__ void encode_row(const RowCtx& rc, const RowSmem<NPTS>* __restrict__ rsm,
-                                           const uint16_t* __restrict__ x_row,
+                                           TeamSmem<D>* ts, const uint16_t* __restrict__ x_row,
                                            const float* __restrict__ pred_row,
                                            uint8_t* __restrict__ codes_row,
                                            uint16_t* __restrict__ scales_row,
                                            uint16_t* __restrict__ hat_row) {
-  constexpr int NC = D / 256, NV = NC * 8;
+  using RT = RowTeam<D>;
+  constexpr int NC = RT::NC, CPM = RT::CPM, NV = RT::NV;
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
   const int lane = rc.lane;
+  const int c0 = rc.member * CPM;                    // first chunk of this warp
   const float inv_g = exp2f(-static_cast<float>(rc.log_g));
   const float rs = exp2f(-0.5f * static_cast<float>(rc.log_h));
   float v[NV];
   // ---- residual r = x - pred -------------------------------------------------------------------
   {
-    uint4 raw[NC];
+    uint4 raw[CPM];
 #pragma unroll
-    for (int c = 0; c < NC; ++c)
-      raw[c] = *reinterpret_cast<const uint4*>(x_row + c * 256 + lane * 8);
+    for (int c = 0; c < CPM; ++c)
+      raw[c] = *reinterpret_cast<const uint4*>(x_row + (c0 + c) * 256 + lane * 8);
+    float4 pq[CPM][2];
     if (pred_row != nullptr) {
-      float4 pq[NC][2];
 #pragma unroll
-      for (int c = 0; c < NC; ++c) {
-        pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + c * 256 + lane * 8));
-        pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + c * 256 + lane * 8 + 4));
+      for (int c = 0; c < CPM; ++c) {
+        pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + lane * 8));
+        pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + lane * 8 + 4));
       }
+    }
 #pragma unroll
-      for (int c = 0; c < NC; ++c) {
-        const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
+    for (int c = 0; c < CPM; ++c) {
+      const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        v[c * 8 + 2 * i] = load16<kBf16>(uint16_t(w[i] & 0xffffu));
+        v[c * 8 + 2 * i + 1] = load16<kBf16>(uint16_t(w[i] >> 16));
+      }
+      if (pred_row != nullptr) {
         const float pp[8] = {pq[c][0].x, pq[c][0].y, pq[c][0].z, pq[c][0].w,
                              pq[c][1].x, pq[c][1].y, pq[c][1].z, pq[c][1].w};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          v[c * 8 + 2 * i] = __fsub_rn(load16<kBf16>(uint16_t(w[i] & 0xffffu)), pp[2 * i]);
-          v[c * 8 + 2 * i + 1] = __fsub_rn(load16<kBf16>(uint16_t(w[i] >> 16)), pp[2 * i + 1]);
-        }
-      }
-    } else {
-#pragma unroll
-      for (int c = 0; c < NC; ++c) {
-        const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          v[c * 8 + 2 * i] = load16<kBf16>(uint16_t(w[i] & 0xffffu));
-          v[c * 8 + 2 * i + 1] = load16<kBf16>(uint16_t(w[i] >> 16));
-        }
+        for (int i = 0; i < 8; ++i) v[c * 8 + i] = __fsub_rn(v[c * 8 + i], pp[i]);
       }
     }
   }
-  // ---- group scale: root mean square, stored as fp16; normalise with the rounded value --------
-  float ss[NC], sf[NC], inv[NC];
-  group_sums<NC>(v, ss, rc.log_g);
+  // ---- per-chunk sums of squares (lane bits reduced by shuffles), sign flip ---------------------
+  float ss[CPM];
 #pragma unroll
-  for (int c = 0; c < NC; ++c) {
-    const float s = fminf(sqrtf(ss[c] * inv_g), 65504.0f);
-    const __half s16 = __float2half_rn(s);
-    sf[c] = __half2float(s16);
-    if (rc.log_g >= 8) {                 // one lane per group writes the scale
+  for (int c = 0; c < CPM; ++c) {
+    float s = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s = fmaf(v[c * 8 + i], v[c * 8 + i], s);
+#pragma unroll
+    for (int b = 3; b < 8; ++b)
+      if (b < rc.log_g) s += __shfl_xor_sync(0xffffffffu, s, 1 << (b - 3));
+    ss[c] = s;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[c * 8 + i] = apply_sign(v[c * 8 + i], rc.signmask, (c0 + c) * 8 + i);
+  }
+  // ---- rotate (the division by the scale is applied afterwards: the rotation is linear) ---------
+  fwht_regs_and_lanes<NV>(v, rc.log_h, lane);
+  float all_ss[NC];
+#pragma unroll
+  for (int c = 0; c < NC; ++c) all_ss[c] = 0.0f;
+  if constexpr (RT::TEAM == 2) {
+    if (RT::CROSS_BIT < rc.log_g) {          // scale groups (and maybe Hadamard blocks) span both warps
+      float o[NV], oss[CPM];
+      team_exchange<D, true>(rc, ts, v, o, ss, oss);
+      if (RT::CROSS_BIT < rc.log_h) cross_butterfly<NV>(v, o, rc.member);
+#pragma unroll
+      for (int c = 0; c < CPM; ++c) {
+        all_ss[c0 + c] = ss[c];
+        all_ss[(c0 ^ CPM) + c] = oss[c];
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < CPM; ++c) all_ss[c0 + c] = ss[c];
+    }
+  } else {
+#pragma unroll
+    for (int c = 0; c < CPM; ++c) all_ss[c] = ss[c];
+  }
+  // ---- group scale: root mean square, stored as fp16; normalise with the rounded value ----------
+  float sf[CPM];
+#pragma unroll
+  for (int c = 0; c < CPM; ++c) {
+    float tot = ss[c];
+    if (rc.log_g > 8) {                      // groups of several chunks: add them in ascending order
       const int cpg = 1 << (rc.log_g - 8);
-      if (lane == 0 && (c % cpg) == 0) scales_row[c / cpg] = __half_as_ushort(s16);
+      tot = 0.0f;
+#pragma unroll
+      for (int c2 = 0; c2 < NC; ++c2)
+        if ((c2 / cpg) == ((c0 + c) / cpg)) tot += all_ss[c2];
+    }
+    const float sc = fminf(sqrtf(tot * inv_g), 65504.0f);
+    const __half s16 = __float2half_rn(sc);
+    sf[c] = __half2float(s16);
+    const int cg = c0 + c;
+    if (rc.log_g >= 8) {                     // one lane per group writes the scale
+      const int cpg = 1 << (rc.log_g - 8);
+      if (lane == 0 && (cg % cpg) == 0) scales_row[cg / cpg] = __half_as_ushort(s16);
     } else {
       const int lpg = 1 << (rc.log_g - 3);   // lanes per group
-      if ((lane % lpg) == 0) scales_row[c * (256 >> rc.log_g) + lane / lpg] = __half_as_ushort(s16);
+      if ((lane % lpg) == 0) scales_row[cg * (256 >> rc.log_g) + lane / lpg] = __half_as_ushort(s16);
     }
-    // the rotation is linear: the division by the scale is applied after it, merged with 1/sqrt(h)
-    inv[c] = (sf[c] > 0.0f ? 1.0f / sf[c] : 0.0f) * rs;
+    const float inv = (sf[c] > 0.0f ? 1.0f / sf[c] : 0.0f) * rs;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[c * 8 + i] = apply_sign(v[c * 8 + i], rc.signmask, c * 8 + i);
+    for (int i = 0; i < 8; ++i) v[c * 8 + i] *= inv;
   }
-  // ---- rotate ------------------------------------------------------------------------------------
-  fwht_regs_and_lanes<NV>(v, rc.log_h, lane);
-#pragma unroll
-  for (int c = 0; c < NC; ++c)
-#pragma unroll
-    for (int i = 0; i < 8; ++i) v[c * 8 + i] *= inv[c];
   // ---- nearest grid point per pair: all table entries first, then the candidates ----------------
   uint32_t entry[NV / 2];
   uint32_t any_brute = 0;
@@ -336,7 +414,7 @@ __device__ __forceinline__ void encode_row(const RowCtx& rc, const RowSmem<NPTS>
   }
   const bool slow = __any_sync(0xffffffffu, any_brute != 0);
 #pragma unroll
-  for (int c = 0; c < NC; ++c) {
+  for (int c = 0; c < CPM; ++c) {
     uint32_t word = 0;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
@@ -354,24 +432,24 @@ __device__ __forceinline__ void encode_row(const RowCtx& rc, const RowSmem<NPTS>
       v[2 * j] = g.x;
       v[2 * j + 1] = g.y;
     }
-    store_code_word<BITS>(codes_row, c, lane, word);
+    store_code_word<BITS>(codes_row, c0 + c, lane, word);
   }
   // ---- reconstruction: hat = round16(pred + Q^-1(codes)) ---------------------------------------
-  if (hat_row != nullptr) {
-    float4 pq[NC][2];
+  if (hat_row != nullptr) {      // uniform over the team
+    float4 pq[CPM][2];
     if (pred_row != nullptr) {
 #pragma unroll
-      for (int c = 0; c < NC; ++c) {
-        pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + c * 256 + lane * 8));
-        pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + c * 256 + lane * 8 + 4));
+      for (int c = 0; c < CPM; ++c) {
+        pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + lane * 8));
+        pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + lane * 8 + 4));
       }
     } else {
 #pragma unroll
-      for (int c = 0; c < NC; ++c) pq[c][0] = pq[c][1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+      for (int c = 0; c < CPM; ++c) pq[c][0] = pq[c][1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
     }
-    rotate_back_and_scale<NV>(v, sf, rc.signmask, rc.log_h, lane);
+    team_rotate_back_and_scale<D>(rc, ts, v, sf);
 #pragma unroll
-    for (int c = 0; c < NC; ++c) {
+    for (int c = 0; c < CPM; ++c) {
       const float pp[8] = {pq[c][0].x, pq[c][0].y, pq[c][0].z, pq[c][0].w,
                            pq[c][1].x, pq[c][1].y, pq[c][1].z, pq[c][1].w};
       uint32_t o[4];
@@ -381,73 +459,90 @@ __device__ __forceinline__ void encode_row(const RowCtx& rc, const RowSmem<NPTS>
         const uint32_t hi = store16<kBf16>(__fadd_rn(pp[2 * i + 1], v[c * 8 + 2 * i + 1]));
         o[i] = lo | (hi << 16);
       }
-      *reinterpret_cast<uint4*>(hat_row + c * 256 + lane * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+      *reinterpret_cast<uint4*>(hat_row + (c0 + c) * 256 + lane * 8) = make_uint4(o[0], o[1], o[2], o[3]);
     }
   }
+}
+
+// Shared memory of the stand-alone row kernels: search tables plus one exchange buffer per team.
+template <int D, int NPTS>
+struct RowKernelSmem {
+  RowSmem<NPTS> tables;
+  TeamSmem<D> team[kCodecWarps / RowTeam<D>::TEAM];
+};
+
+__device__ __forceinline__ RowCtx make_row_ctx(const CodecArgs& a, int team_size, int first_barrier) {
+  RowCtx rc;
+  const int warp = threadIdx.x >> 5;
+  rc.lane = threadIdx.x & 31;
+  rc.signmask = a.signmask[rc.lane];
+  rc.inv_w = a.search.inv_w;
+  rc.log_h = a.log_h;
+  rc.log_g = a.log_g;
+  rc.member = warp % team_size;
+  rc.barrier = first_barrier + warp / team_size;
+  return rc;
 }
 
 template <int D, int NPTS, bool kBf16>
 __global__ void __launch_bounds__(kCodecThreads, 2) encode_rows_kernel(const CodecArgs a) {
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
   constexpr int CODE_BYTES = D / 2 * BITS / 8;
-  __shared__ RowSmem<NPTS> rsm;
-  row_smem_fill<NPTS>(&rsm, a.search.table, a.grid4);
+  constexpr int TEAM = RowTeam<D>::TEAM, TEAMS = kCodecWarps / TEAM;
+  __shared__ RowKernelSmem<D, NPTS> sm;
+  row_smem_fill<NPTS>(&sm.tables, a.search.table, a.grid4);
   __syncthreads();
-  RowCtx rc;
-  rc.lane = threadIdx.x & 31;
-  rc.signmask = a.signmask[rc.lane];
-  rc.inv_w = a.search.inv_w;
-  rc.log_h = a.log_h;
-  rc.log_g = a.log_g;
-  const int warp = threadIdx.x >> 5;
+  const RowCtx rc = make_row_ctx(a, TEAM, 1);
+  const int team = (threadIdx.x >> 5) / TEAM;
   const int n_groups = D >> a.log_g;
-  for (long long row = (long long)blockIdx.x * kCodecWarps + warp; row < a.T;
-       row += (long long)gridDim.x * kCodecWarps) {
-    encode_row<D, NPTS, kBf16>(rc, &rsm, a.X + row * a.ldX,
+  for (long long row = (long long)blockIdx.x * TEAMS + team; row < a.T; row += (long long)gridDim.x * TEAMS) {
+    encode_row<D, NPTS, kBf16>(rc, &sm.tables, &sm.team[team], a.X + row * a.ldX,
                                a.P != nullptr ? a.P + row * a.ldP : nullptr,
                                a.codes + row * CODE_BYTES, a.scales + row * n_groups,
                                a.hat != nullptr ? a.hat + row * a.ldHat : nullptr);
   }
 }
 
-// One token row of Algorithm 3 line 5 / 7 given the prediction:
+// This warp's part of one token row of Algorithm 3 line 5 / 7 given the prediction:
 //   hat = round16(pred + Q^-1(codes, scales)).  pred_row == nullptr: no predictor.
-template <int D, int NPTS, bool kBf16, typename GridT>
-__device__ __forceinline__ void decode_row(const RowCtx& rc, const GridT* __restrict__ grid_s,
-                                           const uint8_t* __restrict__ codes_row,
+template <int D, int NPTS, bool kBf16>
+__device__ __forceinline__ void decode_row(const RowCtx& rc, const float2* __restrict__ grid_s,
+                                           TeamSmem<D>* ts, const uint8_t* __restrict__ codes_row,
                                            const uint16_t* __restrict__ scales_row,
                                            const float* __restrict__ pred_row,
                                            uint16_t* __restrict__ hat_row) {
-  constexpr int NC = D / 256, NV = NC * 8;
+  using RT = RowTeam<D>;
+  constexpr int CPM = RT::CPM, NV = RT::NV;
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
   const int lane = rc.lane;
-  float w[NV], sf[NC];
-  float4 pq[NC][2];
+  const int c0 = rc.member * CPM;
+  float w[NV], sf[CPM];
+  float4 pq[CPM][2];
   if (pred_row != nullptr) {
 #pragma unroll
-    for (int c = 0; c < NC; ++c) {
-      pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + c * 256 + lane * 8));
-      pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + c * 256 + lane * 8 + 4));
+    for (int c = 0; c < CPM; ++c) {
+      pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + lane * 8));
+      pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + lane * 8 + 4));
     }
   } else {
 #pragma unroll
-    for (int c = 0; c < NC; ++c) pq[c][0] = pq[c][1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    for (int c = 0; c < CPM; ++c) pq[c][0] = pq[c][1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
   }
 #pragma unroll
-  for (int c = 0; c < NC; ++c) {
-    const uint32_t word = load_code_word<BITS>(codes_row, c, lane);
+  for (int c = 0; c < CPM; ++c) {
+    const uint32_t word = load_code_word<BITS>(codes_row, c0 + c, lane);
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      const GridT g = grid_s[(word >> (k * BITS)) & (NPTS - 1)];
+      const float2 g = grid_s[(word >> (k * BITS)) & (NPTS - 1)];
       w[c * 8 + 2 * k] = g.x;
       w[c * 8 + 2 * k + 1] = g.y;
     }
-    const int e0 = c * 256 + lane * 8;
+    const int e0 = (c0 + c) * 256 + lane * 8;
     sf[c] = __half2float(__ushort_as_half(scales_row[e0 >> rc.log_g]));
   }
-  rotate_back_and_scale<NV>(w, sf, rc.signmask, rc.log_h, lane);
+  team_rotate_back_and_scale<D>(rc, ts, w, sf);
 #pragma unroll
-  for (int c = 0; c < NC; ++c) {
+  for (int c = 0; c < CPM; ++c) {
     const float pp[8] = {pq[c][0].x, pq[c][0].y, pq[c][0].z, pq[c][0].w,
                          pq[c][1].x, pq[c][1].y, pq[c][1].z, pq[c][1].w};
     uint32_t o[4];
@@ -457,31 +552,28 @@ __device__ __forceinline__ void decode_row(const RowCtx& rc, const GridT* __rest
       const uint32_t hi = store16<kBf16>(__fadd_rn(pp[2 * i + 1], w[c * 8 + 2 * i + 1]));
       o[i] = lo | (hi << 16);
     }
-    *reinterpret_cast<uint4*>(hat_row + c * 256 + lane * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+    *reinterpret_cast<uint4*>(hat_row + (c0 + c) * 256 + lane * 8) = make_uint4(o[0], o[1], o[2], o[3]);
   }
 }
 
 template <int D, int NPTS, bool kBf16>
-__global__ void __launch_bounds__(kCodecThreads) decode_rows_kernel(const CodecArgs a) {
+__global__ void __launch_bounds__(kCodecThreads, 2) decode_rows_kernel(const CodecArgs a) {
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
   constexpr int CODE_BYTES = D / 2 * BITS / 8;
+  constexpr int TEAM = RowTeam<D>::TEAM, TEAMS = kCodecWarps / TEAM;
   __shared__ float2 grid_s[NPTS];
+  __shared__ TeamSmem<D> team_s[TEAMS];
   for (int i = threadIdx.x; i < NPTS; i += blockDim.x) {
     const float4 g = a.grid4[i];
     grid_s[i] = make_float2(g.x, g.y);
   }
   __syncthreads();
-  RowCtx rc;
-  rc.lane = threadIdx.x & 31;
-  rc.signmask = a.signmask[rc.lane];
-  rc.inv_w = a.search.inv_w;
-  rc.log_h = a.log_h;
-  rc.log_g = a.log_g;
-  const int warp = threadIdx.x >> 5;
+  const RowCtx rc = make_row_ctx(a, TEAM, 1);
+  const int team = (threadIdx.x >> 5) / TEAM;
   const int n_groups = D >> a.log_g;
-  for (long long row = (long long)blockIdx.x * kCodecWarps + warp; row < a.T;
-       row += (long long)gridDim.x * kCodecWarps) {
-    decode_row<D, NPTS, kBf16>(rc, grid_s, a.codes + row * CODE_BYTES, a.scales + row * n_groups,
+  for (long long row = (long long)blockIdx.x * TEAMS + team; row < a.T; row += (long long)gridDim.x * TEAMS) {
+    decode_row<D, NPTS, kBf16>(rc, grid_s, &team_s[team], a.codes + row * CODE_BYTES,
+                               a.scales + row * n_groups,
                                a.P != nullptr ? a.P + row * a.ldP : nullptr, a.hat + row * a.ldHat);
   }
 }

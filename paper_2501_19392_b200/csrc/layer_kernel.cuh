@@ -33,9 +33,9 @@
 
 namespace aquakv {
 
-constexpr int kRowWarps = 8;
+constexpr int kRowWarps = 16;
 constexpr int kLayerThreads = 32 * (6 + kRowWarps);
-constexpr int kLayerStages = 4;
+constexpr int kLayerStages = 3;
 
 struct LayerSmemTail {
   uint64_t full[kLayerStages];
@@ -46,9 +46,15 @@ struct LayerSmemTail {
   int abort_flag;
 };
 
-template <int NPTS>
+template <int D, int NPTS>
+struct LayerRowSmem {
+  RowSmem<NPTS> tables;
+  TeamSmem<D> team[kRowWarps / RowTeam<D>::TEAM];
+};
+
+template <int D, int NPTS>
 constexpr size_t layer_smem_bytes() {
-  return 1024 + size_t(kLayerStages) * kStageBytes + sizeof(LayerSmemTail) + 16 + sizeof(RowSmem<NPTS>);
+  return 1024 + size_t(kLayerStages) * kStageBytes + sizeof(LayerSmemTail) + 16 + sizeof(LayerRowSmem<D, NPTS>);
 }
 
 struct LayerArgs {
@@ -140,7 +146,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~uintptr_t(1023));
   LayerSmemTail* tail = reinterpret_cast<LayerSmemTail*>(smem + size_t(kLayerStages) * kStageBytes);
-  RowSmem<NPTS>* rsm = reinterpret_cast<RowSmem<NPTS>*>(
+  LayerRowSmem<D, NPTS>* rsm = reinterpret_cast<LayerRowSmem<D, NPTS>*>(
       (reinterpret_cast<uintptr_t>(tail) + sizeof(LayerSmemTail) + 15) & ~uintptr_t(15));
 
   const int warp = threadIdx.x >> 5;
@@ -161,7 +167,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
     tail->abort_flag = 0;
     mbar_fence_init();
   }
-  row_smem_fill<NPTS>(rsm, a.search.table, a.grid4);
+  row_smem_fill<NPTS>(&rsm->tables, a.search.table, a.grid4);
   if (warp == 1) {
     tmem_alloc(&tail->tmem_base, kTmemCols);
     tmem_relinquish();
@@ -327,29 +333,51 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       if (warp == 2 && lane == 0) atomicAdd(a.gemm_done + j * a.mw + ml, 1);
     }
   } else {
-    // ------------------------------- row warps ------------------------------------------------
+    // ------------------------------- row warps (teams of TEAM warps per row) -------------------
+    constexpr int TEAM = RowTeam<D>::TEAM, TEAMS = kRowWarps / TEAM;
     const int rw = warp - 6;
-    RowCtx rck, rcv;
-    rck.lane = rcv.lane = lane;
+    const int team = rw / TEAM;
+    RowCtx rck;
+    rck.lane = lane;
     rck.signmask = a.signmask_k[lane];
+    rck.inv_w = a.search.inv_w;
+    rck.log_h = a.log_h;
+    rck.log_g = a.log_g;
+    rck.member = rw % TEAM;
+    rck.barrier = 3 + team;
+    RowCtx rcv = rck;
     rcv.signmask = a.signmask_v[lane];
-    rck.inv_w = rcv.inv_w = a.search.inv_w;
-    rck.log_h = rcv.log_h = a.log_h;
-    rck.log_g = rcv.log_g = a.log_g;
+    TeamSmem<D>* ts = &rsm->team[team];
     const int n_groups = D >> a.log_g;
     for (int j = 0; j < n_jobs; ++j) {
       int ph, wave;
       layer_job(j, a.n_waves, ph, wave);
       const int m = wave * a.mw + ml;
       if (m >= a.n_mblocks) continue;
+      if constexpr (kEncode) {
+        // pull this job's input rows towards L2 while the prediction is still being produced
+        const uint16_t* xin = ph == 0 ? a.K : a.V;
+        for (int r = n_blk * RJ + team; r < (n_blk + 1) * RJ; r += TEAMS) {
+          const long long g = (long long)m * kBM + r;
+          if (g < a.T && lane < D / 256 / TEAM * 4)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(xin + g * a.ldX + rck.member * (D / TEAM) + lane * 64));
+        }
+      }
       bool ok = true;
       if (lane == 0) ok = counter_wait_bounded(a.gemm_done + j * a.mw + ml, NTN, abort_flag, a.status);
       ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (TEAM == 2) {
+        // both warps of a team must take the same path: agree through shared memory
+        if (!ok) *abort_flag = 1;
+        team_barrier(rck.barrier);
+        ok = *abort_flag == 0;
+        team_barrier(rck.barrier);
+      }
       if (ok) {
         const float* pbuf = a.P + (size_t(j % a.nb) * a.mw * kBM + size_t(ml) * kBM) * D;
         const size_t khat_base = a.khat_ring ? size_t((wave % a.khat_ring) * a.mw + ml) * kBM
                                              : size_t(m) * kBM;
-        for (int r = n_blk * RJ + rw; r < (n_blk + 1) * RJ; r += kRowWarps) {
+        for (int r = n_blk * RJ + team; r < (n_blk + 1) * RJ; r += TEAMS) {
           const long long g = (long long)m * kBM + r;
           if (g >= a.T) break;
           const float* pred_row = pbuf + size_t(r) * D;
@@ -360,10 +388,11 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
           uint16_t* scales_row = (ph == 0 ? a.Kscales : a.Vscales) + g * n_groups;
           if constexpr (kEncode) {
             const uint16_t* x_row = (ph == 0 ? a.K : a.V) + g * a.ldX;
-            encode_row<D, NPTS, kBf16>(ph == 0 ? rck : rcv, rsm, x_row, pred_row, codes_row, scales_row,
-                                       hat_row);
+            encode_row<D, NPTS, kBf16>(ph == 0 ? rck : rcv, &rsm->tables, ts, x_row, pred_row, codes_row,
+                                       scales_row, hat_row);
           } else {
-            decode_row<D, NPTS, kBf16>(ph == 0 ? rck : rcv, rsm->grid, codes_row, scales_row, pred_row, hat_row);
+            decode_row<D, NPTS, kBf16>(ph == 0 ? rck : rcv, rsm->tables.grid, ts, codes_row, scales_row,
+                                       pred_row, hat_row);
           }
         }
       }
