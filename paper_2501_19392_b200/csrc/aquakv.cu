@@ -394,14 +394,14 @@ LayerWs layer_ws(const aquakv_ctx* c, int64_t T) {
 template <bool ENC, int D, int NPTS, bool BF>
 int launch_layer_t(cudaStream_t st, int grid, const CUtensorMap* tm, const LayerArgs& a) {
   static bool attr_set = false;   // per instantiation; contexts are used from one thread at a time
-  constexpr size_t smem = layer_smem_bytes<D, NPTS>();
+  constexpr size_t smem = layer_smem_bytes<ENC, D, NPTS>();
   if (!attr_set) {
     if (cudaFuncSetAttribute(layer_kernel<ENC, D, NPTS, BF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              int(smem)) != cudaSuccess)
       return AQUAKV_ERR_CUDA;
     attr_set = true;
   }
-  layer_kernel<ENC, D, NPTS, BF><<<grid, kLayerThreads, smem, st>>>(tm[0], tm[1], tm[2], tm[3], tm[4], a);
+  layer_kernel<ENC, D, NPTS, BF><<<grid, kLayerThreads, smem, st>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], a);
   return AQUAKV_OK;
 }
 template <int D, int NPTS, bool BF>
@@ -411,6 +411,13 @@ void launch_layer_enc_t(int* rc, cudaStream_t st, int grid, const CUtensorMap* t
 template <int D, int NPTS, bool BF>
 void launch_layer_dec_t(int* rc, cudaStream_t st, int grid, const CUtensorMap* tm, const LayerArgs& a) {
   *rc = launch_layer_t<false, D, NPTS, BF>(st, grid, tm, a);
+}
+
+// The fused kernel needs its whole shared-memory budget in one CTA; the largest grid (256 points)
+// does not fit next to the encoder's search table, so that combination uses the separate GEMM and
+// row kernels instead.
+bool layer_kernel_fits(const aquakv_ctx* c, bool encode) {
+  return !(encode && c->p.grid_size == 256);
 }
 
 // Algorithm 2 (encode = true) or Algorithm 3 for one layer with predictors, all tokens, one launch.
@@ -461,7 +468,18 @@ int launch_layer(aquakv_ctx* c, cudaStream_t st, bool encode, int64_t T, const v
   a.log_g = c->log_g;
   a.status = c->d_status;
 
-  CUtensorMap tm[5];
+  CUtensorMap tm[6];
+  {
+    // the prediction ring as a 2-D fp32 tensor for the epilogue's TMA stores (32 x 32 boxes)
+    const cuuint64_t dims[2] = {cuuint64_t(d), cuuint64_t(kLayerRing) * ws.mw * kBM};
+    const cuuint64_t strides[1] = {cuuint64_t(d) * sizeof(float)};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    if (c->encode_tiled(&tm[5], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, a.P, dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return AQUAKV_ERR_CUDA;
+  }
   int rc = make_tmap(c, &tm[0], Khat_prev, uint64_t(T), uint64_t(d), uint64_t(ld_prev), kBM);
   if (rc) return rc;
   if ((rc = make_tmap(c, &tm[1], Vhat_prev, uint64_t(T), uint64_t(d), uint64_t(ld_prev), kBM))) return rc;
@@ -818,6 +836,8 @@ int aquakv_encode(aquakv_ctx* c, int64_t n_tokens, const void* K, const void* V,
     if (workspace == nullptr || workspace_bytes < aquakv_workspace_bytes(c, n_tokens, AQUAKV_OP_ENCODE))
       return AQUAKV_ERR_WORKSPACE;
     if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
+  }
+  if (has_pred && layer_kernel_fits(c, true)) {
     if (n_tokens > (int64_t(1) << 30)) return AQUAKV_ERR_UNSUPPORTED;
     return launch_layer(c, static_cast<cudaStream_t>(cuda_stream), true, n_tokens, K, V, ld_kv, Khat_prev,
                         Vhat_prev, ld_prev, Wk, Wv, bk, bv, Kcodes, Kscales, Vcodes, Vscales, Khat, Vhat,

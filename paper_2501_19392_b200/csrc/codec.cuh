@@ -72,48 +72,89 @@ struct CodecArgs {
   int log_g;                // log2 of the scale group
 };
 
+// Packed pairs of fp32 values: sm_100 executes add/sub/fma on two fp32 lanes of a 64-bit register
+// pair in one instruction (add.f32x2 / fma.rn.f32x2), each lane rounded exactly like the scalar
+// operation.  The rotation keeps (v[2k], v[2k+1]) packed, which halves its arithmetic instructions.
+typedef unsigned long long f32x2_t;
+__device__ __forceinline__ f32x2_t pack2(float lo, float hi) {
+  f32x2_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2_t p, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
+}
+__device__ __forceinline__ f32x2_t add2(f32x2_t a, f32x2_t b) {
+  f32x2_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ f32x2_t sub2(f32x2_t a, f32x2_t b) {
+  f32x2_t r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ f32x2_t fma2(f32x2_t a, f32x2_t b, f32x2_t c) {
+  f32x2_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ f32x2_t mul2(f32x2_t a, f32x2_t b) {
+  f32x2_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+
+// Hadamard butterflies of one warp's NV values per lane (element index bits 0-2 in registers,
+// 3-7 across lanes, the next bit between the warp's two chunks when NV == 16), by ascending bit.
+// vp[k] holds (v[2k], v[2k+1]).
 template <int NV>
-__device__ __forceinline__ void fwht_regs_and_lanes(float (&v)[NV], int log_h, int lane) {
-  // index bits 0..2: inside each 8-element register chunk (h >= 64, so always applied)
+__device__ __forceinline__ void fwht_packed(f32x2_t (&vp)[NV / 2], int log_h, int lane) {
+  // bit 0: inside each packed pair
 #pragma unroll
-  for (int b = 0; b < 3; ++b) {
+  for (int k = 0; k < NV / 2; ++k) {
+    float a, b;
+    unpack2(vp[k], a, b);
+    vp[k] = pack2(a + b, a - b);
+  }
+  // bits 1, 2: between packed pairs k and k ^ 1, k ^ 2
 #pragma unroll
-    for (int i = 0; i < NV; ++i) {
-      if ((i & (1 << b)) == 0) {
-        const float a = v[i], c = v[i | (1 << b)];
-        v[i] = a + c;
-        v[i | (1 << b)] = a - c;
+  for (int b = 1; b < 3; ++b) {
+    const int m = 1 << (b - 1);
+#pragma unroll
+    for (int k = 0; k < NV / 2; ++k) {
+      if ((k & m) == 0) {
+        const f32x2_t x = vp[k], y = vp[k | m];
+        vp[k] = add2(x, y);
+        vp[k | m] = sub2(x, y);
       }
     }
   }
-  // index bits 3..7: lane bits 0..4
+  // bits 3..7: lane bits 0..4
 #pragma unroll
   for (int b = 3; b < 8; ++b) {
     if (b < log_h) {
       const int m = 1 << (b - 3);
       const float sg = (lane & m) ? -1.0f : 1.0f;
+      const f32x2_t sg2 = pack2(sg, sg);
 #pragma unroll
-      for (int i = 0; i < NV; ++i) {
-        const float o = __shfl_xor_sync(0xffffffffu, v[i], m);
-        v[i] = fmaf(sg, v[i], o);   // lower partner: v + o; upper partner: o - v (both exact adds)
+      for (int k = 0; k < NV / 2; ++k) {
+        float a, c;
+        unpack2(vp[k], a, c);
+        const float oa = __shfl_xor_sync(0xffffffffu, a, m);
+        const float oc = __shfl_xor_sync(0xffffffffu, c, m);
+        vp[k] = fma2(sg2, vp[k], pack2(oa, oc));   // lower partner: v + o; upper partner: o - v
       }
     }
   }
-  // index bits 8..9: register chunk index
+  // bit 8: between the two chunks of a 16-value warp
+  if constexpr (NV == 16) {
+    if (8 < log_h) {
 #pragma unroll
-  for (int b = 8; b < 10; ++b) {
-    if ((NV >> 3) > (1 << (b - 8)) && b < log_h) {
-      const int cm = 1 << (b - 8);
-#pragma unroll
-      for (int i = 0; i < NV; ++i) {
-        if (((i >> 3) & cm) == 0) {
-          const int j = i + (cm << 3);
-          if (j < NV) {
-            const float a = v[i], c = v[j];
-            v[i] = a + c;
-            v[j] = a - c;
-          }
-        }
+      for (int k = 0; k < 4; ++k) {
+        const f32x2_t x = vp[k], y = vp[k + 4];
+        vp[k] = add2(x, y);
+        vp[k + 4] = sub2(x, y);
       }
     }
   }
@@ -211,19 +252,36 @@ struct RowTeam {
 // Exchange buffer of one team (only used when TEAM == 2).
 template <int D>
 struct TeamSmem {
-  float4 x[2][RowTeam<D>::CPM * 2][32];   // [member][16-byte piece][lane]
+  ulonglong2 x[2][RowTeam<D>::CPM * 2][32];   // [member][16-byte piece][lane]
   float ss[2][2];                         // [member][chunk] sums of squares
 };
 
 // Per-warp constants of the row routines.
 struct RowCtx {
-  uint32_t signmask;       // this lane's entry of CodecArgs::signmask
+  uint32_t signmask;       // this lane's sign bits for this warp's values: bit i <=> value i is flipped
   float inv_w;             // SearchDev::inv_w
+  float inv_g;             // 1 / scale group
+  float rs;                // 1 / sqrt(Hadamard block)
   int log_h, log_g;
   int lane;
   int member;              // 0 or 1: which half of the row this warp holds
   int barrier;             // named barrier shared by the two warps of the team
 };
+
+// Fills the fields that depend only on the parameters and on the warp's place in its team.
+__device__ __forceinline__ void row_ctx_init(RowCtx& rc, const uint32_t* signmask, float inv_w, int log_h,
+                                             int log_g, int lane, int member, int values_per_warp,
+                                             int barrier) {
+  rc.lane = lane;
+  rc.member = member;
+  rc.barrier = barrier;
+  rc.signmask = signmask[lane] >> (member * values_per_warp);
+  rc.inv_w = inv_w;
+  rc.log_h = log_h;
+  rc.log_g = log_g;
+  rc.inv_g = __int_as_float((127 - log_g) << 23);                       // 2^-log_g, exact
+  rc.rs = __int_as_float((127 - (log_h >> 1)) << 23) * ((log_h & 1) ? 0.70710678118654752f : 1.0f);
+}
 
 __device__ __forceinline__ void team_barrier(int id) {
   asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory");
@@ -232,14 +290,15 @@ __device__ __forceinline__ void team_barrier(int id) {
 // Publishes this warp's values (and optionally its chunk sums) and reads the partner's.
 template <int D, bool kWithSums>
 __device__ __forceinline__ void team_exchange(const RowCtx& rc, TeamSmem<D>* ts,
-                                              const float (&v)[RowTeam<D>::NV], float (&o)[RowTeam<D>::NV],
+                                              const f32x2_t (&vp)[RowTeam<D>::NV / 2],
+                                              f32x2_t (&op)[RowTeam<D>::NV / 2],
                                               const float (&ss)[RowTeam<D>::CPM],
                                               float (&oss)[RowTeam<D>::CPM]) {
   constexpr int NV = RowTeam<D>::NV, CPM = RowTeam<D>::CPM;
   team_barrier(rc.barrier);                // the partner has finished reading the previous exchange
 #pragma unroll
   for (int q = 0; q < NV / 4; ++q)
-    ts->x[rc.member][q][rc.lane] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+    ts->x[rc.member][q][rc.lane] = make_ulonglong2(vp[2 * q], vp[2 * q + 1]);
   if (kWithSums && rc.lane == 0) {
 #pragma unroll
     for (int c = 0; c < CPM; ++c) ts->ss[rc.member][c] = ss[c];
@@ -247,8 +306,9 @@ __device__ __forceinline__ void team_exchange(const RowCtx& rc, TeamSmem<D>* ts,
   team_barrier(rc.barrier);
 #pragma unroll
   for (int q = 0; q < NV / 4; ++q) {
-    const float4 t = ts->x[rc.member ^ 1][q][rc.lane];
-    o[4 * q] = t.x; o[4 * q + 1] = t.y; o[4 * q + 2] = t.z; o[4 * q + 3] = t.w;
+    const ulonglong2 t = ts->x[rc.member ^ 1][q][rc.lane];
+    op[2 * q] = t.x;
+    op[2 * q + 1] = t.y;
   }
   if (kWithSums) {
 #pragma unroll
@@ -258,10 +318,12 @@ __device__ __forceinline__ void team_exchange(const RowCtx& rc, TeamSmem<D>* ts,
 
 // Butterfly over the index bit that separates the two warps: the lower half keeps a + b, the upper
 // half a - b (a = lower half's value, b = upper half's).
-template <int NV>
-__device__ __forceinline__ void cross_butterfly(float (&v)[NV], const float (&o)[NV], int member) {
+template <int NP>
+__device__ __forceinline__ void cross_butterfly(f32x2_t (&vp)[NP], const f32x2_t (&op)[NP], int member) {
+  const float sg = member ? -1.0f : 1.0f;
+  const f32x2_t sg2 = pack2(sg, sg);
 #pragma unroll
-  for (int i = 0; i < NV; ++i) v[i] = member == 0 ? __fadd_rn(v[i], o[i]) : __fsub_rn(o[i], v[i]);
+  for (int k = 0; k < NP; ++k) vp[k] = fma2(sg2, vp[k], op[k]);
 }
 
 // Q^-1 without the prediction for this warp's part of the row: `w` enters holding the gathered grid
@@ -273,19 +335,27 @@ __device__ __forceinline__ void team_rotate_back_and_scale(const RowCtx& rc, Tea
                                                            float (&w)[RowTeam<D>::NV],
                                                            const float (&sf)[RowTeam<D>::CPM]) {
   using RT = RowTeam<D>;
-  fwht_regs_and_lanes<RT::NV>(w, rc.log_h, rc.lane);
+  f32x2_t wp[RT::NV / 2];
+#pragma unroll
+  for (int k = 0; k < RT::NV / 2; ++k) wp[k] = pack2(w[2 * k], w[2 * k + 1]);
+  fwht_packed<RT::NV>(wp, rc.log_h, rc.lane);
   if constexpr (RT::TEAM == 2) {
     if (RT::CROSS_BIT < rc.log_h) {
-      float o[RT::NV], dummy_a[RT::CPM] = {}, dummy_b[RT::CPM];
-      team_exchange<D, false>(rc, ts, w, o, dummy_a, dummy_b);
-      cross_butterfly<RT::NV>(w, o, rc.member);
+      f32x2_t op[RT::NV / 2];
+      float dummy_a[RT::CPM] = {}, dummy_b[RT::CPM];
+      team_exchange<D, false>(rc, ts, wp, op, dummy_a, dummy_b);
+      cross_butterfly<RT::NV / 2>(wp, op, rc.member);
     }
   }
-  const float rs = exp2f(-0.5f * static_cast<float>(rc.log_h));   // exact for even log_h
+  const f32x2_t rs2 = pack2(rc.rs, rc.rs);
 #pragma unroll
-  for (int i = 0; i < RT::NV; ++i)
-    w[i] = apply_sign(__fmul_rn(__fmul_rn(w[i], rs), sf[i >> 3]), rc.signmask,
-                      rc.member * RT::NV + i);
+  for (int k = 0; k < RT::NV / 2; ++k) {
+    const float s = sf[(2 * k) >> 3];
+    float a, b;
+    unpack2(mul2(mul2(wp[k], rs2), pack2(s, s)), a, b);
+    w[2 * k] = apply_sign(a, rc.signmask, 2 * k);
+    w[2 * k + 1] = apply_sign(b, rc.signmask, 2 * k + 1);
+  }
 }
 
 // This warp's part of one token row of Q and of the reconstruction (Algorithm 2 lines 6-7 / 9):
@@ -295,51 +365,37 @@ __device__ __forceinline__ void team_rotate_back_and_scale(const RowCtx& rc, Tea
 // again for the reconstruction) instead of being held in registers across the rotation and the
 // search; both reads bypass L1 (ld.global.cg) because the prediction may have been written by
 // another SM of the same kernel just before.  Both warps of a team must call this together.
-template <int D, int NPTS, bool kBf16>
-__device__ __forceinline__ void encode_row(const RowCtx& rc, const RowSmem<NPTS>* __restrict__ rsm,
-                                           TeamSmem<D>* ts, const uint16_t* __restrict__ x_row,
-                                           const float* __restrict__ pred_row,
-                                           uint8_t* __restrict__ codes_row,
-                                           uint16_t* __restrict__ scales_row,
-                                           uint16_t* __restrict__ hat_row) {
+template <int D, int NPTS, bool kBf16, typename AfterLoad>
+__device__ __forceinline__ void encode_row_core(const RowCtx& rc, const RowSmem<NPTS>* __restrict__ rsm,
+                                                TeamSmem<D>* ts, const uint4 (&raw)[RowTeam<D>::CPM],
+                                                const float4 (&pq0)[RowTeam<D>::CPM][2],
+                                                const float* __restrict__ pred_row,
+                                                uint8_t* __restrict__ codes_row,
+                                                uint16_t* __restrict__ scales_row,
+                                                uint16_t* __restrict__ hat_row, AfterLoad after_load) {
   using RT = RowTeam<D>;
   constexpr int NC = RT::NC, CPM = RT::CPM, NV = RT::NV;
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
   const int lane = rc.lane;
   const int c0 = rc.member * CPM;                    // first chunk of this warp
-  const float inv_g = exp2f(-static_cast<float>(rc.log_g));
-  const float rs = exp2f(-0.5f * static_cast<float>(rc.log_h));
   float v[NV];
-  // ---- residual r = x - pred -------------------------------------------------------------------
-  {
-    uint4 raw[CPM];
+  // ---- residual r = x - pred (raw = this lane's 16-bit inputs, pq0 = its prediction values) -----
 #pragma unroll
-    for (int c = 0; c < CPM; ++c)
-      raw[c] = *reinterpret_cast<const uint4*>(x_row + (c0 + c) * 256 + lane * 8);
-    float4 pq[CPM][2];
-    if (pred_row != nullptr) {
+  for (int c = 0; c < CPM; ++c) {
+    const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
 #pragma unroll
-      for (int c = 0; c < CPM; ++c) {
-        pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + lane * 8));
-        pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + lane * 8 + 4));
-      }
+    for (int i = 0; i < 4; ++i) {
+      v[c * 8 + 2 * i] = load16<kBf16>(uint16_t(w[i] & 0xffffu));
+      v[c * 8 + 2 * i + 1] = load16<kBf16>(uint16_t(w[i] >> 16));
     }
+    if (pred_row != nullptr) {
+      const float pp[8] = {pq0[c][0].x, pq0[c][0].y, pq0[c][0].z, pq0[c][0].w,
+                           pq0[c][1].x, pq0[c][1].y, pq0[c][1].z, pq0[c][1].w};
 #pragma unroll
-    for (int c = 0; c < CPM; ++c) {
-      const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        v[c * 8 + 2 * i] = load16<kBf16>(uint16_t(w[i] & 0xffffu));
-        v[c * 8 + 2 * i + 1] = load16<kBf16>(uint16_t(w[i] >> 16));
-      }
-      if (pred_row != nullptr) {
-        const float pp[8] = {pq[c][0].x, pq[c][0].y, pq[c][0].z, pq[c][0].w,
-                             pq[c][1].x, pq[c][1].y, pq[c][1].z, pq[c][1].w};
-#pragma unroll
-        for (int i = 0; i < 8; ++i) v[c * 8 + i] = __fsub_rn(v[c * 8 + i], pp[i]);
-      }
+      for (int i = 0; i < 8; ++i) v[c * 8 + i] = __fsub_rn(v[c * 8 + i], pp[i]);
     }
   }
+  after_load();   // raw and pq0 are consumed: the caller may start fetching the next row's inputs
   // ---- per-chunk sums of squares (lane bits reduced by shuffles), sign flip ---------------------
   float ss[CPM];
 #pragma unroll
@@ -352,18 +408,22 @@ __device__ __forceinline__ void encode_row(const RowCtx& rc, const RowSmem<NPTS>
       if (b < rc.log_g) s += __shfl_xor_sync(0xffffffffu, s, 1 << (b - 3));
     ss[c] = s;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[c * 8 + i] = apply_sign(v[c * 8 + i], rc.signmask, (c0 + c) * 8 + i);
+    for (int i = 0; i < 8; ++i) v[c * 8 + i] = apply_sign(v[c * 8 + i], rc.signmask, c * 8 + i);
   }
   // ---- rotate (the division by the scale is applied afterwards: the rotation is linear) ---------
-  fwht_regs_and_lanes<NV>(v, rc.log_h, lane);
+  f32x2_t vp[NV / 2];
+#pragma unroll
+  for (int k = 0; k < NV / 2; ++k) vp[k] = pack2(v[2 * k], v[2 * k + 1]);
+  fwht_packed<NV>(vp, rc.log_h, lane);
   float all_ss[NC];
 #pragma unroll
   for (int c = 0; c < NC; ++c) all_ss[c] = 0.0f;
   if constexpr (RT::TEAM == 2) {
     if (RT::CROSS_BIT < rc.log_g) {          // scale groups (and maybe Hadamard blocks) span both warps
-      float o[NV], oss[CPM];
-      team_exchange<D, true>(rc, ts, v, o, ss, oss);
-      if (RT::CROSS_BIT < rc.log_h) cross_butterfly<NV>(v, o, rc.member);
+      f32x2_t op[NV / 2];
+      float oss[CPM];
+      team_exchange<D, true>(rc, ts, vp, op, ss, oss);
+      if (RT::CROSS_BIT < rc.log_h) cross_butterfly<NV / 2>(vp, op, rc.member);
 #pragma unroll
       for (int c = 0; c < CPM; ++c) {
         all_ss[c0 + c] = ss[c];
@@ -389,7 +449,7 @@ __device__ __forceinline__ void encode_row(const RowCtx& rc, const RowSmem<NPTS>
       for (int c2 = 0; c2 < NC; ++c2)
         if ((c2 / cpg) == ((c0 + c) / cpg)) tot += all_ss[c2];
     }
-    const float sc = fminf(sqrtf(tot * inv_g), 65504.0f);
+    const float sc = fminf(sqrtf(tot * rc.inv_g), 65504.0f);
     const __half s16 = __float2half_rn(sc);
     sf[c] = __half2float(s16);
     const int cg = c0 + c;
@@ -400,9 +460,22 @@ __device__ __forceinline__ void encode_row(const RowCtx& rc, const RowSmem<NPTS>
       const int lpg = 1 << (rc.log_g - 3);   // lanes per group
       if ((lane % lpg) == 0) scales_row[cg * (256 >> rc.log_g) + lane / lpg] = __half_as_ushort(s16);
     }
-    const float inv = (sf[c] > 0.0f ? 1.0f / sf[c] : 0.0f) * rs;
+    const float inv = (sf[c] > 0.0f ? __frcp_rn(sf[c]) : 0.0f) * rc.rs;
+    const f32x2_t inv2 = pack2(inv, inv);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[c * 8 + i] *= inv;
+    for (int k = 0; k < 4; ++k) unpack2(mul2(vp[c * 4 + k], inv2), v[c * 8 + 2 * k], v[c * 8 + 2 * k + 1]);
+  }
+  // the prediction is needed again for the reconstruction: start reading it now, the search hides it
+  float4 pq[CPM][2];
+  if (hat_row != nullptr && pred_row != nullptr) {
+#pragma unroll
+    for (int c = 0; c < CPM; ++c) {
+      pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + lane * 8));
+      pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + lane * 8 + 4));
+    }
+  } else {
+#pragma unroll
+    for (int c = 0; c < CPM; ++c) pq[c][0] = pq[c][1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
   }
   // ---- nearest grid point per pair: all table entries first, then the candidates ----------------
   uint32_t entry[NV / 2];
@@ -436,17 +509,6 @@ __device__ __forceinline__ void encode_row(const RowCtx& rc, const RowSmem<NPTS>
   }
   // ---- reconstruction: hat = round16(pred + Q^-1(codes)) ---------------------------------------
   if (hat_row != nullptr) {      // uniform over the team
-    float4 pq[CPM][2];
-    if (pred_row != nullptr) {
-#pragma unroll
-      for (int c = 0; c < CPM; ++c) {
-        pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + lane * 8));
-        pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + lane * 8 + 4));
-      }
-    } else {
-#pragma unroll
-      for (int c = 0; c < CPM; ++c) pq[c][0] = pq[c][1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-    }
     team_rotate_back_and_scale<D>(rc, ts, v, sf);
 #pragma unroll
     for (int c = 0; c < CPM; ++c) {
@@ -454,14 +516,36 @@ __device__ __forceinline__ void encode_row(const RowCtx& rc, const RowSmem<NPTS>
                            pq[c][1].x, pq[c][1].y, pq[c][1].z, pq[c][1].w};
       uint32_t o[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint32_t lo = store16<kBf16>(__fadd_rn(pp[2 * i], v[c * 8 + 2 * i]));
-        const uint32_t hi = store16<kBf16>(__fadd_rn(pp[2 * i + 1], v[c * 8 + 2 * i + 1]));
-        o[i] = lo | (hi << 16);
-      }
+      for (int i = 0; i < 4; ++i)
+        o[i] = store16x2<kBf16>(__fadd_rn(pp[2 * i], v[c * 8 + 2 * i]), __fadd_rn(pp[2 * i + 1], v[c * 8 + 2 * i + 1]));
       *reinterpret_cast<uint4*>(hat_row + (c0 + c) * 256 + lane * 8) = make_uint4(o[0], o[1], o[2], o[3]);
     }
   }
+}
+
+// encode_row_core with the row's inputs read straight from global memory.
+template <int D, int NPTS, bool kBf16>
+__device__ __forceinline__ void encode_row(const RowCtx& rc, const RowSmem<NPTS>* __restrict__ rsm,
+                                           TeamSmem<D>* ts, const uint16_t* __restrict__ x_row,
+                                           const float* __restrict__ pred_row,
+                                           uint8_t* __restrict__ codes_row,
+                                           uint16_t* __restrict__ scales_row,
+                                           uint16_t* __restrict__ hat_row) {
+  constexpr int CPM = RowTeam<D>::CPM;
+  const int c0 = rc.member * CPM;
+  uint4 raw[CPM];
+  float4 pq[CPM][2];
+#pragma unroll
+  for (int c = 0; c < CPM; ++c) {
+    raw[c] = *reinterpret_cast<const uint4*>(x_row + (c0 + c) * 256 + rc.lane * 8);
+    if (pred_row != nullptr) {
+      pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + rc.lane * 8));
+      pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + rc.lane * 8 + 4));
+    } else {
+      pq[c][0] = pq[c][1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    }
+  }
+  encode_row_core<D, NPTS, kBf16>(rc, rsm, ts, raw, pq, pred_row, codes_row, scales_row, hat_row, [] {});
 }
 
 // Shared memory of the stand-alone row kernels: search tables plus one exchange buffer per team.
@@ -471,16 +555,12 @@ struct RowKernelSmem {
   TeamSmem<D> team[kCodecWarps / RowTeam<D>::TEAM];
 };
 
-__device__ __forceinline__ RowCtx make_row_ctx(const CodecArgs& a, int team_size, int first_barrier) {
+__device__ __forceinline__ RowCtx make_row_ctx(const CodecArgs& a, int team_size, int values_per_warp,
+                                               int first_barrier) {
   RowCtx rc;
   const int warp = threadIdx.x >> 5;
-  rc.lane = threadIdx.x & 31;
-  rc.signmask = a.signmask[rc.lane];
-  rc.inv_w = a.search.inv_w;
-  rc.log_h = a.log_h;
-  rc.log_g = a.log_g;
-  rc.member = warp % team_size;
-  rc.barrier = first_barrier + warp / team_size;
+  row_ctx_init(rc, a.signmask, a.search.inv_w, a.log_h, a.log_g, threadIdx.x & 31, warp % team_size,
+               values_per_warp, first_barrier + warp / team_size);
   return rc;
 }
 
@@ -492,7 +572,7 @@ __global__ void __launch_bounds__(kCodecThreads, 2) encode_rows_kernel(const Cod
   __shared__ RowKernelSmem<D, NPTS> sm;
   row_smem_fill<NPTS>(&sm.tables, a.search.table, a.grid4);
   __syncthreads();
-  const RowCtx rc = make_row_ctx(a, TEAM, 1);
+  const RowCtx rc = make_row_ctx(a, TEAM, RowTeam<D>::NV, 1);
   const int team = (threadIdx.x >> 5) / TEAM;
   const int n_groups = D >> a.log_g;
   for (long long row = (long long)blockIdx.x * TEAMS + team; row < a.T; row += (long long)gridDim.x * TEAMS) {
@@ -504,56 +584,89 @@ __global__ void __launch_bounds__(kCodecThreads, 2) encode_rows_kernel(const Cod
 }
 
 // This warp's part of one token row of Algorithm 3 line 5 / 7 given the prediction:
-//   hat = round16(pred + Q^-1(codes, scales)).  pred_row == nullptr: no predictor.
-template <int D, int NPTS, bool kBf16>
-__device__ __forceinline__ void decode_row(const RowCtx& rc, const float2* __restrict__ grid_s,
-                                           TeamSmem<D>* ts, const uint8_t* __restrict__ codes_row,
-                                           const uint16_t* __restrict__ scales_row,
-                                           const float* __restrict__ pred_row,
-                                           uint16_t* __restrict__ hat_row) {
+//   hat = round16(pred + Q^-1(codes, scales)).  words = this lane's packed codes per chunk, sf = the
+// scale of each chunk; get_pred(pq) delivers the prediction values of this lane just before they are
+// added, so a caller can fetch them while the rotation runs.
+template <int D, int NPTS, bool kBf16, typename GetPred>
+__device__ __forceinline__ void decode_row_core(const RowCtx& rc, const float2* __restrict__ grid_s,
+                                                TeamSmem<D>* ts, const uint32_t (&words)[RowTeam<D>::CPM],
+                                                const float (&sf)[RowTeam<D>::CPM], GetPred get_pred,
+                                                uint16_t* __restrict__ hat_row) {
   using RT = RowTeam<D>;
   constexpr int CPM = RT::CPM, NV = RT::NV;
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
   const int lane = rc.lane;
   const int c0 = rc.member * CPM;
-  float w[NV], sf[CPM];
-  float4 pq[CPM][2];
-  if (pred_row != nullptr) {
-#pragma unroll
-    for (int c = 0; c < CPM; ++c) {
-      pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + lane * 8));
-      pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + lane * 8 + 4));
-    }
-  } else {
-#pragma unroll
-    for (int c = 0; c < CPM; ++c) pq[c][0] = pq[c][1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-  }
+  float w[NV];
 #pragma unroll
   for (int c = 0; c < CPM; ++c) {
-    const uint32_t word = load_code_word<BITS>(codes_row, c0 + c, lane);
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      const float2 g = grid_s[(word >> (k * BITS)) & (NPTS - 1)];
+      const float2 g = grid_s[(words[c] >> (k * BITS)) & (NPTS - 1)];
       w[c * 8 + 2 * k] = g.x;
       w[c * 8 + 2 * k + 1] = g.y;
     }
-    const int e0 = (c0 + c) * 256 + lane * 8;
-    sf[c] = __half2float(__ushort_as_half(scales_row[e0 >> rc.log_g]));
   }
   team_rotate_back_and_scale<D>(rc, ts, w, sf);
+  float4 pq[CPM][2];
+  get_pred(pq);     // the prediction values of this lane (zeros without a predictor)
 #pragma unroll
   for (int c = 0; c < CPM; ++c) {
     const float pp[8] = {pq[c][0].x, pq[c][0].y, pq[c][0].z, pq[c][0].w,
                          pq[c][1].x, pq[c][1].y, pq[c][1].z, pq[c][1].w};
     uint32_t o[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const uint32_t lo = store16<kBf16>(__fadd_rn(pp[2 * i], w[c * 8 + 2 * i]));
-      const uint32_t hi = store16<kBf16>(__fadd_rn(pp[2 * i + 1], w[c * 8 + 2 * i + 1]));
-      o[i] = lo | (hi << 16);
-    }
+    for (int i = 0; i < 4; ++i)
+      o[i] = store16x2<kBf16>(__fadd_rn(pp[2 * i], w[c * 8 + 2 * i]), __fadd_rn(pp[2 * i + 1], w[c * 8 + 2 * i + 1]));
     *reinterpret_cast<uint4*>(hat_row + (c0 + c) * 256 + lane * 8) = make_uint4(o[0], o[1], o[2], o[3]);
   }
+}
+
+// This lane's codes and scales of one row (the small inputs of decode_row_core).
+template <int D, int NPTS>
+__device__ __forceinline__ void decode_row_load_codes(const RowCtx& rc, const uint8_t* __restrict__ codes_row,
+                                                      const uint16_t* __restrict__ scales_row,
+                                                      uint32_t (&words)[RowTeam<D>::CPM],
+                                                      float (&sf)[RowTeam<D>::CPM]) {
+  constexpr int CPM = RowTeam<D>::CPM;
+  constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
+  const int c0 = rc.member * CPM;
+#pragma unroll
+  for (int c = 0; c < CPM; ++c) {
+    words[c] = load_code_word<BITS>(codes_row, c0 + c, rc.lane);
+    const int e0 = (c0 + c) * 256 + rc.lane * 8;
+    sf[c] = __half2float(__ushort_as_half(scales_row[e0 >> rc.log_g]));
+  }
+}
+
+// decode_row_core with the row's inputs read straight from global memory.
+template <int D, int NPTS, bool kBf16>
+__device__ __forceinline__ void decode_row(const RowCtx& rc, const float2* __restrict__ grid_s,
+                                           TeamSmem<D>* ts, const uint8_t* __restrict__ codes_row,
+                                           const uint16_t* __restrict__ scales_row,
+                                           const float* __restrict__ pred_row,
+                                           uint16_t* __restrict__ hat_row) {
+  constexpr int CPM = RowTeam<D>::CPM;
+  const int c0 = rc.member * CPM;
+  float4 pq[CPM][2];
+#pragma unroll
+  for (int c = 0; c < CPM; ++c) {
+    if (pred_row != nullptr) {
+      pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + rc.lane * 8));
+      pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + rc.lane * 8 + 4));
+    } else {
+      pq[c][0] = pq[c][1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    }
+  }
+  uint32_t words[CPM];
+  float sf[CPM];
+  decode_row_load_codes<D, NPTS>(rc, codes_row, scales_row, words, sf);
+  decode_row_core<D, NPTS, kBf16>(rc, grid_s, ts, words, sf,
+                                  [&](float4 (&out)[CPM][2]) {
+#pragma unroll
+                                    for (int c = 0; c < CPM; ++c) { out[c][0] = pq[c][0]; out[c][1] = pq[c][1]; }
+                                  },
+                                  hat_row);
 }
 
 template <int D, int NPTS, bool kBf16>
@@ -568,7 +681,7 @@ __global__ void __launch_bounds__(kCodecThreads, 2) decode_rows_kernel(const Cod
     grid_s[i] = make_float2(g.x, g.y);
   }
   __syncthreads();
-  const RowCtx rc = make_row_ctx(a, TEAM, 1);
+  const RowCtx rc = make_row_ctx(a, TEAM, RowTeam<D>::NV, 1);
   const int team = (threadIdx.x >> 5) / TEAM;
   const int n_groups = D >> a.log_g;
   for (long long row = (long long)blockIdx.x * TEAMS + team; row < a.T; row += (long long)gridDim.x * TEAMS) {

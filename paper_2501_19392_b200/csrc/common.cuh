@@ -196,4 +196,16 @@ __device__ __forceinline__ uint16_t store16(float x) {   // round to nearest eve
   }
 }
 
+// Two values rounded to nearest even and packed: `lo` in bits 0..15, `hi` in bits 16..31.
+template <bool kBf16>
+__device__ __forceinline__ uint32_t store16x2(float lo, float hi) {
+  if constexpr (kBf16) {
+    const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&p);
+  } else {
+    const __half2 p = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&p);
+  }
+}
+
 }  // namespace aquakv

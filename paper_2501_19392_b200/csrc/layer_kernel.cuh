@@ -46,15 +46,42 @@ struct LayerSmemTail {
   int abort_flag;
 };
 
-template <int D, int NPTS>
+// Grid only (decode needs no search table).
+template <int NPTS>
+struct GridSmem {
+  float2 grid[NPTS];
+};
+template <bool kEncode, int NPTS> struct LayerTables { typedef RowSmem<NPTS> type; };
+template <int NPTS> struct LayerTables<false, NPTS> { typedef GridSmem<NPTS> type; };
+
+template <bool kEncode, int D, int NPTS>
 struct LayerRowSmem {
-  RowSmem<NPTS> tables;
+  typename LayerTables<kEncode, NPTS>::type tables;
   TeamSmem<D> team[kRowWarps / RowTeam<D>::TEAM];
 };
 
-template <int D, int NPTS>
+// The GEMM epilogue stages each 32-row x 32-column fp32 piece of a tile in shared memory (128-byte
+// swizzle) and hands it to a TMA store: two 4 KB buffers per epilogue warp.
+constexpr int kEpiPieceBytes = 32 * 32 * 4;
+constexpr int kEpiBytes = 4 * 2 * kEpiPieceBytes;
+
+template <bool kEncode, int D, int NPTS>
 constexpr size_t layer_smem_bytes() {
-  return 1024 + size_t(kLayerStages) * kStageBytes + sizeof(LayerSmemTail) + 16 + sizeof(LayerRowSmem<D, NPTS>);
+  return 1024 + size_t(kLayerStages) * kStageBytes + kEpiBytes + sizeof(LayerSmemTail) + 16 +
+         sizeof(LayerRowSmem<kEncode, D, NPTS>);
+}
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* smem_src, int32_t x, int32_t y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
+                   reinterpret_cast<uint64_t>(map)),
+               "r"(smem_u32(smem_src)), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
 struct LayerArgs {
@@ -136,7 +163,8 @@ template <bool kEncode, int D, int NPTS, bool kBf16>
 __global__ void __launch_bounds__(kLayerThreads, 1)
 layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant__ CUtensorMap tmVprev,
              const __grid_constant__ CUtensorMap tmKhat, const __grid_constant__ CUtensorMap tmWk,
-             const __grid_constant__ CUtensorMap tmWv, const LayerArgs a) {
+             const __grid_constant__ CUtensorMap tmWv, const __grid_constant__ CUtensorMap tmP,
+             const LayerArgs a) {
   constexpr int NTN = D / kBN;             // feature tiles per token block = CTAs per token block
   constexpr int RJ = kBM / NTN;            // rows of a token block whose row work this CTA does
   constexpr int NKD = D / kBK;             // k-blocks per d_kv input features
@@ -145,8 +173,9 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~uintptr_t(1023));
-  LayerSmemTail* tail = reinterpret_cast<LayerSmemTail*>(smem + size_t(kLayerStages) * kStageBytes);
-  LayerRowSmem<D, NPTS>* rsm = reinterpret_cast<LayerRowSmem<D, NPTS>*>(
+  uint8_t* epi_smem = smem + size_t(kLayerStages) * kStageBytes;      // 1024-byte aligned
+  LayerSmemTail* tail = reinterpret_cast<LayerSmemTail*>(epi_smem + kEpiBytes);
+  LayerRowSmem<kEncode, D, NPTS>* rsm = reinterpret_cast<LayerRowSmem<kEncode, D, NPTS>*>(
       (reinterpret_cast<uintptr_t>(tail) + sizeof(LayerSmemTail) + 15) & ~uintptr_t(15));
 
   const int warp = threadIdx.x >> 5;
@@ -167,7 +196,14 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
     tail->abort_flag = 0;
     mbar_fence_init();
   }
-  row_smem_fill<NPTS>(&rsm->tables, a.search.table, a.grid4);
+  if constexpr (kEncode) {
+    row_smem_fill<NPTS>(&rsm->tables, a.search.table, a.grid4);
+  } else {
+    for (int i = threadIdx.x; i < NPTS; i += blockDim.x) {
+      const float4 g = a.grid4[i];
+      rsm->tables.grid[i] = make_float2(g.x, g.y);
+    }
+  }
   if (warp == 1) {
     tmem_alloc(&tail->tmem_base, kTmemCols);
     tmem_relinquish();
@@ -186,6 +222,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       tma_prefetch_desc(&tmKhat);
       tma_prefetch_desc(&tmWk);
       tma_prefetch_desc(&tmWv);
+      tma_prefetch_desc(&tmP);
       int stage = 0;
       uint32_t phase_bit = 0;
       bool ok = true;
@@ -303,29 +340,45 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       if (ok) ok = mbar_wait_bounded(&tail->acc_full[acc], acc_phase, abort_flag, a.status);
       if (ok) {
         tc_fence_after_sync();
-        const int r = quarter * 32 + lane;
-        const bool valid = m * kBM + r < a.T;
         const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * kBN);
-        float* out = a.P + (size_t(j % a.nb) * a.mw * kBM + size_t(ml) * kBM + r) * D + n_blk * kBN;
+        // ring row of this warp's 32 tokens; rows past the last token are written too (never read)
+        const int ring_row = (j % a.nb) * a.mw * kBM + ml * kBM + quarter * 32;
         const float* bias = ph == 0 ? a.bk : a.bv;
+        uint8_t* my_epi = epi_smem + (warp - 2) * 2 * kEpiPieceBytes;
 #pragma unroll 1
         for (int c = 0; c < kBN / 32; ++c) {
           float v[32];
           tmem_ld_32x32b_x32(taddr + uint32_t(c * 32), v);
-          if (valid) {
-            if (bias != nullptr) {
-              const float* b = bias + n_blk * kBN + c * 32;
+          if (bias != nullptr) {
+            const float* b = bias + n_blk * kBN + c * 32;
 #pragma unroll
-              for (int i = 0; i < 32; ++i) v[i] = __fadd_rn(v[i], __ldg(b + i));
-            }
+            for (int i = 0; i < 32; ++i) v[i] = __fadd_rn(v[i], __ldg(b + i));
+          }
+          uint8_t* buf = my_epi + (c & 1) * kEpiPieceBytes;
+          if (c >= 2) {                  // the store that last read this buffer must be done with it
+            if (lane == 0) bulk_wait_read_1();
+            __syncwarp();
+          }
+          // lane = row of the piece; 16-byte chunk q of row r sits at chunk position q ^ (r % 8)
 #pragma unroll
-            for (int i = 0; i < 32; i += 4)
-              __stcg(reinterpret_cast<float4*>(out + c * 32 + i), make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]));
+          for (int q = 0; q < 8; ++q)
+            *reinterpret_cast<float4*>(buf + lane * 128 + ((q ^ (lane & 7)) << 4)) =
+                make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&tmP, buf, n_blk * kBN + c * 32, ring_row);
+            bulk_commit();
           }
         }
         tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&tail->acc_empty[acc]);
+        if (lane == 0) {
+          mbar_arrive(&tail->acc_empty[acc]);
+          bulk_wait_all();               // the tile's rows are written
+          fence_proxy_async_all();
+        }
+        __syncwarp();
       }
       __threadfence();
       named_barrier(1, 128);
@@ -337,16 +390,9 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
     constexpr int TEAM = RowTeam<D>::TEAM, TEAMS = kRowWarps / TEAM;
     const int rw = warp - 6;
     const int team = rw / TEAM;
-    RowCtx rck;
-    rck.lane = lane;
-    rck.signmask = a.signmask_k[lane];
-    rck.inv_w = a.search.inv_w;
-    rck.log_h = a.log_h;
-    rck.log_g = a.log_g;
-    rck.member = rw % TEAM;
-    rck.barrier = 3 + team;
-    RowCtx rcv = rck;
-    rcv.signmask = a.signmask_v[lane];
+    RowCtx rck, rcv;
+    row_ctx_init(rck, a.signmask_k, a.search.inv_w, a.log_h, a.log_g, lane, rw % TEAM, RowTeam<D>::NV, 3 + team);
+    row_ctx_init(rcv, a.signmask_v, a.search.inv_w, a.log_h, a.log_g, lane, rw % TEAM, RowTeam<D>::NV, 3 + team);
     TeamSmem<D>* ts = &rsm->team[team];
     const int n_groups = D >> a.log_g;
     for (int j = 0; j < n_jobs; ++j) {
