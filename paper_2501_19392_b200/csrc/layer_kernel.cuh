@@ -15,7 +15,7 @@
 //
 // Dependencies (all counted per job j and token-block slot ml, targets NTN):
 //   gemm_done[j][ml]  -- feature tiles of job j written to the ring        (row warps wait)
-//   rows_done[j][ml]  -- row slices of job j finished                       (the value-phase TMA
+//   rows_done[j][ml]  -- row teams that finished job j (target NTN x teams per CTA)                      (the value-phase TMA
 //                        producer waits for the key rows of its wave; the GEMM epilogue waits for
 //                        job j - ring size before it overwrites that ring slot)
 // Every job waits only on jobs with a smaller index (or the same index of the other role), so the
@@ -36,6 +36,7 @@ namespace aquakv {
 constexpr int kRowWarps = 16;
 constexpr int kLayerThreads = 32 * (6 + kRowWarps);
 constexpr int kLayerStages = 3;
+template <int D> constexpr int kRowTeamsOf = kRowWarps / RowTeam<D>::TEAM;
 
 struct LayerSmemTail {
   uint64_t full[kLayerStages];
@@ -237,7 +238,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         for (int kb = 0; kb < nk; ++kb) {
           if (ph == 1 && kb == NKD) {
             // the remaining k-blocks read this wave's reconstructed keys, written by row warps
-            if (!counter_wait_bounded(a.rows_done + layer_key_job(wave) * a.mw + ml, NTN, abort_flag,
+            if (!counter_wait_bounded(a.rows_done + layer_key_job(wave) * a.mw + ml, NTN * kRowTeamsOf<D>, abort_flag,
                                       a.status)) {
               ok = false;
               break;
@@ -334,7 +335,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       bool ok = true;
       // the ring slot of this job was last used by job j - nb: its row work must be over
       if (j >= a.nb) {
-        if (lane == 0) ok = counter_wait_bounded(a.rows_done + (j - a.nb) * a.mw + ml, NTN, abort_flag, a.status);
+        if (lane == 0) ok = counter_wait_bounded(a.rows_done + (j - a.nb) * a.mw + ml, NTN * kRowTeamsOf<D>, abort_flag, a.status);
         ok = __shfl_sync(0xffffffffu, ok, 0);
       }
       if (ok) ok = mbar_wait_bounded(&tail->acc_full[acc], acc_phase, abort_flag, a.status);
@@ -442,11 +443,12 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
           }
         }
       }
+      // each team reports on its own, so a slow team never holds the others back
       __threadfence();
       fence_proxy_async_all();
-      named_barrier(2, kRowWarps * 32);
+      if (TEAM == 2) team_barrier(rck.barrier); else __syncwarp();
       if (*abort_flag) break;
-      if (rw == 0 && lane == 0) atomicAdd(a.rows_done + j * a.mw + ml, 1);
+      if (rck.member == 0 && lane == 0) atomicAdd(a.rows_done + j * a.mw + ml, 1);
     }
   }
 
