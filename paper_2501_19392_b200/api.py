@@ -22,7 +22,7 @@ OP_DECODE_ATTN = 2
 ROLE_KEY = 0
 ROLE_VALUE = 1
 NOALLOC_MAX_TOKENS = 1024
-KERNEL_PREDICT, KERNEL_ENCODE_ROWS, KERNEL_DECODE_ROWS, KERNEL_ATTN = 0, 1, 2, 3
+KERNEL_PREDICT, KERNEL_ENCODE_ROWS, KERNEL_DECODE_ROWS, KERNEL_ATTN, KERNEL_LAYER = 0, 1, 2, 3, 4
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libaquakv.so")

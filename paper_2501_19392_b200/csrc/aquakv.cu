@@ -336,33 +336,6 @@ EncodeWs encode_ws(const aquakv_ctx* c, int64_t T) {
   return w;
 }
 
-struct AttnWs {
-  size_t p_off, khat_off, vhat_off, ml_off, o_off, total;
-  int chunk_blocks;     // split-KV blocks per chunk
-  int n_splits;
-};
-
-AttnWs attn_ws(const aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_heads,
-               int32_t head_dim) {
-  AttnWs w;
-  const int tb = c->attn_block_tokens;
-  w.n_splits = int((ctx_len + tb - 1) / tb);
-  int cb = c->chunk_tokens / tb;
-  if (cb < 1) cb = 1;
-  const int64_t total_blocks = int64_t(batch) * w.n_splits;
-  if (cb > total_blocks) cb = int(total_blocks);
-  w.chunk_blocks = cb;
-  const size_t chunk_rows = size_t(cb) * tb;
-  const size_t d = size_t(c->p.d_kv);
-  w.p_off = 0;
-  w.khat_off = round_up(chunk_rows * d * sizeof(float), 256);
-  w.vhat_off = w.khat_off + round_up(chunk_rows * d * 2, 256);
-  w.ml_off = w.vhat_off + round_up(chunk_rows * d * 2, 256);
-  w.o_off = w.ml_off + round_up(size_t(total_blocks) * n_q_heads * 2 * sizeof(float), 256);
-  w.total = w.o_off + round_up(size_t(total_blocks) * n_q_heads * head_dim * sizeof(float), 256);
-  return w;
-}
-
 // ---------------------------------------------------------------------------------------------
 // fused layer kernel (predictor GEMMs + row work in one persistent launch)
 // ---------------------------------------------------------------------------------------------
@@ -388,6 +361,38 @@ LayerWs layer_ws(const aquakv_ctx* c, int64_t T) {
   w.flags_off = w.khat_off + round_up(size_t(kKhatRing) * mw * kBM * d * 2, 256);
   w.flags_bytes = size_t(2) * 2 * w.n_waves * mw * sizeof(int);
   w.total = w.flags_off + round_up(w.flags_bytes, 256);
+  return w;
+}
+
+struct AttnWs {
+  size_t layer_off, khat_off, vhat_off, ml_off, o_off, total;
+  int chunk_blocks;     // split-KV blocks per chunk
+  int n_splits;
+};
+
+// The decode of a long cache runs chunk by chunk (about eight waves of the fused kernel) so that
+// the attention kernel finds most of a chunk's freshly decoded keys/values still in L2.
+AttnWs attn_ws(const aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_heads,
+               int32_t head_dim) {
+  AttnWs w;
+  const int tb = c->attn_block_tokens;
+  const size_t d = size_t(c->p.d_kv);
+  w.n_splits = int((ctx_len + tb - 1) / tb);
+  const int wave_tokens = (c->sm_count / int(d / kBN) > 0 ? c->sm_count / int(d / kBN) : 1) * kBM;
+  int cb = 8 * wave_tokens / tb;
+  if (cb < 1) cb = 1;
+  const int64_t total_blocks = int64_t(batch) * w.n_splits;
+  if (cb > total_blocks) cb = int(total_blocks);
+  w.chunk_blocks = cb;
+  const size_t chunk_rows = size_t(cb) * tb;
+  const size_t phase_bytes = round_up(chunk_rows * d * sizeof(float), 256);   // separate-kernel path
+  const size_t layer_bytes = layer_ws(c, int64_t(chunk_rows)).total;
+  w.layer_off = 0;
+  w.khat_off = phase_bytes > layer_bytes ? phase_bytes : layer_bytes;
+  w.vhat_off = w.khat_off + round_up(chunk_rows * d * 2, 256);
+  w.ml_off = w.vhat_off + round_up(chunk_rows * d * 2, 256);
+  w.o_off = w.ml_off + round_up(size_t(total_blocks) * n_q_heads * 2 * sizeof(float), 256);
+  w.total = w.o_off + round_up(size_t(total_blocks) * n_q_heads * head_dim * sizeof(float), 256);
   return w;
 }
 
@@ -1035,7 +1040,6 @@ int aquakv_decode_attn(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_
 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   uint8_t* wsb = static_cast<uint8_t*>(workspace);
-  float* P = has_pred ? reinterpret_cast<float*>(wsb + ws.p_off) : nullptr;
   float* part_ml = reinterpret_cast<float*>(wsb + ws.ml_off);
   float* part_o = reinterpret_cast<float*>(wsb + ws.o_off);
   const int cb = c->code_bytes, ng = c->n_groups, tb = c->attn_block_tokens;
@@ -1056,17 +1060,18 @@ int aquakv_decode_attn(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_
                                    : reinterpret_cast<uint16_t*>(wsb + ws.vhat_off);
     const int64_t ldh = Khat != nullptr ? ld_hat : d;
     if (has_pred) {
-      rc = launch_predict(c, st, rows, Kpv + t0 * ld_prev, nullptr, ld_prev, 0, Wk, bk, P, d);
+      // Algorithm 3 for the chunk in one fused launch (predictor GEMMs + row work)
+      rc = launch_layer(c, st, false, rows, nullptr, nullptr, 0, Kpv + t0 * ld_prev, Vpv + t0 * ld_prev,
+                        ld_prev, Wk, Wv, bk, bv, const_cast<uint8_t*>(Kcodes) + t0 * cb,
+                        const_cast<uint16_t*>(Kscales) + t0 * ng, const_cast<uint8_t*>(Vcodes) + t0 * cb,
+                        const_cast<uint16_t*>(Vscales) + t0 * ng, kh, vh, ldh, wsb + ws.layer_off);
+      if (rc) return rc;
+    } else {
+      rc = launch_decode_rows(c, st, kRoleK, rows, Kcodes + t0 * cb, Kscales + t0 * ng, nullptr, d, kh, ldh);
+      if (rc) return rc;
+      rc = launch_decode_rows(c, st, kRoleV, rows, Vcodes + t0 * cb, Vscales + t0 * ng, nullptr, d, vh, ldh);
       if (rc) return rc;
     }
-    rc = launch_decode_rows(c, st, kRoleK, rows, Kcodes + t0 * cb, Kscales + t0 * ng, P, d, kh, ldh);
-    if (rc) return rc;
-    if (has_pred) {
-      rc = launch_predict(c, st, rows, Vpv + t0 * ld_prev, kh, ld_prev, ldh, Wv, bv, P, d);
-      if (rc) return rc;
-    }
-    rc = launch_decode_rows(c, st, kRoleV, rows, Vcodes + t0 * cb, Vscales + t0 * ng, P, d, vh, ldh);
-    if (rc) return rc;
     AttnArgs a;
     a.q = static_cast<const uint16_t*>(q);
     a.Kh = kh;
