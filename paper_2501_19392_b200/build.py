@@ -10,14 +10,13 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libaquakv.so")
 SOURCES = ["aquakv.cu"]
-HEADERS = ["common.cuh", "gemm_pred.cuh", "codec.cuh", "attn.cuh"]
 
 
 def _stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in SOURCES + HEADERS] + [os.path.join(ROOT, "include", "aquakv.h")]
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "aquakv.h")]
     return any(os.path.getmtime(d) > t for d in deps if os.path.exists(d))
 
 
