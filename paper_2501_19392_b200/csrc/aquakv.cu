@@ -351,9 +351,9 @@ LayerWs layer_ws(const aquakv_ctx* c, int64_t T) {
   LayerWs w;
   const int d = c->p.d_kv, ntn = d / kBN;
   w.n_mblocks = int((T + kBM - 1) / kBM);
-  int mw = c->sm_count / ntn;
-  if (mw < 1) mw = 1;
-  if (mw > w.n_mblocks) mw = w.n_mblocks;
+  int mw = (c->sm_count / ntn) & ~1;          // CTAs work in pairs on two token blocks
+  if (mw < 2) mw = 2;
+  if (mw > w.n_mblocks) mw = (w.n_mblocks + 1) & ~1;
   w.mw = mw;
   w.n_waves = (w.n_mblocks + mw - 1) / mw;
   w.p_off = 0;
@@ -406,8 +406,22 @@ int launch_layer_t(cudaStream_t st, int grid, const CUtensorMap* tm, const Layer
       return AQUAKV_ERR_CUDA;
     attr_set = true;
   }
-  layer_kernel<ENC, D, NPTS, BF><<<grid, kLayerThreads, smem, st>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], a);
-  return AQUAKV_OK;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(grid));
+  cfg.blockDim = dim3(kLayerThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, layer_kernel<ENC, D, NPTS, BF>, tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], a) ==
+                 cudaSuccess
+             ? AQUAKV_OK
+             : AQUAKV_ERR_CUDA;
 }
 template <int D, int NPTS, bool BF>
 void launch_layer_enc_t(int* rc, cudaStream_t st, int grid, const CUtensorMap* tm, const LayerArgs& a) {
@@ -490,8 +504,9 @@ int launch_layer(aquakv_ctx* c, cudaStream_t st, bool encode, int64_t T, const v
   if ((rc = make_tmap(c, &tm[1], Vhat_prev, uint64_t(T), uint64_t(d), uint64_t(ld_prev), kBM))) return rc;
   const uint64_t khat_rows = a.khat_ring ? uint64_t(kKhatRing) * ws.mw * kBM : uint64_t(T);
   if ((rc = make_tmap(c, &tm[2], a.Khat, khat_rows, uint64_t(d), uint64_t(a.ldKhat), kBM))) return rc;
-  if ((rc = make_tmap(c, &tm[3], Wk, uint64_t(d), uint64_t(d), uint64_t(d), kBN))) return rc;
-  if ((rc = make_tmap(c, &tm[4], Wv, uint64_t(d), uint64_t(2) * d, uint64_t(2) * d, kBN))) return rc;
+  // weight tiles are fetched half (128 rows) per CTA of a pair
+  if ((rc = make_tmap(c, &tm[3], Wk, uint64_t(d), uint64_t(d), uint64_t(d), kBN / 2))) return rc;
+  if ((rc = make_tmap(c, &tm[4], Wv, uint64_t(d), uint64_t(2) * d, uint64_t(2) * d, kBN / 2))) return rc;
 
   if (cudaMemsetAsync(a.gemm_done, 0, ws.flags_bytes, st) != cudaSuccess) return AQUAKV_ERR_CUDA;
   const int grid = ws.mw * (d / kBN);

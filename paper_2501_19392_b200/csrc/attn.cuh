@@ -46,12 +46,13 @@ __device__ __forceinline__ void unpack8(const uint4& raw, float (&f)[8]) {
 }
 
 template <int HD, int GQ, bool kBf16>
-__global__ void __launch_bounds__(kAttnThreads) attn_partial_kernel(const AttnArgs a) {
+__global__ void __launch_bounds__(kAttnThreads, 2) attn_partial_kernel(const AttnArgs a) {
   constexpr int NP = HD / 64;          // 16-byte pieces per lane per row (8 dims each)
   constexpr int DPL = NP * 8;          // dims per lane
   __shared__ float sm_m[kAttnWarps][GQ];
   __shared__ float sm_l[kAttnWarps][GQ];
   __shared__ float sm_o[kAttnWarps][GQ][HD];
+  __shared__ float sm_q[GQ][HD];       // queries, pre-multiplied by softmax_scale * log2(e)
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int tg = lane >> 3, dl = lane & 7;
   const long long gb = a.blk_begin + blockIdx.x;
@@ -62,18 +63,13 @@ __global__ void __launch_bounds__(kAttnThreads) attn_partial_kernel(const AttnAr
   const int kvh = blockIdx.y;
   const int g0 = blockIdx.z * GQ;      // first query head (within the KV group) of this pass
 
-  float qf[GQ][DPL];
-#pragma unroll
-  for (int g = 0; g < GQ; ++g) {
-    const uint16_t* qp = a.q + ((long long)b * a.n_q_heads + kvh * rep + g0 + g) * HD;
-#pragma unroll
-    for (int pc = 0; pc < NP; ++pc) {
-      float f[8];
-      unpack8<kBf16>(*reinterpret_cast<const uint4*>(qp + pc * 64 + dl * 8), f);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) qf[g][pc * 8 + i] = f[i] * a.scale_log2;
-    }
+  for (int idx = threadIdx.x; idx < GQ * HD; idx += kAttnThreads) {
+    const int g = idx / HD, i = idx % HD;
+    const uint16_t qb = a.q[((long long)b * a.n_q_heads + kvh * rep + g0 + g) * HD + i];
+    sm_q[g][i] = load16<kBf16>(qb) * a.scale_log2;
   }
+  __syncthreads();
+
   float m[GQ], l[GQ], acc[GQ][DPL];
 #pragma unroll
   for (int g = 0; g < GQ; ++g) {
@@ -83,21 +79,34 @@ __global__ void __launch_bounds__(kAttnThreads) attn_partial_kernel(const AttnAr
     for (int i = 0; i < DPL; ++i) acc[g][i] = 0.0f;
   }
   const long long row0 = (long long)b * a.ctx - a.tok_base;
-  // warp w takes tokens t_begin + 4*(w + 8*j) + {0,1,2,3}; its four lane groups take one each
-  for (int tb = t_begin + warp * 4; tb < t_end; tb += 4 * kAttnWarps) {
+  // warp w takes tokens t_begin + 4*(w + 8*j) + {0,1,2,3}; its four lane groups take one each.
+  // The next iteration's key/value pieces are fetched before the current ones are used.
+  uint4 kraw[NP], vraw[NP], kraw_n[NP], vraw_n[NP];
+  auto fetch = [&](int tb, uint4 (&kr)[NP], uint4 (&vr)[NP]) {
     const int t = tb + tg;
-    const bool valid = t < t_end;
-    const long long row = row0 + (valid ? t : t_begin);
+    const long long row = row0 + (t < t_end ? t : t_begin);
     const uint16_t* kp = a.Kh + row * a.ld + kvh * HD + dl * 8;
     const uint16_t* vp = a.Vh + row * a.ld + kvh * HD + dl * 8;
+#pragma unroll
+    for (int pc = 0; pc < NP; ++pc) {
+      kr[pc] = __ldcs(reinterpret_cast<const uint4*>(kp + pc * 64));
+      vr[pc] = __ldcs(reinterpret_cast<const uint4*>(vp + pc * 64));
+    }
+  };
+  int tb = t_begin + warp * 4;
+  if (tb < t_end) fetch(tb, kraw, vraw);
+  for (; tb < t_end; tb += 4 * kAttnWarps) {
+    const int tbn = tb + 4 * kAttnWarps;
+    if (tbn < t_end) fetch(tbn, kraw_n, vraw_n);
+    const bool valid = tb + tg < t_end;
     float kf[DPL], vf[DPL];
 #pragma unroll
     for (int pc = 0; pc < NP; ++pc) {
       float f[8];
-      unpack8<kBf16>(*reinterpret_cast<const uint4*>(kp + pc * 64), f);
+      unpack8<kBf16>(kraw[pc], f);
 #pragma unroll
       for (int i = 0; i < 8; ++i) kf[pc * 8 + i] = f[i];
-      unpack8<kBf16>(*reinterpret_cast<const uint4*>(vp + pc * 64), f);
+      unpack8<kBf16>(vraw[pc], f);
 #pragma unroll
       for (int i = 0; i < 8; ++i) vf[pc * 8 + i] = f[i];
     }
@@ -105,7 +114,14 @@ __global__ void __launch_bounds__(kAttnThreads) attn_partial_kernel(const AttnAr
     for (int g = 0; g < GQ; ++g) {
       float s = 0.0f;
 #pragma unroll
-      for (int i = 0; i < DPL; ++i) s = fmaf(qf[g][i], kf[i], s);
+      for (int pc = 0; pc < NP; ++pc) {
+        const float4 q0 = *reinterpret_cast<const float4*>(&sm_q[g][pc * 64 + dl * 8]);
+        const float4 q1 = *reinterpret_cast<const float4*>(&sm_q[g][pc * 64 + dl * 8 + 4]);
+        s = fmaf(q0.x, kf[pc * 8 + 0], s); s = fmaf(q0.y, kf[pc * 8 + 1], s);
+        s = fmaf(q0.z, kf[pc * 8 + 2], s); s = fmaf(q0.w, kf[pc * 8 + 3], s);
+        s = fmaf(q1.x, kf[pc * 8 + 4], s); s = fmaf(q1.y, kf[pc * 8 + 5], s);
+        s = fmaf(q1.z, kf[pc * 8 + 6], s); s = fmaf(q1.w, kf[pc * 8 + 7], s);
+      }
       s += __shfl_xor_sync(0xffffffffu, s, 1);
       s += __shfl_xor_sync(0xffffffffu, s, 2);
       s += __shfl_xor_sync(0xffffffffu, s, 4);
@@ -118,6 +134,11 @@ __global__ void __launch_bounds__(kAttnThreads) attn_partial_kernel(const AttnAr
 #pragma unroll
         for (int i = 0; i < DPL; ++i) acc[g][i] = fmaf(acc[g][i], corr, pr * vf[i]);
       }
+    }
+#pragma unroll
+    for (int pc = 0; pc < NP; ++pc) {
+      kraw[pc] = kraw_n[pc];
+      vraw[pc] = vraw_n[pc];
     }
   }
   // merge the four token groups of the warp

@@ -7,8 +7,12 @@
 // memory.
 //
 // Work layout.  A token block is 128 tokens; a GEMM tile is one token block x 256 output features,
-// so NTN = d_kv/256 CTAs share a token block.  CTA c owns token-block slot ml = c / NTN and feature
-// tile n = c % NTN in every "wave" of gridDim.x / NTN token blocks.  For each wave a CTA computes
+// so NTN = d_kv/256 CTAs share a token block.  CTAs run as pairs (clusters of two): pair p owns
+// feature tile n = p % NTN and the two token-block slots ml = 2 * (p / NTN) + rank, and computes
+// both tiles with one tcgen05.mma.cta_group::2 of M = 256: each CTA loads its own 128 token rows
+// and HALF of the 256 weight rows, so a k-block costs 32 KB of L2 traffic per CTA instead of 48 KB
+// (the GEMM is bound by L2 bandwidth, not by the tensor pipe).  Every "wave" covers
+// gridDim.x / NTN token blocks.  For each wave a CTA computes
 // its key-phase tile and its value-phase tile, and runs the row work of 128/NTN rows of its token
 // block for both phases.  Jobs are ordered  K0, K1, V0, K2, V1, ..., so that the value-phase GEMM of
 // a wave (which reads the reconstructed keys of that wave) is issued one job after its key rows.
@@ -35,7 +39,9 @@ namespace aquakv {
 
 constexpr int kRowWarps = 16;
 constexpr int kLayerThreads = 32 * (6 + kRowWarps);
-constexpr int kLayerStages = 3;
+constexpr int kLayerStages = 4;
+constexpr int kPairBBytes = (kBN / 2) * kBK * 2;        // this CTA's half of a weight tile k-block
+constexpr int kPairStageBytes = kABytes + kPairBBytes;   // 32 KB
 template <int D> constexpr int kRowTeamsOf = kRowWarps / RowTeam<D>::TEAM;
 
 struct LayerSmemTail {
@@ -68,7 +74,7 @@ constexpr int kEpiBytes = 4 * 2 * kEpiPieceBytes;
 
 template <bool kEncode, int D, int NPTS>
 constexpr size_t layer_smem_bytes() {
-  return 1024 + size_t(kLayerStages) * kStageBytes + kEpiBytes + sizeof(LayerSmemTail) + 16 +
+  return 1024 + size_t(kLayerStages) * kPairStageBytes + kEpiBytes + sizeof(LayerSmemTail) + 16 +
          sizeof(LayerRowSmem<kEncode, D, NPTS>);
 }
 
@@ -174,15 +180,18 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~uintptr_t(1023));
-  uint8_t* epi_smem = smem + size_t(kLayerStages) * kStageBytes;      // 1024-byte aligned
+  uint8_t* epi_smem = smem + size_t(kLayerStages) * kPairStageBytes;      // 1024-byte aligned
   LayerSmemTail* tail = reinterpret_cast<LayerSmemTail*>(epi_smem + kEpiBytes);
   LayerRowSmem<kEncode, D, NPTS>* rsm = reinterpret_cast<LayerRowSmem<kEncode, D, NPTS>*>(
       (reinterpret_cast<uintptr_t>(tail) + sizeof(LayerSmemTail) + 15) & ~uintptr_t(15));
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int ml = blockIdx.x / NTN;
-  const int n_blk = blockIdx.x % NTN;
+  const uint32_t rank = cluster_ctarank();          // 0 = leader of the pair (issues the MMAs)
+  const int pair = blockIdx.x >> 1;
+  const int ml = 2 * (pair / NTN) + int(rank);
+  const int ml0 = 2 * (pair / NTN);                 // the pair is active in a wave iff its first block exists
+  const int n_blk = pair % NTN;
   const int n_jobs = 2 * a.n_waves;
 
   if (threadIdx.x == 0) {
@@ -192,7 +201,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
     }
     for (int s = 0; s < kAccStages; ++s) {
       mbar_init(&tail->acc_full[s], 1);
-      mbar_init(&tail->acc_empty[s], 4);
+      mbar_init(&tail->acc_empty[s], 8);     // 4 epilogue warps of each CTA (used in the leader only)
     }
     tail->abort_flag = 0;
     mbar_fence_init();
@@ -206,11 +215,12 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
     }
   }
   if (warp == 1) {
-    tmem_alloc(&tail->tmem_base, kTmemCols);
-    tmem_relinquish();
+    tmem_alloc_pair(&tail->tmem_base, kTmemCols);
+    tmem_relinquish_pair();
   }
   tc_fence_before_sync();
   __syncthreads();
+  cluster_sync_all();          // the peer's barriers are initialised before anything signals them
   tc_fence_after_sync();
   const uint32_t tmem_base = tail->tmem_base;
   volatile int* abort_flag = &tail->abort_flag;
@@ -232,11 +242,11 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         int ph, wave;
         layer_job(j, a.n_waves, ph, wave);
         const int m = wave * a.mw + ml;
-        if (m >= a.n_mblocks) continue;
+        if (wave * a.mw + ml0 >= a.n_mblocks) continue;
         const int nk = ph == 0 ? NKD : 2 * NKD;
         const int khat_row = a.khat_ring ? ((wave % a.khat_ring) * a.mw + ml) * kBM : m * kBM;
         for (int kb = 0; kb < nk; ++kb) {
-          if (ph == 1 && kb == NKD) {
+          if (ph == 1 && kb == NKD && m < a.n_mblocks) {
             // the remaining k-blocks read this wave's reconstructed keys, written by row warps
             if (!counter_wait_bounded(a.rows_done + layer_key_job(wave) * a.mw + ml, NTN * kRowTeamsOf<D>, abort_flag,
                                       a.status)) {
@@ -249,26 +259,28 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
             ok = false;
             break;
           }
-          uint8_t* a_dst = smem + size_t(stage) * kStageBytes;
+          uint8_t* a_dst = smem + size_t(stage) * kPairStageBytes;
           uint8_t* b_dst = a_dst + kABytes;
-          mbar_arrive_expect_tx(&tail->full[stage], kStageBytes);
+          // the leader's barrier collects the bytes of both CTAs
+          if (rank == 0) mbar_arrive_expect_tx(&tail->full[stage], 2 * kPairStageBytes);
+          const int w_row = n_blk * kBN + int(rank) * (kBN / 2);     // this CTA's half of the weight rows
           if (ph == 0) {
-            tma_load_2d(a_dst, &tmKprev, &tail->full[stage], kb * kBK, m * kBM);
-            tma_load_2d(b_dst, &tmWk, &tail->full[stage], kb * kBK, n_blk * kBN);
+            tma_load_2d_pair(a_dst, &tmKprev, &tail->full[stage], kb * kBK, m * kBM);
+            tma_load_2d_pair(b_dst, &tmWk, &tail->full[stage], kb * kBK, w_row);
           } else {
             if (kb < NKD) {
-              tma_load_2d(a_dst, &tmVprev, &tail->full[stage], kb * kBK, m * kBM);
+              tma_load_2d_pair(a_dst, &tmVprev, &tail->full[stage], kb * kBK, m * kBM);
             } else {
-              tma_load_2d(a_dst, &tmKhat, &tail->full[stage], (kb - NKD) * kBK, khat_row);
+              tma_load_2d_pair(a_dst, &tmKhat, &tail->full[stage], (kb - NKD) * kBK, khat_row);
             }
-            tma_load_2d(b_dst, &tmWv, &tail->full[stage], kb * kBK, n_blk * kBN);
+            tma_load_2d_pair(b_dst, &tmWv, &tail->full[stage], kb * kBK, w_row);
           }
           ++issued;
           if (++stage == kLayerStages) { stage = 0; phase_bit ^= 1u; }
         }
       }
-      if (!ok) {
-        // let this CTA's copies in flight land before its shared memory is released
+      if (!ok && rank == 0) {
+        // let the copies in flight land before the shared memory is released
         int s = stage;
         uint32_t pb = phase_bit;
         const int pending = issued < kLayerStages ? issued : kLayerStages;
@@ -283,8 +295,8 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
     }
   } else if (warp == 1) {
     // ------------------------------- MMA issuer ----------------------------------------------
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_f16(kBM, kBN, kBf16);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = umma_idesc_f16(2 * kBM, kBN, kBf16);
       int stage = 0;
       uint32_t phase_bit = 0;
       bool ok = true;
@@ -292,7 +304,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       for (int j = 0; ok && j < n_jobs; ++j) {
         int ph, wave;
         layer_job(j, a.n_waves, ph, wave);
-        if (wave * a.mw + ml >= a.n_mblocks) continue;
+        if (wave * a.mw + ml0 >= a.n_mblocks) continue;
         const int nk = ph == 0 ? NKD : 2 * NKD;
         const int acc = it & 1;
         const uint32_t acc_phase = (it >> 1) & 1u;
@@ -306,18 +318,18 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
             break;
           }
           tc_fence_after_sync();
-          const uint32_t a_addr = smem_u32(smem + size_t(stage) * kStageBytes);
+          const uint32_t a_addr = smem_u32(smem + size_t(stage) * kPairStageBytes);
           const uint32_t b_addr = a_addr + kABytes;
 #pragma unroll
           for (int k = 0; k < kBK / kUmmaK; ++k) {
             const uint64_t da = umma_smem_desc_k128(a_addr + k * kUmmaK * 2);
             const uint64_t db = umma_smem_desc_k128(b_addr + k * kUmmaK * 2);
-            umma_f16(tmem_d, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            umma_f16_pair(tmem_d, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
           }
-          umma_commit(&tail->empty[stage]);
+          umma_commit_pair(&tail->empty[stage]);   // frees the stage in both CTAs
           if (++stage == kLayerStages) { stage = 0; phase_bit ^= 1u; }
         }
-        if (ok) umma_commit(&tail->acc_full[acc]);
+        if (ok) umma_commit_pair(&tail->acc_full[acc]);
       }
     }
   } else if (warp < 6) {
@@ -327,8 +339,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
     for (int j = 0; j < n_jobs; ++j) {
       int ph, wave;
       layer_job(j, a.n_waves, ph, wave);
-      const int m = wave * a.mw + ml;
-      if (m >= a.n_mblocks) continue;
+      if (wave * a.mw + ml0 >= a.n_mblocks) continue;
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1u;
       ++it;
@@ -375,7 +386,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) {
-          mbar_arrive(&tail->acc_empty[acc]);
+          mbar_arrive_leader(&tail->acc_empty[acc]);   // the leader's MMA issuer waits for both CTAs
           bulk_wait_all();               // the tile's rows are written
           fence_proxy_async_all();
         }
@@ -454,9 +465,10 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
 
   tc_fence_before_sync();
   __syncthreads();
+  cluster_sync_all();          // neither CTA leaves while its peer may still signal its barriers
   if (warp == 1) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, kTmemCols);
+    tmem_dealloc_pair(tmem_base, kTmemCols);
   }
 }
 
