@@ -411,7 +411,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       int ph, wave;
       layer_job(j, a.n_waves, ph, wave);
       const int m = wave * a.mw + ml;
-      if (m >= a.n_mblocks) continue;
+      if (wave * a.mw + ml0 >= a.n_mblocks) continue;   // (a missing second block of a pair has no rows)
       if constexpr (kEncode) {
         // pull this job's input rows towards L2 while the prediction is still being produced
         const uint16_t* xin = ph == 0 ? a.K : a.V;
