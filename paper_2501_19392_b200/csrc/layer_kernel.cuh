@@ -19,7 +19,8 @@
 //
 // Dependencies (all counted per job j and token-block slot ml, targets NTN):
 //   gemm_done[j][ml]  -- feature tiles of job j written to the ring        (row warps wait)
-//   rows_done[j][ml]  -- row teams that finished job j (target NTN x teams per CTA)                      (the value-phase TMA
+//   rows_done[j][ml]  -- row teams that finished job j on token block ml (target: CTAs per block
+//                        x teams per CTA)                                    (the value-phase TMA
 //                        producer waits for the key rows of its wave; the GEMM epilogue waits for
 //                        job j - ring size before it overwrites that ring slot)
 // Every job waits only on jobs with a smaller index (or the same index of the other role), so the
@@ -133,6 +134,34 @@ __device__ __forceinline__ void layer_job(int j, int n_waves, int& phase, int& w
 }
 __device__ __forceinline__ int layer_key_job(int wave) { return wave == 0 ? 0 : 2 * wave - 1; }
 
+// Row work of a wave is spread evenly over ALL CTAs: CTA slot s takes rows [s*rpc, (s+1)*rpc) of
+// the wave, rpc = the power of two >= rows / CTAs.  For a full wave this is rpc = 128 / NTN rows of
+// the CTA's own token block; in the short last wave it keeps every SM busy instead of a few.
+struct WaveRows {
+  int tokens;      // rows of the wave
+  int blocks;      // token blocks of the wave
+  int rpc;         // rows per CTA slot (power of two, <= 128 / NTN)
+};
+__device__ __forceinline__ WaveRows wave_rows(int wave, int T, int mw, int n_ctas) {
+  WaveRows w;
+  const long long left = (long long)T - (long long)wave * mw * kBM;
+  w.tokens = left < (long long)mw * kBM ? int(left) : mw * kBM;
+  w.blocks = (w.tokens + kBM - 1) / kBM;
+  const int need = (w.tokens + n_ctas - 1) / n_ctas;
+  int rpc = 1;
+  while (rpc < need) rpc <<= 1;
+  w.rpc = rpc;
+  return w;
+}
+
+// Number of row teams that report on token block `block` of that wave (CTA slots on the block x teams).
+__device__ __forceinline__ int wave_block_teams(const WaveRows& w, int block, int n_ctas, int teams) {
+  const int per_block = kBM / w.rpc;
+  const int hi = (block + 1) * per_block < n_ctas ? (block + 1) * per_block : n_ctas;
+  const int n = hi - block * per_block;
+  return (n > 0 ? n : 0) * teams;
+}
+
 __device__ __forceinline__ int ld_acquire(const int* p) {
   int v;
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -173,7 +202,6 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
              const __grid_constant__ CUtensorMap tmWv, const __grid_constant__ CUtensorMap tmP,
              const LayerArgs a) {
   constexpr int NTN = D / kBN;             // feature tiles per token block = CTAs per token block
-  constexpr int RJ = kBM / NTN;            // rows of a token block whose row work this CTA does
   constexpr int NKD = D / kBK;             // k-blocks per d_kv input features
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
   constexpr int CODE_BYTES = D / 2 * BITS / 8;
@@ -248,7 +276,8 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         for (int kb = 0; kb < nk; ++kb) {
           if (ph == 1 && kb == NKD && m < a.n_mblocks) {
             // the remaining k-blocks read this wave's reconstructed keys, written by row warps
-            if (!counter_wait_bounded(a.rows_done + layer_key_job(wave) * a.mw + ml, NTN * kRowTeamsOf<D>, abort_flag,
+            const int target = wave_block_teams(wave_rows(wave, a.T, a.mw, gridDim.x), ml, gridDim.x, kRowTeamsOf<D>);
+            if (!counter_wait_bounded(a.rows_done + layer_key_job(wave) * a.mw + ml, target, abort_flag,
                                       a.status)) {
               ok = false;
               break;
@@ -346,7 +375,10 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       bool ok = true;
       // the ring slot of this job was last used by job j - nb: its row work must be over
       if (j >= a.nb) {
-        if (lane == 0) ok = counter_wait_bounded(a.rows_done + (j - a.nb) * a.mw + ml, NTN * kRowTeamsOf<D>, abort_flag, a.status);
+        int ph_old, wave_old;
+        layer_job(j - a.nb, a.n_waves, ph_old, wave_old);
+        const int target = wave_block_teams(wave_rows(wave_old, a.T, a.mw, gridDim.x), ml, gridDim.x, kRowTeamsOf<D>);
+        if (lane == 0) ok = counter_wait_bounded(a.rows_done + (j - a.nb) * a.mw + ml, target, abort_flag, a.status);
         ok = __shfl_sync(0xffffffffu, ok, 0);
       }
       if (ok) ok = mbar_wait_bounded(&tail->acc_full[acc], acc_phase, abort_flag, a.status);
@@ -410,19 +442,26 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
     for (int j = 0; j < n_jobs; ++j) {
       int ph, wave;
       layer_job(j, a.n_waves, ph, wave);
-      const int m = wave * a.mw + ml;
-      if (wave * a.mw + ml0 >= a.n_mblocks) continue;   // (a missing second block of a pair has no rows)
+      const WaveRows wr = wave_rows(wave, a.T, a.mw, gridDim.x);
+      if (wr.tokens <= 0) continue;
+      const int slot_row = (ml * NTN + n_blk) * wr.rpc;      // first row (within the wave) of this CTA's slice
+      const int rb = slot_row / kBM;                         // token block (within the wave) the slice lies in
+      if (rb >= wr.blocks) continue;                         // nothing assigned, nobody waits for this CTA
+      const int r_begin = slot_row % kBM;
+      const int m = wave * a.mw + rb;
+      const long long rows_left = (long long)a.T - (long long)m * kBM;
+      const int r_end = rows_left < r_begin + wr.rpc ? int(rows_left) : r_begin + wr.rpc;
       if constexpr (kEncode) {
         // pull this job's input rows towards L2 while the prediction is still being produced
         const uint16_t* xin = ph == 0 ? a.K : a.V;
-        for (int r = n_blk * RJ + team; r < (n_blk + 1) * RJ; r += TEAMS) {
+        for (int r = r_begin + team; r < r_end; r += TEAMS) {
           const long long g = (long long)m * kBM + r;
-          if (g < a.T && lane < D / 256 / TEAM * 4)
+          if (lane < D / 256 / TEAM * 4)
             asm volatile("prefetch.global.L2 [%0];" ::"l"(xin + g * a.ldX + rck.member * (D / TEAM) + lane * 64));
         }
       }
       bool ok = true;
-      if (lane == 0) ok = counter_wait_bounded(a.gemm_done + j * a.mw + ml, NTN, abort_flag, a.status);
+      if (lane == 0) ok = counter_wait_bounded(a.gemm_done + j * a.mw + rb, NTN, abort_flag, a.status);
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (TEAM == 2) {
         // both warps of a team must take the same path: agree through shared memory
@@ -432,12 +471,11 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         team_barrier(rck.barrier);
       }
       if (ok) {
-        const float* pbuf = a.P + (size_t(j % a.nb) * a.mw * kBM + size_t(ml) * kBM) * D;
-        const size_t khat_base = a.khat_ring ? size_t((wave % a.khat_ring) * a.mw + ml) * kBM
+        const float* pbuf = a.P + (size_t(j % a.nb) * a.mw * kBM + size_t(rb) * kBM) * D;
+        const size_t khat_base = a.khat_ring ? size_t((wave % a.khat_ring) * a.mw + rb) * kBM
                                              : size_t(m) * kBM;
-        for (int r = n_blk * RJ + team; r < (n_blk + 1) * RJ; r += TEAMS) {
+        for (int r = r_begin + team; r < r_end; r += TEAMS) {
           const long long g = (long long)m * kBM + r;
-          if (g >= a.T) break;
           const float* pred_row = pbuf + size_t(r) * D;
           uint16_t* hat_row;
           if (ph == 0) hat_row = a.Khat + (khat_base + r) * a.ldKhat;
@@ -459,7 +497,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       fence_proxy_async_all();
       if (TEAM == 2) team_barrier(rck.barrier); else __syncwarp();
       if (*abort_flag) break;
-      if (rck.member == 0 && lane == 0) atomicAdd(a.rows_done + j * a.mw + ml, 1);
+      if (rck.member == 0 && lane == 0) atomicAdd(a.rows_done + j * a.mw + rb, 1);
     }
   }
 
