@@ -182,3 +182,84 @@ def test_full_size_layer_on_sampled_rows(T, n):
     Kc4, Ks4, Vc4, Vs4, _, _ = codec.encode(g(K), g(V), g(prevK), g(prevV), g(Wk), g(Wv), want_hat=False)
     torch.cuda.synchronize()
     assert torch.equal(Kc4, Kc) and torch.equal(Vc4, Vc) and torch.equal(Ks4, Ks) and torch.equal(Vs4, Vs)
+
+
+@pytest.mark.parametrize("d,hd,h,g,n,dtype,T", [
+    (256, 64, 256, 256, 16, synth.BF16, 131),     # one 256-wide feature tile per token block, one-warp teams
+    (512, 64, 64, 64, 16, synth.F16, 1),          # a single token
+    (512, 64, 128, 256, 64, synth.BF16, 259),     # Hadamard block < scale group < row, four candidates per cell
+    (1024, 128, 1024, 1024, 256, synth.BF16, 200),  # 256-point grid: encode takes the separate-kernel path
+    (1024, 128, 512, 1024, 16, synth.F16, 385),   # Hadamard block = one warp's half row, group = whole row
+])
+def test_fused_layer_shapes_strides_and_bias(d, hd, h, g, n, dtype, T):
+    """The fused layer kernel (and its separate-kernel fallback) on the other supported shapes, with
+    predictor biases and row strides larger than d_kv, against the oracle (teacher-forced)."""
+    from paper_2501_19392_b200 import api
+    shape = dataclasses.replace(synth.CONFIGS[2], n_kv_heads=d // hd, head_dim=hd, n_tokens=T, n_layers=2,
+                                dtype=dtype, had_block=h, scale_group=g, grid_size=n, channel_scales=False)
+    kv = synth.kv_chain(shape, seed=77 + d + T)
+    ad = synth.random_adapters(shape, seed=78 + d + T, bias=True)
+    codec, ora = make(d, h, g, n, dtype)
+    bits = shape.code_bits
+    b = synth.to_bits
+    ld = d + 64                                     # padded rows: ld % 8 == 0, ld > d_kv
+    def padded(t):
+        buf = torch.zeros((T, ld), dtype=t.dtype, device=DEV)
+        buf[:, :d] = t.to(DEV)
+        return buf[:, :d]
+    K, V, pK, pV = padded(kv.K[1]), padded(kv.V[1]), padded(kv.K[0]), padded(kv.V[0])
+    Kh = torch.zeros((T, ld), dtype=codec.torch_dtype, device=DEV)[:, :d]
+    Vh = torch.zeros((T, ld), dtype=codec.torch_dtype, device=DEV)[:, :d]
+    Wk, Wv, bk, bv = ad.Wk[1].to(DEV), ad.Wv[1].to(DEV), ad.bk[1].to(DEV), ad.bv[1].to(DEV)
+    Kc, Ks, Vc, Vs, _, _ = codec.encode(K, V, pK, pV, Wk, Wv, bk, bv, Khat=Kh, Vhat=Vh)
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    ok_ = ora.encode_phase(b(kv.K[1]), [b(kv.K[0])], b(ad.Wk[1]), ad.bk[1].numpy(), "k")
+    rows_ok, n_bad = scale_rows_ok(gpu_bits(Ks.view(torch.float16)), ok_["scales"], ok_["scales_exact"])
+    assert n_bad <= 2
+    check_codes(Kc.cpu().numpy(), ok_, bits, rows_ok)
+    same = rows_ok & (Kc.cpu().numpy() == ok_["codes"]).all(axis=1)
+    check_recon(gpu_bits(Kh), ok_["hat_exact"], ok_["hat"], dtype, same)
+    ov_ = ora.encode_phase(b(kv.V[1]), [b(kv.V[0]), gpu_bits(Kh)], b(ad.Wv[1]), ad.bv[1].numpy(), "v")
+    rows_ok_v, n_bad = scale_rows_ok(gpu_bits(Vs.view(torch.float16)), ov_["scales"], ov_["scales_exact"])
+    assert n_bad <= 2
+    check_codes(Vc.cpu().numpy(), ov_, bits, rows_ok_v)
+    same_v = rows_ok_v & (Vc.cpu().numpy() == ov_["codes"]).all(axis=1)
+    check_recon(gpu_bits(Vh), ov_["hat_exact"], ov_["hat"], dtype, same_v)
+    # decode of the oracle's codes (fused kernel) against the oracle's reconstruction
+    oc = lambda o: (torch.from_numpy(o["codes"]).to(DEV), torch.from_numpy(o["scales"]).view(torch.float16).to(DEV))
+    Kd = torch.zeros((T, ld), dtype=codec.torch_dtype, device=DEV)[:, :d]
+    Vd = torch.zeros((T, ld), dtype=codec.torch_dtype, device=DEV)[:, :d]
+    codec.decode(*oc(ok_), *oc(ov_), pK, pV, Wk, Wv, bk, bv, Khat=Kd, Vhat=Vd)
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    check_recon(gpu_bits(Kd), ok_["hat_exact"], ok_["hat"], dtype)
+    same_k = (gpu_bits(Kd) == gpu_bits(Kh)).all(axis=1)       # rows whose value predictor saw the same keys
+    check_recon(gpu_bits(Vd)[same_k], ov_["hat_exact"][same_k], ov_["hat"][same_k], dtype)
+    # own codes decode to the encoder's reconstruction bit for bit; the row padding is untouched
+    Kd2, Vd2 = codec.decode(Kc, Ks, Vc, Vs, pK, pV, Wk, Wv, bk, bv)
+    assert torch.equal(Kd2, Kh) and torch.equal(Vd2, Vh)
+    assert not Kh._base[:, d:].any() and not Vh._base[:, d:].any()
+
+
+def test_empty_and_argument_errors_on_device():
+    from paper_2501_19392_b200 import api
+    codec, _ = make(1024, 1024, 1024, 16, synth.BF16)
+    e = torch.empty((0, 1024), dtype=torch.bfloat16, device=DEV)
+    out = codec.encode(e, e)                       # zero tokens: no launch, no error
+    assert out[0].shape[0] == 0 and codec.launch_count() == 0
+    x = synth.random_16bit((8, 1024), synth.BF16, 1).to(DEV)
+    w = synth.random_16bit((1024, 1024), synth.BF16, 2).to(DEV)
+    with pytest.raises(api.AquaKVError) as err:    # adapters must come as a full set
+        codec.encode(x, x, x, None, w, None)
+    assert err.value.status == -1
+    with pytest.raises(api.AquaKVError) as err:    # misaligned row stride
+        codec.encode(x[:, :1024], x, Khat=torch.empty((8, 1028), dtype=torch.bfloat16, device=DEV)[:, :1024],
+                     Vhat=torch.empty((8, 1028), dtype=torch.bfloat16, device=DEV)[:, :1024])
+    assert err.value.status == -3
+    wv = synth.random_16bit((1024, 2048), synth.BF16, 3).to(DEV)
+    small = torch.empty(1024, dtype=torch.uint8, device=DEV)
+    with pytest.raises(api.AquaKVError) as err:    # workspace too small
+        codec.encode(x, x, x, x, w, wv, workspace=small)
+    assert err.value.status == -4
+    assert codec.poll_status() == 0
