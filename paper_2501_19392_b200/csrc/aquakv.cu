@@ -189,7 +189,7 @@ void launch_decode_rows_t(aquakv_ctx*, cudaStream_t st, const CodecArgs& a, int 
   } while (0)
 
 int codec_grid(const aquakv_ctx* c, int rows) {
-  const int rows_per_block = kCodecWarps / (c->p.d_kv >= 512 ? 2 : 1);   // two-warp teams above 256
+  const int rows_per_block = kCodecWarps / (c->p.d_kv / 256);   // one warp per 256-element chunk
   const int blocks = (rows + rows_per_block - 1) / rows_per_block;
   const int cap = c->sm_count * 8;
   return blocks < cap ? blocks : cap;

@@ -3,15 +3,15 @@
 // 2-D grid, packed codes) and of the residual / add-back steps of Algorithm 2 (lines 6-7, 9) and
 // Algorithm 3 (lines 5, 7).
 //
-// A team of one warp (d_kv = 256) or two warps (d_kv = 512, 1024) owns one token row; each warp
-// holds one or two 256-element chunks.  Element e of the row lives in warp (e/256)/chunks-per-warp,
-// lane (e/8)%32, register ((e/256)%chunks-per-warp)*8 + e%8, so every global access is a 16-byte
-// (16-bit data) or 2x16-byte (fp32) vector per lane and a warp touches whole 128-byte lines.  The
-// Hadamard butterflies over index bits 0-2 are register-local, bits 3-7 are warp shuffles, the
-// next bit (two-chunk warps) is register-local again and the top bit crosses the two warps through
-// shared memory.  Splitting a row over two warps halves the registers per thread, which is what
-// lets enough warps be resident to hide the latencies of this shuffle- and load-heavy code.  The
-// value pair (2j, 2j+1) that shares one code always sits in one lane.
+// A team of d_kv/256 warps (1, 2 or 4) owns one token row; each warp holds one 256-element chunk.
+// Element e of the row lives in warp e/256, lane (e/8)%32, register e%8, so every global access is
+// a 16-byte (16-bit data) or 2x16-byte (fp32) vector per lane and a warp touches whole 128-byte
+// lines.  The Hadamard butterflies over index bits 0-2 are register-local, bits 3-7 are warp
+// shuffles, bits 8-9 cross the warps of the team through shared memory.  The row code is a long
+// chain of dependent shuffles and shared-memory gathers whose throughput grows with the number of
+// resident warps; eight values per lane keep it near 64 registers per thread, which lets 24 row
+// warps sit beside the GEMM warps of the fused kernel.  The value pair (2j, 2j+1) that shares one
+// code always sits in one lane.
 #pragma once
 
 #include "common.cuh"
@@ -239,21 +239,21 @@ __device__ __noinline__ int nearest_exhaustive(float y0, float y1, const float2*
   return idx;
 }
 
-// Geometry of a row team.
+// Geometry of a row team: one warp per 256-element chunk of the row.
 template <int D>
 struct RowTeam {
   static constexpr int NC = D / 256;                 // 256-element chunks per row
-  static constexpr int TEAM = NC >= 2 ? 2 : 1;       // warps per row
-  static constexpr int CPM = NC / TEAM;              // chunks per warp
-  static constexpr int NV = CPM * 8;                 // values per lane
-  static constexpr int CROSS_BIT = 8 + (CPM == 2 ? 1 : 0);   // index bit that separates the warps
+  static constexpr int TEAM = NC;                    // warps per row (1, 2 or 4)
+  static constexpr int LOG_TEAM = NC == 4 ? 2 : (NC == 2 ? 1 : 0);
+  static constexpr int CPM = 1;                      // chunks per warp
+  static constexpr int NV = 8;                       // values per lane
 };
 
-// Exchange buffer of one team (only used when TEAM == 2).
+// Exchange buffer of one team (only used when TEAM > 1).
 template <int D>
 struct TeamSmem {
-  ulonglong2 x[2][RowTeam<D>::CPM * 2][32];   // [member][16-byte piece][lane]
-  float ss[2][2];                         // [member][chunk] sums of squares
+  ulonglong2 x[RowTeam<D>::TEAM][RowTeam<D>::NV / 4][32];   // [member][16-byte piece][lane]
+  float ss[RowTeam<D>::TEAM];                               // [member] sum of squares of its chunk
 };
 
 // Per-warp constants of the row routines.
@@ -264,8 +264,8 @@ struct RowCtx {
   float rs;                // 1 / sqrt(Hadamard block)
   int log_h, log_g;
   int lane;
-  int member;              // 0 or 1: which half of the row this warp holds
-  int barrier;             // named barrier shared by the two warps of the team
+  int member;              // which chunk of the row this warp holds
+  int barrier;             // named barrier shared by the warps of the team
 };
 
 // Fills the fields that depend only on the parameters and on the warp's place in its team.
@@ -283,47 +283,70 @@ __device__ __forceinline__ void row_ctx_init(RowCtx& rc, const uint32_t* signmas
   rc.rs = __int_as_float((127 - (log_h >> 1)) << 23) * ((log_h & 1) ? 0.70710678118654752f : 1.0f);
 }
 
+template <int D>
 __device__ __forceinline__ void team_barrier(int id) {
-  asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory");
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(RowTeam<D>::TEAM * 32) : "memory");
 }
 
-// Publishes this warp's values (and optionally its chunk sums) and reads the partner's.
-template <int D, bool kWithSums>
-__device__ __forceinline__ void team_exchange(const RowCtx& rc, TeamSmem<D>* ts,
+// Publishes this warp's values (and optionally its sum of squares) and reads those of `partner`.
+template <int D, bool kWithSum>
+__device__ __forceinline__ void team_exchange(const RowCtx& rc, TeamSmem<D>* ts, int partner,
                                               const f32x2_t (&vp)[RowTeam<D>::NV / 2],
-                                              f32x2_t (&op)[RowTeam<D>::NV / 2],
-                                              const float (&ss)[RowTeam<D>::CPM],
-                                              float (&oss)[RowTeam<D>::CPM]) {
-  constexpr int NV = RowTeam<D>::NV, CPM = RowTeam<D>::CPM;
-  team_barrier(rc.barrier);                // the partner has finished reading the previous exchange
+                                              f32x2_t (&op)[RowTeam<D>::NV / 2], float ss) {
+  constexpr int NV = RowTeam<D>::NV;
+  team_barrier<D>(rc.barrier);             // everybody has finished reading the previous exchange
 #pragma unroll
   for (int q = 0; q < NV / 4; ++q)
     ts->x[rc.member][q][rc.lane] = make_ulonglong2(vp[2 * q], vp[2 * q + 1]);
-  if (kWithSums && rc.lane == 0) {
-#pragma unroll
-    for (int c = 0; c < CPM; ++c) ts->ss[rc.member][c] = ss[c];
-  }
-  team_barrier(rc.barrier);
+  if (kWithSum && rc.lane == 0) ts->ss[rc.member] = ss;
+  team_barrier<D>(rc.barrier);
 #pragma unroll
   for (int q = 0; q < NV / 4; ++q) {
-    const ulonglong2 t = ts->x[rc.member ^ 1][q][rc.lane];
+    const ulonglong2 t = ts->x[partner][q][rc.lane];
     op[2 * q] = t.x;
     op[2 * q + 1] = t.y;
   }
-  if (kWithSums) {
-#pragma unroll
-    for (int c = 0; c < CPM; ++c) oss[c] = ts->ss[rc.member ^ 1][c];
-  }
 }
 
-// Butterfly over the index bit that separates the two warps: the lower half keeps a + b, the upper
-// half a - b (a = lower half's value, b = upper half's).
+// Publishes only the sums of squares (scale groups that span warps while Hadamard blocks do not).
+template <int D>
+__device__ __forceinline__ void team_exchange_sums(const RowCtx& rc, TeamSmem<D>* ts, float ss) {
+  team_barrier<D>(rc.barrier);
+  if (rc.lane == 0) ts->ss[rc.member] = ss;
+  team_barrier<D>(rc.barrier);
+}
+
+// Butterfly over an index bit that separates warps: the lower warp keeps a + b, the upper one a - b
+// (a = lower warp's value, b = upper warp's).
 template <int NP>
-__device__ __forceinline__ void cross_butterfly(f32x2_t (&vp)[NP], const f32x2_t (&op)[NP], int member) {
-  const float sg = member ? -1.0f : 1.0f;
+__device__ __forceinline__ void cross_butterfly(f32x2_t (&vp)[NP], const f32x2_t (&op)[NP], bool upper) {
+  const float sg = upper ? -1.0f : 1.0f;
   const f32x2_t sg2 = pack2(sg, sg);
 #pragma unroll
   for (int k = 0; k < NP; ++k) vp[k] = fma2(sg2, vp[k], op[k]);
+}
+
+// The Hadamard stages over the index bits that separate the warps of a team (bits 8, 9), ascending.
+// kWithSum: the first exchange also publishes this warp's sum of squares; returns whether it did.
+template <int D, bool kWithSum>
+__device__ __forceinline__ bool team_cross_stages(const RowCtx& rc, TeamSmem<D>* ts,
+                                                  f32x2_t (&vp)[RowTeam<D>::NV / 2], float ss) {
+  using RT = RowTeam<D>;
+  bool published = false;
+#pragma unroll
+  for (int k = 0; k < RT::LOG_TEAM; ++k) {
+    if (8 + k < rc.log_h) {
+      f32x2_t op[RT::NV / 2];
+      if (kWithSum && k == 0) {
+        team_exchange<D, true>(rc, ts, rc.member ^ (1 << k), vp, op, ss);
+        published = true;
+      } else {
+        team_exchange<D, false>(rc, ts, rc.member ^ (1 << k), vp, op, 0.0f);
+      }
+      cross_butterfly<RT::NV / 2>(vp, op, (rc.member >> k) & 1);
+    }
+  }
+  return published;
 }
 
 // Q^-1 without the prediction for this warp's part of the row: `w` enters holding the gathered grid
@@ -339,14 +362,7 @@ __device__ __forceinline__ void team_rotate_back_and_scale(const RowCtx& rc, Tea
 #pragma unroll
   for (int k = 0; k < RT::NV / 2; ++k) wp[k] = pack2(w[2 * k], w[2 * k + 1]);
   fwht_packed<RT::NV>(wp, rc.log_h, rc.lane);
-  if constexpr (RT::TEAM == 2) {
-    if (RT::CROSS_BIT < rc.log_h) {
-      f32x2_t op[RT::NV / 2];
-      float dummy_a[RT::CPM] = {}, dummy_b[RT::CPM];
-      team_exchange<D, false>(rc, ts, wp, op, dummy_a, dummy_b);
-      cross_butterfly<RT::NV / 2>(wp, op, rc.member);
-    }
-  }
+  team_cross_stages<D, false>(rc, ts, wp, 0.0f);
   const f32x2_t rs2 = pack2(rc.rs, rc.rs);
 #pragma unroll
   for (int k = 0; k < RT::NV / 2; ++k) {
@@ -415,39 +431,25 @@ __device__ __forceinline__ void encode_row_core(const RowCtx& rc, const RowSmem<
 #pragma unroll
   for (int k = 0; k < NV / 2; ++k) vp[k] = pack2(v[2 * k], v[2 * k + 1]);
   fwht_packed<NV>(vp, rc.log_h, lane);
-  float all_ss[NC];
-#pragma unroll
-  for (int c = 0; c < NC; ++c) all_ss[c] = 0.0f;
-  if constexpr (RT::TEAM == 2) {
-    if (RT::CROSS_BIT < rc.log_g) {          // scale groups (and maybe Hadamard blocks) span both warps
-      f32x2_t op[NV / 2];
-      float oss[CPM];
-      team_exchange<D, true>(rc, ts, vp, op, ss, oss);
-      if (RT::CROSS_BIT < rc.log_h) cross_butterfly<NV / 2>(vp, op, rc.member);
-#pragma unroll
-      for (int c = 0; c < CPM; ++c) {
-        all_ss[c0 + c] = ss[c];
-        all_ss[(c0 ^ CPM) + c] = oss[c];
-      }
-    } else {
-#pragma unroll
-      for (int c = 0; c < CPM; ++c) all_ss[c0 + c] = ss[c];
-    }
-  } else {
-#pragma unroll
-    for (int c = 0; c < CPM; ++c) all_ss[c] = ss[c];
+  {
+    // stages across warps; the sums of squares travel with the first exchange when groups span warps
+    const bool need_sums = RT::TEAM > 1 && rc.log_g > 8;
+    bool published = false;
+    if (need_sums) published = team_cross_stages<D, true>(rc, ts, vp, ss[0]);
+    else team_cross_stages<D, false>(rc, ts, vp, 0.0f);
+    if (need_sums && !published) team_exchange_sums<D>(rc, ts, ss[0]);
   }
   // ---- group scale: root mean square, stored as fp16; normalise with the rounded value ----------
   float sf[CPM];
 #pragma unroll
   for (int c = 0; c < CPM; ++c) {
     float tot = ss[c];
-    if (rc.log_g > 8) {                      // groups of several chunks: add them in ascending order
+    if (RT::TEAM > 1 && rc.log_g > 8) {      // groups of several chunks: add them in ascending order
       const int cpg = 1 << (rc.log_g - 8);
       tot = 0.0f;
 #pragma unroll
       for (int c2 = 0; c2 < NC; ++c2)
-        if ((c2 / cpg) == ((c0 + c) / cpg)) tot += all_ss[c2];
+        if ((c2 / cpg) == ((c0 + c) / cpg)) tot += ts->ss[c2];
     }
     const float sc = fminf(sqrtf(tot * rc.inv_g), 65504.0f);
     const __half s16 = __float2half_rn(sc);

@@ -38,7 +38,7 @@
 
 namespace aquakv {
 
-constexpr int kRowWarps = 16;
+constexpr int kRowWarps = 24;
 constexpr int kLayerThreads = 32 * (6 + kRowWarps);
 constexpr int kLayerStages = 4;
 constexpr int kPairBBytes = (kBN / 2) * kBK * 2;        // this CTA's half of a weight tile k-block
@@ -454,7 +454,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       if constexpr (kEncode) {
         // pull this job's input rows towards L2 while the prediction is still being produced
         const uint16_t* xin = ph == 0 ? a.K : a.V;
-        for (int r = r_begin + team; r < r_end; r += TEAMS) {
+        for (int r = r_begin + (team + j) % TEAMS; r < r_end; r += TEAMS) {
           const long long g = (long long)m * kBM + r;
           if (lane < D / 256 / TEAM * 4)
             asm volatile("prefetch.global.L2 [%0];" ::"l"(xin + g * a.ldX + rck.member * (D / TEAM) + lane * 64));
@@ -463,18 +463,18 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       bool ok = true;
       if (lane == 0) ok = counter_wait_bounded(a.gemm_done + j * a.mw + rb, NTN, abort_flag, a.status);
       ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (TEAM == 2) {
-        // both warps of a team must take the same path: agree through shared memory
+      if (TEAM > 1) {
+        // all warps of a team must take the same path: agree through shared memory
         if (!ok) *abort_flag = 1;
-        team_barrier(rck.barrier);
+        team_barrier<D>(rck.barrier);
         ok = *abort_flag == 0;
-        team_barrier(rck.barrier);
+        team_barrier<D>(rck.barrier);
       }
       if (ok) {
         const float* pbuf = a.P + (size_t(j % a.nb) * a.mw * kBM + size_t(rb) * kBM) * D;
         const size_t khat_base = a.khat_ring ? size_t((wave % a.khat_ring) * a.mw + rb) * kBM
                                              : size_t(m) * kBM;
-        for (int r = r_begin + team; r < r_end; r += TEAMS) {
+        for (int r = r_begin + (team + j) % TEAMS; r < r_end; r += TEAMS) {   // rotated per job for balance
           const long long g = (long long)m * kBM + r;
           const float* pred_row = pbuf + size_t(r) * D;
           uint16_t* hat_row;
@@ -495,7 +495,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       // each team reports on its own, so a slow team never holds the others back
       __threadfence();
       fence_proxy_async_all();
-      if (TEAM == 2) team_barrier(rck.barrier); else __syncwarp();
+      if (TEAM > 1) team_barrier<D>(rck.barrier); else __syncwarp();
       if (*abort_flag) break;
       if (rck.member == 0 && lane == 0) atomicAdd(a.rows_done + j * a.mw + rb, 1);
     }
