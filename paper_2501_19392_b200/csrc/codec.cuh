@@ -249,11 +249,14 @@ struct RowTeam {
   static constexpr int NV = 8;                       // values per lane
 };
 
-// Exchange buffer of one team (only used when TEAM > 1).
+// Exchange buffers of one team (only used when TEAM > 1).  Two copies used alternately: a warp
+// writes copy n % 2 in its n-th exchange after passing the barrier of exchange n - 1, which every
+// warp reaches only after it has read copy n % 2 in exchange n - 2, so one barrier per exchange
+// is enough.
 template <int D>
 struct TeamSmem {
-  ulonglong2 x[RowTeam<D>::TEAM][RowTeam<D>::NV / 4][32];   // [member][16-byte piece][lane]
-  float ss[RowTeam<D>::TEAM];                               // [member] sum of squares of its chunk
+  ulonglong2 x[2][RowTeam<D>::TEAM][RowTeam<D>::NV / 4][32];   // [copy][member][16-byte piece][lane]
+  float ss[2][RowTeam<D>::TEAM];                               // [copy][member] sum of squares of its chunk
 };
 
 // Per-warp constants of the row routines.
@@ -266,6 +269,7 @@ struct RowCtx {
   int lane;
   int member;              // which chunk of the row this warp holds
   int barrier;             // named barrier shared by the warps of the team
+  mutable int xcopy;       // exchange-buffer copy the next exchange uses (same in all warps of a team)
 };
 
 // Fills the fields that depend only on the parameters and on the warp's place in its team.
@@ -275,6 +279,7 @@ __device__ __forceinline__ void row_ctx_init(RowCtx& rc, const uint32_t* signmas
   rc.lane = lane;
   rc.member = member;
   rc.barrier = barrier;
+  rc.xcopy = 0;
   rc.signmask = signmask[lane] >> (member * values_per_warp);
   rc.inv_w = inv_w;
   rc.log_h = log_h;
@@ -289,31 +294,36 @@ __device__ __forceinline__ void team_barrier(int id) {
 }
 
 // Publishes this warp's values (and optionally its sum of squares) and reads those of `partner`.
+// Returns the buffer copy that was used (the sums of all members can be read from it).
 template <int D, bool kWithSum>
-__device__ __forceinline__ void team_exchange(const RowCtx& rc, TeamSmem<D>* ts, int partner,
-                                              const f32x2_t (&vp)[RowTeam<D>::NV / 2],
-                                              f32x2_t (&op)[RowTeam<D>::NV / 2], float ss) {
+__device__ __forceinline__ int team_exchange(const RowCtx& rc, TeamSmem<D>* ts, int partner,
+                                             const f32x2_t (&vp)[RowTeam<D>::NV / 2],
+                                             f32x2_t (&op)[RowTeam<D>::NV / 2], float ss) {
   constexpr int NV = RowTeam<D>::NV;
-  team_barrier<D>(rc.barrier);             // everybody has finished reading the previous exchange
+  const int cp = rc.xcopy;
+  rc.xcopy ^= 1;
 #pragma unroll
   for (int q = 0; q < NV / 4; ++q)
-    ts->x[rc.member][q][rc.lane] = make_ulonglong2(vp[2 * q], vp[2 * q + 1]);
-  if (kWithSum && rc.lane == 0) ts->ss[rc.member] = ss;
+    ts->x[cp][rc.member][q][rc.lane] = make_ulonglong2(vp[2 * q], vp[2 * q + 1]);
+  if (kWithSum && rc.lane == 0) ts->ss[cp][rc.member] = ss;
   team_barrier<D>(rc.barrier);
 #pragma unroll
   for (int q = 0; q < NV / 4; ++q) {
-    const ulonglong2 t = ts->x[partner][q][rc.lane];
+    const ulonglong2 t = ts->x[cp][partner][q][rc.lane];
     op[2 * q] = t.x;
     op[2 * q + 1] = t.y;
   }
+  return cp;
 }
 
 // Publishes only the sums of squares (scale groups that span warps while Hadamard blocks do not).
 template <int D>
-__device__ __forceinline__ void team_exchange_sums(const RowCtx& rc, TeamSmem<D>* ts, float ss) {
+__device__ __forceinline__ int team_exchange_sums(const RowCtx& rc, TeamSmem<D>* ts, float ss) {
+  const int cp = rc.xcopy;
+  rc.xcopy ^= 1;
+  if (rc.lane == 0) ts->ss[cp][rc.member] = ss;
   team_barrier<D>(rc.barrier);
-  if (rc.lane == 0) ts->ss[rc.member] = ss;
-  team_barrier<D>(rc.barrier);
+  return cp;
 }
 
 // Butterfly over an index bit that separates warps: the lower warp keeps a + b, the upper one a - b
@@ -327,26 +337,26 @@ __device__ __forceinline__ void cross_butterfly(f32x2_t (&vp)[NP], const f32x2_t
 }
 
 // The Hadamard stages over the index bits that separate the warps of a team (bits 8, 9), ascending.
-// kWithSum: the first exchange also publishes this warp's sum of squares; returns whether it did.
+// kWithSum: the first exchange also publishes this warp's sum of squares; returns the buffer copy
+// holding the sums, or -1 if no exchange published them.
 template <int D, bool kWithSum>
-__device__ __forceinline__ bool team_cross_stages(const RowCtx& rc, TeamSmem<D>* ts,
-                                                  f32x2_t (&vp)[RowTeam<D>::NV / 2], float ss) {
+__device__ __forceinline__ int team_cross_stages(const RowCtx& rc, TeamSmem<D>* ts,
+                                                 f32x2_t (&vp)[RowTeam<D>::NV / 2], float ss) {
   using RT = RowTeam<D>;
-  bool published = false;
+  int sums_copy = -1;
 #pragma unroll
   for (int k = 0; k < RT::LOG_TEAM; ++k) {
     if (8 + k < rc.log_h) {
       f32x2_t op[RT::NV / 2];
       if (kWithSum && k == 0) {
-        team_exchange<D, true>(rc, ts, rc.member ^ (1 << k), vp, op, ss);
-        published = true;
+        sums_copy = team_exchange<D, true>(rc, ts, rc.member ^ (1 << k), vp, op, ss);
       } else {
         team_exchange<D, false>(rc, ts, rc.member ^ (1 << k), vp, op, 0.0f);
       }
       cross_butterfly<RT::NV / 2>(vp, op, (rc.member >> k) & 1);
     }
   }
-  return published;
+  return sums_copy;
 }
 
 // Q^-1 without the prediction for this warp's part of the row: `w` enters holding the gathered grid
@@ -431,13 +441,16 @@ __device__ __forceinline__ void encode_row_core(const RowCtx& rc, const RowSmem<
 #pragma unroll
   for (int k = 0; k < NV / 2; ++k) vp[k] = pack2(v[2 * k], v[2 * k + 1]);
   fwht_packed<NV>(vp, rc.log_h, lane);
+  int sums_copy = 0;
   {
     // stages across warps; the sums of squares travel with the first exchange when groups span warps
     const bool need_sums = RT::TEAM > 1 && rc.log_g > 8;
-    bool published = false;
-    if (need_sums) published = team_cross_stages<D, true>(rc, ts, vp, ss[0]);
-    else team_cross_stages<D, false>(rc, ts, vp, 0.0f);
-    if (need_sums && !published) team_exchange_sums<D>(rc, ts, ss[0]);
+    if (need_sums) {
+      sums_copy = team_cross_stages<D, true>(rc, ts, vp, ss[0]);
+      if (sums_copy < 0) sums_copy = team_exchange_sums<D>(rc, ts, ss[0]);
+    } else {
+      team_cross_stages<D, false>(rc, ts, vp, 0.0f);
+    }
   }
   // ---- group scale: root mean square, stored as fp16; normalise with the rounded value ----------
   float sf[CPM];
@@ -449,7 +462,7 @@ __device__ __forceinline__ void encode_row_core(const RowCtx& rc, const RowSmem<
       tot = 0.0f;
 #pragma unroll
       for (int c2 = 0; c2 < NC; ++c2)
-        if ((c2 / cpg) == ((c0 + c) / cpg)) tot += ts->ss[c2];
+        if ((c2 / cpg) == ((c0 + c) / cpg)) tot += ts->ss[sums_copy][c2];
     }
     const float sc = fminf(sqrtf(tot * rc.inv_g), 65504.0f);
     const __half s16 = __float2half_rn(sc);

@@ -434,9 +434,10 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
     constexpr int TEAM = RowTeam<D>::TEAM, TEAMS = kRowWarps / TEAM;
     const int rw = warp - 6;
     const int team = rw / TEAM;
-    RowCtx rck, rcv;
+    RowCtx rck;     // one context per warp; the sign bits are switched between key and value jobs
     row_ctx_init(rck, a.signmask_k, a.search.inv_w, a.log_h, a.log_g, lane, rw % TEAM, RowTeam<D>::NV, 3 + team);
-    row_ctx_init(rcv, a.signmask_v, a.search.inv_w, a.log_h, a.log_g, lane, rw % TEAM, RowTeam<D>::NV, 3 + team);
+    const uint32_t signs_k = rck.signmask;
+    const uint32_t signs_v = a.signmask_v[lane] >> (rck.member * RowTeam<D>::NV);
     TeamSmem<D>* ts = &rsm->team[team];
     const int n_groups = D >> a.log_g;
     for (int j = 0; j < n_jobs; ++j) {
@@ -444,6 +445,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       layer_job(j, a.n_waves, ph, wave);
       const WaveRows wr = wave_rows(wave, a.T, a.mw, gridDim.x);
       if (wr.tokens <= 0) continue;
+      rck.signmask = ph == 0 ? signs_k : signs_v;
       const int slot_row = (ml * NTN + n_blk) * wr.rpc;      // first row (within the wave) of this CTA's slice
       const int rb = slot_row / kBM;                         // token block (within the wave) the slice lies in
       if (rb >= wr.blocks) continue;                         // nothing assigned, nobody waits for this CTA
@@ -484,10 +486,10 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
           uint16_t* scales_row = (ph == 0 ? a.Kscales : a.Vscales) + g * n_groups;
           if constexpr (kEncode) {
             const uint16_t* x_row = (ph == 0 ? a.K : a.V) + g * a.ldX;
-            encode_row<D, NPTS, kBf16>(ph == 0 ? rck : rcv, &rsm->tables, ts, x_row, pred_row, codes_row,
+            encode_row<D, NPTS, kBf16>(rck, &rsm->tables, ts, x_row, pred_row, codes_row,
                                        scales_row, hat_row);
           } else {
-            decode_row<D, NPTS, kBf16>(ph == 0 ? rck : rcv, rsm->tables.grid, ts, codes_row, scales_row,
+            decode_row<D, NPTS, kBf16>(rck, rsm->tables.grid, ts, codes_row, scales_row,
                                        pred_row, hat_row);
           }
         }
