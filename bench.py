@@ -374,7 +374,8 @@ def main():
 def run_e2e(args, codec, chain, shape, kv, ad, cache, bufs, q, out, ctx_len, scale, dev, world):
     """Same step, but every input starts in pinned host memory and every product ends there:
     per layer H2D(K, V) -> encode -> D2H(codes, scales); then H2D(codes, scales, q) -> decode +
-    attention -> D2H(attention output).  Copies are inside the timed region."""
+    attention -> D2H(attention output).  Copies are inside the timed region (on copy streams that
+    the timed stream waits for)."""
     T, L, d = shape.n_tokens, shape.n_layers, shape.d_kv
     pin = lambda t: torch.empty(t.shape, dtype=t.dtype, device="cpu", pin_memory=True).copy_(t)
     hK = [pin(t) for t in kv.K]
@@ -383,35 +384,76 @@ def run_e2e(args, codec, chain, shape, kv, ad, cache, bufs, q, out, ctx_len, sca
     hc = [[torch.empty(t.shape, dtype=t.dtype, device="cpu", pin_memory=True) for t in lst]
           for lst in (cache.Kcodes, cache.Kscales, cache.Vcodes, cache.Vscales)]
     ho = [torch.empty(t.shape, dtype=t.dtype, device="cpu", pin_memory=True) for t in out]
-    dK = torch.empty_like(kv.K[0])
-    dV = torch.empty_like(kv.V[0])
-    dq = torch.empty_like(q[0])
+    # Copies run on their own streams (PCIe is full duplex) and overlap the kernels of other layers:
+    # inputs are double-buffered on the device, events order copy -> kernel -> copy per layer.
+    dK = [torch.empty_like(kv.K[0]) for _ in range(2)]
+    dV = [torch.empty_like(kv.V[0]) for _ in range(2)]
+    dq = [torch.empty_like(q[0]) for _ in range(2)]
     dlists = (cache.Kcodes, cache.Kscales, cache.Vcodes, cache.Vscales)
+    main = torch.cuda.current_stream()
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    ev = lambda: torch.cuda.Event()
 
     def e2e_step():
+        start = ev()
+        start.record(main)
+        s_in.wait_event(start)
+        s_out.wait_event(start)
+        used = [None, None]            # event: the kernel that last read input buffer b has been issued
+        d2h_done = []
         for l in range(L):
-            dK.copy_(hK[l], non_blocking=True)
-            dV.copy_(hV[l], non_blocking=True)
+            b = l % 2
+            with torch.cuda.stream(s_in):
+                if used[b] is not None:
+                    s_in.wait_event(used[b])
+                dK[b].copy_(hK[l], non_blocking=True)
+                dV[b].copy_(hV[l], non_blocking=True)
+                arrived = ev()
+                arrived.record(s_in)
+            main.wait_event(arrived)
             cur, prv = l % 2, (l + 1) % 2
             has = l > 0
-            codec.encode(dK, dV, bufs.K[prv] if has else None, bufs.V[prv] if has else None,
+            codec.encode(dK[b], dV[b], bufs.K[prv] if has else None, bufs.V[prv] if has else None,
                          ad.Wk[l] if has else None, ad.Wv[l] if has else None, None, None,
                          cache.Kcodes[l], cache.Kscales[l], cache.Vcodes[l], cache.Vscales[l],
                          bufs.K[cur], bufs.V[cur])
-            for h, dl in zip(hc, dlists):
-                h[l].copy_(dl[l], non_blocking=True)
+            used[b] = ev()
+            used[b].record(main)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(used[b])
+                for h, dl in zip(hc, dlists):
+                    h[l].copy_(dl[l], non_blocking=True)
+                done = ev()
+                done.record(s_out)
+                d2h_done.append(done)
+        usedq = [None, None]
         for l in range(L):
-            for h, dl in zip(hc, dlists):
-                dl[l].copy_(h[l], non_blocking=True)
-            dq.copy_(hq[l], non_blocking=True)
+            b = l % 2
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(d2h_done[l])          # the codes of this layer have reached the host
+                if usedq[b] is not None:
+                    s_in.wait_event(usedq[b])
+                for h, dl in zip(hc, dlists):
+                    dl[l].copy_(h[l], non_blocking=True)
+                dq[b].copy_(hq[l], non_blocking=True)
+                arrived = ev()
+                arrived.record(s_in)
+            main.wait_event(arrived)
             cur, prv = l % 2, (l + 1) % 2
             has = l > 0
-            codec.decode_attn(dq, cache.Kcodes[l], cache.Kscales[l], cache.Vcodes[l], cache.Vscales[l],
+            codec.decode_attn(dq[b], cache.Kcodes[l], cache.Kscales[l], cache.Vcodes[l], cache.Vscales[l],
                               ctx_len, shape.n_kv_heads, scale,
                               bufs.K[prv] if has else None, bufs.V[prv] if has else None,
                               ad.Wk[l] if has else None, ad.Wv[l] if has else None, None, None,
                               out=out[l], Khat=bufs.K[cur], Vhat=bufs.V[cur])
-            ho[l].copy_(out[l], non_blocking=True)
+            usedq[b] = ev()
+            usedq[b].record(main)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(usedq[b])
+                ho[l].copy_(out[l], non_blocking=True)
+        end_out = ev()
+        end_out.record(s_out)
+        main.wait_event(end_out)              # the step ends when its last result is on the host
 
     nbytes = lambda ts: sum(t.numel() * t.element_size() for t in ts)
     code_bytes = sum(nbytes(lst) for lst in hc)
