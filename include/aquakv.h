@@ -95,8 +95,9 @@ int aquakv_create(const aquakv_params* params, const float* grid_host, const int
  * rotated values goes to the nearest grid point).  The square [-half_extent, half_extent)^2 is cut
  * into cells_per_side^2 cells; entry [iy*cells_per_side + ix] holds, in bytes 0..3, the ascending
  * indices of every grid point that is nearest somewhere in that cell (short lists repeat the last
- * index; at most three distinct ones for grid_size 16, four otherwise), and the value 1 means
- * "more than that: search all points".  The kernels use the same
+ * index; at most three distinct ones for grid_size 16, four otherwise), and 0xFFFFFFFF means "search
+ * all points" (cells with more candidates, and the border cells, which also stand for everything
+ * outside the square).  The kernels use the same
  * table, so a host test can check that it never excludes the true nearest point.  HOST memory
  * only, no GPU needed.  table == NULL: only report the dimensions.
  */

@@ -18,60 +18,6 @@
 
 namespace aquakv {
 
-constexpr int kCodecWarps = 8;
-constexpr int kCodecThreads = kCodecWarps * 32;
-
-// Nearest-point search.  dist_i(y) = (y0 - g_i.x)^2 + (y1 - g_i.y)^2; the lowest index wins ties.
-// A cell table built on the host (search_table.h) lists, for the cell that holds y, every point
-// that can win there, so only three (n = 16) or four distances are evaluated; cells with more candidates and
-// values outside the table's square fall back to the exhaustive loop.  Both paths evaluate the same
-// fp32 expression, so the result is the exhaustive arg-min bit for bit.  The table (64 x 64
-// entries) and the grid live in shared memory: the row kernels are bound by the load/store and
-// shuffle pipe, and shared-memory gathers of 4 and 8 bytes cost far fewer cycles there than
-// global gathers or 16-byte records.
-constexpr int kSearchCells = 64;          // cells per side of the table (see search_table.h)
-constexpr int kSearchLogCells = 6;
-constexpr uint32_t kCellBruteDev = 1u;    // the one non-ascending entry: search all points
-
-struct SearchDev {
-  const uint32_t* table;   // global copy [64*64] of the candidate lists
-  float inv_w;             // cells / (2 * half extent)
-};
-
-// Shared-memory tables of the row routines.
-template <int NPTS>
-struct RowSmem {
-  uint32_t table[kSearchCells * kSearchCells];
-  float2 grid[NPTS];
-};
-
-template <int NPTS>
-__device__ __forceinline__ void row_smem_fill(RowSmem<NPTS>* rs, const uint32_t* table, const float4* grid4) {
-  for (int i = threadIdx.x; i < kSearchCells * kSearchCells; i += blockDim.x) rs->table[i] = table[i];
-  for (int i = threadIdx.x; i < NPTS; i += blockDim.x) {
-    const float4 g = grid4[i];
-    rs->grid[i] = make_float2(g.x, g.y);
-  }
-}
-
-struct CodecArgs {
-  const uint16_t* X;        // encode: target rows (16-bit)              [T, ldX]
-  long long ldX;
-  const float* P;           // prediction rows (fp32) or nullptr          [T, ldP]
-  long long ldP;
-  const uint32_t* signmask; // [32]: bit (c*8+i) of entry `lane` set <=> sign of element
-                            //       c*256 + lane*8 + i is -1
-  const float4* grid4;      // [n]: (g_x, g_y, 0, 0)
-  SearchDev search;
-  uint8_t* codes;           // [T, code_bytes]
-  uint16_t* scales;         // [T, D/G] fp16 bits
-  uint16_t* hat;            // reconstruction rows (16-bit) or nullptr    [T, ldHat]
-  long long ldHat;
-  int T;
-  int log_h;                // log2 of the Hadamard block
-  int log_g;                // log2 of the scale group
-};
-
 // Packed pairs of fp32 values: sm_100 executes add/sub/fma on two fp32 lanes of a 64-bit register
 // pair in one instruction (add.f32x2 / fma.rn.f32x2), each lane rounded exactly like the scalar
 // operation.  The rotation keeps (v[2k], v[2k+1]) packed, which halves its arithmetic instructions.
@@ -104,6 +50,60 @@ __device__ __forceinline__ f32x2_t mul2(f32x2_t a, f32x2_t b) {
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
   return r;
 }
+
+constexpr int kCodecWarps = 8;
+constexpr int kCodecThreads = kCodecWarps * 32;
+
+// Nearest-point search.  dist_i(y) = (y0 - g_i.x)^2 + (y1 - g_i.y)^2; the lowest index wins ties.
+// A cell table built on the host (search_table.h) lists, for the cell that holds y, every point
+// that can win there, so only three (n = 16) or four distances are evaluated; cells with more candidates and
+// values outside the table's square fall back to the exhaustive loop.  Both paths evaluate the same
+// fp32 expression, so the result is the exhaustive arg-min bit for bit.  The table (64 x 64
+// entries) and the grid live in shared memory: the row kernels are bound by the load/store and
+// shuffle pipe, and shared-memory gathers of 4 and 8 bytes cost far fewer cycles there than
+// global gathers or 16-byte records.
+constexpr int kSearchCells = 64;          // cells per side of the table (see search_table.h)
+constexpr int kSearchLogCells = 6;
+constexpr uint32_t kCellBruteDev = 0xFFFFFFFFu;   // "search all points" (the largest entry value)
+
+struct SearchDev {
+  const uint32_t* table;   // global copy [64*64] of the candidate lists
+  float inv_w;             // cells / (2 * half extent)
+};
+
+// Shared-memory tables of the row routines.
+template <int NPTS>
+struct RowSmem {
+  uint32_t table[kSearchCells * kSearchCells];
+  f32x2_t grid[NPTS];      // (g.x, g.y) as packed fp32 pairs
+};
+
+template <int NPTS>
+__device__ __forceinline__ void row_smem_fill(RowSmem<NPTS>* rs, const uint32_t* table, const float4* grid4) {
+  for (int i = threadIdx.x; i < kSearchCells * kSearchCells; i += blockDim.x) rs->table[i] = table[i];
+  for (int i = threadIdx.x; i < NPTS; i += blockDim.x) {
+    const float4 g = grid4[i];
+    rs->grid[i] = pack2(g.x, g.y);
+  }
+}
+
+struct CodecArgs {
+  const uint16_t* X;        // encode: target rows (16-bit)              [T, ldX]
+  long long ldX;
+  const float* P;           // prediction rows (fp32) or nullptr          [T, ldP]
+  long long ldP;
+  const uint32_t* signmask; // [32]: bit (c*8+i) of entry `lane` set <=> sign of element
+                            //       c*256 + lane*8 + i is -1
+  const float4* grid4;      // [n]: (g_x, g_y, 0, 0)
+  SearchDev search;
+  uint8_t* codes;           // [T, code_bytes]
+  uint16_t* scales;         // [T, D/G] fp16 bits
+  uint16_t* hat;            // reconstruction rows (16-bit) or nullptr    [T, ldHat]
+  long long ldHat;
+  int T;
+  int log_h;                // log2 of the Hadamard block
+  int log_g;                // log2 of the scale group
+};
 
 // Hadamard butterflies of one warp's NV values per lane (element index bits 0-2 in registers,
 // 3-7 across lanes, the next bit between the warp's two chunks when NV == 16), by ascending bit.
@@ -193,47 +193,48 @@ __device__ __forceinline__ void store_code_word(uint8_t* row_codes, int chunk, i
   }
 }
 
-// Cell-table entry of one value pair (marked exhaustive outside the square).
+// Cell-table entry of one value pair.  The cell coordinates saturate at the table's border cells,
+// which the host marks "search all points", so values outside the square need no separate test.
 __device__ __forceinline__ uint32_t search_entry(float y0, float y1, float inv_w,
                                                  const uint32_t* __restrict__ table_s) {
-  const int ix = __float2int_rd(fmaf(y0, inv_w, 0.5f * kSearchCells));
-  const int iy = __float2int_rd(fmaf(y1, inv_w, 0.5f * kSearchCells));
-  const bool inside = static_cast<unsigned>(ix | iy) < unsigned(kSearchCells);
-  const uint32_t e = table_s[inside ? ((iy << kSearchLogCells) + ix) : 0];
-  return inside ? e : kCellBruteDev;
+  const unsigned ix = min(__float2uint_rd(fmaf(y0, inv_w, 0.5f * kSearchCells)), unsigned(kSearchCells - 1));
+  const unsigned iy = min(__float2uint_rd(fmaf(y1, inv_w, 0.5f * kSearchCells)), unsigned(kSearchCells - 1));
+  return table_s[(iy << kSearchLogCells) + ix];
 }
 
-__device__ __forceinline__ float pair_dist(float y0, float y1, float2 g) {
-  const float dx = __fsub_rn(y0, g.x), dy = __fsub_rn(y1, g.y);
-  return fmaf(dy, dy, __fmul_rn(dx, dx));
+// Squared distance of the packed pair y to the grid point g (both as packed fp32 pairs).
+__device__ __forceinline__ float pair_dist(f32x2_t y, f32x2_t g) {
+  const f32x2_t d = sub2(y, g);
+  float qx, qy;
+  unpack2(mul2(d, d), qx, qy);
+  return __fadd_rn(qx, qy);
 }
 
 // Arg-min over the ascending candidates of a table entry (three for n = 16, else four).
 template <int NPTS>
-__device__ __forceinline__ int nearest_of_candidates(float y0, float y1, uint32_t e,
-                                                     const float2* __restrict__ grid_s) {
+__device__ __forceinline__ int nearest_of_candidates(f32x2_t y, uint32_t e, const f32x2_t* __restrict__ grid_s) {
   const int c0 = e & 0xffu, c1 = (e >> 8) & 0xffu, c2 = (e >> 16) & 0xffu;
-  const float t0 = pair_dist(y0, y1, grid_s[c0]);
-  const float t1 = pair_dist(y0, y1, grid_s[c1]);
-  const float t2 = pair_dist(y0, y1, grid_s[c2]);
+  const float t0 = pair_dist(y, grid_s[c0]);
+  const float t1 = pair_dist(y, grid_s[c1]);
+  const float t2 = pair_dist(y, grid_s[c2]);
   int idx = c0;
   float best = t0;
   if (t1 < best) { best = t1; idx = c1; }
   if (t2 < best) { best = t2; idx = c2; }
   if constexpr (NPTS > 16) {
     const int c3 = e >> 24;
-    const float t3 = pair_dist(y0, y1, grid_s[c3]);
+    const float t3 = pair_dist(y, grid_s[c3]);
     if (t3 < best) { idx = c3; }
   }
   return idx;
 }
 
 template <int NPTS>
-__device__ __noinline__ int nearest_exhaustive(float y0, float y1, const float2* __restrict__ grid_s) {
+__device__ __noinline__ int nearest_exhaustive(f32x2_t y, const f32x2_t* __restrict__ grid_s) {
   float best = 3.0e38f;
   int idx = 0;
   for (int i = 0; i < NPTS; ++i) {
-    const float t = pair_dist(y0, y1, grid_s[i]);
+    const float t = pair_dist(y, grid_s[i]);
     if (t < best) { best = t; idx = i; }             // strict: lowest index wins ties
   }
   return idx;
@@ -261,7 +262,7 @@ struct TeamSmem {
 
 // Per-warp constants of the row routines.
 struct RowCtx {
-  uint32_t signmask;       // this lane's sign bits for this warp's values: bit i <=> value i is flipped
+  f32x2_t sgn2[4];         // this lane's Hadamard signs as packed (+-1, +-1) multipliers, pair k = values 2k, 2k+1
   float inv_w;             // SearchDev::inv_w
   float inv_g;             // 1 / scale group
   float rs;                // 1 / sqrt(Hadamard block)
@@ -272,6 +273,13 @@ struct RowCtx {
   mutable int xcopy;       // exchange-buffer copy the next exchange uses (same in all warps of a team)
 };
 
+// bits: bit i set <=> value i of this lane is multiplied by -1.
+__device__ __forceinline__ void row_ctx_set_signs(RowCtx& rc, uint32_t bits) {
+#pragma unroll
+  for (int k = 0; k < 4; ++k)
+    rc.sgn2[k] = pack2((bits >> (2 * k)) & 1u ? -1.0f : 1.0f, (bits >> (2 * k + 1)) & 1u ? -1.0f : 1.0f);
+}
+
 // Fills the fields that depend only on the parameters and on the warp's place in its team.
 __device__ __forceinline__ void row_ctx_init(RowCtx& rc, const uint32_t* signmask, float inv_w, int log_h,
                                              int log_g, int lane, int member, int values_per_warp,
@@ -280,7 +288,7 @@ __device__ __forceinline__ void row_ctx_init(RowCtx& rc, const uint32_t* signmas
   rc.member = member;
   rc.barrier = barrier;
   rc.xcopy = 0;
-  rc.signmask = signmask[lane] >> (member * values_per_warp);
+  row_ctx_set_signs(rc, signmask[lane] >> (member * values_per_warp));
   rc.inv_w = inv_w;
   rc.log_h = log_h;
   rc.log_g = log_g;
@@ -359,29 +367,35 @@ __device__ __forceinline__ int team_cross_stages(const RowCtx& rc, TeamSmem<D>* 
   return sums_copy;
 }
 
-// Q^-1 without the prediction for this warp's part of the row: `w` enters holding the gathered grid
-// coordinates and leaves holding xhat.  The operation order (rotation stages by ascending index bit,
-// multiply by 1/sqrt(h), then by the scale, sign flip) is shared by encode and decode so that both
-// produce bit-identical reconstructions.
+// Q^-1 without the prediction for this warp's chunk of the row: `wp` enters holding the gathered grid
+// points (packed pairs) and leaves holding xhat.  The operation order (rotation stages by ascending
+// index bit, multiply by 1/sqrt(h), then by the signed scale) is shared by encode and decode so that
+// both produce bit-identical reconstructions.
 template <int D>
 __device__ __forceinline__ void team_rotate_back_and_scale(const RowCtx& rc, TeamSmem<D>* ts,
-                                                           float (&w)[RowTeam<D>::NV],
-                                                           const float (&sf)[RowTeam<D>::CPM]) {
-  using RT = RowTeam<D>;
-  f32x2_t wp[RT::NV / 2];
-#pragma unroll
-  for (int k = 0; k < RT::NV / 2; ++k) wp[k] = pack2(w[2 * k], w[2 * k + 1]);
-  fwht_packed<RT::NV>(wp, rc.log_h, rc.lane);
+                                                           f32x2_t (&wp)[4], float scale) {
+  fwht_packed<8>(wp, rc.log_h, rc.lane);
   team_cross_stages<D, false>(rc, ts, wp, 0.0f);
-  const f32x2_t rs2 = pack2(rc.rs, rc.rs);
+  const f32x2_t rs2 = pack2(rc.rs, rc.rs), s2 = pack2(scale, scale);
 #pragma unroll
-  for (int k = 0; k < RT::NV / 2; ++k) {
-    const float s = sf[(2 * k) >> 3];
-    float a, b;
-    unpack2(mul2(mul2(wp[k], rs2), pack2(s, s)), a, b);
-    w[2 * k] = apply_sign(a, rc.signmask, 2 * k);
-    w[2 * k + 1] = apply_sign(b, rc.signmask, 2 * k + 1);
+  for (int k = 0; k < 4; ++k) wp[k] = mul2(mul2(wp[k], rs2), mul2(s2, rc.sgn2[k]));
+}
+
+// (lo, hi) 16-bit values of a 32-bit word as a packed fp32 pair.
+template <bool kBf16>
+__device__ __forceinline__ f32x2_t load16x2(uint32_t w) {
+  if constexpr (kBf16) {
+    return pack2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+  } else {
+    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w));
+    return pack2(f.x, f.y);
   }
+}
+template <bool kBf16>
+__device__ __forceinline__ uint32_t store16x2p(f32x2_t v) {
+  float lo, hi;
+  unpack2(v, lo, hi);
+  return store16x2<kBf16>(lo, hi);
 }
 
 // This warp's part of one token row of Q and of the reconstruction (Algorithm 2 lines 6-7 / 9):
@@ -393,81 +407,73 @@ __device__ __forceinline__ void team_rotate_back_and_scale(const RowCtx& rc, Tea
 // another SM of the same kernel just before.  Both warps of a team must call this together.
 template <int D, int NPTS, bool kBf16, typename AfterLoad>
 __device__ __forceinline__ void encode_row_core(const RowCtx& rc, const RowSmem<NPTS>* __restrict__ rsm,
-                                                TeamSmem<D>* ts, const uint4 (&raw)[RowTeam<D>::CPM],
-                                                const float4 (&pq0)[RowTeam<D>::CPM][2],
+                                                TeamSmem<D>* ts, const uint4 (&raw)[1],
+                                                const float4 (&pq0)[1][2],
                                                 const float* __restrict__ pred_row,
                                                 uint8_t* __restrict__ codes_row,
                                                 uint16_t* __restrict__ scales_row,
                                                 uint16_t* __restrict__ hat_row, AfterLoad after_load) {
   using RT = RowTeam<D>;
-  constexpr int NC = RT::NC, CPM = RT::CPM, NV = RT::NV;
+  constexpr int NC = RT::NC;
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
   const int lane = rc.lane;
-  const int c0 = rc.member * CPM;                    // first chunk of this warp
-  float v[NV];
+  const int cg = rc.member;                          // this warp's chunk
   // ---- residual r = x - pred (raw = this lane's 16-bit inputs, pq0 = its prediction values) -----
+  f32x2_t vp[4];
+  {
+    const uint32_t w[4] = {raw[0].x, raw[0].y, raw[0].z, raw[0].w};
 #pragma unroll
-  for (int c = 0; c < CPM; ++c) {
-    const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      v[c * 8 + 2 * i] = load16<kBf16>(uint16_t(w[i] & 0xffffu));
-      v[c * 8 + 2 * i + 1] = load16<kBf16>(uint16_t(w[i] >> 16));
-    }
+    for (int k = 0; k < 4; ++k) vp[k] = load16x2<kBf16>(w[k]);
     if (pred_row != nullptr) {
-      const float pp[8] = {pq0[c][0].x, pq0[c][0].y, pq0[c][0].z, pq0[c][0].w,
-                           pq0[c][1].x, pq0[c][1].y, pq0[c][1].z, pq0[c][1].w};
-#pragma unroll
-      for (int i = 0; i < 8; ++i) v[c * 8 + i] = __fsub_rn(v[c * 8 + i], pp[i]);
+      vp[0] = sub2(vp[0], pack2(pq0[0][0].x, pq0[0][0].y));
+      vp[1] = sub2(vp[1], pack2(pq0[0][0].z, pq0[0][0].w));
+      vp[2] = sub2(vp[2], pack2(pq0[0][1].x, pq0[0][1].y));
+      vp[3] = sub2(vp[3], pack2(pq0[0][1].z, pq0[0][1].w));
     }
   }
   after_load();   // raw and pq0 are consumed: the caller may start fetching the next row's inputs
-  // ---- per-chunk sums of squares (lane bits reduced by shuffles), sign flip ---------------------
-  float ss[CPM];
+  // ---- sum of squares of the chunk (lane bits reduced by shuffles), sign flip --------------------
+  float ss;
+  {
+    f32x2_t acc = mul2(vp[0], vp[0]);
 #pragma unroll
-  for (int c = 0; c < CPM; ++c) {
-    float s = 0.0f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) s = fmaf(v[c * 8 + i], v[c * 8 + i], s);
+    for (int k = 1; k < 4; ++k) acc = fma2(vp[k], vp[k], acc);
+    float lo, hi;
+    unpack2(acc, lo, hi);
+    ss = lo + hi;
 #pragma unroll
     for (int b = 3; b < 8; ++b)
-      if (b < rc.log_g) s += __shfl_xor_sync(0xffffffffu, s, 1 << (b - 3));
-    ss[c] = s;
+      if (b < rc.log_g) ss += __shfl_xor_sync(0xffffffffu, ss, 1 << (b - 3));
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[c * 8 + i] = apply_sign(v[c * 8 + i], rc.signmask, c * 8 + i);
+    for (int k = 0; k < 4; ++k) vp[k] = mul2(vp[k], rc.sgn2[k]);
   }
   // ---- rotate (the division by the scale is applied afterwards: the rotation is linear) ---------
-  f32x2_t vp[NV / 2];
-#pragma unroll
-  for (int k = 0; k < NV / 2; ++k) vp[k] = pack2(v[2 * k], v[2 * k + 1]);
-  fwht_packed<NV>(vp, rc.log_h, lane);
+  fwht_packed<8>(vp, rc.log_h, lane);
   int sums_copy = 0;
   {
     // stages across warps; the sums of squares travel with the first exchange when groups span warps
     const bool need_sums = RT::TEAM > 1 && rc.log_g > 8;
     if (need_sums) {
-      sums_copy = team_cross_stages<D, true>(rc, ts, vp, ss[0]);
-      if (sums_copy < 0) sums_copy = team_exchange_sums<D>(rc, ts, ss[0]);
+      sums_copy = team_cross_stages<D, true>(rc, ts, vp, ss);
+      if (sums_copy < 0) sums_copy = team_exchange_sums<D>(rc, ts, ss);
     } else {
       team_cross_stages<D, false>(rc, ts, vp, 0.0f);
     }
   }
   // ---- group scale: root mean square, stored as fp16; normalise with the rounded value ----------
-  float sf[CPM];
-#pragma unroll
-  for (int c = 0; c < CPM; ++c) {
-    float tot = ss[c];
+  float sf;
+  {
+    float tot = ss;
     if (RT::TEAM > 1 && rc.log_g > 8) {      // groups of several chunks: add them in ascending order
       const int cpg = 1 << (rc.log_g - 8);
       tot = 0.0f;
 #pragma unroll
       for (int c2 = 0; c2 < NC; ++c2)
-        if ((c2 / cpg) == ((c0 + c) / cpg)) tot += ts->ss[sums_copy][c2];
+        if ((c2 / cpg) == (cg / cpg)) tot += ts->ss[sums_copy][c2];
     }
     const float sc = fminf(sqrtf(tot * rc.inv_g), 65504.0f);
     const __half s16 = __float2half_rn(sc);
-    sf[c] = __half2float(s16);
-    const int cg = c0 + c;
+    sf = __half2float(s16);
     if (rc.log_g >= 8) {                     // one lane per group writes the scale
       const int cpg = 1 << (rc.log_g - 8);
       if (lane == 0 && (cg % cpg) == 0) scales_row[cg / cpg] = __half_as_ushort(s16);
@@ -475,66 +481,53 @@ __device__ __forceinline__ void encode_row_core(const RowCtx& rc, const RowSmem<
       const int lpg = 1 << (rc.log_g - 3);   // lanes per group
       if ((lane % lpg) == 0) scales_row[cg * (256 >> rc.log_g) + lane / lpg] = __half_as_ushort(s16);
     }
-    const float inv = (sf[c] > 0.0f ? __frcp_rn(sf[c]) : 0.0f) * rc.rs;
+    const float inv = (sf > 0.0f ? __frcp_rn(sf) : 0.0f) * rc.rs;
     const f32x2_t inv2 = pack2(inv, inv);
 #pragma unroll
-    for (int k = 0; k < 4; ++k) unpack2(mul2(vp[c * 4 + k], inv2), v[c * 8 + 2 * k], v[c * 8 + 2 * k + 1]);
+    for (int k = 0; k < 4; ++k) vp[k] = mul2(vp[k], inv2);
   }
   // the prediction is needed again for the reconstruction: start reading it now, the search hides it
-  float4 pq[CPM][2];
+  float4 pq[2];
   if (hat_row != nullptr && pred_row != nullptr) {
-#pragma unroll
-    for (int c = 0; c < CPM; ++c) {
-      pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + lane * 8));
-      pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + lane * 8 + 4));
-    }
+    pq[0] = __ldcg(reinterpret_cast<const float4*>(pred_row + cg * 256 + lane * 8));
+    pq[1] = __ldcg(reinterpret_cast<const float4*>(pred_row + cg * 256 + lane * 8 + 4));
   } else {
-#pragma unroll
-    for (int c = 0; c < CPM; ++c) pq[c][0] = pq[c][1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    pq[0] = pq[1] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
   }
   // ---- nearest grid point per pair: all table entries first, then the candidates ----------------
-  uint32_t entry[NV / 2];
-  uint32_t any_brute = 0;
+  uint32_t entry[4];
+  uint32_t emax = 0;
 #pragma unroll
-  for (int j = 0; j < NV / 2; ++j) {
-    entry[j] = search_entry(v[2 * j], v[2 * j + 1], rc.inv_w, rsm->table);
-    any_brute |= uint32_t(entry[j] == kCellBruteDev);
+  for (int k = 0; k < 4; ++k) {
+    float y0, y1;
+    unpack2(vp[k], y0, y1);
+    entry[k] = search_entry(y0, y1, rc.inv_w, rsm->table);
+    emax = max(emax, entry[k]);
   }
-  const bool slow = __any_sync(0xffffffffu, any_brute != 0);
+  const bool slow = __any_sync(0xffffffffu, emax == kCellBruteDev);
+  uint32_t word = 0;
 #pragma unroll
-  for (int c = 0; c < CPM; ++c) {
-    uint32_t word = 0;
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const int j = c * 4 + k;
-      int idx;
-      if (!slow) {
-        idx = nearest_of_candidates<NPTS>(v[2 * j], v[2 * j + 1], entry[j], rsm->grid);
-      } else {
-        idx = entry[j] == kCellBruteDev
-                  ? nearest_exhaustive<NPTS>(v[2 * j], v[2 * j + 1], rsm->grid)
-                  : nearest_of_candidates<NPTS>(v[2 * j], v[2 * j + 1], entry[j], rsm->grid);
-      }
-      word |= uint32_t(idx) << (k * BITS);
-      const float2 g = rsm->grid[idx];
-      v[2 * j] = g.x;
-      v[2 * j + 1] = g.y;
+  for (int k = 0; k < 4; ++k) {
+    int idx;
+    if (!slow) {
+      idx = nearest_of_candidates<NPTS>(vp[k], entry[k], rsm->grid);
+    } else {
+      idx = entry[k] == kCellBruteDev ? nearest_exhaustive<NPTS>(vp[k], rsm->grid)
+                                      : nearest_of_candidates<NPTS>(vp[k], entry[k], rsm->grid);
     }
-    store_code_word<BITS>(codes_row, c0 + c, lane, word);
+    word |= uint32_t(idx) << (k * BITS);
+    vp[k] = rsm->grid[idx];
   }
+  store_code_word<BITS>(codes_row, cg, lane, word);
   // ---- reconstruction: hat = round16(pred + Q^-1(codes)) ---------------------------------------
   if (hat_row != nullptr) {      // uniform over the team
-    team_rotate_back_and_scale<D>(rc, ts, v, sf);
-#pragma unroll
-    for (int c = 0; c < CPM; ++c) {
-      const float pp[8] = {pq[c][0].x, pq[c][0].y, pq[c][0].z, pq[c][0].w,
-                           pq[c][1].x, pq[c][1].y, pq[c][1].z, pq[c][1].w};
-      uint32_t o[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        o[i] = store16x2<kBf16>(__fadd_rn(pp[2 * i], v[c * 8 + 2 * i]), __fadd_rn(pp[2 * i + 1], v[c * 8 + 2 * i + 1]));
-      *reinterpret_cast<uint4*>(hat_row + (c0 + c) * 256 + lane * 8) = make_uint4(o[0], o[1], o[2], o[3]);
-    }
+    team_rotate_back_and_scale<D>(rc, ts, vp, sf);
+    uint32_t o[4];
+    o[0] = store16x2p<kBf16>(add2(pack2(pq[0].x, pq[0].y), vp[0]));
+    o[1] = store16x2p<kBf16>(add2(pack2(pq[0].z, pq[0].w), vp[1]));
+    o[2] = store16x2p<kBf16>(add2(pack2(pq[1].x, pq[1].y), vp[2]));
+    o[3] = store16x2p<kBf16>(add2(pack2(pq[1].z, pq[1].w), vp[3]));
+    *reinterpret_cast<uint4*>(hat_row + cg * 256 + lane * 8) = make_uint4(o[0], o[1], o[2], o[3]);
   }
 }
 
@@ -603,38 +596,23 @@ __global__ void __launch_bounds__(kCodecThreads, 2) encode_rows_kernel(const Cod
 // scale of each chunk; get_pred(pq) delivers the prediction values of this lane just before they are
 // added, so a caller can fetch them while the rotation runs.
 template <int D, int NPTS, bool kBf16, typename GetPred>
-__device__ __forceinline__ void decode_row_core(const RowCtx& rc, const float2* __restrict__ grid_s,
-                                                TeamSmem<D>* ts, const uint32_t (&words)[RowTeam<D>::CPM],
-                                                const float (&sf)[RowTeam<D>::CPM], GetPred get_pred,
+__device__ __forceinline__ void decode_row_core(const RowCtx& rc, const f32x2_t* __restrict__ grid_s,
+                                                TeamSmem<D>* ts, const uint32_t (&words)[1],
+                                                const float (&sf)[1], GetPred get_pred,
                                                 uint16_t* __restrict__ hat_row) {
-  using RT = RowTeam<D>;
-  constexpr int CPM = RT::CPM, NV = RT::NV;
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
-  const int lane = rc.lane;
-  const int c0 = rc.member * CPM;
-  float w[NV];
+  f32x2_t wp[4];
 #pragma unroll
-  for (int c = 0; c < CPM; ++c) {
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const float2 g = grid_s[(words[c] >> (k * BITS)) & (NPTS - 1)];
-      w[c * 8 + 2 * k] = g.x;
-      w[c * 8 + 2 * k + 1] = g.y;
-    }
-  }
-  team_rotate_back_and_scale<D>(rc, ts, w, sf);
-  float4 pq[CPM][2];
+  for (int k = 0; k < 4; ++k) wp[k] = grid_s[(words[0] >> (k * BITS)) & (NPTS - 1)];
+  team_rotate_back_and_scale<D>(rc, ts, wp, sf[0]);
+  float4 pq[1][2];
   get_pred(pq);     // the prediction values of this lane (zeros without a predictor)
-#pragma unroll
-  for (int c = 0; c < CPM; ++c) {
-    const float pp[8] = {pq[c][0].x, pq[c][0].y, pq[c][0].z, pq[c][0].w,
-                         pq[c][1].x, pq[c][1].y, pq[c][1].z, pq[c][1].w};
-    uint32_t o[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-      o[i] = store16x2<kBf16>(__fadd_rn(pp[2 * i], w[c * 8 + 2 * i]), __fadd_rn(pp[2 * i + 1], w[c * 8 + 2 * i + 1]));
-    *reinterpret_cast<uint4*>(hat_row + (c0 + c) * 256 + lane * 8) = make_uint4(o[0], o[1], o[2], o[3]);
-  }
+  uint32_t o[4];
+  o[0] = store16x2p<kBf16>(add2(pack2(pq[0][0].x, pq[0][0].y), wp[0]));
+  o[1] = store16x2p<kBf16>(add2(pack2(pq[0][0].z, pq[0][0].w), wp[1]));
+  o[2] = store16x2p<kBf16>(add2(pack2(pq[0][1].x, pq[0][1].y), wp[2]));
+  o[3] = store16x2p<kBf16>(add2(pack2(pq[0][1].z, pq[0][1].w), wp[3]));
+  *reinterpret_cast<uint4*>(hat_row + rc.member * 256 + rc.lane * 8) = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
 // This lane's codes and scales of one row (the small inputs of decode_row_core).
@@ -656,7 +634,7 @@ __device__ __forceinline__ void decode_row_load_codes(const RowCtx& rc, const ui
 
 // decode_row_core with the row's inputs read straight from global memory.
 template <int D, int NPTS, bool kBf16>
-__device__ __forceinline__ void decode_row(const RowCtx& rc, const float2* __restrict__ grid_s,
+__device__ __forceinline__ void decode_row(const RowCtx& rc, const f32x2_t* __restrict__ grid_s,
                                            TeamSmem<D>* ts, const uint8_t* __restrict__ codes_row,
                                            const uint16_t* __restrict__ scales_row,
                                            const float* __restrict__ pred_row,
@@ -689,11 +667,11 @@ __global__ void __launch_bounds__(kCodecThreads, 2) decode_rows_kernel(const Cod
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
   constexpr int CODE_BYTES = D / 2 * BITS / 8;
   constexpr int TEAM = RowTeam<D>::TEAM, TEAMS = kCodecWarps / TEAM;
-  __shared__ float2 grid_s[NPTS];
+  __shared__ f32x2_t grid_s[NPTS];
   __shared__ TeamSmem<D> team_s[TEAMS];
   for (int i = threadIdx.x; i < NPTS; i += blockDim.x) {
     const float4 g = a.grid4[i];
-    grid_s[i] = make_float2(g.x, g.y);
+    grid_s[i] = pack2(g.x, g.y);
   }
   __syncthreads();
   const RowCtx rc = make_row_ctx(a, TEAM, RowTeam<D>::NV, 1);

@@ -57,7 +57,7 @@ struct LayerSmemTail {
 // Grid only (decode needs no search table).
 template <int NPTS>
 struct GridSmem {
-  float2 grid[NPTS];
+  f32x2_t grid[NPTS];
 };
 template <bool kEncode, int NPTS> struct LayerTables { typedef RowSmem<NPTS> type; };
 template <int NPTS> struct LayerTables<false, NPTS> { typedef GridSmem<NPTS> type; };
@@ -239,7 +239,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
   } else {
     for (int i = threadIdx.x; i < NPTS; i += blockDim.x) {
       const float4 g = a.grid4[i];
-      rsm->tables.grid[i] = make_float2(g.x, g.y);
+      rsm->tables.grid[i] = pack2(g.x, g.y);
     }
   }
   if (warp == 1) {
@@ -436,7 +436,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
     const int team = rw / TEAM;
     RowCtx rck;     // one context per warp; the sign bits are switched between key and value jobs
     row_ctx_init(rck, a.signmask_k, a.search.inv_w, a.log_h, a.log_g, lane, rw % TEAM, RowTeam<D>::NV, 3 + team);
-    const uint32_t signs_k = rck.signmask;
+    const uint32_t signs_k = a.signmask_k[lane] >> (rck.member * RowTeam<D>::NV);
     const uint32_t signs_v = a.signmask_v[lane] >> (rck.member * RowTeam<D>::NV);
     TeamSmem<D>* ts = &rsm->team[team];
     const int n_groups = D >> a.log_g;
@@ -445,7 +445,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       layer_job(j, a.n_waves, ph, wave);
       const WaveRows wr = wave_rows(wave, a.T, a.mw, gridDim.x);
       if (wr.tokens <= 0) continue;
-      rck.signmask = ph == 0 ? signs_k : signs_v;
+      row_ctx_set_signs(rck, ph == 0 ? signs_k : signs_v);
       const int slot_row = (ml * NTN + n_blk) * wr.rpc;      // first row (within the wave) of this CTA's slice
       const int rb = slot_row / kBM;                         // token block (within the wave) the slice lies in
       if (rb >= wr.blocks) continue;                         // nothing assigned, nobody waits for this CTA

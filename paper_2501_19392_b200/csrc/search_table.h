@@ -10,8 +10,8 @@
 // result, it only skips points that cannot win.
 //
 // Entry layout (uint32): bytes 0..3 = candidate indices in ascending order (short lists repeat
-// their last index); the single descending pattern 0x00000001 marks a cell that must be searched
-// exhaustively.
+// their last index); 0xFFFFFFFF marks a cell that must be searched exhaustively, which includes all
+// border cells: the kernel clamps cell coordinates, so they stand for everything outside the square.
 #pragma once
 
 #include <cmath>
@@ -20,7 +20,8 @@
 
 namespace aquakv {
 
-constexpr uint32_t kCellBrute = 1u;   // bytes (1, 0, 0, 0): not ascending, so never a candidate list
+constexpr uint32_t kCellBrute = 0xFFFFFFFFu;   // the largest entry value; as a candidate list it could only
+                                               // mean "point 255 alone", for which searching all points is right too
 
 struct SearchTableSpec {
   int cells;        // C, cells per side (power of two)
@@ -101,7 +102,9 @@ inline void build_search_table(const float* grid, int n, const SearchTableSpec& 
         if (!poly.empty()) cand.push_back(i);
       }
       uint32_t e;
-      if (cand.empty() || int(cand.size()) > s.max_cand) {
+      // border cells also catch every value outside the square (the kernel's cell index saturates)
+      const bool border = ix == 0 || iy == 0 || ix == C - 1 || iy == C - 1;
+      if (border || cand.empty() || int(cand.size()) > s.max_cand) {
         e = kCellBrute;
       } else {
         e = 0;

@@ -10,11 +10,10 @@ from paper_2501_19392_b200 import synth
 
 def _candidates(table, cells, half, y):
     w = 2.0 * half / cells
-    ix = np.floor((y[:, 0] + half) / w).astype(np.int64)
-    iy = np.floor((y[:, 1] + half) / w).astype(np.int64)
-    inside = (ix >= 0) & (ix < cells) & (iy >= 0) & (iy < cells)
-    e = table[np.clip(iy, 0, cells - 1), np.clip(ix, 0, cells - 1)]
-    brute = (e == 1) | ~inside
+    ix = np.clip(np.floor((y[:, 0] + half) / w).astype(np.int64), 0, cells - 1)   # the kernel's cell index saturates
+    iy = np.clip(np.floor((y[:, 1] + half) / w).astype(np.int64), 0, cells - 1)
+    e = table[iy, ix]
+    brute = e == 0xFFFFFFFF
     cand = np.stack([e & 0xFF, (e >> 8) & 0xFF, (e >> 16) & 0xFF, (e >> 24) & 0xFF], axis=1).astype(np.int64)
     return cand, brute
 
@@ -59,5 +58,8 @@ def test_table_keeps_the_nearest_point(n):
         assert np.all(np.diff(cand[asc], axis=1) >= 0)
         if n == 16:     # the kernel evaluates three candidates there: the fourth byte only repeats the third
             assert np.all(cand[asc][:, 3] == cand[asc][:, 2])
+        # values outside the square land in border cells, which must all say "search all points"
+        assert np.all(table[0, :] == 0xFFFFFFFF) and np.all(table[-1, :] == 0xFFFFFFFF)
+        assert np.all(table[:, 0] == 0xFFFFFFFF) and np.all(table[:, -1] == 0xFFFFFFFF)
         if name == "gauss":
             assert brute.mean() < (0.02 if n <= 64 else 0.25), brute.mean()
