@@ -79,3 +79,51 @@ def test_decode_attn_matches_dequantize_then_attend(batch, ctx, n_q, n_kv, hd, d
     # (4) without the optional K_hat/V_hat outputs the result is bit-identical
     out_b, lse_b = codec.decode_attn(*args, want_lse=True)
     assert torch.equal(out_b, out) and torch.equal(lse_b, lse)
+
+
+def test_decode_attn_at_the_full_llama31_8b_shape():
+    """Batch 32 x context 32768 (1,048,576 cached tokens), 32 query heads / 8 KV heads x 128, bf16, 2-bit
+    cache from seed, adapters on the previous layer's reconstruction: the full decode-attention
+    workload in one call.  The oracle checks sampled decoded rows, and attends over the decoded rows of
+    two whole sequences (softmax needs the full context)."""
+    from paper_2501_19392_b200 import api
+    batch, ctx, n_q, n_kv, hd, dtype = 32, 32768, 32, 8, 128, synth.BF16
+    d, T = n_kv * hd, batch * ctx
+    shape = dataclasses.replace(synth.CONFIGS[5], n_tokens=T, n_layers=2)
+    grid = synth.lloyd_grid(16, seed=7, n_samples=1 << 14, iters=25)
+    sk, sv = synth.hadamard_signs(d, 11), synth.hadamard_signs(d, 12)
+    codec = api.Codec(d, d, d, grid, dtype, sk, sv)
+    ora = oracle.Oracle(d, d, d, grid, dtype, sk, sv)
+    cache = synth.random_cache(shape, seed=5101, device=DEV, n_layers=1)
+    ad = synth.random_adapters(shape, seed=5102, device=DEV)
+    pK = synth.random_16bit((T, d), dtype, 5103, device=DEV)
+    pV = synth.random_16bit((T, d), dtype, 5104, device=DEV)
+    q = synth.random_16bit((batch, n_q, hd), dtype, 5105, device=DEV)
+    Kh = torch.empty((T, d), dtype=torch.bfloat16, device=DEV)
+    Vh = torch.empty_like(Kh)
+    scale = 1.0 / np.sqrt(hd)
+    out, lse = codec.decode_attn(q, cache.Kcodes[0], cache.Kscales[0], cache.Vcodes[0], cache.Vscales[0], ctx,
+                                 n_kv, scale, pK, pV, ad.Wk[1], ad.Wv[1], Khat=Kh, Vhat=Vh, want_lse=True)
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    b = synth.to_bits
+    rng = np.random.default_rng(5106)
+    rows = np.unique(np.concatenate([[0, 1, 127, 128, 4607, 4608, 36863, 36864, T - 129, T - 1],
+                                     rng.integers(0, T, 150)]))
+    idx = torch.from_numpy(rows).to(DEV)
+    kd = ora.decode_phase(cache.Kcodes[0][idx].cpu().numpy(), b(cache.Kscales[0][idx]), [b(pK[idx])],
+                          b(ad.Wk[1]), None, "k")
+    check_recon(gpu_bits(Kh[idx]), kd["hat_exact"], kd["hat"], dtype)
+    vd = ora.decode_phase(cache.Vcodes[0][idx].cpu().numpy(), b(cache.Vscales[0][idx]),
+                          [b(pV[idx]), gpu_bits(Kh[idx])], b(ad.Wv[1]), None, "v")
+    check_recon(gpu_bits(Vh[idx]), vd["hat_exact"], vd["hat"], dtype)
+    for s in (0, batch - 1):
+        sl = slice(s * ctx, (s + 1) * ctx)
+        ref, ref_lse = oracle.attention(dtype, 1, ctx, n_q, n_kv, hd, scale, b(q[s:s + 1]), gpu_bits(Kh[sl]),
+                                        gpu_bits(Vh[sl]))
+        o = out[s:s + 1].to(torch.float64).cpu().numpy()
+        ref_bits = synth.to_bits(torch.from_numpy(ref).to(torch.bfloat16)).astype(np.int64)
+        adjacent = np.abs(gpu_bits(out[s:s + 1]).astype(np.int64) - ref_bits) <= 1
+        denom = np.abs(ref).max(axis=-1, keepdims=True)
+        assert np.all((np.abs(o - ref) <= 2e-3 * denom) | adjacent)
+        assert np.abs(lse[s:s + 1].cpu().numpy() - ref_lse).max() <= 1e-4

@@ -263,3 +263,65 @@ def test_empty_and_argument_errors_on_device():
         codec.encode(x, x, x, x, w, wv, workspace=small)
     assert err.value.status == -4
     assert codec.poll_status() == 0
+
+
+def test_bulk_decode_shape_on_sampled_rows():
+    """Llama-3.3-70B-shaped bulk decode (131072 cached tokens, d_kv 1024, 2-bit codes and fp16 scales
+    drawn from seed, adapters on the previous layer's reconstruction), one layer in the launch
+    configuration of a real call (all tokens in one fused launch), against the oracle on sampled rows."""
+    T = 131072
+    shape = dataclasses.replace(synth.CONFIGS[4], n_tokens=T, n_layers=2)
+    d, dtype = shape.d_kv, shape.dtype
+    codec, ora = make(d, shape.had_block, shape.scale_group, shape.grid_size, dtype)
+    cache = synth.random_cache(shape, seed=4001, device=DEV, n_layers=1)
+    ad = synth.random_adapters(shape, seed=4002, device=DEV)
+    pK = synth.random_16bit((T, d), dtype, 4003, device=DEV)
+    pV = synth.random_16bit((T, d), dtype, 4004, device=DEV)
+    Kh, Vh = codec.decode(cache.Kcodes[0], cache.Kscales[0], cache.Vcodes[0], cache.Vscales[0], pK, pV,
+                          ad.Wk[1], ad.Wv[1])
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    rows = _sample_rows(T, seed=4005)
+    idx = torch.from_numpy(rows).to(DEV)
+    b = synth.to_bits
+    kd = ora.decode_phase(cache.Kcodes[0][idx].cpu().numpy(), b(cache.Kscales[0][idx]), [b(pK[idx])],
+                          b(ad.Wk[1]), None, "k")
+    check_recon(gpu_bits(Kh[idx]), kd["hat_exact"], kd["hat"], dtype)
+    vd = ora.decode_phase(cache.Vcodes[0][idx].cpu().numpy(), b(cache.Vscales[0][idx]),
+                          [b(pV[idx]), gpu_bits(Kh[idx])], b(ad.Wv[1]), None, "v")
+    check_recon(gpu_bits(Vh[idx]), vd["hat_exact"], vd["hat"], dtype)
+
+
+def test_free_running_chain_tracks_the_oracle_chain():
+    """Six layers with each side feeding itself (no teacher forcing): codes may drift apart after
+    near-ties, so the chains are compared statistically: per layer, the library's relative
+    reconstruction error stays within 2 % (relative) of the oracle's, and most codes still agree."""
+    from paper_2501_19392_b200 import chain as chain_mod
+    T, L = 512, 6
+    shape, kv, ad = chain(2, T, L)
+    d, dtype, bits = shape.d_kv, shape.dtype, shape.code_bits
+    codec, ora = make(d, shape.had_block, shape.scale_group, shape.grid_size, dtype)
+    g = lambda t: None if t is None else t.to(DEV)
+    adg = dataclasses.replace(ad, Wk=[g(w) for w in ad.Wk], Wv=[g(w) for w in ad.Wv])
+    cache = chain_mod.CompressedCache.empty(codec, L, T, DEV)
+    bufs = chain_mod.PingPong(codec, T, DEV)
+    Kg, Vg = [g(t) for t in kv.K], [g(t) for t in kv.V]
+    b = synth.to_bits
+    pk = pv = None
+    for l in range(L):
+        has = l > 0
+        cur, prv = l % 2, (l + 1) % 2
+        codec.encode(Kg[l], Vg[l], bufs.K[prv] if has else None, bufs.V[prv] if has else None,
+                     adg.Wk[l] if has else None, adg.Wv[l] if has else None, None, None,
+                     cache.Kcodes[l], cache.Kscales[l], cache.Vcodes[l], cache.Vscales[l], bufs.K[cur], bufs.V[cur])
+        ok_, ov_ = ora.encode_layer(b(kv.K[l]), b(kv.V[l]), pk, pv, b(ad.Wk[l]) if has else None,
+                                    b(ad.Wv[l]) if has else None)
+        pk, pv = ok_["hat"], ov_["hat"]
+        for x, hat_gpu, o in ((kv.K[l], bufs.K[cur], ok_), (kv.V[l], bufs.V[cur], ov_)):
+            x64 = x.to(torch.float64).numpy()
+            err_gpu = ((hat_gpu.to(torch.float64).cpu().numpy() - x64) ** 2).sum() / (x64 ** 2).sum()
+            err_ora = ((bits_to_f64(o["hat"], dtype) - x64) ** 2).sum() / (x64 ** 2).sum()
+            assert abs(err_gpu - err_ora) <= 0.02 * err_ora, (l, err_gpu, err_ora)
+        agree = (cache.Kcodes[l].cpu().numpy() == ok_["codes"]).mean()
+        assert agree > 0.9, (l, agree)
+    assert codec.poll_status() == 0
