@@ -230,9 +230,10 @@ __device__ __forceinline__ int nearest_of_candidates(f32x2_t y, uint32_t e, cons
 }
 
 template <int NPTS>
-__device__ __noinline__ int nearest_exhaustive(f32x2_t y, const f32x2_t* __restrict__ grid_s) {
+__device__ __forceinline__ int nearest_exhaustive(f32x2_t y, const f32x2_t* __restrict__ grid_s) {
   float best = 3.0e38f;
   int idx = 0;
+#pragma unroll 1
   for (int i = 0; i < NPTS; ++i) {
     const float t = pair_dist(y, grid_s[i]);
     if (t < best) { best = t; idx = i; }             // strict: lowest index wins ties
@@ -505,18 +506,19 @@ __device__ __forceinline__ void encode_row_core(const RowCtx& rc, const RowSmem<
     emax = max(emax, entry[k]);
   }
   const bool slow = __any_sync(0xffffffffu, emax == kCellBruteDev);
+  int idx[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) idx[k] = nearest_of_candidates<NPTS>(vp[k], entry[k], rsm->grid);
+  if (slow) {                    // rare: some lane of the warp has a pair that needs the exhaustive search
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (entry[k] == kCellBruteDev) idx[k] = nearest_exhaustive<NPTS>(vp[k], rsm->grid);
+  }
   uint32_t word = 0;
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
-    int idx;
-    if (!slow) {
-      idx = nearest_of_candidates<NPTS>(vp[k], entry[k], rsm->grid);
-    } else {
-      idx = entry[k] == kCellBruteDev ? nearest_exhaustive<NPTS>(vp[k], rsm->grid)
-                                      : nearest_of_candidates<NPTS>(vp[k], entry[k], rsm->grid);
-    }
-    word |= uint32_t(idx) << (k * BITS);
-    vp[k] = rsm->grid[idx];
+    word |= uint32_t(idx[k]) << (k * BITS);
+    vp[k] = rsm->grid[idx[k]];
   }
   store_code_word<BITS>(codes_row, cg, lane, word);
   // ---- reconstruction: hat = round16(pred + Q^-1(codes)) ---------------------------------------

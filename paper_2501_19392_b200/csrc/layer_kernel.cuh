@@ -175,7 +175,7 @@ __device__ __forceinline__ bool counter_wait_bounded(const int* ctr, int target,
   const unsigned long long t0 = global_timer_ns();
   uint32_t spins = 0;
   while (ld_acquire(ctr) < target) {
-    __nanosleep(64);
+    __nanosleep(256);
     if ((++spins & 0x3Fu) == 0) {
       if (*abort_flag) return false;
       if (global_timer_ns() - t0 > kWaitLimitNs) {
