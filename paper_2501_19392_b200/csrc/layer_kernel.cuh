@@ -424,10 +424,14 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         }
         __syncwarp();
       }
-      __threadfence();
+      // release by one thread after the barrier: its fence also covers the stores of the threads it
+      // has synchronised with, and only that thread waits for them to become visible
       named_barrier(1, 128);
       if (*abort_flag) break;
-      if (warp == 2 && lane == 0) atomicAdd(a.gemm_done + j * a.mw + ml, 1);
+      if (warp == 2 && lane == 0) {
+        __threadfence();
+        atomicAdd(a.gemm_done + j * a.mw + ml, 1);
+      }
     }
   } else {
     // ------------------------------- row warps (teams of TEAM warps per row) -------------------
@@ -495,11 +499,13 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         }
       }
       // each team reports on its own, so a slow team never holds the others back
-      __threadfence();
-      fence_proxy_async_all();
       if (TEAM > 1) team_barrier<D>(rck.barrier); else __syncwarp();
       if (*abort_flag) break;
-      if (rck.member == 0 && lane == 0) atomicAdd(a.rows_done + j * a.mw + rb, 1);
+      if (rck.member == 0 && lane == 0) {   // one releasing thread per team (see the epilogue)
+        __threadfence();
+        fence_proxy_async_all();
+        atomicAdd(a.rows_done + j * a.mw + rb, 1);
+      }
     }
   }
 
