@@ -174,8 +174,10 @@ __device__ __forceinline__ bool counter_wait_bounded(const int* ctr, int target,
   if (ld_acquire(ctr) >= target) return true;
   const unsigned long long t0 = global_timer_ns();
   uint32_t spins = 0;
+  uint32_t pause = 64;          // polls cost issue slots the row warps need: back off up to 2 us
   while (ld_acquire(ctr) < target) {
-    __nanosleep(256);
+    __nanosleep(pause);
+    if (pause < 2048) pause <<= 1;
     if ((++spins & 0x3Fu) == 0) {
       if (*abort_flag) return false;
       if (global_timer_ns() - t0 > kWaitLimitNs) {
@@ -378,8 +380,11 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         int ph_old, wave_old;
         layer_job(j - a.nb, a.n_waves, ph_old, wave_old);
         const int target = wave_block_teams(wave_rows(wave_old, a.T, a.mw, gridDim.x), ml, gridDim.x, kRowTeamsOf<D>);
-        if (lane == 0) ok = counter_wait_bounded(a.rows_done + (j - a.nb) * a.mw + ml, target, abort_flag, a.status);
-        ok = __shfl_sync(0xffffffffu, ok, 0);
+        // one thread polls for the four warps; a failed wait has set the abort flag
+        if (warp == 2 && lane == 0)
+          counter_wait_bounded(a.rows_done + (j - a.nb) * a.mw + ml, target, abort_flag, a.status);
+        named_barrier(1, 128);
+        ok = *abort_flag == 0;
       }
       if (ok) ok = mbar_wait_bounded(&tail->acc_full[acc], acc_phase, abort_flag, a.status);
       if (ok) {
@@ -467,14 +472,17 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         }
       }
       bool ok = true;
-      if (lane == 0) ok = counter_wait_bounded(a.gemm_done + j * a.mw + rb, NTN, abort_flag, a.status);
-      ok = __shfl_sync(0xffffffffu, ok, 0);
       if (TEAM > 1) {
-        // all warps of a team must take the same path: agree through shared memory
-        if (!ok) *abort_flag = 1;
+        // one thread polls for the team; all its warps must take the same path, so they agree
+        // through the abort flag (set by a failed wait) between two barriers
+        if (rck.member == 0 && lane == 0)
+          counter_wait_bounded(a.gemm_done + j * a.mw + rb, NTN, abort_flag, a.status);
         team_barrier<D>(rck.barrier);
         ok = *abort_flag == 0;
         team_barrier<D>(rck.barrier);
+      } else {
+        if (lane == 0) ok = counter_wait_bounded(a.gemm_done + j * a.mw + rb, NTN, abort_flag, a.status);
+        ok = __shfl_sync(0xffffffffu, ok, 0);
       }
       if (ok) {
         const float* pbuf = a.P + (size_t(j % a.nb) * a.mw * kBM + size_t(rb) * kBM) * D;
