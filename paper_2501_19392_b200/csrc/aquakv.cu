@@ -396,12 +396,12 @@ AttnWs attn_ws(const aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_
   return w;
 }
 
-template <bool ENC, int D, int NPTS, bool BF>
+template <bool ENC, int D, int NPTS, bool BF, bool FULL>
 int launch_layer_t(cudaStream_t st, int grid, const CUtensorMap* tm, const LayerArgs& a) {
   static bool attr_set = false;   // per instantiation; contexts are used from one thread at a time
   constexpr size_t smem = layer_smem_bytes<ENC, D, NPTS>();
   if (!attr_set) {
-    if (cudaFuncSetAttribute(layer_kernel<ENC, D, NPTS, BF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(layer_kernel<ENC, D, NPTS, BF, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              int(smem)) != cudaSuccess)
       return AQUAKV_ERR_CUDA;
     attr_set = true;
@@ -418,18 +418,22 @@ int launch_layer_t(cudaStream_t st, int grid, const CUtensorMap* tm, const Layer
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, layer_kernel<ENC, D, NPTS, BF>, tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], a) ==
+  return cudaLaunchKernelEx(&cfg, layer_kernel<ENC, D, NPTS, BF, FULL>, tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], a) ==
                  cudaSuccess
              ? AQUAKV_OK
              : AQUAKV_ERR_CUDA;
 }
 template <int D, int NPTS, bool BF>
 void launch_layer_enc_t(int* rc, cudaStream_t st, int grid, const CUtensorMap* tm, const LayerArgs& a) {
-  *rc = launch_layer_t<true, D, NPTS, BF>(st, grid, tm, a);
+  // Hadamard block = scale group = the whole row: the encoder has an instantiation with those sizes
+  // fixed at compile time (measured 3-6 % faster; the decoder measured no gain and has none)
+  const bool full = a.log_h == a.log_g && (1 << a.log_h) == D;
+  *rc = full ? launch_layer_t<true, D, NPTS, BF, true>(st, grid, tm, a)
+             : launch_layer_t<true, D, NPTS, BF, false>(st, grid, tm, a);
 }
 template <int D, int NPTS, bool BF>
 void launch_layer_dec_t(int* rc, cudaStream_t st, int grid, const CUtensorMap* tm, const LayerArgs& a) {
-  *rc = launch_layer_t<false, D, NPTS, BF>(st, grid, tm, a);
+  *rc = launch_layer_t<false, D, NPTS, BF, false>(st, grid, tm, a);
 }
 
 // The fused kernel needs its whole shared-memory budget in one CTA; the largest grid (256 points)

@@ -197,7 +197,9 @@ __device__ __forceinline__ void fence_proxy_async_all() {
   asm volatile("fence.proxy.async;" ::: "memory");
 }
 
-template <bool kEncode, int D, int NPTS, bool kBf16>
+// kFull: the Hadamard block and the scale group both span the whole row (the paper's setting for
+// d_kv = 1024, Section 4.1); their logarithms are then compile-time constants of the row code.
+template <bool kEncode, int D, int NPTS, bool kBf16, bool kFull>
 __global__ void __launch_bounds__(kLayerThreads, 1)
 layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant__ CUtensorMap tmVprev,
              const __grid_constant__ CUtensorMap tmKhat, const __grid_constant__ CUtensorMap tmWk,
@@ -444,11 +446,13 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
     const int rw = warp - 6;
     const int team = rw / TEAM;
     RowCtx rck;     // one context per warp; the sign bits are switched between key and value jobs
-    row_ctx_init(rck, a.signmask_k, a.search.inv_w, a.log_h, a.log_g, lane, rw % TEAM, RowTeam<D>::NV, 3 + team);
+    constexpr int LOG_D = D == 1024 ? 10 : (D == 512 ? 9 : 8);
+    const int log_h = kFull ? LOG_D : a.log_h, log_g = kFull ? LOG_D : a.log_g;
+    row_ctx_init(rck, a.signmask_k, a.search.inv_w, log_h, log_g, lane, rw % TEAM, RowTeam<D>::NV, 3 + team);
     const uint32_t signs_k = a.signmask_k[lane] >> (rck.member * RowTeam<D>::NV);
     const uint32_t signs_v = a.signmask_v[lane] >> (rck.member * RowTeam<D>::NV);
     TeamSmem<D>* ts = &rsm->team[team];
-    const int n_groups = D >> a.log_g;
+    const int n_groups = D >> log_g;
     for (int j = 0; j < n_jobs; ++j) {
       int ph, wave;
       layer_job(j, a.n_waves, ph, wave);
