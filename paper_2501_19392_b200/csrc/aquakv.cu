@@ -246,34 +246,19 @@ int launch_decode_rows(aquakv_ctx* c, cudaStream_t st, int role, int rows, const
   return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
 }
 
-template <int HD, int GQ, bool BF>
-void launch_attn_partial_t(cudaStream_t st, const AttnArgs& a, dim3 grid) {
-  attn_partial_kernel<HD, GQ, BF><<<grid, kAttnThreads, 0, st>>>(a);
-}
-
-int attn_gq(int rep, int* passes) {
-  switch (rep) {
-    case 1: case 2: case 3: case 4: *passes = 1; return rep;
-    case 6: *passes = 2; return 3;
-    case 8: *passes = 2; return 4;
-    default: *passes = 0; return 0;
-  }
-}
-
-int launch_attn_partial(aquakv_ctx* c, cudaStream_t st, const AttnArgs& a, int head_dim,
-                        int n_blocks) {
-  int passes = 0;
-  const int gq = attn_gq(a.n_q_heads / a.n_kv_heads, &passes);
+int launch_attn_partial(aquakv_ctx* c, cudaStream_t st, AttnArgs a, int head_dim, int n_blocks) {
+  const int rep = a.n_q_heads / a.n_kv_heads;
+  const int passes = (rep + kAttnMmaMaxGq - 1) / kAttnMmaMaxGq;
+  a.gq = (rep + passes - 1) / passes;
   const dim3 grid(n_blocks, a.n_kv_heads, passes);
   ProfScope prof(c, st, AQUAKV_KERNEL_ATTN);
-#define AQ_ATTN(HD, GQ)                                                   \
-  if (head_dim == HD && gq == GQ) {                                       \
-    if (c->bf16) launch_attn_partial_t<HD, GQ, true>(st, a, grid);        \
-    else launch_attn_partial_t<HD, GQ, false>(st, a, grid);               \
+  if (head_dim == 64) {
+    if (c->bf16) attn_partial_kernel<64, true><<<grid, kAttnMmaThreads, 0, st>>>(a);
+    else attn_partial_kernel<64, false><<<grid, kAttnMmaThreads, 0, st>>>(a);
+  } else {
+    if (c->bf16) attn_partial_kernel<128, true><<<grid, kAttnMmaThreads, 0, st>>>(a);
+    else attn_partial_kernel<128, false><<<grid, kAttnMmaThreads, 0, st>>>(a);
   }
-  AQ_ATTN(64, 1) AQ_ATTN(64, 2) AQ_ATTN(64, 3) AQ_ATTN(64, 4)
-  AQ_ATTN(128, 1) AQ_ATTN(128, 2) AQ_ATTN(128, 3) AQ_ATTN(128, 4)
-#undef AQ_ATTN
   ++c->launches;
   return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
 }
@@ -1035,8 +1020,7 @@ int aquakv_decode_attn(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_
   const int d = c->p.d_kv;
   if (n_q_heads <= 0 || n_kv_heads <= 0 || head_dim <= 0) return AQUAKV_ERR_INVALID_ARG;
   if (n_kv_heads * head_dim != d || n_q_heads % n_kv_heads) return AQUAKV_ERR_INVALID_ARG;
-  int passes = 0;
-  if ((head_dim != 64 && head_dim != 128) || attn_gq(n_q_heads / n_kv_heads, &passes) == 0)
+  if ((head_dim != 64 && head_dim != 128) || n_q_heads / n_kv_heads > kAttnMmaMaxGq)
     return AQUAKV_ERR_UNSUPPORTED;
   if (ctx_len > (int64_t(1) << 30)) return AQUAKV_ERR_UNSUPPORTED;
   if (q == nullptr || out == nullptr || Kcodes == nullptr || Kscales == nullptr ||

@@ -3,19 +3,14 @@
 // tokens of one sequence to per-query-head partials (running max, sum, unnormalised output), a
 // second kernel merges the partials of a sequence by log-sum-exp.  All accumulation is fp32.
 //
-// One CTA owns (token block, KV head) and up to four of that KV head's query heads at once, so
-// K/V bytes are read once per KV head.  Inside a warp, 8 lanes share one token (each lane owns
-// HD/8 head dimensions as 16-byte pieces) and the 4 lane groups take consecutive tokens; the 8
-// warps interleave over the block's tokens and merge through shared memory.
+// One CTA owns (token block, KV head) and up to eight of that KV head's query heads at once, so
+// K/V bytes are read once per KV head.
 #pragma once
 
 #include "common.cuh"
 
 namespace aquakv {
 
-constexpr int kAttnWarps = 8;
-constexpr int kAttnThreads = kAttnWarps * 32;
-constexpr int kAttnMaxGq = 4;       // query heads per KV head processed by one pass
 constexpr float kNegBig = -1.0e30f;
 
 struct AttnArgs {
@@ -30,165 +25,215 @@ struct AttnArgs {
   int n_kv_heads;
   int n_splits;           // blocks per sequence
   int block_tokens;       // tokens per block
+  int gq;                 // query heads of a KV group handled by one pass (grid z = passes), <= 8
   float scale_log2;       // softmax_scale * log2(e)
   float* part_ml;         // [batch][n_splits][n_q_heads][2]  (max in log2 units, sum)
   float* part_o;          // [batch][n_splits][n_q_heads][HD]
 };
 
+// D += A * B for one m16n8k16 tile (fp32 accumulate), A and B in the cache's 16-bit type.
 template <bool kBf16>
-__device__ __forceinline__ void unpack8(const uint4& raw, float (&f)[8]) {
-  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    f[2 * i] = load16<kBf16>(uint16_t(w[i] & 0xffffu));
-    f[2 * i + 1] = load16<kBf16>(uint16_t(w[i] >> 16));
+__device__ __forceinline__ void mma_16x8x16(float& d0, float& d1, float& d2, float& d3, uint32_t a0,
+                                            uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  if constexpr (kBf16) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(d0), "+f"(d1), "+f"(d2), "+f"(d3)
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  } else {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(d0), "+f"(d1), "+f"(d2), "+f"(d3)
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
   }
 }
 
-template <int HD, int GQ, bool kBf16>
-__global__ void __launch_bounds__(kAttnThreads, 2) attn_partial_kernel(const AttnArgs a) {
-  constexpr int NP = HD / 64;          // 16-byte pieces per lane per row (8 dims each)
-  constexpr int DPL = NP * 8;          // dims per lane
-  __shared__ float sm_m[kAttnWarps][GQ];
-  __shared__ float sm_l[kAttnWarps][GQ];
-  __shared__ float sm_o[kAttnWarps][GQ][HD];
-  __shared__ float sm_q[GQ][HD];       // queries, pre-multiplied by softmax_scale * log2(e)
+// The kernel is bound by reading K^ and V^ once (HD * 4 bytes per token and KV head), so it is built
+// to issue few instructions per byte: both contractions run as warp-level 16x8x16 matrix products
+// with the query heads of the KV group on the M side (up to 8 rows used, the other 8 are zero) and
+// every operand fragment filled straight from 16-byte global loads.
+//   scores: A = queries, B = keys.  The product sums over head dimensions, so their order inside a
+//           32-dimension chunk is free: lane (n, j) loads dimensions [32c + 8j, 32c + 8j + 8) of
+//           token n as one 16-byte piece and uses it as the B fragments of two k-steps; the query
+//           fragments use the same order.
+//   output: A = probabilities (the score accumulators, rounded to the 16-bit type, already have the
+//           A-fragment layout), B = values.  A B register pairs two consecutive tokens at one
+//           dimension; it is made from the 16-byte pieces of those two token rows with one byte
+//           permute.  Column n of output tile u stands for head dimension 8n + u (u < 8) or
+//           64 + 8n + (u - 8), so lane group n reads contiguous 16-byte pieces.
+// A warp takes 32 tokens at a time (four 8-token score tiles, two 16-token k-steps of the output
+// product) with an online softmax across its groups; the warps of a CTA merge through shared memory.
+constexpr int kAttnMmaWarps = 4;
+constexpr int kAttnMmaThreads = kAttnMmaWarps * 32;
+constexpr int kAttnMmaMaxGq = 8;    // query heads per KV head in one pass (rows of the M = 16 tile in use)
+
+template <int HD, bool kBf16>
+__global__ void __launch_bounds__(kAttnMmaThreads, 2) attn_partial_kernel(const AttnArgs a) {
+  constexpr int NCH = HD / 32;         // 32-dimension chunks of the score product
+  constexpr int NVH = HD / 64;         // 64-dimension halves of a value row (one 16-byte piece per lane each)
+  constexpr int NOT = HD / 8;          // output tiles of 8 dimensions
+  __shared__ float sm_m[kAttnMmaWarps][kAttnMmaMaxGq];
+  __shared__ float sm_l[kAttnMmaWarps][kAttnMmaMaxGq];
+  __shared__ float sm_o[kAttnMmaWarps][kAttnMmaMaxGq][HD];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int tg = lane >> 3, dl = lane & 7;
+  const int g = lane >> 2, j = lane & 3;
   const long long gb = a.blk_begin + blockIdx.x;
   const int b = int(gb / a.n_splits), split = int(gb % a.n_splits);
   const int t_begin = split * a.block_tokens;
   const int t_end = min(a.ctx, t_begin + a.block_tokens);
   const int rep = a.n_q_heads / a.n_kv_heads;
   const int kvh = blockIdx.y;
-  const int g0 = blockIdx.z * GQ;      // first query head (within the KV group) of this pass
+  const int g0 = blockIdx.z * a.gq;    // first query head (within the KV group) of this pass
+  const int gq = min(a.gq, rep - g0);  // query heads of this pass
 
-  for (int idx = threadIdx.x; idx < GQ * HD; idx += kAttnThreads) {
-    const int g = idx / HD, i = idx % HD;
-    const uint16_t qb = a.q[((long long)b * a.n_q_heads + kvh * rep + g0 + g) * HD + i];
-    sm_q[g][i] = load16<kBf16>(qb) * a.scale_log2;
+  // query fragments: row g = query head g0 + g of the KV group (rows >= gq and rows 8..15 are zero)
+  uint32_t qa[NCH][2][2];
+  {
+    const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
+        a.q + ((long long)b * a.n_q_heads + kvh * rep + g0 + (g < gq ? g : 0)) * HD);
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      const uint4 w = *reinterpret_cast<const uint4*>(qrow + (c * 32 + j * 8) / 2);
+      const bool on = g < gq;
+      qa[c][0][0] = on ? w.x : 0u;
+      qa[c][0][1] = on ? w.y : 0u;
+      qa[c][1][0] = on ? w.z : 0u;
+      qa[c][1][1] = on ? w.w : 0u;
+    }
   }
-  __syncthreads();
+  float m_run = kNegBig, l_run = 0.0f;     // row g's running maximum (log2 units) and this lane's part of its sum
+  float o[NOT][2];
+#pragma unroll
+  for (int u = 0; u < NOT; ++u) o[u][0] = o[u][1] = 0.0f;
+  float dz0 = 0.0f, dz1 = 0.0f;            // rows 8..15 of every product: stay zero
 
-  float m[GQ], l[GQ], acc[GQ][DPL];
-#pragma unroll
-  for (int g = 0; g < GQ; ++g) {
-    m[g] = kNegBig;
-    l[g] = 0.0f;
-#pragma unroll
-    for (int i = 0; i < DPL; ++i) acc[g][i] = 0.0f;
-  }
   const long long row0 = (long long)b * a.ctx - a.tok_base;
-  // warp w takes tokens t_begin + 4*(w + 8*j) + {0,1,2,3}; its four lane groups take one each.
-  // The next iteration's key/value pieces are fetched before the current ones are used.
-  uint4 kraw[NP], vraw[NP], kraw_n[NP], vraw_n[NP];
-  auto fetch = [&](int tb, uint4 (&kr)[NP], uint4 (&vr)[NP]) {
-    const int t = tb + tg;
-    const long long row = row0 + (t < t_end ? t : t_begin);
-    const uint16_t* kp = a.Kh + row * a.ld + kvh * HD + dl * 8;
-    const uint16_t* vp = a.Vh + row * a.ld + kvh * HD + dl * 8;
+  const uint16_t* kbase = a.Kh + kvh * HD;
+  const uint16_t* vbase = a.Vh + kvh * HD;
+  for (int tb = t_begin + warp * 32; tb < t_end; tb += 32 * kAttnMmaWarps) {
+    // ---- all loads of the group: keys (score tile t, token g of it), values (k-step ks, tokens 2j.. of it) ----
+    uint4 kq[4][NCH];
 #pragma unroll
-    for (int pc = 0; pc < NP; ++pc) {
-      kr[pc] = __ldcs(reinterpret_cast<const uint4*>(kp + pc * 64));
-      vr[pc] = __ldcs(reinterpret_cast<const uint4*>(vp + pc * 64));
+    for (int t = 0; t < 4; ++t) {
+      const int tok = tb + 8 * t + g;
+      const uint16_t* kp = kbase + (row0 + (tok < t_end ? tok : t_begin)) * a.ld + j * 8;
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) kq[t][c] = __ldcs(reinterpret_cast<const uint4*>(kp + c * 32));
     }
-  };
-  int tb = t_begin + warp * 4;
-  if (tb < t_end) fetch(tb, kraw, vraw);
-  for (; tb < t_end; tb += 4 * kAttnWarps) {
-    const int tbn = tb + 4 * kAttnWarps;
-    if (tbn < t_end) fetch(tbn, kraw_n, vraw_n);
-    const bool valid = tb + tg < t_end;
-    float kf[DPL], vf[DPL];
+    uint4 vq[2][4][NVH];
 #pragma unroll
-    for (int pc = 0; pc < NP; ++pc) {
-      float f[8];
-      unpack8<kBf16>(kraw[pc], f);
+    for (int ks = 0; ks < 2; ++ks) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) kf[pc * 8 + i] = f[i];
-      unpack8<kBf16>(vraw[pc], f);
+      for (int r = 0; r < 4; ++r) {
+        const int tok = tb + 16 * ks + (r >> 1) * 8 + 2 * j + (r & 1);
+        const uint16_t* vp = vbase + (row0 + (tok < t_end ? tok : t_begin)) * a.ld + g * 8;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) vf[pc * 8 + i] = f[i];
-    }
-#pragma unroll
-    for (int g = 0; g < GQ; ++g) {
-      float s = 0.0f;
-#pragma unroll
-      for (int pc = 0; pc < NP; ++pc) {
-        const float4 q0 = *reinterpret_cast<const float4*>(&sm_q[g][pc * 64 + dl * 8]);
-        const float4 q1 = *reinterpret_cast<const float4*>(&sm_q[g][pc * 64 + dl * 8 + 4]);
-        s = fmaf(q0.x, kf[pc * 8 + 0], s); s = fmaf(q0.y, kf[pc * 8 + 1], s);
-        s = fmaf(q0.z, kf[pc * 8 + 2], s); s = fmaf(q0.w, kf[pc * 8 + 3], s);
-        s = fmaf(q1.x, kf[pc * 8 + 4], s); s = fmaf(q1.y, kf[pc * 8 + 5], s);
-        s = fmaf(q1.z, kf[pc * 8 + 6], s); s = fmaf(q1.w, kf[pc * 8 + 7], s);
-      }
-      s += __shfl_xor_sync(0xffffffffu, s, 1);
-      s += __shfl_xor_sync(0xffffffffu, s, 2);
-      s += __shfl_xor_sync(0xffffffffu, s, 4);
-      if (valid) {
-        const float m_new = fmaxf(m[g], s);
-        const float corr = exp2f(m[g] - m_new);
-        const float pr = exp2f(s - m_new);
-        m[g] = m_new;
-        l[g] = fmaf(l[g], corr, pr);
-#pragma unroll
-        for (int i = 0; i < DPL; ++i) acc[g][i] = fmaf(acc[g][i], corr, pr * vf[i]);
+        for (int h = 0; h < NVH; ++h) vq[ks][r][h] = __ldcs(reinterpret_cast<const uint4*>(vp + h * 64));
       }
     }
+    // ---- scores ---------------------------------------------------------------------------------
+    float sc[4][2];
 #pragma unroll
-    for (int pc = 0; pc < NP; ++pc) {
-      kraw[pc] = kraw_n[pc];
-      vraw[pc] = vraw_n[pc];
+    for (int t = 0; t < 4; ++t) {
+      float s0 = 0.0f, s1 = 0.0f;
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) {
+        mma_16x8x16<kBf16>(s0, s1, dz0, dz1, qa[c][0][0], 0u, qa[c][0][1], 0u, kq[t][c].x, kq[t][c].y);
+        mma_16x8x16<kBf16>(s0, s1, dz0, dz1, qa[c][1][0], 0u, qa[c][1][1], 0u, kq[t][c].z, kq[t][c].w);
+      }
+      const int tok = tb + 8 * t + 2 * j;
+      sc[t][0] = tok < t_end ? s0 * a.scale_log2 : kNegBig;
+      sc[t][1] = tok + 1 < t_end ? s1 * a.scale_log2 : kNegBig;
+    }
+    // ---- online softmax of row g over the group's 32 tokens (8 per lane, 4 lanes per row) ------
+    float mx = fmaxf(fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1])),
+                     fmaxf(fmaxf(sc[2][0], sc[2][1]), fmaxf(sc[3][0], sc[3][1])));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    const float m_new = fmaxf(m_run, mx);
+    const float corr = exp2f(m_run - m_new);
+    m_run = m_new;
+    // probabilities as 16-bit A fragments.  bf16 keeps 8 bits, too few for the output's tolerance, so
+    // a probability goes in as two terms (rounded value + rounded remainder, together good to 2^-17).
+    uint32_t pa[4], pb[4];
+    float lsum = 0.0f;
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      // masked tokens get probability 0 even when the whole group is masked (sc == m_new == kNegBig)
+      const float p0 = sc[t][0] > 0.5f * kNegBig ? exp2f(sc[t][0] - m_new) : 0.0f;
+      const float p1 = sc[t][1] > 0.5f * kNegBig ? exp2f(sc[t][1] - m_new) : 0.0f;
+      pa[t] = store16x2<kBf16>(p0, p1);
+      if constexpr (kBf16) {
+        pb[t] = store16x2<kBf16>(p0 - load16<kBf16>(uint16_t(pa[t] & 0xffffu)),
+                                 p1 - load16<kBf16>(uint16_t(pa[t] >> 16)));
+        lsum += p0 + p1;
+      } else {
+        pb[t] = 0u;
+        // the row sum uses the rounded probabilities, the ones the output product multiplies by
+        lsum += load16<kBf16>(uint16_t(pa[t] & 0xffffu)) + load16<kBf16>(uint16_t(pa[t] >> 16));
+      }
+    }
+    l_run = fmaf(l_run, corr, lsum);
+#pragma unroll
+    for (int u = 0; u < NOT; ++u) {
+      o[u][0] *= corr;
+      o[u][1] *= corr;
+    }
+    // ---- output: O[g][:] += P[g][tokens] * V[tokens][:] ---------------------------------------------
+#pragma unroll
+    for (int ks = 0; ks < 2; ++ks) {
+#pragma unroll
+      for (int h = 0; h < NVH; ++h) {
+        const uint32_t w0[4] = {vq[ks][0][h].x, vq[ks][0][h].y, vq[ks][0][h].z, vq[ks][0][h].w};
+        const uint32_t w1[4] = {vq[ks][1][h].x, vq[ks][1][h].y, vq[ks][1][h].z, vq[ks][1][h].w};
+        const uint32_t w2[4] = {vq[ks][2][h].x, vq[ks][2][h].y, vq[ks][2][h].z, vq[ks][2][h].w};
+        const uint32_t w3[4] = {vq[ks][3][h].x, vq[ks][3][h].y, vq[ks][3][h].z, vq[ks][3][h].w};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;
+          const uint32_t b0 = __byte_perm(w0[e >> 1], w1[e >> 1], sel);
+          const uint32_t b1 = __byte_perm(w2[e >> 1], w3[e >> 1], sel);
+          mma_16x8x16<kBf16>(o[h * 8 + e][0], o[h * 8 + e][1], dz0, dz1, pa[2 * ks], 0u, pa[2 * ks + 1], 0u, b0, b1);
+          if constexpr (kBf16)
+            mma_16x8x16<kBf16>(o[h * 8 + e][0], o[h * 8 + e][1], dz0, dz1, pb[2 * ks], 0u, pb[2 * ks + 1], 0u, b0, b1);
+        }
+      }
     }
   }
-  // merge the four token groups of the warp
-#pragma unroll
-  for (int mask = 8; mask <= 16; mask <<= 1) {
-#pragma unroll
-    for (int g = 0; g < GQ; ++g) {
-      const float m_o = __shfl_xor_sync(0xffffffffu, m[g], mask);
-      const float l_o = __shfl_xor_sync(0xffffffffu, l[g], mask);
-      const float m_new = fmaxf(m[g], m_o);
-      const float c_s = exp2f(m[g] - m_new), c_o = exp2f(m_o - m_new);
-      l[g] = l[g] * c_s + l_o * c_o;
-#pragma unroll
-      for (int i = 0; i < DPL; ++i) {
-        const float a_o = __shfl_xor_sync(0xffffffffu, acc[g][i], mask);
-        acc[g][i] = acc[g][i] * c_s + a_o * c_o;
-      }
-      m[g] = m_new;
+  // ---- merge the warps of the CTA -----------------------------------------------------------------
+  l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+  l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+  if (g < gq) {
+    if (j == 0) {
+      sm_m[warp][g] = m_run;
+      sm_l[warp][g] = l_run;
     }
-  }
-  if (tg == 0) {
 #pragma unroll
-    for (int g = 0; g < GQ; ++g) {
-      if (dl == 0) {
-        sm_m[warp][g] = m[g];
-        sm_l[warp][g] = l[g];
-      }
-#pragma unroll
-      for (int pc = 0; pc < NP; ++pc)
-#pragma unroll
-        for (int i = 0; i < 8; ++i) sm_o[warp][g][pc * 64 + dl * 8 + i] = acc[g][pc * 8 + i];
+    for (int u = 0; u < NOT; ++u) {
+      const int base = (u < 8 ? 0 : 64) + (u & 7);
+      sm_o[warp][g][base + (2 * j) * 8] = o[u][0];
+      sm_o[warp][g][base + (2 * j + 1) * 8] = o[u][1];
     }
   }
   __syncthreads();
-  // merge the warps; thread -> (query head g, dimension i)
-  for (int idx = threadIdx.x; idx < GQ * HD; idx += kAttnThreads) {
-    const int g = idx / HD, i = idx % HD;
+  // thread -> (query head q, dimension i)
+  for (int idx = threadIdx.x; idx < gq * HD; idx += kAttnMmaThreads) {
+    const int qi = idx / HD, i = idx % HD;
     float M = kNegBig;
 #pragma unroll
-    for (int w = 0; w < kAttnWarps; ++w) M = fmaxf(M, sm_m[w][g]);
-    float o = 0.0f, L = 0.0f;
+    for (int w = 0; w < kAttnMmaWarps; ++w) M = fmaxf(M, sm_m[w][qi]);
+    float ov = 0.0f, L = 0.0f;
 #pragma unroll
-    for (int w = 0; w < kAttnWarps; ++w) {
-      const float sc = exp2f(sm_m[w][g] - M);
-      o = fmaf(sm_o[w][g][i], sc, o);
-      L = fmaf(sm_l[w][g], sc, L);
+    for (int w = 0; w < kAttnMmaWarps; ++w) {
+      const float scl = exp2f(sm_m[w][qi] - M);
+      ov = fmaf(sm_o[w][qi][i], scl, ov);
+      L = fmaf(sm_l[w][qi], scl, L);
     }
-    const int qh = kvh * rep + g0 + g;
+    const int qh = kvh * rep + g0 + qi;
     const long long pidx = ((long long)b * a.n_splits + split) * a.n_q_heads + qh;
-    a.part_o[pidx * HD + i] = o;
+    a.part_o[pidx * HD + i] = ov;
     if (i == 0) {
       a.part_ml[pidx * 2] = M;
       a.part_ml[pidx * 2 + 1] = L;
