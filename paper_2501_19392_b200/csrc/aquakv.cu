@@ -578,7 +578,7 @@ int aquakv_create(const aquakv_params* params, const float* grid_host, const int
   c->code_bytes = d / 2 * c->bits / 8;
   c->n_groups = d / params->scale_group;
   c->bf16 = params->dtype == AQUAKV_BF16;
-  c->attn_block_tokens = 256;
+  c->attn_block_tokens = 1024;
 
   float4 g4[256];
   for (int i = 0; i < n; ++i) {

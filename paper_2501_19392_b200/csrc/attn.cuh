@@ -112,9 +112,9 @@ __global__ void __launch_bounds__(kAttnMmaThreads, 2) attn_partial_kernel(const 
   const long long row0 = (long long)b * a.ctx - a.tok_base;
   const uint16_t* kbase = a.Kh + kvh * HD;
   const uint16_t* vbase = a.Vh + kvh * HD;
-  for (int tb = t_begin + warp * 32; tb < t_end; tb += 32 * kAttnMmaWarps) {
-    // ---- all loads of the group: keys (score tile t, token g of it), values (k-step ks, tokens 2j.. of it) ----
-    uint4 kq[4][NCH];
+  // keys of a group: score tile t, token g of it, 16-byte piece j of every 32-dimension chunk
+  uint4 kq[4][NCH];
+  auto load_keys = [&](int tb) {
 #pragma unroll
     for (int t = 0; t < 4; ++t) {
       const int tok = tb + 8 * t + g;
@@ -122,6 +122,10 @@ __global__ void __launch_bounds__(kAttnMmaThreads, 2) attn_partial_kernel(const 
 #pragma unroll
       for (int c = 0; c < NCH; ++c) kq[t][c] = __ldcs(reinterpret_cast<const uint4*>(kp + c * 32));
     }
+  };
+  if (t_begin + warp * 32 < t_end) load_keys(t_begin + warp * 32);
+  for (int tb = t_begin + warp * 32; tb < t_end; tb += 32 * kAttnMmaWarps) {
+    // ---- values of this group (k-step ks, tokens 2j.. of it); its keys were fetched one group ahead ----
     uint4 vq[2][4][NVH];
 #pragma unroll
     for (int ks = 0; ks < 2; ++ks) {
@@ -147,6 +151,7 @@ __global__ void __launch_bounds__(kAttnMmaThreads, 2) attn_partial_kernel(const 
       sc[t][0] = tok < t_end ? s0 * a.scale_log2 : kNegBig;
       sc[t][1] = tok + 1 < t_end ? s1 * a.scale_log2 : kNegBig;
     }
+    if (tb + 32 * kAttnMmaWarps < t_end) load_keys(tb + 32 * kAttnMmaWarps);   // in flight during the rest
     // ---- online softmax of row g over the group's 32 tokens (8 per lane, 4 lanes per row) ------
     float mx = fmaxf(fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1])),
                      fmaxf(fmaxf(sc[2][0], sc[2][1]), fmaxf(sc[3][0], sc[3][1])));
