@@ -19,7 +19,9 @@ CASES = [
     (2, 300, 32, 8, 128, synth.BF16, True),     # Llama-3.1-8B head layout, ragged split blocks
     (3, 700, 24, 8, 128, synth.BF16, True),     # 3 query heads per KV head
     (1, 1, 32, 8, 128, synth.BF16, False),      # single cached token
-    (2, 257, 64, 8, 128, synth.F16, True),      # 8 query heads per KV head (two passes)
+    (2, 257, 64, 8, 128, synth.F16, True),      # 8 query heads per KV head (all rows of the tile in use)
+    (2, 2500, 40, 8, 128, synth.BF16, True),    # 5 query heads per KV head, three split blocks, ragged last one
+    (1, 1025, 56, 8, 64, synth.F16, False),     # 7 per KV head, head_dim 64, one token past a block boundary
     (2, 130, 32, 8, 64, synth.F16, True),       # head_dim 64 (d_kv = 512)
     (1, 2100, 8, 8, 128, synth.BF16, False),    # MHA-style, several chunks of blocks
 ]
