@@ -93,16 +93,23 @@ int aquakv_create(const aquakv_params* params, const float* grid_host, const int
 /*
  * The host-built cell table that prunes the nearest-point search of Q (Section 2: each pair of
  * rotated values goes to the nearest grid point).  The square [-half_extent, half_extent)^2 is cut
- * into cells_per_side^2 cells; entry [iy*cells_per_side + ix] holds, in bytes 0..3, the ascending
- * indices of every grid point that is nearest somewhere in that cell (short lists repeat the last
- * index; at most three distinct ones for grid_size 16, four otherwise), and 0xFFFFFFFF means "search
- * all points" (cells with more candidates, and the border cells, which also stand for everything
- * outside the square).  The kernels use the same
- * table, so a host test can check that it never excludes the true nearest point.  HOST memory
- * only, no GPU needed.  table == NULL: only report the dimensions.
+ * into cells_per_side^2 cells; entry [iy*cells_per_side + ix] holds, in bytes 3, 2, 1, 0, the
+ * ascending indices of every grid point that is nearest somewhere in that cell (byte 3 the lowest;
+ * short lists repeat the last index; at most three distinct ones for grid_size 16, four otherwise).
+ * For grid_size 256 a cell with more candidates, up to eight, holds 0xFF000000 + i, a reference to
+ * second-level list i (the smaller grids practically never need one and have none):
+ * words [cells^2 + 2i, cells^2 + 2i + 1] of the same buffer hold its eight ascending candidates, one
+ * per byte, byte 0 of the first word the lowest.  0xFFFFFFFF means "search all points" (cells with
+ * still more candidates, and the border cells, which also stand for everything outside the square).
+ * The kernels use the same table, so a host test can check that it never excludes the true nearest
+ * point.  HOST memory only, no GPU needed.  table == NULL: only report the dimensions; otherwise
+ * table_capacity (in words) must be at least cells^2 + AQUAKV_SEARCH_TABLE_LIST_WORDS.
+ * second_level_lists (may be NULL) receives the number of second-level lists in use.
  */
+#define AQUAKV_SEARCH_TABLE_LIST_WORDS 4096
 int aquakv_search_table_host(const float* grid_host, int32_t grid_size, int32_t* cells_per_side,
-                             float* half_extent, uint32_t* table, size_t table_capacity);
+                             float* half_extent, uint32_t* table, size_t table_capacity,
+                             int32_t* second_level_lists);
 
 /* Frees the context's device tables.  NULL is accepted.  Pending work must have completed. */
 int aquakv_destroy(aquakv_ctx* ctx);

@@ -56,7 +56,8 @@ def _load():
     L.aquakv_code_bytes.restype = ctypes.c_int
     L.aquakv_code_bytes.argtypes = [ctypes.POINTER(Params)]
     L.aquakv_search_table_host.restype = ctypes.c_int
-    L.aquakv_search_table_host.argtypes = [vp, i32, ctypes.POINTER(i32), ctypes.POINTER(f32), vp, sz]
+    L.aquakv_search_table_host.argtypes = [vp, i32, ctypes.POINTER(i32), ctypes.POINTER(f32), vp, sz,
+                                           ctypes.POINTER(i32)]
     L.aquakv_create.restype = ctypes.c_int
     L.aquakv_create.argtypes = [ctypes.POINTER(Params), vp, vp, vp, ctypes.POINTER(vp)]
     L.aquakv_destroy.restype = ctypes.c_int
@@ -109,19 +110,26 @@ def code_bytes(d_kv: int, grid_size: int, had_block: int = 64, scale_group: int 
     return int(lib.aquakv_code_bytes(ctypes.byref(p)))
 
 
+SEARCH_TABLE_LIST_WORDS = 4096
+
+
 def search_table(grid: np.ndarray):
-    """(cells_per_side, half_extent, table uint32 [cells, cells]) of aquakv_search_table_host."""
+    """(cells_per_side, half_extent, table uint32 [cells, cells], lists uint8 [n_lists, 8]) of
+    aquakv_search_table_host: the cell entries and the second-level candidate lists they refer to."""
     g = np.ascontiguousarray(grid, dtype=np.float32)
-    cells, half = ctypes.c_int32(0), ctypes.c_float(0.0)
-    rc = lib.aquakv_search_table_host(g.ctypes.data, g.shape[0], ctypes.byref(cells), ctypes.byref(half), None, 0)
+    cells, half, n_lists = ctypes.c_int32(0), ctypes.c_float(0.0), ctypes.c_int32(0)
+    rc = lib.aquakv_search_table_host(g.ctypes.data, g.shape[0], ctypes.byref(cells), ctypes.byref(half), None, 0,
+                                      None)
     if rc:
         raise AquaKVError(rc, "aquakv_search_table_host")
-    table = np.zeros((cells.value, cells.value), dtype=np.uint32)
+    c = cells.value
+    buf = np.zeros(c * c + SEARCH_TABLE_LIST_WORDS, dtype=np.uint32)
     rc = lib.aquakv_search_table_host(g.ctypes.data, g.shape[0], ctypes.byref(cells), ctypes.byref(half),
-                                      table.ctypes.data, table.size)
+                                      buf.ctypes.data, buf.size, ctypes.byref(n_lists))
     if rc:
         raise AquaKVError(rc, "aquakv_search_table_host")
-    return int(cells.value), float(half.value), table
+    lists = buf[c * c:c * c + 2 * n_lists.value].view(np.uint8).reshape(n_lists.value, 8)
+    return int(c), float(half.value), buf[:c * c].reshape(c, c).copy(), lists.copy()
 
 
 def _ptr(t) -> Optional[int]:

@@ -543,7 +543,8 @@ const char* aquakv_status_string(int status) {
 }
 
 int aquakv_search_table_host(const float* grid_host, int32_t grid_size, int32_t* cells_per_side,
-                             float* half_extent, uint32_t* table, size_t table_capacity) {
+                             float* half_extent, uint32_t* table, size_t table_capacity,
+                             int32_t* second_level_lists) {
   if (grid_host == nullptr || cells_per_side == nullptr || half_extent == nullptr)
     return AQUAKV_ERR_INVALID_ARG;
   if (grid_size != 16 && grid_size != 64 && grid_size != 256) return AQUAKV_ERR_UNSUPPORTED;
@@ -553,8 +554,9 @@ int aquakv_search_table_host(const float* grid_host, int32_t grid_size, int32_t*
   *cells_per_side = spec.cells;
   *half_extent = spec.half;
   if (table == nullptr) return AQUAKV_OK;
-  if (table_capacity < size_t(spec.cells) * spec.cells) return AQUAKV_ERR_INVALID_ARG;
-  build_search_table(grid_host, grid_size, spec, table);
+  if (table_capacity < search_table_words(spec)) return AQUAKV_ERR_INVALID_ARG;
+  const int n_lists = build_search_table(grid_host, grid_size, spec, table);
+  if (second_level_lists != nullptr) *second_level_lists = n_lists;
   return AQUAKV_OK;
 }
 
@@ -591,7 +593,7 @@ int aquakv_create(const aquakv_params* params, const float* grid_host, const int
     g4[i] = make_float4(gx, gy, 0.0f, 0.0f);
   }
   c->search_spec = search_table_spec(grid_host, n);
-  std::vector<uint32_t> table(size_t(c->search_spec.cells) * c->search_spec.cells);
+  std::vector<uint32_t> table(search_table_words(c->search_spec));
   build_search_table(grid_host, n, c->search_spec, table.data());
   uint32_t masks[2][32];
   std::memset(masks, 0, sizeof(masks));

@@ -65,9 +65,10 @@ constexpr int kCodecThreads = kCodecWarps * 32;
 constexpr int kSearchCells = 64;          // cells per side of the table (see search_table.h)
 constexpr int kSearchLogCells = 6;
 constexpr uint32_t kCellBruteDev = 0xFFFFFFFFu;   // "search all points" (the largest entry value)
+constexpr uint32_t kCellSpecialDev = 0xFF000000u; // entries from here up: second-level list (low 24 bits) or kCellBruteDev
 
 struct SearchDev {
-  const uint32_t* table;   // global copy [64*64] of the candidate lists
+  const uint32_t* table;   // global copy [64*64] of the candidate lists, then the second-level lists (two words each)
   float inv_w;             // cells / (2 * half extent)
 };
 
@@ -76,11 +77,13 @@ template <int NPTS>
 struct RowSmem {
   uint32_t table[kSearchCells * kSearchCells];
   f32x2_t grid[NPTS];      // (g.x, g.y) as packed fp32 pairs
+  const uint2* lists;      // second-level candidate lists (global memory: only the rare path reads them)
 };
 
 template <int NPTS>
 __device__ __forceinline__ void row_smem_fill(RowSmem<NPTS>* rs, const uint32_t* table, const float4* grid4) {
   for (int i = threadIdx.x; i < kSearchCells * kSearchCells; i += blockDim.x) rs->table[i] = table[i];
+  if (threadIdx.x == 0) rs->lists = reinterpret_cast<const uint2*>(table + kSearchCells * kSearchCells);
   for (int i = threadIdx.x; i < NPTS; i += blockDim.x) {
     const float4 g = grid4[i];
     rs->grid[i] = pack2(g.x, g.y);
@@ -210,10 +213,11 @@ __device__ __forceinline__ float pair_dist(f32x2_t y, f32x2_t g) {
   return __fadd_rn(qx, qy);
 }
 
-// Arg-min over the ascending candidates of a table entry (three for n = 16, else four).
+// Arg-min over the ascending candidates of a table entry (bytes 3, 2, 1 and, for n > 16, 0).  Indices
+// are masked to the grid so that special entries, whose result is replaced afterwards, stay in range.
 template <int NPTS>
 __device__ __forceinline__ int nearest_of_candidates(f32x2_t y, uint32_t e, const f32x2_t* __restrict__ grid_s) {
-  const int c0 = e & 0xffu, c1 = (e >> 8) & 0xffu, c2 = (e >> 16) & 0xffu;
+  const int c0 = (e >> 24) & (NPTS - 1), c1 = (e >> 16) & (NPTS - 1), c2 = (e >> 8) & (NPTS - 1);
   const float t0 = pair_dist(y, grid_s[c0]);
   const float t1 = pair_dist(y, grid_s[c1]);
   const float t2 = pair_dist(y, grid_s[c2]);
@@ -222,21 +226,38 @@ __device__ __forceinline__ int nearest_of_candidates(f32x2_t y, uint32_t e, cons
   if (t1 < best) { best = t1; idx = c1; }
   if (t2 < best) { best = t2; idx = c2; }
   if constexpr (NPTS > 16) {
-    const int c3 = e >> 24;
+    const int c3 = e & (NPTS - 1);
     const float t3 = pair_dist(y, grid_s[c3]);
     if (t3 < best) { idx = c3; }
   }
   return idx;
 }
 
+// The pair's nearest point for a special table entry: arg-min over all points or, for the large grid
+// (the host builds second-level lists only for n > 64: smaller grids practically never need them),
+// over the entry's list of eight ascending candidates (repeats at the end change nothing).  One
+// rolled loop, so that this rarely taken path adds little code and no registers to the row loop.
 template <int NPTS>
-__device__ __forceinline__ int nearest_exhaustive(f32x2_t y, const f32x2_t* __restrict__ grid_s) {
+__device__ __forceinline__ int nearest_special(f32x2_t y, uint32_t e, const RowSmem<NPTS>* rsm) {
   float best = 3.0e38f;
   int idx = 0;
+  if constexpr (NPTS > 64) {
+    const bool all = e == kCellBruteDev;
+    uint2 lst = make_uint2(0u, 0u);
+    if (!all) lst = __ldg(rsm->lists + (e & 0x00FFFFFFu));
+    const int count = all ? NPTS : 8;
 #pragma unroll 1
-  for (int i = 0; i < NPTS; ++i) {
-    const float t = pair_dist(y, grid_s[i]);
-    if (t < best) { best = t; idx = i; }             // strict: lowest index wins ties
+    for (int i = 0; i < count; ++i) {
+      const int c = all ? i : int((((i & 4) ? lst.y : lst.x) >> (8 * (i & 3))) & (NPTS - 1));
+      const float t = pair_dist(y, rsm->grid[c]);
+      if (t < best) { best = t; idx = c; }             // strict: lowest index wins ties
+    }
+  } else {
+#pragma unroll 1
+    for (int i = 0; i < NPTS; ++i) {
+      const float t = pair_dist(y, rsm->grid[i]);
+      if (t < best) { best = t; idx = i; }
+    }
   }
   return idx;
 }
@@ -505,14 +526,14 @@ __device__ __forceinline__ void encode_row_core(const RowCtx& rc, const RowSmem<
     entry[k] = search_entry(y0, y1, rc.inv_w, rsm->table);
     emax = max(emax, entry[k]);
   }
-  const bool slow = __any_sync(0xffffffffu, emax == kCellBruteDev);
+  const bool slow = __any_sync(0xffffffffu, emax >= kCellSpecialDev);
   int idx[4];
 #pragma unroll
   for (int k = 0; k < 4; ++k) idx[k] = nearest_of_candidates<NPTS>(vp[k], entry[k], rsm->grid);
-  if (slow) {                    // rare: some lane of the warp has a pair that needs the exhaustive search
+  if (slow) {     // some lane of the warp has a pair in a cell with more candidates (rare for n <= 64)
 #pragma unroll
     for (int k = 0; k < 4; ++k)
-      if (entry[k] == kCellBruteDev) idx[k] = nearest_exhaustive<NPTS>(vp[k], rsm->grid);
+      if (entry[k] >= kCellSpecialDev) idx[k] = nearest_special<NPTS>(vp[k], entry[k], rsm);
   }
   uint32_t word = 0;
 #pragma unroll

@@ -5,13 +5,19 @@
 // The square [-B, B)^2 is cut into C x C cells.  For each cell the table lists every grid point
 // whose Voronoi region meets the (slightly inflated) cell, so the exact arg-min over ALL points
 // equals the arg-min over the listed ones for any y inside the cell.  Cells that need more
-// candidates than the kernel evaluates (three for n = 16, four for larger grids), and values
-// outside the square, are searched exhaustively by the kernel; the table therefore never changes a
-// result, it only skips points that cannot win.
+// candidates than the kernel evaluates in its fast path (three for n = 16, four for larger grids)
+// are searched exhaustively by the kernel, and so are values outside the square; for n > 64, where
+// such cells are common, those with at most eight candidates point to a second-level list of eight
+// instead.  The table therefore never changes a result,
+// it only skips points that cannot win.
 //
-// Entry layout (uint32): bytes 0..3 = candidate indices in ascending order (short lists repeat
-// their last index); 0xFFFFFFFF marks a cell that must be searched exhaustively, which includes all
-// border cells: the kernel clamps cell coordinates, so they stand for everything outside the square.
+// Entry layout (uint32): bytes 3, 2, 1, 0 = candidate indices in ascending order (byte 3 the
+// lowest; short lists repeat their last index), so every plain entry is below 0xFF000000 unless
+// its only candidate is point 255.  0xFF000000 + i points to second-level list i (two uint32 after
+// the cells: eight ascending candidates, byte 0 of the first word the lowest, short lists repeat
+// their last index).  0xFFFFFFFF marks a cell that must be searched exhaustively, which includes
+// all border cells: the kernel clamps cell coordinates, so they stand for everything outside the
+// square.  The kernel finds the special entries with one unsigned comparison.
 #pragma once
 
 #include <cmath>
@@ -22,6 +28,9 @@ namespace aquakv {
 
 constexpr uint32_t kCellBrute = 0xFFFFFFFFu;   // the largest entry value; as a candidate list it could only
                                                // mean "point 255 alone", for which searching all points is right too
+constexpr uint32_t kCellSpecial = 0xFF000000u; // entries >= this are second-level references or kCellBrute
+constexpr int kSearchMaxLists = 2048;          // second-level lists the table has room for
+constexpr int kSearchListLen = 8;
 
 struct SearchTableSpec {
   int cells;        // C, cells per side (power of two)
@@ -63,8 +72,14 @@ inline void clip(std::vector<Pt>& poly, double ax, double ay, double b) {
 }
 }  // namespace detail
 
-// Fills table[cells*cells] (row = y cell, column = x cell).
-inline void build_search_table(const float* grid, int n, const SearchTableSpec& s, uint32_t* table) {
+// Words of a table buffer: the cells followed by the second-level lists (two words each).
+inline size_t search_table_words(const SearchTableSpec& s) {
+  return size_t(s.cells) * s.cells + size_t(2) * kSearchMaxLists;
+}
+
+// Fills table[cells*cells] (row = y cell, column = x cell) and the second-level lists behind it;
+// returns the number of lists used (the rest of the buffer is zeroed).
+inline int build_search_table(const float* grid, int n, const SearchTableSpec& s, uint32_t* table) {
   const int C = s.cells;
   const double w = 1.0 / double(s.inv_w);
   const double eps = 1e-3 * w + 1e-5;        // covers fp32 rounding of the cell index and scores
@@ -72,6 +87,9 @@ inline void build_search_table(const float* grid, int n, const SearchTableSpec& 
   std::vector<double> dist(n);
   std::vector<int> pre, cand;
   std::vector<detail::Pt> poly;
+  uint32_t* lists = table + size_t(C) * C;
+  for (int i = 0; i < 2 * kSearchMaxLists; ++i) lists[i] = 0;
+  int n_lists = 0;
   for (int iy = 0; iy < C; ++iy) {
     for (int ix = 0; ix < C; ++ix) {
       const double x0 = (ix - C / 2) * w - eps, x1 = (ix + 1 - C / 2) * w + eps;
@@ -104,16 +122,26 @@ inline void build_search_table(const float* grid, int n, const SearchTableSpec& 
       uint32_t e;
       // border cells also catch every value outside the square (the kernel's cell index saturates)
       const bool border = ix == 0 || iy == 0 || ix == C - 1 || iy == C - 1;
-      if (border || cand.empty() || int(cand.size()) > s.max_cand) {
+      const int nc = int(cand.size());
+      auto at = [&](int k) { return uint32_t(cand[k < nc ? k : nc - 1]); };
+      const bool may_list = n > 64 && nc <= kSearchListLen && n_lists < kSearchMaxLists;
+      if (border || cand.empty() || (nc > s.max_cand && !may_list)) {
         e = kCellBrute;
+      } else if (nc > s.max_cand) {
+        e = kCellSpecial + uint32_t(n_lists);
+        for (int k = 0; k < 4; ++k) {
+          lists[2 * n_lists] |= at(k) << (8 * k);
+          lists[2 * n_lists + 1] |= at(4 + k) << (8 * k);
+        }
+        ++n_lists;
       } else {
         e = 0;
-        for (int k = 0; k < 4; ++k)
-          e |= uint32_t(cand[k < int(cand.size()) ? k : int(cand.size()) - 1]) << (8 * k);
+        for (int k = 0; k < 4; ++k) e |= at(k) << (8 * (3 - k));
       }
       table[size_t(iy) * C + ix] = e;
     }
   }
+  return n_lists;
 }
 
 }  // namespace aquakv

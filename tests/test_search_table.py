@@ -8,21 +8,28 @@ import pytest
 from paper_2501_19392_b200 import synth
 
 
-def _candidates(table, cells, half, y):
+def _candidates(table, lists, cells, half, y):
+    """Candidate lists (8 wide, ascending, padded by repetition) of the cells the points fall in; `brute`
+    marks cells that say "search all points", `second` those that refer to a second-level list."""
     w = 2.0 * half / cells
     ix = np.clip(np.floor((y[:, 0] + half) / w).astype(np.int64), 0, cells - 1)   # the kernel's cell index saturates
     iy = np.clip(np.floor((y[:, 1] + half) / w).astype(np.int64), 0, cells - 1)
-    e = table[iy, ix]
+    e = table[iy, ix].astype(np.int64)
     brute = e == 0xFFFFFFFF
-    cand = np.stack([e & 0xFF, (e >> 8) & 0xFF, (e >> 16) & 0xFF, (e >> 24) & 0xFF], axis=1).astype(np.int64)
-    return cand, brute
+    second = (e >= 0xFF000000) & ~brute
+    first = np.stack([(e >> 24) & 0xFF, (e >> 16) & 0xFF, (e >> 8) & 0xFF, e & 0xFF], axis=1)
+    cand = np.concatenate([first, first[:, 3:4].repeat(4, axis=1)], axis=1)
+    if second.any():
+        cand[second] = lists[e[second] & 0xFFFFFF].astype(np.int64)
+    return cand, brute, second
 
 
 @pytest.mark.parametrize("n", [16, 64, 256])
 def test_table_keeps_the_nearest_point(n):
     from paper_2501_19392_b200 import api
     grid = synth.lloyd_grid(n, seed=7, n_samples=1 << 14, iters=25)
-    cells, half, table = api.search_table(grid)
+    cells, half, table, lists = api.search_table(grid)
+    assert len(lists) <= api.SEARCH_TABLE_LIST_WORDS // 2
     assert cells == 64 and half >= np.abs(grid).max() + 2.0
     G = grid.astype(np.float64)
     rng = np.random.default_rng(n)
@@ -46,7 +53,7 @@ def test_table_keeps_the_nearest_point(n):
         order = np.argsort(dist, axis=1)
         best = order[:, 0]
         margin = (np.take_along_axis(dist, order[:, 1:2], 1)[:, 0] - dist[np.arange(len(y)), best])
-        cand, brute = _candidates(table, cells, half, y)
+        cand, brute, lvl2 = _candidates(table, lists, cells, half, y)
         listed = (cand == best[:, None]).any(axis=1)
         assert np.all(listed | brute), "%s: nearest point missing from %d cells" % (name, (~(listed | brute)).sum())
         # near-ties (fp32 could pick either point): both contenders must be listed
@@ -56,10 +63,20 @@ def test_table_keeps_the_nearest_point(n):
         # candidates are ascending so that the first minimum is the lowest index
         asc = ~brute
         assert np.all(np.diff(cand[asc], axis=1) >= 0)
-        if n == 16:     # the kernel evaluates three candidates there: the fourth byte only repeats the third
-            assert np.all(cand[asc][:, 3] == cand[asc][:, 2])
+        # the kernel's fast path evaluates three candidates for n = 16 and four otherwise: cells with
+        # more must go through a second-level list
+        plain = ~brute & ~lvl2
+        distinct = (np.diff(cand[plain][:, :4], axis=1) > 0).sum(axis=1) + 1
+        assert np.all(distinct <= (3 if n == 16 else 4))
+        if n == 16:     # the fourth byte only repeats the third
+            assert np.all(cand[plain][:, 3] == cand[plain][:, 2])
+        if lvl2.any():
+            assert np.all((np.diff(cand[lvl2], axis=1) > 0).sum(axis=1) + 1 > (3 if n == 16 else 4))
         # values outside the square land in border cells, which must all say "search all points"
         assert np.all(table[0, :] == 0xFFFFFFFF) and np.all(table[-1, :] == 0xFFFFFFFF)
         assert np.all(table[:, 0] == 0xFFFFFFFF) and np.all(table[:, -1] == 0xFFFFFFFF)
-        if name == "gauss":
-            assert brute.mean() < (0.02 if n <= 64 else 0.25), brute.mean()
+        if n <= 64:             # second-level lists exist only for the 256-point grid
+            assert not lvl2.any() and len(lists) == 0
+        if name == "gauss":     # the exhaustive search must stay rare
+            assert brute.mean() < (0.02 if n <= 64 else 1e-3), brute.mean()
+            assert lvl2.mean() < 0.25, lvl2.mean()
