@@ -1,8 +1,8 @@
 // Host side of the AQUA-KV codec library: the C ABI declared in include/aquakv.h, argument
 // validation, workspace carving, tensor-map construction and kernel launches.  Every step of
 // Algorithm 2 / Algorithm 3 / the attention read of Algorithm 4 runs in the kernels of
-// gemm_pred.cuh, codec.cuh and attn.cuh; nothing is computed on the host and there is no
-// fallback path.
+// layer_kernel.cuh, gemm_pred.cuh, codec.cuh and attn.cuh; nothing is computed on the host and
+// there is no fallback path.
 //
 // Large calls are cut into token chunks sized so that one chunk's fp32 prediction (and, for the
 // fused attention, its decoded keys/values) stays resident in the 126 MB L2 between the kernel
@@ -426,13 +426,6 @@ void launch_layer_dec_t(int* rc, int device, cudaStream_t st, int grid, const CU
   *rc = launch_layer_t<false, D, NPTS, BF, false>(device, st, grid, tm, a);
 }
 
-// The fused kernel needs its whole shared-memory budget in one CTA; the largest grid (256 points)
-// does not fit next to the encoder's search table, so that combination uses the separate GEMM and
-// row kernels instead.
-bool layer_kernel_fits(const aquakv_ctx* c, bool encode) {
-  return !(encode && c->p.grid_size == 256);
-}
-
 // Algorithm 2 (encode = true) or Algorithm 3 for one layer with predictors, all tokens, one launch.
 int launch_layer(aquakv_ctx* c, cudaStream_t st, bool encode, int64_t T, const void* K, const void* V,
                  int64_t ld_kv, const void* Khat_prev, const void* Vhat_prev, int64_t ld_prev,
@@ -853,43 +846,26 @@ int aquakv_encode(aquakv_ctx* c, int64_t n_tokens, const void* K, const void* V,
       return AQUAKV_ERR_WORKSPACE;
     if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
   }
-  if (has_pred && layer_kernel_fits(c, true)) {
+  if (has_pred) {
     if (n_tokens > (int64_t(1) << 30)) return AQUAKV_ERR_UNSUPPORTED;
     return launch_layer(c, static_cast<cudaStream_t>(cuda_stream), true, n_tokens, K, V, ld_kv, Khat_prev,
                         Vhat_prev, ld_prev, Wk, Wv, bk, bv, Kcodes, Kscales, Vcodes, Vscales, Khat, Vhat,
                         ld_hat, workspace);
   }
+  // no predictor (layer 0): the row kernels alone
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  uint8_t* wsb = static_cast<uint8_t*>(workspace);
-  float* P = has_pred ? reinterpret_cast<float*>(wsb + ws.p_off) : nullptr;
   const int cb = c->code_bytes, ng = c->n_groups;
   const uint16_t* Kp = static_cast<const uint16_t*>(K);
   const uint16_t* Vp = static_cast<const uint16_t*>(V);
-  const uint16_t* Kpv = static_cast<const uint16_t*>(Khat_prev);
-  const uint16_t* Vpv = static_cast<const uint16_t*>(Vhat_prev);
   for (int64_t t0 = 0; t0 < n_tokens; t0 += ws.chunk) {
     const int rows = int(n_tokens - t0 < ws.chunk ? n_tokens - t0 : ws.chunk);
-    // keys: Algorithm 2 lines 5-7
-    uint16_t* khat_c = Khat != nullptr ? static_cast<uint16_t*>(Khat) + t0 * ld_hat
-                                       : reinterpret_cast<uint16_t*>(wsb + ws.khat_off);
-    const int64_t ld_khat_c = Khat != nullptr ? ld_hat : d;
-    if (has_pred) {
-      rc = launch_predict(c, st, rows, Kpv + t0 * ld_prev, nullptr, ld_prev, 0, Wk, bk, P, d);
-      if (rc) return rc;
-    }
-    rc = launch_encode_rows(c, st, kRoleK, rows, Kp + t0 * ld_kv, ld_kv, P, d, Kcodes + t0 * cb,
-                            Kscales + t0 * ng, (has_pred || Khat != nullptr) ? khat_c : nullptr,
-                            ld_khat_c);
+    rc = launch_encode_rows(c, st, kRoleK, rows, Kp + t0 * ld_kv, ld_kv, nullptr, d, Kcodes + t0 * cb,
+                            Kscales + t0 * ng,
+                            Khat != nullptr ? static_cast<uint16_t*>(Khat) + t0 * ld_hat : nullptr, ld_hat);
     if (rc) return rc;
-    // values: Algorithm 2 lines 8-9 (the value predictor reads the rounded Khat)
-    if (has_pred) {
-      rc = launch_predict(c, st, rows, Vpv + t0 * ld_prev, khat_c, ld_prev, ld_khat_c, Wv, bv, P, d);
-      if (rc) return rc;
-    }
-    rc = launch_encode_rows(c, st, kRoleV, rows, Vp + t0 * ld_kv, ld_kv, P, d, Vcodes + t0 * cb,
+    rc = launch_encode_rows(c, st, kRoleV, rows, Vp + t0 * ld_kv, ld_kv, nullptr, d, Vcodes + t0 * cb,
                             Vscales + t0 * ng,
-                            Vhat != nullptr ? static_cast<uint16_t*>(Vhat) + t0 * ld_hat : nullptr,
-                            ld_hat);
+                            Vhat != nullptr ? static_cast<uint16_t*>(Vhat) + t0 * ld_hat : nullptr, ld_hat);
     if (rc) return rc;
   }
   return AQUAKV_OK;
@@ -923,27 +899,17 @@ int aquakv_decode(aquakv_ctx* c, int64_t n_tokens, const uint8_t* Kcodes, const 
                         const_cast<uint16_t*>(Kscales), const_cast<uint8_t*>(Vcodes),
                         const_cast<uint16_t*>(Vscales), Khat, Vhat, ld_hat, workspace);
   }
+  // no predictor (layer 0): the row kernels alone
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  float* P = has_pred ? reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + ws.p_off) : nullptr;
   const int cb = c->code_bytes, ng = c->n_groups;
-  const uint16_t* Kpv = static_cast<const uint16_t*>(Khat_prev);
-  const uint16_t* Vpv = static_cast<const uint16_t*>(Vhat_prev);
   uint16_t* Kh = static_cast<uint16_t*>(Khat);
   uint16_t* Vh = static_cast<uint16_t*>(Vhat);
   for (int64_t t0 = 0; t0 < n_tokens; t0 += ws.chunk) {
     const int rows = int(n_tokens - t0 < ws.chunk ? n_tokens - t0 : ws.chunk);
-    if (has_pred) {
-      rc = launch_predict(c, st, rows, Kpv + t0 * ld_prev, nullptr, ld_prev, 0, Wk, bk, P, d);
-      if (rc) return rc;
-    }
-    rc = launch_decode_rows(c, st, kRoleK, rows, Kcodes + t0 * cb, Kscales + t0 * ng, P, d,
+    rc = launch_decode_rows(c, st, kRoleK, rows, Kcodes + t0 * cb, Kscales + t0 * ng, nullptr, d,
                             Kh + t0 * ld_hat, ld_hat);
     if (rc) return rc;
-    if (has_pred) {
-      rc = launch_predict(c, st, rows, Vpv + t0 * ld_prev, Kh + t0 * ld_hat, ld_prev, ld_hat, Wv, bv, P, d);
-      if (rc) return rc;
-    }
-    rc = launch_decode_rows(c, st, kRoleV, rows, Vcodes + t0 * cb, Vscales + t0 * ng, P, d,
+    rc = launch_decode_rows(c, st, kRoleV, rows, Vcodes + t0 * cb, Vscales + t0 * ng, nullptr, d,
                             Vh + t0 * ld_hat, ld_hat);
     if (rc) return rc;
   }

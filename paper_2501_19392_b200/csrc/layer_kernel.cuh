@@ -69,13 +69,16 @@ struct LayerRowSmem {
 };
 
 // The GEMM epilogue stages each 32-row x 32-column fp32 piece of a tile in shared memory (128-byte
-// swizzle) and hands it to a TMA store: two 4 KB buffers per epilogue warp.
+// swizzle) and hands it to a TMA store: two 4 KB buffers per epilogue warp, or one for the encoder
+// with the 256-point grid, whose 2 KB grid would otherwise not fit (its row work is so much longer
+// than its GEMM that the epilogue's overlap does not matter).
 constexpr int kEpiPieceBytes = 32 * 32 * 4;
-constexpr int kEpiBytes = 4 * 2 * kEpiPieceBytes;
+template <bool kEncode, int NPTS> constexpr int kEpiBufs = (kEncode && NPTS > 64) ? 1 : 2;
+template <bool kEncode, int NPTS> constexpr int kEpiBytes = 4 * kEpiBufs<kEncode, NPTS> * kEpiPieceBytes;
 
 template <bool kEncode, int D, int NPTS>
 constexpr size_t layer_smem_bytes() {
-  return 1024 + size_t(kLayerStages) * kPairStageBytes + kEpiBytes + sizeof(LayerSmemTail) + 16 +
+  return 1024 + size_t(kLayerStages) * kPairStageBytes + kEpiBytes<kEncode, NPTS> + sizeof(LayerSmemTail) + 16 +
          sizeof(LayerRowSmem<kEncode, D, NPTS>);
 }
 
@@ -87,6 +90,7 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void*
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -213,7 +217,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~uintptr_t(1023));
   uint8_t* epi_smem = smem + size_t(kLayerStages) * kPairStageBytes;      // 1024-byte aligned
-  LayerSmemTail* tail = reinterpret_cast<LayerSmemTail*>(epi_smem + kEpiBytes);
+  LayerSmemTail* tail = reinterpret_cast<LayerSmemTail*>(epi_smem + kEpiBytes<kEncode, NPTS>);
   LayerRowSmem<kEncode, D, NPTS>* rsm = reinterpret_cast<LayerRowSmem<kEncode, D, NPTS>*>(
       (reinterpret_cast<uintptr_t>(tail) + sizeof(LayerSmemTail) + 15) & ~uintptr_t(15));
 
@@ -395,7 +399,8 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         // ring row of this warp's 32 tokens; rows past the last token are written too (never read)
         const int ring_row = (j % a.nb) * a.mw * kBM + ml * kBM + quarter * 32;
         const float* bias = ph == 0 ? a.bk : a.bv;
-        uint8_t* my_epi = epi_smem + (warp - 2) * 2 * kEpiPieceBytes;
+        constexpr int EB = kEpiBufs<kEncode, NPTS>;
+        uint8_t* my_epi = epi_smem + (warp - 2) * EB * kEpiPieceBytes;
 #pragma unroll 1
         for (int c = 0; c < kBN / 32; ++c) {
           float v[32];
@@ -405,9 +410,11 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = __fadd_rn(v[i], __ldg(b + i));
           }
-          uint8_t* buf = my_epi + (c & 1) * kEpiPieceBytes;
-          if (c >= 2) {                  // the store that last read this buffer must be done with it
-            if (lane == 0) bulk_wait_read_1();
+          uint8_t* buf = my_epi + (c & (EB - 1)) * kEpiPieceBytes;
+          if (c >= EB) {                 // the store that last read this buffer must be done with it
+            if (lane == 0) {
+              if constexpr (EB == 2) bulk_wait_read_1(); else bulk_wait_read_0();
+            }
             __syncwarp();
           }
           // lane = row of the piece; 16-byte chunk q of row r sits at chunk position q ^ (r % 8)

@@ -188,11 +188,11 @@ def test_full_size_layer_on_sampled_rows(T, n):
     (256, 64, 256, 256, 16, synth.BF16, 131),     # one 256-wide feature tile per token block, one-warp teams
     (512, 64, 64, 64, 16, synth.F16, 1),          # a single token
     (512, 64, 128, 256, 64, synth.BF16, 259),     # Hadamard block < scale group < row, four candidates per cell
-    (1024, 128, 1024, 1024, 256, synth.BF16, 200),  # 256-point grid: encode takes the separate-kernel path
+    (1024, 128, 1024, 1024, 256, synth.BF16, 200),  # 256-point grid: second-level search lists, single-buffered GEMM epilogue
     (1024, 128, 512, 1024, 16, synth.F16, 385),   # Hadamard block = one warp's half row, group = whole row
 ])
 def test_fused_layer_shapes_strides_and_bias(d, hd, h, g, n, dtype, T):
-    """The fused layer kernel (and its separate-kernel fallback) on the other supported shapes, with
+    """The fused layer kernel on the other supported shapes, with
     predictor biases and row strides larger than d_kv, against the oracle (teacher-forced)."""
     from paper_2501_19392_b200 import api
     shape = dataclasses.replace(synth.CONFIGS[2], n_kv_heads=d // hd, head_dim=hd, n_tokens=T, n_layers=2,
