@@ -332,6 +332,7 @@ constexpr int kKhatRing = 3;        // waves of reconstructed keys kept when the
 struct LayerWs {
   size_t p_off, khat_off, flags_off, flags_bytes, total;
   int mw, n_waves, n_mblocks;
+  int grid_mw;     // token-block slots the launched grid covers (>= mw)
 };
 
 LayerWs layer_ws(const aquakv_ctx* c, int64_t T) {
@@ -340,6 +341,10 @@ LayerWs layer_ws(const aquakv_ctx* c, int64_t T) {
   w.n_mblocks = int((T + kBM - 1) / kBM);
   int mw = (c->sm_count / ntn) & ~1;          // CTAs work in pairs on two token blocks
   if (mw < 2) mw = 2;
+  // A call with fewer token blocks than a wave keeps its buffers small (mw shrinks) but still
+  // launches the whole grid: the CTAs without a GEMM tile take their share of the row work, which is
+  // what the latency of a small call consists of.
+  w.grid_mw = mw;
   if (mw > w.n_mblocks) mw = (w.n_mblocks + 1) & ~1;
   w.mw = mw;
   w.n_waves = (w.n_mblocks + mw - 1) / mw;
@@ -496,7 +501,7 @@ int launch_layer(aquakv_ctx* c, cudaStream_t st, bool encode, int64_t T, const v
   if ((rc = make_tmap(c, &tm[4], Wv, uint64_t(d), uint64_t(2) * d, uint64_t(2) * d, kBN / 2))) return rc;
 
   if (cudaMemsetAsync(a.gemm_done, 0, ws.flags_bytes, st) != cudaSuccess) return AQUAKV_ERR_CUDA;
-  const int grid = ws.mw * (d / kBN);
+  const int grid = ws.grid_mw * (d / kBN);
   ProfScope prof(c, st, AQUAKV_KERNEL_LAYER);
   if (encode) {
     AQ_DISPATCH_DNB(launch_layer_enc_t, &rc, c->device, st, grid, tm, a);
