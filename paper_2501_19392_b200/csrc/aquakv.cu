@@ -4,9 +4,10 @@
 // layer_kernel.cuh, gemm_pred.cuh, codec.cuh and attn.cuh; nothing is computed on the host and
 // there is no fallback path.
 //
-// Large calls are cut into token chunks sized so that one chunk's fp32 prediction (and, for the
-// fused attention, its decoded keys/values) stays resident in the 126 MB L2 between the kernel
-// that writes it and the kernel that reads it.
+// The single-phase entry points cut large calls into token chunks sized so that one chunk's fp32
+// prediction stays resident in the 126 MB L2 between the GEMM that writes it and the row kernel
+// that reads it; the fused attention entry point works on chunks of about 32 waves of the layer
+// kernel.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -362,8 +363,11 @@ struct AttnWs {
   int n_splits;
 };
 
-// The decode of a long cache runs chunk by chunk (about eight waves of the fused kernel) so that
-// the attention kernel finds most of a chunk's freshly decoded keys/values still in L2.
+// The decode of a long cache runs chunk by chunk, about 32 waves of the fused kernel each: long
+// enough that the kernel's fill and drain cost little (eight-wave chunks measured 9 % slower; the
+// attention kernel read the decoded rows from DRAM either way), short enough to bound the
+// workspace that holds a chunk's decoded keys/values when the caller does not ask for them
+// (0.6 GB at d_kv = 1024).
 AttnWs attn_ws(const aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_heads,
                int32_t head_dim) {
   AttnWs w;
@@ -371,7 +375,7 @@ AttnWs attn_ws(const aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_
   const size_t d = size_t(c->p.d_kv);
   w.n_splits = int((ctx_len + tb - 1) / tb);
   const int wave_tokens = (c->sm_count / int(d / kBN) > 0 ? c->sm_count / int(d / kBN) : 1) * kBM;
-  int cb = 8 * wave_tokens / tb;
+  int cb = 32 * wave_tokens / tb;
   if (cb < 1) cb = 1;
   const int64_t total_blocks = int64_t(batch) * w.n_splits;
   if (cb > total_blocks) cb = int(total_blocks);
