@@ -849,7 +849,6 @@ int aquakv_encode(aquakv_ctx* c, int64_t n_tokens, const void* K, const void* V,
   if ((Khat != nullptr && (Khat == Khat_prev || Khat == K || Khat == Vhat_prev)) ||
       (Vhat != nullptr && (Vhat == Vhat_prev || Vhat == V || Vhat == Khat_prev || Vhat == Khat)))
     return AQUAKV_ERR_INVALID_ARG;
-  const EncodeWs ws = encode_ws(c, n_tokens);
   if (has_pred) {
     if (workspace == nullptr || workspace_bytes < aquakv_workspace_bytes(c, n_tokens, AQUAKV_OP_ENCODE))
       return AQUAKV_ERR_WORKSPACE;
@@ -861,13 +860,15 @@ int aquakv_encode(aquakv_ctx* c, int64_t n_tokens, const void* K, const void* V,
                         Vhat_prev, ld_prev, Wk, Wv, bk, bv, Kcodes, Kscales, Vcodes, Vscales, Khat, Vhat,
                         ld_hat, workspace);
   }
-  // no predictor (layer 0): the row kernels alone
+  // no predictor (layer 0): the row kernels alone, in launches of up to 2^30 rows (no prediction
+  // buffer bounds them)
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int cb = c->code_bytes, ng = c->n_groups;
   const uint16_t* Kp = static_cast<const uint16_t*>(K);
   const uint16_t* Vp = static_cast<const uint16_t*>(V);
-  for (int64_t t0 = 0; t0 < n_tokens; t0 += ws.chunk) {
-    const int rows = int(n_tokens - t0 < ws.chunk ? n_tokens - t0 : ws.chunk);
+  const int64_t chunk = int64_t(1) << 30;
+  for (int64_t t0 = 0; t0 < n_tokens; t0 += chunk) {
+    const int rows = int(n_tokens - t0 < chunk ? n_tokens - t0 : chunk);
     rc = launch_encode_rows(c, st, kRoleK, rows, Kp + t0 * ld_kv, ld_kv, nullptr, d, Kcodes + t0 * cb,
                             Kscales + t0 * ng,
                             Khat != nullptr ? static_cast<uint16_t*>(Khat) + t0 * ld_hat : nullptr, ld_hat);
@@ -897,7 +898,6 @@ int aquakv_decode(aquakv_ctx* c, int64_t n_tokens, const uint8_t* Kcodes, const 
   if ((rc = check_adapters(Khat_prev, Vhat_prev, ld_prev, Wk, Wv, bk, bv, d, &has_pred))) return rc;
   if (Khat == Khat_prev || Khat == Vhat_prev || Vhat == Vhat_prev || Vhat == Khat_prev || Vhat == Khat)
     return AQUAKV_ERR_INVALID_ARG;
-  const EncodeWs ws = encode_ws(c, n_tokens);
   if (has_pred) {
     if (workspace == nullptr || workspace_bytes < aquakv_workspace_bytes(c, n_tokens, AQUAKV_OP_DECODE))
       return AQUAKV_ERR_WORKSPACE;
@@ -908,13 +908,14 @@ int aquakv_decode(aquakv_ctx* c, int64_t n_tokens, const uint8_t* Kcodes, const 
                         const_cast<uint16_t*>(Kscales), const_cast<uint8_t*>(Vcodes),
                         const_cast<uint16_t*>(Vscales), Khat, Vhat, ld_hat, workspace);
   }
-  // no predictor (layer 0): the row kernels alone
+  // no predictor (layer 0): the row kernels alone, in launches of up to 2^30 rows
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int cb = c->code_bytes, ng = c->n_groups;
   uint16_t* Kh = static_cast<uint16_t*>(Khat);
   uint16_t* Vh = static_cast<uint16_t*>(Vhat);
-  for (int64_t t0 = 0; t0 < n_tokens; t0 += ws.chunk) {
-    const int rows = int(n_tokens - t0 < ws.chunk ? n_tokens - t0 : ws.chunk);
+  const int64_t chunk = int64_t(1) << 30;
+  for (int64_t t0 = 0; t0 < n_tokens; t0 += chunk) {
+    const int rows = int(n_tokens - t0 < chunk ? n_tokens - t0 : chunk);
     rc = launch_decode_rows(c, st, kRoleK, rows, Kcodes + t0 * cb, Kscales + t0 * ng, nullptr, d,
                             Kh + t0 * ld_hat, ld_hat);
     if (rc) return rc;
