@@ -125,6 +125,9 @@ size_t aquakv_workspace_bytes(const aquakv_ctx* ctx, int64_t n_tokens, int op);
 /*
  * Workspace of aquakv_decode_attn for this problem shape (its split-KV partials depend on the
  * batch and head counts, which aquakv_workspace_bytes does not see).  0 on invalid arguments.
+ * The cache is decoded in chunks of up to about 147 K tokens; the workspace holds one chunk's
+ * decoded keys and values (4 * d_kv bytes per token: about 0.6 GB at d_kv = 1024 for long caches,
+ * whether or not Khat/Vhat are passed) besides the fused kernel's buffers.
  */
 size_t aquakv_decode_attn_workspace_bytes(const aquakv_ctx* ctx, int32_t batch, int64_t ctx_len,
                                           int32_t n_q_heads, int32_t head_dim);
