@@ -135,11 +135,13 @@ def _sample_rows(T, seed):
     return np.array(rows, dtype=np.int64)
 
 
-@pytest.mark.parametrize("T,n", [(32768, 16), (9549, 16), (4737, 64)])
+@pytest.mark.parametrize("T,n", [(32768, 16), (9549, 16), (4737, 64), (2500, 16), (2500, 256)])
 def test_full_size_layer_on_sampled_rows(T, n):
     """One layer of the benchmark's launch configuration (all tokens in one call: several waves of
     token blocks through the fused layer kernel, ragged last block) against the oracle on sampled
-    rows; rows are independent, so the oracle's result for a row does not depend on the others."""
+    rows; rows are independent, so the oracle's result for a row does not depend on the others.
+    2500 tokens are less than one wave: most CTAs of the grid have no GEMM tile and only share the
+    row work; with 256 grid points the search goes through the second-level lists."""
     shape, kv, ad = chain(2, T, 2, grid_size=n)
     d, dtype, bits = shape.d_kv, shape.dtype, shape.code_bits
     codec, ora = make(d, shape.had_block, shape.scale_group, n, dtype)
