@@ -568,7 +568,7 @@ __device__ __forceinline__ void encode_row(const RowCtx& rc, const RowSmem<NPTS>
   float4 pq[CPM][2];
 #pragma unroll
   for (int c = 0; c < CPM; ++c) {
-    raw[c] = *reinterpret_cast<const uint4*>(x_row + (c0 + c) * 256 + rc.lane * 8);
+    raw[c] = __ldcs(reinterpret_cast<const uint4*>(x_row + (c0 + c) * 256 + rc.lane * 8));   // read once
     if (pred_row != nullptr) {
       pq[c][0] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + rc.lane * 8));
       pq[c][1] = __ldcg(reinterpret_cast<const float4*>(pred_row + (c0 + c) * 256 + rc.lane * 8 + 4));

@@ -88,6 +88,13 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void*
                "r"(smem_u32(smem_src)), "r"(x), "r"(y)
                : "memory");
 }
+__device__ __forceinline__ void tma_store_2d_hint(const CUtensorMap* map, const void* smem_src, int32_t x, int32_t y,
+                                                  uint64_t policy) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;" ::"l"(
+                   reinterpret_cast<uint64_t>(map)),
+               "r"(smem_u32(smem_src)), "r"(x), "r"(y), "l"(policy)
+               : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
@@ -270,6 +277,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       tma_prefetch_desc(&tmWk);
       tma_prefetch_desc(&tmWv);
       tma_prefetch_desc(&tmP);
+      const uint64_t pol_stream = l2_policy_evict_first(), pol_keep = l2_policy_evict_last();
       int stage = 0;
       uint32_t phase_bit = 0;
       bool ok = true;
@@ -301,16 +309,17 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
           // the leader's barrier collects the bytes of both CTAs
           if (rank == 0) mbar_arrive_expect_tx(&tail->full[stage], 2 * kPairStageBytes);
           const int w_row = n_blk * kBN + int(rank) * (kBN / 2);     // this CTA's half of the weight rows
+          // token rows stream through L2 once; the adapter tiles are read again by every wave
           if (ph == 0) {
-            tma_load_2d_pair(a_dst, &tmKprev, &tail->full[stage], kb * kBK, m * kBM);
-            tma_load_2d_pair(b_dst, &tmWk, &tail->full[stage], kb * kBK, w_row);
+            tma_load_2d_pair_hint(a_dst, &tmKprev, &tail->full[stage], kb * kBK, m * kBM, pol_stream);
+            tma_load_2d_pair_hint(b_dst, &tmWk, &tail->full[stage], kb * kBK, w_row, pol_keep);
           } else {
             if (kb < NKD) {
-              tma_load_2d_pair(a_dst, &tmVprev, &tail->full[stage], kb * kBK, m * kBM);
+              tma_load_2d_pair_hint(a_dst, &tmVprev, &tail->full[stage], kb * kBK, m * kBM, pol_stream);
             } else {
-              tma_load_2d_pair(a_dst, &tmKhat, &tail->full[stage], (kb - NKD) * kBK, khat_row);
+              tma_load_2d_pair_hint(a_dst, &tmKhat, &tail->full[stage], (kb - NKD) * kBK, khat_row, pol_stream);
             }
-            tma_load_2d_pair(b_dst, &tmWv, &tail->full[stage], kb * kBK, w_row);
+            tma_load_2d_pair_hint(b_dst, &tmWv, &tail->full[stage], kb * kBK, w_row, pol_keep);
           }
           ++issued;
           if (++stage == kLayerStages) { stage = 0; phase_bit ^= 1u; }
@@ -400,6 +409,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         const int ring_row = (j % a.nb) * a.mw * kBM + ml * kBM + quarter * 32;
         const float* bias = ph == 0 ? a.bk : a.bv;
         constexpr int EB = kEpiBufs<kEncode, NPTS>;
+        const uint64_t pol_keep = l2_policy_evict_last();
         uint8_t* my_epi = epi_smem + (warp - 2) * EB * kEpiPieceBytes;
 #pragma unroll 1
         for (int c = 0; c < kBN / 32; ++c) {
@@ -425,7 +435,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
           fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) {
-            tma_store_2d(&tmP, buf, n_blk * kBN + c * 32, ring_row);
+            tma_store_2d_hint(&tmP, buf, n_blk * kBN + c * 32, ring_row, pol_keep);   // read back soon by the row warps
             bulk_commit();
           }
         }
@@ -514,6 +524,14 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
           } else {
             decode_row<D, NPTS, kBf16>(rck, rsm->tables.grid, ts, codes_row, scales_row,
                                        pred_row, hat_row);
+          }
+          // The row's prediction has been read for the last time: drop its lines from L2 without
+          // writing them back (the ring is scratch; only whole, 128-byte aligned lines are dropped).
+          if (hat_row != nullptr || !kEncode) {
+            __syncwarp();
+            const float* mine = pred_row + rck.member * 256 + lane * 8;
+            if ((lane & 3) == 0 && (reinterpret_cast<uintptr_t>(mine) & 127) == 0)
+              asm volatile("discard.global.L2 [%0], 128;" ::"l"(mine) : "memory");
           }
         }
       }
