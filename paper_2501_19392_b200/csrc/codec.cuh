@@ -550,7 +550,9 @@ __device__ __forceinline__ void encode_row_core(const RowCtx& rc, const RowSmem<
     o[1] = store16x2p<kBf16>(add2(pack2(pq[0].z, pq[0].w), vp[1]));
     o[2] = store16x2p<kBf16>(add2(pack2(pq[1].x, pq[1].y), vp[2]));
     o[3] = store16x2p<kBf16>(add2(pack2(pq[1].z, pq[1].w), vp[3]));
-    *reinterpret_cast<uint4*>(hat_row + cg * 256 + lane * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+    // streaming store: the reconstruction is read at most once more (by the value-phase GEMM) before it
+    // leaves L2
+    __stcs(reinterpret_cast<uint4*>(hat_row + cg * 256 + lane * 8), make_uint4(o[0], o[1], o[2], o[3]));
   }
 }
 
@@ -635,7 +637,7 @@ __device__ __forceinline__ void decode_row_core(const RowCtx& rc, const f32x2_t*
   o[1] = store16x2p<kBf16>(add2(pack2(pq[0][0].z, pq[0][0].w), wp[1]));
   o[2] = store16x2p<kBf16>(add2(pack2(pq[0][1].x, pq[0][1].y), wp[2]));
   o[3] = store16x2p<kBf16>(add2(pack2(pq[0][1].z, pq[0][1].w), wp[3]));
-  *reinterpret_cast<uint4*>(hat_row + rc.member * 256 + rc.lane * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+  __stcs(reinterpret_cast<uint4*>(hat_row + rc.member * 256 + rc.lane * 8), make_uint4(o[0], o[1], o[2], o[3]));
 }
 
 // This lane's codes and scales of one row (the small inputs of decode_row_core).
