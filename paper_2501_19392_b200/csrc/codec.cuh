@@ -598,7 +598,7 @@ __device__ __forceinline__ RowCtx make_row_ctx(const CodecArgs& a, int team_size
 }
 
 template <int D, int NPTS, bool kBf16>
-__global__ void __launch_bounds__(kCodecThreads, 2) encode_rows_kernel(const CodecArgs a) {
+__global__ void __launch_bounds__(kCodecThreads, 4) encode_rows_kernel(const CodecArgs a) {
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
   constexpr int CODE_BYTES = D / 2 * BITS / 8;
   constexpr int TEAM = RowTeam<D>::TEAM, TEAMS = kCodecWarps / TEAM;
@@ -688,7 +688,7 @@ __device__ __forceinline__ void decode_row(const RowCtx& rc, const f32x2_t* __re
 }
 
 template <int D, int NPTS, bool kBf16>
-__global__ void __launch_bounds__(kCodecThreads, 2) decode_rows_kernel(const CodecArgs a) {
+__global__ void __launch_bounds__(kCodecThreads, 4) decode_rows_kernel(const CodecArgs a) {
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
   constexpr int CODE_BYTES = D / 2 * BITS / 8;
   constexpr int TEAM = RowTeam<D>::TEAM, TEAMS = kCodecWarps / TEAM;
