@@ -58,7 +58,8 @@ def workload(args):
 
 
 def algorithmic_bytes(shape, n_rows_per_call):
-    """Bytes the method itself must move per token-layer (SURVEY 8d style accounting)."""
+    """Bytes the method itself must move per token-layer: inputs, outputs, codes, scales and the
+    adapters once per call; re-reads and the fp32 prediction scratch are implementation traffic."""
     d, g = shape.d_kv, shape.scale_group
     codes = 2 * (d // 2 * shape.code_bits // 8) + 2 * 2 * (d // g)
     weights = 6 * d * d / n_rows_per_call
