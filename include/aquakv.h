@@ -29,6 +29,8 @@
  *                   = even pair; n = 64: four codes per three bytes; n = 256: one byte each);
  *       scales[t] : d_kv/scale_group IEEE fp16 bit patterns, the group's root-mean-square
  *                   residual rounded to nearest even.
+ *     Code arrays are 16-byte aligned (a token's codes are a multiple of 16 bytes, and the kernels
+ *     move them as 16-byte vectors), scale arrays 2-byte aligned; AQUAKV_ERR_ALIGNMENT otherwise.
  *     Bits per value = log2(n)/2 + 16/scale_group (2.02 at n = 16, group 1024).
  *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
  *     legacy default stream).  They never synchronise, print, abort or throw.  Every function

@@ -86,6 +86,12 @@ inline int ilog2(int v) {
 inline bool is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t round_up(size_t v, size_t m) { return (v + m - 1) / m * m; }
+// The kernels want their scratch on 128-byte lines (32-byte vector loads, whole-line L2 discards); the
+// caller's workspace need only be 16-byte aligned, so every workspace size includes this slack.
+constexpr size_t kWsSlack = 128;
+inline uint8_t* ws_base(void* workspace) {
+  return reinterpret_cast<uint8_t*>(round_up(reinterpret_cast<uintptr_t>(workspace), kWsSlack));
+}
 
 int check_params(const aquakv_params* p) {
   if (p == nullptr) return AQUAKV_ERR_INVALID_ARG;
@@ -157,13 +163,28 @@ int launch_predict(aquakv_ctx* c, cudaStream_t st, int M, const void* in0, const
   return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
 }
 
+// d_kv = 1024 with the Hadamard block and the scale group spanning the row: one warp per row.
+inline bool warp_rows(const CodecArgs& a, int d) { return d == 1024 && a.log_h == 10 && a.log_g == 10; }
+
 template <int D, int NPTS, bool BF>
 void launch_encode_rows_t(aquakv_ctx*, cudaStream_t st, const CodecArgs& a, int grid) {
+  if constexpr (D == 1024) {
+    if (warp_rows(a, D)) {
+      encode_rows_warp_kernel<NPTS, BF><<<grid, kWrKernelWarps * 32, 0, st>>>(a);
+      return;
+    }
+  }
   encode_rows_kernel<D, NPTS, BF><<<grid, kCodecThreads, 0, st>>>(a);
 }
 
 template <int D, int NPTS, bool BF>
 void launch_decode_rows_t(aquakv_ctx*, cudaStream_t st, const CodecArgs& a, int grid) {
+  if constexpr (D == 1024) {
+    if (warp_rows(a, D)) {
+      decode_rows_warp_kernel<NPTS, BF><<<grid, kWrKernelWarps * 32, 0, st>>>(a);
+      return;
+    }
+  }
   decode_rows_kernel<D, NPTS, BF><<<grid, kCodecThreads, 0, st>>>(a);
 }
 
@@ -192,7 +213,8 @@ void launch_decode_rows_t(aquakv_ctx*, cudaStream_t st, const CodecArgs& a, int 
   } while (0)
 
 int codec_grid(const aquakv_ctx* c, int rows) {
-  const int rows_per_block = kCodecWarps / (c->p.d_kv / 256);   // one warp per 256-element chunk
+  const bool wr = c->p.d_kv == 1024 && c->log_h == 10 && c->log_g == 10;   // one warp per row, four per CTA
+  const int rows_per_block = wr ? kWrKernelWarps : kCodecWarps / (c->p.d_kv / 256);   // else one warp per 256-element chunk
   const int blocks = (rows + rows_per_block - 1) / rows_per_block;
   const int cap = c->sm_count * 8;
   return blocks < cap ? blocks : cap;
@@ -309,6 +331,17 @@ int check_rows(const void* p, int64_t ld, int d, bool required) {
   return AQUAKV_OK;
 }
 
+// Packed codes are read and written as 16-byte vectors (every token's codes are a multiple of 16
+// bytes), scales as 16-bit words.
+int check_cache(const void* Kcodes, const void* Kscales, const void* Vcodes, const void* Vscales) {
+  if (Kcodes == nullptr || Kscales == nullptr || Vcodes == nullptr || Vscales == nullptr)
+    return AQUAKV_ERR_INVALID_ARG;
+  if (!aligned16(Kcodes) || !aligned16(Vcodes)) return AQUAKV_ERR_ALIGNMENT;
+  if ((reinterpret_cast<uintptr_t>(Kscales) & 1u) || (reinterpret_cast<uintptr_t>(Vscales) & 1u))
+    return AQUAKV_ERR_ALIGNMENT;
+  return AQUAKV_OK;
+}
+
 struct EncodeWs {
   size_t p_off, khat_off, total;
   int chunk;
@@ -320,7 +353,7 @@ EncodeWs encode_ws(const aquakv_ctx* c, int64_t T) {
   w.chunk = int(t128 < c->chunk_tokens ? t128 : c->chunk_tokens);
   w.p_off = 0;
   w.khat_off = round_up(size_t(w.chunk) * c->p.d_kv * sizeof(float), 256);
-  w.total = w.khat_off + round_up(size_t(w.chunk) * c->p.d_kv * 2, 256);
+  w.total = w.khat_off + round_up(size_t(w.chunk) * c->p.d_kv * 2, 256) + kWsSlack;
   return w;
 }
 
@@ -353,7 +386,7 @@ LayerWs layer_ws(const aquakv_ctx* c, int64_t T) {
   w.khat_off = round_up(size_t(kLayerRing) * mw * kBM * d * sizeof(float), 256);
   w.flags_off = w.khat_off + round_up(size_t(kKhatRing) * mw * kBM * d * 2, 256);
   w.flags_bytes = size_t(2) * 2 * w.n_waves * mw * sizeof(int);
-  w.total = w.flags_off + round_up(w.flags_bytes, 256);
+  w.total = w.flags_off + round_up(w.flags_bytes, 256) + kWsSlack;
   return w;
 }
 
@@ -388,7 +421,7 @@ AttnWs attn_ws(const aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_
   w.vhat_off = w.khat_off + round_up(chunk_rows * d * 2, 256);
   w.ml_off = w.vhat_off + round_up(chunk_rows * d * 2, 256);
   w.o_off = w.ml_off + round_up(size_t(total_blocks) * n_q_heads * 2 * sizeof(float), 256);
-  w.total = w.o_off + round_up(size_t(total_blocks) * n_q_heads * head_dim * sizeof(float), 256);
+  w.total = w.o_off + round_up(size_t(total_blocks) * n_q_heads * head_dim * sizeof(float), 256) + kWsSlack;
   return w;
 }
 
@@ -397,7 +430,7 @@ int launch_layer_t(int device, cudaStream_t st, int grid, const CUtensorMap* tm,
   // the shared-memory opt-in is a per-device attribute of the function: one bit per device and
   // instantiation (setting it twice from two threads is harmless)
   static std::atomic<unsigned long long> attr_devices{0};
-  constexpr size_t smem = layer_smem_bytes<ENC, D, NPTS>();
+  constexpr size_t smem = layer_smem_bytes<ENC, D, NPTS, FULL>();
   const unsigned long long bit = 1ull << (device & 63);
   if (device >= 64 || !(attr_devices.load(std::memory_order_acquire) & bit)) {
     if (cudaFuncSetAttribute(layer_kernel<ENC, D, NPTS, BF, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -407,7 +440,7 @@ int launch_layer_t(int device, cudaStream_t st, int grid, const CUtensorMap* tm,
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(unsigned(grid));
-  cfg.blockDim = dim3(kLayerThreads);
+  cfg.blockDim = dim3(unsigned(LayerGeom<D, FULL>::THREADS));
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -432,6 +465,13 @@ void launch_layer_enc_t(int* rc, int device, cudaStream_t st, int grid, const CU
 }
 template <int D, int NPTS, bool BF>
 void launch_layer_dec_t(int* rc, int device, cudaStream_t st, int grid, const CUtensorMap* tm, const LayerArgs& a) {
+  // the decoder has the fixed-size instantiation only where it selects the one-warp-per-row routines
+  if constexpr (D == 1024) {
+    if (a.log_h == 10 && a.log_g == 10) {
+      *rc = launch_layer_t<false, D, NPTS, BF, true>(device, st, grid, tm, a);
+      return;
+    }
+  }
   *rc = launch_layer_t<false, D, NPTS, BF, false>(device, st, grid, tm, a);
 }
 
@@ -443,7 +483,7 @@ int launch_layer(aquakv_ctx* c, cudaStream_t st, bool encode, int64_t T, const v
                  int64_t ld_hat, void* workspace) {
   const int d = c->p.d_kv;
   const LayerWs ws = layer_ws(c, T);
-  uint8_t* wsb = static_cast<uint8_t*>(workspace);
+  uint8_t* wsb = ws_base(workspace);
   LayerArgs a;
   std::memset(&a, 0, sizeof(a));
   a.T = int(T);
@@ -750,7 +790,7 @@ int aquakv_encode_phase(aquakv_ctx* c, int role, int64_t n_tokens, const void* X
   int rc;
   if ((rc = check_rows(X, ld_x, d, true))) return rc;
   if ((rc = check_rows(hat, ld_hat, d, false))) return rc;
-  if (codes == nullptr || scales == nullptr) return AQUAKV_ERR_INVALID_ARG;
+  if ((rc = check_cache(codes, scales, codes, scales))) return rc;
   const bool has_pred = W != nullptr;
   if (has_pred) {
     if ((rc = check_rows(in0, ld_in, d, true))) return rc;
@@ -766,7 +806,7 @@ int aquakv_encode_phase(aquakv_ctx* c, int role, int64_t n_tokens, const void* X
     if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
   }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  float* P = has_pred ? reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + ws.p_off) : nullptr;
+  float* P = has_pred ? reinterpret_cast<float*>(ws_base(workspace) + ws.p_off) : nullptr;
   const int cb = c->code_bytes, ng = c->n_groups;
   const uint16_t* Xp = static_cast<const uint16_t*>(X);
   const uint16_t* a0 = static_cast<const uint16_t*>(in0);
@@ -795,7 +835,7 @@ int aquakv_decode_phase(aquakv_ctx* c, int role, int64_t n_tokens, const uint8_t
   const int d = c->p.d_kv;
   int rc;
   if ((rc = check_rows(hat, ld_hat, d, true))) return rc;
-  if (codes == nullptr || scales == nullptr) return AQUAKV_ERR_INVALID_ARG;
+  if ((rc = check_cache(codes, scales, codes, scales))) return rc;
   const bool has_pred = W != nullptr;
   if (has_pred) {
     if ((rc = check_rows(in0, ld_in, d, true))) return rc;
@@ -811,7 +851,7 @@ int aquakv_decode_phase(aquakv_ctx* c, int role, int64_t n_tokens, const uint8_t
     if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
   }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  float* P = has_pred ? reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + ws.p_off) : nullptr;
+  float* P = has_pred ? reinterpret_cast<float*>(ws_base(workspace) + ws.p_off) : nullptr;
   const int cb = c->code_bytes, ng = c->n_groups;
   const uint16_t* a0 = static_cast<const uint16_t*>(in0);
   const uint16_t* a1 = static_cast<const uint16_t*>(in1);
@@ -842,8 +882,7 @@ int aquakv_encode(aquakv_ctx* c, int64_t n_tokens, const void* K, const void* V,
   if ((rc = check_rows(V, ld_kv, d, true))) return rc;
   if ((rc = check_rows(Khat, ld_hat, d, false))) return rc;
   if ((rc = check_rows(Vhat, ld_hat, d, false))) return rc;
-  if (Kcodes == nullptr || Kscales == nullptr || Vcodes == nullptr || Vscales == nullptr)
-    return AQUAKV_ERR_INVALID_ARG;
+  if ((rc = check_cache(Kcodes, Kscales, Vcodes, Vscales))) return rc;
   bool has_pred = false;
   if ((rc = check_adapters(Khat_prev, Vhat_prev, ld_prev, Wk, Wv, bk, bv, d, &has_pred))) return rc;
   if ((Khat != nullptr && (Khat == Khat_prev || Khat == K || Khat == Vhat_prev)) ||
@@ -892,8 +931,7 @@ int aquakv_decode(aquakv_ctx* c, int64_t n_tokens, const uint8_t* Kcodes, const 
   int rc;
   if ((rc = check_rows(Khat, ld_hat, d, true))) return rc;
   if ((rc = check_rows(Vhat, ld_hat, d, true))) return rc;
-  if (Kcodes == nullptr || Kscales == nullptr || Vcodes == nullptr || Vscales == nullptr)
-    return AQUAKV_ERR_INVALID_ARG;
+  if ((rc = check_cache(Kcodes, Kscales, Vcodes, Vscales))) return rc;
   bool has_pred = false;
   if ((rc = check_adapters(Khat_prev, Vhat_prev, ld_prev, Wk, Wv, bk, bv, d, &has_pred))) return rc;
   if (Khat == Khat_prev || Khat == Vhat_prev || Vhat == Vhat_prev || Vhat == Khat_prev || Vhat == Khat)
@@ -971,8 +1009,7 @@ int aquakv_decode_noalloc(aquakv_ctx* c, int64_t n_tokens, const uint8_t* Kcodes
   int rc;
   if ((rc = check_rows(Khat, ld_hat, d, true))) return rc;
   if ((rc = check_rows(Vhat, ld_hat, d, true))) return rc;
-  if (Kcodes == nullptr || Kscales == nullptr || Vcodes == nullptr || Vscales == nullptr)
-    return AQUAKV_ERR_INVALID_ARG;
+  if ((rc = check_cache(Kcodes, Kscales, Vcodes, Vscales))) return rc;
   bool has_pred = false;
   if ((rc = check_adapters(Khat_prev, Vhat_prev, ld_prev, Wk, Wv, bk, bv, d, &has_pred))) return rc;
   if (Khat == Khat_prev || Khat == Vhat_prev || Vhat == Vhat_prev || Vhat == Khat_prev || Vhat == Khat)
@@ -1012,6 +1049,7 @@ int aquakv_decode_attn(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_
   if (!aligned16(q) || !aligned16(out)) return AQUAKV_ERR_ALIGNMENT;
   if (!(softmax_scale == softmax_scale)) return AQUAKV_ERR_INVALID_ARG;
   int rc;
+  if ((rc = check_cache(Kcodes, Kscales, Vcodes, Vscales))) return rc;
   if ((Khat == nullptr) != (Vhat == nullptr)) return AQUAKV_ERR_INVALID_ARG;
   if ((rc = check_rows(Khat, ld_hat, d, false))) return rc;
   if ((rc = check_rows(Vhat, ld_hat, d, false))) return rc;
@@ -1025,7 +1063,7 @@ int aquakv_decode_attn(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_
   if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  uint8_t* wsb = static_cast<uint8_t*>(workspace);
+  uint8_t* wsb = ws_base(workspace);
   float* part_ml = reinterpret_cast<float*>(wsb + ws.ml_off);
   float* part_o = reinterpret_cast<float*>(wsb + ws.o_off);
   const int cb = c->code_bytes, ng = c->n_groups, tb = c->attn_block_tokens;

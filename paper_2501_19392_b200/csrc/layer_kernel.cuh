@@ -35,15 +35,26 @@
 #include "codec.cuh"
 #include "common.cuh"
 #include "gemm_pred.cuh"
+#include "rowwarp.cuh"
 
 namespace aquakv {
 
-constexpr int kRowWarps = 24;
-constexpr int kLayerThreads = 32 * (6 + kRowWarps);
 constexpr int kLayerStages = 4;
 constexpr int kPairBBytes = (kBN / 2) * kBK * 2;        // this CTA's half of a weight tile k-block
 constexpr int kPairStageBytes = kABytes + kPairBBytes;   // 32 KB
-template <int D> constexpr int kRowTeamsOf = kRowWarps / RowTeam<D>::TEAM;
+
+// Row warps of a CTA.  With d_kv = 1024 and the Hadamard block and scale group spanning the whole row
+// (kFull) a single warp owns a row (rowwarp.cuh): 12 such warps at up to 112 registers; otherwise
+// teams of d_kv/256 warps share a row (codec.cuh): 24 warps at 64 registers.
+constexpr int kWrLayerWarps = 12;
+template <int D, bool kFull>
+struct LayerGeom {
+  static constexpr bool WR = D == 1024 && kFull;
+  static constexpr int ROW_WARPS = WR ? kWrLayerWarps : 24;
+  static constexpr int TEAM = WR ? 1 : RowTeam<D>::TEAM;
+  static constexpr int TEAMS = ROW_WARPS / TEAM;          // rows a CTA works on at a time
+  static constexpr int THREADS = 32 * (6 + ROW_WARPS);
+};
 
 struct LayerSmemTail {
   uint64_t full[kLayerStages];
@@ -62,10 +73,13 @@ struct GridSmem {
 template <bool kEncode, int NPTS> struct LayerTables { typedef RowSmem<NPTS> type; };
 template <int NPTS> struct LayerTables<false, NPTS> { typedef GridSmem<NPTS> type; };
 
-template <bool kEncode, int D, int NPTS>
+template <int D, bool WR> struct LayerRowScratch { TeamSmem<D> team[24 / RowTeam<D>::TEAM]; };
+template <int D> struct LayerRowScratch<D, true> { unsigned long long xbuf[kWrLayerWarps][kWrItems]; };
+
+template <bool kEncode, int D, int NPTS, bool kFull>
 struct LayerRowSmem {
   typename LayerTables<kEncode, NPTS>::type tables;
-  TeamSmem<D> team[kRowWarps / RowTeam<D>::TEAM];
+  LayerRowScratch<D, LayerGeom<D, kFull>::WR> scratch;
 };
 
 // The GEMM epilogue stages each 32-row x 32-column fp32 piece of a tile in shared memory (128-byte
@@ -76,10 +90,10 @@ constexpr int kEpiPieceBytes = 32 * 32 * 4;
 template <bool kEncode, int NPTS> constexpr int kEpiBufs = (kEncode && NPTS > 64) ? 1 : 2;
 template <bool kEncode, int NPTS> constexpr int kEpiBytes = 4 * kEpiBufs<kEncode, NPTS> * kEpiPieceBytes;
 
-template <bool kEncode, int D, int NPTS>
+template <bool kEncode, int D, int NPTS, bool kFull>
 constexpr size_t layer_smem_bytes() {
   return 1024 + size_t(kLayerStages) * kPairStageBytes + kEpiBytes<kEncode, NPTS> + sizeof(LayerSmemTail) + 16 +
-         sizeof(LayerRowSmem<kEncode, D, NPTS>);
+         sizeof(LayerRowSmem<kEncode, D, NPTS, kFull>);
 }
 
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* smem_src, int32_t x, int32_t y) {
@@ -211,11 +225,12 @@ __device__ __forceinline__ void fence_proxy_async_all() {
 // kFull: the Hadamard block and the scale group both span the whole row (the paper's setting for
 // d_kv = 1024, Section 4.1); their logarithms are then compile-time constants of the row code.
 template <bool kEncode, int D, int NPTS, bool kBf16, bool kFull>
-__global__ void __launch_bounds__(kLayerThreads, 1)
+__global__ void __launch_bounds__((LayerGeom<D, kFull>::THREADS), 1)
 layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant__ CUtensorMap tmVprev,
              const __grid_constant__ CUtensorMap tmKhat, const __grid_constant__ CUtensorMap tmWk,
              const __grid_constant__ CUtensorMap tmWv, const __grid_constant__ CUtensorMap tmP,
              const LayerArgs a) {
+  using G = LayerGeom<D, kFull>;
   constexpr int NTN = D / kBN;             // feature tiles per token block = CTAs per token block
   constexpr int NKD = D / kBK;             // k-blocks per d_kv input features
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
@@ -225,7 +240,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
                                              ~uintptr_t(1023));
   uint8_t* epi_smem = smem + size_t(kLayerStages) * kPairStageBytes;      // 1024-byte aligned
   LayerSmemTail* tail = reinterpret_cast<LayerSmemTail*>(epi_smem + kEpiBytes<kEncode, NPTS>);
-  LayerRowSmem<kEncode, D, NPTS>* rsm = reinterpret_cast<LayerRowSmem<kEncode, D, NPTS>*>(
+  LayerRowSmem<kEncode, D, NPTS, kFull>* rsm = reinterpret_cast<LayerRowSmem<kEncode, D, NPTS, kFull>*>(
       (reinterpret_cast<uintptr_t>(tail) + sizeof(LayerSmemTail) + 15) & ~uintptr_t(15));
 
   const int warp = threadIdx.x >> 5;
@@ -292,7 +307,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         for (int kb = 0; kb < nk; ++kb) {
           if (ph == 1 && kb == NKD && m < a.n_mblocks) {
             // the remaining k-blocks read this wave's reconstructed keys, written by row warps
-            const int target = wave_block_teams(wave_rows(wave, a.T, a.mw, gridDim.x), ml, gridDim.x, kRowTeamsOf<D>);
+            const int target = wave_block_teams(wave_rows(wave, a.T, a.mw, gridDim.x), ml, gridDim.x, G::TEAMS);
             if (!counter_wait_bounded(a.rows_done + layer_key_job(wave) * a.mw + ml, target, abort_flag,
                                       a.status)) {
               ok = false;
@@ -394,7 +409,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       if (j >= a.nb) {
         int ph_old, wave_old;
         layer_job(j - a.nb, a.n_waves, ph_old, wave_old);
-        const int target = wave_block_teams(wave_rows(wave_old, a.T, a.mw, gridDim.x), ml, gridDim.x, kRowTeamsOf<D>);
+        const int target = wave_block_teams(wave_rows(wave_old, a.T, a.mw, gridDim.x), ml, gridDim.x, G::TEAMS);
         // one thread polls for the four warps; a failed wait has set the abort flag
         if (warp == 2 && lane == 0)
           counter_wait_bounded(a.rows_done + (j - a.nb) * a.mw + ml, target, abort_flag, a.status);
@@ -458,24 +473,37 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       }
     }
   } else {
-    // ------------------------------- row warps (teams of TEAM warps per row) -------------------
-    constexpr int TEAM = RowTeam<D>::TEAM, TEAMS = kRowWarps / TEAM;
+    // ------------------------------- row warps (TEAM warps per row; TEAMS rows at a time) ------
+    constexpr int TEAM = G::TEAM, TEAMS = G::TEAMS;
     const int rw = warp - 6;
     const int team = rw / TEAM;
-    RowCtx rck;     // one context per warp; the sign bits are switched between key and value jobs
     constexpr int LOG_D = D == 1024 ? 10 : (D == 512 ? 9 : 8);
     const int log_h = kFull ? LOG_D : a.log_h, log_g = kFull ? LOG_D : a.log_g;
-    row_ctx_init(rck, a.signmask_k, a.search.inv_w, log_h, log_g, lane, rw % TEAM, RowTeam<D>::NV, 3 + team);
-    const uint32_t signs_k = a.signmask_k[lane] >> (rck.member * RowTeam<D>::NV);
-    const uint32_t signs_v = a.signmask_v[lane] >> (rck.member * RowTeam<D>::NV);
-    TeamSmem<D>* ts = &rsm->team[team];
+    // one context per warp; the sign bits are switched between key and value jobs
+    RowCtx rck;
+    WarpRowCtx wrc;
+    uint32_t signs_k, signs_v;
+    if constexpr (G::WR) {
+      wrc.lane = lane;
+      wrc.inv_w = a.search.inv_w;
+      wrc.signs = 0u;
+      signs_k = a.signmask_k[lane];
+      signs_v = a.signmask_v[lane];
+      rck.member = 0;
+      rck.barrier = 0;
+    } else {
+      row_ctx_init(rck, a.signmask_k, a.search.inv_w, log_h, log_g, lane, rw % TEAM, RowTeam<D>::NV, 3 + team);
+      signs_k = a.signmask_k[lane] >> (rck.member * RowTeam<D>::NV);
+      signs_v = a.signmask_v[lane] >> (rck.member * RowTeam<D>::NV);
+    }
     const int n_groups = D >> log_g;
     for (int j = 0; j < n_jobs; ++j) {
       int ph, wave;
       layer_job(j, a.n_waves, ph, wave);
       const WaveRows wr = wave_rows(wave, a.T, a.mw, gridDim.x);
       if (wr.tokens <= 0) continue;
-      row_ctx_set_signs(rck, ph == 0 ? signs_k : signs_v);
+      if constexpr (G::WR) wrc.signs = ph == 0 ? signs_k : signs_v;
+      else row_ctx_set_signs(rck, ph == 0 ? signs_k : signs_v);
       const int slot_row = (ml * NTN + n_blk) * wr.rpc;      // first row (within the wave) of this CTA's slice
       const int rb = slot_row / kBM;                         // token block (within the wave) the slice lies in
       if (rb >= wr.blocks) continue;                         // nothing assigned, nobody waits for this CTA
@@ -517,21 +545,38 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
           else hat_row = a.Vhat != nullptr ? a.Vhat + g * a.ldVhat : nullptr;
           uint8_t* codes_row = (ph == 0 ? a.Kcodes : a.Vcodes) + g * CODE_BYTES;
           uint16_t* scales_row = (ph == 0 ? a.Kscales : a.Vscales) + g * n_groups;
-          if constexpr (kEncode) {
-            const uint16_t* x_row = (ph == 0 ? a.K : a.V) + g * a.ldX;
-            encode_row<D, NPTS, kBf16>(rck, &rsm->tables, ts, x_row, pred_row, codes_row,
-                                       scales_row, hat_row);
+          if constexpr (G::WR) {
+            unsigned long long* xbuf = rsm->scratch.xbuf[rw];
+            if constexpr (kEncode) {
+              const uint16_t* x_row = (ph == 0 ? a.K : a.V) + g * a.ldX;
+              wr_encode_row<NPTS, kBf16>(wrc, &rsm->tables, xbuf, x_row, pred_row, codes_row, scales_row, hat_row);
+            } else {
+              wr_decode_row<NPTS, kBf16>(wrc, rsm->tables.grid, xbuf, codes_row, scales_row, pred_row, hat_row);
+            }
           } else {
-            decode_row<D, NPTS, kBf16>(rck, rsm->tables.grid, ts, codes_row, scales_row,
-                                       pred_row, hat_row);
+            TeamSmem<D>* ts = &rsm->scratch.team[team];
+            if constexpr (kEncode) {
+              const uint16_t* x_row = (ph == 0 ? a.K : a.V) + g * a.ldX;
+              encode_row<D, NPTS, kBf16>(rck, &rsm->tables, ts, x_row, pred_row, codes_row,
+                                         scales_row, hat_row);
+            } else {
+              decode_row<D, NPTS, kBf16>(rck, rsm->tables.grid, ts, codes_row, scales_row,
+                                         pred_row, hat_row);
+            }
           }
           // The row's prediction has been read for the last time: drop its lines from L2 without
           // writing them back (the ring is scratch; only whole, 128-byte aligned lines are dropped).
           if (hat_row != nullptr || !kEncode) {
             __syncwarp();
-            const float* mine = pred_row + rck.member * 256 + lane * 8;
-            if ((lane & 3) == 0 && (reinterpret_cast<uintptr_t>(mine) & 127) == 0)
-              asm volatile("discard.global.L2 [%0], 128;" ::"l"(mine) : "memory");
+            if constexpr (G::WR) {
+              const float* mine = pred_row + lane * 32;             // the row's 32 lines, one per lane
+              if ((reinterpret_cast<uintptr_t>(mine) & 127) == 0)
+                asm volatile("discard.global.L2 [%0], 128;" ::"l"(mine) : "memory");
+            } else {
+              const float* mine = pred_row + rck.member * 256 + lane * 8;
+              if ((lane & 3) == 0 && (reinterpret_cast<uintptr_t>(mine) & 127) == 0)
+                asm volatile("discard.global.L2 [%0], 128;" ::"l"(mine) : "memory");
+            }
           }
         }
       }
