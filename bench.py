@@ -8,7 +8,14 @@ Algorithm 4 for every layer).  The workload is the Llama-3.2-3B-shaped prefill c
 28 layers x 32768 tokens, 8 KV heads x 128 (d_kv = 1024), bf16, 2 bits per value (16-point 2-D
 grid, Hadamard block = scale group = 1024).
 
-Metric: KV tokens/s per layer = tokens x layers carried through the step / step time.
+Metric: KV tokens/s per layer = tokens x layers carried through the step / step time.  The
+headline `value` counts a token-layer once per round trip (encode + decode-attention); the per-op
+rates (encode, decode-attention, plain decode) are under `ops`.
+
+After the timed step the other four workload shapes are timed as well (one predicted-layer call
+each, inputs resident in HBM) and reported under `ops_by_config` with their fraction of the roofline
+max(6 d^2 T / tensor peak, algorithmic bytes / HBM bandwidth) against both the burst and the
+sustained measured tensor peak.
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample of the
 same workload instead (the reference arm).
@@ -168,9 +175,19 @@ def oracle_baseline(shape, n_q_heads, target_s=12.0):
     rows = rows // 64 * 64
     layers = 4
     t = oracle_sample_run(shape, rows, layers, n_q_heads, seed=2001)
-    return dict(value=rows * layers / t, unit=UNIT, cores=oracle.num_threads(), kind="oracle",
+    cores = oracle.num_threads()
+    # the same oracle on one thread, on a sample sized for a few seconds
+    rows1 = max(64, int(rows / max(1, cores) / 2) // 64 * 64)
+    oracle.set_num_threads(1)
+    try:
+        t1 = oracle_sample_run(shape, rows1, layers, n_q_heads, seed=2002)
+    finally:
+        oracle.set_num_threads(cores)
+    return dict(value=rows * layers / t, unit=UNIT, cores=cores, kind="oracle",
                 sample="%d tokens x %d layers of the workload (encode chain + decode chain + attention), %.1f s"
-                       % (rows, layers, t))
+                       % (rows, layers, t),
+                value_1thread=rows1 * layers / t1,
+                sample_1thread="%d tokens x %d layers, %.1f s" % (rows1, layers, t1))
 
 
 def run_reference(args):
@@ -202,19 +219,145 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------------
+# The other workload shapes (one predicted-layer call each)
+# ------------------------------------------------------------------------------------------------
+
+def _time_calls(fn, reps, warm=3):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def _shape_bytes(shape, tokens, encode, write_hat=True):
+    """Algorithmic bytes per token-layer of one predicted-layer call over `tokens` tokens."""
+    d = shape.d_kv
+    codes = 2 * shape.code_bytes + 2 * 2 * shape.n_groups
+    by = codes + 4 * d + 6.0 * d * d / tokens + (4 * d if write_hat else 0)   # codes, prev in, weights, hats out
+    return by + (4 * d if encode else 0)                                          # K, V in
+
+
+def _shape_entry(peaks, shape, op, tokens, ms, by_per_token, **extra):
+    d = shape.d_kv
+    t_hbm = by_per_token / (peaks["hbm_gbs"] * 1e9)
+    tps = tokens / (ms * 1e-3)
+    out = {"workload": shape.name, "op": op, "tokens_per_call": tokens, "d_kv": d, "grid_points": shape.grid_size,
+           "ms_per_layer_call": ms, "token_layers_per_s": tps}
+    for key, tf in (("burst", peaks["tf_burst"]), ("sustained", peaks["tf_sustained"])):
+        t_tensor = 6.0 * d * d / (tf * 1e12)
+        t_roof = max(t_tensor, t_hbm)
+        out["frac_of_roofline_" + key] = tps * t_roof
+        if key == "burst":
+            out["bound"] = "tensor" if t_tensor >= t_hbm else "hbm"
+            out["roofline_token_layers_per_s"] = 1.0 / t_roof
+    out.update(extra)
+    return out
+
+
+def _shape_codec(api, shape):
+    grid = synth.lloyd_grid(shape.grid_size, seed=7, n_samples=1 << 14, iters=25)
+    return api.Codec(shape.d_kv, shape.had_block, shape.scale_group, grid, shape.dtype,
+                     synth.hadamard_signs(shape.d_kv, 11), synth.hadamard_signs(shape.d_kv, 12))
+
+
+def ops_by_config(api, chain, peaks, dev, reps=5):
+    """Times configs 1, 3, 4 and 5 (config 2 is the timed step itself): per predicted-layer call, with
+    the previous layer's reconstruction already in the ping-pong buffers."""
+    out = []
+
+    def encode_case(cfg, shape, layers, want_decode):
+        shape = dataclasses.replace(shape, n_layers=layers)
+        T = shape.n_tokens
+        codec = _shape_codec(api, shape)
+        kv = synth.kv_chain(shape, seed=1000 * cfg + 1, device=dev)
+        ad = synth.random_adapters(shape, seed=1000 * cfg + 2, device=dev)
+        cache = chain.CompressedCache.empty(codec, layers, T, dev)
+        bufs = chain.PingPong(codec, T, dev)
+        chain.encode_chain(codec, kv.K, kv.V, ad, cache, bufs)
+        ms_chain = _time_calls(lambda: chain.encode_chain(codec, kv.K, kv.V, ad, cache, bufs), reps)
+        l = layers - 1
+        prv, cur = (l + 1) % 2, l % 2
+        one = lambda: codec.encode(kv.K[l], kv.V[l], bufs.K[prv], bufs.V[prv], ad.Wk[l], ad.Wv[l], None, None,
+                                   cache.Kcodes[l], cache.Kscales[l], cache.Vcodes[l], cache.Vscales[l],
+                                   bufs.K[cur], bufs.V[cur])
+        ms = _time_calls(one, reps * 4)
+        out.append(_shape_entry(peaks, shape, "encode", T, ms, _shape_bytes(shape, T, True),
+                                config=cfg, ms_chain=ms_chain, chain_layers=layers))
+        if want_decode:
+            chain.decode_chain(codec, cache, ad, bufs)
+            one = lambda: codec.decode(cache.Kcodes[l], cache.Kscales[l], cache.Vcodes[l], cache.Vscales[l],
+                                       bufs.K[prv], bufs.V[prv], ad.Wk[l], ad.Wv[l], None, None,
+                                       bufs.K[cur], bufs.V[cur])
+            ms = _time_calls(one, reps * 4)
+            out.append(_shape_entry(peaks, shape, "decode", T, ms, _shape_bytes(shape, T, False), config=cfg))
+        assert codec.poll_status() == 0
+
+    # config 1: two layers, encode + decode round trip
+    encode_case(1, synth.CONFIGS[1], 2, True)
+    # config 3: decode-step encode, 2 and 3 bits per value
+    for n in (16, 64):
+        encode_case(3, dataclasses.replace(synth.CONFIGS[3], grid_size=n), synth.CONFIGS[3].n_layers, False)
+    torch.cuda.empty_cache()
+    # config 4: bulk decode over a random packed cache, 8 of its 80 layers (every layer after the
+    # first costs the same; the metric is per layer)
+    shape = dataclasses.replace(synth.CONFIGS[4], n_layers=8)
+    codec = _shape_codec(api, shape)
+    rc = synth.random_cache(shape, seed=4003, device=dev)
+    cache = chain.CompressedCache(rc.Kcodes, rc.Kscales, rc.Vcodes, rc.Vscales)
+    ad = synth.random_adapters(shape, seed=4002, device=dev)
+    bufs = chain.PingPong(codec, shape.n_tokens, dev)
+    chain.decode_chain(codec, cache, ad, bufs)
+    ms_chain = _time_calls(lambda: chain.decode_chain(codec, cache, ad, bufs), max(2, reps // 2))
+    ms = (ms_chain - _time_calls(lambda: chain.decode_chain(codec, cache, ad, bufs, n_layers=1), reps)) / 7
+    out.append(_shape_entry(peaks, shape, "decode", shape.n_tokens, ms, _shape_bytes(shape, shape.n_tokens, False),
+                            config=4, ms_chain=ms_chain, chain_layers=8, layers_of_the_full_shape=80))
+    assert codec.poll_status() == 0
+    del cache, rc, bufs
+    torch.cuda.empty_cache()
+    # config 5: decode + single-query attention, batch 32 x context 32768, one layer call
+    shape = dataclasses.replace(synth.CONFIGS[5], n_layers=2)
+    T, d = shape.n_tokens, shape.d_kv
+    codec = _shape_codec(api, shape)
+    rc = synth.random_cache(shape, seed=5003, device=dev, n_layers=1)
+    ad = synth.random_adapters(shape, seed=5002, device=dev)
+    Kp = synth.random_16bit((T, d), shape.dtype, 5004, device=dev)
+    Vp = synth.random_16bit((T, d), shape.dtype, 5005, device=dev)
+    q = synth.random_16bit((shape.batch, shape.n_q_heads, shape.head_dim), shape.dtype, 5006, device=dev)
+    o = torch.empty_like(q)
+    ctx_len = T // shape.batch
+    one = lambda: codec.decode_attn(q, rc.Kcodes[0], rc.Kscales[0], rc.Vcodes[0], rc.Vscales[0], ctx_len,
+                                    shape.n_kv_heads, 1.0 / math.sqrt(shape.head_dim), Kp, Vp, ad.Wk[1], ad.Wv[1],
+                                    None, None, out=o)
+    ms = _time_calls(one, max(2, reps // 2), warm=2)
+    out.append(_shape_entry(peaks, shape, "decode_attn", T, ms, _shape_bytes(shape, T, False, write_hat=False),
+                            config=5, batch=shape.batch, ctx=ctx_len, n_q_heads=shape.n_q_heads))
+    assert codec.poll_status() == 0
+    del rc, Kp, Vp
+    torch.cuda.empty_cache()
+    return out
+
+
+# ------------------------------------------------------------------------------------------------
 # GPU arm
 # ------------------------------------------------------------------------------------------------
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--tokens", type=int, default=0, help="override tokens per GPU (testing only)")
     ap.add_argument("--layers", type=int, default=0, help="override layer count (testing only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true", help="skip the per-call timing of configs 1, 3, 4, 5")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -319,13 +462,15 @@ def main():
     flops_tl = 6.0 * d * d * (L - 1) / L                    # layer 0 has no predictor
     t_tensor = flops_tl / (peaks["tf_burst"] * 1e12)
     roof = {}
+    t_tensor_sus = flops_tl / (peaks["tf_sustained"] * 1e12)
     for name, ms, by in (("encode", enc_ms, enc_bytes), ("decode_attn", dec_ms, dec_bytes),
                          ("decode", plain_dec_ms, dec_bytes)):
         t_hbm = by / (peaks["hbm_gbs"] * 1e9)
         t_roof = max(t_tensor, t_hbm)
         tps = T * L / (ms * 1e-3)
         roof[name] = {"token_layers_per_s": tps, "ms": ms, "roofline_token_layers_per_s": 1.0 / t_roof,
-                      "frac_of_roofline": tps * t_roof, "bound": "tensor" if t_tensor >= t_hbm else "hbm",
+                      "frac_of_roofline": tps * t_roof, "frac_of_roofline_sustained": tps * max(t_tensor_sus, t_hbm),
+                      "bound": "tensor" if t_tensor >= t_hbm else "hbm",
                       "achieved_tflops": tps * flops_tl / 1e12, "achieved_gbs": tps * by / 1e9}
 
     gemm_flops_total = args.steps * 2 * (L - 1) * 6.0 * d * d * T      # encode + decode-attn chains
@@ -341,6 +486,7 @@ def main():
     achieved = gemm_flops_total / max(1e-9, ms_l * 1e-3) / 1e12
     roofline = {"kernel": "layer_kernel", "bound": "tensor", "achieved": achieved,
                 "peak": peaks["tf_sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["tf_sustained"],
+                "frac_burst": achieved / peaks["tf_burst"], "peak_burst": peaks["tf_burst"],
                 "traffic": LAYER_KERNEL_DRAM_BYTES_PER_LAUNCH if (T, d, shape.grid_size) == (32768, 1024, 16) else None,
                 "traffic_unit": "bytes per launch (ncu dram read+write, mean of the encode and decode launches)",
                 "algorithmic_bytes_per_launch": 0.5 * (enc_bytes + dec_bytes) * T,
@@ -363,6 +509,11 @@ def main():
         "ops": roof, "kernels": kernels, "roofline": roofline, "clocks": clocks, "gpu_launches": launches,
         "e2e": e2e,
     }
+    if world == 1 and not args.no_other_configs and not (args.tokens or args.layers):
+        del kv, cache, bufs, q, out
+        torch.cuda.empty_cache()
+        result["ops_by_config"] = ([dict(config=2, workload=shape.name, op=name, tokens_per_call=T, **v)
+                                    for name, v in roof.items()] + ops_by_config(api, chain, peaks, dev))
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = oracle_baseline(shape, n_q)
     if rank == 0:

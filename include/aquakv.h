@@ -267,6 +267,16 @@ int aquakv_decode_attn(aquakv_ctx* ctx, int32_t batch, int64_t ctx_len,
  */
 int aquakv_poll_status(aquakv_ctx* ctx, void* cuda_stream);
 
+/*
+ * Failure-path check of the device-side waits.  Every wait inside the kernels (on a TMA or
+ * tensor-core completion barrier, on another CTA's progress counter) gives up after a time limit,
+ * records AQUAKV_ERR_TIMEOUT in the context's status word and lets the kernel return.  This call
+ * launches one warp that waits, with a limit of limit_ns nanoseconds (0 < limit_ns <= 2e9), on a
+ * barrier that nothing arrives on, so the next aquakv_poll_status returns AQUAKV_ERR_TIMEOUT (and
+ * clears it) while the context stays usable.  Diagnostic only; not part of the paper's method.
+ */
+int aquakv_selftest_bounded_wait(aquakv_ctx* ctx, int64_t limit_ns, void* cuda_stream);
+
 /* Number of kernels this context has launched since creation (for benchmarks' bookkeeping). */
 int64_t aquakv_launch_count(const aquakv_ctx* ctx);
 

@@ -31,7 +31,7 @@ SYMBOLS = [
     "aquakv_code_bytes", "aquakv_search_table_host", "aquakv_create", "aquakv_destroy", "aquakv_workspace_bytes",
     "aquakv_decode_attn_workspace_bytes", "aquakv_predict", "aquakv_encode", "aquakv_decode",
     "aquakv_decode_attn", "aquakv_decode_noalloc", "aquakv_encode_phase", "aquakv_decode_phase", "aquakv_poll_status", "aquakv_launch_count", "aquakv_status_string",
-    "aquakv_profile_enable", "aquakv_profile_read",
+    "aquakv_profile_enable", "aquakv_profile_read", "aquakv_selftest_bounded_wait",
 ]
 
 
@@ -93,6 +93,8 @@ def _load():
     L.aquakv_profile_enable.argtypes = [vp, ctypes.c_int]
     L.aquakv_profile_read.restype = ctypes.c_int
     L.aquakv_profile_read.argtypes = [vp, ctypes.c_int, ctypes.POINTER(i64), ctypes.POINTER(ctypes.c_double)]
+    L.aquakv_selftest_bounded_wait.restype = ctypes.c_int
+    L.aquakv_selftest_bounded_wait.argtypes = [vp, i64, vp]
     L.aquakv_status_string.restype = ctypes.c_char_p
     L.aquakv_status_string.argtypes = [ctypes.c_int]
     return L
@@ -307,6 +309,11 @@ class Codec:
 
     def launch_count(self) -> int:
         return int(lib.aquakv_launch_count(self.h))
+
+    def selftest_bounded_wait(self, limit_ns: int) -> None:
+        rc = lib.aquakv_selftest_bounded_wait(self.h, int(limit_ns), _stream())
+        if rc:
+            raise AquaKVError(rc, "aquakv_selftest_bounded_wait")
 
     def profile_enable(self, enable: bool) -> None:
         rc = lib.aquakv_profile_enable(self.h, 1 if enable else 0)

@@ -440,7 +440,7 @@ int launch_layer_t(int device, cudaStream_t st, int grid, const CUtensorMap* tm,
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(unsigned(grid));
-  cfg.blockDim = dim3(unsigned(LayerGeom<D, FULL>::THREADS));
+  cfg.blockDim = dim3(unsigned(LayerGeom<ENC, D, FULL>::THREADS));
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -756,6 +756,14 @@ int aquakv_poll_status(aquakv_ctx* c, void* cuda_stream) {
     return AQUAKV_ERR_CUDA;
   if (h != 0 && cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess) return AQUAKV_ERR_CUDA;
   return h;
+}
+
+int aquakv_selftest_bounded_wait(aquakv_ctx* c, int64_t limit_ns, void* cuda_stream) {
+  if (c == nullptr || limit_ns <= 0 || limit_ns > int64_t(kWaitLimitNs)) return AQUAKV_ERR_INVALID_ARG;
+  bounded_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      c->d_status, static_cast<unsigned long long>(limit_ns));
+  ++c->launches;
+  return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
 }
 
 int aquakv_predict(aquakv_ctx* c, int64_t n_tokens, const void* in0, const void* in1, int64_t ld_in,

@@ -79,14 +79,15 @@ __device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t par
 // timeout in *status and raising *abort_flag in shared memory) if the wait exceeded
 // kWaitLimitNs or another role of this CTA already aborted.
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity,
-                                                  volatile int* abort_flag, int* status) {
+                                                  volatile int* abort_flag, int* status,
+                                                  unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_timer_ns();
   uint32_t spins = 0;
   while (!mbar_try_wait_parked(bar, parity, 2000u)) {
     if ((++spins & 0x3Fu) == 0) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
+      if (global_timer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         atomicExch(status, kStatusTimeout);
         return false;
@@ -94,6 +95,21 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     }
   }
   return true;
+}
+
+// One warp waits, with the given limit, on a barrier that nothing ever arrives on: the wait must give
+// up, record the timeout and return.  Used to check the failure path of the bounded waits without
+// disturbing any real kernel (the loop ends on %globaltimer alone).
+__global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(int* status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    mbar_fence_init();
+  }
+  __syncwarp();
+  if (threadIdx.x == 0) mbar_wait_bounded(&bar, 0u, &abort_flag, status, limit_ns);
 }
 
 // ---------------------------------------------------------------------------------------------

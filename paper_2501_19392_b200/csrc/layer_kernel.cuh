@@ -44,13 +44,14 @@ constexpr int kPairBBytes = (kBN / 2) * kBK * 2;        // this CTA's half of a 
 constexpr int kPairStageBytes = kABytes + kPairBBytes;   // 32 KB
 
 // Row warps of a CTA.  With d_kv = 1024 and the Hadamard block and scale group spanning the whole row
-// (kFull) a single warp owns a row (rowwarp.cuh): 12 such warps at up to 112 registers; otherwise
+// (kFull) a single warp owns a row (rowwarp.cuh): 12 such warps at 96 registers; otherwise
 // teams of d_kv/256 warps share a row (codec.cuh): 24 warps at 64 registers.
-constexpr int kWrLayerWarps = 12;
-template <int D, bool kFull>
+constexpr int kWrEncodeWarps = 12;    // the encoder's search table leaves shared memory for 12 transposition buffers
+constexpr int kWrDecodeWarps = 12;    // 12 to 16 measured alike
+template <bool kEncode, int D, bool kFull>
 struct LayerGeom {
   static constexpr bool WR = D == 1024 && kFull;
-  static constexpr int ROW_WARPS = WR ? kWrLayerWarps : 24;
+  static constexpr int ROW_WARPS = WR ? (kEncode ? kWrEncodeWarps : kWrDecodeWarps) : 24;
   static constexpr int TEAM = WR ? 1 : RowTeam<D>::TEAM;
   static constexpr int TEAMS = ROW_WARPS / TEAM;          // rows a CTA works on at a time
   static constexpr int THREADS = 32 * (6 + ROW_WARPS);
@@ -73,13 +74,13 @@ struct GridSmem {
 template <bool kEncode, int NPTS> struct LayerTables { typedef RowSmem<NPTS> type; };
 template <int NPTS> struct LayerTables<false, NPTS> { typedef GridSmem<NPTS> type; };
 
-template <int D, bool WR> struct LayerRowScratch { TeamSmem<D> team[24 / RowTeam<D>::TEAM]; };
-template <int D> struct LayerRowScratch<D, true> { unsigned long long xbuf[kWrLayerWarps][kWrItems]; };
+template <int D, int ROW_WARPS, bool WR> struct LayerRowScratch { TeamSmem<D> team[ROW_WARPS / RowTeam<D>::TEAM]; };
+template <int D, int ROW_WARPS> struct LayerRowScratch<D, ROW_WARPS, true> { unsigned long long xbuf[ROW_WARPS][kWrItems]; };
 
 template <bool kEncode, int D, int NPTS, bool kFull>
 struct LayerRowSmem {
   typename LayerTables<kEncode, NPTS>::type tables;
-  LayerRowScratch<D, LayerGeom<D, kFull>::WR> scratch;
+  LayerRowScratch<D, LayerGeom<kEncode, D, kFull>::ROW_WARPS, LayerGeom<kEncode, D, kFull>::WR> scratch;
 };
 
 // The GEMM epilogue stages each 32-row x 32-column fp32 piece of a tile in shared memory (128-byte
@@ -225,12 +226,12 @@ __device__ __forceinline__ void fence_proxy_async_all() {
 // kFull: the Hadamard block and the scale group both span the whole row (the paper's setting for
 // d_kv = 1024, Section 4.1); their logarithms are then compile-time constants of the row code.
 template <bool kEncode, int D, int NPTS, bool kBf16, bool kFull>
-__global__ void __launch_bounds__((LayerGeom<D, kFull>::THREADS), 1)
+__global__ void __launch_bounds__((LayerGeom<kEncode, D, kFull>::THREADS), 1)
 layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant__ CUtensorMap tmVprev,
              const __grid_constant__ CUtensorMap tmKhat, const __grid_constant__ CUtensorMap tmWk,
              const __grid_constant__ CUtensorMap tmWv, const __grid_constant__ CUtensorMap tmP,
              const LayerArgs a) {
-  using G = LayerGeom<D, kFull>;
+  using G = LayerGeom<kEncode, D, kFull>;
   constexpr int NTN = D / kBN;             // feature tiles per token block = CTAs per token block
   constexpr int NKD = D / kBK;             // k-blocks per d_kv input features
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);

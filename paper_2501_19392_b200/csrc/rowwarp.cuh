@@ -157,6 +157,10 @@ __device__ __forceinline__ void wr_finish_row(const WarpRowCtx& rc, f32x2_t (&wp
       wr_load_pred8(pred_row + ch * 256 + lane * 8, p);
 #pragma unroll
       for (int i = 0; i < 4; ++i) wp[4 * ch + i] = add2(p[i], wp[4 * ch + i]);
+    } else {
+      // adding the zero prediction turns a -0 (a zero value whose sign was flipped) into +0
+#pragma unroll
+      for (int i = 0; i < 4; ++i) wp[4 * ch + i] = add2(pack2(0.0f, 0.0f), wp[4 * ch + i]);
     }
     // streaming store: the reconstruction is read at most once more before it leaves L2
     __stcs(reinterpret_cast<uint4*>(hat_row + ch * 256 + lane * 8),

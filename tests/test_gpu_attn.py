@@ -75,9 +75,21 @@ def test_decode_attn_matches_dequantize_then_attend(batch, ctx, n_q, n_kv, hd, d
     denom = np.abs(ref2).max(axis=-1, keepdims=True)
     assert np.all((np.abs(o - ref2) <= 2e-3 * denom) | adjacent)
     assert np.abs(lse.cpu().numpy() - ref2_lse).max() <= 1e-4
-    # (3) end to end against the oracle's own dequantize-then-attend: the flips add a little
-    assert np.abs(o - ref).max() <= 1e-2 * np.abs(ref).max()
-    assert np.abs(lse.cpu().numpy() - ref_lse).max() <= 2e-3
+    # (3) end to end against the oracle's own dequantize-then-attend.  What separates it from (2) is
+    #     the effect that the one-ulp flips in the decoded rows have on the ORACLE's own output: a
+    #     flipped key element moves its token's score by about 1e-3, and a diffuse softmax over random
+    #     values yields outputs several times smaller than the values themselves, so relative to the
+    #     head's largest output this reaches a few 1e-3 (largest measured over these cases: 2.3e-3).
+    #     It is bounded at 5e-3; the end-to-end bar is therefore 2e-3 + 5e-3 of the head's largest
+    #     output, or a one-ulp flip of the 16-bit output.
+    denom1 = np.abs(ref).max(axis=-1, keepdims=True)
+    flips = np.abs(ref2 - ref) / denom1
+    print("effect of one-ulp flips in the decoded rows on the oracle's attention output: %.2e" % flips.max())
+    assert flips.max() <= 5e-3, flips.max()
+    ref_bits = synth.to_bits(torch.from_numpy(ref).to(codec.torch_dtype)).astype(np.int64)
+    adjacent1 = np.abs(gpu_bits(out).astype(np.int64) - ref_bits) <= 1
+    assert np.all((np.abs(o - ref) <= 7e-3 * denom1) | adjacent1)
+    assert np.abs(lse.cpu().numpy() - ref_lse).max() <= 5e-4
     # (4) without the optional K_hat/V_hat outputs the result is bit-identical
     out_b, lse_b = codec.decode_attn(*args, want_lse=True)
     assert torch.equal(out_b, out) and torch.equal(lse_b, lse)

@@ -9,7 +9,7 @@ import torch
 
 import oracle
 from paper_2501_19392_b200 import synth
-from parity import check_codes, check_recon, gpu_bits, scale_rows_ok
+from parity import check_codes, check_recon, check_same_rows, gpu_bits, scale_rows_ok
 from util import bits_to_f64
 
 pytestmark = pytest.mark.gpu
@@ -97,7 +97,7 @@ def test_encode_with_adapters_teacher_forced(cfg, T, n):
         check_codes(Kc.cpu().numpy(), ok_, bits, rows_ok)
         # reconstruction: rows whose codes agree (a near-tie flip legitimately moves its whole Hadamard block)
         same_codes = rows_ok & (Kc.cpu().numpy() == ok_["codes"]).all(axis=1)
-        assert same_codes.mean() > 0.9
+        check_same_rows(same_codes, shape.d_kv, int((~rows_ok).sum()))
         check_recon(gpu_bits(Kh), ok_["hat_exact"], ok_["hat"], shape.dtype, same_codes)
         # values, teacher-forced inside the layer too: the value phase is given the ORACLE's K_hat
         from paper_2501_19392_b200 import api
@@ -109,7 +109,7 @@ def test_encode_with_adapters_teacher_forced(cfg, T, n):
         rows_ok_v, _ = scale_rows_ok(gpu_bits(Vs2.view(torch.float16)), ov_["scales"], ov_["scales_exact"])
         check_codes(Vc2.cpu().numpy(), ov_, bits, rows_ok_v)
         same_codes_v = rows_ok_v & (Vc2.cpu().numpy() == ov_["codes"]).all(axis=1)
-        assert same_codes_v.mean() > 0.9
+        check_same_rows(same_codes_v, shape.d_kv, int((~rows_ok_v).sum()))
         check_recon(gpu_bits(Vh2), ov_["hat_exact"], ov_["hat"], shape.dtype, same_codes_v)
         # the one-call encode agrees with its own phases wherever its K_hat equals the oracle's
         same_k = (gpu_bits(Kh) == ok_["hat"]).all(axis=1)
@@ -159,7 +159,7 @@ def test_full_size_layer_on_sampled_rows(T, n):
     assert n_bad <= 2
     check_codes(Kc.cpu().numpy()[rows], ok_, bits, rows_ok)
     same = rows_ok & (Kc.cpu().numpy()[rows] == ok_["codes"]).all(axis=1)
-    assert same.mean() > 0.9
+    check_same_rows(same, d, int((~rows_ok).sum()))
     check_recon(gpu_bits(Kh)[rows], ok_["hat_exact"], ok_["hat"], dtype, same)
     # values: the oracle is given the library's reconstructed keys of those rows (teacher forcing)
     ov_ = ora.encode_phase(sel(V), [sel(prevV), gpu_bits(Kh)[rows]], b(Wv), None, "v")
@@ -167,7 +167,7 @@ def test_full_size_layer_on_sampled_rows(T, n):
     assert n_bad <= 2
     check_codes(Vc.cpu().numpy()[rows], ov_, bits, rows_ok_v)
     same_v = rows_ok_v & (Vc.cpu().numpy()[rows] == ov_["codes"]).all(axis=1)
-    assert same_v.mean() > 0.9
+    check_same_rows(same_v, d, int((~rows_ok_v).sum()))
     check_recon(gpu_bits(Vh)[rows], ov_["hat_exact"], ov_["hat"], dtype, same_v)
     # decode of the library's own codes reproduces the encoder's reconstruction bit for bit, all rows
     Kh2, Vh2 = codec.decode(Kc, Ks, Vc, Vs, g(prevK), g(prevV), g(Wk), g(Wv))
@@ -221,12 +221,14 @@ def test_fused_layer_shapes_strides_and_bias(d, hd, h, g, n, dtype, T):
     assert n_bad <= 2
     check_codes(Kc.cpu().numpy(), ok_, bits, rows_ok)
     same = rows_ok & (Kc.cpu().numpy() == ok_["codes"]).all(axis=1)
+    check_same_rows(same, d, int((~rows_ok).sum()))
     check_recon(gpu_bits(Kh), ok_["hat_exact"], ok_["hat"], dtype, same)
     ov_ = ora.encode_phase(b(kv.V[1]), [b(kv.V[0]), gpu_bits(Kh)], b(ad.Wv[1]), ad.bv[1].numpy(), "v")
     rows_ok_v, n_bad = scale_rows_ok(gpu_bits(Vs.view(torch.float16)), ov_["scales"], ov_["scales_exact"])
     assert n_bad <= 2
     check_codes(Vc.cpu().numpy(), ov_, bits, rows_ok_v)
     same_v = rows_ok_v & (Vc.cpu().numpy() == ov_["codes"]).all(axis=1)
+    check_same_rows(same_v, d, int((~rows_ok_v).sum()))
     check_recon(gpu_bits(Vh), ov_["hat_exact"], ov_["hat"], dtype, same_v)
     # decode of the oracle's codes (fused kernel) against the oracle's reconstruction
     oc = lambda o: (torch.from_numpy(o["codes"]).to(DEV), torch.from_numpy(o["scales"]).view(torch.float16).to(DEV))
@@ -294,12 +296,13 @@ def test_bulk_decode_shape_on_sampled_rows():
     check_recon(gpu_bits(Vh[idx]), vd["hat_exact"], vd["hat"], dtype)
 
 
-def test_free_running_chain_tracks_the_oracle_chain():
-    """Six layers with each side feeding itself (no teacher forcing): codes may drift apart after
-    near-ties, so the chains are compared statistically: per layer, the library's relative
-    reconstruction error stays within 2 % (relative) of the oracle's, and most codes still agree."""
+@pytest.mark.parametrize("T,L", [(512, 6), (512, 28)])
+def test_free_running_chain_tracks_the_oracle_chain(T, L):
+    """Each side feeds itself through all layers (no teacher forcing; 28 layers is the depth the
+    benchmark's chain runs): codes may drift apart after near-ties, so the chains are compared
+    statistically: per layer, the library's relative reconstruction error stays within 1 % (relative)
+    of the oracle's, and in the first layers most codes still agree."""
     from paper_2501_19392_b200 import chain as chain_mod
-    T, L = 512, 6
     shape, kv, ad = chain(2, T, L)
     d, dtype, bits = shape.d_kv, shape.dtype, shape.code_bits
     codec, ora = make(d, shape.had_block, shape.scale_group, shape.grid_size, dtype)
@@ -310,6 +313,7 @@ def test_free_running_chain_tracks_the_oracle_chain():
     Kg, Vg = [g(t) for t in kv.K], [g(t) for t in kv.V]
     b = synth.to_bits
     pk = pv = None
+    worst, least = 0.0, 1.0
     for l in range(L):
         has = l > 0
         cur, prv = l % 2, (l + 1) % 2
@@ -323,7 +327,161 @@ def test_free_running_chain_tracks_the_oracle_chain():
             x64 = x.to(torch.float64).numpy()
             err_gpu = ((hat_gpu.to(torch.float64).cpu().numpy() - x64) ** 2).sum() / (x64 ** 2).sum()
             err_ora = ((bits_to_f64(o["hat"], dtype) - x64) ** 2).sum() / (x64 ** 2).sum()
-            assert abs(err_gpu - err_ora) <= 0.02 * err_ora, (l, err_gpu, err_ora)
+            worst = max(worst, abs(err_gpu - err_ora) / err_ora)
+            assert abs(err_gpu - err_ora) <= 0.01 * err_ora, (l, err_gpu, err_ora)
+        # a row whose codes differ once keeps drifting (its residuals differ from then on), so the share
+        # of equal code bytes falls with depth; it is a requirement only for the first layers
         agree = (cache.Kcodes[l].cpu().numpy() == ok_["codes"]).mean()
-        assert agree > 0.9, (l, agree)
+        least = min(least, agree)
+        if l < 4:
+            assert agree > 0.9, (l, agree)
+    print("free-running chain, %d layers: largest relative gap of the reconstruction error %.2e, "
+          "smallest share of equal key code bytes %.3f" % (L, worst, least))
     assert codec.poll_status() == 0
+
+
+# ---------------------------------------------------------------------------------------------------
+# Degenerate cases of the quantizer (Section 2 "Vector Quantization": group-wise scales, round to the
+# nearest grid point), each against the oracle
+# ---------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("d,h,g,dtype", [(1024, 1024, 1024, synth.BF16), (512, 64, 64, synth.F16), (512, 128, 256, synth.BF16)])
+def test_zero_rows_and_zero_groups(d, h, g, dtype):
+    """Rows and scale groups that are exactly zero (what padded batches look like): scale 0, every
+    pair takes the code of the grid point nearest the origin, the reconstruction is the prediction.
+    Checked without a predictor and with one (zero previous-layer rows give a zero prediction)."""
+    n, T = 16, 70
+    codec, ora = make(d, h, g, n, dtype)
+    X = synth.random_16bit((T, d), dtype, seed=31, std=1.3)
+    X[3] = 0                                 # a whole row
+    X[T - 1] = 0                             # the last row of the call
+    X[10, :g] = 0                            # the first group of a row
+    X[11, d - g:] = 0                        # the last group of a row
+    Xv = synth.random_16bit((T, d), dtype, seed=32)
+    Xv[0] = 0
+    b = synth.to_bits
+    ok_, ov_ = ora.encode_layer(b(X), b(Xv))
+    Kc, Ks, Vc, Vs, Kh, Vh = codec.encode(X.to(DEV), Xv.to(DEV))
+    assert codec.poll_status() == 0
+    origin = int(np.argmin((codec_grid(n) ** 2).sum(axis=1)))
+    for o, c, sc, hat in ((ok_, Kc, Ks, Kh), (ov_, Vc, Vs, Vh)):
+        rows_ok, n_bad = scale_rows_ok(gpu_bits(sc.view(torch.float16)), o["scales"], o["scales_exact"])
+        assert n_bad <= 1
+        check_codes(c.cpu().numpy(), o, 4, rows_ok)
+    ks = gpu_bits(Ks.view(torch.float16))
+    assert (ks[3] == 0).all() and (ks[T - 1] == 0).all() and ks[10, 0] == 0 and ks[11, -1] == 0
+    from util import unpack_codes
+    ki = unpack_codes(Kc.cpu().numpy(), 4)
+    assert (ki[3] == origin).all() and (ki[T - 1] == origin).all()
+    assert (ki[10, :g // 2] == origin).all() and (ki[11, -(g // 2):] == origin).all()
+    assert np.array_equal(ki[3], unpack_codes(ok_["codes"], 4)[3])
+    for rows_hat, o, r in ((Kh, ok_, 3), (Kh, ok_, T - 1), (Vh, ov_, 0)):       # zero, as the oracle's (+0)
+        assert not gpu_bits(rows_hat)[r].any() and np.array_equal(gpu_bits(rows_hat)[r], o["hat"][r])
+    # with a predictor: previous-layer rows of zeros predict zero, so zero targets leave a zero residual
+    shape = dataclasses.replace(synth.CONFIGS[2], n_kv_heads=d // 64, head_dim=64, n_tokens=T, n_layers=2, dtype=dtype,
+                                had_block=h, scale_group=g, grid_size=n, channel_scales=False)
+    ad = synth.random_adapters(shape, seed=33)
+    pK = synth.random_16bit((T, d), dtype, seed=34)
+    pV = synth.random_16bit((T, d), dtype, seed=35)
+    pK[3] = 0
+    pV[3] = 0
+    Xv[3] = 0
+    dev = lambda t: t.to(DEV)
+    ok2, ov2 = ora.encode_layer(b(X), b(Xv), b(pK), b(pV), b(ad.Wk[1]), b(ad.Wv[1]))
+    Kc2, Ks2, Vc2, Vs2, Kh2, Vh2 = codec.encode(dev(X), dev(Xv), dev(pK), dev(pV), dev(ad.Wk[1]), dev(ad.Wv[1]))
+    assert codec.poll_status() == 0
+    assert (gpu_bits(Ks2.view(torch.float16))[3] == 0).all() and (gpu_bits(Vs2.view(torch.float16))[3] == 0).all()
+    assert (unpack_codes(Kc2.cpu().numpy(), 4)[3] == origin).all() and (unpack_codes(Vc2.cpu().numpy(), 4)[3] == origin).all()
+    assert np.array_equal(Kc2.cpu().numpy()[3], ok2["codes"][3]) and np.array_equal(Vc2.cpu().numpy()[3], ov2["codes"][3])
+    assert not gpu_bits(Kh2)[3].any() and not gpu_bits(Vh2)[3].any()
+    Kd, Vd = codec.decode(Kc2, Ks2, Vc2, Vs2, dev(pK), dev(pV), dev(ad.Wk[1]), dev(ad.Wv[1]))
+    assert torch.equal(Kd, Kh2) and torch.equal(Vd, Vh2)
+
+
+def codec_grid(n):
+    return synth.lloyd_grid(n, seed=7, n_samples=1 << 14, iters=25).astype(np.float64)
+
+
+@pytest.mark.parametrize("d,h", [(1024, 1024), (512, 64)])
+def test_scale_is_clamped_to_the_largest_fp16(d, h):
+    """A bf16 row whose residual RMS exceeds 65504 (finite values only): the stored scale is the
+    largest finite fp16 and the codes follow from dividing by it, as in the oracle."""
+    n, T, dtype = 16, 40, synth.BF16
+    codec, ora = make(d, h, h, n, dtype)
+    X = synth.random_16bit((T, d), dtype, seed=41, std=1.5e5)        # RMS about 1.5e5 in every group
+    X[1] = synth.random_16bit((d,), dtype, seed=42, std=4.0e4)       # below the clamp
+    X[2] = synth.random_16bit((d,), dtype, seed=43, std=3.0e6)       # far above: rotated values of about 45 grid units
+    Xv = synth.random_16bit((T, d), dtype, seed=44)
+    b = synth.to_bits
+    ok_, ov_ = ora.encode_layer(b(X), b(Xv))
+    Kc, Ks, Vc, Vs, Kh, Vh = codec.encode(X.to(DEV), Xv.to(DEV))
+    assert codec.poll_status() == 0
+    ks = gpu_bits(Ks.view(torch.float16))
+    assert (ks[0] == 0x7BFF).all() and (ks[2] == 0x7BFF).all() and (ks[1] < 0x7BFF).all()
+    rows_ok, n_bad = scale_rows_ok(ks, ok_["scales"], ok_["scales_exact"])
+    assert n_bad <= 1
+    check_codes(Kc.cpu().numpy(), ok_, 4, rows_ok)
+    Kd, Vd = codec.decode(torch.from_numpy(ok_["codes"]).to(DEV), torch.from_numpy(ok_["scales"]).view(torch.float16).to(DEV),
+                          torch.from_numpy(ov_["codes"]).to(DEV), torch.from_numpy(ov_["scales"]).view(torch.float16).to(DEV))
+    check_recon(gpu_bits(Kd), ok_["hat_exact"], ok_["hat"], dtype)
+
+
+@pytest.mark.parametrize("d,h,dtype", [(512, 64, synth.F16), (1024, 1024, synth.BF16)])
+def test_exact_ties_go_to_the_lowest_index(d, h, dtype):
+    """Inputs built so that the rotated, normalised values are small dyadic numbers that land exactly
+    on Voronoi boundaries of a symmetric 4 x 4 grid (margin 0): both sides must pick the lowest index,
+    so every code is compared with the oracle's, ties included."""
+    from paper_2501_19392_b200 import api
+    from util import unpack_codes
+    side = np.array([-1.5, -0.5, 0.5, 1.5])
+    grid = np.array([[x, y] for x in side for y in side], dtype=np.float32)       # sorted lexicographically
+    sk, sv = synth.hadamard_signs(d, 11), synth.hadamard_signs(d, 12)
+    codec, ora = api.Codec(d, h, h, grid, dtype, sk, sv), oracle.Oracle(d, h, h, grid, dtype, sk, sv)
+    rng = np.random.default_rng(51)
+    T = 64
+    H = np.array([[1.0]])
+    while H.shape[0] < h:
+        H = np.block([[H, H], [H, -H]])
+    X = np.zeros((T, d))
+    for t in range(T):
+        for blk in range(d // h):
+            # rotated target with mean square exactly 1: a quarter zeros, half +-1, an eighth +-2, an eighth zeros
+            y = np.concatenate([np.zeros(h // 4), rng.choice([-1.0, 1.0], h // 2), rng.choice([-2.0, 2.0], h // 8),
+                                np.zeros(h // 8)])
+            y = y[rng.permutation(h)]
+            s = 2.0 ** rng.integers(-3, 3)                       # the group's scale: a power of two
+            u = s * (H @ y) / np.sqrt(h)                         # H / sqrt(h) is orthonormal and symmetric
+            X[t, blk * h:(blk + 1) * h] = u * sk[blk * h:(blk + 1) * h]
+    Xt = torch.from_numpy(X).to(synth.torch_dtype(dtype))
+    assert np.array_equal(Xt.to(torch.float64).numpy(), X), "the construction must be exact in the 16-bit type"
+    Xv = synth.random_16bit((T, d), dtype, seed=52)
+    b = synth.to_bits
+    ok_, ov_ = ora.encode_layer(b(Xt), b(Xv))
+    assert (ok_["margins"] == 0).mean() > 0.3, "the construction must produce exact ties"
+    Kc, Ks, Vc, Vs, Kh, Vh = codec.encode(Xt.to(DEV), Xv.to(DEV))
+    assert codec.poll_status() == 0
+    assert np.array_equal(gpu_bits(Ks.view(torch.float16)), ok_["scales"])
+    assert np.array_equal(unpack_codes(Kc.cpu().numpy(), 4), unpack_codes(ok_["codes"], 4))
+    assert np.array_equal(gpu_bits(Kh), ok_["hat"])              # every step of this case is exact
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
+    """One warp waits 1 ms on a barrier that nothing arrives on: the kernel returns, the status word
+    reads AQUAKV_ERR_TIMEOUT once, and an ordinary decode on the same context then succeeds."""
+    codec, ora = make(1024, 1024, 1024, 16, synth.BF16)
+    assert codec.poll_status() == 0
+    codec.selftest_bounded_wait(1_000_000)
+    assert codec.poll_status() == -6              # AQUAKV_ERR_TIMEOUT
+    assert codec.poll_status() == 0               # cleared by the poll
+    shape = dataclasses.replace(synth.CONFIGS[4], n_tokens=200, n_layers=2)
+    cache = synth.random_cache(shape, seed=61, n_layers=1)
+    ad = synth.random_adapters(shape, seed=62)
+    pK = synth.random_16bit((200, 1024), synth.BF16, seed=63)
+    pV = synth.random_16bit((200, 1024), synth.BF16, seed=64)
+    g = lambda t: t.to(DEV)
+    Kh, Vh = codec.decode(g(cache.Kcodes[0]), g(cache.Kscales[0]), g(cache.Vcodes[0]), g(cache.Vscales[0]),
+                          g(pK), g(pV), g(ad.Wk[1]), g(ad.Wv[1]))
+    assert codec.poll_status() == 0
+    b = synth.to_bits
+    kd = ora.decode_phase(cache.Kcodes[0].numpy(), b(cache.Kscales[0]), [b(pK)], b(ad.Wk[1]), None, "k")
+    check_recon(gpu_bits(Kh), kd["hat_exact"], kd["hat"], synth.BF16)
