@@ -125,11 +125,14 @@ int aquakv_destroy(aquakv_ctx* ctx);
 size_t aquakv_workspace_bytes(const aquakv_ctx* ctx, int64_t n_tokens, int op);
 
 /*
- * Workspace of aquakv_decode_attn for this problem shape (its split-KV partials depend on the
+ * Workspace of aquakv_decode_attn for this problem shape (its attention partials depend on the
  * batch and head counts, which aquakv_workspace_bytes does not see).  0 on invalid arguments.
- * The cache is decoded in chunks of up to about 147 K tokens; the workspace holds one chunk's
- * decoded keys and values (4 * d_kv bytes per token: about 0.6 GB at d_kv = 1024 for long caches,
- * whether or not Khat/Vhat are passed) besides the fused kernel's buffers.
+ * With predictors at d_kv = 1024 (Hadamard block = scale group = d_kv) decode and attention run as
+ * one kernel: the workspace holds that kernel's buffers (the prediction ring and, when Khat/Vhat
+ * are not requested, rings of three waves of decoded keys and values: about 0.1 GB in all) and one
+ * attention partial per 128-token block and query head (about 130 bytes per token at 32 query
+ * heads).  In the other cases the cache is decoded in chunks of up to about 147 K tokens into the
+ * workspace (4 * d_kv bytes per token of a chunk) and a second kernel attends over each chunk.
  */
 size_t aquakv_decode_attn_workspace_bytes(const aquakv_ctx* ctx, int32_t batch, int64_t ctx_len,
                                           int32_t n_q_heads, int32_t head_dim);
@@ -245,8 +248,15 @@ int aquakv_decode_noalloc(aquakv_ctx* ctx, int64_t n_tokens,
  * n_kv_heads * head_dim must equal d_kv; head_dim must be 64 or 128; n_q_heads a multiple of
  * n_kv_heads with n_q_heads/n_kv_heads <= 8.  q, out: [batch][n_q_heads][head_dim] 16-bit,
  * contiguous.  lse: optional fp32 [batch][n_q_heads] log-sum-exp of the scaled scores (NULL =
- * not written).  Khat, Vhat: optional outputs [n_tokens, ld_hat] for the next layer's decode
- * (NULL = the reconstruction lives only in the workspace, chunk by chunk).
+ * not written).  Khat, Vhat: optional outputs [n_tokens, ld_hat] for the next layer's decode.
+ *
+ * With predictors at d_kv = 1024 and Hadamard block = scale group = d_kv (the paper's setting) this
+ * is ONE kernel: while the tensor cores form the predictions and the row warps reconstruct token
+ * rows, attention warps of the same kernel take every 128-token block as soon as its keys and
+ * values exist and reduce it to per-block softmax partials; a small second kernel merges the
+ * partials of each sequence.  Without Khat/Vhat the decoded rows live only in a ring of three
+ * waves of tokens in the workspace.  Without predictors (layer 0) and for the other shapes decode
+ * and attention are separate kernels behind this entry point (see the workspace note above).
  */
 int aquakv_decode_attn(aquakv_ctx* ctx, int32_t batch, int64_t ctx_len,
                        int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, float softmax_scale,

@@ -364,12 +364,12 @@ constexpr int kLayerRing = 3;       // prediction buffers
 constexpr int kKhatRing = 3;        // waves of reconstructed keys kept when the caller wants none
 
 struct LayerWs {
-  size_t p_off, khat_off, flags_off, flags_bytes, total;
+  size_t p_off, khat_off, vhat_off, flags_off, flags_bytes, total;
   int mw, n_waves, n_mblocks;
   int grid_mw;     // token-block slots the launched grid covers (>= mw)
 };
 
-LayerWs layer_ws(const aquakv_ctx* c, int64_t T) {
+LayerWs layer_ws(const aquakv_ctx* c, int64_t T, bool with_attn = false) {
   LayerWs w;
   const int d = c->p.d_kv, ntn = d / kBN;
   w.n_mblocks = int((T + kBM - 1) / kBM);
@@ -384,28 +384,47 @@ LayerWs layer_ws(const aquakv_ctx* c, int64_t T) {
   w.n_waves = (w.n_mblocks + mw - 1) / mw;
   w.p_off = 0;
   w.khat_off = round_up(size_t(kLayerRing) * mw * kBM * d * sizeof(float), 256);
-  w.flags_off = w.khat_off + round_up(size_t(kKhatRing) * mw * kBM * d * 2, 256);
-  w.flags_bytes = size_t(2) * 2 * w.n_waves * mw * sizeof(int);
+  w.vhat_off = w.khat_off + round_up(size_t(kKhatRing) * mw * kBM * d * 2, 256);
+  w.flags_off = with_attn ? w.vhat_off + round_up(size_t(kKhatRing) * mw * kBM * d * 2, 256) : w.vhat_off;
+  w.flags_bytes = size_t(with_attn ? 5 : 4) * w.n_waves * mw * sizeof(int);   // gemm_done, rows_done (two jobs per wave each), attn_done
   w.total = w.flags_off + round_up(w.flags_bytes, 256) + kWsSlack;
   return w;
 }
 
 struct AttnWs {
   size_t layer_off, khat_off, vhat_off, ml_off, o_off, total;
-  int chunk_blocks;     // split-KV blocks per chunk
-  int n_splits;
+  int chunk_blocks;     // split-KV blocks per chunk (two-kernel path)
+  int n_splits;         // partial slots per sequence
+  bool fused;           // decode and attention in one launch of the layer kernel
 };
 
-// The decode of a long cache runs chunk by chunk, about 32 waves of the fused kernel each: long
-// enough that the kernel's fill and drain cost little (eight-wave chunks measured 9 % slower; the
-// attention kernel read the decoded rows from DRAM either way), short enough to bound the
-// workspace that holds a chunk's decoded keys/values when the caller does not ask for them
-// (0.6 GB at d_kv = 1024).
+bool fused_attn_supported(const aquakv_ctx* c);
+
+// Workspace of aquakv_decode_attn.  With predictors at d_kv = 1024 (Hadamard block = scale group =
+// the row) decode and attention are ONE launch of the layer kernel: the workspace holds that
+// kernel's buffers (prediction ring, rings of three waves of decoded keys / values, counters) and
+// the attention partials, one slot per 128-token block that overlaps a sequence.  Otherwise (no
+// predictor, other shapes) the cache is decoded chunk by chunk, about 32 waves each, into the
+// workspace (or the caller's Khat/Vhat) and a separate kernel attends over each chunk in blocks of
+// 1024 tokens.
 AttnWs attn_ws(const aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_heads,
-               int32_t head_dim) {
+               int32_t head_dim, bool has_pred) {
   AttnWs w;
-  const int tb = c->attn_block_tokens;
   const size_t d = size_t(c->p.d_kv);
+  w.fused = has_pred && fused_attn_supported(c);
+  if (w.fused) {
+    w.n_splits = int((ctx_len + kAttnSubTokens - 2) / kAttnSubTokens) + 1;   // sub-blocks of the flattened token
+                                                                             // index a sequence can overlap
+    w.chunk_blocks = 0;
+    const int64_t slots = int64_t(batch) * w.n_splits;
+    w.layer_off = 0;
+    w.khat_off = w.vhat_off = 0;
+    w.ml_off = round_up(layer_ws(c, int64_t(batch) * ctx_len, true).total, 256);
+    w.o_off = w.ml_off + round_up(size_t(slots) * n_q_heads * 2 * sizeof(float), 256);
+    w.total = w.o_off + round_up(size_t(slots) * n_q_heads * head_dim * sizeof(float), 256) + kWsSlack;
+    return w;
+  }
+  const int tb = c->attn_block_tokens;
   w.n_splits = int((ctx_len + tb - 1) / tb);
   const int wave_tokens = (c->sm_count / int(d / kBN) > 0 ? c->sm_count / int(d / kBN) : 1) * kBM;
   int cb = 32 * wave_tokens / tb;
@@ -425,7 +444,7 @@ AttnWs attn_ws(const aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_
   return w;
 }
 
-template <bool ENC, int D, int NPTS, bool BF, bool FULL>
+template <bool ENC, int D, int NPTS, bool BF, bool FULL, int AHD = 0>
 int launch_layer_t(int device, cudaStream_t st, int grid, const CUtensorMap* tm, const LayerArgs& a) {
   // the shared-memory opt-in is a per-device attribute of the function: one bit per device and
   // instantiation (setting it twice from two threads is harmless)
@@ -433,14 +452,14 @@ int launch_layer_t(int device, cudaStream_t st, int grid, const CUtensorMap* tm,
   constexpr size_t smem = layer_smem_bytes<ENC, D, NPTS, FULL>();
   const unsigned long long bit = 1ull << (device & 63);
   if (device >= 64 || !(attr_devices.load(std::memory_order_acquire) & bit)) {
-    if (cudaFuncSetAttribute(layer_kernel<ENC, D, NPTS, BF, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(layer_kernel<ENC, D, NPTS, BF, FULL, AHD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              int(smem)) != cudaSuccess)
       return AQUAKV_ERR_CUDA;
     if (device < 64) attr_devices.fetch_or(bit, std::memory_order_release);
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(unsigned(grid));
-  cfg.blockDim = dim3(unsigned(LayerGeom<ENC, D, FULL>::THREADS));
+  cfg.blockDim = dim3(unsigned(layer_threads<ENC, D, FULL, AHD>()));
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -450,7 +469,7 @@ int launch_layer_t(int device, cudaStream_t st, int grid, const CUtensorMap* tm,
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, layer_kernel<ENC, D, NPTS, BF, FULL>, tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], a) ==
+  return cudaLaunchKernelEx(&cfg, layer_kernel<ENC, D, NPTS, BF, FULL, AHD>, tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], a) ==
                  cudaSuccess
              ? AQUAKV_OK
              : AQUAKV_ERR_CUDA;
@@ -468,21 +487,38 @@ void launch_layer_dec_t(int* rc, int device, cudaStream_t st, int grid, const CU
   // the decoder has the fixed-size instantiation only where it selects the one-warp-per-row routines
   if constexpr (D == 1024) {
     if (a.log_h == 10 && a.log_g == 10) {
+      if (a.q != nullptr) {       // decode + single-query attention in one kernel
+        *rc = a.n_kv_heads * 128 == D ? launch_layer_t<false, D, NPTS, BF, true, 128>(device, st, grid, tm, a)
+                                      : launch_layer_t<false, D, NPTS, BF, true, 64>(device, st, grid, tm, a);
+        return;
+      }
       *rc = launch_layer_t<false, D, NPTS, BF, true>(device, st, grid, tm, a);
       return;
     }
   }
-  *rc = launch_layer_t<false, D, NPTS, BF, false>(device, st, grid, tm, a);
+  *rc = a.q != nullptr ? AQUAKV_ERR_UNSUPPORTED : launch_layer_t<false, D, NPTS, BF, false>(device, st, grid, tm, a);
 }
+
+// The attention a decode launch also computes (Algorithm 4 lines 5-9); q == nullptr: none.
+struct LayerAttnArgs {
+  const void* q;
+  int ctx, n_q_heads, n_kv_heads, n_splits;
+  float scale_log2;
+  float* part_ml;
+  float* part_o;
+};
+
+// True if decode + attention runs as one launch of the layer kernel for this context.
+bool fused_attn_supported(const aquakv_ctx* c) { return c->p.d_kv == 1024 && c->log_h == 10 && c->log_g == 10; }
 
 // Algorithm 2 (encode = true) or Algorithm 3 for one layer with predictors, all tokens, one launch.
 int launch_layer(aquakv_ctx* c, cudaStream_t st, bool encode, int64_t T, const void* K, const void* V,
                  int64_t ld_kv, const void* Khat_prev, const void* Vhat_prev, int64_t ld_prev,
                  const void* Wk, const void* Wv, const float* bk, const float* bv, uint8_t* Kcodes,
                  uint16_t* Kscales, uint8_t* Vcodes, uint16_t* Vscales, void* Khat, void* Vhat,
-                 int64_t ld_hat, void* workspace) {
+                 int64_t ld_hat, void* workspace, const LayerAttnArgs* attn = nullptr) {
   const int d = c->p.d_kv;
-  const LayerWs ws = layer_ws(c, T);
+  const LayerWs ws = layer_ws(c, T, attn != nullptr);
   uint8_t* wsb = ws_base(workspace);
   LayerArgs a;
   std::memset(&a, 0, sizeof(a));
@@ -514,6 +550,22 @@ int launch_layer(aquakv_ctx* c, cudaStream_t st, bool encode, int64_t T, const v
   }
   a.Vhat = static_cast<uint16_t*>(Vhat);
   a.ldVhat = ld_hat;
+  if (attn != nullptr) {
+    if (Vhat == nullptr) {       // decoded values the caller does not want: a ring like the keys'
+      a.vhat_ring = kKhatRing;
+      a.Vhat = reinterpret_cast<uint16_t*>(wsb + ws.vhat_off);
+      a.ldVhat = d;
+    }
+    a.q = static_cast<const uint16_t*>(attn->q);
+    a.ctx = attn->ctx;
+    a.n_q_heads = attn->n_q_heads;
+    a.n_kv_heads = attn->n_kv_heads;
+    a.n_splits = attn->n_splits;
+    a.scale_log2 = attn->scale_log2;
+    a.part_ml = attn->part_ml;
+    a.part_o = attn->part_o;
+    a.attn_done = a.rows_done + size_t(2) * ws.n_waves * ws.mw;
+  }
   a.signmask_k = c->d_signmask[kRoleK];
   a.signmask_v = c->d_signmask[kRoleV];
   const CodecArgs ca = codec_args(c, kRoleK, 0);
@@ -712,7 +764,10 @@ size_t aquakv_workspace_bytes(const aquakv_ctx* c, int64_t n_tokens, int op) {
 size_t aquakv_decode_attn_workspace_bytes(const aquakv_ctx* c, int32_t batch, int64_t ctx_len,
                                           int32_t n_q_heads, int32_t head_dim) {
   if (c == nullptr || batch <= 0 || ctx_len <= 0 || n_q_heads <= 0 || head_dim <= 0) return 0;
-  return attn_ws(c, batch, ctx_len, n_q_heads, head_dim).total;
+  // the caller may or may not pass predictors: the larger of the two layouts
+  const size_t a = attn_ws(c, batch, ctx_len, n_q_heads, head_dim, true).total;
+  const size_t b = attn_ws(c, batch, ctx_len, n_q_heads, head_dim, false).total;
+  return a > b ? a : b;
 }
 
 int64_t aquakv_launch_count(const aquakv_ctx* c) { return c ? c->launches : 0; }
@@ -1066,9 +1121,40 @@ int aquakv_decode_attn(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_
   if (Khat != nullptr && (Khat == Khat_prev || Khat == Vhat_prev || Vhat == Vhat_prev ||
                           Vhat == Khat_prev || Vhat == Khat))
     return AQUAKV_ERR_INVALID_ARG;
-  const AttnWs ws = attn_ws(c, batch, ctx_len, n_q_heads, head_dim);
+  const AttnWs ws = attn_ws(c, batch, ctx_len, n_q_heads, head_dim, has_pred);
   if (workspace == nullptr || workspace_bytes < ws.total) return AQUAKV_ERR_WORKSPACE;
   if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
+  if (ws.fused) {
+    // Algorithm 3 and the attention read of Algorithm 4 in ONE launch: the attention warps of the layer
+    // kernel consume every token block's decoded rows from L2 as soon as they exist
+    if (int64_t(batch) * ctx_len > (int64_t(1) << 30)) return AQUAKV_ERR_UNSUPPORTED;
+    uint8_t* wsb = ws_base(workspace);
+    LayerAttnArgs at;
+    at.q = q;
+    at.ctx = int(ctx_len);
+    at.n_q_heads = n_q_heads;
+    at.n_kv_heads = n_kv_heads;
+    at.n_splits = ws.n_splits;
+    at.scale_log2 = softmax_scale * 1.4426950408889634f;
+    at.part_ml = reinterpret_cast<float*>(wsb + ws.ml_off);
+    at.part_o = reinterpret_cast<float*>(wsb + ws.o_off);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    rc = launch_layer(c, st, false, int64_t(batch) * ctx_len, nullptr, nullptr, 0, Khat_prev, Vhat_prev, ld_prev, Wk, Wv,
+                      bk, bv, const_cast<uint8_t*>(Kcodes), const_cast<uint16_t*>(Kscales),
+                      const_cast<uint8_t*>(Vcodes), const_cast<uint16_t*>(Vscales), Khat, Vhat, ld_hat,
+                      wsb + ws.layer_off, &at);
+    if (rc) return rc;
+    AttnCombineArgs ca;
+    ca.part_ml = at.part_ml;
+    ca.part_o = at.part_o;
+    ca.out = static_cast<uint16_t*>(out);
+    ca.lse = lse;
+    ca.n_q_heads = n_q_heads;
+    ca.n_splits = ws.n_splits;
+    ca.ctx = int(ctx_len);
+    ca.block_tokens = kAttnSubTokens;
+    return launch_attn_combine(c, st, ca, head_dim, batch);
+  }
 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   uint8_t* wsb = ws_base(workspace);
@@ -1129,6 +1215,8 @@ int aquakv_decode_attn(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_
   ca.lse = lse;
   ca.n_q_heads = n_q_heads;
   ca.n_splits = ws.n_splits;
+  ca.ctx = int(ctx_len);
+  ca.block_tokens = 0;
   return launch_attn_combine(c, st, ca, head_dim, batch);
 }
 

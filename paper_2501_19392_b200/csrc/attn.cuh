@@ -246,13 +246,145 @@ __global__ void __launch_bounds__(kAttnMmaThreads, 2) attn_partial_kernel(const 
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// The same product for ONE warp, at most 128 consecutive tokens of one sequence, one KV head and 64 of
+// its output dimensions: the attention role of the fused decode kernel (layer_kernel.cuh) calls it
+// on every token block as soon as the block's reconstructed rows exist, so the rows are read from L2
+// and never need to come back from DRAM.  With head_dim 128 two warps share a head: both form the
+// scores (the keys are read twice, from L2), each accumulates one half of the output dimensions, so a
+// warp holds 16 accumulator registers and can keep its loads one phase ahead within the fused
+// kernel's register budget: the values of a step are requested before its scores are formed, the
+// keys of the next step right after them.  16 tokens per step (two 8-token score tiles, one
+// 16-token k-step of the output product).  Rows are read with ld.global.cg: other SMs of the same
+// kernel have just written them.
+//   Krows: row r = token r of the segment, offset to the KV head's first dimension.
+//   Vrows: the same, offset to the first of this warp's 64 output dimensions.
+//   qrows: query head 0 of the KV group (gq heads, HD values each), re-read every step (L1 hits).
+//   ml_out[q][2] = (running maximum in log2 units, sum) or nullptr (the head's other warp writes it);
+//   o_out[q][HD]: unnormalised output, offset to this warp's first dimension.
+// ---------------------------------------------------------------------------------------------
+template <int HD, bool kBf16>
+__device__ __forceinline__ void attn_segment_warp(const uint16_t* __restrict__ Krows, const uint16_t* __restrict__ Vrows,
+                                                  long long ldK, long long ldV, int n_tok,
+                                                  const uint16_t* __restrict__ qrows, int gq, float scale_log2,
+                                                  float* __restrict__ ml_out, float* __restrict__ o_out, int lane) {
+  constexpr int NCH = HD / 32;
+  const int g = lane >> 2, j = lane & 3;
+  float m_run = kNegBig, l_run = 0.0f;
+  float o[8][2];
+#pragma unroll
+  for (int u = 0; u < 8; ++u) o[u][0] = o[u][1] = 0.0f;
+  float dz0 = 0.0f, dz1 = 0.0f;            // rows 8..15 of every product: stay zero
+  const uint32_t* qrow = reinterpret_cast<const uint32_t*>(qrows + (g < gq ? g : 0) * HD);
+  const bool q_on = g < gq;
+  uint4 kq[2][NCH];
+  auto load_keys = [&](int tb) {
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      const int tok = tb + 8 * t + g;
+      const uint16_t* kp = Krows + (long long)(tok < n_tok ? tok : 0) * ldK + j * 8;
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) kq[t][c] = __ldcg(reinterpret_cast<const uint4*>(kp + c * 32));
+    }
+  };
+  load_keys(0);
+#pragma unroll 1
+  for (int tb = 0; tb < n_tok; tb += 16) {
+    // ---- this step's values: requested now, used after the softmax -----------------------------------
+    uint4 w[4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int tok = tb + (r >> 1) * 8 + 2 * j + (r & 1);
+      w[r] = __ldcg(reinterpret_cast<const uint4*>(Vrows + (long long)(tok < n_tok ? tok : 0) * ldV + g * 8));
+    }
+    // ---- scores of 16 tokens ------------------------------------------------------------------------
+    float sc[2][2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      float s0 = 0.0f, s1 = 0.0f;
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) {
+        const uint4 qw = __ldg(reinterpret_cast<const uint4*>(qrow + (c * 32 + j * 8) / 2));
+        mma_16x8x16<kBf16>(s0, s1, dz0, dz1, q_on ? qw.x : 0u, 0u, q_on ? qw.y : 0u, 0u, kq[t][c].x, kq[t][c].y);
+        mma_16x8x16<kBf16>(s0, s1, dz0, dz1, q_on ? qw.z : 0u, 0u, q_on ? qw.w : 0u, 0u, kq[t][c].z, kq[t][c].w);
+      }
+      const int tok = tb + 8 * t + 2 * j;
+      sc[t][0] = tok < n_tok ? s0 * scale_log2 : kNegBig;
+      sc[t][1] = tok + 1 < n_tok ? s1 * scale_log2 : kNegBig;
+    }
+    if (tb + 16 < n_tok) load_keys(tb + 16);     // in flight during the softmax and the output product
+    // ---- online softmax of row g (4 tokens per lane, 4 lanes per row) -------------------------------
+    float mx = fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1]));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    const float m_new = fmaxf(m_run, mx);
+    const float corr = exp2f(m_run - m_new);
+    m_run = m_new;
+    uint32_t pa[2], pb[2];
+    float lsum = 0.0f;
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      const float p0 = sc[t][0] > 0.5f * kNegBig ? exp2f(sc[t][0] - m_new) : 0.0f;
+      const float p1 = sc[t][1] > 0.5f * kNegBig ? exp2f(sc[t][1] - m_new) : 0.0f;
+      pa[t] = store16x2<kBf16>(p0, p1);
+      if constexpr (kBf16) {     // two terms: 8 bits are too few for the output's tolerance
+        pb[t] = store16x2<kBf16>(p0 - load16<kBf16>(uint16_t(pa[t] & 0xffffu)),
+                                 p1 - load16<kBf16>(uint16_t(pa[t] >> 16)));
+        lsum += p0 + p1;
+      } else {
+        pb[t] = 0u;
+        lsum += load16<kBf16>(uint16_t(pa[t] & 0xffffu)) + load16<kBf16>(uint16_t(pa[t] >> 16));
+      }
+    }
+    l_run = fmaf(l_run, corr, lsum);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      o[u][0] *= corr;
+      o[u][1] *= corr;
+    }
+    // ---- output: O[g][dims] += P[g][tokens] * V[tokens][dims] ------------------------------------------
+    {
+      const uint32_t w0[4] = {w[0].x, w[0].y, w[0].z, w[0].w};
+      const uint32_t w1[4] = {w[1].x, w[1].y, w[1].z, w[1].w};
+      const uint32_t w2[4] = {w[2].x, w[2].y, w[2].z, w[2].w};
+      const uint32_t w3[4] = {w[3].x, w[3].y, w[3].z, w[3].w};
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;
+        const uint32_t b0 = __byte_perm(w0[e >> 1], w1[e >> 1], sel);
+        const uint32_t b1 = __byte_perm(w2[e >> 1], w3[e >> 1], sel);
+        mma_16x8x16<kBf16>(o[e][0], o[e][1], dz0, dz1, pa[0], 0u, pa[1], 0u, b0, b1);
+        if constexpr (kBf16)
+          mma_16x8x16<kBf16>(o[e][0], o[e][1], dz0, dz1, pb[0], 0u, pb[1], 0u, b0, b1);
+      }
+    }
+  }
+  l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+  l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+  if (g < gq) {
+    if (j == 0 && ml_out != nullptr) {
+      ml_out[g * 2] = m_run;
+      ml_out[g * 2 + 1] = l_run;
+    }
+    // column n of output tile u stands for dimension 8n + u of the warp's 64
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      o_out[g * HD + u + (2 * j) * 8] = o[u][0];
+      o_out[g * HD + u + (2 * j + 1) * 8] = o[u][1];
+    }
+  }
+}
+
 struct AttnCombineArgs {
   const float* part_ml;
   const float* part_o;
   uint16_t* out;      // [batch][n_q_heads][HD] 16-bit
   float* lse;         // [batch][n_q_heads] natural-log sum-exp, or nullptr
   int n_q_heads;
-  int n_splits;
+  int n_splits;       // slots per sequence in the partial arrays
+  int ctx;            // tokens per sequence
+  int block_tokens;   // > 0: partials per block of that many tokens of the FLATTENED token index (a sequence
+                      // uses as many slots as blocks overlap it); 0: every sequence uses all n_splits slots
 };
 
 // One CTA per (sequence, query head); thread i owns output dimension i.
@@ -260,15 +392,50 @@ template <int HD, bool kBf16>
 __global__ void __launch_bounds__(HD) attn_combine_kernel(const AttnCombineArgs a) {
   const int b = blockIdx.x / a.n_q_heads, qh = blockIdx.x % a.n_q_heads;
   const int i = threadIdx.x;
+  int n_s = a.n_splits;
+  if (a.block_tokens > 0) {
+    const long long t0 = (long long)b * a.ctx, t1 = t0 + a.ctx - 1;
+    n_s = int(t1 / a.block_tokens - t0 / a.block_tokens) + 1;
+  }
+  // Both passes keep several independent loads in flight: with many slots per sequence the kernel is
+  // bound by the latency of its loads, not by their number.
+  const float* ml = a.part_ml + ((long long)b * a.n_splits * a.n_q_heads + qh) * 2;
+  const float* po = a.part_o + ((long long)b * a.n_splits * a.n_q_heads + qh) * HD + i;
+  const long long ml_step = (long long)a.n_q_heads * 2, o_step = (long long)a.n_q_heads * HD;
   float M = kNegBig;
-  for (int s = 0; s < a.n_splits; ++s)
-    M = fmaxf(M, a.part_ml[(((long long)b * a.n_splits + s) * a.n_q_heads + qh) * 2]);
+  {
+    float m4[4] = {kNegBig, kNegBig, kNegBig, kNegBig};
+    int s = 0;
+    for (; s + 4 <= n_s; s += 4) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) m4[u] = fmaxf(m4[u], ml[(s + u) * ml_step]);
+    }
+    for (; s < n_s; ++s) m4[0] = fmaxf(m4[0], ml[s * ml_step]);
+    M = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+  }
   float L = 0.0f, o = 0.0f;
-  for (int s = 0; s < a.n_splits; ++s) {
-    const long long pidx = ((long long)b * a.n_splits + s) * a.n_q_heads + qh;
-    const float w = exp2f(a.part_ml[pidx * 2] - M);
-    L = fmaf(a.part_ml[pidx * 2 + 1], w, L);
-    o = fmaf(a.part_o[pidx * HD + i], w, o);
+  {
+    int s = 0;
+    for (; s + 4 <= n_s; s += 4) {
+      float mv[4], lv[4], ov[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        mv[u] = ml[(s + u) * ml_step];
+        lv[u] = ml[(s + u) * ml_step + 1];
+        ov[u] = po[(s + u) * o_step];
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {          // accumulated in slot order
+        const float w = exp2f(mv[u] - M);
+        L = fmaf(lv[u], w, L);
+        o = fmaf(ov[u], w, o);
+      }
+    }
+    for (; s < n_s; ++s) {
+      const float w = exp2f(ml[s * ml_step] - M);
+      L = fmaf(ml[s * ml_step + 1], w, L);
+      o = fmaf(po[s * o_step], w, o);
+    }
   }
   a.out[((long long)b * a.n_q_heads + qh) * HD + i] = store16<kBf16>(o / L);
   if (a.lse != nullptr && i == 0)

@@ -29,9 +29,15 @@
 // all its roles leave their loops.
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = tensor-memory owner + MMA issuer, warps 2..5 =
-// GEMM epilogue (tensor memory -> fp32 rows in the ring), warps 6.. = row warps.
+// GEMM epilogue (tensor memory -> fp32 rows in the ring), then the row warps and, in the decoder
+// instantiation that also attends (Algorithm 4 lines 5-9), four attention warps: as soon as the value
+// rows of the CTA's token block are reconstructed they read the block's keys and values back from
+// L2, form the single-query attention partials of the CTA's share of the KV heads for every sequence
+// the block overlaps, and release the block's rows (attn_done), so that decoded rows which the
+// caller does not ask for live only in a ring of three waves that never needs to reach DRAM.
 #pragma once
 
+#include "attn.cuh"
 #include "codec.cuh"
 #include "common.cuh"
 #include "gemm_pred.cuh"
@@ -48,14 +54,22 @@ constexpr int kPairStageBytes = kABytes + kPairBBytes;   // 32 KB
 // teams of d_kv/256 warps share a row (codec.cuh): 24 warps at 64 registers.
 constexpr int kWrEncodeWarps = 12;    // the encoder's search table leaves shared memory for 12 transposition buffers
 constexpr int kWrDecodeWarps = 12;    // 12 to 16 measured alike
-template <bool kEncode, int D, bool kFull>
+constexpr int kWrAttnDecodeWarps = 10; // beside four attention warps: 640 threads, which keeps the 96-register budget
+template <bool kEncode, int D, bool kFull, int kAttnHD = 0>
 struct LayerGeom {
   static constexpr bool WR = D == 1024 && kFull;
-  static constexpr int ROW_WARPS = WR ? (kEncode ? kWrEncodeWarps : kWrDecodeWarps) : 24;
+  static constexpr int ROW_WARPS =
+      WR ? (kEncode ? kWrEncodeWarps : (kAttnHD > 0 ? kWrAttnDecodeWarps : kWrDecodeWarps)) : 24;
   static constexpr int TEAM = WR ? 1 : RowTeam<D>::TEAM;
   static constexpr int TEAMS = ROW_WARPS / TEAM;          // rows a CTA works on at a time
   static constexpr int THREADS = 32 * (6 + ROW_WARPS);
 };
+constexpr int kAttnWarps = 4;
+constexpr int kAttnSubTokens = 128;  // tokens of a token block that one attention warp covers (one partial slot each)
+template <bool kEncode, int D, bool kFull, int kAttnHD>
+constexpr int layer_threads() {
+  return LayerGeom<kEncode, D, kFull, kAttnHD>::THREADS + (kAttnHD > 0 ? 32 * kAttnWarps : 0);
+}
 
 struct LayerSmemTail {
   uint64_t full[kLayerStages];
@@ -150,6 +164,16 @@ struct LayerArgs {
   SearchDev search;
   int log_h, log_g;
   int* status;
+  // single-query attention over the decoded rows (decoder instantiations with kAttnHD > 0)
+  int vhat_ring;            // like khat_ring, for V^ (both rings or neither)
+  const uint16_t* q;        // [batch][n_q_heads][head_dim]
+  int ctx;                  // tokens per sequence: token t belongs to sequence t / ctx
+  int n_q_heads, n_kv_heads;
+  int n_splits;             // partial slots per sequence: slot s of sequence b = sub-block (of kAttnSubTokens tokens) b*ctx/kAttnSubTokens + s
+  float scale_log2;         // softmax scale * log2(e)
+  float* part_ml;           // [batch][n_splits][n_q_heads][2]
+  float* part_o;            // [batch][n_splits][n_q_heads][head_dim]
+  int* attn_done;           // [n_waves][mw], zero at launch: attention warps that are done with the block
 };
 
 __device__ __forceinline__ void layer_job(int j, int n_waves, int& phase, int& wave) {
@@ -159,6 +183,9 @@ __device__ __forceinline__ void layer_job(int j, int n_waves, int& phase, int& w
   else { phase = 1; wave = (j >> 1) - 1; }
 }
 __device__ __forceinline__ int layer_key_job(int wave) { return wave == 0 ? 0 : 2 * wave - 1; }
+__device__ __forceinline__ int layer_value_job(int wave, int n_waves) {
+  return wave == n_waves - 1 ? 2 * n_waves - 1 : 2 * wave + 2;
+}
 
 // Row work of a wave is spread evenly over ALL CTAs: CTA slot s takes rows [s*rpc, (s+1)*rpc) of
 // the wave, rpc = the power of two >= rows / CTAs.  For a full wave this is rpc = 128 / NTN rows of
@@ -225,13 +252,14 @@ __device__ __forceinline__ void fence_proxy_async_all() {
 
 // kFull: the Hadamard block and the scale group both span the whole row (the paper's setting for
 // d_kv = 1024, Section 4.1); their logarithms are then compile-time constants of the row code.
-template <bool kEncode, int D, int NPTS, bool kBf16, bool kFull>
-__global__ void __launch_bounds__((LayerGeom<kEncode, D, kFull>::THREADS), 1)
+// kAttnHD: 0, or the head dimension (64 / 128) of the attention the decoder also computes.
+template <bool kEncode, int D, int NPTS, bool kBf16, bool kFull, int kAttnHD = 0>
+__global__ void __launch_bounds__((layer_threads<kEncode, D, kFull, kAttnHD>()), 1)
 layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant__ CUtensorMap tmVprev,
              const __grid_constant__ CUtensorMap tmKhat, const __grid_constant__ CUtensorMap tmWk,
              const __grid_constant__ CUtensorMap tmWv, const __grid_constant__ CUtensorMap tmP,
              const LayerArgs a) {
-  using G = LayerGeom<kEncode, D, kFull>;
+  using G = LayerGeom<kEncode, D, kFull, kAttnHD>;
   constexpr int NTN = D / kBN;             // feature tiles per token block = CTAs per token block
   constexpr int NKD = D / kBK;             // k-blocks per d_kv input features
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
@@ -473,7 +501,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         atomicAdd(a.gemm_done + j * a.mw + ml, 1);
       }
     }
-  } else {
+  } else if (warp < 6 + G::ROW_WARPS) {
     // ------------------------------- row warps (TEAM warps per row; TEAMS rows at a time) ------
     constexpr int TEAM = G::TEAM, TEAMS = G::TEAMS;
     const int rw = warp - 6;
@@ -522,7 +550,19 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         }
       }
       bool ok = true;
-      if (TEAM > 1) {
+      if constexpr (kAttnHD > 0) {
+        // the key rows of this wave reuse the ring rows of wave - ring depth: the attention warps must
+        // be done with them (they trail the rows by about one job, so this rarely waits)
+        if (ph == 0 && a.khat_ring > 0 && wave >= a.khat_ring) {
+          if (lane == 0)
+            ok = counter_wait_bounded(a.attn_done + (wave - a.khat_ring) * a.mw + rb, NTN * kAttnWarps, abort_flag,
+                                      a.status);
+          ok = __shfl_sync(0xffffffffu, ok, 0);
+        }
+      }
+      if (!ok) {
+        // fall through to the report below with the abort flag set
+      } else if (TEAM > 1) {
         // one thread polls for the team; all its warps must take the same path, so they agree
         // through the abort flag (set by a failed wait) between two barriers
         if (rck.member == 0 && lane == 0)
@@ -543,6 +583,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
           const float* pred_row = pbuf + size_t(r) * D;
           uint16_t* hat_row;
           if (ph == 0) hat_row = a.Khat + (khat_base + r) * a.ldKhat;
+          else if (a.vhat_ring) hat_row = a.Vhat + (khat_base + r) * a.ldVhat;     // same ring geometry as K^
           else hat_row = a.Vhat != nullptr ? a.Vhat + g * a.ldVhat : nullptr;
           uint8_t* codes_row = (ph == 0 ? a.Kcodes : a.Vcodes) + g * CODE_BYTES;
           uint16_t* scales_row = (ph == 0 ? a.Kscales : a.Vscales) + g * n_groups;
@@ -588,6 +629,59 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         __threadfence();
         fence_proxy_async_all();
         atomicAdd(a.rows_done + j * a.mw + rb, 1);
+      }
+    }
+  } else {
+    // ------------------------------- attention warps ------------------------------------------------
+    if constexpr (kAttnHD > 0) {
+      // A warp takes one KV head, 64 of its output dimensions (with head_dim 128 two warps share a head)
+      // and one sub-block of kAttnSubTokens tokens of the token block; every (sub-block, sequence) has
+      // its own partial slot.  (Eight warps on 64-token sub-blocks measured slower than four on whole
+      // blocks: the kernel then runs at 80 registers and the row warps spill.)
+      constexpr int WPH = kAttnHD / 64;                // warps per head and sub-block
+      constexpr int NSUB = kBM / kAttnSubTokens;       // sub-blocks of a token block
+      constexpr int HPAR = kAttnWarps / (WPH * NSUB);  // heads in flight per CTA
+      const int aw = warp - 6 - G::ROW_WARPS;
+      const int half = aw % WPH;
+      const int sub = (aw / WPH) % NSUB;
+      const int hpc = a.n_kv_heads / NTN;              // KV heads of a token block that this CTA attends over
+      const int rep = a.n_q_heads / a.n_kv_heads;
+      for (int wave = 0; wave < a.n_waves; ++wave) {
+        const WaveRows wr = wave_rows(wave, a.T, a.mw, gridDim.x);
+        if (ml >= wr.blocks) continue;                  // this CTA's block does not exist in the (last) wave
+        bool ok = true;
+        if (lane == 0)
+          ok = counter_wait_bounded(a.rows_done + layer_value_job(wave, a.n_waves) * a.mw + ml,
+                                    wave_block_teams(wr, ml, gridDim.x, G::TEAMS), abort_flag, a.status);
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        const long long blk = (long long)wave * a.mw + ml;       // token block of the call
+        const long long sblk = blk * NSUB + sub;                 // this warp's sub-block of the call
+        const long long tok0 = sblk * kAttnSubTokens;
+        const long long tok1 = tok0 + kAttnSubTokens < a.T ? tok0 + kAttnSubTokens : a.T;
+        const long long ring_row0 =
+            a.khat_ring ? ((long long)(wave % a.khat_ring) * a.mw + ml) * kBM + sub * kAttnSubTokens : tok0;
+        for (int h = n_blk * hpc + aw / (WPH * NSUB); h < (n_blk + 1) * hpc; h += HPAR) {
+          long long t = tok0;
+          while (t < tok1) {                            // one segment per sequence the sub-block overlaps
+            const long long b = t / a.ctx;
+            const long long seg_end = (b + 1) * a.ctx < tok1 ? (b + 1) * a.ctx : tok1;
+            const long long row = ring_row0 + (t - tok0);
+            const long long split = sblk - (b * a.ctx) / kAttnSubTokens;
+            const long long pidx = (b * a.n_splits + split) * a.n_q_heads + (long long)h * rep;
+            attn_segment_warp<kAttnHD, kBf16>(a.Khat + row * a.ldKhat + h * kAttnHD,
+                                              a.Vhat + row * a.ldVhat + h * kAttnHD + half * 64, a.ldKhat, a.ldVhat,
+                                              int(seg_end - t), a.q + (b * a.n_q_heads + (long long)h * rep) * kAttnHD,
+                                              rep, a.scale_log2, half == 0 ? a.part_ml + pidx * 2 : nullptr,
+                                              a.part_o + pidx * kAttnHD + half * 64, lane);
+            t = seg_end;
+          }
+        }
+        __syncwarp();
+        if (lane == 0) {
+          __threadfence();
+          atomicAdd(a.attn_done + wave * a.mw + ml, 1);
+        }
       }
     }
   }
