@@ -207,6 +207,51 @@ int aquakv_decode(aquakv_ctx* ctx, int64_t n_tokens,
                   void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Algorithm 4's loop over layers for SMALL calls -- a decode step of a batch of sequences, a short
+ * prompt -- in ONE launch: Algorithm 2 (encode_chain) or Algorithm 3 (decode_chain) for n_layers
+ * consecutive layers, each layer's predictors reading the previous layer's reconstruction (Algorithm
+ * 4 lines 4 and 14; Section 3.3).  A per-layer call of a few tokens is bound by launch and hand-off
+ * latency and by a handful of SMs streaming the adapter weights; here every SM streams a share of
+ * the weights, the key chain runs ahead of the value chain, and the layers hand over through
+ * counters in device memory.
+ *
+ * Per-layer arguments are HOST arrays of n_layers DEVICE pointers (read during the call only):
+ * K[l], V[l] (encode), Wk[l], Wv[l] (both NULL: layer l has no predictor, e.g. the model's first
+ * layer), bk[l], bv[l] (the arrays or single entries may be NULL), codes and scales, and the optional
+ * outputs Khat[l], Vhat[l] ([n_tokens, ld_hat]; arrays or entries NULL: that layer's reconstruction
+ * stays in the workspace; give both or neither of a layer).  If layer 0 has a predictor, Khat_init /
+ * Vhat_init ([n_tokens, ld_init]) are the reconstruction of the layer before it; otherwise they must
+ * be NULL.  n_tokens <= 2048 and n_layers <= 128 (AQUAKV_ERR_TOO_LARGE beyond: use the per-layer
+ * calls, which are built for large token counts).  d_kv = 1024 requires Hadamard block = scale group
+ * = 1024 (AQUAKV_ERR_UNSUPPORTED otherwise).  Workspace: aquakv_chain_workspace_bytes.
+ *
+ * Results satisfy the same bounds against the definition as the per-layer calls; the fp32 prediction
+ * is summed in a different order, so a reconstruction can differ from aquakv_encode / aquakv_decode in
+ * the last bit of the 16-bit type.  decode_chain reproduces encode_chain's reconstructions bit for bit.
+ * Calls on one context must not overlap on the device, and no other kernel may occupy the device's
+ * SMs while a chain call runs (its CTAs wait for one another; a wait that finds no partner expires
+ * after two seconds with AQUAKV_ERR_TIMEOUT in the status word).
+ */
+size_t aquakv_chain_workspace_bytes(const aquakv_ctx* ctx, int64_t n_tokens, int32_t n_layers);
+int aquakv_encode_chain(aquakv_ctx* ctx, int64_t n_tokens, int32_t n_layers,
+                        const void* const* K, const void* const* V, int64_t ld_kv,
+                        const void* Khat_init, const void* Vhat_init, int64_t ld_init,
+                        const void* const* Wk, const void* const* Wv,
+                        const float* const* bk, const float* const* bv,
+                        uint8_t* const* Kcodes, uint16_t* const* Kscales,
+                        uint8_t* const* Vcodes, uint16_t* const* Vscales,
+                        void* const* Khat, void* const* Vhat, int64_t ld_hat,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+int aquakv_decode_chain(aquakv_ctx* ctx, int64_t n_tokens, int32_t n_layers,
+                        const uint8_t* const* Kcodes, const uint16_t* const* Kscales,
+                        const uint8_t* const* Vcodes, const uint16_t* const* Vscales,
+                        const void* Khat_init, const void* Vhat_init, int64_t ld_init,
+                        const void* const* Wk, const void* const* Wv,
+                        const float* const* bk, const float* const* bv,
+                        void* const* Khat, void* const* Vhat, int64_t ld_hat,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * aquakv_decode for callers that cannot allocate device memory and therefore have no workspace to
  * hand over.  (The paper has no counterpart: this is a packaging variant of aquakv_decode, same
  * arithmetic, same kernels.)  Who needs it: a decode step running inside a region where
@@ -303,6 +348,7 @@ int64_t aquakv_launch_count(const aquakv_ctx* ctx);
 #define AQUAKV_KERNEL_DECODE_ROWS 2 /* unpack, gather, inverse rotation, add-back */
 #define AQUAKV_KERNEL_ATTN 3        /* split-KV attention partials and combine   */
 #define AQUAKV_KERNEL_LAYER 4       /* fused layer kernel: predictor GEMMs + row work */
+#define AQUAKV_KERNEL_CHAIN 5       /* all layers of a small call in one launch       */
 int aquakv_profile_enable(aquakv_ctx* ctx, int enable);
 int aquakv_profile_read(aquakv_ctx* ctx, int kernel_class, int64_t* launches, double* total_ms);
 

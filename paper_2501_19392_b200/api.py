@@ -22,7 +22,8 @@ OP_DECODE_ATTN = 2
 ROLE_KEY = 0
 ROLE_VALUE = 1
 NOALLOC_MAX_TOKENS = 1024
-KERNEL_PREDICT, KERNEL_ENCODE_ROWS, KERNEL_DECODE_ROWS, KERNEL_ATTN, KERNEL_LAYER = 0, 1, 2, 3, 4
+KERNEL_PREDICT, KERNEL_ENCODE_ROWS, KERNEL_DECODE_ROWS, KERNEL_ATTN, KERNEL_LAYER, KERNEL_CHAIN = 0, 1, 2, 3, 4, 5
+CHAIN_MAX_TOKENS, CHAIN_MAX_LAYERS = 2048, 128
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libaquakv.so")
@@ -32,6 +33,7 @@ SYMBOLS = [
     "aquakv_decode_attn_workspace_bytes", "aquakv_predict", "aquakv_encode", "aquakv_decode",
     "aquakv_decode_attn", "aquakv_decode_noalloc", "aquakv_encode_phase", "aquakv_decode_phase", "aquakv_poll_status", "aquakv_launch_count", "aquakv_status_string",
     "aquakv_profile_enable", "aquakv_profile_read", "aquakv_selftest_bounded_wait",
+    "aquakv_chain_workspace_bytes", "aquakv_encode_chain", "aquakv_decode_chain",
 ]
 
 
@@ -93,6 +95,13 @@ def _load():
     L.aquakv_profile_enable.argtypes = [vp, ctypes.c_int]
     L.aquakv_profile_read.restype = ctypes.c_int
     L.aquakv_profile_read.argtypes = [vp, ctypes.c_int, ctypes.POINTER(i64), ctypes.POINTER(ctypes.c_double)]
+    L.aquakv_chain_workspace_bytes.restype = sz
+    L.aquakv_chain_workspace_bytes.argtypes = [vp, i64, i32]
+    L.aquakv_encode_chain.restype = ctypes.c_int
+    L.aquakv_encode_chain.argtypes = [vp, i64, i32, vp, vp, i64, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64,
+                                      vp, sz, vp]
+    L.aquakv_decode_chain.restype = ctypes.c_int
+    L.aquakv_decode_chain.argtypes = [vp, i64, i32, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, i64, vp, sz, vp]
     L.aquakv_selftest_bounded_wait.restype = ctypes.c_int
     L.aquakv_selftest_bounded_wait.argtypes = [vp, i64, vp]
     L.aquakv_status_string.restype = ctypes.c_char_p
@@ -303,6 +312,45 @@ class Codec:
         if rc:
             raise AquaKVError(rc, "aquakv_decode_phase")
         return hat
+
+    # -- all layers of a small call in one launch ---------------------------------------------------
+    @staticmethod
+    def _ptr_array(tensors, n):
+        """Host array of n device pointers (None entries and a None list give NULL)."""
+        if tensors is None:
+            return None
+        assert len(tensors) == n
+        return (ctypes.c_void_p * n)(*[_ptr(t) for t in tensors])
+
+    def chain_workspace_bytes(self, n_tokens: int, n_layers: int) -> int:
+        return int(lib.aquakv_chain_workspace_bytes(self.h, n_tokens, n_layers))
+
+    def encode_chain(self, K, V, Wk, Wv, Kcodes, Kscales, Vcodes, Vscales, bk=None, bv=None, Khat=None, Vhat=None,
+                     Khat_init=None, Vhat_init=None, workspace=None):
+        """Lists with one entry per layer (Wk[l] = Wv[l] = None: no predictor for layer l)."""
+        L, T = len(K), int(K[0].shape[0])
+        ws = workspace if workspace is not None else self._workspace(self.chain_workspace_bytes(T, L), K[0].device)
+        arr = lambda ts: self._ptr_array(ts, L)
+        hats = [t for t in (Khat or []) if t is not None]
+        rc = lib.aquakv_encode_chain(self.h, T, L, arr(K), arr(V), _ld(K[0], self.d), _ptr(Khat_init), _ptr(Vhat_init),
+                                     _ld(Khat_init, self.d), arr(Wk), arr(Wv), arr(bk), arr(bv), arr(Kcodes),
+                                     arr(Kscales), arr(Vcodes), arr(Vscales), arr(Khat), arr(Vhat),
+                                     _ld(hats[0] if hats else None, self.d), _ptr(ws), ws.numel(), _stream())
+        if rc:
+            raise AquaKVError(rc, "aquakv_encode_chain")
+
+    def decode_chain(self, Kcodes, Kscales, Vcodes, Vscales, Wk, Wv, bk=None, bv=None, Khat=None, Vhat=None,
+                     Khat_init=None, Vhat_init=None, workspace=None):
+        L, T = len(Kcodes), int(Kcodes[0].shape[0])
+        ws = workspace if workspace is not None else self._workspace(self.chain_workspace_bytes(T, L), Kcodes[0].device)
+        arr = lambda ts: self._ptr_array(ts, L)
+        hats = [t for t in (Khat or []) if t is not None]
+        rc = lib.aquakv_decode_chain(self.h, T, L, arr(Kcodes), arr(Kscales), arr(Vcodes), arr(Vscales), _ptr(Khat_init),
+                                     _ptr(Vhat_init), _ld(Khat_init, self.d), arr(Wk), arr(Wv), arr(bk), arr(bv),
+                                     arr(Khat), arr(Vhat), _ld(hats[0] if hats else None, self.d), _ptr(ws), ws.numel(),
+                                     _stream())
+        if rc:
+            raise AquaKVError(rc, "aquakv_decode_chain")
 
     def poll_status(self) -> int:
         return int(lib.aquakv_poll_status(self.h, _stream()))

@@ -22,6 +22,7 @@
 
 #include "aquakv.h"
 #include "attn.cuh"
+#include "chain_kernel.cuh"
 #include "codec.cuh"
 #include "gemm_pred.cuh"
 #include "layer_kernel.cuh"
@@ -609,6 +610,152 @@ int launch_layer(aquakv_ctx* c, cudaStream_t st, bool encode, int64_t T, const v
   return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
 }
 
+// ---------------------------------------------------------------------------------------------
+// chain kernel (all layers of a small call in one persistent launch)
+// ---------------------------------------------------------------------------------------------
+constexpr int64_t kChainMaxTokens = 2048;
+
+struct ChainWs {
+  size_t pk_off, pv_off, cnt_off, cnt_bytes, hat_off, hat_bytes, total;
+};
+
+ChainWs chain_ws(const aquakv_ctx* c, int64_t T, int L) {
+  ChainWs w;
+  const size_t d = size_t(c->p.d_kv);
+  const size_t n_mt = size_t((T + kChainMT - 1) / kChainMT);
+  w.pk_off = 0;
+  w.pv_off = round_up(size_t(T) * d * sizeof(float), 256);
+  w.cnt_off = w.pv_off + round_up(size_t(T) * d * sizeof(float), 256);
+  w.cnt_bytes = size_t(4) * L * n_mt * sizeof(int);
+  w.hat_off = w.cnt_off + round_up(w.cnt_bytes, 256);
+  w.hat_bytes = round_up(size_t(T) * d * 2, 256);           // one layer's K^ or V^
+  w.total = w.hat_off + size_t(2) * L * w.hat_bytes + kWsSlack;
+  return w;
+}
+
+template <bool ENC, int D, int NPTS, bool BF>
+int launch_chain_t(int device, cudaStream_t st, int grid, const ChainArgs& a) {
+  static std::atomic<unsigned long long> attr_devices{0};
+  constexpr size_t smem = sizeof(ChainSmem<D, NPTS, ENC>);
+  const unsigned long long bit = 1ull << (device & 63);
+  if (device >= 64 || !(attr_devices.load(std::memory_order_acquire) & bit)) {
+    if (cudaFuncSetAttribute(chain_kernel<ENC, D, NPTS, BF>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) !=
+        cudaSuccess)
+      return AQUAKV_ERR_CUDA;
+    if (device < 64) attr_devices.fetch_or(bit, std::memory_order_release);
+  }
+  chain_kernel<ENC, D, NPTS, BF><<<grid, kChainThreads, smem, st>>>(a);
+  return AQUAKV_OK;
+}
+template <int D, int NPTS, bool BF>
+void launch_chain_dnb(int* rc, bool encode, int device, cudaStream_t st, int grid, const ChainArgs& a) {
+  *rc = encode ? launch_chain_t<true, D, NPTS, BF>(device, st, grid, a) : launch_chain_t<false, D, NPTS, BF>(device, st, grid, a);
+}
+
+// Algorithm 2 (encode) or Algorithm 3 for n_layers layers in one launch; argument checks included.
+int run_chain(aquakv_ctx* c, bool encode, int64_t T, int32_t L, const void* const* K, const void* const* V,
+              int64_t ld_kv, const void* Khat_init, const void* Vhat_init, int64_t ld_init, const void* const* Wk,
+              const void* const* Wv, const float* const* bk, const float* const* bv, uint8_t* const* Kcodes,
+              uint16_t* const* Kscales, uint8_t* const* Vcodes, uint16_t* const* Vscales, void* const* Khat,
+              void* const* Vhat, int64_t ld_hat, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (c == nullptr || T < 0 || L < 0) return AQUAKV_ERR_INVALID_ARG;
+  if (T == 0 || L == 0) return AQUAKV_OK;
+  if (T > kChainMaxTokens || L > kChainMaxLayers) return AQUAKV_ERR_TOO_LARGE;
+  const int d = c->p.d_kv;
+  if (d == 1024 && !(c->log_h == 10 && c->log_g == 10)) return AQUAKV_ERR_UNSUPPORTED;
+  if (Wk == nullptr || Wv == nullptr || Kcodes == nullptr || Kscales == nullptr || Vcodes == nullptr || Vscales == nullptr)
+    return AQUAKV_ERR_INVALID_ARG;
+  if (encode && (K == nullptr || V == nullptr)) return AQUAKV_ERR_INVALID_ARG;
+  int rc;
+  const ChainWs ws = chain_ws(c, T, L);
+  bool any_hat = false;
+  for (int l = 0; l < L; ++l) {
+    if ((rc = check_cache(Kcodes[l], Kscales[l], Vcodes[l], Vscales[l]))) return rc;
+    if (encode) {
+      if ((rc = check_rows(K[l], ld_kv, d, true))) return rc;
+      if ((rc = check_rows(V[l], ld_kv, d, true))) return rc;
+    }
+    if ((Wk[l] == nullptr) != (Wv[l] == nullptr)) return AQUAKV_ERR_INVALID_ARG;
+    if (Wk[l] != nullptr && (!aligned16(Wk[l]) || !aligned16(Wv[l]))) return AQUAKV_ERR_ALIGNMENT;
+    const float* b0 = bk ? bk[l] : nullptr;
+    const float* b1 = bv ? bv[l] : nullptr;
+    if (Wk[l] == nullptr && (b0 != nullptr || b1 != nullptr)) return AQUAKV_ERR_INVALID_ARG;
+    if ((b0 != nullptr && !aligned16(b0)) || (b1 != nullptr && !aligned16(b1))) return AQUAKV_ERR_ALIGNMENT;
+    const void* kh = Khat ? Khat[l] : nullptr;
+    const void* vh = Vhat ? Vhat[l] : nullptr;
+    if ((rc = check_rows(kh, ld_hat, d, false))) return rc;
+    if ((rc = check_rows(vh, ld_hat, d, false))) return rc;
+    if (kh != nullptr && (kh == vh || (encode && (kh == K[l] || kh == V[l])))) return AQUAKV_ERR_INVALID_ARG;
+    any_hat = any_hat || kh != nullptr || vh != nullptr;
+  }
+  if (Wk[0] != nullptr) {
+    if ((rc = check_rows(Khat_init, ld_init, d, true))) return rc;
+    if ((rc = check_rows(Vhat_init, ld_init, d, true))) return rc;
+  } else if (Khat_init != nullptr || Vhat_init != nullptr) {
+    return AQUAKV_ERR_INVALID_ARG;
+  }
+  if (workspace == nullptr || workspace_bytes < ws.total) return AQUAKV_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
+  (void)any_hat;
+
+  uint8_t* wsb = ws_base(workspace);
+  ChainArgs a;
+  std::memset(&a, 0, sizeof(a));
+  a.T = int(T);
+  a.L = L;
+  a.ldX = ld_kv;
+  a.Khat_init = static_cast<const uint16_t*>(Khat_init);
+  a.Vhat_init = static_cast<const uint16_t*>(Vhat_init);
+  a.ldInit = ld_init;
+  a.Pk = reinterpret_cast<float*>(wsb + ws.pk_off);
+  a.Pv = reinterpret_cast<float*>(wsb + ws.pv_off);
+  a.counters = reinterpret_cast<int*>(wsb + ws.cnt_off);
+  a.signmask_k = c->d_signmask[kRoleK];
+  a.signmask_v = c->d_signmask[kRoleV];
+  const CodecArgs ca = codec_args(c, kRoleK, 0);
+  a.grid4 = ca.grid4;
+  a.search = ca.search;
+  a.log_h = c->log_h;
+  a.log_g = c->log_g;
+  a.status = c->d_status;
+  for (int l = 0; l < L; ++l) {
+    ChainLayer& y = a.layer[l];
+    y.K = encode ? static_cast<const uint16_t*>(K[l]) : nullptr;
+    y.V = encode ? static_cast<const uint16_t*>(V[l]) : nullptr;
+    y.Wk = static_cast<const uint16_t*>(Wk[l]);
+    y.Wv = static_cast<const uint16_t*>(Wv[l]);
+    y.bk = bk ? bk[l] : nullptr;
+    y.bv = bv ? bv[l] : nullptr;
+    y.Kcodes = Kcodes[l];
+    y.Kscales = Kscales[l];
+    y.Vcodes = Vcodes[l];
+    y.Vscales = Vscales[l];
+    void* kh = Khat ? Khat[l] : nullptr;
+    void* vh = Vhat ? Vhat[l] : nullptr;
+    // the K and V reconstructions of a layer share ld: both the caller's or both the workspace's
+    if ((kh == nullptr) != (vh == nullptr)) return AQUAKV_ERR_INVALID_ARG;
+    if (kh != nullptr) {
+      y.Khat = static_cast<uint16_t*>(kh);
+      y.Vhat = static_cast<uint16_t*>(vh);
+      y.ldHat = ld_hat;
+    } else {
+      y.Khat = reinterpret_cast<uint16_t*>(wsb + ws.hat_off + size_t(2 * l) * ws.hat_bytes);
+      y.Vhat = reinterpret_cast<uint16_t*>(wsb + ws.hat_off + size_t(2 * l + 1) * ws.hat_bytes);
+      y.ldHat = d;
+    }
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(a.counters, 0, ws.cnt_bytes, st) != cudaSuccess) return AQUAKV_ERR_CUDA;
+  const int grid = c->sm_count;
+  a.n_ctas_k = grid * 2 / 5 > 0 ? grid * 2 / 5 : 1;
+  if (grid < 2) return AQUAKV_ERR_UNSUPPORTED;
+  ProfScope prof(c, st, AQUAKV_KERNEL_CHAIN);
+  AQ_DISPATCH_DNB(launch_chain_dnb, &rc, encode, c->device, st, grid, a);
+  if (rc) return rc;
+  ++c->launches;
+  return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
+}
+
 }  // namespace
 
 // =============================================================================================
@@ -1025,6 +1172,32 @@ int aquakv_decode(aquakv_ctx* c, int64_t n_tokens, const uint8_t* Kcodes, const 
     if (rc) return rc;
   }
   return AQUAKV_OK;
+}
+
+size_t aquakv_chain_workspace_bytes(const aquakv_ctx* c, int64_t n_tokens, int32_t n_layers) {
+  if (c == nullptr || n_tokens <= 0 || n_layers <= 0 || n_tokens > kChainMaxTokens || n_layers > kChainMaxLayers) return 0;
+  return chain_ws(c, n_tokens, n_layers).total;
+}
+
+int aquakv_encode_chain(aquakv_ctx* c, int64_t n_tokens, int32_t n_layers, const void* const* K, const void* const* V,
+                        int64_t ld_kv, const void* Khat_init, const void* Vhat_init, int64_t ld_init,
+                        const void* const* Wk, const void* const* Wv, const float* const* bk, const float* const* bv,
+                        uint8_t* const* Kcodes, uint16_t* const* Kscales, uint8_t* const* Vcodes,
+                        uint16_t* const* Vscales, void* const* Khat, void* const* Vhat, int64_t ld_hat, void* workspace,
+                        size_t workspace_bytes, void* cuda_stream) {
+  return run_chain(c, true, n_tokens, n_layers, K, V, ld_kv, Khat_init, Vhat_init, ld_init, Wk, Wv, bk, bv, Kcodes, Kscales,
+                   Vcodes, Vscales, Khat, Vhat, ld_hat, workspace, workspace_bytes, cuda_stream);
+}
+
+int aquakv_decode_chain(aquakv_ctx* c, int64_t n_tokens, int32_t n_layers, const uint8_t* const* Kcodes,
+                        const uint16_t* const* Kscales, const uint8_t* const* Vcodes, const uint16_t* const* Vscales,
+                        const void* Khat_init, const void* Vhat_init, int64_t ld_init, const void* const* Wk,
+                        const void* const* Wv, const float* const* bk, const float* const* bv, void* const* Khat,
+                        void* const* Vhat, int64_t ld_hat, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return run_chain(c, false, n_tokens, n_layers, nullptr, nullptr, 0, Khat_init, Vhat_init, ld_init, Wk, Wv, bk, bv,
+                   const_cast<uint8_t* const*>(Kcodes), const_cast<uint16_t* const*>(Kscales),
+                   const_cast<uint8_t* const*>(Vcodes), const_cast<uint16_t* const*>(Vscales), Khat, Vhat, ld_hat, workspace,
+                   workspace_bytes, cuda_stream);
 }
 
 // ---------------------------------------------------------------------------------------------
