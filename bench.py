@@ -296,6 +296,20 @@ def ops_by_config(api, chain, peaks, dev, reps=5):
                                        bufs.K[cur], bufs.V[cur])
             ms = _time_calls(one, reps * 4)
             out.append(_shape_entry(peaks, shape, "decode", T, ms, _shape_bytes(shape, T, False), config=cfg))
+        # the same layers through the chain entry points (all layers in one launch)
+        mk = lambda cols, dt: [torch.empty((T, cols), dtype=dt, device=dev) for _ in range(layers)]
+        Kc, Ks = mk(codec.code_bytes, torch.uint8), mk(codec.n_groups, torch.float16)
+        Vc, Vs = mk(codec.code_bytes, torch.uint8), mk(codec.n_groups, torch.float16)
+        Kh, Vh = mk(shape.d_kv, codec.torch_dtype), mk(shape.d_kv, codec.torch_dtype)
+        ms = _time_calls(lambda: codec.encode_chain(kv.K, kv.V, ad.Wk, ad.Wv, Kc, Ks, Vc, Vs), reps * 4)
+        out.append(_shape_entry(peaks, shape, "encode_chain", T, ms / layers, _shape_bytes(shape, T, True),
+                                config=cfg, ms_chain=ms, chain_layers=layers,
+                                note="aquakv_encode_chain: all layers in one launch; per layer = launch time / layers"))
+        if want_decode:
+            ms = _time_calls(lambda: codec.decode_chain(Kc, Ks, Vc, Vs, ad.Wk, ad.Wv, Khat=Kh, Vhat=Vh), reps * 4)
+            out.append(_shape_entry(peaks, shape, "decode_chain", T, ms / layers, _shape_bytes(shape, T, False),
+                                    config=cfg, ms_chain=ms, chain_layers=layers,
+                                    note="aquakv_decode_chain: all layers in one launch; per layer = launch time / layers"))
         assert codec.poll_status() == 0
 
     # config 1: two layers, encode + decode round trip
@@ -432,7 +446,7 @@ def main():
     enc_ms = sum(a.elapsed_time(b) for a, b, _ in mids) / args.steps
     dec_ms = sum(b.elapsed_time(c) for _, b, c in mids) / args.steps
     prof = {name: codec.profile_read(k) for name, k in
-            (("layer_fused", api.KERNEL_LAYER), ("predict_gemm", api.KERNEL_PREDICT),
+            (("layer_fused", api.KERNEL_LAYER), ("chain", api.KERNEL_CHAIN), ("predict_gemm", api.KERNEL_PREDICT),
              ("encode_rows", api.KERNEL_ENCODE_ROWS), ("decode_rows", api.KERNEL_DECODE_ROWS),
              ("attention", api.KERNEL_ATTN))}
     codec.profile_enable(False)

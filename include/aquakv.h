@@ -39,6 +39,12 @@
  *   - Non-finite inputs are memory-safe; the resulting codes/scales are unspecified.
  *   - A context may be used from one host thread at a time, on the device that was current
  *     when it was created.
+ *   - The layer calls with predictors (encode, decode, decode_attn) and the chain calls run
+ *     persistent kernels whose CTAs wait for one another and therefore must all be resident: do
+ *     not let them overlap other kernels on the same device (other streams, other contexts).  If
+ *     the grid cannot fit an idle device the call returns AQUAKV_ERR_UNSUPPORTED; if it is
+ *     crowded out at run time, its waits expire after two seconds and the call's outputs are
+ *     invalid, which only aquakv_poll_status reports (AQUAKV_ERR_TIMEOUT).
  */
 #ifndef AQUAKV_H_
 #define AQUAKV_H_

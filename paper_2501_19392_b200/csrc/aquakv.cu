@@ -470,6 +470,16 @@ int launch_layer_t(int device, cudaStream_t st, int grid, const CUtensorMap* tm,
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  // The CTAs of this kernel wait for one another, so all CTA pairs of the grid must fit the device at
+  // once (asked once per device and instantiation; an idle device is assumed, see the header).
+  static std::atomic<unsigned long long> fits_devices{0};
+  if (device >= 64 || !(fits_devices.load(std::memory_order_acquire) & bit)) {
+    int max_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&max_clusters, layer_kernel<ENC, D, NPTS, BF, FULL, AHD>, &cfg) != cudaSuccess)
+      return AQUAKV_ERR_CUDA;
+    if (max_clusters * 2 < grid) return AQUAKV_ERR_UNSUPPORTED;
+    if (device < 64) fits_devices.fetch_or(bit, std::memory_order_release);
+  }
   return cudaLaunchKernelEx(&cfg, layer_kernel<ENC, D, NPTS, BF, FULL, AHD>, tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], a) ==
                  cudaSuccess
              ? AQUAKV_OK
@@ -643,6 +653,16 @@ int launch_chain_t(int device, cudaStream_t st, int grid, const ChainArgs& a) {
         cudaSuccess)
       return AQUAKV_ERR_CUDA;
     if (device < 64) attr_devices.fetch_or(bit, std::memory_order_release);
+  }
+  // all CTAs wait for one another: one per SM must fit (asked once per device and instantiation)
+  static std::atomic<unsigned long long> fits_devices{0};
+  if (device >= 64 || !(fits_devices.load(std::memory_order_acquire) & bit)) {
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, chain_kernel<ENC, D, NPTS, BF>, kChainThreads, smem) !=
+        cudaSuccess)
+      return AQUAKV_ERR_CUDA;
+    if (per_sm < 1) return AQUAKV_ERR_UNSUPPORTED;
+    if (device < 64) fits_devices.fetch_or(bit, std::memory_order_release);
   }
   chain_kernel<ENC, D, NPTS, BF><<<grid, kChainThreads, smem, st>>>(a);
   return AQUAKV_OK;
