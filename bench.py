@@ -41,8 +41,8 @@ sys.path.insert(0, ROOT)
 from paper_2501_19392_b200 import synth  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per layer_kernel launch (32768 tokens, d_kv 1024, n 16):
-# mean of the encode (456 MB) and decode (281 MB) launches of profiles/layer_kernel_3layer_32768tok.md
-LAYER_KERNEL_DRAM_BYTES_PER_LAUNCH = 368.5e6
+# mean of the encode (438 MB) and decode + attention (390 MB) launches of profiles/layer_kernel_3layer_32768tok.md
+LAYER_KERNEL_DRAM_BYTES_PER_LAUNCH = 414.0e6
 
 METRIC = "KV tokens/s per layer (encode + decode-attention round trip) at 2 bits/value"
 UNIT = "token-layers/s"
@@ -502,7 +502,7 @@ def main():
                 "peak": peaks["tf_sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["tf_sustained"],
                 "frac_burst": achieved / peaks["tf_burst"], "peak_burst": peaks["tf_burst"],
                 "traffic": LAYER_KERNEL_DRAM_BYTES_PER_LAUNCH if (T, d, shape.grid_size) == (32768, 1024, 16) else None,
-                "traffic_unit": "bytes per launch (ncu dram read+write, mean of the encode and decode launches)",
+                "traffic_unit": "bytes per launch (ncu dram read+write, mean of the encode and decode + attention launches)",
                 "algorithmic_bytes_per_launch": 0.5 * (enc_bytes + dec_bytes) * T,
                 "peak_source": peaks["source"] + " (sustained)", "dominant_by_time": dominant,
                 "launches": n_l, "avg_launch_ms": ms_l / max(1, n_l)}
