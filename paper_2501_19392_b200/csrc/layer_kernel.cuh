@@ -45,16 +45,30 @@
 
 namespace aquakv {
 
-constexpr int kLayerStages = 4;
+// Operand stages of 32 KB per CTA: four, except three for the encoder with one warp per row (kWarpRows),
+// whose row work is the longer side and whose shared memory is better spent on more row warps
+// (measured: 3 and 4 stages alike).
+constexpr int kLayerStagesMax = 4;
+template <bool kEncode, bool kWarpRows> constexpr int kLayerStagesT = (kEncode && kWarpRows) ? 3 : 4;
 constexpr int kPairBBytes = (kBN / 2) * kBK * 2;        // this CTA's half of a weight tile k-block
 constexpr int kPairStageBytes = kABytes + kPairBBytes;   // 32 KB
 
 // Row warps of a CTA.  With d_kv = 1024 and the Hadamard block and scale group spanning the whole row
-// (kFull) a single warp owns a row (rowwarp.cuh): 12 such warps at 96 registers; otherwise
-// teams of d_kv/256 warps share a row (codec.cuh): 24 warps at 64 registers.
-constexpr int kWrEncodeWarps = 12;    // the encoder's search table leaves shared memory for 12 transposition buffers
-constexpr int kWrDecodeWarps = 12;    // 12 to 16 measured alike
-constexpr int kWrAttnDecodeWarps = 10; // beside four attention warps: 640 threads, which keeps the 96-register budget
+// (kFull) a single warp owns a row (rowwarp.cuh); otherwise teams of d_kv/256 warps share a row
+// (codec.cuh): 24 warps at 64 registers.  The register file is split over the SM's four schedulers, so
+// the budget per thread follows from the warps per scheduler: 4 -> 128, 5 -> 96, 6 -> 80 registers.
+//   encoder: its row work is the longer side of the kernel and gains from every resident warp, even at
+//            80 registers (12 / 14 / 16 / 18-20 row warps measured: 1.51 / 1.48 / 1.38 / 1.46-1.48 ms per
+//            131072 tokens);
+//   decoder: the GEMM is the longer side; 10 row warps keep the CTA at 16 warps and 128 registers, which
+//            lets a row issue its prediction loads before the look-ups and the rotation (8 / 10 / 12 row
+//            warps: 0.836 / 0.801-0.809 / 0.835 ms per 131072 tokens).
+constexpr int kWrEncodeWarps = 16;
+constexpr int kWrDecodeWarps = 10;
+constexpr int kWrAttnDecodeWarps = 6;  // beside four attention warps: again 16 warps and 128 registers, which the
+                                       // attention warps need as much as the row warps (4 / 5 / 6 / 7 / 10 row warps:
+                                       // 2.19 / 2.07 / 2.07 / 2.35 / 2.22 ms per 8 x 32768 tokens)
+static_assert(kWrAttnDecodeWarps <= kWrDecodeWarps, "the decoder's shared memory is sized for kWrDecodeWarps row warps");
 template <bool kEncode, int D, bool kFull, int kAttnHD = 0>
 struct LayerGeom {
   static constexpr bool WR = D == 1024 && kFull;
@@ -63,6 +77,9 @@ struct LayerGeom {
   static constexpr int TEAM = WR ? 1 : RowTeam<D>::TEAM;
   static constexpr int TEAMS = ROW_WARPS / TEAM;          // rows a CTA works on at a time
   static constexpr int THREADS = 32 * (6 + ROW_WARPS);
+  // With at most 16 warps per CTA (four per scheduler) a thread may use 128 registers: the row
+  // routines then load ahead (next row's input, the prediction before the rotation).
+  static constexpr bool AHEAD = WR && 6 + ROW_WARPS + (kAttnHD > 0 ? 4 : 0) <= 16;
 };
 constexpr int kAttnWarps = 4;
 constexpr int kAttnSubTokens = 128;  // tokens of a token block that one attention warp covers (one partial slot each)
@@ -72,8 +89,8 @@ constexpr int layer_threads() {
 }
 
 struct LayerSmemTail {
-  uint64_t full[kLayerStages];
-  uint64_t empty[kLayerStages];
+  uint64_t full[kLayerStagesMax];
+  uint64_t empty[kLayerStagesMax];
   uint64_t acc_full[kAccStages];
   uint64_t acc_empty[kAccStages];
   uint32_t tmem_base;
@@ -98,16 +115,20 @@ struct LayerRowSmem {
 };
 
 // The GEMM epilogue stages each 32-row x 32-column fp32 piece of a tile in shared memory (128-byte
-// swizzle) and hands it to a TMA store: two 4 KB buffers per epilogue warp, or one for the encoder
-// with the 256-point grid, whose 2 KB grid would otherwise not fit (its row work is so much longer
-// than its GEMM that the epilogue's overlap does not matter).
+// swizzle) and hands it to a TMA store.  With one warp per row: one 4 KB buffer per epilogue warp
+// (two measured 2-3 % slower in the decoder and no faster in the encoder, where the space goes to
+// the row warps).  With row teams: two, which the short calls of that path gain from, or one for the
+// encoder with the 256-point grid, whose 2 KB grid would otherwise not fit.
 constexpr int kEpiPieceBytes = 32 * 32 * 4;
-template <bool kEncode, int NPTS> constexpr int kEpiBufs = (kEncode && NPTS > 64) ? 1 : 2;
-template <bool kEncode, int NPTS> constexpr int kEpiBytes = 4 * kEpiBufs<kEncode, NPTS> * kEpiPieceBytes;
+template <bool kEncode, int NPTS, bool kWarpRows>
+constexpr int kEpiBufs = (kWarpRows || (kEncode && NPTS > 64)) ? 1 : 2;
+template <bool kEncode, int NPTS, bool kWarpRows>
+constexpr int kEpiBytes = 4 * kEpiBufs<kEncode, NPTS, kWarpRows> * kEpiPieceBytes;
 
 template <bool kEncode, int D, int NPTS, bool kFull>
 constexpr size_t layer_smem_bytes() {
-  return 1024 + size_t(kLayerStages) * kPairStageBytes + kEpiBytes<kEncode, NPTS> + sizeof(LayerSmemTail) + 16 +
+  constexpr bool WR = LayerGeom<kEncode, D, kFull>::WR;
+  return 1024 + size_t(kLayerStagesT<kEncode, WR>) * kPairStageBytes + kEpiBytes<kEncode, NPTS, WR> + sizeof(LayerSmemTail) + 16 +
          sizeof(LayerRowSmem<kEncode, D, NPTS, kFull>);
 }
 
@@ -246,6 +267,7 @@ __device__ __forceinline__ bool counter_wait_bounded(const int* ctr, int target,
 __device__ __forceinline__ void named_barrier(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
+__device__ __forceinline__ void fence_acq_rel_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_all() {
   asm volatile("fence.proxy.async;" ::: "memory");
 }
@@ -267,8 +289,8 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~uintptr_t(1023));
-  uint8_t* epi_smem = smem + size_t(kLayerStages) * kPairStageBytes;      // 1024-byte aligned
-  LayerSmemTail* tail = reinterpret_cast<LayerSmemTail*>(epi_smem + kEpiBytes<kEncode, NPTS>);
+  uint8_t* epi_smem = smem + size_t(kLayerStagesT<kEncode, G::WR>) * kPairStageBytes;      // 1024-byte aligned
+  LayerSmemTail* tail = reinterpret_cast<LayerSmemTail*>(epi_smem + kEpiBytes<kEncode, NPTS, G::WR>);
   LayerRowSmem<kEncode, D, NPTS, kFull>* rsm = reinterpret_cast<LayerRowSmem<kEncode, D, NPTS, kFull>*>(
       (reinterpret_cast<uintptr_t>(tail) + sizeof(LayerSmemTail) + 15) & ~uintptr_t(15));
 
@@ -282,7 +304,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
   const int n_jobs = 2 * a.n_waves;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kLayerStages; ++s) {
+    for (int s = 0; s < kLayerStagesT<kEncode, G::WR>; ++s) {
       mbar_init(&tail->full[s], 1);
       mbar_init(&tail->empty[s], 1);
     }
@@ -366,16 +388,16 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
             tma_load_2d_pair_hint(b_dst, &tmWv, &tail->full[stage], kb * kBK, w_row, pol_keep);
           }
           ++issued;
-          if (++stage == kLayerStages) { stage = 0; phase_bit ^= 1u; }
+          if (++stage == kLayerStagesT<kEncode, G::WR>) { stage = 0; phase_bit ^= 1u; }
         }
       }
       if (!ok && rank == 0) {
         // let the copies in flight land before the shared memory is released
         int s = stage;
         uint32_t pb = phase_bit;
-        const int pending = issued < kLayerStages ? issued : kLayerStages;
+        const int pending = issued < kLayerStagesT<kEncode, G::WR> ? issued : kLayerStagesT<kEncode, G::WR>;
         for (int i = 0; i < pending; ++i) {
-          if (s == 0) { s = kLayerStages; pb ^= 1u; }
+          if (s == 0) { s = kLayerStagesT<kEncode, G::WR>; pb ^= 1u; }
           --s;
           const unsigned long long t0 = global_timer_ns();
           while (!mbar_try_wait(&tail->full[s], pb) && global_timer_ns() - t0 < kWaitLimitNs) {
@@ -417,7 +439,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
             umma_f16_pair(tmem_d, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
           }
           umma_commit_pair(&tail->empty[stage]);   // frees the stage in both CTAs
-          if (++stage == kLayerStages) { stage = 0; phase_bit ^= 1u; }
+          if (++stage == kLayerStagesT<kEncode, G::WR>) { stage = 0; phase_bit ^= 1u; }
         }
         if (ok) umma_commit_pair(&tail->acc_full[acc]);
       }
@@ -452,7 +474,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         // ring row of this warp's 32 tokens; rows past the last token are written too (never read)
         const int ring_row = (j % a.nb) * a.mw * kBM + ml * kBM + quarter * 32;
         const float* bias = ph == 0 ? a.bk : a.bv;
-        constexpr int EB = kEpiBufs<kEncode, NPTS>;
+        constexpr int EB = kEpiBufs<kEncode, NPTS, G::WR>;
         const uint64_t pol_keep = l2_policy_evict_last();
         uint8_t* my_epi = epi_smem + (warp - 2) * EB * kEpiPieceBytes;
 #pragma unroll 1
@@ -578,6 +600,8 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         const float* pbuf = a.P + (size_t(j % a.nb) * a.mw * kBM + size_t(rb) * kBM) * D;
         const size_t khat_base = a.khat_ring ? size_t((wave % a.khat_ring) * a.mw + rb) * kBM
                                              : size_t(m) * kBM;
+        [[maybe_unused]] uint4 xraw[4];
+        [[maybe_unused]] bool first_row = true;
         for (int r = r_begin + (team + j) % TEAMS; r < r_end; r += TEAMS) {   // rotated per job for balance
           const long long g = (long long)m * kBM + r;
           const float* pred_row = pbuf + size_t(r) * D;
@@ -591,9 +615,18 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
             unsigned long long* xbuf = rsm->scratch.xbuf[rw];
             if constexpr (kEncode) {
               const uint16_t* x_row = (ph == 0 ? a.K : a.V) + g * a.ldX;
-              wr_encode_row<NPTS, kBf16>(wrc, &rsm->tables, xbuf, x_row, pred_row, codes_row, scales_row, hat_row);
+              if constexpr (G::AHEAD) {
+                if (first_row) wr_load_x_row(x_row, lane, xraw);
+                first_row = false;
+                const uint16_t* x_next = r + TEAMS < r_end ? x_row + TEAMS * a.ldX : nullptr;
+                wr_encode_row_x<NPTS, kBf16, true>(wrc, &rsm->tables, xbuf, xraw, x_next, pred_row, codes_row, scales_row,
+                                                   hat_row);
+              } else {
+                wr_encode_row<NPTS, kBf16>(wrc, &rsm->tables, xbuf, x_row, pred_row, codes_row, scales_row, hat_row);
+              }
             } else {
-              wr_decode_row<NPTS, kBf16>(wrc, rsm->tables.grid, xbuf, codes_row, scales_row, pred_row, hat_row);
+              wr_decode_row<NPTS, kBf16, false, G::AHEAD>(wrc, rsm->tables.grid, xbuf, codes_row, scales_row, pred_row,
+                                                          hat_row);
             }
           } else {
             TeamSmem<D>* ts = &rsm->scratch.team[team];
@@ -626,8 +659,17 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       if (TEAM > 1) team_barrier<D>(rck.barrier); else __syncwarp();
       if (*abort_flag) break;
       if (rck.member == 0 && lane == 0) {   // one releasing thread per team (see the epilogue)
-        __threadfence();
-        fence_proxy_async_all();
+        // Key rows are read back by other CTAs' TMA loads (value-phase GEMM) and, like the value rows,
+        // by other CTAs' attention warps: those need the stores released, the TMA also across the
+        // proxies.  Value rows without attention are read by nobody in this launch; the counter then
+        // only tells the epilogue that the ring slot's prediction has been read (the row's stores
+        // depend on those loads, so they have completed).
+        if (ph == 0) {
+          fence_acq_rel_gpu();
+          fence_proxy_async_all();
+        } else if (kAttnHD > 0) {
+          fence_acq_rel_gpu();
+        }
         atomicAdd(a.rows_done + j * a.mw + rb, 1);
       }
     }

@@ -139,13 +139,27 @@ __device__ __forceinline__ int wr_code_chunk(int lane) {
   return (lane >> 4) + 2 * ((lane >> 2) & 1) + 4 * ((lane >> 3) & 1);
 }
 
+// The lane's 32 fp32 prediction values in the load layout (pair 4c + i = elements 256c + 8 lane + 2i, +1).
+// The loads are issued here and their values first used by wr_finish_row, so that the trip to L2
+// overlaps the rotation in between (32 registers: only where the register budget allows it).
+__device__ __forceinline__ void wr_load_pred_row(const float* __restrict__ pred_row, int lane, f32x2_t (&pr)[16]) {
+#pragma unroll
+  for (int ch = 0; ch < 4; ++ch) {
+    f32x2_t p[4];
+    wr_load_pred8(pred_row + ch * 256 + lane * 8, p);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) pr[4 * ch + i] = p[i];
+  }
+}
+
 // hat = round16(pred + c * sign * wp) for the lane's 32 values in the load layout; `wp` holds the
-// rotated-back grid points, c = scale / sqrt(1024).
+// rotated-back grid points, c = scale / sqrt(1024).  kEarly: the prediction was loaded into `pr`
+// before the rotation; otherwise it is read here, chunk by chunk.
 // kKeep stores the rows with the default policy instead of as streaming data (measured 2-4 % slower
 // even when the attention warps of the same kernel read them back, so nothing selects it).
-template <bool kBf16, bool kKeep = false>
+template <bool kBf16, bool kKeep = false, bool kEarly = false>
 __device__ __forceinline__ void wr_finish_row(const WarpRowCtx& rc, f32x2_t (&wp)[16], float c,
-                                              const float* __restrict__ pred_row,
+                                              const float* __restrict__ pred_row, const f32x2_t (&pr)[16],
                                               uint16_t* __restrict__ hat_row) {
   const int lane = rc.lane;
   const f32x2_t c2 = pack2(c, c);
@@ -155,10 +169,15 @@ __device__ __forceinline__ void wr_finish_row(const WarpRowCtx& rc, f32x2_t (&wp
 #pragma unroll
   for (int ch = 0; ch < 4; ++ch) {
     if (pred_row != nullptr) {
-      f32x2_t p[4];
-      wr_load_pred8(pred_row + ch * 256 + lane * 8, p);
+      if constexpr (kEarly) {
 #pragma unroll
-      for (int i = 0; i < 4; ++i) wp[4 * ch + i] = add2(p[i], wp[4 * ch + i]);
+        for (int i = 0; i < 4; ++i) wp[4 * ch + i] = add2(pr[4 * ch + i], wp[4 * ch + i]);
+      } else {
+        f32x2_t p[4];
+        wr_load_pred8(pred_row + ch * 256 + lane * 8, p);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) wp[4 * ch + i] = add2(p[i], wp[4 * ch + i]);
+      }
     } else {
       // adding the zero prediction turns a -0 (a zero value whose sign was flipped) into +0
 #pragma unroll
@@ -179,13 +198,23 @@ __device__ __forceinline__ void wr_finish_row(const WarpRowCtx& rc, f32x2_t (&wp
 // reconstruction) instead of being held in 32 registers across the rotation and the search; both
 // reads bypass L1 because another SM of the same kernel may have written it just before.  The
 // prediction rows must be 32-byte aligned.
-template <int NPTS, bool kBf16>
-__device__ __forceinline__ void wr_encode_row(const WarpRowCtx& rc, const RowSmem<NPTS>* __restrict__ rsm,
-                                              unsigned long long* xbuf, const uint16_t* __restrict__ x_row,
-                                              const float* __restrict__ pred_row,
-                                              uint8_t* __restrict__ codes_row,
-                                              uint16_t* __restrict__ scales_row,
-                                              uint16_t* __restrict__ hat_row) {
+// The lane's 32 input values of a row (16-bit, load layout) as loaded.
+__device__ __forceinline__ void wr_load_x_row(const uint16_t* __restrict__ x_row, int lane, uint4 (&xraw)[4]) {
+#pragma unroll
+  for (int ch = 0; ch < 4; ++ch) xraw[ch] = __ldcs(reinterpret_cast<const uint4*>(x_row + ch * 256 + lane * 8));   // read once
+}
+
+// kAhead (for callers with registers to spare): `xraw` holds this row's input on entry and, if x_next
+// is not null, the next row's on return (its loads are issued before the reconstruction so that they
+// overlap it), and the second prediction read is issued before the rotation back.
+template <int NPTS, bool kBf16, bool kAhead>
+__device__ __forceinline__ void wr_encode_row_x(const WarpRowCtx& rc, const RowSmem<NPTS>* __restrict__ rsm,
+                                                unsigned long long* xbuf, uint4 (&xraw)[4],
+                                                const uint16_t* __restrict__ x_next,
+                                                const float* __restrict__ pred_row,
+                                                uint8_t* __restrict__ codes_row,
+                                                uint16_t* __restrict__ scales_row,
+                                                uint16_t* __restrict__ hat_row) {
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
   constexpr int NW = 2 * BITS;               // 32-bit words of a 64-code chunk
   const int lane = rc.lane;
@@ -193,7 +222,7 @@ __device__ __forceinline__ void wr_encode_row(const WarpRowCtx& rc, const RowSme
   f32x2_t vp[16];
 #pragma unroll
   for (int ch = 0; ch < 4; ++ch) {
-    const uint4 raw = __ldcs(reinterpret_cast<const uint4*>(x_row + ch * 256 + lane * 8));   // read once
+    const uint4 raw = xraw[ch];
     vp[4 * ch + 0] = load16x2<kBf16>(raw.x);
     vp[4 * ch + 1] = load16x2<kBf16>(raw.y);
     vp[4 * ch + 2] = load16x2<kBf16>(raw.z);
@@ -302,15 +331,34 @@ __device__ __forceinline__ void wr_encode_row(const WarpRowCtx& rc, const RowSme
     }
   }
   // ---- reconstruction: hat = round16(pred + Q^-1(codes)) ---------------------------------------
-  if (hat_row != nullptr) {      // uniform over the warp
-    wr_rotate_back(vp, xbuf, lane);
-    wr_finish_row<kBf16>(rc, vp, sf * (1.0f / 32.0f), pred_row, hat_row);
+  if constexpr (kAhead) {
+    if (x_next != nullptr) wr_load_x_row(x_next, lane, xraw);
   }
+  if (hat_row != nullptr) {      // uniform over the warp
+    f32x2_t pr[16];
+    if constexpr (kAhead) {
+      if (pred_row != nullptr) wr_load_pred_row(pred_row, lane, pr);
+    }
+    wr_rotate_back(vp, xbuf, lane);
+    wr_finish_row<kBf16, false, kAhead>(rc, vp, sf * (1.0f / 32.0f), pred_row, pr, hat_row);
+  }
+}
+
+template <int NPTS, bool kBf16>
+__device__ __forceinline__ void wr_encode_row(const WarpRowCtx& rc, const RowSmem<NPTS>* __restrict__ rsm,
+                                              unsigned long long* xbuf, const uint16_t* __restrict__ x_row,
+                                              const float* __restrict__ pred_row,
+                                              uint8_t* __restrict__ codes_row,
+                                              uint16_t* __restrict__ scales_row,
+                                              uint16_t* __restrict__ hat_row) {
+  uint4 xraw[4];
+  wr_load_x_row(x_row, rc.lane, xraw);
+  wr_encode_row_x<NPTS, kBf16, false>(rc, rsm, xbuf, xraw, nullptr, pred_row, codes_row, scales_row, hat_row);
 }
 
 // One token row of Algorithm 3 line 5 / 7 given the prediction:
 //   hat = round16(pred + Q^-1(codes, scale)).
-template <int NPTS, bool kBf16, bool kKeep = false>
+template <int NPTS, bool kBf16, bool kKeep = false, bool kEarly = false>
 __device__ __forceinline__ void wr_decode_row(const WarpRowCtx& rc, const f32x2_t* __restrict__ grid_s,
                                               unsigned long long* xbuf,
                                               const uint8_t* __restrict__ codes_row,
@@ -320,6 +368,10 @@ __device__ __forceinline__ void wr_decode_row(const WarpRowCtx& rc, const f32x2_
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
   constexpr int NW = 2 * BITS;
   const int lane = rc.lane;
+  f32x2_t pr[16];
+  if constexpr (kEarly) {
+    if (pred_row != nullptr) wr_load_pred_row(pred_row, lane, pr);   // in flight during the look-ups and the rotation
+  }
   // the chunk of 64 codes this lane's group of four covers (each of the four lanes reads all of it)
   uint32_t W[NW];
   {
@@ -346,7 +398,7 @@ __device__ __forceinline__ void wr_decode_row(const WarpRowCtx& rc, const f32x2_
     wp[m] = grid_s[(W[pos >> 5] >> (pos & 31)) & uint32_t(NPTS - 1)];
   }
   wr_rotate_back(wp, xbuf, lane);
-  wr_finish_row<kBf16, kKeep>(rc, wp, sf * (1.0f / 32.0f), pred_row, hat_row);
+  wr_finish_row<kBf16, kKeep, kEarly>(rc, wp, sf * (1.0f / 32.0f), pred_row, pr, hat_row);
 }
 
 // ---------------------------------------------------------------------------------------------
