@@ -41,8 +41,8 @@ sys.path.insert(0, ROOT)
 from paper_2501_19392_b200 import synth  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per layer_kernel launch (32768 tokens, d_kv 1024, n 16):
-# mean of the encode (438 MB) and decode + attention (390 MB) launches of profiles/layer_kernel_3layer_32768tok.md
-LAYER_KERNEL_DRAM_BYTES_PER_LAUNCH = 414.0e6
+# mean of the encode (526 MB) and decode + attention (377 MB) launches of profiles/layer_kernel_3layer_32768tok.md
+LAYER_KERNEL_DRAM_BYTES_PER_LAUNCH = 451.5e6
 
 METRIC = "KV tokens/s per layer (encode + decode-attention round trip) at 2 bits/value"
 UNIT = "token-layers/s"

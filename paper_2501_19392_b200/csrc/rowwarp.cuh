@@ -191,19 +191,20 @@ __device__ __forceinline__ void wr_finish_row(const WarpRowCtx& rc, f32x2_t (&wp
   }
 }
 
-// One token row of Q and of the reconstruction (Algorithm 2 lines 6-7 / 9):
-//   codes, scale = Q(x - pred);  hat = round16(pred + Q^-1(codes, scale)).
-// Row pointers address the start of the row.  pred_row == nullptr: no predictor.  hat_row == nullptr:
-// reconstruction not wanted.  The prediction is read twice (for the residual and again for the
-// reconstruction) instead of being held in 32 registers across the rotation and the search; both
-// reads bypass L1 because another SM of the same kernel may have written it just before.  The
-// prediction rows must be 32-byte aligned.
 // The lane's 32 input values of a row (16-bit, load layout) as loaded.
 __device__ __forceinline__ void wr_load_x_row(const uint16_t* __restrict__ x_row, int lane, uint4 (&xraw)[4]) {
 #pragma unroll
   for (int ch = 0; ch < 4; ++ch) xraw[ch] = __ldcs(reinterpret_cast<const uint4*>(x_row + ch * 256 + lane * 8));   // read once
 }
 
+// One token row of Q and of the reconstruction (Algorithm 2 lines 6-7 / 9):
+//   codes, scale = Q(x - pred);  hat = round16(pred + Q^-1(codes, scale)).
+// Row pointers address the start of the row.  pred_row == nullptr: no predictor.  hat_row == nullptr:
+// reconstruction not wanted.  The prediction is read twice (for the residual and again for the
+// reconstruction) instead of being held in 32 registers across the rotation and the search (a copy in
+// the warp's shared memory measured 4 % slower than the second read: that pipe is the scarcer one); both
+// reads bypass L1 because another SM of the same kernel may have written it just before.  The
+// prediction rows must be 32-byte aligned.
 // kAhead (for callers with registers to spare): `xraw` holds this row's input on entry and, if x_next
 // is not null, the next row's on return (its loads are issued before the reconstruction so that they
 // overlap it), and the second prediction read is issued before the rotation back.
