@@ -67,6 +67,7 @@ extern "C" {
 #define AQUAKV_ERR_CUDA (-5)        /* a CUDA runtime/driver call failed                     */
 #define AQUAKV_ERR_TIMEOUT (-6)     /* a bounded device-side wait expired (see poll_status)  */
 #define AQUAKV_ERR_TOO_LARGE (-7)   /* more tokens than the fixed scratch of a *_noalloc call  */
+#define AQUAKV_ERR_NUMERIC (-8)     /* a fit's normal equations were not positive definite (poll_status) */
 
 #define AQUAKV_OP_ENCODE 0
 #define AQUAKV_OP_DECODE 1
@@ -320,6 +321,34 @@ int aquakv_decode_attn(aquakv_ctx* ctx, int32_t batch, int64_t ctx_len,
                        void* Khat, void* Vhat, int64_t ld_hat,
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Calibration of one predictor (Algorithm 1, the two arg-min lines; Section 3.2: linear regression
+ * with "closed-form training"; Appendix A: "closed form solution with regularizer rate 1e-3"):
+ *
+ *   W = argmin_W || [in0 ; in1] W^T (+ b) - target ||^2 + rate * trace(X^T X) / n_in * ||W||^2
+ *
+ * over n_tokens calibration tokens.  in0 / in1 (in1 may be NULL: one input tensor, the key predictor;
+ * two: the value predictor on [V_old ; K_rec]) and target are 16-bit device rows [n_tokens][ld],
+ * ld_in / ld_target >= d_kv and multiples of 8, pointers 16-byte aligned.  rate >= 0.  fit_bias != 0
+ * fits an intercept (inputs and targets centred; b = mean(target) - mean(X) W^T) into bias_out
+ * (fp32 [d_kv], device); otherwise bias_out is not touched and may be NULL.  W_out receives the
+ * matrix rounded once to the ctx's 16-bit type, laid out [d_kv][n_in * d_kv] like every adapter of this
+ * library; W32_out (may be NULL) the same matrix in fp32.  The normal equations are formed on the
+ * tensor cores with fp32 accumulation and solved by a Cholesky factorisation in double precision,
+ * all inside this library's kernels.  Algorithm 1's loop over layers (fit the key predictor, encode
+ * the keys, fit the value predictor on the reconstructed keys, encode the values, hand the
+ * reconstructions to the next layer) is made of this call and aquakv_encode_phase.
+ * Workspace: aquakv_fit_workspace_bytes(ctx, n_tokens, n_inputs) bytes of device memory, owned by the
+ * caller, not read after the call's kernels finish.  Asynchronous on cuda_stream.  Errors: the usual
+ * argument codes and nothing launched; a matrix that is not positive definite (possible only with
+ * rate == 0 and dependent inputs) is reported by aquakv_poll_status as AQUAKV_ERR_NUMERIC.
+ * d_kv must be a multiple of 256 (AQUAKV_ERR_UNSUPPORTED otherwise).                                */
+size_t aquakv_fit_workspace_bytes(const aquakv_ctx* ctx, int64_t n_tokens, int32_t n_inputs);
+int aquakv_fit_predictor(aquakv_ctx* ctx, int64_t n_tokens, const void* in0, const void* in1, int64_t ld_in,
+                         const void* target, int64_t ld_target, double rate, int fit_bias, void* W_out,
+                         float* W32_out, float* bias_out, void* workspace, size_t workspace_bytes,
+                         void* cuda_stream);
+
 /*
  * Synchronises `cuda_stream` and returns the context's device status word: AQUAKV_OK, or
  * AQUAKV_ERR_TIMEOUT if a bounded wait inside a kernel (on a TMA or tensor-core completion
@@ -355,6 +384,7 @@ int64_t aquakv_launch_count(const aquakv_ctx* ctx);
 #define AQUAKV_KERNEL_ATTN 3        /* split-KV attention partials and combine   */
 #define AQUAKV_KERNEL_LAYER 4       /* fused layer kernel: predictor GEMMs + row work */
 #define AQUAKV_KERNEL_CHAIN 5       /* all layers of a small call in one launch       */
+#define AQUAKV_KERNEL_FIT 6         /* calibration: transposes, normal equations, solve */
 int aquakv_profile_enable(aquakv_ctx* ctx, int enable);
 int aquakv_profile_read(aquakv_ctx* ctx, int kernel_class, int64_t* launches, double* total_ms);
 

@@ -23,6 +23,8 @@ ROLE_KEY = 0
 ROLE_VALUE = 1
 NOALLOC_MAX_TOKENS = 1024
 KERNEL_PREDICT, KERNEL_ENCODE_ROWS, KERNEL_DECODE_ROWS, KERNEL_ATTN, KERNEL_LAYER, KERNEL_CHAIN = 0, 1, 2, 3, 4, 5
+KERNEL_FIT = 6
+ERR_NUMERIC = -8
 CHAIN_MAX_TOKENS, CHAIN_MAX_LAYERS = 2048, 128
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -34,6 +36,7 @@ SYMBOLS = [
     "aquakv_decode_attn", "aquakv_decode_noalloc", "aquakv_encode_phase", "aquakv_decode_phase", "aquakv_poll_status", "aquakv_launch_count", "aquakv_status_string",
     "aquakv_profile_enable", "aquakv_profile_read", "aquakv_selftest_bounded_wait",
     "aquakv_chain_workspace_bytes", "aquakv_encode_chain", "aquakv_decode_chain",
+    "aquakv_fit_workspace_bytes", "aquakv_fit_predictor",
 ]
 
 
@@ -95,6 +98,11 @@ def _load():
     L.aquakv_profile_enable.argtypes = [vp, ctypes.c_int]
     L.aquakv_profile_read.restype = ctypes.c_int
     L.aquakv_profile_read.argtypes = [vp, ctypes.c_int, ctypes.POINTER(i64), ctypes.POINTER(ctypes.c_double)]
+    L.aquakv_fit_workspace_bytes.restype = sz
+    L.aquakv_fit_workspace_bytes.argtypes = [vp, i64, i32]
+    L.aquakv_fit_predictor.restype = ctypes.c_int
+    L.aquakv_fit_predictor.argtypes = [vp, i64, vp, vp, i64, vp, i64, ctypes.c_double, ctypes.c_int, vp, vp, vp,
+                                       vp, sz, vp]
     L.aquakv_chain_workspace_bytes.restype = sz
     L.aquakv_chain_workspace_bytes.argtypes = [vp, i64, i32]
     L.aquakv_encode_chain.restype = ctypes.c_int
@@ -288,6 +296,26 @@ class Codec:
         if rc:
             raise AquaKVError(rc, "aquakv_decode_attn")
         return out, lse
+
+    def fit_workspace_bytes(self, n_tokens: int, n_inputs: int) -> int:
+        return int(lib.aquakv_fit_workspace_bytes(self.h, n_tokens, n_inputs))
+
+    def fit_predictor(self, target, in0, in1=None, rate: float = 1e-3, fit_bias: bool = False,
+                      want_fp32: bool = False, workspace=None):
+        """One predictor of Algorithm 1 (aquakv_fit_predictor): returns (W [d, n_in*d] 16-bit, bias or None,
+        W in fp32 or None)."""
+        T, dev = target.shape[0], target.device
+        n_in = 2 if in1 is not None else 1
+        W = torch.empty((self.d, n_in * self.d), dtype=self.torch_dtype, device=dev)
+        W32 = torch.empty((self.d, n_in * self.d), dtype=torch.float32, device=dev) if want_fp32 else None
+        bias = torch.empty((self.d,), dtype=torch.float32, device=dev) if fit_bias else None
+        ws = workspace if workspace is not None else self._workspace(self.fit_workspace_bytes(T, n_in), dev)
+        rc = lib.aquakv_fit_predictor(self.h, T, _ptr(in0), _ptr(in1), _ld(in0, self.d), _ptr(target),
+                                      _ld(target, self.d), float(rate), int(bool(fit_bias)), _ptr(W), _ptr(W32),
+                                      _ptr(bias), _ptr(ws), ws.numel(), _stream())
+        if rc:
+            raise AquaKVError(rc, "aquakv_fit_predictor")
+        return W, bias, W32
 
     def encode_phase(self, role: int, X, in0=None, in1=None, W=None, bias=None, want_hat: bool = True):
         T, dev = X.shape[0], X.device

@@ -22,6 +22,7 @@
 
 #include "aquakv.h"
 #include "attn.cuh"
+#include "calib.cuh"
 #include "chain_kernel.cuh"
 #include "codec.cuh"
 #include "gemm_pred.cuh"
@@ -356,6 +357,66 @@ EncodeWs encode_ws(const aquakv_ctx* c, int64_t T) {
   w.khat_off = round_up(size_t(w.chunk) * c->p.d_kv * sizeof(float), 256);
   w.total = w.khat_off + round_up(size_t(w.chunk) * c->p.d_kv * 2, 256) + kWsSlack;
   return w;
+}
+
+// ---------------------------------------------------------------------------------------------
+// calibration of one predictor (calib.cuh)
+// ---------------------------------------------------------------------------------------------
+struct FitWs {
+  size_t xt_off, yt_off, g_off, c_off, gd_off, cd_off, sums_off, ridge_off, total;
+  int64_t Tp;
+  int n;           // input features
+};
+
+FitWs fit_ws(const aquakv_ctx* c, int64_t T, int n_inputs) {
+  FitWs w;
+  const size_t d = size_t(c->p.d_kv);
+  w.n = int(d) * n_inputs;
+  w.Tp = (T + 63) / 64 * 64;
+  const size_t n = size_t(w.n);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { const size_t o = off; off += round_up(bytes, 256); return o; };
+  w.xt_off = take(n * size_t(w.Tp) * 2);
+  w.yt_off = take(d * size_t(w.Tp) * 2);
+  w.g_off = take(n * n * sizeof(float));
+  w.c_off = take(n * d * sizeof(float));
+  w.gd_off = take(n * n * sizeof(double));
+  w.cd_off = take(n * d * sizeof(double));
+  w.sums_off = take((n + d) * sizeof(double));
+  w.ridge_off = take(sizeof(double));
+  w.total = off + kWsSlack;
+  return w;
+}
+
+// out[M][N] (fp32) = A B^T for token-contiguous 16-bit A [M][Tp], B [N][Tp] on the tensor cores.
+int launch_gram(aquakv_ctx* c, cudaStream_t st, const void* A, int M, const void* B, int N, int64_t Tp, float* out) {
+  CUtensorMap tA, tB;
+  int rc = make_tmap(c, &tA, A, uint64_t(M), uint64_t(Tp), uint64_t(Tp), kBM);
+  if (rc) return rc;
+  if ((rc = make_tmap(c, &tB, B, uint64_t(N), uint64_t(Tp), uint64_t(Tp), kBN))) return rc;
+  GemmArgs g;
+  g.M = M;
+  g.N = N;
+  g.nk0 = int(Tp / kBK);
+  g.nk1 = 0;
+  g.P = out;
+  g.ldP = N;
+  g.bias = nullptr;
+  g.status = c->d_status;
+  const int tiles = (M / kBM) * (N / kBN);
+  const int grid = tiles < c->sm_count ? tiles : c->sm_count;
+  if (c->bf16) gemm_pred_kernel<true><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(tA, tA, tB, g);
+  else gemm_pred_kernel<false><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(tA, tA, tB, g);
+  ++c->launches;
+  return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
+}
+
+void launch_fit_update(aquakv_ctx* c, cudaStream_t st, double* C, long long ldc, const double* A, long long lda,
+                       int transA, const double* B, long long ldb, int transB, int M, int N, int lower_only) {
+  if (M <= 0 || N <= 0) return;
+  const dim3 grid((N + 63) / 64, (M + 63) / 64), block(16, 16);
+  fit_update_kernel<<<grid, block, 0, st>>>(C, ldc, A, lda, transA, B, ldb, transB, M, N, lower_only);
+  ++c->launches;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -799,6 +860,7 @@ const char* aquakv_status_string(int status) {
     case AQUAKV_ERR_CUDA: return "CUDA call failed";
     case AQUAKV_ERR_TIMEOUT: return "bounded device-side wait expired";
     case AQUAKV_ERR_TOO_LARGE: return "more tokens than the fixed scratch of the no-allocation call holds";
+    case AQUAKV_ERR_NUMERIC: return "normal equations of a fit not positive definite";
     default: return "unknown status";
   }
 }
@@ -967,6 +1029,123 @@ int aquakv_profile_read(aquakv_ctx* c, int kernel_class, int64_t* launches, doub
     ++*launches;
   }
   return AQUAKV_OK;
+}
+
+size_t aquakv_fit_workspace_bytes(const aquakv_ctx* c, int64_t n_tokens, int32_t n_inputs) {
+  if (c == nullptr || n_tokens <= 0 || n_inputs < 1 || n_inputs > 2) return 0;
+  return fit_ws(c, n_tokens, n_inputs).total;
+}
+
+int aquakv_fit_predictor(aquakv_ctx* c, int64_t n_tokens, const void* in0, const void* in1, int64_t ld_in,
+                         const void* target, int64_t ld_target, double rate, int fit_bias, void* W_out,
+                         float* W32_out, float* bias_out, void* workspace, size_t workspace_bytes,
+                         void* cuda_stream) {
+  if (c == nullptr || n_tokens <= 0 || !(rate >= 0.0) || W_out == nullptr) return AQUAKV_ERR_INVALID_ARG;
+  const int d = c->p.d_kv;
+  if (d % kBN) return AQUAKV_ERR_UNSUPPORTED;
+  if (n_tokens > (int64_t(1) << 30)) return AQUAKV_ERR_TOO_LARGE;
+  int rc;
+  if ((rc = check_rows(in0, ld_in, d, true))) return rc;
+  if ((rc = check_rows(in1, ld_in, d, false))) return rc;
+  if ((rc = check_rows(target, ld_target, d, true))) return rc;
+  if (fit_bias && bias_out == nullptr) return AQUAKV_ERR_INVALID_ARG;
+  if (!aligned16(W_out) || !aligned16(W32_out) || (fit_bias && !aligned16(bias_out))) return AQUAKV_ERR_ALIGNMENT;
+  const int n_inputs = in1 != nullptr ? 2 : 1;
+  const FitWs w = fit_ws(c, n_tokens, n_inputs);
+  if (workspace == nullptr || !aligned16(workspace) || workspace_bytes < w.total) return AQUAKV_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  uint8_t* ws = ws_base(workspace);
+  uint16_t* Xt = reinterpret_cast<uint16_t*>(ws + w.xt_off);
+  uint16_t* Yt = reinterpret_cast<uint16_t*>(ws + w.yt_off);
+  float* G = reinterpret_cast<float*>(ws + w.g_off);
+  float* C = reinterpret_cast<float*>(ws + w.c_off);
+  double* Gd = reinterpret_cast<double*>(ws + w.gd_off);
+  double* Cd = reinterpret_cast<double*>(ws + w.cd_off);
+  double* sx = reinterpret_cast<double*>(ws + w.sums_off);
+  double* sy = sx + w.n;
+  double* ridge = reinterpret_cast<double*>(ws + w.ridge_off);
+  const int n = w.n;
+  const long long T = n_tokens, Tp = w.Tp;
+  ProfScope prof(c, st, AQUAKV_KERNEL_FIT);
+
+  // 1. token-contiguous copies
+  {
+    const dim3 block(32, 8);
+    const dim3 grid_x((unsigned)(Tp / 32), (unsigned)(d / 32));
+    fit_transpose_kernel<<<grid_x, block, 0, st>>>(static_cast<const uint16_t*>(in0), ld_in, T, Tp, Xt);
+    if (in1 != nullptr)
+      fit_transpose_kernel<<<grid_x, block, 0, st>>>(static_cast<const uint16_t*>(in1), ld_in, T, Tp,
+                                                     Xt + size_t(d) * size_t(Tp));
+    fit_transpose_kernel<<<grid_x, block, 0, st>>>(static_cast<const uint16_t*>(target), ld_target, T, Tp, Yt);
+    c->launches += in1 != nullptr ? 3 : 2;
+  }
+  // 2. normal equations on the tensor cores
+  if ((rc = launch_gram(c, st, Xt, n, Xt, n, Tp, G))) return rc;
+  if ((rc = launch_gram(c, st, Xt, n, Yt, d, Tp, C))) return rc;
+  // column sums for the intercept
+  if (fit_bias) {
+    if (cudaMemsetAsync(sx, 0, size_t(n + d) * sizeof(double), st) != cudaSuccess) return AQUAKV_ERR_CUDA;
+    const dim3 block(32, 8);
+    const dim3 grid_s((unsigned)((T + 255) / 256), (unsigned)(d / 32));
+    if (c->bf16) {
+      fit_colsum_kernel<true><<<grid_s, block, 0, st>>>(static_cast<const uint16_t*>(in0), ld_in, T, sx);
+      if (in1) fit_colsum_kernel<true><<<grid_s, block, 0, st>>>(static_cast<const uint16_t*>(in1), ld_in, T, sx + d);
+      fit_colsum_kernel<true><<<grid_s, block, 0, st>>>(static_cast<const uint16_t*>(target), ld_target, T, sy);
+    } else {
+      fit_colsum_kernel<false><<<grid_s, block, 0, st>>>(static_cast<const uint16_t*>(in0), ld_in, T, sx);
+      if (in1) fit_colsum_kernel<false><<<grid_s, block, 0, st>>>(static_cast<const uint16_t*>(in1), ld_in, T, sx + d);
+      fit_colsum_kernel<false><<<grid_s, block, 0, st>>>(static_cast<const uint16_t*>(target), ld_target, T, sy);
+    }
+    c->launches += in1 != nullptr ? 3 : 2;
+  }
+  const double* sxp = fit_bias ? sx : nullptr;
+  const double* syp = fit_bias ? sy : nullptr;
+  fit_ridge_kernel<<<1, 256, 0, st>>>(G, n, double(T), sxp, rate, ridge);
+  {
+    const int wide = n > d ? n : d;
+    const dim3 grid_p((wide + 255) / 256, n);
+    fit_prepare_kernel<<<grid_p, 256, 0, st>>>(G, C, n, d, double(T), sxp, syp, ridge, Gd, Cd);
+  }
+  c->launches += 2;
+  // 3. Cholesky factorisation, panel by panel
+  for (int k = 0; k < n; k += kFitNB) {
+    fit_chol_diag_kernel<<<1, dim3(kFitNB, kFitNB), 0, st>>>(Gd, n, k, c->d_status);
+    ++c->launches;
+    const int below = n - k - kFitNB;
+    if (below > 0) {
+      fit_chol_panel_kernel<<<below / kFitNB, kFitNB, 0, st>>>(Gd, n, k);
+      ++c->launches;
+      double* A22 = Gd + size_t(k + kFitNB) * n + (k + kFitNB);
+      const double* L21 = Gd + size_t(k + kFitNB) * n + k;
+      launch_fit_update(c, st, A22, n, L21, n, 0, L21, n, 1, below, below, 1);
+    }
+  }
+  // forward solve L Z = Cd, then backward solve L^T Wt = Z (both in place in Cd)
+  const int solve_grid = (d + 127) / 128;
+  for (int k = 0; k < n; k += kFitNB) {
+    fit_solve_diag_kernel<<<solve_grid, 128, 0, st>>>(Gd, n, k, Cd, d, 0);
+    ++c->launches;
+    const int below = n - k - kFitNB;
+    launch_fit_update(c, st, Cd + size_t(k + kFitNB) * d, d, Gd + size_t(k + kFitNB) * n + k, n, 0,
+                      Cd + size_t(k) * d, d, 0, below, d, 0);
+  }
+  for (int k = n - kFitNB; k >= 0; k -= kFitNB) {
+    fit_solve_diag_kernel<<<solve_grid, 128, 0, st>>>(Gd, n, k, Cd, d, 1);
+    ++c->launches;
+    launch_fit_update(c, st, Cd, d, Gd + size_t(k) * n, n, 1, Cd + size_t(k) * d, d, 0, k, d, 0);
+  }
+  // 4. the adapter in its storage layout, and the intercept
+  {
+    const dim3 block(32, 8), grid_o(n / 32, d / 32);
+    if (c->bf16) fit_store_kernel<true><<<grid_o, block, 0, st>>>(Cd, n, d, static_cast<uint16_t*>(W_out), W32_out);
+    else fit_store_kernel<false><<<grid_o, block, 0, st>>>(Cd, n, d, static_cast<uint16_t*>(W_out), W32_out);
+    ++c->launches;
+    if (fit_bias) {
+      fit_bias_kernel<<<(d + 127) / 128, 128, 0, st>>>(Cd, n, d, sx, sy, double(T), bias_out);
+      ++c->launches;
+    }
+  }
+  return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
 }
 
 int aquakv_poll_status(aquakv_ctx* c, void* cuda_stream) {

@@ -13,6 +13,7 @@ namespace aquakv {
 
 // Status word values written by kernels (mirrors AQUAKV_ERR_TIMEOUT in the public header).
 constexpr int kStatusTimeout = -6;
+constexpr int kStatusNumeric = -8;   // AQUAKV_ERR_NUMERIC: the normal equations of a fit were not positive definite
 
 // A bounded wait gives up after this many nanoseconds of %globaltimer.
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
