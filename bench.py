@@ -357,6 +357,65 @@ def ops_by_config(api, chain, peaks, dev, reps=5):
     return out
 
 
+def calibration_entry(api, peaks, dev, reps=3):
+    """Algorithm 1 on the prefill-shaped workload: three layers of 32768 calibration tokens (two fitted
+    layers), d_kv 1024, 2 bits.  Time per fitted layer (key fit, key reconstruction, value fit, value
+    reconstruction), against the time the normal equations need on the tensor cores plus the time the
+    solve needs on the fp64 units; and what the fitted predictors buy: relative reconstruction error
+    of the last layer with fitted predictors, with the seeded random adapters, and without predictors
+    at 2 and at 3 bits per value."""
+    from paper_2501_19392_b200 import calibrate as gcal
+    shape = dataclasses.replace(synth.CONFIGS[2], n_layers=3)
+    T, d, L = shape.n_tokens, shape.d_kv, shape.n_layers
+    codec = _shape_codec(api, shape)
+    kv = synth.kv_chain(shape, seed=6001, device=dev)
+    run = lambda: gcal.calibrate(codec, kv.K, kv.V, rate=1e-3, keep_reconstructions=True)
+    preds, recs = run()
+    ms_all = _time_calls(run, reps, warm=1)
+    ms_layer0 = _time_calls(lambda: (codec.encode_phase(api.ROLE_KEY, kv.K[0]), codec.encode_phase(api.ROLE_VALUE, kv.V[0])),
+                            reps, warm=1)
+    ms_layer = (ms_all - ms_layer0) / (L - 1)
+    ms_fit_k = _time_calls(lambda: codec.fit_predictor(kv.K[1], recs[0][0], None, 1e-3), reps, warm=1)
+    ms_fit_v = _time_calls(lambda: codec.fit_predictor(kv.V[1], recs[0][1], recs[1][0], 1e-3), reps, warm=1)
+    assert codec.poll_status() == 0
+    gram_flops = 2.0 * T * (d * (d + d) + 2 * d * (2 * d + d))            # X^T X and X^T Y of both fits
+    solve_flops = sum(n ** 3 / 3.0 + 2.0 * n * n * d for n in (d, 2 * d)) * 2.0   # Cholesky + two triangular solves, multiply-adds x 2
+    fp64_peak = 148 * 64 * 2 * 1.965e9                                      # 64 fp64 FMA lanes per SM at the maximum clock
+    t_roof_ms = (gram_flops / (peaks["tf_burst"] * 1e12) + solve_flops / fp64_peak) * 1e3
+
+    def rel_err(X, Xh):
+        X, Xh = X.float(), Xh.float()
+        return float(((X - Xh) ** 2).sum() / ((X - X.mean(dim=0)) ** 2).sum())
+
+    last = L - 1
+    quality = {"fitted_2bit": {"K": rel_err(kv.K[last], recs[last][0]), "V": rel_err(kv.V[last], recs[last][1])}}
+    # the same chain with the seeded random adapters of the throughput runs
+    ad = synth.random_adapters(shape, seed=6002, device=dev)
+    _, _, Kh = codec.encode_phase(api.ROLE_KEY, kv.K[0])
+    _, _, Vh = codec.encode_phase(api.ROLE_VALUE, kv.V[0])
+    for l in range(1, L):
+        _, _, Kn = codec.encode_phase(api.ROLE_KEY, kv.K[l], Kh, None, ad.Wk[l])
+        _, _, Vh = codec.encode_phase(api.ROLE_VALUE, kv.V[l], Vh, Kn, ad.Wv[l])
+        Kh = Kn
+    quality["random_adapters_2bit"] = {"K": rel_err(kv.K[last], Kh), "V": rel_err(kv.V[last], Vh)}
+    for n, name in ((16, "no_predictor_2bit"), (64, "no_predictor_3bit")):
+        c = _shape_codec(api, dataclasses.replace(shape, grid_size=n))
+        _, _, Kd = c.encode_phase(api.ROLE_KEY, kv.K[last])
+        _, _, Vd = c.encode_phase(api.ROLE_VALUE, kv.V[last])
+        quality[name] = {"K": rel_err(kv.K[last], Kd), "V": rel_err(kv.V[last], Vd)}
+    torch.cuda.empty_cache()
+    return {"config": "calibration", "workload": shape.name + " (3 layers of calibration tokens)", "op": "calibrate",
+            "tokens_per_call": T, "d_kv": d, "grid_points": shape.grid_size, "regularizer_rate": 1e-3,
+            "ms_per_fitted_layer": ms_layer, "ms_fit_key_predictor": ms_fit_k, "ms_fit_value_predictor": ms_fit_v,
+            "token_layers_per_s": T / (ms_layer * 1e-3), "gram_tflop_per_layer": gram_flops / 1e12,
+            "solve_fp64_gflop_per_layer": solve_flops / 1e9, "roofline_ms_per_layer": t_roof_ms,
+            "frac_of_roofline_burst": t_roof_ms / (ms_fit_k + ms_fit_v), "bound": "tensor + fp64 alu",
+            "fp64_peak_tflops": fp64_peak / 1e12,
+            "note": "roofline = normal equations at the tensor peak + solve at 148 SMs x 64 fp64 lanes x 2 x 1.965 GHz; "
+                    "fraction taken over the two fits (the reconstructions between them are encode calls)",
+            "relative_error_last_layer": quality}
+
+
 # ------------------------------------------------------------------------------------------------
 # GPU arm
 # ------------------------------------------------------------------------------------------------
@@ -527,7 +586,8 @@ def main():
         del kv, cache, bufs, q, out
         torch.cuda.empty_cache()
         result["ops_by_config"] = ([dict(config=2, workload=shape.name, op=name, tokens_per_call=T, **v)
-                                    for name, v in roof.items()] + ops_by_config(api, chain, peaks, dev))
+                                    for name, v in roof.items()] + ops_by_config(api, chain, peaks, dev) +
+                                   [calibration_entry(api, peaks, dev)])
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = oracle_baseline(shape, n_q)
     if rank == 0:
