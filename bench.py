@@ -431,6 +431,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-other-configs", action="store_true", help="skip the per-call timing of configs 1, 3, 4, 5")
+    ap.add_argument("--only-calibration", action="store_true",
+                    help="run only the calibration entry of ops_by_config and print it (profiling aid)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -448,6 +450,10 @@ def main():
     from paper_2501_19392_b200 import api, chain    # raises if the CUDA library is missing
 
     peaks = load_peaks()
+    if args.only_calibration:
+        if rank == 0:
+            print(json.dumps(calibration_entry(api, peaks, dev, reps=1)))
+        return
     shape, batch = workload(args)
     T, L, d = shape.n_tokens, shape.n_layers, shape.d_kv
     ctx_len = T // batch
