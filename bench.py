@@ -354,6 +354,32 @@ def ops_by_config(api, chain, peaks, dev, reps=5):
     assert codec.poll_status() == 0
     del rc, Kp, Vp
     torch.cuda.empty_cache()
+
+    # configs 6 / 7 (second workload): Qwen-2.5-shaped caches, only the 20 % of a 131072-token context that a
+    # pruning policy keeps are compressed, first layer left in 16 bits; time of one predicted layer
+    # (gather of the kept keys and values + encode of the compact rows)
+    for cfg in (6, 7):
+        shape = dataclasses.replace(synth.CONFIGS[cfg], n_layers=3)
+        codec = _shape_codec(api, shape)
+        kv = synth.kv_chain(shape, seed=1000 * cfg + 1, device=dev)
+        ad = synth.random_adapters(shape, seed=1000 * cfg + 2, device=dev)
+        idx = torch.from_numpy(synth.kept_tokens(shape.n_tokens, 0.2, seed=1000 * cfg + 3)).to(dev)
+        n_keep = int(idx.shape[0])
+        cache = chain.CompressedCache.empty(codec, shape.n_layers, n_keep, dev)
+        bufs = chain.PingPong(codec, n_keep, dev)
+        sk, sv = torch.empty_like(bufs.K[0]), torch.empty_like(bufs.V[0])
+        run = lambda: chain.encode_chain_kept(codec, kv.K, kv.V, idx, ad, cache, bufs, sk, sv, first_layer_16bit=True)
+        run()
+        ms_chain = _time_calls(run, reps)
+        first = lambda: (codec.gather_rows(kv.K[0], idx, bufs.K[0]), codec.gather_rows(kv.V[0], idx, bufs.V[0]))
+        ms = (ms_chain - _time_calls(first, reps)) / (shape.n_layers - 1)
+        out.append(_shape_entry(peaks, shape, "encode_kept_tokens", n_keep, ms, _shape_bytes(shape, n_keep, True),
+                                config=cfg, context_tokens=shape.n_tokens, kept_fraction=0.2, ms_chain=ms_chain,
+                                chain_layers=shape.n_layers,
+                                note="per predicted layer: gather of the kept K and V rows + encode; first layer in 16 bits"))
+        assert codec.poll_status() == 0
+        del kv, cache, bufs, sk, sv
+        torch.cuda.empty_cache()
     return out
 
 

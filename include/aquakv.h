@@ -322,6 +322,19 @@ int aquakv_decode_attn(aquakv_ctx* ctx, int32_t batch, int64_t ctx_len,
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Row gather for compressing a subset of the tokens (Section 4.3: a pruning policy such as H2O
+ * selects the tokens to keep, "and [we] apply AQUA-KV compression [to] those tokens"): dst row i =
+ * src row idx[i], 16-bit rows of d_kv values; the compact rows then go through aquakv_encode like any
+ * other batch (their previous-layer reconstructions are compact in the same order).  idx is a device
+ * array of n_rows int64 values in [0, n_src_rows), or NULL for the identity (a plain row copy, which is
+ * how an unquantised first layer - the Qwen-2.5 setting of the appendix tables - enters the chain's
+ * buffers).  src / dst: device, 16-byte aligned, ld multiples of 8 and >= d_kv, no overlap.
+ * Asynchronous on cuda_stream.  An index out of range zero-fills its row and is reported by
+ * aquakv_poll_status as AQUAKV_ERR_INVALID_ARG.                                                       */
+int aquakv_gather_rows(aquakv_ctx* ctx, int64_t n_rows, const int64_t* idx, int64_t n_src_rows, const void* src,
+                       int64_t ld_src, void* dst, int64_t ld_dst, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Calibration of one predictor (Algorithm 1, the two arg-min lines; Section 3.2: linear regression
  * with "closed-form training"; Appendix A: "closed form solution with regularizer rate 1e-3"):
  *

@@ -36,7 +36,7 @@ SYMBOLS = [
     "aquakv_decode_attn", "aquakv_decode_noalloc", "aquakv_encode_phase", "aquakv_decode_phase", "aquakv_poll_status", "aquakv_launch_count", "aquakv_status_string",
     "aquakv_profile_enable", "aquakv_profile_read", "aquakv_selftest_bounded_wait",
     "aquakv_chain_workspace_bytes", "aquakv_encode_chain", "aquakv_decode_chain",
-    "aquakv_fit_workspace_bytes", "aquakv_fit_predictor",
+    "aquakv_fit_workspace_bytes", "aquakv_fit_predictor", "aquakv_gather_rows",
 ]
 
 
@@ -98,6 +98,8 @@ def _load():
     L.aquakv_profile_enable.argtypes = [vp, ctypes.c_int]
     L.aquakv_profile_read.restype = ctypes.c_int
     L.aquakv_profile_read.argtypes = [vp, ctypes.c_int, ctypes.POINTER(i64), ctypes.POINTER(ctypes.c_double)]
+    L.aquakv_gather_rows.restype = ctypes.c_int
+    L.aquakv_gather_rows.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp]
     L.aquakv_fit_workspace_bytes.restype = sz
     L.aquakv_fit_workspace_bytes.argtypes = [vp, i64, i32]
     L.aquakv_fit_predictor.restype = ctypes.c_int
@@ -296,6 +298,17 @@ class Codec:
         if rc:
             raise AquaKVError(rc, "aquakv_decode_attn")
         return out, lse
+
+    def gather_rows(self, src, idx=None, out=None):
+        """Rows idx (int64 device tensor; None = all rows in order) of a 16-bit [T, d] tensor, compact."""
+        n = src.shape[0] if idx is None else idx.shape[0]
+        if out is None:
+            out = torch.empty((n, self.d), dtype=src.dtype, device=src.device)
+        rc = lib.aquakv_gather_rows(self.h, n, _ptr(idx), src.shape[0], _ptr(src), _ld(src, self.d), _ptr(out),
+                                    _ld(out, self.d), _stream())
+        if rc:
+            raise AquaKVError(rc, "aquakv_gather_rows")
+        return out
 
     def fit_workspace_bytes(self, n_tokens: int, n_inputs: int) -> int:
         return int(lib.aquakv_fit_workspace_bytes(self.h, n_tokens, n_inputs))

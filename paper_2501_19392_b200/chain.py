@@ -58,6 +58,30 @@ def encode_chain(codec: api.Codec, K: List[torch.Tensor], V: List[torch.Tensor],
                      bufs.K[cur], bufs.V[cur])
 
 
+def encode_chain_kept(codec: api.Codec, K: List[torch.Tensor], V: List[torch.Tensor], idx: torch.Tensor,
+                      adapters, cache: CompressedCache, bufs: PingPong, stage_k: torch.Tensor,
+                      stage_v: torch.Tensor, first_layer_16bit: bool = False) -> None:
+    """Algorithm 2 over the tokens a pruning policy keeps (Section 4.3): each layer's kept rows are
+    gathered into the compact staging tensors and encoded like any batch; cache and buffers hold
+    len(idx) tokens.  first_layer_16bit leaves the first layer unquantised (the Qwen-2.5 setting of the
+    appendix tables): its kept rows are carried into the buffers as they are and nothing is stored for it."""
+    for l in range(len(K)):
+        cur, prv = l % 2, (l + 1) % 2
+        has = l > 0
+        if l == 0 and first_layer_16bit:
+            codec.gather_rows(K[0], idx, bufs.K[cur])
+            codec.gather_rows(V[0], idx, bufs.V[cur])
+            continue
+        codec.gather_rows(K[l], idx, stage_k)
+        codec.gather_rows(V[l], idx, stage_v)
+        codec.encode(stage_k, stage_v,
+                     bufs.K[prv] if has else None, bufs.V[prv] if has else None,
+                     adapters.Wk[l] if has else None, adapters.Wv[l] if has else None,
+                     adapters.bk[l] if has else None, adapters.bv[l] if has else None,
+                     cache.Kcodes[l], cache.Kscales[l], cache.Vcodes[l], cache.Vscales[l],
+                     bufs.K[cur], bufs.V[cur])
+
+
 def decode_chain(codec: api.Codec, cache: CompressedCache, adapters, bufs: PingPong,
                  n_layers: Optional[int] = None) -> int:
     """Algorithm 3 for every layer in order; returns the index of the buffer pair holding the last

@@ -1031,6 +1031,27 @@ int aquakv_profile_read(aquakv_ctx* c, int kernel_class, int64_t* launches, doub
   return AQUAKV_OK;
 }
 
+int aquakv_gather_rows(aquakv_ctx* c, int64_t n_rows, const int64_t* idx, int64_t n_src_rows, const void* src,
+                       int64_t ld_src, void* dst, int64_t ld_dst, void* cuda_stream) {
+  if (c == nullptr || n_rows < 0 || n_src_rows < 0) return AQUAKV_ERR_INVALID_ARG;
+  if (n_rows == 0) return AQUAKV_OK;
+  const int d = c->p.d_kv;
+  int rc;
+  if ((rc = check_rows(src, ld_src, d, true))) return rc;
+  if ((rc = check_rows(dst, ld_dst, d, true))) return rc;
+  if (src == dst || (idx == nullptr && n_rows > n_src_rows)) return AQUAKV_ERR_INVALID_ARG;
+  if (idx != nullptr && (reinterpret_cast<uintptr_t>(idx) & 7u)) return AQUAKV_ERR_ALIGNMENT;
+  const int warps_per_block = 8;
+  int64_t blocks = (n_rows + warps_per_block - 1) / warps_per_block;
+  const int64_t cap = int64_t(c->sm_count) * 16;
+  if (blocks > cap) blocks = cap;
+  gather_rows_kernel<<<int(blocks), warps_per_block * 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      static_cast<const uint16_t*>(src), ld_src, reinterpret_cast<const long long*>(idx), n_rows, n_src_rows, d,
+      static_cast<uint16_t*>(dst), ld_dst, c->d_status);
+  ++c->launches;
+  return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
+}
+
 size_t aquakv_fit_workspace_bytes(const aquakv_ctx* c, int64_t n_tokens, int32_t n_inputs) {
   if (c == nullptr || n_tokens <= 0 || n_inputs < 1 || n_inputs > 2) return 0;
   return fit_ws(c, n_tokens, n_inputs).total;

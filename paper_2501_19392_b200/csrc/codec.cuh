@@ -709,4 +709,28 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_rows_kernel(const Cod
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Row gather (Section 4.3 "Compatibility with Pruning": a token-pruning policy picks the tokens to
+// keep and only those are compressed).  dst[i][0..d) = src[idx[i]][0..d) for 16-bit rows; idx ==
+// nullptr copies row i (used to carry an unquantised first layer into the chain's buffers).  One warp
+// per row, 16-byte accesses.  An index outside [0, n_src_rows) zero-fills the row and records
+// kStatusBadIndex.
+// ---------------------------------------------------------------------------------------------
+constexpr int kStatusBadIndex = -1;     // AQUAKV_ERR_INVALID_ARG
+__global__ void gather_rows_kernel(const uint16_t* __restrict__ src, long long ld_src, const long long* __restrict__ idx,
+                                   long long n_rows, long long n_src_rows, int d, uint16_t* __restrict__ dst,
+                                   long long ld_dst, int* __restrict__ status) {
+  const int lane = threadIdx.x & 31;
+  const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long n_warps = (long long)gridDim.x * (blockDim.x >> 5);
+  for (long long i = warp; i < n_rows; i += n_warps) {
+    const long long r = idx != nullptr ? idx[i] : i;
+    const bool ok = r >= 0 && r < n_src_rows;
+    if (!ok && lane == 0) atomicExch(status, kStatusBadIndex);
+    uint4* out = reinterpret_cast<uint4*>(dst + i * ld_dst);
+    const uint4* in = reinterpret_cast<const uint4*>(src + (ok ? r : 0) * ld_src);
+    for (int c = lane; c < d / 8; c += 32) out[c] = ok ? __ldcs(in + c) : make_uint4(0u, 0u, 0u, 0u);
+  }
+}
+
 }  // namespace aquakv

@@ -86,6 +86,10 @@ CONFIGS = {
     4: Shape("llama3.3-70b-bulk-decode", 8, 128, 64, 80, 131072, BF16, 1024, 1024, 16),
     5: Shape("llama3.1-8b-decode-attn", 8, 128, 32, 1, 32 * 32768, BF16, 1024, 1024, 16,
              batch=32),
+    # second workload: Qwen-2.5-shaped caches (2 and 4 KV heads of 128: d_kv 256 / 512, group = d_kv, first
+    # layer left in 16 bits), compressed for the 20 % of a 131072-token context that a pruning policy keeps
+    6: Shape("qwen2.5-3b-kept-token-encode", 2, 128, 16, 36, 131072, BF16, 256, 256, 16),
+    7: Shape("qwen2.5-7b-kept-token-encode", 4, 128, 28, 28, 131072, BF16, 512, 512, 16),
 }
 
 
@@ -240,6 +244,15 @@ def random_16bit(shape_, dtype: int, seed: int, device="cpu", std: float = 1.0) 
 # Token sharding for multi-GPU runs (tokens are independent through all layers, so ranks take
 # disjoint token ranges and exchange nothing)
 # --------------------------------------------------------------------------------------------
+
+def kept_tokens(n_tokens: int, fraction: float, seed: int) -> np.ndarray:
+    """Sorted indices of the tokens a pruning policy keeps: a seeded random subset of round(fraction *
+    n_tokens) tokens (stand-in for a heavy-hitter selection, which depends on attention scores the
+    harness does not have)."""
+    rng = np.random.default_rng(seed)
+    n_keep = int(round(fraction * n_tokens))
+    return np.sort(rng.choice(n_tokens, size=n_keep, replace=False)).astype(np.int64)
+
 
 def shard_range(n: int, rank: int, world: int, multiple: int = 1):
     """Contiguous [begin, end) of rank's share of n items, every share but the last a multiple
