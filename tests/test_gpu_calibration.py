@@ -96,6 +96,18 @@ def test_fit_matches_the_oracle(heads, T, dtype, two_inputs, bias, scales):
     compare_fit(ora, W16, W32, b, ref, X64, bias)
 
 
+def test_fit_at_the_benchmark_size():
+    # the key fit bench.py times: 32768 calibration tokens, d_kv 1024, outlier channels
+    shape = small_shape(8, 32768, 2, oracle.BF16, channel_scales=True)
+    codec, ora = make(shape)
+    kv = synth.kv_chain(shape, seed=6001)
+    W16, _, W32 = codec.fit_predictor(kv.K[1].to(DEV), kv.K[0].to(DEV), None, rate=1e-3, want_fp32=True)
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    ref = cal.fit_predictor([synth.to_bits(kv.K[0])], synth.to_bits(kv.K[1]), shape.dtype, 1e-3)
+    compare_fit(ora, W16, W32, None, ref, cal.bits_to_double(synth.to_bits(kv.K[0]), shape.dtype), False)
+
+
 def test_rows_with_padding_and_rate_zero_on_a_planted_map():
     # strided inputs (ld > d_kv) and an exactly linear target: W is the planted matrix up to 16-bit rounding
     shape = small_shape(2, 2048, 2, oracle.BF16)

@@ -104,3 +104,40 @@ def test_kept_token_encode_matches_the_oracle_on_the_kept_rows(cfg, T, L, n):
         assert torch.equal(Ks, cache.Kscales[l]) and torch.equal(Vs, cache.Vscales[l])
     assert torch.equal(Kh_prev, bufs.K[(L - 1) % 2]) and torch.equal(Vh_prev, bufs.V[(L - 1) % 2])
     assert codec.poll_status() == 0
+
+
+def test_kept_token_encode_at_the_benchmark_size_on_sampled_rows():
+    # the launch configuration bench.py times for config 6: 26214 kept tokens of a 131072-token context, d_kv 256;
+    # rows are independent, so the oracle checks a sample of them
+    from paper_2501_19392_b200 import api
+    shape = dataclasses.replace(synth.CONFIGS[6], n_layers=2)
+    codec, ora = make(shape)
+    kv = synth.kv_chain(shape, seed=6001, device=DEV)
+    ad = synth.random_adapters(shape, seed=6002, device=DEV)
+    keep = synth.kept_tokens(shape.n_tokens, 0.2, seed=6003)
+    idx = torch.from_numpy(keep).to(DEV)
+    K0, V0 = codec.gather_rows(kv.K[0], idx), codec.gather_rows(kv.V[0], idx)          # first layer in 16 bits
+    K1, V1 = codec.gather_rows(kv.K[1], idx), codec.gather_rows(kv.V[1], idx)
+    Kc, Ks, Vc, Vs, Kh, Vh = codec.encode(K1, V1, K0, V0, ad.Wk[1], ad.Wv[1])
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    assert Kc.shape[0] == len(keep) == 26214
+    rng = np.random.default_rng(5)
+    sample = np.sort(np.concatenate([rng.choice(len(keep), 1500, replace=False), [0, len(keep) - 1]]))
+    sel = torch.from_numpy(sample).to(DEV)
+    b = lambda t: synth.to_bits(t[sel].cpu())
+    src = lambda t: synth.to_bits(t[idx[sel]].cpu())
+    assert np.array_equal(b(K1), src(kv.K[1])) and np.array_equal(b(V0), src(kv.V[0]))
+    ok_ = ora.encode_phase(src(kv.K[1]), [src(kv.K[0])], synth.to_bits(ad.Wk[1].cpu()), None, "k")
+    rows_ok, _ = scale_rows_ok(gpu_bits(Ks[sel].view(torch.float16)), ok_["scales"], ok_["scales_exact"])
+    check_codes(Kc[sel].cpu().numpy(), ok_, shape.code_bits, rows_ok)
+    same = rows_ok & (Kc[sel].cpu().numpy() == ok_["codes"]).all(axis=1)
+    check_same_rows(same, shape.d_kv, int((~rows_ok).sum()))
+    check_recon(b(Kh), ok_["hat_exact"], ok_["hat"], shape.dtype, same)
+    # values: the oracle is given the GPU's reconstructed keys of the sampled rows (teacher forcing inside the layer)
+    ov_ = ora.encode_phase(src(kv.V[1]), [src(kv.V[0]), b(Kh)], synth.to_bits(ad.Wv[1].cpu()), None, "v")
+    rows_ok_v, _ = scale_rows_ok(gpu_bits(Vs[sel].view(torch.float16)), ov_["scales"], ov_["scales_exact"])
+    check_codes(Vc[sel].cpu().numpy(), ov_, shape.code_bits, rows_ok_v)
+    same_v = rows_ok_v & (Vc[sel].cpu().numpy() == ov_["codes"]).all(axis=1)
+    check_same_rows(same_v, shape.d_kv, int((~rows_ok_v).sum()))
+    check_recon(b(Vh), ov_["hat_exact"], ov_["hat"], shape.dtype, same_v)
