@@ -1,0 +1,96 @@
+"""CPU oracle of the alternative backbone quantizer: round-to-nearest on a uniform grid with absmax
+normalisation per group, applied per token (Section 4.1 "Alternative quantizers": "Quanto ... simple
+round-to-nearest quantization with absmax normalization ... the default group size 64 and per-token
+compression"; Section 3.2: the method "is agnostic to the choice of Q").
+
+TEST INFRASTRUCTURE ONLY, like the rest of this package: plain numpy in double precision.
+
+Reading (the paper names the scheme, not its arithmetic).  For b bits per value the levels are the
+2^b signed integers -2^(b-1) .. 2^(b-1)-1 times the group scale; the scale is absmax / 2^(b-1), stored
+as fp16 (clamped to the largest finite fp16) and it is the ROUNDED scale that normalises, so encoder
+and decoder agree; a value goes to the nearest level, the lower one on an exact tie (the codec's rule
+"lowest index wins"), and saturates at the ends (the group's positive maximum maps to 2^(b-1)-1); a
+group of zeros has scale 0 and level 0.  The code of a value is its level + 2^(b-1) as an unsigned
+b-bit number; codes are packed LSB-first in value order; no rotation, no sign flips.  Predictors,
+residual and add-back are those of Algorithms 2 and 3: codes = Q(x - pred), hat = round16(pred + Q^-1).
+"""
+from __future__ import annotations
+
+from typing import Optional, Sequence
+
+import numpy as np
+
+from . import F16, Oracle
+from .calibration import bits_to_double, double_to_bits
+
+
+def _pack(levels_unsigned: np.ndarray, b: int) -> np.ndarray:
+    """[T, d] unsigned b-bit numbers -> [T, d*b/8] bytes, LSB-first in value order."""
+    T, d = levels_unsigned.shape
+    bits = ((levels_unsigned[:, :, None] >> np.arange(b)[None, None, :]) & 1).astype(np.uint8).reshape(T, d * b)
+    return np.packbits(bits, axis=1, bitorder="little")
+
+
+def _unpack(codes: np.ndarray, b: int, d: int) -> np.ndarray:
+    T = codes.shape[0]
+    bits = np.unpackbits(np.ascontiguousarray(codes, dtype=np.uint8), axis=1, bitorder="little")[:, :d * b]
+    return (bits.reshape(T, d, b).astype(np.int64) << np.arange(b)[None, None, :]).sum(axis=2)
+
+
+def quantize(R: np.ndarray, b: int, g: int):
+    """Q on double residuals R [T, d].  Returns codes, scales (fp16 bits), margins (distance of every
+    normalised value from the nearest decision boundary, in level spacings) and the unrounded scales."""
+    R = np.asarray(R, dtype=np.float64)
+    T, d = R.shape
+    half = 1 << (b - 1)
+    G = R.reshape(T, d // g, g)
+    s_exact = np.abs(G).max(axis=2) / half
+    s16_bits = double_to_bits(np.minimum(s_exact, 65504.0), F16)
+    s16 = bits_to_double(s16_bits, F16)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        x = np.where(s16[:, :, None] > 0, G / np.where(s16 > 0, s16, 1.0)[:, :, None], 0.0)
+    q = np.ceil(x - 0.5)                                   # nearest integer, the lower one on a tie
+    q = np.clip(q, -half, half - 1)
+    # decision boundaries are the half-integers between neighbouring levels: -half + 0.5 .. half - 1.5
+    boundary = np.clip(np.floor(x) + 0.5, -half + 0.5, half - 1.5)
+    margins = np.abs(x - boundary)
+    codes = _pack((q + half).astype(np.int64).reshape(T, d), b)
+    return dict(codes=codes, scales=s16_bits, margins=margins.reshape(T, d), scales_exact=s_exact)
+
+
+def dequantize(codes: np.ndarray, scales: np.ndarray, b: int, g: int, d: int) -> np.ndarray:
+    """Q^-1 to double: level * scale."""
+    T = codes.shape[0]
+    q = _unpack(codes, b, d) - (1 << (b - 1))
+    s16 = bits_to_double(np.ascontiguousarray(scales, dtype=np.uint16).reshape(T, d // g), F16)
+    return (q.reshape(T, d // g, g) * s16[:, :, None]).reshape(T, d)
+
+
+class UniformOracle:
+    """Algorithm 2 / 3 phases with the uniform backbone.  `linear` is a codec oracle of the same width
+    and 16-bit type, used for the predictor product only."""
+
+    def __init__(self, linear: Oracle, bits: int, group: int):
+        self.linear, self.b, self.g = linear, bits, group
+        self.d, self.dtype = linear.d, linear.dtype
+        self.code_bytes = self.d * bits // 8
+        self.n_groups = self.d // group
+
+    def _pred(self, T, inputs, W, bias):
+        if W is None:
+            return np.zeros((T, self.d), np.float64)
+        return self.linear.predict(list(inputs), W, bias)
+
+    def encode_phase(self, X: np.ndarray, inputs: Sequence[np.ndarray], W: Optional[np.ndarray],
+                     bias: Optional[np.ndarray] = None):
+        x = bits_to_double(X, self.dtype)
+        pred = self._pred(x.shape[0], inputs, W, bias)
+        out = quantize(x - pred, self.b, self.g)                                   # Algorithm 2 lines 6 / 8
+        hat_exact = pred + dequantize(out["codes"], out["scales"], self.b, self.g, self.d)   # lines 7 / 9
+        out.update(hat=double_to_bits(hat_exact, self.dtype), hat_exact=hat_exact, pred=pred)
+        return out
+
+    def decode_phase(self, codes, scales, inputs, W, bias=None):
+        T = codes.shape[0]
+        hat_exact = self._pred(T, inputs, W, bias) + dequantize(codes, scales, self.b, self.g, self.d)   # Algorithm 3 lines 5 / 7
+        return dict(hat=double_to_bits(hat_exact, self.dtype), hat_exact=hat_exact)
