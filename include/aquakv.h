@@ -85,7 +85,8 @@ typedef struct aquakv_params {
 
 typedef struct aquakv_ctx aquakv_ctx; /* opaque; owns the device copies of grid, signs, status */
 
-/* Bytes of one token's codes for these parameters (d_kv/2 * log2(n) / 8), or a negative error. */
+/* Bytes of one token's codes for these parameters (d_kv/2 * log2(n) / 8; with grid_dim = 1, see
+ * aquakv_create, d_kv * log2(n) / 8), or a negative error. */
 int aquakv_code_bytes(const aquakv_params* params);
 
 /*
@@ -95,6 +96,18 @@ int aquakv_code_bytes(const aquakv_params* params);
  * for keys and for values.  All three are copied; the caller may free them after the call.
  * This is the only entry point that allocates device memory (a few KB) and it synchronises the
  * device once.  Errors: INVALID_ARG (NULL, sign not +-1, non-finite grid), UNSUPPORTED, CUDA.
+ *
+ * Alternative backbone (Section 4.1 "Alternative quantizers": Quanto-style "round-to-nearest quantization
+ * with absmax normalization", group size 64, per token; Section 3.2: the method is agnostic to Q):
+ * grid_dim = 1 selects it.  grid_size = 2^b in {4, 8, 16} is then the number of levels PER VALUE (b bits
+ * per value): the signed integers -2^(b-1) .. 2^(b-1)-1 times the group scale, scale = absmax / 2^(b-1)
+ * stored as fp16, nearest level with the lower one on a tie, saturation at the ends, code = level +
+ * 2^(b-1), codes packed LSB-first in value order (d_kv * b / 8 bytes per token); had_block must be 1 (no
+ * rotation), scale_group in {32, 64, 128, 256}; grid_host and the sign arrays are not read and may be
+ * NULL.  Such a ctx serves aquakv_encode / aquakv_decode (with predictors: two launches per phase, and
+ * Khat is required because the value phase reads it), the *_phase entry points, aquakv_predict,
+ * aquakv_fit_predictor and aquakv_gather_rows; the chain, no-allocation and attention entry points return
+ * AQUAKV_ERR_UNSUPPORTED.
  */
 int aquakv_create(const aquakv_params* params, const float* grid_host, const int8_t* signs_k_host,
                   const int8_t* signs_v_host, aquakv_ctx** out);

@@ -173,15 +173,21 @@ class Codec:
     """One aquakv_ctx.  Tensors are torch CUDA tensors: 16-bit rows [T, d_kv] (stride(1) == 1),
     codes uint8 [T, code_bytes], scales float16 [T, d_kv/scale_group] (both contiguous)."""
 
-    def __init__(self, d_kv: int, had_block: int, scale_group: int, grid: np.ndarray, dtype: int,
-                 signs_k: np.ndarray, signs_v: np.ndarray):
-        self.params = Params(d_kv, had_block, scale_group, 2, int(np.asarray(grid).shape[0]), dtype)
-        g = np.ascontiguousarray(grid, dtype=np.float32)
-        sk = np.ascontiguousarray(signs_k, dtype=np.int8)
-        sv = np.ascontiguousarray(signs_v, dtype=np.int8)
+    def __init__(self, d_kv: int, had_block: int, scale_group: int, grid: Optional[np.ndarray], dtype: int,
+                 signs_k: Optional[np.ndarray] = None, signs_v: Optional[np.ndarray] = None, levels: int = 0):
+        """grid [n, 2] with sign vectors: the rotated 2-D vector quantizer.  grid None with `levels` = 2^b: the
+        uniform round-to-nearest backbone with absmax normalisation (had_block must be 1)."""
         h = ctypes.c_void_p()
-        rc = lib.aquakv_create(ctypes.byref(self.params), g.ctypes.data, sk.ctypes.data, sv.ctypes.data,
-                               ctypes.byref(h))
+        if grid is None:
+            self.params = Params(d_kv, had_block, scale_group, 1, int(levels), dtype)
+            rc = lib.aquakv_create(ctypes.byref(self.params), None, None, None, ctypes.byref(h))
+        else:
+            self.params = Params(d_kv, had_block, scale_group, 2, int(np.asarray(grid).shape[0]), dtype)
+            g = np.ascontiguousarray(grid, dtype=np.float32)
+            sk = np.ascontiguousarray(signs_k, dtype=np.int8)
+            sv = np.ascontiguousarray(signs_v, dtype=np.int8)
+            rc = lib.aquakv_create(ctypes.byref(self.params), g.ctypes.data, sk.ctypes.data, sv.ctypes.data,
+                                   ctypes.byref(h))
         if rc:
             raise AquaKVError(rc, "aquakv_create")
         self.h = h

@@ -28,6 +28,7 @@
 #include "gemm_pred.cuh"
 #include "layer_kernel.cuh"
 #include "search_table.h"
+#include "uniform.cuh"
 
 using namespace aquakv;
 
@@ -100,6 +101,15 @@ int check_params(const aquakv_params* p) {
   if (p->d_kv <= 0 || p->had_block <= 0 || p->scale_group <= 0 || p->grid_size <= 0)
     return AQUAKV_ERR_INVALID_ARG;
   if (p->dtype != AQUAKV_F16 && p->dtype != AQUAKV_BF16) return AQUAKV_ERR_INVALID_ARG;
+  if (p->grid_dim == 1) {
+    // uniform round-to-nearest backbone with absmax normalisation: grid_size = 2^b levels per value,
+    // no rotation (had_block 1), groups of 32 .. 256 values
+    if (p->d_kv != 256 && p->d_kv != 512 && p->d_kv != 1024) return AQUAKV_ERR_UNSUPPORTED;
+    if (p->grid_size != 4 && p->grid_size != 8 && p->grid_size != 16) return AQUAKV_ERR_UNSUPPORTED;
+    if (p->had_block != 1) return AQUAKV_ERR_UNSUPPORTED;
+    if (!is_pow2(p->scale_group) || p->scale_group < 32 || p->scale_group > 256) return AQUAKV_ERR_UNSUPPORTED;
+    return AQUAKV_OK;
+  }
   if (p->grid_dim != 2) return AQUAKV_ERR_UNSUPPORTED;
   if (p->d_kv != 256 && p->d_kv != 512 && p->d_kv != 1024) return AQUAKV_ERR_UNSUPPORTED;
   if (p->grid_size != 16 && p->grid_size != 64 && p->grid_size != 256) return AQUAKV_ERR_UNSUPPORTED;
@@ -236,9 +246,51 @@ CodecArgs codec_args(const aquakv_ctx* c, int role, int rows) {
 }
 
 // One phase of Algorithm 2 on `rows` rows: codes/scales = Q(X - P), hat = round16(P + Q^-1(..)).
+inline bool uniform_backbone(const aquakv_ctx* c) { return c->p.grid_dim == 1; }
+
+// Row kernels of the uniform backbone (uniform.cuh): X == nullptr decodes.
+int launch_uniform_rows(aquakv_ctx* c, cudaStream_t st, int rows, const void* X, int64_t ldX, const float* P,
+                        int64_t ldP, uint8_t* codes, uint16_t* scales, void* hat, int64_t ldHat) {
+  UniformArgs a;
+  a.X = static_cast<const uint16_t*>(X);
+  a.ldX = ldX;
+  a.P = P;
+  a.ldP = ldP;
+  a.codes = codes;
+  a.scales = scales;
+  a.hat = static_cast<uint16_t*>(hat);
+  a.ldHat = ldHat;
+  a.T = rows;
+  a.d = c->p.d_kv;
+  a.log_g = c->log_g;
+  int64_t blocks = (int64_t(rows) + kUniformWarps - 1) / kUniformWarps;
+  const int64_t cap = int64_t(c->sm_count) * 16;
+  if (blocks > cap) blocks = cap;
+  const int grid = int(blocks), threads = kUniformWarps * 32;
+  const bool enc = X != nullptr;
+  ProfScope prof(c, st, enc ? AQUAKV_KERNEL_ENCODE_ROWS : AQUAKV_KERNEL_DECODE_ROWS);
+#define AQ_UNIFORM(BITS)                                                                              \
+  do {                                                                                                \
+    if (enc) {                                                                                        \
+      if (c->bf16) uniform_encode_rows_kernel<BITS, true><<<grid, threads, 0, st>>>(a);               \
+      else uniform_encode_rows_kernel<BITS, false><<<grid, threads, 0, st>>>(a);                      \
+    } else {                                                                                          \
+      if (c->bf16) uniform_decode_rows_kernel<BITS, true><<<grid, threads, 0, st>>>(a);               \
+      else uniform_decode_rows_kernel<BITS, false><<<grid, threads, 0, st>>>(a);                      \
+    }                                                                                                 \
+  } while (0)
+  if (c->bits == 2) AQ_UNIFORM(2);
+  else if (c->bits == 3) AQ_UNIFORM(3);
+  else AQ_UNIFORM(4);
+#undef AQ_UNIFORM
+  ++c->launches;
+  return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
+}
+
 int launch_encode_rows(aquakv_ctx* c, cudaStream_t st, int role, int rows, const void* X,
                        int64_t ldX, const float* P, int64_t ldP, uint8_t* codes, uint16_t* scales,
                        void* hat, int64_t ldHat) {
+  if (uniform_backbone(c)) return launch_uniform_rows(c, st, rows, X, ldX, P, ldP, codes, scales, hat, ldHat);
   CodecArgs a = codec_args(c, role, rows);
   a.X = static_cast<const uint16_t*>(X);
   a.ldX = ldX;
@@ -259,6 +311,9 @@ int launch_encode_rows(aquakv_ctx* c, cudaStream_t st, int role, int rows, const
 int launch_decode_rows(aquakv_ctx* c, cudaStream_t st, int role, int rows, const uint8_t* codes,
                        const uint16_t* scales, const float* P, int64_t ldP, void* hat,
                        int64_t ldHat) {
+  if (uniform_backbone(c))
+    return launch_uniform_rows(c, st, rows, nullptr, 0, P, ldP, const_cast<uint8_t*>(codes),
+                               const_cast<uint16_t*>(scales), hat, ldHat);
   CodecArgs a = codec_args(c, role, rows);
   a.P = P;
   a.ldP = ldP;
@@ -739,6 +794,7 @@ int run_chain(aquakv_ctx* c, bool encode, int64_t T, int32_t L, const void* cons
               const void* const* Wv, const float* const* bk, const float* const* bv, uint8_t* const* Kcodes,
               uint16_t* const* Kscales, uint8_t* const* Vcodes, uint16_t* const* Vscales, void* const* Khat,
               void* const* Vhat, int64_t ld_hat, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (c != nullptr && uniform_backbone(c)) return AQUAKV_ERR_UNSUPPORTED;   // per-layer entry points only
   if (c == nullptr || T < 0 || L < 0) return AQUAKV_ERR_INVALID_ARG;
   if (T == 0 || L == 0) return AQUAKV_OK;
   if (T > kChainMaxTokens || L > kChainMaxLayers) return AQUAKV_ERR_TOO_LARGE;
@@ -847,6 +903,7 @@ extern "C" {
 int aquakv_code_bytes(const aquakv_params* params) {
   const int rc = check_params(params);
   if (rc) return rc;
+  if (params->grid_dim == 1) return params->d_kv * ilog2(params->grid_size) / 8;
   return params->d_kv / 2 * ilog2(params->grid_size) / 8;
 }
 
@@ -889,14 +946,17 @@ int aquakv_create(const aquakv_params* params, const float* grid_host, const int
   *out = nullptr;
   int rc = check_params(params);
   if (rc) return rc;
-  if (grid_host == nullptr || signs_k_host == nullptr || signs_v_host == nullptr)
+  const bool uniform = params->grid_dim == 1;      // its levels are implied: grid and signs are not read
+  if (!uniform && (grid_host == nullptr || signs_k_host == nullptr || signs_v_host == nullptr))
     return AQUAKV_ERR_INVALID_ARG;
   const int d = params->d_kv, n = params->grid_size;
-  for (int i = 0; i < 2 * n; ++i)
-    if (!std::isfinite(grid_host[i])) return AQUAKV_ERR_INVALID_ARG;
-  for (int i = 0; i < d; ++i) {
-    if (signs_k_host[i] != 1 && signs_k_host[i] != -1) return AQUAKV_ERR_INVALID_ARG;
-    if (signs_v_host[i] != 1 && signs_v_host[i] != -1) return AQUAKV_ERR_INVALID_ARG;
+  if (!uniform) {
+    for (int i = 0; i < 2 * n; ++i)
+      if (!std::isfinite(grid_host[i])) return AQUAKV_ERR_INVALID_ARG;
+    for (int i = 0; i < d; ++i) {
+      if (signs_k_host[i] != 1 && signs_k_host[i] != -1) return AQUAKV_ERR_INVALID_ARG;
+      if (signs_v_host[i] != 1 && signs_v_host[i] != -1) return AQUAKV_ERR_INVALID_ARG;
+    }
   }
   aquakv_ctx* c = new (std::nothrow) aquakv_ctx();
   if (c == nullptr) return AQUAKV_ERR_CUDA;
@@ -905,22 +965,26 @@ int aquakv_create(const aquakv_params* params, const float* grid_host, const int
   c->log_h = ilog2(params->had_block);
   c->log_g = ilog2(params->scale_group);
   c->bits = ilog2(n);
-  c->code_bytes = d / 2 * c->bits / 8;
+  c->code_bytes = uniform ? d * c->bits / 8 : d / 2 * c->bits / 8;
   c->n_groups = d / params->scale_group;
   c->bf16 = params->dtype == AQUAKV_BF16;
   c->attn_block_tokens = 1024;
 
   float4 g4[256];
-  for (int i = 0; i < n; ++i) {
-    const float gx = grid_host[2 * i], gy = grid_host[2 * i + 1];
-    g4[i] = make_float4(gx, gy, 0.0f, 0.0f);
+  std::memset(g4, 0, sizeof(g4));
+  std::vector<uint32_t> table(4, 0u);
+  if (!uniform) {
+    for (int i = 0; i < n; ++i) {
+      const float gx = grid_host[2 * i], gy = grid_host[2 * i + 1];
+      g4[i] = make_float4(gx, gy, 0.0f, 0.0f);
+    }
+    c->search_spec = search_table_spec(grid_host, n);
+    table.assign(search_table_words(c->search_spec), 0u);
+    build_search_table(grid_host, n, c->search_spec, table.data());
   }
-  c->search_spec = search_table_spec(grid_host, n);
-  std::vector<uint32_t> table(search_table_words(c->search_spec));
-  build_search_table(grid_host, n, c->search_spec, table.data());
   uint32_t masks[2][32];
   std::memset(masks, 0, sizeof(masks));
-  for (int role = 0; role < 2; ++role) {
+  for (int role = 0; role < 2 && !uniform; ++role) {
     const int8_t* s = role == kRoleK ? signs_k_host : signs_v_host;
     for (int e = 0; e < d; ++e)
       if (s[e] < 0) masks[role][(e >> 3) & 31] |= 1u << (((e >> 8) << 3) | (e & 7));
@@ -984,7 +1048,9 @@ int aquakv_destroy(aquakv_ctx* c) {
 size_t aquakv_workspace_bytes(const aquakv_ctx* c, int64_t n_tokens, int op) {
   if (c == nullptr || n_tokens <= 0) return 0;
   if (op == AQUAKV_OP_ENCODE || op == AQUAKV_OP_DECODE) {
-    const size_t phase_bytes = encode_ws(c, n_tokens).total, layer_bytes = layer_ws(c, n_tokens).total;
+    const size_t phase_bytes = encode_ws(c, n_tokens).total;
+    if (uniform_backbone(c)) return phase_bytes;
+    const size_t layer_bytes = layer_ws(c, n_tokens).total;
     return phase_bytes > layer_bytes ? phase_bytes : layer_bytes;
   }
   return 0;
@@ -992,6 +1058,7 @@ size_t aquakv_workspace_bytes(const aquakv_ctx* c, int64_t n_tokens, int op) {
 
 size_t aquakv_decode_attn_workspace_bytes(const aquakv_ctx* c, int32_t batch, int64_t ctx_len,
                                           int32_t n_q_heads, int32_t head_dim) {
+  if (c != nullptr && uniform_backbone(c)) return 0;
   if (c == nullptr || batch <= 0 || ctx_len <= 0 || n_q_heads <= 0 || head_dim <= 0) return 0;
   // the caller may or may not pass predictors: the larger of the two layouts
   const size_t a = attn_ws(c, batch, ctx_len, n_q_heads, head_dim, true).total;
@@ -1323,6 +1390,16 @@ int aquakv_encode(aquakv_ctx* c, int64_t n_tokens, const void* K, const void* V,
       return AQUAKV_ERR_WORKSPACE;
     if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
   }
+  if (has_pred && uniform_backbone(c)) {
+    // no fused kernel for this backbone: the key phase, then the value phase on the reconstructed keys
+    if (Khat == nullptr) return AQUAKV_ERR_INVALID_ARG;
+    if (ld_prev != ld_hat) return AQUAKV_ERR_UNSUPPORTED;   // the value phase reads both inputs with one stride
+    if ((rc = aquakv_encode_phase(c, AQUAKV_ROLE_KEY, n_tokens, K, ld_kv, Khat_prev, nullptr, ld_prev, Wk, bk, Kcodes,
+                                  Kscales, Khat, ld_hat, workspace, workspace_bytes, cuda_stream)))
+      return rc;
+    return aquakv_encode_phase(c, AQUAKV_ROLE_VALUE, n_tokens, V, ld_kv, Vhat_prev, Khat, ld_prev, Wv, bv, Vcodes,
+                               Vscales, Vhat, ld_hat, workspace, workspace_bytes, cuda_stream);
+  }
   if (has_pred) {
     if (n_tokens > (int64_t(1) << 30)) return AQUAKV_ERR_UNSUPPORTED;
     return launch_layer(c, static_cast<cudaStream_t>(cuda_stream), true, n_tokens, K, V, ld_kv, Khat_prev,
@@ -1370,6 +1447,14 @@ int aquakv_decode(aquakv_ctx* c, int64_t n_tokens, const uint8_t* Kcodes, const 
     if (workspace == nullptr || workspace_bytes < aquakv_workspace_bytes(c, n_tokens, AQUAKV_OP_DECODE))
       return AQUAKV_ERR_WORKSPACE;
     if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
+    if (uniform_backbone(c)) {
+      if (ld_prev != ld_hat) return AQUAKV_ERR_UNSUPPORTED;
+      if ((rc = aquakv_decode_phase(c, AQUAKV_ROLE_KEY, n_tokens, Kcodes, Kscales, Khat_prev, nullptr, ld_prev, Wk, bk,
+                                    Khat, ld_hat, workspace, workspace_bytes, cuda_stream)))
+        return rc;
+      return aquakv_decode_phase(c, AQUAKV_ROLE_VALUE, n_tokens, Vcodes, Vscales, Vhat_prev, Khat, ld_prev, Wv, bv,
+                                 Vhat, ld_hat, workspace, workspace_bytes, cuda_stream);
+    }
     if (n_tokens > (int64_t(1) << 30)) return AQUAKV_ERR_UNSUPPORTED;
     return launch_layer(c, static_cast<cudaStream_t>(cuda_stream), false, n_tokens, nullptr, nullptr, 0,
                         Khat_prev, Vhat_prev, ld_prev, Wk, Wv, bk, bv, const_cast<uint8_t*>(Kcodes),
@@ -1395,6 +1480,7 @@ int aquakv_decode(aquakv_ctx* c, int64_t n_tokens, const uint8_t* Kcodes, const 
 }
 
 size_t aquakv_chain_workspace_bytes(const aquakv_ctx* c, int64_t n_tokens, int32_t n_layers) {
+  if (c != nullptr && uniform_backbone(c)) return 0;
   if (c == nullptr || n_tokens <= 0 || n_layers <= 0 || n_tokens > kChainMaxTokens || n_layers > kChainMaxLayers) return 0;
   return chain_ws(c, n_tokens, n_layers).total;
 }
@@ -1458,6 +1544,7 @@ int aquakv_decode_noalloc(aquakv_ctx* c, int64_t n_tokens, const uint8_t* Kcodes
                           const void* Khat_prev, const void* Vhat_prev, int64_t ld_prev,
                           const void* Wk, const void* Wv, const float* bk, const float* bv,
                           void* Khat, void* Vhat, int64_t ld_hat, void* cuda_stream) {
+  if (c != nullptr && uniform_backbone(c)) return AQUAKV_ERR_UNSUPPORTED;
   if (c == nullptr || n_tokens < 0) return AQUAKV_ERR_INVALID_ARG;
   if (n_tokens > AQUAKV_NOALLOC_MAX_TOKENS) return AQUAKV_ERR_TOO_LARGE;
   if (n_tokens == 0) return AQUAKV_OK;
@@ -1491,6 +1578,7 @@ int aquakv_decode_attn(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_
                        int64_t ld_prev, const void* Wk, const void* Wv, const float* bk,
                        const float* bv, void* out, float* lse, void* Khat, void* Vhat,
                        int64_t ld_hat, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (c != nullptr && uniform_backbone(c)) return AQUAKV_ERR_UNSUPPORTED;
   if (c == nullptr || batch < 0 || ctx_len < 0) return AQUAKV_ERR_INVALID_ARG;
   if (batch == 0 || ctx_len == 0) return AQUAKV_OK;
   const int d = c->p.d_kv;

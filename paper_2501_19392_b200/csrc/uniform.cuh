@@ -1,0 +1,158 @@
+// Alternative backbone quantizer (Section 4.1 "Alternative quantizers": Quanto-style "simple
+// round-to-nearest quantization with absmax normalization", "group size 64 and per-token compression";
+// Section 3.2: the method is agnostic to the choice of Q) for the residual / add-back steps of
+// Algorithm 2 (lines 6-7, 9) and Algorithm 3 (lines 5, 7).
+//
+// For b bits per value the levels are the 2^b signed integers -2^(b-1) .. 2^(b-1)-1 times the group
+// scale; scale = absmax / 2^(b-1), stored as fp16 (clamped to 65504), and the ROUNDED scale normalises;
+// a value goes to the nearest level, the lower one on an exact tie, saturating at the ends; a group of
+// zeros has scale 0 and level 0.  The code of a value is level + 2^(b-1); codes are packed LSB-first in
+// value order.  No rotation, no sign flips.
+//
+// One warp per row.  Lane L holds the 8 consecutive values 256 c + 8 L .. + 7 of every 256-value chunk c
+// (16-byte accesses); a group of g values (32 <= g <= 256) is g/8 neighbouring lanes, so its absmax is
+// log2(g/8) shuffle steps.  The lane's 8 codes are b contiguous bytes of the row's code stream.
+#pragma once
+
+#include "codec.cuh"
+
+namespace aquakv {
+
+struct UniformArgs {
+  const uint16_t* X;        // encode: target rows (16-bit) [T, ldX]
+  long long ldX;
+  const float* P;           // prediction rows (fp32) or nullptr [T, ldP]
+  long long ldP;
+  uint8_t* codes;           // [T, d * b / 8]
+  uint16_t* scales;         // [T, d / g] fp16 bits
+  uint16_t* hat;            // reconstruction rows or nullptr (encode) [T, ldHat]
+  long long ldHat;
+  int T;
+  int d;                    // 256, 512 or 1024
+  int log_g;                // 5 .. 8
+};
+
+constexpr int kUniformWarps = 4;
+
+template <bool kBf16>
+__device__ __forceinline__ void uniform_store8(uint16_t* dst, const float (&v)[8]) {
+  uint4 out;
+  out.x = store16x2p<kBf16>(pack2(v[0], v[1]));
+  out.y = store16x2p<kBf16>(pack2(v[2], v[3]));
+  out.z = store16x2p<kBf16>(pack2(v[4], v[5]));
+  out.w = store16x2p<kBf16>(pack2(v[6], v[7]));
+  __stcs(reinterpret_cast<uint4*>(dst), out);
+}
+
+__device__ __forceinline__ void uniform_load_pred8(const float* p, float (&v)[8]) {
+  const float4 a = __ldcs(reinterpret_cast<const float4*>(p));
+  const float4 b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+  v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+
+// codes, scales = Q(x - pred);  hat = round16(pred + Q^-1(codes, scales)).
+template <int BITS, bool kBf16>
+__global__ void __launch_bounds__(kUniformWarps * 32)
+uniform_encode_rows_kernel(const UniformArgs a) {
+  constexpr int HALF = 1 << (BITS - 1);
+  const int lane = threadIdx.x & 31;
+  const long long warp = (long long)blockIdx.x * kUniformWarps + (threadIdx.x >> 5);
+  const long long n_warps = (long long)gridDim.x * kUniformWarps;
+  const int lanes_per_group = 1 << (a.log_g - 3);
+  const int n_groups = a.d >> a.log_g;
+  for (long long t = warp; t < a.T; t += n_warps) {
+    for (int c = 0; c < a.d / 256; ++c) {
+      const int e0 = 256 * c + 8 * lane;
+      float r[8], pred[8];
+      {
+        const uint4 raw = __ldcs(reinterpret_cast<const uint4*>(a.X + t * a.ldX + e0));
+        float lo, hi;
+        unpack2(load16x2<kBf16>(raw.x), lo, hi); r[0] = lo; r[1] = hi;
+        unpack2(load16x2<kBf16>(raw.y), lo, hi); r[2] = lo; r[3] = hi;
+        unpack2(load16x2<kBf16>(raw.z), lo, hi); r[4] = lo; r[5] = hi;
+        unpack2(load16x2<kBf16>(raw.w), lo, hi); r[6] = lo; r[7] = hi;
+      }
+      if (a.P != nullptr) {
+        uniform_load_pred8(a.P + t * a.ldP + e0, pred);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) r[i] -= pred[i];
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) pred[i] = 0.0f;
+      }
+      float m = 0.0f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) m = fmaxf(m, fabsf(r[i]));
+      for (int off = 1; off < lanes_per_group; off <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+      const __half s16 = __float2half_rn(fminf(m * (1.0f / HALF), 65504.0f));
+      const float sf = __half2float(s16);
+      if ((lane & (lanes_per_group - 1)) == 0)
+        a.scales[t * n_groups + ((e0) >> a.log_g)] = __half_as_ushort(s16);
+      uint32_t word = 0;
+      float q[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        // nearest level, the lower one on a tie: ceil(x - 0.5); the division is IEEE
+        const float x = sf > 0.0f ? __fdiv_rn(r[i], sf) : 0.0f;
+        float lv = ceilf(x - 0.5f);
+        lv = fminf(fmaxf(lv, float(-HALF)), float(HALF - 1));
+        q[i] = lv;
+        word |= uint32_t(int(lv) + HALF) << (BITS * i);
+      }
+      uint8_t* cdst = a.codes + t * (long long)(a.d * BITS / 8) + (32 * c + lane) * BITS;
+      if constexpr (BITS == 2) {
+        *reinterpret_cast<uint16_t*>(cdst) = uint16_t(word);
+      } else if constexpr (BITS == 4) {
+        *reinterpret_cast<uint32_t*>(cdst) = word;
+      } else {
+        cdst[0] = uint8_t(word);
+        cdst[1] = uint8_t(word >> 8);
+        cdst[2] = uint8_t(word >> 16);
+      }
+      if (a.hat != nullptr) {
+        float h[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) h[i] = fmaf(q[i], sf, pred[i]);
+        uniform_store8<kBf16>(a.hat + t * a.ldHat + e0, h);
+      }
+    }
+  }
+}
+
+// hat = round16(pred + Q^-1(codes, scales)).
+template <int BITS, bool kBf16>
+__global__ void __launch_bounds__(kUniformWarps * 32)
+uniform_decode_rows_kernel(const UniformArgs a) {
+  constexpr int HALF = 1 << (BITS - 1);
+  const int lane = threadIdx.x & 31;
+  const long long warp = (long long)blockIdx.x * kUniformWarps + (threadIdx.x >> 5);
+  const long long n_warps = (long long)gridDim.x * kUniformWarps;
+  const int n_groups = a.d >> a.log_g;
+  for (long long t = warp; t < a.T; t += n_warps) {
+    for (int c = 0; c < a.d / 256; ++c) {
+      const int e0 = 256 * c + 8 * lane;
+      const uint8_t* csrc = a.codes + t * (long long)(a.d * BITS / 8) + (32 * c + lane) * BITS;
+      uint32_t word;
+      if constexpr (BITS == 2) word = *reinterpret_cast<const uint16_t*>(csrc);
+      else if constexpr (BITS == 4) word = *reinterpret_cast<const uint32_t*>(csrc);
+      else word = uint32_t(csrc[0]) | (uint32_t(csrc[1]) << 8) | (uint32_t(csrc[2]) << 16);
+      const float sf = __half2float(__ushort_as_half(a.scales[t * n_groups + (e0 >> a.log_g)]));
+      float pred[8], h[8];
+      if (a.P != nullptr) {
+        uniform_load_pred8(a.P + t * a.ldP + e0, pred);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) pred[i] = 0.0f;
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float lv = float(int((word >> (BITS * i)) & uint32_t((1 << BITS) - 1)) - HALF);
+        h[i] = fmaf(lv, sf, pred[i]);
+      }
+      uniform_store8<kBf16>(a.hat + t * a.ldHat + e0, h);
+    }
+  }
+}
+
+}  // namespace aquakv
