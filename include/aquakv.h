@@ -334,6 +334,30 @@ int aquakv_decode_attn(aquakv_ctx* ctx, int32_t batch, int64_t ctx_len,
                        void* Khat, void* Vhat, int64_t ld_hat,
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * The same with the cache policy of Section 3.3 / Section 4.1 around it: "the first 4 tokens (attention
+ * sinks)" and "a buffer of 128 most recent tokens" stay uncompressed, and every query attends to both
+ * the compressed cache and those rows.  K16 / V16: [batch][n_uncompressed][ld16] 16-bit rows of the
+ * ctx's type (device, 16-byte aligned, ld16 >= d_kv and a multiple of 8), each sequence's uncompressed
+ * rows in any order (attention does not depend on it; position encoding is the caller's business, as in
+ * aquakv_decode_attn).  Their split-KV partials are formed by the library's attention kernel and merged
+ * with the partials of the compressed cache in fp32 before the single rounding of `out`, so the result
+ * is the attention over the concatenation [compressed ; uncompressed] (Algorithm 4 lines 5-9 with
+ * the buffered rows appended to the decoded ones).  ctx_len may be 0 (nothing compressed yet: the cache
+ * pointers are then ignored), n_uncompressed may be 0 (identical to aquakv_decode_attn); both 0 does
+ * nothing.  Workspace: aquakv_decode_attn_buffered_workspace_bytes.  Everything else as aquakv_decode_attn.
+ */
+size_t aquakv_decode_attn_buffered_workspace_bytes(const aquakv_ctx* ctx, int32_t batch, int64_t ctx_len,
+                                                   int64_t n_uncompressed, int32_t n_q_heads, int32_t head_dim);
+int aquakv_decode_attn_buffered(aquakv_ctx* ctx, int32_t batch, int64_t ctx_len, int32_t n_q_heads,
+                                int32_t n_kv_heads, int32_t head_dim, float softmax_scale, const void* q,
+                                const uint8_t* Kcodes, const uint16_t* Kscales, const uint8_t* Vcodes,
+                                const uint16_t* Vscales, const void* Khat_prev, const void* Vhat_prev,
+                                int64_t ld_prev, const void* Wk, const void* Wv, const float* bk,
+                                const float* bv, const void* K16, const void* V16, int64_t n_uncompressed,
+                                int64_t ld16, void* out, float* lse, void* Khat, void* Vhat, int64_t ld_hat,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Row gather for compressing a subset of the tokens (Section 4.3: a pruning policy such as H2O
  * selects the tokens to keep, "and [we] apply AQUA-KV compression [to] those tokens"): dst row i =

@@ -37,6 +37,7 @@ SYMBOLS = [
     "aquakv_profile_enable", "aquakv_profile_read", "aquakv_selftest_bounded_wait",
     "aquakv_chain_workspace_bytes", "aquakv_encode_chain", "aquakv_decode_chain",
     "aquakv_fit_workspace_bytes", "aquakv_fit_predictor", "aquakv_gather_rows",
+    "aquakv_decode_attn_buffered_workspace_bytes", "aquakv_decode_attn_buffered",
 ]
 
 
@@ -98,6 +99,12 @@ def _load():
     L.aquakv_profile_enable.argtypes = [vp, ctypes.c_int]
     L.aquakv_profile_read.restype = ctypes.c_int
     L.aquakv_profile_read.argtypes = [vp, ctypes.c_int, ctypes.POINTER(i64), ctypes.POINTER(ctypes.c_double)]
+    L.aquakv_decode_attn_buffered_workspace_bytes.restype = sz
+    L.aquakv_decode_attn_buffered_workspace_bytes.argtypes = [vp, i32, i64, i64, i32, i32]
+    L.aquakv_decode_attn_buffered.restype = ctypes.c_int
+    L.aquakv_decode_attn_buffered.argtypes = [vp, i32, i64, i32, i32, i32, f32, vp, vp, vp, vp, vp,
+                                              vp, vp, i64, vp, vp, vp, vp, vp, vp, i64, i64, vp, vp, vp, vp, i64,
+                                              vp, sz, vp]
     L.aquakv_gather_rows.restype = ctypes.c_int
     L.aquakv_gather_rows.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp]
     L.aquakv_fit_workspace_bytes.restype = sz
@@ -335,6 +342,32 @@ class Codec:
         if rc:
             raise AquaKVError(rc, "aquakv_fit_predictor")
         return W, bias, W32
+
+    def decode_attn_buffered(self, q, Kcodes, Kscales, Vcodes, Vscales, ctx_len: int, n_kv_heads: int,
+                             softmax_scale: float, K16, V16, Khat_prev=None, Vhat_prev=None, Wk=None, Wv=None,
+                             bk=None, bv=None, out=None, lse=None, Khat=None, Vhat=None, want_lse: bool = False,
+                             workspace=None):
+        """decode_attn over the compressed cache plus uncompressed rows K16 / V16 [batch, n, d] (sinks, recent
+        tokens); ctx_len may be 0."""
+        batch, n_q_heads, head_dim = q.shape
+        dev = q.device
+        n16 = 0 if K16 is None else K16.shape[1]
+        if out is None:
+            out = torch.empty_like(q)
+        if want_lse and lse is None:
+            lse = torch.empty((batch, n_q_heads), dtype=torch.float32, device=dev)
+        ws = workspace if workspace is not None else self._workspace(int(
+            lib.aquakv_decode_attn_buffered_workspace_bytes(self.h, batch, ctx_len, n16, n_q_heads, head_dim)), dev)
+        ld16 = self.d if K16 is None else int(K16.stride(1))
+        rc = lib.aquakv_decode_attn_buffered(self.h, batch, ctx_len, n_q_heads, n_kv_heads, head_dim, softmax_scale,
+                                             _ptr(q), _ptr(Kcodes), _ptr(Kscales), _ptr(Vcodes), _ptr(Vscales),
+                                             _ptr(Khat_prev), _ptr(Vhat_prev), _ld(Khat_prev, self.d), _ptr(Wk),
+                                             _ptr(Wv), _ptr(bk), _ptr(bv), _ptr(K16), _ptr(V16), n16, ld16, _ptr(out),
+                                             _ptr(lse), _ptr(Khat), _ptr(Vhat), _ld(Khat, self.d), _ptr(ws),
+                                             ws.numel(), _stream())
+        if rc:
+            raise AquaKVError(rc, "aquakv_decode_attn_buffered")
+        return out, lse
 
     def encode_phase(self, role: int, X, in0=None, in1=None, W=None, bias=None, want_hat: bool = True):
         T, dev = X.shape[0], X.device

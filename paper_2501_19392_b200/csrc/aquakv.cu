@@ -1571,17 +1571,85 @@ int aquakv_decode_noalloc(aquakv_ctx* c, int64_t n_tokens, const uint8_t* Kcodes
   return launch_decode_rows(c, st, kRoleV, rows, Vcodes, Vscales, P, d, Vh, ld_hat);
 }
 
-int aquakv_decode_attn(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_heads,
-                       int32_t n_kv_heads, int32_t head_dim, float softmax_scale, const void* q,
-                       const uint8_t* Kcodes, const uint16_t* Kscales, const uint8_t* Vcodes,
-                       const uint16_t* Vscales, const void* Khat_prev, const void* Vhat_prev,
-                       int64_t ld_prev, const void* Wk, const void* Wv, const float* bk,
-                       const float* bv, void* out, float* lse, void* Khat, void* Vhat,
-                       int64_t ld_hat, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+// Partial-result arrays of the uncompressed rows that are attended to beside the compressed cache.
+struct AttnExtWs {
+  size_t ml_off, o_off, total;
+  int splits;
+};
+static AttnExtWs attn_ext_ws(const aquakv_ctx* c, size_t base_total, int32_t batch, int64_t n16, int32_t n_q_heads,
+                             int32_t head_dim) {
+  AttnExtWs w;
+  const int tb = c->attn_block_tokens;
+  w.splits = n16 > 0 ? int((n16 + tb - 1) / tb) : 0;
+  const size_t slots = size_t(batch) * size_t(w.splits);
+  w.ml_off = round_up(base_total, 256);
+  w.o_off = w.ml_off + round_up(slots * n_q_heads * 2 * sizeof(float), 256);
+  w.total = w.o_off + round_up(slots * n_q_heads * head_dim * sizeof(float), 256) + kWsSlack;
+  return w;
+}
+
+static int decode_attn_impl(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_heads,
+                            int32_t n_kv_heads, int32_t head_dim, float softmax_scale, const void* q,
+                            const uint8_t* Kcodes, const uint16_t* Kscales, const uint8_t* Vcodes,
+                            const uint16_t* Vscales, const void* Khat_prev, const void* Vhat_prev,
+                            int64_t ld_prev, const void* Wk, const void* Wv, const float* bk,
+                            const float* bv, void* out, float* lse, void* Khat, void* Vhat,
+                            int64_t ld_hat, const void* K16, const void* V16, int64_t n16, int64_t ld16,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream) {
   if (c != nullptr && uniform_backbone(c)) return AQUAKV_ERR_UNSUPPORTED;
-  if (c == nullptr || batch < 0 || ctx_len < 0) return AQUAKV_ERR_INVALID_ARG;
-  if (batch == 0 || ctx_len == 0) return AQUAKV_OK;
+  if (c == nullptr || batch < 0 || ctx_len < 0 || n16 < 0) return AQUAKV_ERR_INVALID_ARG;
+  if (batch == 0 || (ctx_len == 0 && n16 == 0)) return AQUAKV_OK;
   const int d = c->p.d_kv;
+  if (n16 > 0) {
+    int rc16;
+    if ((rc16 = check_rows(K16, ld16, d, true))) return rc16;
+    if ((rc16 = check_rows(V16, ld16, d, true))) return rc16;
+    if (n16 > (int64_t(1) << 24)) return AQUAKV_ERR_UNSUPPORTED;
+  }
+  if (ctx_len == 0) {
+    // nothing compressed yet: the uncompressed rows alone
+    if (n_q_heads <= 0 || n_kv_heads <= 0 || head_dim <= 0) return AQUAKV_ERR_INVALID_ARG;
+    if (n_kv_heads * head_dim != d || n_q_heads % n_kv_heads) return AQUAKV_ERR_INVALID_ARG;
+    if ((head_dim != 64 && head_dim != 128) || n_q_heads / n_kv_heads > kAttnMmaMaxGq) return AQUAKV_ERR_UNSUPPORTED;
+    if (q == nullptr || out == nullptr) return AQUAKV_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out)) return AQUAKV_ERR_ALIGNMENT;
+    if (!(softmax_scale == softmax_scale)) return AQUAKV_ERR_INVALID_ARG;
+    const AttnExtWs xw = attn_ext_ws(c, 0, batch, n16, n_q_heads, head_dim);
+    if (workspace == nullptr || workspace_bytes < xw.total) return AQUAKV_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
+    cudaStream_t st0 = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* wsb0 = ws_base(workspace);
+    AttnArgs a;
+    a.q = static_cast<const uint16_t*>(q);
+    a.Kh = static_cast<const uint16_t*>(K16);
+    a.Vh = static_cast<const uint16_t*>(V16);
+    a.ld = ld16;
+    a.tok_base = 0;
+    a.blk_begin = 0;
+    a.ctx = int(n16);
+    a.n_q_heads = n_q_heads;
+    a.n_kv_heads = n_kv_heads;
+    a.n_splits = xw.splits;
+    a.block_tokens = c->attn_block_tokens;
+    a.scale_log2 = softmax_scale * 1.4426950408889634f;
+    a.part_ml = reinterpret_cast<float*>(wsb0 + xw.ml_off);
+    a.part_o = reinterpret_cast<float*>(wsb0 + xw.o_off);
+    int rc0 = launch_attn_partial(c, st0, a, head_dim, batch * xw.splits);
+    if (rc0) return rc0;
+    AttnCombineArgs ca;
+    ca.part_ml = a.part_ml;
+    ca.part_o = a.part_o;
+    ca.out = static_cast<uint16_t*>(out);
+    ca.lse = lse;
+    ca.n_q_heads = n_q_heads;
+    ca.n_splits = xw.splits;
+    ca.ctx = int(n16);
+    ca.block_tokens = 0;
+    ca.extra_ml = nullptr;
+    ca.extra_o = nullptr;
+    ca.extra_splits = 0;
+    return launch_attn_combine(c, st0, ca, head_dim, batch);
+  }
   if (n_q_heads <= 0 || n_kv_heads <= 0 || head_dim <= 0) return AQUAKV_ERR_INVALID_ARG;
   if (n_kv_heads * head_dim != d || n_q_heads % n_kv_heads) return AQUAKV_ERR_INVALID_ARG;
   if ((head_dim != 64 && head_dim != 128) || n_q_heads / n_kv_heads > kAttnMmaMaxGq)
@@ -1603,8 +1671,34 @@ int aquakv_decode_attn(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_
                           Vhat == Khat_prev || Vhat == Khat))
     return AQUAKV_ERR_INVALID_ARG;
   const AttnWs ws = attn_ws(c, batch, ctx_len, n_q_heads, head_dim, has_pred);
-  if (workspace == nullptr || workspace_bytes < ws.total) return AQUAKV_ERR_WORKSPACE;
+  const AttnExtWs xw = attn_ext_ws(c, ws.total, batch, n16, n_q_heads, head_dim);
+  if (workspace == nullptr || workspace_bytes < (n16 > 0 ? xw.total : ws.total)) return AQUAKV_ERR_WORKSPACE;
   if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
+  // partials of the uncompressed rows (attention sinks, recent-token buffer), merged by the combine kernel
+  const float* extra_ml = nullptr;
+  const float* extra_o = nullptr;
+  if (n16 > 0) {
+    uint8_t* wsx = ws_base(workspace);
+    AttnArgs a;
+    a.q = static_cast<const uint16_t*>(q);
+    a.Kh = static_cast<const uint16_t*>(K16);
+    a.Vh = static_cast<const uint16_t*>(V16);
+    a.ld = ld16;
+    a.tok_base = 0;
+    a.blk_begin = 0;
+    a.ctx = int(n16);
+    a.n_q_heads = n_q_heads;
+    a.n_kv_heads = n_kv_heads;
+    a.n_splits = xw.splits;
+    a.block_tokens = c->attn_block_tokens;
+    a.scale_log2 = softmax_scale * 1.4426950408889634f;
+    a.part_ml = reinterpret_cast<float*>(wsx + xw.ml_off);
+    a.part_o = reinterpret_cast<float*>(wsx + xw.o_off);
+    if ((rc = launch_attn_partial(c, static_cast<cudaStream_t>(cuda_stream), a, head_dim, batch * xw.splits))) return rc;
+    extra_ml = a.part_ml;
+    extra_o = a.part_o;
+  }
+  const int extra_splits = n16 > 0 ? xw.splits : 0;
   if (ws.fused) {
     // Algorithm 3 and the attention read of Algorithm 4 in ONE launch: the attention warps of the layer
     // kernel consume every token block's decoded rows from L2 as soon as they exist
@@ -1634,6 +1728,9 @@ int aquakv_decode_attn(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_
     ca.n_splits = ws.n_splits;
     ca.ctx = int(ctx_len);
     ca.block_tokens = kAttnSubTokens;
+    ca.extra_ml = extra_ml;
+    ca.extra_o = extra_o;
+    ca.extra_splits = extra_splits;
     return launch_attn_combine(c, st, ca, head_dim, batch);
   }
 
@@ -1698,7 +1795,43 @@ int aquakv_decode_attn(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_
   ca.n_splits = ws.n_splits;
   ca.ctx = int(ctx_len);
   ca.block_tokens = 0;
+  ca.extra_ml = extra_ml;
+  ca.extra_o = extra_o;
+  ca.extra_splits = extra_splits;
   return launch_attn_combine(c, st, ca, head_dim, batch);
+}
+
+int aquakv_decode_attn(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_heads,
+                       int32_t n_kv_heads, int32_t head_dim, float softmax_scale, const void* q,
+                       const uint8_t* Kcodes, const uint16_t* Kscales, const uint8_t* Vcodes,
+                       const uint16_t* Vscales, const void* Khat_prev, const void* Vhat_prev,
+                       int64_t ld_prev, const void* Wk, const void* Wv, const float* bk,
+                       const float* bv, void* out, float* lse, void* Khat, void* Vhat,
+                       int64_t ld_hat, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return decode_attn_impl(c, batch, ctx_len, n_q_heads, n_kv_heads, head_dim, softmax_scale, q, Kcodes, Kscales, Vcodes,
+                          Vscales, Khat_prev, Vhat_prev, ld_prev, Wk, Wv, bk, bv, out, lse, Khat, Vhat, ld_hat, nullptr,
+                          nullptr, 0, 0, workspace, workspace_bytes, cuda_stream);
+}
+
+size_t aquakv_decode_attn_buffered_workspace_bytes(const aquakv_ctx* c, int32_t batch, int64_t ctx_len,
+                                                   int64_t n_uncompressed, int32_t n_q_heads, int32_t head_dim) {
+  if (c == nullptr || batch <= 0 || ctx_len < 0 || n_uncompressed < 0 || n_q_heads <= 0 || head_dim <= 0) return 0;
+  if (uniform_backbone(c)) return 0;
+  const size_t base = ctx_len > 0 ? aquakv_decode_attn_workspace_bytes(c, batch, ctx_len, n_q_heads, head_dim) : 0;
+  return attn_ext_ws(c, base, batch, n_uncompressed, n_q_heads, head_dim).total;
+}
+
+int aquakv_decode_attn_buffered(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_heads,
+                                int32_t n_kv_heads, int32_t head_dim, float softmax_scale, const void* q,
+                                const uint8_t* Kcodes, const uint16_t* Kscales, const uint8_t* Vcodes,
+                                const uint16_t* Vscales, const void* Khat_prev, const void* Vhat_prev,
+                                int64_t ld_prev, const void* Wk, const void* Wv, const float* bk,
+                                const float* bv, const void* K16, const void* V16, int64_t n_uncompressed,
+                                int64_t ld16, void* out, float* lse, void* Khat, void* Vhat, int64_t ld_hat,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return decode_attn_impl(c, batch, ctx_len, n_q_heads, n_kv_heads, head_dim, softmax_scale, q, Kcodes, Kscales, Vcodes,
+                          Vscales, Khat_prev, Vhat_prev, ld_prev, Wk, Wv, bk, bv, out, lse, Khat, Vhat, ld_hat, K16, V16,
+                          n_uncompressed, ld16, workspace, workspace_bytes, cuda_stream);
 }
 
 }  // extern "C"

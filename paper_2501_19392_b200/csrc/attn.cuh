@@ -385,6 +385,11 @@ struct AttnCombineArgs {
   int ctx;            // tokens per sequence
   int block_tokens;   // > 0: partials per block of that many tokens of the FLATTENED token index (a sequence
                       // uses as many slots as blocks overlap it); 0: every sequence uses all n_splits slots
+  // a second set of partials per sequence, merged after the first (the uncompressed rows a cache policy keeps
+  // beside the compressed ones: attention sinks and the recent-token buffer, Section 3.3); 0 slots = none
+  const float* extra_ml;   // [batch][extra_splits][n_q_heads][2]
+  const float* extra_o;    // [batch][extra_splits][n_q_heads][HD]
+  int extra_splits;
 };
 
 // One CTA per (sequence, query head); thread i owns output dimension i.
@@ -393,10 +398,14 @@ __global__ void __launch_bounds__(HD) attn_combine_kernel(const AttnCombineArgs 
   const int b = blockIdx.x / a.n_q_heads, qh = blockIdx.x % a.n_q_heads;
   const int i = threadIdx.x;
   int n_s = a.n_splits;
-  if (a.block_tokens > 0) {
+  if (a.ctx == 0) {
+    n_s = 0;
+  } else if (a.block_tokens > 0) {
     const long long t0 = (long long)b * a.ctx, t1 = t0 + a.ctx - 1;
     n_s = int(t1 / a.block_tokens - t0 / a.block_tokens) + 1;
   }
+  const float* xml = a.extra_ml + ((long long)b * a.extra_splits * a.n_q_heads + qh) * 2;
+  const float* xpo = a.extra_o + ((long long)b * a.extra_splits * a.n_q_heads + qh) * HD + i;
   // Both passes keep several independent loads in flight: with many slots per sequence the kernel is
   // bound by the latency of its loads, not by their number.
   const float* ml = a.part_ml + ((long long)b * a.n_splits * a.n_q_heads + qh) * 2;
@@ -411,6 +420,7 @@ __global__ void __launch_bounds__(HD) attn_combine_kernel(const AttnCombineArgs 
       for (int u = 0; u < 4; ++u) m4[u] = fmaxf(m4[u], ml[(s + u) * ml_step]);
     }
     for (; s < n_s; ++s) m4[0] = fmaxf(m4[0], ml[s * ml_step]);
+    for (int x = 0; x < a.extra_splits; ++x) m4[1] = fmaxf(m4[1], xml[x * ml_step]);
     M = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
   }
   float L = 0.0f, o = 0.0f;
@@ -435,6 +445,11 @@ __global__ void __launch_bounds__(HD) attn_combine_kernel(const AttnCombineArgs 
       const float w = exp2f(ml[s * ml_step] - M);
       L = fmaf(ml[s * ml_step + 1], w, L);
       o = fmaf(po[s * o_step], w, o);
+    }
+    for (int x = 0; x < a.extra_splits; ++x) {
+      const float w = exp2f(xml[x * ml_step] - M);
+      L = fmaf(xml[x * ml_step + 1], w, L);
+      o = fmaf(xpo[x * o_step], w, o);
     }
   }
   a.out[((long long)b * a.n_q_heads + qh) * HD + i] = store16<kBf16>(o / L);
