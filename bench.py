@@ -351,6 +351,19 @@ def ops_by_config(api, chain, peaks, dev, reps=5):
     ms = _time_calls(one, max(2, reps // 2), warm=2)
     out.append(_shape_entry(peaks, shape, "decode_attn", T, ms, _shape_bytes(shape, T, False, write_hat=False),
                             config=5, batch=shape.batch, ctx=ctx_len, n_q_heads=shape.n_q_heads))
+    # the same with the cache policy's uncompressed rows beside the compressed cache: 4 attention sinks and 128
+    # recent tokens per sequence (Section 4.1), merged in the same combine kernel
+    n16 = 132
+    K16 = synth.random_16bit((shape.batch, n16, d), shape.dtype, 5007, device=dev)
+    V16 = synth.random_16bit((shape.batch, n16, d), shape.dtype, 5008, device=dev)
+    buf = lambda: codec.decode_attn_buffered(q, rc.Kcodes[0], rc.Kscales[0], rc.Vcodes[0], rc.Vscales[0], ctx_len,
+                                             shape.n_kv_heads, 1.0 / math.sqrt(shape.head_dim), K16, V16, Kp, Vp,
+                                             ad.Wk[1], ad.Wv[1], None, None, out=o)
+    ms_b = _time_calls(buf, max(2, reps // 2), warm=2)
+    out.append(_shape_entry(peaks, shape, "decode_attn_buffered", T, ms_b,
+                            _shape_bytes(shape, T, False, write_hat=False), config=5, batch=shape.batch, ctx=ctx_len,
+                            n_q_heads=shape.n_q_heads, uncompressed_rows_per_sequence=n16,
+                            note="compressed cache + 4 sink and 128 recent tokens per sequence in 16 bits"))
     assert codec.poll_status() == 0
     del rc, Kp, Vp
     torch.cuda.empty_cache()
