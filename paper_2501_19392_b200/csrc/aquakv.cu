@@ -759,13 +759,13 @@ ChainWs chain_ws(const aquakv_ctx* c, int64_t T, int L) {
   return w;
 }
 
-template <bool ENC, int D, int NPTS, bool BF>
+template <bool ENC, int D, int NPTS, bool BF, bool WROWS>
 int launch_chain_t(int device, cudaStream_t st, int grid, const ChainArgs& a) {
   static std::atomic<unsigned long long> attr_devices{0};
-  constexpr size_t smem = sizeof(ChainSmem<D, NPTS, ENC>);
+  constexpr size_t smem = sizeof(ChainSmem<D, NPTS, ENC, WROWS>);
   const unsigned long long bit = 1ull << (device & 63);
   if (device >= 64 || !(attr_devices.load(std::memory_order_acquire) & bit)) {
-    if (cudaFuncSetAttribute(chain_kernel<ENC, D, NPTS, BF>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) !=
+    if (cudaFuncSetAttribute(chain_kernel<ENC, D, NPTS, BF, WROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) !=
         cudaSuccess)
       return AQUAKV_ERR_CUDA;
     if (device < 64) attr_devices.fetch_or(bit, std::memory_order_release);
@@ -774,18 +774,28 @@ int launch_chain_t(int device, cudaStream_t st, int grid, const ChainArgs& a) {
   static std::atomic<unsigned long long> fits_devices{0};
   if (device >= 64 || !(fits_devices.load(std::memory_order_acquire) & bit)) {
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, chain_kernel<ENC, D, NPTS, BF>, kChainThreads, smem) !=
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, chain_kernel<ENC, D, NPTS, BF, WROWS>, kChainThreads, smem) !=
         cudaSuccess)
       return AQUAKV_ERR_CUDA;
     if (per_sm < 1) return AQUAKV_ERR_UNSUPPORTED;
     if (device < 64) fits_devices.fetch_or(bit, std::memory_order_release);
   }
-  chain_kernel<ENC, D, NPTS, BF><<<grid, kChainThreads, smem, st>>>(a);
+  chain_kernel<ENC, D, NPTS, BF, WROWS><<<grid, kChainThreads, smem, st>>>(a);
   return AQUAKV_OK;
 }
 template <int D, int NPTS, bool BF>
 void launch_chain_dnb(int* rc, bool encode, int device, cudaStream_t st, int grid, const ChainArgs& a) {
-  *rc = encode ? launch_chain_t<true, D, NPTS, BF>(device, st, grid, a) : launch_chain_t<false, D, NPTS, BF>(device, st, grid, a);
+  // one warp per row once the teams of four warps no longer cover every row of a layer at once
+  if constexpr (D == 1024) {
+    const bool warp_rows = 2 * a.T > grid * (kChainWarps / RowTeam<D>::TEAM);
+    if (warp_rows) {
+      *rc = encode ? launch_chain_t<true, D, NPTS, BF, true>(device, st, grid, a)
+                   : launch_chain_t<false, D, NPTS, BF, true>(device, st, grid, a);
+      return;
+    }
+  }
+  *rc = encode ? launch_chain_t<true, D, NPTS, BF, false>(device, st, grid, a)
+               : launch_chain_t<false, D, NPTS, BF, false>(device, st, grid, a);
 }
 
 // Algorithm 2 (encode) or Algorithm 3 for n_layers layers in one launch; argument checks included.

@@ -40,6 +40,7 @@ CASES = [
     (1, 1024, 2, 16),     # Llama-3.2-1B-shaped round trip: d_kv 512, fp16, Hadamard block 64
     (3, 37, 3, 256),      # ragged 16-token tiles, 4 bits
     (1, 1, 3, 16),        # a single token
+    (3, 600, 3, 16),      # d_kv 1024 with more rows than four-warp teams at once: one warp per row
 ]
 
 
@@ -91,7 +92,8 @@ def test_chain_free_running_and_decode_reproduces_encode(cfg, T, L, n):
         assert torch.equal(Kc2[l], Kc[l]) and torch.equal(Vc2[l], Vc[l]) and torch.equal(Ks2[l], Ks[l]) and torch.equal(Vs2[l], Vs[l])
 
 
-@pytest.mark.parametrize("cfg,T,n,bias", [(3, 64, 16, False), (3, 64, 64, True), (1, 300, 16, False), (2, 200, 16, True)])
+@pytest.mark.parametrize("cfg,T,n,bias", [(3, 64, 16, False), (3, 64, 64, True), (1, 300, 16, False), (2, 200, 16, True),
+                                          (2, 700, 16, False)])     # the last: d_kv 1024 on the one-warp-per-row routines
 def test_chain_teacher_forced_layers(cfg, T, n, bias):
     """A chain of ONE predicted layer started from the oracle's reconstruction of the layer before it:
     codes, scales and reconstructions against the oracle under the rules of the per-layer tests; then
