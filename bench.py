@@ -517,6 +517,8 @@ def main():
     ap.add_argument("--no-other-configs", action="store_true", help="skip the per-call timing of configs 1, 3, 4, 5")
     ap.add_argument("--only-calibration", action="store_true",
                     help="run only the calibration entry of ops_by_config and print it (profiling aid)")
+    ap.add_argument("--only-uniform-backbone", action="store_true",
+                    help="run only the uniform-backbone entries of ops_by_config and print them (profiling aid)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -537,6 +539,10 @@ def main():
     if args.only_calibration:
         if rank == 0:
             print(json.dumps(calibration_entry(api, peaks, dev, reps=1)))
+        return
+    if args.only_uniform_backbone:
+        if rank == 0:
+            print(json.dumps(uniform_backbone_entries(api, chain, peaks, dev, reps=2)))
         return
     shape, batch = workload(args)
     T, L, d = shape.n_tokens, shape.n_layers, shape.d_kv
