@@ -272,7 +272,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) chain_kernel(const __grid_co
         if (int(threadIdx.x) < tiles_per_round) {      // one releasing thread per tile, after the barrier
           const int tile2 = q * tiles_per_round + int(threadIdx.x);
           if (tile2 < n_tiles) {
-            __threadfence();
+            asm volatile("fence.acq_rel.gpu;" ::: "memory");     // release: the barrier above ordered the CTA's stores before it
             atomicAdd(g_done + l * n_mt + tile2 / NTILES, 1);
           }
         }
@@ -331,7 +331,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) chain_kernel(const __grid_co
       }
       if (TEAM > 1) team_barrier<D>(rck.barrier); else __syncwarp();
       if (rck.member == 0 && lane == 0) {
-        __threadfence();
+        asm volatile("fence.acq_rel.gpu;" ::: "memory");
         atomicAdd(r_done + l * n_mt + mt, 1);
       }
     }
