@@ -103,7 +103,7 @@ int aquakv_code_bytes(const aquakv_params* params);
  * per value): the signed integers -2^(b-1) .. 2^(b-1)-1 times the group scale, scale = absmax / 2^(b-1)
  * stored as fp16, nearest level with the lower one on a tie, saturation at the ends, code = level +
  * 2^(b-1), codes packed LSB-first in value order (d_kv * b / 8 bytes per token); had_block must be 1 (no
- * rotation), scale_group in {32, 64, 128, 256}; grid_host and the sign arrays are not read and may be
+ * rotation), scale_group a power of two from 32 to d_kv; grid_host and the sign arrays are not read and may be
  * NULL.  Such a ctx serves aquakv_encode / aquakv_decode (with predictors: two launches per phase, and
  * Khat is required because the value phase reads it), the *_phase entry points, aquakv_predict,
  * aquakv_fit_predictor and aquakv_gather_rows; the chain, no-allocation and attention entry points return

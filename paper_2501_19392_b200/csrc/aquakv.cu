@@ -103,11 +103,11 @@ int check_params(const aquakv_params* p) {
   if (p->dtype != AQUAKV_F16 && p->dtype != AQUAKV_BF16) return AQUAKV_ERR_INVALID_ARG;
   if (p->grid_dim == 1) {
     // uniform round-to-nearest backbone with absmax normalisation: grid_size = 2^b levels per value,
-    // no rotation (had_block 1), groups of 32 .. 256 values
+    // no rotation (had_block 1), groups of 32 .. d_kv values
     if (p->d_kv != 256 && p->d_kv != 512 && p->d_kv != 1024) return AQUAKV_ERR_UNSUPPORTED;
     if (p->grid_size != 4 && p->grid_size != 8 && p->grid_size != 16) return AQUAKV_ERR_UNSUPPORTED;
     if (p->had_block != 1) return AQUAKV_ERR_UNSUPPORTED;
-    if (!is_pow2(p->scale_group) || p->scale_group < 32 || p->scale_group > 256) return AQUAKV_ERR_UNSUPPORTED;
+    if (!is_pow2(p->scale_group) || p->scale_group < 32 || p->scale_group > p->d_kv) return AQUAKV_ERR_UNSUPPORTED;
     return AQUAKV_OK;
   }
   if (p->grid_dim != 2) return AQUAKV_ERR_UNSUPPORTED;

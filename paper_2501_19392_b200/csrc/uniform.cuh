@@ -10,8 +10,10 @@
 // value order.  No rotation, no sign flips.
 //
 // One warp per row.  Lane L holds the 8 consecutive values 256 c + 8 L .. + 7 of every 256-value chunk c
-// (16-byte accesses); a group of g values (32 <= g <= 256) is g/8 neighbouring lanes, so its absmax is
-// log2(g/8) shuffle steps.  The lane's 8 codes are b contiguous bytes of the row's code stream.
+// (16-byte accesses); a group of g <= 256 values is g/8 neighbouring lanes, so its absmax is log2(g/8)
+// shuffle steps; a larger group (512 or 1024 values: whole chunks) takes a first pass over its chunks for
+// the absmax and reads them again to quantize.  The lane's 8 codes are b contiguous bytes of the row's
+// code stream.
 #pragma once
 
 #include "codec.cuh"
@@ -29,8 +31,30 @@ struct UniformArgs {
   long long ldHat;
   int T;
   int d;                    // 256, 512 or 1024
-  int log_g;                // 5 .. 8
+  int log_g;                // 5 .. 10
 };
+
+// |x - pred| maximum of this lane's 8 values of chunk c of row t.
+template <bool kBf16>
+__device__ __forceinline__ float uniform_chunk_absmax(const UniformArgs& a, long long t, int c, int lane) {
+  const int e0 = 256 * c + 8 * lane;
+  const uint4 raw = __ldg(reinterpret_cast<const uint4*>(a.X + t * a.ldX + e0));
+  float r[8], lo, hi;
+  unpack2(load16x2<kBf16>(raw.x), lo, hi); r[0] = lo; r[1] = hi;
+  unpack2(load16x2<kBf16>(raw.y), lo, hi); r[2] = lo; r[3] = hi;
+  unpack2(load16x2<kBf16>(raw.z), lo, hi); r[4] = lo; r[5] = hi;
+  unpack2(load16x2<kBf16>(raw.w), lo, hi); r[6] = lo; r[7] = hi;
+  if (a.P != nullptr) {
+    const float4 p0 = *reinterpret_cast<const float4*>(a.P + t * a.ldP + e0);
+    const float4 p1 = *(reinterpret_cast<const float4*>(a.P + t * a.ldP + e0) + 1);
+    r[0] -= p0.x; r[1] -= p0.y; r[2] -= p0.z; r[3] -= p0.w;
+    r[4] -= p1.x; r[5] -= p1.y; r[6] -= p1.z; r[7] -= p1.w;
+  }
+  float m = 0.0f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) m = fmaxf(m, fabsf(r[i]));
+  return m;
+}
 
 constexpr int kUniformWarps = 4;
 
@@ -59,10 +83,16 @@ uniform_encode_rows_kernel(const UniformArgs a) {
   const int lane = threadIdx.x & 31;
   const long long warp = (long long)blockIdx.x * kUniformWarps + (threadIdx.x >> 5);
   const long long n_warps = (long long)gridDim.x * kUniformWarps;
-  const int lanes_per_group = 1 << (a.log_g - 3);
+  const int lanes_per_group = a.log_g >= 8 ? 32 : 1 << (a.log_g - 3);
+  const int chunks_per_group = a.log_g > 8 ? 1 << (a.log_g - 8) : 1;
   const int n_groups = a.d >> a.log_g;
   for (long long t = warp; t < a.T; t += n_warps) {
+    float m_group = 0.0f;      // groups of several chunks: their absmax, found before the first chunk is quantized
     for (int c = 0; c < a.d / 256; ++c) {
+      if (chunks_per_group > 1 && (c & (chunks_per_group - 1)) == 0) {
+        m_group = 0.0f;
+        for (int cc = c; cc < c + chunks_per_group; ++cc) m_group = fmaxf(m_group, uniform_chunk_absmax<kBf16>(a, t, cc, lane));
+      }
       const int e0 = 256 * c + 8 * lane;
       float r[8], pred[8];
       {
@@ -84,10 +114,11 @@ uniform_encode_rows_kernel(const UniformArgs a) {
       float m = 0.0f;
 #pragma unroll
       for (int i = 0; i < 8; ++i) m = fmaxf(m, fabsf(r[i]));
+      if (chunks_per_group > 1) m = m_group;
       for (int off = 1; off < lanes_per_group; off <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
       const __half s16 = __float2half_rn(fminf(m * (1.0f / HALF), 65504.0f));
       const float sf = __half2float(s16);
-      if ((lane & (lanes_per_group - 1)) == 0)
+      if ((lane & (lanes_per_group - 1)) == 0 && (c & (chunks_per_group - 1)) == 0)
         a.scales[t * n_groups + ((e0) >> a.log_g)] = __half_as_ushort(s16);
       uint32_t word = 0;
       float q[8];

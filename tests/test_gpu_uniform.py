@@ -50,7 +50,7 @@ def check_levels(gpu_codes, ora, b, d, rows_ok):
 
 
 CASES = [(256, 2, 64, oracle.BF16, 700), (512, 3, 64, oracle.F16, 513), (1024, 4, 32, oracle.BF16, 300),
-         (1024, 2, 256, oracle.BF16, 1000)]
+         (1024, 2, 256, oracle.BF16, 1000), (1024, 2, 1024, oracle.BF16, 600), (512, 4, 512, oracle.F16, 257)]
 
 
 @pytest.mark.parametrize("d,b,g,dtype,T", CASES)
@@ -123,7 +123,7 @@ def test_zero_rows_ties_and_saturation_on_the_gpu():
 
 def test_parameter_checks_and_unsupported_entry_points():
     from paper_2501_19392_b200 import api
-    for bad in (dict(had_block=64), dict(levels=32), dict(scale_group=16), dict(scale_group=512)):
+    for bad in (dict(had_block=64), dict(levels=32), dict(scale_group=16), dict(scale_group=512), dict(scale_group=96)):
         kw = dict(had_block=1, scale_group=64, levels=4)
         kw.update(bad)
         with pytest.raises(api.AquaKVError) as e:
