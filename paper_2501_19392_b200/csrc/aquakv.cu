@@ -561,15 +561,15 @@ AttnWs attn_ws(const aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_
   return w;
 }
 
-template <bool ENC, int D, int NPTS, bool BF, bool FULL, int AHD = 0>
-int launch_layer_t(int device, cudaStream_t st, int grid, const CUtensorMap* tm, const LayerArgs& a) {
+template <bool ENC, int D, int NPTS, bool BF, bool FULL, int AHD, int NB>
+int launch_layer_t(int device, cudaStream_t st, int grid, const LayerBatch<NB>& B) {
   // the shared-memory opt-in is a per-device attribute of the function: one bit per device and
   // instantiation (setting it twice from two threads is harmless)
   static std::atomic<unsigned long long> attr_devices{0};
   constexpr size_t smem = layer_smem_bytes<ENC, D, NPTS, FULL>();
   const unsigned long long bit = 1ull << (device & 63);
   if (device >= 64 || !(attr_devices.load(std::memory_order_acquire) & bit)) {
-    if (cudaFuncSetAttribute(layer_kernel<ENC, D, NPTS, BF, FULL, AHD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(layer_kernel<ENC, D, NPTS, BF, FULL, AHD, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              int(smem)) != cudaSuccess)
       return AQUAKV_ERR_CUDA;
     if (device < 64) attr_devices.fetch_or(bit, std::memory_order_release);
@@ -591,39 +591,53 @@ int launch_layer_t(int device, cudaStream_t st, int grid, const CUtensorMap* tm,
   static std::atomic<unsigned long long> fits_devices{0};
   if (device >= 64 || !(fits_devices.load(std::memory_order_acquire) & bit)) {
     int max_clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&max_clusters, layer_kernel<ENC, D, NPTS, BF, FULL, AHD>, &cfg) != cudaSuccess)
+    if (cudaOccupancyMaxActiveClusters(&max_clusters, layer_kernel<ENC, D, NPTS, BF, FULL, AHD, NB>, &cfg) != cudaSuccess)
       return AQUAKV_ERR_CUDA;
     if (max_clusters * 2 < grid) return AQUAKV_ERR_UNSUPPORTED;
     if (device < 64) fits_devices.fetch_or(bit, std::memory_order_release);
   }
-  return cudaLaunchKernelEx(&cfg, layer_kernel<ENC, D, NPTS, BF, FULL, AHD>, tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], a) ==
-                 cudaSuccess
-             ? AQUAKV_OK
-             : AQUAKV_ERR_CUDA;
+  return cudaLaunchKernelEx(&cfg, layer_kernel<ENC, D, NPTS, BF, FULL, AHD, NB>, B) == cudaSuccess ? AQUAKV_OK
+                                                                                                      : AQUAKV_ERR_CUDA;
 }
-template <int D, int NPTS, bool BF>
-void launch_layer_enc_t(int* rc, int device, cudaStream_t st, int grid, const CUtensorMap* tm, const LayerArgs& a) {
+// Launches of several layers exist for the paper's main setting only (d_kv = 1024, Hadamard block = scale
+// group = the row); everything else runs layer by layer.
+template <int D, int NPTS, bool BF, int NB>
+void launch_layer_enc_t(int* rc, int device, cudaStream_t st, int grid, const LayerBatch<NB>& B) {
   // Hadamard block = scale group = the whole row: the encoder has an instantiation with those sizes
   // fixed at compile time (measured 8-10 % faster; the decoder measured no gain and has none)
+  const LayerArgs& a = B.layer[0];
   const bool full = a.log_h == a.log_g && (1 << a.log_h) == D;
-  *rc = full ? launch_layer_t<true, D, NPTS, BF, true>(device, st, grid, tm, a)
-             : launch_layer_t<true, D, NPTS, BF, false>(device, st, grid, tm, a);
+  if constexpr (NB > 1) {
+    if constexpr (D == 1024) {
+      *rc = full ? launch_layer_t<true, D, NPTS, BF, true, 0, NB>(device, st, grid, B) : AQUAKV_ERR_UNSUPPORTED;
+    } else {
+      *rc = AQUAKV_ERR_UNSUPPORTED;
+    }
+  } else {
+    *rc = full ? launch_layer_t<true, D, NPTS, BF, true, 0, NB>(device, st, grid, B)
+               : launch_layer_t<true, D, NPTS, BF, false, 0, NB>(device, st, grid, B);
+  }
 }
-template <int D, int NPTS, bool BF>
-void launch_layer_dec_t(int* rc, int device, cudaStream_t st, int grid, const CUtensorMap* tm, const LayerArgs& a) {
+template <int D, int NPTS, bool BF, int NB>
+void launch_layer_dec_t(int* rc, int device, cudaStream_t st, int grid, const LayerBatch<NB>& B) {
   // the decoder has the fixed-size instantiation only where it selects the one-warp-per-row routines
+  const LayerArgs& a = B.layer[0];
   if constexpr (D == 1024) {
     if (a.log_h == 10 && a.log_g == 10) {
       if (a.q != nullptr) {       // decode + single-query attention in one kernel
-        *rc = a.n_kv_heads * 128 == D ? launch_layer_t<false, D, NPTS, BF, true, 128>(device, st, grid, tm, a)
-                                      : launch_layer_t<false, D, NPTS, BF, true, 64>(device, st, grid, tm, a);
+        *rc = a.n_kv_heads * 128 == D ? launch_layer_t<false, D, NPTS, BF, true, 128, NB>(device, st, grid, B)
+                                      : launch_layer_t<false, D, NPTS, BF, true, 64, NB>(device, st, grid, B);
         return;
       }
-      *rc = launch_layer_t<false, D, NPTS, BF, true>(device, st, grid, tm, a);
+      *rc = launch_layer_t<false, D, NPTS, BF, true, 0, NB>(device, st, grid, B);
       return;
     }
   }
-  *rc = a.q != nullptr ? AQUAKV_ERR_UNSUPPORTED : launch_layer_t<false, D, NPTS, BF, false>(device, st, grid, tm, a);
+  if constexpr (NB > 1) {
+    *rc = AQUAKV_ERR_UNSUPPORTED;
+  } else {
+    *rc = a.q != nullptr ? AQUAKV_ERR_UNSUPPORTED : launch_layer_t<false, D, NPTS, BF, false, 0, NB>(device, st, grid, B);
+  }
 }
 
 // The attention a decode launch also computes (Algorithm 4 lines 5-9); q == nullptr: none.
@@ -638,16 +652,15 @@ struct LayerAttnArgs {
 // True if decode + attention runs as one launch of the layer kernel for this context.
 bool fused_attn_supported(const aquakv_ctx* c) { return c->p.d_kv == 1024 && c->log_h == 10 && c->log_g == 10; }
 
-// Algorithm 2 (encode = true) or Algorithm 3 for one layer with predictors, all tokens, one launch.
-int launch_layer(aquakv_ctx* c, cudaStream_t st, bool encode, int64_t T, const void* K, const void* V,
-                 int64_t ld_kv, const void* Khat_prev, const void* Vhat_prev, int64_t ld_prev,
-                 const void* Wk, const void* Wv, const float* bk, const float* bv, uint8_t* Kcodes,
-                 uint16_t* Kscales, uint8_t* Vcodes, uint16_t* Vscales, void* Khat, void* Vhat,
-                 int64_t ld_hat, void* workspace, const LayerAttnArgs* attn = nullptr) {
+// Arguments and tensor maps of one layer of a launch.  `flags` is the layer's counter block (gemm_done,
+// rows_done and, with attention, attn_done; zero at launch), `P` the prediction ring.
+int fill_layer(aquakv_ctx* c, const LayerWs& ws, uint8_t* wsb, int* flags, int64_t T, const void* K, const void* V,
+               int64_t ld_kv, const void* Khat_prev, const void* Vhat_prev, int64_t ld_prev, const void* Wk,
+               const void* Wv, const float* bk, const float* bv, uint8_t* Kcodes, uint16_t* Kscales, uint8_t* Vcodes,
+               uint16_t* Vscales, void* Khat, void* Vhat, int64_t ld_hat, const LayerAttnArgs* attn, LayerArgs* out,
+               LayerMaps* maps) {
   const int d = c->p.d_kv;
-  const LayerWs ws = layer_ws(c, T, attn != nullptr);
-  uint8_t* wsb = ws_base(workspace);
-  LayerArgs a;
+  LayerArgs& a = *out;
   std::memset(&a, 0, sizeof(a));
   a.T = int(T);
   a.n_mblocks = ws.n_mblocks;
@@ -657,7 +670,7 @@ int launch_layer(aquakv_ctx* c, cudaStream_t st, bool encode, int64_t T, const v
   a.bk = bk;
   a.bv = bv;
   a.P = reinterpret_cast<float*>(wsb + ws.p_off);
-  a.gemm_done = reinterpret_cast<int*>(wsb + ws.flags_off);
+  a.gemm_done = flags;
   a.rows_done = a.gemm_done + size_t(2) * ws.n_waves * ws.mw;
   a.K = static_cast<const uint16_t*>(K);
   a.V = static_cast<const uint16_t*>(V);
@@ -701,35 +714,49 @@ int launch_layer(aquakv_ctx* c, cudaStream_t st, bool encode, int64_t T, const v
   a.log_h = c->log_h;
   a.log_g = c->log_g;
   a.status = c->d_status;
-
-  CUtensorMap tm[6];
   {
     // the prediction ring as a 2-D fp32 tensor for the epilogue's TMA stores (32 x 32 boxes)
     const cuuint64_t dims[2] = {cuuint64_t(d), cuuint64_t(kLayerRing) * ws.mw * kBM};
     const cuuint64_t strides[1] = {cuuint64_t(d) * sizeof(float)};
     const cuuint32_t box[2] = {32, 32};
     const cuuint32_t estr[2] = {1, 1};
-    if (c->encode_tiled(&tm[5], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, a.P, dims, strides, box, estr,
+    if (c->encode_tiled(&maps->p, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, a.P, dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return AQUAKV_ERR_CUDA;
   }
-  int rc = make_tmap(c, &tm[0], Khat_prev, uint64_t(T), uint64_t(d), uint64_t(ld_prev), kBM);
+  int rc = make_tmap(c, &maps->kprev, Khat_prev, uint64_t(T), uint64_t(d), uint64_t(ld_prev), kBM);
   if (rc) return rc;
-  if ((rc = make_tmap(c, &tm[1], Vhat_prev, uint64_t(T), uint64_t(d), uint64_t(ld_prev), kBM))) return rc;
+  if ((rc = make_tmap(c, &maps->vprev, Vhat_prev, uint64_t(T), uint64_t(d), uint64_t(ld_prev), kBM))) return rc;
   const uint64_t khat_rows = a.khat_ring ? uint64_t(kKhatRing) * ws.mw * kBM : uint64_t(T);
-  if ((rc = make_tmap(c, &tm[2], a.Khat, khat_rows, uint64_t(d), uint64_t(a.ldKhat), kBM))) return rc;
+  if ((rc = make_tmap(c, &maps->khat, a.Khat, khat_rows, uint64_t(d), uint64_t(a.ldKhat), kBM))) return rc;
   // weight tiles are fetched half (128 rows) per CTA of a pair
-  if ((rc = make_tmap(c, &tm[3], Wk, uint64_t(d), uint64_t(d), uint64_t(d), kBN / 2))) return rc;
-  if ((rc = make_tmap(c, &tm[4], Wv, uint64_t(d), uint64_t(2) * d, uint64_t(2) * d, kBN / 2))) return rc;
+  if ((rc = make_tmap(c, &maps->wk, Wk, uint64_t(d), uint64_t(d), uint64_t(d), kBN / 2))) return rc;
+  return make_tmap(c, &maps->wv, Wv, uint64_t(d), uint64_t(2) * d, uint64_t(2) * d, kBN / 2);
+}
 
-  if (cudaMemsetAsync(a.gemm_done, 0, ws.flags_bytes, st) != cudaSuccess) return AQUAKV_ERR_CUDA;
+// Algorithm 2 (encode = true) or Algorithm 3 for one layer with predictors, all tokens, one launch.
+int launch_layer(aquakv_ctx* c, cudaStream_t st, bool encode, int64_t T, const void* K, const void* V,
+                 int64_t ld_kv, const void* Khat_prev, const void* Vhat_prev, int64_t ld_prev,
+                 const void* Wk, const void* Wv, const float* bk, const float* bv, uint8_t* Kcodes,
+                 uint16_t* Kscales, uint8_t* Vcodes, uint16_t* Vscales, void* Khat, void* Vhat,
+                 int64_t ld_hat, void* workspace, const LayerAttnArgs* attn = nullptr) {
+  const int d = c->p.d_kv;
+  const LayerWs ws = layer_ws(c, T, attn != nullptr);
+  uint8_t* wsb = ws_base(workspace);
+  LayerBatch<1> B;
+  B.n_layers = 1;
+  int rc = fill_layer(c, ws, wsb, reinterpret_cast<int*>(wsb + ws.flags_off), T, K, V, ld_kv, Khat_prev, Vhat_prev,
+                      ld_prev, Wk, Wv, bk, bv, Kcodes, Kscales, Vcodes, Vscales, Khat, Vhat, ld_hat, attn, &B.layer[0],
+                      &B.maps[0]);
+  if (rc) return rc;
+  if (cudaMemsetAsync(B.layer[0].gemm_done, 0, ws.flags_bytes, st) != cudaSuccess) return AQUAKV_ERR_CUDA;
   const int grid = ws.grid_mw * (d / kBN);
   ProfScope prof(c, st, AQUAKV_KERNEL_LAYER);
   if (encode) {
-    AQ_DISPATCH_DNB(launch_layer_enc_t, &rc, c->device, st, grid, tm, a);
+    AQ_DISPATCH_DNB(launch_layer_enc_t, &rc, c->device, st, grid, B);
   } else {
-    AQ_DISPATCH_DNB(launch_layer_dec_t, &rc, c->device, st, grid, tm, a);
+    AQ_DISPATCH_DNB(launch_layer_dec_t, &rc, c->device, st, grid, B);
   }
   if (rc) return rc;
   ++c->launches;

@@ -197,6 +197,22 @@ struct LayerArgs {
   int* attn_done;           // [n_waves][mw], zero at launch: attention warps that are done with the block
 };
 
+// The layers of one launch.  A launch of several layers (Algorithm 2 / 3 inside Algorithm 4's loop over
+// layers) runs them back to back without a barrier in between: every role walks the layers on its own,
+// the prediction ring and its counters continue across the layer boundary, and a layer's first jobs start
+// while the previous layer's last wave is still being finished (a layer's wave w needs only wave w of the
+// layer before it).  All layers share T, the wave geometry and the ring.
+struct LayerMaps {
+  CUtensorMap kprev, vprev, khat, wk, wv, p;
+};
+constexpr int kLayerBatchMax = 24;      // 24 x (arguments + six tensor maps) stays inside the 32 KB of kernel parameters
+template <int kBatch>
+struct LayerBatch {
+  int n_layers;
+  LayerArgs layer[kBatch];
+  LayerMaps maps[kBatch];
+};
+
 __device__ __forceinline__ void layer_job(int j, int n_waves, int& phase, int& wave) {
   if (j == 0) { phase = 0; wave = 0; }
   else if (j == 2 * n_waves - 1) { phase = 1; wave = n_waves - 1; }
@@ -275,13 +291,12 @@ __device__ __forceinline__ void fence_proxy_async_all() {
 // kFull: the Hadamard block and the scale group both span the whole row (the paper's setting for
 // d_kv = 1024, Section 4.1); their logarithms are then compile-time constants of the row code.
 // kAttnHD: 0, or the head dimension (64 / 128) of the attention the decoder also computes.
-template <bool kEncode, int D, int NPTS, bool kBf16, bool kFull, int kAttnHD = 0>
+template <bool kEncode, int D, int NPTS, bool kBf16, bool kFull, int kAttnHD = 0, int kBatch = 1>
 __global__ void __launch_bounds__((layer_threads<kEncode, D, kFull, kAttnHD>()), 1)
-layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant__ CUtensorMap tmVprev,
-             const __grid_constant__ CUtensorMap tmKhat, const __grid_constant__ CUtensorMap tmWk,
-             const __grid_constant__ CUtensorMap tmWv, const __grid_constant__ CUtensorMap tmP,
-             const LayerArgs a) {
+layer_kernel(const __grid_constant__ LayerBatch<kBatch> B) {
   using G = LayerGeom<kEncode, D, kFull, kAttnHD>;
+  const LayerArgs& a = B.layer[0];         // what all layers of the launch share: geometry, tables, status word
+  const int n_layers = kBatch == 1 ? 1 : B.n_layers;
   constexpr int NTN = D / kBN;             // feature tiles per token block = CTAs per token block
   constexpr int NKD = D / kBK;             // k-blocks per d_kv input features
   constexpr int BITS = NPTS == 16 ? 4 : (NPTS == 64 ? 6 : 8);
@@ -337,17 +352,19 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
   if (warp == 0) {
     // ------------------------------- TMA producer --------------------------------------------
     if (lane == 0) {
-      tma_prefetch_desc(&tmKprev);
-      tma_prefetch_desc(&tmVprev);
-      tma_prefetch_desc(&tmKhat);
-      tma_prefetch_desc(&tmWk);
-      tma_prefetch_desc(&tmWv);
-      tma_prefetch_desc(&tmP);
       const uint64_t pol_stream = l2_policy_evict_first(), pol_keep = l2_policy_evict_last();
       int stage = 0;
       uint32_t phase_bit = 0;
       bool ok = true;
       int issued = 0;
+      for (int l = 0; ok && l < n_layers; ++l) {
+      const LayerArgs& a = B.layer[l];
+      const LayerMaps& tm = B.maps[l];
+      tma_prefetch_desc(&tm.kprev);
+      tma_prefetch_desc(&tm.vprev);
+      tma_prefetch_desc(&tm.khat);
+      tma_prefetch_desc(&tm.wk);
+      tma_prefetch_desc(&tm.wv);
       for (int j = 0; ok && j < n_jobs; ++j) {
         int ph, wave;
         layer_job(j, a.n_waves, ph, wave);
@@ -356,6 +373,18 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         const int nk = ph == 0 ? NKD : 2 * NKD;
         const int khat_row = a.khat_ring ? ((wave % a.khat_ring) * a.mw + ml) * kBM : m * kBM;
         for (int kb = 0; kb < nk; ++kb) {
+          if (l > 0 && kb == 0 && m < a.n_mblocks) {
+            // the previous layer of this launch wrote this job's first input (its reconstructed keys for
+            // the key phase, values for the value phase): its row warps must be done with this token block
+            const LayerArgs& pa = B.layer[l - 1];
+            const int pj = ph == 0 ? layer_key_job(wave) : layer_value_job(wave, a.n_waves);
+            const int target = wave_block_teams(wave_rows(wave, a.T, a.mw, gridDim.x), ml, gridDim.x, G::TEAMS);
+            if (!counter_wait_bounded(pa.rows_done + pj * a.mw + ml, target, abort_flag, a.status)) {
+              ok = false;
+              break;
+            }
+            fence_proxy_async_all();
+          }
           if (ph == 1 && kb == NKD && m < a.n_mblocks) {
             // the remaining k-blocks read this wave's reconstructed keys, written by row warps
             const int target = wave_block_teams(wave_rows(wave, a.T, a.mw, gridDim.x), ml, gridDim.x, G::TEAMS);
@@ -377,20 +406,21 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
           const int w_row = n_blk * kBN + int(rank) * (kBN / 2);     // this CTA's half of the weight rows
           // token rows stream through L2 once; the adapter tiles are read again by every wave
           if (ph == 0) {
-            tma_load_2d_pair_hint(a_dst, &tmKprev, &tail->full[stage], kb * kBK, m * kBM, pol_stream);
-            tma_load_2d_pair_hint(b_dst, &tmWk, &tail->full[stage], kb * kBK, w_row, pol_keep);
+            tma_load_2d_pair_hint(a_dst, &tm.kprev, &tail->full[stage], kb * kBK, m * kBM, pol_stream);
+            tma_load_2d_pair_hint(b_dst, &tm.wk, &tail->full[stage], kb * kBK, w_row, pol_keep);
           } else {
             if (kb < NKD) {
-              tma_load_2d_pair_hint(a_dst, &tmVprev, &tail->full[stage], kb * kBK, m * kBM, pol_stream);
+              tma_load_2d_pair_hint(a_dst, &tm.vprev, &tail->full[stage], kb * kBK, m * kBM, pol_stream);
             } else {
-              tma_load_2d_pair_hint(a_dst, &tmKhat, &tail->full[stage], (kb - NKD) * kBK, khat_row, pol_stream);
+              tma_load_2d_pair_hint(a_dst, &tm.khat, &tail->full[stage], (kb - NKD) * kBK, khat_row, pol_stream);
             }
-            tma_load_2d_pair_hint(b_dst, &tmWv, &tail->full[stage], kb * kBK, w_row, pol_keep);
+            tma_load_2d_pair_hint(b_dst, &tm.wv, &tail->full[stage], kb * kBK, w_row, pol_keep);
           }
           ++issued;
           if (++stage == kLayerStagesT<kEncode, G::WR>) { stage = 0; phase_bit ^= 1u; }
         }
       }
+      }   // layers
       if (!ok && rank == 0) {
         // let the copies in flight land before the shared memory is released
         int s = stage;
@@ -413,6 +443,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       uint32_t phase_bit = 0;
       bool ok = true;
       int it = 0;
+      for (int l = 0; ok && l < n_layers; ++l)
       for (int j = 0; ok && j < n_jobs; ++j) {
         int ph, wave;
         layer_job(j, a.n_waves, ph, wave);
@@ -421,7 +452,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         const int acc = it & 1;
         const uint32_t acc_phase = (it >> 1) & 1u;
         ++it;
-        if (!mbar_wait_bounded(&tail->acc_empty[acc], acc_phase ^ 1u, abort_flag, a.status)) break;
+        if (!mbar_wait_bounded(&tail->acc_empty[acc], acc_phase ^ 1u, abort_flag, a.status)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t tmem_d = tmem_base + uint32_t(acc * kBN);
         for (int kb = 0; kb < nk; ++kb) {
@@ -448,6 +479,10 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
     // ------------------------------- GEMM epilogue (4 warps) ---------------------------------
     const int quarter = warp & 3;   // tensor-memory lanes [32*quarter, 32*quarter+32)
     int it = 0;
+    bool stop = false;
+    for (int l = 0; !stop && l < n_layers; ++l) {
+    const LayerArgs& a = B.layer[l];
+    const LayerMaps& tm = B.maps[l];
     for (int j = 0; j < n_jobs; ++j) {
       int ph, wave;
       layer_job(j, a.n_waves, ph, wave);
@@ -456,14 +491,17 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       const uint32_t acc_phase = (it >> 1) & 1u;
       ++it;
       bool ok = true;
-      // the ring slot of this job was last used by job j - nb: its row work must be over
-      if (j >= a.nb) {
+      // the ring slot of this job was last used nb jobs earlier (counted through the layers of the launch):
+      // that job's row work must be over
+      const int gj = l * n_jobs + j;
+      if (gj >= a.nb) {
+        const int lo = (gj - a.nb) / n_jobs, jo = (gj - a.nb) % n_jobs;
         int ph_old, wave_old;
-        layer_job(j - a.nb, a.n_waves, ph_old, wave_old);
+        layer_job(jo, a.n_waves, ph_old, wave_old);
         const int target = wave_block_teams(wave_rows(wave_old, a.T, a.mw, gridDim.x), ml, gridDim.x, G::TEAMS);
         // one thread polls for the four warps; a failed wait has set the abort flag
         if (warp == 2 && lane == 0)
-          counter_wait_bounded(a.rows_done + (j - a.nb) * a.mw + ml, target, abort_flag, a.status);
+          counter_wait_bounded(B.layer[lo].rows_done + jo * a.mw + ml, target, abort_flag, a.status);
         named_barrier(1, 128);
         ok = *abort_flag == 0;
       }
@@ -472,7 +510,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         tc_fence_after_sync();
         const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * kBN);
         // ring row of this warp's 32 tokens; rows past the last token are written too (never read)
-        const int ring_row = (j % a.nb) * a.mw * kBM + ml * kBM + quarter * 32;
+        const int ring_row = (gj % a.nb) * a.mw * kBM + ml * kBM + quarter * 32;
         const float* bias = ph == 0 ? a.bk : a.bv;
         constexpr int EB = kEpiBufs<kEncode, NPTS, G::WR>;
         const uint64_t pol_keep = l2_policy_evict_last();
@@ -501,7 +539,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
           fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) {
-            tma_store_2d_hint(&tmP, buf, n_blk * kBN + c * 32, ring_row, pol_keep);   // read back soon by the row warps
+            tma_store_2d_hint(&tm.p, buf, n_blk * kBN + c * 32, ring_row, pol_keep);   // read back soon by the row warps
             bulk_commit();
           }
         }
@@ -517,12 +555,13 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       // release by one thread after the barrier: its fence also covers the stores of the threads it
       // has synchronised with, and only that thread waits for them to become visible
       named_barrier(1, 128);
-      if (*abort_flag) break;
+      if (*abort_flag) { stop = true; break; }
       if (warp == 2 && lane == 0) {
         __threadfence();
         atomicAdd(a.gemm_done + j * a.mw + ml, 1);
       }
     }
+    }   // layers
   } else if (warp < 6 + G::ROW_WARPS) {
     // ------------------------------- row warps (TEAM warps per row; TEAMS rows at a time) ------
     constexpr int TEAM = G::TEAM, TEAMS = G::TEAMS;
@@ -548,9 +587,13 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       signs_v = a.signmask_v[lane] >> (rck.member * RowTeam<D>::NV);
     }
     const int n_groups = D >> log_g;
+    bool stop = false;
+    for (int l = 0; !stop && l < n_layers; ++l) {
+    const LayerArgs& a = B.layer[l];
     for (int j = 0; j < n_jobs; ++j) {
       int ph, wave;
       layer_job(j, a.n_waves, ph, wave);
+      const int gj = l * n_jobs + j;
       const WaveRows wr = wave_rows(wave, a.T, a.mw, gridDim.x);
       if (wr.tokens <= 0) continue;
       if constexpr (G::WR) wrc.signs = ph == 0 ? signs_k : signs_v;
@@ -573,9 +616,16 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       }
       bool ok = true;
       if constexpr (kAttnHD > 0) {
+        // this layer's rows overwrite the reconstructions of two layers earlier (the caller alternates
+        // two buffer pairs), which that layer's attention warps may, in principle, still be reading
+        if (l >= 2) {
+          if (lane == 0)
+            ok = counter_wait_bounded(B.layer[l - 2].attn_done + wave * a.mw + rb, NTN * kAttnWarps, abort_flag, a.status);
+          ok = __shfl_sync(0xffffffffu, ok, 0);
+        }
         // the key rows of this wave reuse the ring rows of wave - ring depth: the attention warps must
         // be done with them (they trail the rows by about one job, so this rarely waits)
-        if (ph == 0 && a.khat_ring > 0 && wave >= a.khat_ring) {
+        if (ok && ph == 0 && a.khat_ring > 0 && wave >= a.khat_ring) {
           if (lane == 0)
             ok = counter_wait_bounded(a.attn_done + (wave - a.khat_ring) * a.mw + rb, NTN * kAttnWarps, abort_flag,
                                       a.status);
@@ -597,7 +647,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         ok = __shfl_sync(0xffffffffu, ok, 0);
       }
       if (ok) {
-        const float* pbuf = a.P + (size_t(j % a.nb) * a.mw * kBM + size_t(rb) * kBM) * D;
+        const float* pbuf = a.P + (size_t(gj % a.nb) * a.mw * kBM + size_t(rb) * kBM) * D;
         const size_t khat_base = a.khat_ring ? size_t((wave % a.khat_ring) * a.mw + rb) * kBM
                                              : size_t(m) * kBM;
         [[maybe_unused]] uint4 xraw[4];
@@ -657,14 +707,15 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       }
       // each team reports on its own, so a slow team never holds the others back
       if (TEAM > 1) team_barrier<D>(rck.barrier); else __syncwarp();
-      if (*abort_flag) break;
+      if (*abort_flag) { stop = true; break; }
       if (rck.member == 0 && lane == 0) {   // one releasing thread per team (see the epilogue)
         // Key rows are read back by other CTAs' TMA loads (value-phase GEMM) and, like the value rows,
         // by other CTAs' attention warps: those need the stores released, the TMA also across the
         // proxies.  Value rows without attention are read by nobody in this launch; the counter then
         // only tells the epilogue that the ring slot's prediction has been read (the row's stores
-        // depend on those loads, so they have completed).
-        if (ph == 0) {
+        // depend on those loads, so they have completed).  With a further layer in the launch the value
+        // rows are read by its TMA loads like the key rows.
+        if (ph == 0 || l + 1 < n_layers) {
           fence_acq_rel_gpu();
           fence_proxy_async_all();
         } else if (kAttnHD > 0) {
@@ -673,6 +724,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
         atomicAdd(a.rows_done + j * a.mw + rb, 1);
       }
     }
+    }   // layers
   } else {
     // ------------------------------- attention warps ------------------------------------------------
     if constexpr (kAttnHD > 0) {
@@ -688,6 +740,9 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
       const int sub = (aw / WPH) % NSUB;
       const int hpc = a.n_kv_heads / NTN;              // KV heads of a token block that this CTA attends over
       const int rep = a.n_q_heads / a.n_kv_heads;
+      bool stop = false;
+      for (int l = 0; !stop && l < n_layers; ++l) {
+      const LayerArgs& a = B.layer[l];
       for (int wave = 0; wave < a.n_waves; ++wave) {
         const WaveRows wr = wave_rows(wave, a.T, a.mw, gridDim.x);
         if (ml >= wr.blocks) continue;                  // this CTA's block does not exist in the (last) wave
@@ -696,7 +751,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
           ok = counter_wait_bounded(a.rows_done + layer_value_job(wave, a.n_waves) * a.mw + ml,
                                     wave_block_teams(wr, ml, gridDim.x, G::TEAMS), abort_flag, a.status);
         ok = __shfl_sync(0xffffffffu, ok, 0);
-        if (!ok) break;
+        if (!ok) { stop = true; break; }
         const long long blk = (long long)wave * a.mw + ml;       // token block of the call
         const long long sblk = blk * NSUB + sub;                 // this warp's sub-block of the call
         const long long tok0 = sblk * kAttnSubTokens;
@@ -725,6 +780,7 @@ layer_kernel(const __grid_constant__ CUtensorMap tmKprev, const __grid_constant_
           atomicAdd(a.attn_done + wave * a.mw + ml, 1);
         }
       }
+      }   // layers
     }
   }
 
