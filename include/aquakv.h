@@ -241,9 +241,19 @@ int aquakv_decode(aquakv_ctx* ctx, int64_t n_tokens,
  * outputs Khat[l], Vhat[l] ([n_tokens, ld_hat]; arrays or entries NULL: that layer's reconstruction
  * stays in the workspace; give both or neither of a layer).  If layer 0 has a predictor, Khat_init /
  * Vhat_init ([n_tokens, ld_init]) are the reconstruction of the layer before it; otherwise they must
- * be NULL.  n_tokens <= 2048 and n_layers <= 128 (AQUAKV_ERR_TOO_LARGE beyond: use the per-layer
- * calls, which are built for large token counts).  d_kv = 1024 requires Hadamard block = scale group
- * = 1024 (AQUAKV_ERR_UNSUPPORTED otherwise).  Workspace: aquakv_chain_workspace_bytes.
+ * be NULL.  n_layers <= 128 (AQUAKV_ERR_TOO_LARGE beyond).  Up to 2048 tokens the call is one launch of
+ * the chain kernel; d_kv = 1024 then requires Hadamard block = scale group = 1024 (AQUAKV_ERR_UNSUPPORTED
+ * otherwise).  Workspace: aquakv_chain_workspace_bytes.
+ *
+ * LARGE calls (n_tokens > 2048; d_kv = 1024 with Hadamard block = scale group = 1024 only,
+ * AQUAKV_ERR_TOO_LARGE otherwise: use the per-layer calls) run the persistent layer kernel of
+ * aquakv_encode / aquakv_decode on up to 24 consecutive predicted layers per launch: no barrier between
+ * the layers, a layer's first token blocks start while the previous layer's last ones are being
+ * finished, which removes the pipeline fill and drain that every per-layer launch pays (about 60 us of
+ * an encode and 20 us of a decode launch).  Every layer then needs its Khat[l] / Vhat[l] from the
+ * caller (AQUAKV_ERR_INVALID_ARG otherwise); a layer may reuse the buffers of the layer TWO before it
+ * (two alternating pairs suffice), not those of the layer before it, which it reads.  Results are
+ * bit-identical to the per-layer calls.
  *
  * Results satisfy the same bounds against the definition as the per-layer calls; the fp32 prediction
  * is summed in a different order, so a reconstruction can differ from aquakv_encode / aquakv_decode in

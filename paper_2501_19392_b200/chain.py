@@ -58,6 +58,25 @@ def encode_chain(codec: api.Codec, K: List[torch.Tensor], V: List[torch.Tensor],
                      bufs.K[cur], bufs.V[cur])
 
 
+def encode_layers(codec: api.Codec, K: List[torch.Tensor], V: List[torch.Tensor], adapters,
+                  cache: CompressedCache, bufs: PingPong) -> None:
+    """encode_chain through aquakv_encode_chain: for large token counts several layers per launch of the
+    layer kernel (no pipeline fill and drain between layers), layer l writing buffer pair l % 2."""
+    L = len(K)
+    codec.encode_chain(K, V, adapters.Wk, adapters.Wv, cache.Kcodes, cache.Kscales, cache.Vcodes, cache.Vscales,
+                       adapters.bk, adapters.bv, [bufs.K[l % 2] for l in range(L)], [bufs.V[l % 2] for l in range(L)])
+
+
+def decode_layers(codec: api.Codec, cache: CompressedCache, adapters, bufs: PingPong,
+                  n_layers: Optional[int] = None) -> int:
+    """decode_chain through aquakv_decode_chain (see encode_layers); returns the buffer pair of the last layer."""
+    L = n_layers or len(cache.Kcodes)
+    codec.decode_chain(cache.Kcodes[:L], cache.Kscales[:L], cache.Vcodes[:L], cache.Vscales[:L], adapters.Wk[:L],
+                       adapters.Wv[:L], adapters.bk[:L], adapters.bv[:L], [bufs.K[l % 2] for l in range(L)],
+                       [bufs.V[l % 2] for l in range(L)])
+    return (L - 1) % 2
+
+
 def encode_chain_kept(codec: api.Codec, K: List[torch.Tensor], V: List[torch.Tensor], idx: torch.Tensor,
                       adapters, cache: CompressedCache, bufs: PingPong, stage_k: torch.Tensor,
                       stage_v: torch.Tensor, first_layer_16bit: bool = False) -> None:

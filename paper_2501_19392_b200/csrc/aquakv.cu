@@ -825,6 +825,135 @@ void launch_chain_dnb(int* rc, bool encode, int device, cudaStream_t st, int gri
                : launch_chain_t<false, D, NPTS, BF, false>(device, st, grid, a);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Several layers of a LARGE call per launch of the layer kernel (the chain entry points beyond the
+// chain kernel's token limit): layers without predictors run through the per-layer row kernels, runs
+// of predicted layers go to the layer kernel kLayerBatchMax at a time.
+// ---------------------------------------------------------------------------------------------
+struct LayersWs {
+  LayerWs layer;
+  size_t flags_off, flags_stride, total;
+};
+LayersWs layers_ws(const aquakv_ctx* c, int64_t T, int L) {
+  LayersWs w;
+  w.layer = layer_ws(c, T);
+  const int nb = L < kLayerBatchMax ? (L > 0 ? L : 1) : kLayerBatchMax;
+  w.flags_stride = round_up(w.layer.flags_bytes, 256);
+  w.flags_off = round_up(w.layer.total, 256);
+  w.total = w.flags_off + size_t(nb) * w.flags_stride + kWsSlack;
+  return w;
+}
+
+bool layers_supported(const aquakv_ctx* c) { return c->p.d_kv == 1024 && c->log_h == 10 && c->log_g == 10 && !uniform_backbone(c); }
+
+int run_layers(aquakv_ctx* c, bool encode, int64_t T, int32_t L, const void* const* K, const void* const* V,
+               int64_t ld_kv, const void* Khat_init, const void* Vhat_init, int64_t ld_init, const void* const* Wk,
+               const void* const* Wv, const float* const* bk, const float* const* bv, uint8_t* const* Kcodes,
+               uint16_t* const* Kscales, uint8_t* const* Vcodes, uint16_t* const* Vscales, void* const* Khat,
+               void* const* Vhat, int64_t ld_hat, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!layers_supported(c)) return AQUAKV_ERR_TOO_LARGE;
+  if (T > (int64_t(1) << 30)) return AQUAKV_ERR_UNSUPPORTED;
+  const int d = c->p.d_kv;
+  if (Wk == nullptr || Wv == nullptr || Kcodes == nullptr || Kscales == nullptr || Vcodes == nullptr || Vscales == nullptr ||
+      Khat == nullptr || Vhat == nullptr)
+    return AQUAKV_ERR_INVALID_ARG;
+  if (encode && (K == nullptr || V == nullptr)) return AQUAKV_ERR_INVALID_ARG;
+  int rc;
+  for (int l = 0; l < L; ++l) {
+    if ((rc = check_cache(Kcodes[l], Kscales[l], Vcodes[l], Vscales[l]))) return rc;
+    if (encode) {
+      if ((rc = check_rows(K[l], ld_kv, d, true))) return rc;
+      if ((rc = check_rows(V[l], ld_kv, d, true))) return rc;
+    }
+    if ((Wk[l] == nullptr) != (Wv[l] == nullptr)) return AQUAKV_ERR_INVALID_ARG;
+    if (Wk[l] != nullptr && (!aligned16(Wk[l]) || !aligned16(Wv[l]))) return AQUAKV_ERR_ALIGNMENT;
+    const float* b0 = bk ? bk[l] : nullptr;
+    const float* b1 = bv ? bv[l] : nullptr;
+    if (Wk[l] == nullptr && (b0 != nullptr || b1 != nullptr)) return AQUAKV_ERR_INVALID_ARG;
+    if ((b0 != nullptr && !aligned16(b0)) || (b1 != nullptr && !aligned16(b1))) return AQUAKV_ERR_ALIGNMENT;
+    if ((rc = check_rows(Khat[l], ld_hat, d, true))) return rc;
+    if ((rc = check_rows(Vhat[l], ld_hat, d, true))) return rc;
+    if (Khat[l] == Vhat[l] || (encode && (Khat[l] == K[l] || Khat[l] == V[l] || Vhat[l] == K[l] || Vhat[l] == V[l])))
+      return AQUAKV_ERR_INVALID_ARG;
+    // a layer reads the reconstructions of the layer before it while it writes its own
+    const void* pk = l == 0 ? Khat_init : Khat[l - 1];
+    const void* pv = l == 0 ? Vhat_init : Vhat[l - 1];
+    if (Wk[l] != nullptr) {
+      if (pk == nullptr || pv == nullptr) return AQUAKV_ERR_INVALID_ARG;
+      if (Khat[l] == pk || Khat[l] == pv || Vhat[l] == pk || Vhat[l] == pv) return AQUAKV_ERR_INVALID_ARG;
+    }
+  }
+  if (Wk[0] != nullptr) {
+    if ((rc = check_rows(Khat_init, ld_init, d, true))) return rc;
+    if ((rc = check_rows(Vhat_init, ld_init, d, true))) return rc;
+  } else if (Khat_init != nullptr || Vhat_init != nullptr) {
+    return AQUAKV_ERR_INVALID_ARG;
+  }
+  const LayersWs ws = layers_ws(c, T, L);
+  if (workspace == nullptr || workspace_bytes < ws.total) return AQUAKV_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  uint8_t* wsb = ws_base(workspace);
+  const int grid = ws.layer.grid_mw * (d / kBN);
+  int l = 0;
+  while (l < L) {
+    if (Wk[l] == nullptr) {
+      // no predictor: the row kernels alone
+      const int cb = c->code_bytes, ng = c->n_groups;
+      const int64_t chunk = int64_t(1) << 30;
+      for (int64_t t0 = 0; t0 < T; t0 += chunk) {
+        const int rows = int(T - t0 < chunk ? T - t0 : chunk);
+        uint16_t* kh = static_cast<uint16_t*>(Khat[l]) + t0 * ld_hat;
+        uint16_t* vh = static_cast<uint16_t*>(Vhat[l]) + t0 * ld_hat;
+        if (encode) {
+          rc = launch_encode_rows(c, st, kRoleK, rows, static_cast<const uint16_t*>(K[l]) + t0 * ld_kv, ld_kv, nullptr, d,
+                                  Kcodes[l] + t0 * cb, Kscales[l] + t0 * ng, kh, ld_hat);
+          if (rc) return rc;
+          rc = launch_encode_rows(c, st, kRoleV, rows, static_cast<const uint16_t*>(V[l]) + t0 * ld_kv, ld_kv, nullptr, d,
+                                  Vcodes[l] + t0 * cb, Vscales[l] + t0 * ng, vh, ld_hat);
+        } else {
+          rc = launch_decode_rows(c, st, kRoleK, rows, Kcodes[l] + t0 * cb, Kscales[l] + t0 * ng, nullptr, d, kh, ld_hat);
+          if (rc) return rc;
+          rc = launch_decode_rows(c, st, kRoleV, rows, Vcodes[l] + t0 * cb, Vscales[l] + t0 * ng, nullptr, d, vh, ld_hat);
+        }
+        if (rc) return rc;
+      }
+      ++l;
+      continue;
+    }
+    // a run of predicted layers, at most kLayerBatchMax per launch
+    int n = 0;
+    while (l + n < L && n < kLayerBatchMax && Wk[l + n] != nullptr) ++n;
+    static thread_local LayerBatch<kLayerBatchMax> B;      // 26 KB: not on the stack of a caller's thread
+    B.n_layers = n;
+    for (int i = 0; i < n; ++i) {
+      const int li = l + i;
+      const void* pk = li == 0 ? Khat_init : Khat[li - 1];
+      const void* pv = li == 0 ? Vhat_init : Vhat[li - 1];
+      const int64_t ldp = li == 0 ? ld_init : ld_hat;
+      rc = fill_layer(c, ws.layer, wsb, reinterpret_cast<int*>(wsb + ws.flags_off + size_t(i) * ws.flags_stride), T,
+                      encode ? K[li] : nullptr, encode ? V[li] : nullptr, ld_kv, pk, pv, ldp, Wk[li], Wv[li],
+                      bk ? bk[li] : nullptr, bv ? bv[li] : nullptr, Kcodes[li], Kscales[li], Vcodes[li], Vscales[li],
+                      Khat[li], Vhat[li], ld_hat, nullptr, &B.layer[i], &B.maps[i]);
+      if (rc) return rc;
+    }
+    if (cudaMemsetAsync(wsb + ws.flags_off, 0, size_t(n) * ws.flags_stride, st) != cudaSuccess) return AQUAKV_ERR_CUDA;
+    {
+      ProfScope prof(c, st, AQUAKV_KERNEL_LAYER);
+      if (encode) {
+        AQ_DISPATCH_DNB(launch_layer_enc_t, &rc, c->device, st, grid, B);
+      } else {
+        AQ_DISPATCH_DNB(launch_layer_dec_t, &rc, c->device, st, grid, B);
+      }
+    }
+    if (rc) return rc;
+    ++c->launches;
+    if (cudaGetLastError() != cudaSuccess) return AQUAKV_ERR_CUDA;
+    l += n;
+  }
+  return AQUAKV_OK;
+}
+
 // Algorithm 2 (encode) or Algorithm 3 for n_layers layers in one launch; argument checks included.
 int run_chain(aquakv_ctx* c, bool encode, int64_t T, int32_t L, const void* const* K, const void* const* V,
               int64_t ld_kv, const void* Khat_init, const void* Vhat_init, int64_t ld_init, const void* const* Wk,
@@ -834,7 +963,10 @@ int run_chain(aquakv_ctx* c, bool encode, int64_t T, int32_t L, const void* cons
   if (c != nullptr && uniform_backbone(c)) return AQUAKV_ERR_UNSUPPORTED;   // per-layer entry points only
   if (c == nullptr || T < 0 || L < 0) return AQUAKV_ERR_INVALID_ARG;
   if (T == 0 || L == 0) return AQUAKV_OK;
-  if (T > kChainMaxTokens || L > kChainMaxLayers) return AQUAKV_ERR_TOO_LARGE;
+  if (L > kChainMaxLayers) return AQUAKV_ERR_TOO_LARGE;
+  if (T > kChainMaxTokens)      // beyond the chain kernel: launches of the layer kernel that take several layers each
+    return run_layers(c, encode, T, L, K, V, ld_kv, Khat_init, Vhat_init, ld_init, Wk, Wv, bk, bv, Kcodes, Kscales, Vcodes,
+                      Vscales, Khat, Vhat, ld_hat, workspace, workspace_bytes, cuda_stream);
   const int d = c->p.d_kv;
   if (d == 1024 && !(c->log_h == 10 && c->log_g == 10)) return AQUAKV_ERR_UNSUPPORTED;
   if (Wk == nullptr || Wv == nullptr || Kcodes == nullptr || Kscales == nullptr || Vcodes == nullptr || Vscales == nullptr)
@@ -1518,7 +1650,8 @@ int aquakv_decode(aquakv_ctx* c, int64_t n_tokens, const uint8_t* Kcodes, const 
 
 size_t aquakv_chain_workspace_bytes(const aquakv_ctx* c, int64_t n_tokens, int32_t n_layers) {
   if (c != nullptr && uniform_backbone(c)) return 0;
-  if (c == nullptr || n_tokens <= 0 || n_layers <= 0 || n_tokens > kChainMaxTokens || n_layers > kChainMaxLayers) return 0;
+  if (c == nullptr || n_tokens <= 0 || n_layers <= 0 || n_layers > kChainMaxLayers) return 0;
+  if (n_tokens > kChainMaxTokens) return layers_supported(c) ? layers_ws(c, n_tokens, n_layers).total : 0;
   return chain_ws(c, n_tokens, n_layers).total;
 }
 

@@ -212,6 +212,7 @@ struct LayerBatch {
   LayerArgs layer[kBatch];
   LayerMaps maps[kBatch];
 };
+static_assert(sizeof(LayerBatch<kLayerBatchMax>) <= 32764, "kernel parameters are limited to 32764 bytes");
 
 __device__ __forceinline__ void layer_job(int j, int n_waves, int& phase, int& wave) {
   if (j == 0) { phase = 0; wave = 0; }
@@ -494,10 +495,16 @@ layer_kernel(const __grid_constant__ LayerBatch<kBatch> B) {
       // the ring slot of this job was last used nb jobs earlier (counted through the layers of the launch):
       // that job's row work must be over
       const int gj = l * n_jobs + j;
-      if (gj >= a.nb) {
-        const int lo = (gj - a.nb) / n_jobs, jo = (gj - a.nb) % n_jobs;
-        int ph_old, wave_old;
-        layer_job(jo, a.n_waves, ph_old, wave_old);
+      // ... the latest such job in whose wave this token block exists (the short last wave may not have it:
+      // nobody then read or reports on this block's part of the slot)
+      int go = gj - a.nb, ph_old = 0, wave_old = 0;
+      while (go >= 0) {
+        layer_job(go % n_jobs, a.n_waves, ph_old, wave_old);
+        if (ml < wave_rows(wave_old, a.T, a.mw, gridDim.x).blocks) break;
+        go -= a.nb;
+      }
+      if (go >= 0) {
+        const int lo = go / n_jobs, jo = go % n_jobs;
         const int target = wave_block_teams(wave_rows(wave_old, a.T, a.mw, gridDim.x), ml, gridDim.x, G::TEAMS);
         // one thread polls for the four warps; a failed wait has set the abort flag
         if (warp == 2 && lane == 0)

@@ -168,8 +168,61 @@ def test_chain_argument_errors():
                            workspace=torch.empty(1024, dtype=torch.uint8, device=DEV))
     assert e.value.status == -4
     big = torch.empty((api.CHAIN_MAX_TOKENS + 1, d), dtype=torch.bfloat16, device=DEV)
-    with pytest.raises(api.AquaKVError) as e:       # too many tokens for this entry point
+    with pytest.raises(api.AquaKVError) as e:       # a large call needs every layer's output buffers
         codec.encode_chain([big], [big], [None], [None], *[[t] for t in (Kc[0], Ks[0], Vc[0], Vs[0])],
                            workspace=torch.empty(1024, dtype=torch.uint8, device=DEV))
-    assert e.value.status == -7
+    assert e.value.status == (-1 if d == 1024 else -7)
     assert codec.launch_count() == 0 and codec.poll_status() == 0
+
+
+@pytest.mark.parametrize("T,L,n,first_pred", [(5000, 5, 16, False), (2304, 27, 16, True), (9549, 3, 64, False)])
+def test_large_calls_run_several_layers_per_launch_and_equal_the_per_layer_calls(T, L, n, first_pred):
+    """Beyond 2048 tokens the chain entry points run the layer kernel on up to 24 layers per launch; the result
+    must be the per-layer calls' bit for bit (27 layers: two launches; first_pred: layer 0 has a predictor and
+    reads Khat_init / Vhat_init)."""
+    from paper_2501_19392_b200 import api, chain
+    shape = dataclasses.replace(synth.CONFIGS[2], n_tokens=T, n_layers=L, grid_size=n)
+    codec, _ = make(shape)
+    kv = synth.kv_chain(shape, seed=8800 + L, device=DEV)
+    ad = synth.random_adapters(shape, seed=8900 + L, device=DEV)
+    Wk, Wv = list(ad.Wk), list(ad.Wv)
+    init_k = init_v = None
+    if first_pred:
+        Wk[0], Wv[0] = ad.Wk[1], ad.Wv[1]
+        init_k = synth.random_16bit((T, shape.d_kv), shape.dtype, 1, device=DEV)
+        init_v = synth.random_16bit((T, shape.d_kv), shape.dtype, 2, device=DEV)
+    ad = dataclasses.replace(ad, Wk=Wk, Wv=Wv)
+    # per-layer reference
+    ref = chain.CompressedCache.empty(codec, L, T, DEV)
+    bufs = chain.PingPong(codec, T, DEV)
+    hats = []
+    for l in range(L):
+        cur, prv = l % 2, (l + 1) % 2
+        has = Wk[l] is not None
+        pk = (init_k if l == 0 else bufs.K[prv]) if has else None
+        pv = (init_v if l == 0 else bufs.V[prv]) if has else None
+        codec.encode(kv.K[l], kv.V[l], pk, pv, Wk[l], Wv[l], None, None, ref.Kcodes[l], ref.Kscales[l], ref.Vcodes[l],
+                     ref.Vscales[l], bufs.K[cur], bufs.V[cur])
+        hats.append((bufs.K[cur].clone(), bufs.V[cur].clone()))
+    before = codec.launch_count()
+    got = chain.CompressedCache.empty(codec, L, T, DEV)
+    bufs2 = chain.PingPong(codec, T, DEV)
+    codec.encode_chain(kv.K, kv.V, Wk, Wv, got.Kcodes, got.Kscales, got.Vcodes, got.Vscales, None, None,
+                       [bufs2.K[l % 2] for l in range(L)], [bufs2.V[l % 2] for l in range(L)], init_k, init_v)
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    n_pred = sum(w is not None for w in Wk)
+    assert codec.launch_count() - before == 2 * (L - n_pred) + (n_pred + 23) // 24       # row kernels of layer 0 + batches
+    for l in range(L):
+        assert torch.equal(got.Kcodes[l], ref.Kcodes[l]) and torch.equal(got.Vcodes[l], ref.Vcodes[l]), l
+        assert torch.equal(got.Kscales[l], ref.Kscales[l]) and torch.equal(got.Vscales[l], ref.Vscales[l]), l
+    assert torch.equal(bufs2.K[(L - 1) % 2], hats[-1][0]) and torch.equal(bufs2.V[(L - 1) % 2], hats[-1][1])
+    assert torch.equal(bufs2.K[(L - 2) % 2], hats[-2][0]) and torch.equal(bufs2.V[(L - 2) % 2], hats[-2][1])
+    # decode through the same entry point reproduces the reconstructions
+    bufs3 = chain.PingPong(codec, T, DEV)
+    codec.decode_chain(got.Kcodes, got.Kscales, got.Vcodes, got.Vscales, Wk, Wv, None, None,
+                       [bufs3.K[l % 2] for l in range(L)], [bufs3.V[l % 2] for l in range(L)], init_k, init_v)
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    assert torch.equal(bufs3.K[(L - 1) % 2], hats[-1][0]) and torch.equal(bufs3.V[(L - 1) % 2], hats[-1][1])
+    assert torch.equal(bufs3.K[(L - 2) % 2], hats[-2][0]) and torch.equal(bufs3.V[(L - 2) % 2], hats[-2][1])
