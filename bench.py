@@ -679,10 +679,21 @@ def main():
         "e2e": e2e,
     }
     if world == 1 and not args.no_other_configs and not (args.tokens or args.layers):
+        # the same encode and plain-decode chains through aquakv_encode_chain / aquakv_decode_chain, which run up
+        # to 24 layers per launch of the layer kernel at this size (no pipeline fill and drain between layers)
+        multi = []
+        for name, fn, enc in (("encode_layers", lambda: chain.encode_layers(codec, kv.K, kv.V, ad, cache, bufs), True),
+                              ("decode_layers", lambda: chain.decode_layers(codec, cache, ad, bufs), False)):
+            ms_chain = _time_calls(fn, 5, warm=2)
+            multi.append(_shape_entry(peaks, shape, name, T, ms_chain / L, _shape_bytes(shape, T, enc), config=2,
+                                      ms_chain=ms_chain, chain_layers=L,
+                                      note="all layers through the chain entry point (24 layers per launch); per layer = "
+                                           "chain time / layers, the unpredicted first layer included"))
+        assert codec.poll_status() == 0
         del kv, cache, bufs, q, out
         torch.cuda.empty_cache()
         result["ops_by_config"] = ([dict(config=2, workload=shape.name, op=name, tokens_per_call=T, **v)
-                                    for name, v in roof.items()] + ops_by_config(api, chain, peaks, dev) +
+                                    for name, v in roof.items()] + multi + ops_by_config(api, chain, peaks, dev) +
                                    [calibration_entry(api, peaks, dev)] + uniform_backbone_entries(api, chain, peaks, dev))
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = oracle_baseline(shape, n_q)
