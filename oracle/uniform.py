@@ -13,6 +13,13 @@ and decoder agree; a value goes to the nearest level, the lower one on an exact 
 group of zeros has scale 0 and level 0.  The code of a value is its level + 2^(b-1) as an unsigned
 b-bit number; codes are packed LSB-first in value order; no rotation, no sign flips.  Predictors,
 residual and add-back are those of Algorithms 2 and 3: codes = Q(x - pred), hat = round16(pred + Q^-1).
+
+Rotated variant (the appendix' additional results for Section 4.1: a backbone that "combines Randomized
+Hadamard Transform (RHT) with standard non-vector quantization", group size 1024).  Reading: the
+residual is multiplied by the role's random signs and rotated by the orthonormal Hadamard matrix in
+blocks of `had_block` values (the transform of Section 3.1's vector quantizer), the ROTATED values are
+quantized as above (the group's absmax is taken after the rotation), and Q^-1 rotates the levels times
+scale back and multiplies by the signs again: Q(r) = U(H (s . r) / sqrt(h)), Q^-1 = s . H(U^-1) / sqrt(h).
 """
 from __future__ import annotations
 
@@ -20,7 +27,7 @@ from typing import Optional, Sequence
 
 import numpy as np
 
-from . import F16, Oracle
+from . import F16, Oracle, hadamard_butterfly
 from .calibration import bits_to_double, double_to_bits
 
 
@@ -66,15 +73,49 @@ def dequantize(codes: np.ndarray, scales: np.ndarray, b: int, g: int, d: int) ->
     return (q.reshape(T, d // g, g) * s16[:, :, None]).reshape(T, d)
 
 
+def rotate(R: np.ndarray, signs: np.ndarray, h: int) -> np.ndarray:
+    """Rows of R times the signs, then the orthonormal Hadamard transform of every block of h values."""
+    R = np.asarray(R, dtype=np.float64) * np.asarray(signs, dtype=np.float64)[None, :]
+    Y = np.empty_like(R)
+    for t in range(R.shape[0]):
+        for o in range(0, R.shape[1], h):
+            Y[t, o:o + h] = hadamard_butterfly(R[t, o:o + h]) / np.sqrt(float(h))
+    return Y
+
+
+def rotate_back(Y: np.ndarray, signs: np.ndarray, h: int) -> np.ndarray:
+    """Inverse of `rotate`: the Hadamard matrix is symmetric and orthonormal, the signs are +-1."""
+    Y = np.asarray(Y, dtype=np.float64)
+    R = np.empty_like(Y)
+    for t in range(Y.shape[0]):
+        for o in range(0, Y.shape[1], h):
+            R[t, o:o + h] = hadamard_butterfly(Y[t, o:o + h]) / np.sqrt(float(h))
+    return R * np.asarray(signs, dtype=np.float64)[None, :]
+
+
 class UniformOracle:
     """Algorithm 2 / 3 phases with the uniform backbone.  `linear` is a codec oracle of the same width
     and 16-bit type, used for the predictor product only."""
 
-    def __init__(self, linear: Oracle, bits: int, group: int):
-        self.linear, self.b, self.g = linear, bits, group
+    def __init__(self, linear: Oracle, bits: int, group: int, had_block: int = 1,
+                 signs_k: Optional[np.ndarray] = None, signs_v: Optional[np.ndarray] = None):
+        self.linear, self.b, self.g, self.h = linear, bits, group, had_block
         self.d, self.dtype = linear.d, linear.dtype
         self.code_bytes = self.d * bits // 8
         self.n_groups = self.d // group
+        self.signs = {"k": signs_k, "v": signs_v}
+        assert had_block == 1 or (signs_k is not None and signs_v is not None)
+
+    def quantize(self, R: np.ndarray, role: str = "k"):
+        """Q on double residuals (rotated first when had_block > 1); `Y` is what the levels were chosen for."""
+        Y = rotate(R, self.signs[role], self.h) if self.h > 1 else np.asarray(R, dtype=np.float64)
+        out = quantize(Y, self.b, self.g)
+        out["Y"] = Y
+        return out
+
+    def dequantize(self, codes, scales, role: str = "k") -> np.ndarray:
+        Yhat = dequantize(codes, scales, self.b, self.g, self.d)
+        return rotate_back(Yhat, self.signs[role], self.h) if self.h > 1 else Yhat
 
     def _pred(self, T, inputs, W, bias):
         if W is None:
@@ -82,15 +123,15 @@ class UniformOracle:
         return self.linear.predict(list(inputs), W, bias)
 
     def encode_phase(self, X: np.ndarray, inputs: Sequence[np.ndarray], W: Optional[np.ndarray],
-                     bias: Optional[np.ndarray] = None):
+                     bias: Optional[np.ndarray] = None, role: str = "k"):
         x = bits_to_double(X, self.dtype)
         pred = self._pred(x.shape[0], inputs, W, bias)
-        out = quantize(x - pred, self.b, self.g)                                   # Algorithm 2 lines 6 / 8
-        hat_exact = pred + dequantize(out["codes"], out["scales"], self.b, self.g, self.d)   # lines 7 / 9
+        out = self.quantize(x - pred, role)                                        # Algorithm 2 lines 6 / 8
+        hat_exact = pred + self.dequantize(out["codes"], out["scales"], role)      # lines 7 / 9
         out.update(hat=double_to_bits(hat_exact, self.dtype), hat_exact=hat_exact, pred=pred)
         return out
 
-    def decode_phase(self, codes, scales, inputs, W, bias=None):
+    def decode_phase(self, codes, scales, inputs, W, bias=None, role: str = "k"):
         T = codes.shape[0]
-        hat_exact = self._pred(T, inputs, W, bias) + dequantize(codes, scales, self.b, self.g, self.d)   # Algorithm 3 lines 5 / 7
+        hat_exact = self._pred(T, inputs, W, bias) + self.dequantize(codes, scales, role)   # Algorithm 3 lines 5 / 7
         return dict(hat=double_to_bits(hat_exact, self.dtype), hat_exact=hat_exact)

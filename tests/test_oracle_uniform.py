@@ -100,3 +100,103 @@ def test_phases_round_trip_and_reduce_to_the_plain_quantizer():
     s = bits_to_double(e1["scales"], oracle.F16).repeat(64, axis=1)
     err = np.abs(x - bits_to_double(e1["hat"], oracle.BF16))
     assert (err <= s * (1 + 2.0 ** -9) + np.abs(x) * 2.0 ** -8).all()
+
+
+# ---- rotated variant (random signs + Hadamard rotation before the uniform levels) -------------------
+
+def _sylvester(h):
+    """Orthonormal Hadamard matrix by Kronecker products (independent of the oracle's butterflies)."""
+    H = np.ones((1, 1))
+    while H.shape[0] < h:
+        H = np.kron(H, np.array([[1.0, 1.0], [1.0, -1.0]]))
+    return H / np.sqrt(float(h))
+
+
+@pytest.mark.parametrize("d,h", [(256, 64), (512, 512), (1024, 256)])
+def test_rotation_is_the_signed_blockwise_hadamard_matrix_and_its_own_inverse(d, h):
+    rng = np.random.default_rng(d + h)
+    R = rng.standard_normal((5, d))
+    s = synth.hadamard_signs(d, 11)
+    Y = uq.rotate(R, s, h)
+    H = _sylvester(h)
+    want = np.concatenate([(R * s)[:, o:o + h] @ H.T for o in range(0, d, h)], axis=1)
+    np.testing.assert_allclose(Y, want, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(np.linalg.norm(Y, axis=1), np.linalg.norm(R, axis=1), rtol=1e-13)
+    np.testing.assert_allclose(uq.rotate_back(Y, s, h), R, rtol=0, atol=1e-12)
+
+
+def _rotated_oracle(d, h, b, g, dtype=oracle.BF16):
+    grid = synth.lloyd_grid(16, seed=7, n_samples=1 << 12, iters=10)
+    sk, sv = synth.hadamard_signs(d, 1), synth.hadamard_signs(d, 2)
+    lin = oracle.Oracle(d, 64, 64, grid, dtype, sk, sv)
+    return uq.UniformOracle(lin, b, g, had_block=h, signs_k=sk, signs_v=sv), sk, sv
+
+
+def test_rotated_quantizer_on_a_single_hadamard_column_has_a_closed_form():
+    # r = a * s . c with c the j-th +-1 Hadamard column: s . r = a * sqrt(h) * (orthonormal column j), which the
+    # orthonormal transform maps to the spike a * sqrt(h) * e_j.
+    d, h, b, g, j, a = 256, 256, 2, 256, 37, 0.75
+    o, sk, sv = _rotated_oracle(d, h, b, g)
+    col = _sylvester(h)[:, j] * np.sqrt(float(h))          # +-1 entries
+    R = (a * sk * col)[None, :]
+    q = o.quantize(R, "k")
+    spike = a * np.sqrt(float(h))                          # 12.0: exactly representable, scale 6.0 exact in fp16
+    assert np.allclose(q["Y"][0, j], spike, atol=1e-12) and np.abs(np.delete(q["Y"][0], j)).max() < 1e-12
+    lv = uq._unpack(q["codes"], b, d)[0] - 2
+    assert lv[j] == 1 and (np.delete(lv, j) == 0).all()     # the positive maximum saturates at the top level
+    assert q["scales"][0, 0] == np.float16(spike / 2).view(np.uint16)
+    back = o.dequantize(q["codes"], q["scales"], "k")
+    np.testing.assert_allclose(back[0], 0.5 * R[0], rtol=0, atol=1e-12)   # level 1 of 2: half the spike
+    # the value signs give another row
+    assert not np.array_equal(o.quantize(R, "v")["codes"], q["codes"])
+
+
+def test_rotated_quantizer_error_is_the_rotated_domain_error_and_had_block_one_is_the_plain_one():
+    d, h, b, g = 512, 128, 4, 64
+    o, sk, sv = _rotated_oracle(d, h, b, g)
+    rng = np.random.default_rng(3)
+    R = rng.standard_normal((32, d))
+    q = o.quantize(R, "v")
+    Yhat = uq.dequantize(q["codes"], q["scales"], b, g, d)
+    back = o.dequantize(q["codes"], q["scales"], "v")
+    np.testing.assert_allclose(np.linalg.norm(R - back, axis=1), np.linalg.norm(q["Y"] - Yhat, axis=1), rtol=1e-12)
+    # levels are those of the plain quantizer applied to the rotated rows
+    assert np.array_equal(q["codes"], uq.quantize(uq.rotate(R, sv, h), b, g)["codes"])
+    plain = uq.UniformOracle(o.linear, b, g)
+    p = plain.quantize(R)
+    assert np.array_equal(p["codes"], uq.quantize(R, b, g)["codes"])
+    assert np.array_equal(plain.dequantize(p["codes"], p["scales"]), uq.dequantize(p["codes"], p["scales"], b, g, d))
+
+
+def test_rotation_spreads_an_outlier_so_that_the_other_values_survive():
+    # Why the appendix' rotated backbone works with one group per row where the plain one collapses:
+    # one outlier sets the plain scale and flattens everything else to level 0 (or -1 .. 0).
+    d, h, b, g = 1024, 1024, 2, 1024
+    o, sk, sv = _rotated_oracle(d, h, b, g)
+    rng = np.random.default_rng(5)
+    R = rng.standard_normal((16, d))
+    R[:, 17] = 60.0
+    plain = uq.UniformOracle(o.linear, b, g)
+    qp = plain.quantize(R)
+    err_plain = np.linalg.norm(np.delete(R - plain.dequantize(qp["codes"], qp["scales"]), 17, axis=1), axis=1)
+    qr = o.quantize(R, "k")
+    err_rot = np.linalg.norm(R - o.dequantize(qr["codes"], qr["scales"], "k"), axis=1)
+    base = np.linalg.norm(np.delete(R, 17, axis=1), axis=1)
+    assert (err_plain > 0.95 * base).all()          # nothing but the outlier is kept
+    assert (err_rot < 0.8 * np.linalg.norm(R, axis=1)).all()
+
+
+def test_rotated_phases_round_trip():
+    d, T = 256, 64
+    o, sk, sv = _rotated_oracle(d, 256, 2, 256)
+    X = synth.to_bits(synth.random_16bit((T, d), oracle.BF16, 3))
+    prev = synth.to_bits(synth.random_16bit((T, d), oracle.BF16, 4))
+    W = synth.to_bits(synth.random_16bit((d, d), oracle.BF16, 5, std=1.0 / 16))
+    for role in ("k", "v"):
+        e = o.encode_phase(X, [prev], W, role=role)
+        dcd = o.decode_phase(e["codes"], e["scales"], [prev], W, role=role)
+        assert np.array_equal(dcd["hat"], e["hat"])
+        x = bits_to_double(X, oracle.BF16)
+        want = e["pred"] + o.dequantize(e["codes"], e["scales"], role)
+        np.testing.assert_allclose(e["hat_exact"], want, rtol=0, atol=0)
+        assert np.array_equal(e["codes"], o.quantize(x - e["pred"], role)["codes"])
