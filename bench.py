@@ -456,47 +456,60 @@ def calibration_entry(api, peaks, dev, reps=3):
 
 
 def uniform_backbone_entries(api, chain, peaks, dev, reps=5):
-    """The alternative backbone (uniform round-to-nearest, absmax normalisation, groups of 64, 2 bits per
-    value = 2.25 with the scales) on the prefill-shaped workload: time of one predicted layer through the
-    per-layer entry points (two launches per phase: predictor GEMM, row kernel), and what fitted predictors
-    buy this backbone (Section 4.1 evaluates each backbone with and without them)."""
+    """The alternative backbones built on uniform round-to-nearest levels with absmax normalisation, 2 bits
+    per value, on the prefill-shaped workload: the plain one with groups of 64 (2.25 bits with the scales)
+    and the rotated one with one group per row (random signs + Hadamard rotation first; 2.02 bits).  Time of
+    one predicted layer through the per-layer entry points (two launches per phase: predictor GEMM, row
+    kernel), and what fitted predictors buy each backbone (Section 4.1 evaluates each backbone with and
+    without them)."""
     from paper_2501_19392_b200 import calibrate as gcal
-    shape = dataclasses.replace(synth.CONFIGS[2], n_layers=3, had_block=1, scale_group=64, grid_size=4)
-    T, d, L = shape.n_tokens, shape.d_kv, shape.n_layers
-    codec = api.Codec(d, 1, 64, None, shape.dtype, levels=4)
-    kv = synth.kv_chain(shape, seed=7001, device=dev)
-    preds, recs = gcal.calibrate(codec, kv.K, kv.V, rate=1e-3, keep_reconstructions=True)
-    l = L - 1
-    mk = lambda cols, dt: torch.empty((T, cols), dtype=dt, device=dev)
-    Kc, Ks, Vc, Vs = mk(codec.code_bytes, torch.uint8), mk(codec.n_groups, torch.float16), \
-        mk(codec.code_bytes, torch.uint8), mk(codec.n_groups, torch.float16)
-    Kh, Vh = mk(d, codec.torch_dtype), mk(d, codec.torch_dtype)
-    enc = lambda: codec.encode(kv.K[l], kv.V[l], recs[l - 1][0], recs[l - 1][1], preds.Wk[l], preds.Wv[l], None, None,
-                               Kc, Ks, Vc, Vs, Kh, Vh)
-    ms_enc = _time_calls(enc, reps)
-    dec = lambda: codec.decode(Kc, Ks, Vc, Vs, recs[l - 1][0], recs[l - 1][1], preds.Wk[l], preds.Wv[l], None, None,
-                               Kh, Vh)
-    ms_dec = _time_calls(dec, reps)
-    assert codec.poll_status() == 0
 
     def rel_err(X, Xh):
         X, Xh = X.float(), Xh.float()
         return float(((X - Xh) ** 2).sum() / ((X - X.mean(dim=0)) ** 2).sum())
 
-    _, _, Kd = codec.encode_phase(api.ROLE_KEY, kv.K[l])
-    _, _, Vd = codec.encode_phase(api.ROLE_VALUE, kv.V[l])
-    quality = {"fitted_predictors": {"K": rel_err(kv.K[l], recs[l][0]), "V": rel_err(kv.V[l], recs[l][1])},
-               "no_predictor": {"K": rel_err(kv.K[l], Kd), "V": rel_err(kv.V[l], Vd)}}
-    code_bytes = 2 * codec.code_bytes + 2 * 2 * codec.n_groups
-    by_enc = 4 * d * 2 + 4 * d + code_bytes + 6.0 * d * d * 2 / T       # K,V in; prev in; K^,V^ out; codes; adapters
-    by_dec = 4 * d + 4 * d + code_bytes + 6.0 * d * d * 2 / T
     out = []
-    for op, ms, by in (("encode_uniform_backbone", ms_enc, by_enc), ("decode_uniform_backbone", ms_dec, by_dec)):
-        out.append(_shape_entry(peaks, shape, op, T, ms, by, config="uniform-backbone", bits_per_value=2.25,
-                                scale_group=64, relative_error_last_layer=quality,
-                                note="per predicted layer; two launches per phase (tcgen05 predictor GEMM, row kernel)"))
-    del kv, recs
-    torch.cuda.empty_cache()
+    for tag, h, g in (("uniform-backbone", 1, 64), ("rotated-uniform-backbone", 1024, 1024)):
+        shape = dataclasses.replace(synth.CONFIGS[2], n_layers=3, had_block=h, scale_group=g, grid_size=4)
+        T, d, L = shape.n_tokens, shape.d_kv, shape.n_layers
+        signs = (synth.hadamard_signs(d, 1), synth.hadamard_signs(d, 2)) if h > 1 else (None, None)
+        codec = api.Codec(d, h, g, None, shape.dtype, levels=4, signs_k=signs[0], signs_v=signs[1])
+        kv = synth.kv_chain(shape, seed=7001, device=dev)
+        preds, recs = gcal.calibrate(codec, kv.K, kv.V, rate=1e-3, keep_reconstructions=True)
+        l = L - 1
+        mk = lambda cols, dt: torch.empty((T, cols), dtype=dt, device=dev)
+        Kc, Ks, Vc, Vs = mk(codec.code_bytes, torch.uint8), mk(codec.n_groups, torch.float16), \
+            mk(codec.code_bytes, torch.uint8), mk(codec.n_groups, torch.float16)
+        Kh, Vh = mk(d, codec.torch_dtype), mk(d, codec.torch_dtype)
+        enc = lambda: codec.encode(kv.K[l], kv.V[l], recs[l - 1][0], recs[l - 1][1], preds.Wk[l], preds.Wv[l], None,
+                                   None, Kc, Ks, Vc, Vs, Kh, Vh)
+        ms_enc = _time_calls(enc, reps)
+        dec = lambda: codec.decode(Kc, Ks, Vc, Vs, recs[l - 1][0], recs[l - 1][1], preds.Wk[l], preds.Wv[l], None,
+                                   None, Kh, Vh)
+        ms_dec = _time_calls(dec, reps)
+        assert codec.poll_status() == 0
+        _, _, Kd = codec.encode_phase(api.ROLE_KEY, kv.K[l])
+        _, _, Vd = codec.encode_phase(api.ROLE_VALUE, kv.V[l])
+        quality = {"fitted_predictors": {"K": rel_err(kv.K[l], recs[l][0]), "V": rel_err(kv.V[l], recs[l][1])},
+                   "no_predictor": {"K": rel_err(kv.K[l], Kd), "V": rel_err(kv.V[l], Vd)}}
+        if h > 1:      # the same group size without the rotation (the appendix' "larger group size" row)
+            plain = api.Codec(d, 1, g, None, shape.dtype, levels=4)
+            _, _, Kp = plain.encode_phase(api.ROLE_KEY, kv.K[l])
+            _, _, Vp = plain.encode_phase(api.ROLE_VALUE, kv.V[l])
+            quality["no_predictor_no_rotation_same_group"] = {"K": rel_err(kv.K[l], Kp), "V": rel_err(kv.V[l], Vp)}
+            assert plain.poll_status() == 0
+            plain.close()
+        code_bytes = 2 * codec.code_bytes + 2 * 2 * codec.n_groups
+        by_enc = 4 * d * 2 + 4 * d + code_bytes + 6.0 * d * d * 2 / T       # K,V in; prev in; K^,V^ out; codes; adapters
+        by_dec = 4 * d + 4 * d + code_bytes + 6.0 * d * d * 2 / T
+        for op, ms, by in (("encode_" + tag.replace("-", "_"), ms_enc, by_enc),
+                           ("decode_" + tag.replace("-", "_"), ms_dec, by_dec)):
+            out.append(_shape_entry(peaks, shape, op, T, ms, by, config=tag, bits_per_value=2.0 + 16.0 / g,
+                                    scale_group=g, had_block=h, relative_error_last_layer=quality,
+                                    note="per predicted layer; two launches per phase (tcgen05 predictor GEMM, row kernel)"))
+        del kv, recs, preds, Kd, Vd
+        codec.close()
+        torch.cuda.empty_cache()
     return out
 
 

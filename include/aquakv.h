@@ -78,7 +78,7 @@ typedef struct aquakv_params {
   int32_t d_kv;        /* values per token row; supported: 256, 512, 1024                       */
   int32_t had_block;   /* h: Hadamard block, power of two, 64 <= h <= d_kv, divides d_kv        */
   int32_t scale_group; /* g: values per fp16 scale; multiple of h that divides d_kv             */
-  int32_t grid_dim;    /* p: values per code; must be 2                                         */
+  int32_t grid_dim;    /* p: values per code; 2 (1: the uniform backbone, see aquakv_create)    */
   int32_t grid_size;   /* n: 16, 64 or 256 grid points (2, 3, 4 bits per value)                 */
   int32_t dtype;       /* AQUAKV_F16 or AQUAKV_BF16                                             */
 } aquakv_params;
@@ -102,9 +102,14 @@ int aquakv_code_bytes(const aquakv_params* params);
  * grid_dim = 1 selects it.  grid_size = 2^b in {4, 8, 16} is then the number of levels PER VALUE (b bits
  * per value): the signed integers -2^(b-1) .. 2^(b-1)-1 times the group scale, scale = absmax / 2^(b-1)
  * stored as fp16, nearest level with the lower one on a tie, saturation at the ends, code = level +
- * 2^(b-1), codes packed LSB-first in value order (d_kv * b / 8 bytes per token); had_block must be 1 (no
- * rotation), scale_group a power of two from 32 to d_kv; grid_host and the sign arrays are not read and may be
- * NULL.  Such a ctx serves aquakv_encode / aquakv_decode (with predictors: two launches per phase, and
+ * 2^(b-1), codes packed LSB-first in value order (d_kv * b / 8 bytes per token); scale_group a power of
+ * two from 32 to d_kv; grid_host is not read and may be NULL.  had_block = 1: no rotation, the sign arrays
+ * are not read and may be NULL.  had_block = h, a power of two from 64 to d_kv (the appendix' additional
+ * results for Section 4.1: a backbone that "combines Randomized Hadamard Transform (RHT) with standard
+ * non-vector quantization"): the residual times the role's signs is rotated by the orthonormal Hadamard
+ * matrix in blocks of h values, the ROTATED values are quantized as above (absmax after the rotation;
+ * scale_group is independent of h), and the inverse rotates level * scale back and applies the signs again;
+ * the sign arrays are then required.  Such a ctx serves aquakv_encode / aquakv_decode (with predictors: two launches per phase, and
  * Khat is required because the value phase reads it), the *_phase entry points, aquakv_predict,
  * aquakv_fit_predictor and aquakv_gather_rows; the chain, no-allocation and attention entry points return
  * AQUAKV_ERR_UNSUPPORTED.

@@ -183,11 +183,15 @@ class Codec:
     def __init__(self, d_kv: int, had_block: int, scale_group: int, grid: Optional[np.ndarray], dtype: int,
                  signs_k: Optional[np.ndarray] = None, signs_v: Optional[np.ndarray] = None, levels: int = 0):
         """grid [n, 2] with sign vectors: the rotated 2-D vector quantizer.  grid None with `levels` = 2^b: the
-        uniform round-to-nearest backbone with absmax normalisation (had_block must be 1)."""
+        uniform round-to-nearest backbone with absmax normalisation; had_block 1 leaves the residual as it is,
+        had_block >= 64 (with sign vectors) rotates it first."""
         h = ctypes.c_void_p()
         if grid is None:
             self.params = Params(d_kv, had_block, scale_group, 1, int(levels), dtype)
-            rc = lib.aquakv_create(ctypes.byref(self.params), None, None, None, ctypes.byref(h))
+            sk = None if signs_k is None else np.ascontiguousarray(signs_k, dtype=np.int8)
+            sv = None if signs_v is None else np.ascontiguousarray(signs_v, dtype=np.int8)
+            rc = lib.aquakv_create(ctypes.byref(self.params), None, None if sk is None else sk.ctypes.data,
+                                   None if sv is None else sv.ctypes.data, ctypes.byref(h))
         else:
             self.params = Params(d_kv, had_block, scale_group, 2, int(np.asarray(grid).shape[0]), dtype)
             g = np.ascontiguousarray(grid, dtype=np.float32)

@@ -103,10 +103,12 @@ int check_params(const aquakv_params* p) {
   if (p->dtype != AQUAKV_F16 && p->dtype != AQUAKV_BF16) return AQUAKV_ERR_INVALID_ARG;
   if (p->grid_dim == 1) {
     // uniform round-to-nearest backbone with absmax normalisation: grid_size = 2^b levels per value,
-    // no rotation (had_block 1), groups of 32 .. d_kv values
+    // groups of 32 .. d_kv values; had_block 1: no rotation, 64 .. d_kv: random signs and a Hadamard
+    // rotation of that block size before the levels
     if (p->d_kv != 256 && p->d_kv != 512 && p->d_kv != 1024) return AQUAKV_ERR_UNSUPPORTED;
     if (p->grid_size != 4 && p->grid_size != 8 && p->grid_size != 16) return AQUAKV_ERR_UNSUPPORTED;
-    if (p->had_block != 1) return AQUAKV_ERR_UNSUPPORTED;
+    if (p->had_block != 1 && (!is_pow2(p->had_block) || p->had_block < 64 || p->had_block > p->d_kv))
+      return AQUAKV_ERR_UNSUPPORTED;
     if (!is_pow2(p->scale_group) || p->scale_group < 32 || p->scale_group > p->d_kv) return AQUAKV_ERR_UNSUPPORTED;
     return AQUAKV_OK;
   }
@@ -249,9 +251,12 @@ CodecArgs codec_args(const aquakv_ctx* c, int role, int rows) {
 inline bool uniform_backbone(const aquakv_ctx* c) { return c->p.grid_dim == 1; }
 
 // Row kernels of the uniform backbone (uniform.cuh): X == nullptr decodes.
-int launch_uniform_rows(aquakv_ctx* c, cudaStream_t st, int rows, const void* X, int64_t ldX, const float* P,
+int launch_uniform_rows(aquakv_ctx* c, cudaStream_t st, int role, int rows, const void* X, int64_t ldX, const float* P,
                         int64_t ldP, uint8_t* codes, uint16_t* scales, void* hat, int64_t ldHat) {
-  UniformArgs a;
+  UniformRotArgs ra;
+  UniformArgs& a = ra.u;
+  ra.signmask = c->d_signmask[role];
+  ra.log_h = c->log_h;
   a.X = static_cast<const uint16_t*>(X);
   a.ldX = ldX;
   a.P = P;
@@ -279,9 +284,31 @@ int launch_uniform_rows(aquakv_ctx* c, cudaStream_t st, int rows, const void* X,
       else uniform_decode_rows_kernel<BITS, false><<<grid, threads, 0, st>>>(a);                      \
     }                                                                                                 \
   } while (0)
-  if (c->bits == 2) AQ_UNIFORM(2);
+#define AQ_UNIFORM_ROT2(BITS, NCH)                                                                    \
+  do {                                                                                                \
+    if (enc) {                                                                                        \
+      if (c->bf16) uniform_rot_encode_rows_kernel<BITS, true, NCH><<<grid, threads, 0, st>>>(ra);     \
+      else uniform_rot_encode_rows_kernel<BITS, false, NCH><<<grid, threads, 0, st>>>(ra);            \
+    } else {                                                                                          \
+      if (c->bf16) uniform_rot_decode_rows_kernel<BITS, true, NCH><<<grid, threads, 0, st>>>(ra);     \
+      else uniform_rot_decode_rows_kernel<BITS, false, NCH><<<grid, threads, 0, st>>>(ra);            \
+    }                                                                                                 \
+  } while (0)
+#define AQ_UNIFORM_ROT(BITS)                                                                          \
+  do {                                                                                                \
+    if (a.d == 256) AQ_UNIFORM_ROT2(BITS, 1);                                                         \
+    else if (a.d == 512) AQ_UNIFORM_ROT2(BITS, 2);                                                    \
+    else AQ_UNIFORM_ROT2(BITS, 4);                                                                    \
+  } while (0)
+  if (c->log_h > 0) {
+    if (c->bits == 2) AQ_UNIFORM_ROT(2);
+    else if (c->bits == 3) AQ_UNIFORM_ROT(3);
+    else AQ_UNIFORM_ROT(4);
+  } else if (c->bits == 2) AQ_UNIFORM(2);
   else if (c->bits == 3) AQ_UNIFORM(3);
   else AQ_UNIFORM(4);
+#undef AQ_UNIFORM_ROT
+#undef AQ_UNIFORM_ROT2
 #undef AQ_UNIFORM
   ++c->launches;
   return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
@@ -290,7 +317,7 @@ int launch_uniform_rows(aquakv_ctx* c, cudaStream_t st, int rows, const void* X,
 int launch_encode_rows(aquakv_ctx* c, cudaStream_t st, int role, int rows, const void* X,
                        int64_t ldX, const float* P, int64_t ldP, uint8_t* codes, uint16_t* scales,
                        void* hat, int64_t ldHat) {
-  if (uniform_backbone(c)) return launch_uniform_rows(c, st, rows, X, ldX, P, ldP, codes, scales, hat, ldHat);
+  if (uniform_backbone(c)) return launch_uniform_rows(c, st, role, rows, X, ldX, P, ldP, codes, scales, hat, ldHat);
   CodecArgs a = codec_args(c, role, rows);
   a.X = static_cast<const uint16_t*>(X);
   a.ldX = ldX;
@@ -312,7 +339,7 @@ int launch_decode_rows(aquakv_ctx* c, cudaStream_t st, int role, int rows, const
                        const uint16_t* scales, const float* P, int64_t ldP, void* hat,
                        int64_t ldHat) {
   if (uniform_backbone(c))
-    return launch_uniform_rows(c, st, rows, nullptr, 0, P, ldP, const_cast<uint8_t*>(codes),
+    return launch_uniform_rows(c, st, role, rows, nullptr, 0, P, ldP, const_cast<uint8_t*>(codes),
                                const_cast<uint16_t*>(scales), hat, ldHat);
   CodecArgs a = codec_args(c, role, rows);
   a.P = P;
@@ -1115,13 +1142,15 @@ int aquakv_create(const aquakv_params* params, const float* grid_host, const int
   *out = nullptr;
   int rc = check_params(params);
   if (rc) return rc;
-  const bool uniform = params->grid_dim == 1;      // its levels are implied: grid and signs are not read
-  if (!uniform && (grid_host == nullptr || signs_k_host == nullptr || signs_v_host == nullptr))
-    return AQUAKV_ERR_INVALID_ARG;
+  const bool uniform = params->grid_dim == 1;      // its levels are implied: the grid is not read
+  const bool rotated = !uniform || params->had_block > 1;   // the signs are read
+  if (!uniform && grid_host == nullptr) return AQUAKV_ERR_INVALID_ARG;
+  if (rotated && (signs_k_host == nullptr || signs_v_host == nullptr)) return AQUAKV_ERR_INVALID_ARG;
   const int d = params->d_kv, n = params->grid_size;
-  if (!uniform) {
+  if (!uniform)
     for (int i = 0; i < 2 * n; ++i)
       if (!std::isfinite(grid_host[i])) return AQUAKV_ERR_INVALID_ARG;
+  if (rotated) {
     for (int i = 0; i < d; ++i) {
       if (signs_k_host[i] != 1 && signs_k_host[i] != -1) return AQUAKV_ERR_INVALID_ARG;
       if (signs_v_host[i] != 1 && signs_v_host[i] != -1) return AQUAKV_ERR_INVALID_ARG;
@@ -1153,7 +1182,7 @@ int aquakv_create(const aquakv_params* params, const float* grid_host, const int
   }
   uint32_t masks[2][32];
   std::memset(masks, 0, sizeof(masks));
-  for (int role = 0; role < 2 && !uniform; ++role) {
+  for (int role = 0; role < 2 && rotated; ++role) {
     const int8_t* s = role == kRoleK ? signs_k_host : signs_v_host;
     for (int e = 0; e < d; ++e)
       if (s[e] < 0) masks[role][(e >> 3) & 31] |= 1u << (((e >> 8) << 3) | (e & 7));

@@ -27,12 +27,15 @@ MARGIN = 1e-4
 SCALE_TOL = 1e-5
 
 
-def make(d, b, g, dtype):
+def make(d, b, g, dtype, h=1):
+    """h > 1: the rotated variant (random signs + Hadamard blocks of h values before the levels)."""
     from paper_2501_19392_b200 import api
-    codec = api.Codec(d, 1, g, None, dtype, levels=1 << b)
+    sk, sv = synth.hadamard_signs(d, 1), synth.hadamard_signs(d, 2)
+    codec = api.Codec(d, h, g, None, dtype, levels=1 << b, signs_k=sk if h > 1 else None,
+                      signs_v=sv if h > 1 else None)
     grid = synth.lloyd_grid(16, seed=7, n_samples=1 << 12, iters=10)
-    lin = oracle.Oracle(d, 64, 64, grid, dtype, synth.hadamard_signs(d, 1), synth.hadamard_signs(d, 2))
-    return codec, uq.UniformOracle(lin, b, g)
+    lin = oracle.Oracle(d, 64, 64, grid, dtype, sk, sv)
+    return codec, uq.UniformOracle(lin, b, g, had_block=h, signs_k=sk, signs_v=sv)
 
 
 def check_levels(gpu_codes, ora, b, d, rows_ok):
@@ -49,14 +52,17 @@ def check_levels(gpu_codes, ora, b, d, rows_ok):
     return rows_ok & (got == exp).all(axis=1)
 
 
-CASES = [(256, 2, 64, oracle.BF16, 700), (512, 3, 64, oracle.F16, 513), (1024, 4, 32, oracle.BF16, 300),
-         (1024, 2, 256, oracle.BF16, 1000), (1024, 2, 1024, oracle.BF16, 600), (512, 4, 512, oracle.F16, 257)]
+CASES = [(256, 2, 64, oracle.BF16, 700, 1), (512, 3, 64, oracle.F16, 513, 1), (1024, 4, 32, oracle.BF16, 300, 1),
+         (1024, 2, 256, oracle.BF16, 1000, 1), (1024, 2, 1024, oracle.BF16, 600, 1), (512, 4, 512, oracle.F16, 257, 1),
+         # rotated variant: one group per row (the appendix' setting), and blocks / groups of other sizes
+         (1024, 2, 1024, oracle.BF16, 700, 1024), (512, 3, 64, oracle.F16, 513, 128), (256, 4, 256, oracle.BF16, 300, 64),
+         (1024, 2, 128, oracle.BF16, 400, 512), (512, 2, 512, oracle.BF16, 257, 512)]
 
 
-@pytest.mark.parametrize("d,b,g,dtype,T", CASES)
-def test_layer0_and_predicted_phases_match_the_oracle(d, b, g, dtype, T):
+@pytest.mark.parametrize("d,b,g,dtype,T,h", CASES)
+def test_layer0_and_predicted_phases_match_the_oracle(d, b, g, dtype, T, h):
     from paper_2501_19392_b200 import api
-    codec, ora = make(d, b, g, dtype)
+    codec, ora = make(d, b, g, dtype, h)
     assert codec.code_bytes == d * b // 8 and codec.n_groups == d // g
     shape = dataclasses.replace(synth.CONFIGS[2], n_kv_heads=d // 128, head_dim=128, n_tokens=T, n_layers=2,
                                 dtype=dtype, channel_scales=True)
@@ -74,15 +80,18 @@ def test_layer0_and_predicted_phases_match_the_oracle(d, b, g, dtype, T):
     check_recon(gpu_bits(Kh), o0["hat_exact"], o0["hat"], dtype, same)
     Khd = codec.decode_phase(api.ROLE_KEY, torch.from_numpy(o0["codes"]).to(DEV),
                              torch.from_numpy(o0["scales"]).view(torch.float16).to(DEV))
-    assert np.array_equal(gpu_bits(Khd), o0["hat"])          # level * scale rounded once: exact
+    if h == 1:
+        assert np.array_equal(gpu_bits(Khd), o0["hat"])      # level * scale rounded once: exact
+    else:
+        check_recon(gpu_bits(Khd), o0["hat_exact"], o0["hat"], dtype)
     # ---- layer 1, teacher-forced on the oracle's reconstructions
-    ov0 = ora.encode_phase(bits(kv.V[0]), [], None)
+    ov0 = ora.encode_phase(bits(kv.V[0]), [], None, role="v")
     ok1 = ora.encode_phase(bits(kv.K[1]), [o0["hat"]], bits(ad.Wk[1]))
     Kc1, Ks1, Kh1 = codec.encode_phase(api.ROLE_KEY, up(kv.K[1]), up(o0["hat"]), None, up(ad.Wk[1]))
     rows_ok, _ = scale_rows_ok(gpu_bits(Ks1.view(torch.float16)), ok1["scales"], ok1["scales_exact"], SCALE_TOL)
     same = check_levels(Kc1.cpu().numpy(), ok1, b, d, rows_ok)
     check_recon(gpu_bits(Kh1), ok1["hat_exact"], ok1["hat"], dtype, same)
-    ov1 = ora.encode_phase(bits(kv.V[1]), [ov0["hat"], ok1["hat"]], bits(ad.Wv[1]))
+    ov1 = ora.encode_phase(bits(kv.V[1]), [ov0["hat"], ok1["hat"]], bits(ad.Wv[1]), role="v")
     Vc1, Vs1, Vh1 = codec.encode_phase(api.ROLE_VALUE, up(kv.V[1]), up(ov0["hat"]), up(ok1["hat"]), up(ad.Wv[1]))
     rows_ok, _ = scale_rows_ok(gpu_bits(Vs1.view(torch.float16)), ov1["scales"], ov1["scales_exact"], SCALE_TOL)
     same_v = check_levels(Vc1.cpu().numpy(), ov1, b, d, rows_ok)
@@ -123,12 +132,15 @@ def test_zero_rows_ties_and_saturation_on_the_gpu():
 
 def test_parameter_checks_and_unsupported_entry_points():
     from paper_2501_19392_b200 import api
-    for bad in (dict(had_block=64), dict(levels=32), dict(scale_group=16), dict(scale_group=512), dict(scale_group=96)):
+    for bad in (dict(had_block=32), dict(had_block=512), dict(had_block=96), dict(levels=32), dict(scale_group=16), dict(scale_group=512), dict(scale_group=96)):
         kw = dict(had_block=1, scale_group=64, levels=4)
         kw.update(bad)
         with pytest.raises(api.AquaKVError) as e:
             api.Codec(256, kw["had_block"], kw["scale_group"], None, api.BF16, levels=kw["levels"])
         assert e.value.status == -2
+    with pytest.raises(api.AquaKVError) as e:          # a rotation needs its signs
+        api.Codec(256, 64, 64, None, api.BF16, levels=4)
+    assert e.value.status == -1
     codec, _ = make(256, 2, 64, oracle.BF16)
     T = 64
     c = torch.zeros((T, codec.code_bytes), dtype=torch.uint8, device=DEV)
@@ -141,6 +153,29 @@ def test_parameter_checks_and_unsupported_entry_points():
         codec.decode_noalloc(c, s, c, s)
     assert e.value.status == -2
     assert codec.chain_workspace_bytes(T, 2) == 0
+
+
+def test_rotated_variant_spike_row_zero_row_and_clamp_on_the_gpu():
+    from paper_2501_19392_b200 import api
+    d, b, g, h = 256, 2, 256, 256
+    codec, ora = make(d, b, g, oracle.BF16, h)
+    sk = synth.hadamard_signs(d, 1).astype(np.float64)
+    j = 37
+    col = np.array([(-1.0) ** bin(i & j).count("1") for i in range(d)])
+    X = torch.zeros((3, d), dtype=torch.bfloat16)
+    X[0] = torch.from_numpy(0.75 * sk * col).to(torch.bfloat16)          # rotates to the spike 12 e_j: scale 6
+    X[2] = torch.from_numpy(1.0e30 * sk * col).to(torch.bfloat16)        # spike far beyond fp16: the scale clamps
+    o = ora.encode_phase(synth.to_bits(X), [], None)
+    Kc, Ks, Kh = codec.encode_phase(api.ROLE_KEY, X.to(DEV))
+    assert np.array_equal(Kc.cpu().numpy(), o["codes"])
+    assert np.array_equal(gpu_bits(Ks.view(torch.float16)), o["scales"])
+    lv = uq._unpack(Kc.cpu().numpy(), b, d) - 2
+    assert lv[0, j] == 1 and (np.delete(lv[0], j) == 0).all() and (lv[1] == 0).all()
+    assert float(Ks.view(torch.float16)[0, 0]) == 6.0 and float(Ks.view(torch.float16)[2, 0]) == 65504.0
+    assert np.array_equal(gpu_bits(Kh[:2]), o["hat"][:2])                 # 0.375 * (+-1) and zeros: exact
+    assert torch.equal(Kh[0].float().cpu(), 0.5 * X[0].float()) and not Kh[1].any()
+    check_recon(gpu_bits(Kh)[[0, 2]], o["hat_exact"][[0, 2]], o["hat"][[0, 2]], oracle.BF16)
+    assert codec.poll_status() == 0
 
 
 def test_fitted_predictors_help_this_backbone_too():
