@@ -364,8 +364,21 @@ def ops_by_config(api, chain, peaks, dev, reps=5):
                             _shape_bytes(shape, T, False, write_hat=False), config=5, batch=shape.batch, ctx=ctx_len,
                             n_q_heads=shape.n_q_heads, uncompressed_rows_per_sequence=n16,
                             note="compressed cache + 4 sink and 128 recent tokens per sequence in 16 bits"))
+    # and with the cached keys taken as pre-RoPE keys, rotated on the fly (Section 3.3): sinks at positions 0 .. 3,
+    # compressed tokens from 4, recent rows after them; decode, rotation and attention are separate kernels here
+    table = codec.rope_table(shape.head_dim, 500000.0, 4 + ctx_len + 128, dev)
+    pos16 = torch.cat([torch.arange(4, dtype=torch.int32), torch.arange(4 + ctx_len, 4 + ctx_len + 128, dtype=torch.int32)]).to(dev)
+    rot = lambda: codec.decode_attn_rope(q, rc.Kcodes[0], rc.Kscales[0], rc.Vcodes[0], rc.Vscales[0], ctx_len,
+                                         shape.n_kv_heads, 1.0 / math.sqrt(shape.head_dim), table, 4, K16, V16, pos16,
+                                         Kp, Vp, ad.Wk[1], ad.Wv[1], None, None, out=o)
+    ms_r = _time_calls(rot, max(2, reps // 2), warm=2)
+    out.append(_shape_entry(peaks, shape, "decode_attn_rope", T, ms_r,
+                            _shape_bytes(shape, T, False, write_hat=False), config=5, batch=shape.batch, ctx=ctx_len,
+                            n_q_heads=shape.n_q_heads, uncompressed_rows_per_sequence=n16,
+                            note="as decode_attn_buffered with rotary position encoding applied to the decoded keys; "
+                                 "three kernels per chunk (layer kernel, rotation, split-KV attention)"))
     assert codec.poll_status() == 0
-    del rc, Kp, Vp
+    del rc, Kp, Vp, table
     torch.cuda.empty_cache()
 
     # configs 6 / 7 (second workload): Qwen-2.5-shaped caches, only the 20 % of a 131072-token context that a

@@ -373,6 +373,46 @@ int aquakv_decode_attn_buffered(aquakv_ctx* ctx, int32_t batch, int64_t ctx_len,
                                 int64_t ld16, void* out, float* lse, void* Khat, void* Vhat, int64_t ld_hat,
                                 void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * Rotary position encoding on the fly (Section 3.3 "Positional embeddings": keys are compressed BEFORE
+ * RoPE, where the predictors work better, so the reconstructed keys are rotated when the block attends to
+ * them).  For a head of head_dim values and a token at position pos, frequency i < head_dim/2 has the
+ * angle pos * theta_base^(-2 i / head_dim) and rotates the pair (x[i], x[i + head_dim/2]):
+ *   y[i] = x[i] cos - x[i + head_dim/2] sin,   y[i + head_dim/2] = x[i + head_dim/2] cos + x[i] sin
+ * (the half-split pairing of the Llama-family models the paper evaluates), computed in fp32 and rounded
+ * once to the ctx's 16-bit type; values are not rotated and q must arrive rotated by its own position.
+ *
+ * aquakv_rope_table fills table[pos][i] = (cos, sin) of that angle as fp32 pairs, evaluated in double
+ * precision, for pos < n_positions (device, 16-byte aligned, n_positions * head_dim/2 * 2 floats; owned by
+ * the caller, reusable by every layer and call with the same head_dim and theta_base).  head_dim 64 or 128,
+ * theta_base > 1 (10000 in the original formulation, 500000 for Llama 3).  Errors: INVALID_ARG,
+ * UNSUPPORTED, ALIGNMENT, CUDA.
+ *
+ * aquakv_decode_attn_rope is aquakv_decode_attn_buffered with the keys rotated: compressed token t of
+ * every sequence sits at position pos0 + t, uncompressed row r of every sequence at pos16[r] (device,
+ * n_uncompressed entries, shared by the sequences of the batch; may be NULL when n_uncompressed is 0).
+ * The decoded rows returned in Khat stay un-rotated (they feed the next layer's predictor); the attention
+ * reads rotated copies that live in the workspace, so decode, rotation and attention are separate
+ * kernels here for every shape.  pos0 + ctx_len must not exceed rope_positions (INVALID_ARG); an entry of
+ * pos16 outside the table sets the status word to AQUAKV_ERR_INVALID_ARG and that key row counts as zero.
+ * Workspace: aquakv_decode_attn_rope_workspace_bytes.  Everything else as aquakv_decode_attn_buffered.
+ */
+int aquakv_rope_table(aquakv_ctx* ctx, int32_t head_dim, double theta_base, int64_t n_positions, float* table,
+                      void* cuda_stream);
+size_t aquakv_decode_attn_rope_workspace_bytes(const aquakv_ctx* ctx, int32_t batch, int64_t ctx_len,
+                                               int64_t n_uncompressed, int32_t n_q_heads, int32_t head_dim);
+int aquakv_decode_attn_rope(aquakv_ctx* ctx, int32_t batch, int64_t ctx_len, int32_t n_q_heads,
+                            int32_t n_kv_heads, int32_t head_dim, float softmax_scale, const void* q,
+                            const uint8_t* Kcodes, const uint16_t* Kscales,
+                            const uint8_t* Vcodes, const uint16_t* Vscales,
+                            const void* Khat_prev, const void* Vhat_prev, int64_t ld_prev,
+                            const void* Wk, const void* Wv, const float* bk, const float* bv,
+                            const void* K16, const void* V16, int64_t n_uncompressed, int64_t ld16,
+                            const float* rope_table, int64_t rope_positions, int64_t pos0, const int32_t* pos16,
+                            void* out, float* lse,
+                            void* Khat, void* Vhat, int64_t ld_hat,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Row gather for compressing a subset of the tokens (Section 4.3: a pruning policy such as H2O
  * selects the tokens to keep, "and [we] apply AQUA-KV compression [to] those tokens"): dst row i =

@@ -38,6 +38,7 @@ SYMBOLS = [
     "aquakv_chain_workspace_bytes", "aquakv_encode_chain", "aquakv_decode_chain",
     "aquakv_fit_workspace_bytes", "aquakv_fit_predictor", "aquakv_gather_rows",
     "aquakv_decode_attn_buffered_workspace_bytes", "aquakv_decode_attn_buffered",
+    "aquakv_rope_table", "aquakv_decode_attn_rope_workspace_bytes", "aquakv_decode_attn_rope",
 ]
 
 
@@ -105,6 +106,14 @@ def _load():
     L.aquakv_decode_attn_buffered.argtypes = [vp, i32, i64, i32, i32, i32, f32, vp, vp, vp, vp, vp,
                                               vp, vp, i64, vp, vp, vp, vp, vp, vp, i64, i64, vp, vp, vp, vp, i64,
                                               vp, sz, vp]
+    L.aquakv_rope_table.restype = ctypes.c_int
+    L.aquakv_rope_table.argtypes = [vp, i32, ctypes.c_double, i64, vp, vp]
+    L.aquakv_decode_attn_rope_workspace_bytes.restype = sz
+    L.aquakv_decode_attn_rope_workspace_bytes.argtypes = [vp, i32, i64, i64, i32, i32]
+    L.aquakv_decode_attn_rope.restype = ctypes.c_int
+    L.aquakv_decode_attn_rope.argtypes = [vp, i32, i64, i32, i32, i32, f32, vp, vp, vp, vp, vp,
+                                          vp, vp, i64, vp, vp, vp, vp, vp, vp, i64, i64, vp, i64, i64, vp,
+                                          vp, vp, vp, vp, i64, vp, sz, vp]
     L.aquakv_gather_rows.restype = ctypes.c_int
     L.aquakv_gather_rows.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp]
     L.aquakv_fit_workspace_bytes.restype = sz
@@ -371,6 +380,42 @@ class Codec:
                                              ws.numel(), _stream())
         if rc:
             raise AquaKVError(rc, "aquakv_decode_attn_buffered")
+        return out, lse
+
+    def rope_table(self, head_dim: int, theta_base: float, n_positions: int, device=None):
+        """fp32 (cos, sin) pairs [n_positions, head_dim/2, 2] of the rotary angles, evaluated in double."""
+        dev = device if device is not None else torch.device("cuda", torch.cuda.current_device())
+        table = torch.empty((n_positions, head_dim // 2, 2), dtype=torch.float32, device=dev)
+        rc = lib.aquakv_rope_table(self.h, head_dim, float(theta_base), n_positions, _ptr(table), _stream())
+        if rc:
+            raise AquaKVError(rc, "aquakv_rope_table")
+        return table
+
+    def decode_attn_rope(self, q, Kcodes, Kscales, Vcodes, Vscales, ctx_len: int, n_kv_heads: int,
+                         softmax_scale: float, rope_table, pos0: int = 0, K16=None, V16=None, pos16=None,
+                         Khat_prev=None, Vhat_prev=None, Wk=None, Wv=None, bk=None, bv=None, out=None, lse=None,
+                         Khat=None, Vhat=None, want_lse: bool = False, workspace=None):
+        """decode_attn_buffered over pre-RoPE keys: compressed token t sits at position pos0 + t, uncompressed
+        row r at pos16[r] (int32, device); q is rotated by the caller."""
+        batch, n_q_heads, head_dim = q.shape
+        dev = q.device
+        n16 = 0 if K16 is None else K16.shape[1]
+        if out is None:
+            out = torch.empty_like(q)
+        if want_lse and lse is None:
+            lse = torch.empty((batch, n_q_heads), dtype=torch.float32, device=dev)
+        ws = workspace if workspace is not None else self._workspace(int(
+            lib.aquakv_decode_attn_rope_workspace_bytes(self.h, batch, ctx_len, n16, n_q_heads, head_dim)), dev)
+        ld16 = self.d if K16 is None else int(K16.stride(1))
+        rc = lib.aquakv_decode_attn_rope(self.h, batch, ctx_len, n_q_heads, n_kv_heads, head_dim, softmax_scale,
+                                         _ptr(q), _ptr(Kcodes), _ptr(Kscales), _ptr(Vcodes), _ptr(Vscales),
+                                         _ptr(Khat_prev), _ptr(Vhat_prev), _ld(Khat_prev, self.d), _ptr(Wk),
+                                         _ptr(Wv), _ptr(bk), _ptr(bv), _ptr(K16), _ptr(V16), n16, ld16,
+                                         _ptr(rope_table), int(rope_table.shape[0]), int(pos0), _ptr(pos16),
+                                         _ptr(out), _ptr(lse), _ptr(Khat), _ptr(Vhat), _ld(Khat, self.d), _ptr(ws),
+                                         ws.numel(), _stream())
+        if rc:
+            raise AquaKVError(rc, "aquakv_decode_attn_rope")
         return out, lse
 
     def encode_phase(self, role: int, X, in0=None, in1=None, W=None, bias=None, want_hat: bool = True):

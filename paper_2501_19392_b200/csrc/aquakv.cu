@@ -27,6 +27,7 @@
 #include "codec.cuh"
 #include "gemm_pred.cuh"
 #include "layer_kernel.cuh"
+#include "rope.cuh"
 #include "search_table.h"
 #include "uniform.cuh"
 
@@ -1770,6 +1771,57 @@ int aquakv_decode_noalloc(aquakv_ctx* c, int64_t n_tokens, const uint8_t* Kcodes
   return launch_decode_rows(c, st, kRoleV, rows, Vcodes, Vscales, P, d, Vh, ld_hat);
 }
 
+// Rotary position encoding of the keys the attention reads (rope.cuh).
+struct RopeSpec {
+  const float* table;     // device, [n_pos][head_dim / 2][2]
+  int64_t n_pos;
+  int64_t pos0;           // position of compressed token 0 of every sequence
+  const int32_t* pos16;   // device, positions of the uncompressed rows [n16], or nullptr when there are none
+};
+
+static int launch_rope_rows(aquakv_ctx* c, cudaStream_t st, const RopeSpec& rope, const uint16_t* in, int64_t ld_in,
+                            uint16_t* out, int64_t ld_out, int64_t rows, int n_kv_heads, int head_dim,
+                            const int32_t* pos_list, int64_t period, int64_t row_base) {
+  if (rows <= 0) return AQUAKV_OK;
+  RopeArgs a;
+  a.in = in;
+  a.ld_in = ld_in;
+  a.out = out;
+  a.ld_out = ld_out;
+  a.rows = rows;
+  a.n_kv_heads = n_kv_heads;
+  a.head_dim = head_dim;
+  a.table = reinterpret_cast<const float2*>(rope.table);
+  a.n_pos = rope.n_pos;
+  a.pos_list = pos_list;
+  a.period = period;
+  a.row_base = row_base;
+  a.pos0 = rope.pos0;
+  a.status = c->d_status;
+  const int64_t units = rows * (c->p.d_kv / 16);
+  int64_t blocks = (units + 255) / 256;
+  const int64_t cap = int64_t(c->sm_count) * 16;
+  if (blocks > cap) blocks = cap;
+  ProfScope prof(c, st, AQUAKV_KERNEL_ATTN);
+  if (c->bf16) rope_rows_kernel<true><<<int(blocks), 256, 0, st>>>(a);
+  else rope_rows_kernel<false><<<int(blocks), 256, 0, st>>>(a);
+  ++c->launches;
+  return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
+}
+
+// Rotated copies of the keys: one chunk of decoded rows and the uncompressed rows.
+struct RopeWs {
+  size_t krot_off, k16_off, total;
+};
+static RopeWs rope_ws(const aquakv_ctx* c, size_t base_total, size_t chunk_rows, int32_t batch, int64_t n16) {
+  RopeWs w;
+  const size_t d = size_t(c->p.d_kv);
+  w.krot_off = round_up(base_total, 256);
+  w.k16_off = w.krot_off + round_up(chunk_rows * d * 2, 256);
+  w.total = w.k16_off + round_up(size_t(batch) * size_t(n16) * d * 2, 256) + kWsSlack;
+  return w;
+}
+
 // Partial-result arrays of the uncompressed rows that are attended to beside the compressed cache.
 struct AttnExtWs {
   size_t ml_off, o_off, total;
@@ -1794,11 +1846,17 @@ static int decode_attn_impl(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32
                             int64_t ld_prev, const void* Wk, const void* Wv, const float* bk,
                             const float* bv, void* out, float* lse, void* Khat, void* Vhat,
                             int64_t ld_hat, const void* K16, const void* V16, int64_t n16, int64_t ld16,
-                            void* workspace, size_t workspace_bytes, void* cuda_stream) {
+                            const RopeSpec* rope, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   if (c != nullptr && uniform_backbone(c)) return AQUAKV_ERR_UNSUPPORTED;
   if (c == nullptr || batch < 0 || ctx_len < 0 || n16 < 0) return AQUAKV_ERR_INVALID_ARG;
   if (batch == 0 || (ctx_len == 0 && n16 == 0)) return AQUAKV_OK;
   const int d = c->p.d_kv;
+  if (rope != nullptr) {
+    if (rope->table == nullptr || rope->n_pos <= 0 || rope->pos0 < 0) return AQUAKV_ERR_INVALID_ARG;
+    if (n16 > 0 && rope->pos16 == nullptr) return AQUAKV_ERR_INVALID_ARG;
+    if (!aligned16(rope->table)) return AQUAKV_ERR_ALIGNMENT;
+    if (rope->pos0 + ctx_len > rope->n_pos) return AQUAKV_ERR_INVALID_ARG;
+  }
   if (n16 > 0) {
     int rc16;
     if ((rc16 = check_rows(K16, ld16, d, true))) return rc16;
@@ -1814,7 +1872,8 @@ static int decode_attn_impl(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32
     if (!aligned16(q) || !aligned16(out)) return AQUAKV_ERR_ALIGNMENT;
     if (!(softmax_scale == softmax_scale)) return AQUAKV_ERR_INVALID_ARG;
     const AttnExtWs xw = attn_ext_ws(c, 0, batch, n16, n_q_heads, head_dim);
-    if (workspace == nullptr || workspace_bytes < xw.total) return AQUAKV_ERR_WORKSPACE;
+    const RopeWs rw0 = rope_ws(c, xw.total, 0, batch, n16);
+    if (workspace == nullptr || workspace_bytes < (rope != nullptr ? rw0.total : xw.total)) return AQUAKV_ERR_WORKSPACE;
     if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
     cudaStream_t st0 = static_cast<cudaStream_t>(cuda_stream);
     uint8_t* wsb0 = ws_base(workspace);
@@ -1823,6 +1882,15 @@ static int decode_attn_impl(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32
     a.Kh = static_cast<const uint16_t*>(K16);
     a.Vh = static_cast<const uint16_t*>(V16);
     a.ld = ld16;
+    a.ld_v = ld16;
+    if (rope != nullptr) {
+      uint16_t* k16rot = reinterpret_cast<uint16_t*>(wsb0 + rw0.k16_off);
+      int rcr = launch_rope_rows(c, st0, *rope, a.Kh, ld16, k16rot, d, int64_t(batch) * n16, n_kv_heads, head_dim,
+                                 rope->pos16, n16, 0);
+      if (rcr) return rcr;
+      a.Kh = k16rot;
+      a.ld = d;
+    }
     a.tok_base = 0;
     a.blk_begin = 0;
     a.ctx = int(n16);
@@ -1869,9 +1937,14 @@ static int decode_attn_impl(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32
   if (Khat != nullptr && (Khat == Khat_prev || Khat == Vhat_prev || Vhat == Vhat_prev ||
                           Vhat == Khat_prev || Vhat == Khat))
     return AQUAKV_ERR_INVALID_ARG;
-  const AttnWs ws = attn_ws(c, batch, ctx_len, n_q_heads, head_dim, has_pred);
+  // with rotary keys the attention reads a rotated copy of the decoded rows: the two-kernel layout
+  const AttnWs ws = attn_ws(c, batch, ctx_len, n_q_heads, head_dim, has_pred && rope == nullptr);
   const AttnExtWs xw = attn_ext_ws(c, ws.total, batch, n16, n_q_heads, head_dim);
-  if (workspace == nullptr || workspace_bytes < (n16 > 0 ? xw.total : ws.total)) return AQUAKV_ERR_WORKSPACE;
+  const RopeWs rw = rope_ws(c, n16 > 0 ? xw.total : ws.total,
+                            rope != nullptr ? size_t(ws.chunk_blocks) * size_t(c->attn_block_tokens) : 0, batch, n16);
+  if (workspace == nullptr ||
+      workspace_bytes < (rope != nullptr ? rw.total : (n16 > 0 ? xw.total : ws.total)))
+    return AQUAKV_ERR_WORKSPACE;
   if (!aligned16(workspace)) return AQUAKV_ERR_ALIGNMENT;
   // partials of the uncompressed rows (attention sinks, recent-token buffer), merged by the combine kernel
   const float* extra_ml = nullptr;
@@ -1883,6 +1956,7 @@ static int decode_attn_impl(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32
     a.Kh = static_cast<const uint16_t*>(K16);
     a.Vh = static_cast<const uint16_t*>(V16);
     a.ld = ld16;
+    a.ld_v = ld16;
     a.tok_base = 0;
     a.blk_begin = 0;
     a.ctx = int(n16);
@@ -1893,6 +1967,14 @@ static int decode_attn_impl(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32
     a.scale_log2 = softmax_scale * 1.4426950408889634f;
     a.part_ml = reinterpret_cast<float*>(wsx + xw.ml_off);
     a.part_o = reinterpret_cast<float*>(wsx + xw.o_off);
+    if (rope != nullptr) {
+      uint16_t* k16rot = reinterpret_cast<uint16_t*>(wsx + rw.k16_off);
+      if ((rc = launch_rope_rows(c, static_cast<cudaStream_t>(cuda_stream), *rope, a.Kh, ld16, k16rot, d,
+                                 int64_t(batch) * n16, n_kv_heads, head_dim, rope->pos16, n16, 0)))
+        return rc;
+      a.Kh = k16rot;
+      a.ld = d;
+    }
     if ((rc = launch_attn_partial(c, static_cast<cudaStream_t>(cuda_stream), a, head_dim, batch * xw.splits))) return rc;
     extra_ml = a.part_ml;
     extra_o = a.part_o;
@@ -1972,6 +2054,15 @@ static int decode_attn_impl(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32
     a.Kh = kh;
     a.Vh = vh;
     a.ld = ldh;
+    a.ld_v = ldh;
+    if (rope != nullptr) {
+      // global row t0 + r is token (t0 + r) mod ctx_len of its sequence
+      uint16_t* krot = reinterpret_cast<uint16_t*>(wsb + rw.krot_off);
+      if ((rc = launch_rope_rows(c, st, *rope, kh, ldh, krot, d, rows, n_kv_heads, head_dim, nullptr, ctx_len, t0)))
+        return rc;
+      a.Kh = krot;
+      a.ld = d;
+    }
     a.tok_base = t0;
     a.blk_begin = gb0;
     a.ctx = int(ctx_len);
@@ -2009,7 +2100,7 @@ int aquakv_decode_attn(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_
                        int64_t ld_hat, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   return decode_attn_impl(c, batch, ctx_len, n_q_heads, n_kv_heads, head_dim, softmax_scale, q, Kcodes, Kscales, Vcodes,
                           Vscales, Khat_prev, Vhat_prev, ld_prev, Wk, Wv, bk, bv, out, lse, Khat, Vhat, ld_hat, nullptr,
-                          nullptr, 0, 0, workspace, workspace_bytes, cuda_stream);
+                          nullptr, 0, 0, nullptr, workspace, workspace_bytes, cuda_stream);
 }
 
 size_t aquakv_decode_attn_buffered_workspace_bytes(const aquakv_ctx* c, int32_t batch, int64_t ctx_len,
@@ -2030,7 +2121,59 @@ int aquakv_decode_attn_buffered(aquakv_ctx* c, int32_t batch, int64_t ctx_len, i
                                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
   return decode_attn_impl(c, batch, ctx_len, n_q_heads, n_kv_heads, head_dim, softmax_scale, q, Kcodes, Kscales, Vcodes,
                           Vscales, Khat_prev, Vhat_prev, ld_prev, Wk, Wv, bk, bv, out, lse, Khat, Vhat, ld_hat, K16, V16,
-                          n_uncompressed, ld16, workspace, workspace_bytes, cuda_stream);
+                          n_uncompressed, ld16, nullptr, workspace, workspace_bytes, cuda_stream);
+}
+
+int aquakv_rope_table(aquakv_ctx* c, int32_t head_dim, double theta_base, int64_t n_positions, float* table,
+                      void* cuda_stream) {
+  if (c == nullptr || table == nullptr || n_positions < 0) return AQUAKV_ERR_INVALID_ARG;
+  if (head_dim != 64 && head_dim != 128) return AQUAKV_ERR_UNSUPPORTED;
+  if (!(theta_base > 1.0) || !std::isfinite(theta_base)) return AQUAKV_ERR_INVALID_ARG;
+  if (!aligned16(table)) return AQUAKV_ERR_ALIGNMENT;
+  if (n_positions == 0) return AQUAKV_OK;
+  if (n_positions > (int64_t(1) << 31)) return AQUAKV_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int half = head_dim / 2;
+  int64_t blocks = (n_positions * half + 255) / 256;
+  const int64_t cap = int64_t(c->sm_count) * 16;
+  if (blocks > cap) blocks = cap;
+  ProfScope prof(c, st, AQUAKV_KERNEL_ATTN);
+  rope_table_kernel<<<int(blocks), 256, 0, st>>>(reinterpret_cast<float2*>(table), n_positions, half, theta_base);
+  ++c->launches;
+  return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
+}
+
+size_t aquakv_decode_attn_rope_workspace_bytes(const aquakv_ctx* c, int32_t batch, int64_t ctx_len,
+                                               int64_t n_uncompressed, int32_t n_q_heads, int32_t head_dim) {
+  if (c == nullptr || batch <= 0 || ctx_len < 0 || n_uncompressed < 0 || n_q_heads <= 0 || head_dim <= 0) return 0;
+  if (uniform_backbone(c)) return 0;
+  size_t base = 0, chunk_rows = 0;
+  if (ctx_len > 0) {
+    const AttnWs ws = attn_ws(c, batch, ctx_len, n_q_heads, head_dim, false);
+    base = ws.total;
+    chunk_rows = size_t(ws.chunk_blocks) * size_t(c->attn_block_tokens);
+  }
+  if (n_uncompressed > 0 || ctx_len == 0) base = attn_ext_ws(c, base, batch, n_uncompressed, n_q_heads, head_dim).total;
+  return rope_ws(c, base, chunk_rows, batch, n_uncompressed).total;
+}
+
+int aquakv_decode_attn_rope(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_heads,
+                            int32_t n_kv_heads, int32_t head_dim, float softmax_scale, const void* q,
+                            const uint8_t* Kcodes, const uint16_t* Kscales, const uint8_t* Vcodes,
+                            const uint16_t* Vscales, const void* Khat_prev, const void* Vhat_prev,
+                            int64_t ld_prev, const void* Wk, const void* Wv, const float* bk,
+                            const float* bv, const void* K16, const void* V16, int64_t n_uncompressed,
+                            int64_t ld16, const float* rope_table, int64_t rope_positions, int64_t pos0,
+                            const int32_t* pos16, void* out, float* lse, void* Khat, void* Vhat, int64_t ld_hat,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  RopeSpec rope;
+  rope.table = rope_table;
+  rope.n_pos = rope_positions;
+  rope.pos0 = pos0;
+  rope.pos16 = pos16;
+  return decode_attn_impl(c, batch, ctx_len, n_q_heads, n_kv_heads, head_dim, softmax_scale, q, Kcodes, Kscales, Vcodes,
+                          Vscales, Khat_prev, Vhat_prev, ld_prev, Wk, Wv, bk, bv, out, lse, Khat, Vhat, ld_hat, K16, V16,
+                          n_uncompressed, ld16, &rope, workspace, workspace_bytes, cuda_stream);
 }
 
 }  // extern "C"

@@ -16,8 +16,9 @@ constexpr float kNegBig = -1.0e30f;
 struct AttnArgs {
   const uint16_t* q;      // [batch][n_q_heads][HD]
   const uint16_t* Kh;     // decoded keys, row r = global token (tok_base + r)   [*, ld]
-  const uint16_t* Vh;
+  const uint16_t* Vh;     // decoded values                                      [*, ld_v]
   long long ld;
+  long long ld_v;
   long long tok_base;
   long long blk_begin;    // first global block (sequence * n_splits + split) of this launch
   int ctx;                // tokens per sequence
@@ -132,7 +133,7 @@ __global__ void __launch_bounds__(kAttnMmaThreads, 2) attn_partial_kernel(const 
 #pragma unroll
       for (int r = 0; r < 4; ++r) {
         const int tok = tb + 16 * ks + (r >> 1) * 8 + 2 * j + (r & 1);
-        const uint16_t* vp = vbase + (row0 + (tok < t_end ? tok : t_begin)) * a.ld + g * 8;
+        const uint16_t* vp = vbase + (row0 + (tok < t_end ? tok : t_begin)) * a.ld_v + g * 8;
 #pragma unroll
         for (int h = 0; h < NVH; ++h) vq[ks][r][h] = __ldcs(reinterpret_cast<const uint4*>(vp + h * 64));
       }

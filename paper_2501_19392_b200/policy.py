@@ -8,7 +8,10 @@ Host policy only: bookkeeping of which rows are where.  Compression is chain.enc
 flushed chunk (all layers, the chunk's own reconstructions feeding the next layer), row movement is
 aquakv_gather_rows, attention is aquakv_decode_attn_buffered.  Sequences of a batch advance in lockstep
 (the same number of tokens each); every sequence has its own cache arrays and is served by its own
-calls.  Position encoding is not applied here (keys are cached as given, as in aquakv_decode_attn).
+calls.  Keys are cached as given; with a rotary table (`attend(..., rope_table=...)`, Section 3.3
+"Positional embeddings": keys are compressed before RoPE) they are taken as pre-RoPE keys of tokens 0, 1, ...
+and rotated by their positions when attended to (aquakv_decode_attn_rope): sinks at 0 .. n_sink-1, compressed
+token t at n_sink + t, the recent rows after them.
 """
 from __future__ import annotations
 
@@ -112,11 +115,19 @@ class BufferedKVCache:
     def n_uncompressed(self) -> int:
         return self.n_sinks_held + self.fill
 
-    def attend(self, q: List[torch.Tensor], n_kv_heads: int, softmax_scale: float) -> List[torch.Tensor]:
+    def attend(self, q: List[torch.Tensor], n_kv_heads: int, softmax_scale: float,
+               rope_table: Optional[torch.Tensor] = None) -> List[torch.Tensor]:
         """Algorithm 4 lines 4-9 for every layer: q[l] [batch, n_q_heads, head_dim] -> outputs of the same shape.
-        The decoded compressed rows of layer l feed layer l + 1's predictors and are dropped afterwards."""
+        The decoded compressed rows of layer l feed layer l + 1's predictors and are dropped afterwards.
+        rope_table (Codec.rope_table): the cached keys are pre-RoPE and are rotated by their positions; q[l] must
+        be rotated by the caller."""
         out = [torch.empty_like(x) for x in q]
         n16 = self.n_uncompressed
+        pos16 = None
+        if rope_table is not None and n16:
+            first_recent = self.n_sinks_held + self.ctx
+            pos16 = torch.cat([torch.arange(self.n_sinks_held, dtype=torch.int32, device=self.dev),
+                               torch.arange(first_recent, first_recent + self.fill, dtype=torch.int32, device=self.dev)])
         if self.ctx > 0 and (self._dec is None or self._dec.K[0].shape[0] < self.ctx):
             self._dec = chain.PingPong(self.codec, self.max_ctx, self.dev)
         for b in range(self.B):
@@ -126,12 +137,15 @@ class BufferedKVCache:
                 has = l > 0 and self.ctx > 0
                 kh = self._dec.K[cur][:self.ctx] if self.ctx > 0 else None
                 vh = self._dec.V[cur][:self.ctx] if self.ctx > 0 else None
-                cdc.decode_attn_buffered(
-                    q[l][b:b + 1], self.Kcodes[l][b, :self.ctx], self.Kscales[l][b, :self.ctx],
-                    self.Vcodes[l][b, :self.ctx], self.Vscales[l][b, :self.ctx], self.ctx, n_kv_heads, softmax_scale,
-                    self.K16[l][b:b + 1, :n16] if n16 else None, self.V16[l][b:b + 1, :n16] if n16 else None,
-                    self._dec.K[prv][:self.ctx] if has else None, self._dec.V[prv][:self.ctx] if has else None,
-                    self.ad.Wk[l] if has else None, self.ad.Wv[l] if has else None,
-                    self.ad.bk[l] if has else None, self.ad.bv[l] if has else None,
-                    out=out[l][b:b + 1], Khat=kh, Vhat=vh)
+                cache = (q[l][b:b + 1], self.Kcodes[l][b, :self.ctx], self.Kscales[l][b, :self.ctx],
+                         self.Vcodes[l][b, :self.ctx], self.Vscales[l][b, :self.ctx], self.ctx, n_kv_heads, softmax_scale)
+                rows16 = (self.K16[l][b:b + 1, :n16] if n16 else None, self.V16[l][b:b + 1, :n16] if n16 else None)
+                pred = (self._dec.K[prv][:self.ctx] if has else None, self._dec.V[prv][:self.ctx] if has else None,
+                        self.ad.Wk[l] if has else None, self.ad.Wv[l] if has else None,
+                        self.ad.bk[l] if has else None, self.ad.bv[l] if has else None)
+                if rope_table is None:
+                    cdc.decode_attn_buffered(*cache, *rows16, *pred, out=out[l][b:b + 1], Khat=kh, Vhat=vh)
+                else:
+                    cdc.decode_attn_rope(*cache, rope_table, self.n_sinks_held, *rows16, pos16, *pred,
+                                         out=out[l][b:b + 1], Khat=kh, Vhat=vh)
         return out

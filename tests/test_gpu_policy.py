@@ -132,3 +132,29 @@ def test_policy_keeps_sinks_and_recent_tokens_and_compresses_the_rest():
             rows_k = np.concatenate([gpu_bits(Kh), gpu_bits(cache.K16[l][b, :n16])], axis=0)
             rows_v = np.concatenate([gpu_bits(Vh), gpu_bits(cache.V16[l][b, :n16])], axis=0)
             attn_check(outs[l][b:b + 1], q[l][b:b + 1], rows_k, rows_v, shape, scale)
+    # the same with the cached keys taken as pre-RoPE keys of tokens 0 .. total-1 (Section 3.3): sinks at
+    # 0 .. 3, compressed tokens at 4 .. 131, recent rows at 132 ..
+    from oracle import rope as orope
+    base = 500000.0
+    table = codec.rope_table(shape.head_dim, base, total, DEV)
+    outs_r = cache.attend(q, shape.n_kv_heads, scale, rope_table=table)
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0 and codec0.poll_status() == 0
+    positions = np.concatenate([4 + np.arange(128), np.arange(4), np.arange(132, total)])
+    for b in range(B):
+        Kh = Vh = None
+        for l in range(L):
+            cdc = codec0 if l == 0 else codec
+            args = (cache.Kcodes[l][b, :128], cache.Kscales[l][b, :128], cache.Vcodes[l][b, :128], cache.Vscales[l][b, :128])
+            Kh, Vh = cdc.decode(*args, Kh, Vh, ad.Wk[l] if l else None, ad.Wv[l] if l else None)
+            n16 = cache.n_uncompressed
+            rows_k = np.concatenate([gpu_bits(Kh), gpu_bits(cache.K16[l][b, :n16])], axis=0)
+            rows_v = np.concatenate([gpu_bits(Vh), gpu_bits(cache.V16[l][b, :n16])], axis=0)
+            ref, _ = orope.attention_rope(dt, 1, rows_k.shape[0], shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
+                                          scale, synth.to_bits(q[l][b:b + 1].cpu()), rows_k, rows_v, positions, base)
+            o = outs_r[l][b:b + 1]
+            ref_bits = synth.to_bits(torch.from_numpy(ref).to(o.dtype)).astype(np.int64)
+            adjacent = np.abs(gpu_bits(o).astype(np.int64) - ref_bits) <= 1
+            assert np.all((np.abs(o.to(torch.float64).cpu().numpy() - ref) <= 2e-3 * np.abs(ref).max(axis=-1, keepdims=True))
+                          | adjacent)
+            assert not torch.equal(o, outs[l][b:b + 1])
