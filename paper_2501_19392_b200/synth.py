@@ -107,25 +107,29 @@ def _randn(shape, g: torch.Generator, device) -> torch.Tensor:
 # Grid and signs
 # --------------------------------------------------------------------------------------------
 
-def lloyd_grid(n: int, seed: int = 7, n_samples: int = 1 << 18, iters: int = 60) -> np.ndarray:
-    """A 2-D, n-point codebook fitted to N(0, I_2) samples by Lloyd's algorithm.
+def lloyd_grid(n: int, seed: int = 7, n_samples: int = 1 << 18, iters: int = 60, dim: int = 2) -> np.ndarray:
+    """A dim-dimensional, n-point codebook fitted to N(0, I) samples by Lloyd's algorithm.
 
     Stands in for the fixed Gaussian-optimal grid of the paper's backbone quantizer (Section 4.1
-    "Alternative quantizers": p = 2, n in {16, 64, 256}).  Deterministic for a given seed; rows
-    are sorted lexicographically so that code indices are canonical.  Returned as float32 [n, 2]
-    (the storage type of the library's grid argument).
+    "Alternative quantizers": p = 2, n in {16, 64, 256}, and the slower p = 4, n = 256 grid).
+    Deterministic for a given seed; rows are sorted lexicographically so that code indices are
+    canonical.  Returned as float32 [n, dim] (the storage type of the library's grid argument).
     """
     rng = np.random.default_rng(seed)
-    x = rng.standard_normal((n_samples, 2))
+    x = rng.standard_normal((n_samples, dim))
     c = x[rng.choice(n_samples, size=n, replace=False)].copy()
     for _ in range(iters):
-        d2 = ((x[:, None, :] - c[None, :, :]) ** 2).sum(-1)
-        a = d2.argmin(1)
+        # squared distances up to the sample's own norm, by blocks of samples (memory)
+        a = np.empty(n_samples, dtype=np.int64)
+        for lo in range(0, n_samples, 1 << 16):
+            blk = x[lo:lo + (1 << 16)]
+            a[lo:lo + (1 << 16)] = ((c * c).sum(1)[None, :] - 2.0 * blk @ c.T).argmin(1) if dim > 2 else \
+                ((blk[:, None, :] - c[None, :, :]) ** 2).sum(-1).argmin(1)
         for i in range(n):
             m = a == i
             if m.any():
                 c[i] = x[m].mean(0)
-    order = np.lexsort((c[:, 1], c[:, 0]))
+    order = np.lexsort(tuple(c[:, k] for k in range(dim - 1, -1, -1)))
     return np.ascontiguousarray(c[order], dtype=np.float32)
 
 
