@@ -469,9 +469,10 @@ def calibration_entry(api, peaks, dev, reps=3):
 
 
 def uniform_backbone_entries(api, chain, peaks, dev, reps=5):
-    """The alternative backbones built on uniform round-to-nearest levels with absmax normalisation, 2 bits
-    per value, on the prefill-shaped workload: the plain one with groups of 64 (2.25 bits with the scales)
-    and the rotated one with one group per row (random signs + Hadamard rotation first; 2.02 bits).  Time of
+    """The alternative backbones, 2 bits per value, on the prefill-shaped workload: uniform round-to-nearest
+    levels with absmax normalisation, plain with groups of 64 (2.25 bits with the scales) and rotated with one
+    group per row (random signs + Hadamard rotation first; 2.02 bits), and the vector quantizer with the
+    256-point grid in four dimensions (2.02 bits; the paper's grid "without fast GPU support").  Time of
     one predicted layer through the per-layer entry points (two launches per phase: predictor GEMM, row
     kernel), and what fitted predictors buy each backbone (Section 4.1 evaluates each backbone with and
     without them)."""
@@ -482,11 +483,17 @@ def uniform_backbone_entries(api, chain, peaks, dev, reps=5):
         return float(((X - Xh) ** 2).sum() / ((X - X.mean(dim=0)) ** 2).sum())
 
     out = []
-    for tag, h, g in (("uniform-backbone", 1, 64), ("rotated-uniform-backbone", 1024, 1024)):
+    for tag, h, g in (("uniform-backbone", 1, 64), ("rotated-uniform-backbone", 1024, 1024),
+                      ("four-dimensional-grid-backbone", 1024, 1024)):
         shape = dataclasses.replace(synth.CONFIGS[2], n_layers=3, had_block=h, scale_group=g, grid_size=4)
         T, d, L = shape.n_tokens, shape.d_kv, shape.n_layers
         signs = (synth.hadamard_signs(d, 1), synth.hadamard_signs(d, 2)) if h > 1 else (None, None)
-        codec = api.Codec(d, h, g, None, shape.dtype, levels=4, signs_k=signs[0], signs_v=signs[1])
+        grid4 = tag.startswith("four")     # the 256-point grid in four dimensions (2 bits per value, exhaustive search)
+        if grid4:
+            codec = api.Codec(d, h, g, synth.lloyd_grid(256, seed=9, n_samples=1 << 16, iters=20, dim=4), shape.dtype,
+                              signs[0], signs[1])
+        else:
+            codec = api.Codec(d, h, g, None, shape.dtype, levels=4, signs_k=signs[0], signs_v=signs[1])
         kv = synth.kv_chain(shape, seed=7001, device=dev)
         preds, recs = gcal.calibrate(codec, kv.K, kv.V, rate=1e-3, keep_reconstructions=True)
         l = L - 1
@@ -505,7 +512,7 @@ def uniform_backbone_entries(api, chain, peaks, dev, reps=5):
         _, _, Vd = codec.encode_phase(api.ROLE_VALUE, kv.V[l])
         quality = {"fitted_predictors": {"K": rel_err(kv.K[l], recs[l][0]), "V": rel_err(kv.V[l], recs[l][1])},
                    "no_predictor": {"K": rel_err(kv.K[l], Kd), "V": rel_err(kv.V[l], Vd)}}
-        if h > 1:      # the same group size without the rotation (the appendix' "larger group size" row)
+        if h > 1 and not grid4:      # the same group size without the rotation (the appendix' "larger group size" row)
             plain = api.Codec(d, 1, g, None, shape.dtype, levels=4)
             _, _, Kp = plain.encode_phase(api.ROLE_KEY, kv.K[l])
             _, _, Vp = plain.encode_phase(api.ROLE_VALUE, kv.V[l])

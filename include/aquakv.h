@@ -78,7 +78,7 @@ typedef struct aquakv_params {
   int32_t d_kv;        /* values per token row; supported: 256, 512, 1024                       */
   int32_t had_block;   /* h: Hadamard block, power of two, 64 <= h <= d_kv, divides d_kv        */
   int32_t scale_group; /* g: values per fp16 scale; multiple of h that divides d_kv             */
-  int32_t grid_dim;    /* p: values per code; 2 (1: the uniform backbone, see aquakv_create)    */
+  int32_t grid_dim;    /* p: values per code; 2 (1: uniform backbone, 4: see aquakv_create)     */
   int32_t grid_size;   /* n: 16, 64 or 256 grid points (2, 3, 4 bits per value)                 */
   int32_t dtype;       /* AQUAKV_F16 or AQUAKV_BF16                                             */
 } aquakv_params;
@@ -109,7 +109,16 @@ int aquakv_code_bytes(const aquakv_params* params);
  * non-vector quantization"): the residual times the role's signs is rotated by the orthonormal Hadamard
  * matrix in blocks of h values, the ROTATED values are quantized as above (absmax after the rotation;
  * scale_group is independent of h), and the inverse rotates level * scale back and applies the signs again;
- * the sign arrays are then required.  Such a ctx serves aquakv_encode / aquakv_decode (with predictors: two launches per phase, and
+ * the sign arrays are then required.
+ *
+ * Four-dimensional grid (Section 4.1: "one grid without fast GPU support (2-bit precision, d = 4, n = 256)",
+ * the paper's d being the grid dimension): grid_dim = 4 with grid_size = 256.  grid_host is then 256 x 4
+ * floats; every consecutive 4-tuple of rotated normalised values goes to the nearest of the 256 points
+ * (exhaustive search, lowest index on a tie) and takes one byte (d_kv / 4 bytes per token); scale,
+ * signs, rotation and reconstruction are those of the planar grids, with the same rules for had_block and
+ * scale_group.  It is served like the uniform backbone.
+ *
+ * A ctx with grid_dim 1 or 4 serves aquakv_encode / aquakv_decode (with predictors: two launches per phase, and
  * Khat is required because the value phase reads it), the *_phase entry points, aquakv_predict,
  * aquakv_fit_predictor and aquakv_gather_rows; the chain, no-allocation and attention entry points return
  * AQUAKV_ERR_UNSUPPORTED.

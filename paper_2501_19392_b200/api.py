@@ -191,7 +191,7 @@ class Codec:
 
     def __init__(self, d_kv: int, had_block: int, scale_group: int, grid: Optional[np.ndarray], dtype: int,
                  signs_k: Optional[np.ndarray] = None, signs_v: Optional[np.ndarray] = None, levels: int = 0):
-        """grid [n, 2] with sign vectors: the rotated 2-D vector quantizer.  grid None with `levels` = 2^b: the
+        """grid [n, 2] (or [256, 4]) with sign vectors: the rotated vector quantizer.  grid None with `levels` = 2^b: the
         uniform round-to-nearest backbone with absmax normalisation; had_block 1 leaves the residual as it is,
         had_block >= 64 (with sign vectors) rotates it first."""
         h = ctypes.c_void_p()
@@ -202,7 +202,9 @@ class Codec:
             rc = lib.aquakv_create(ctypes.byref(self.params), None, None if sk is None else sk.ctypes.data,
                                    None if sv is None else sv.ctypes.data, ctypes.byref(h))
         else:
-            self.params = Params(d_kv, had_block, scale_group, 2, int(np.asarray(grid).shape[0]), dtype)
+            # grid [n, 2], or [256, 4]: the four-dimensional grid (per-layer entry points only)
+            self.params = Params(d_kv, had_block, scale_group, int(np.asarray(grid).shape[1]),
+                                 int(np.asarray(grid).shape[0]), dtype)
             g = np.ascontiguousarray(grid, dtype=np.float32)
             sk = np.ascontiguousarray(signs_k, dtype=np.int8)
             sv = np.ascontiguousarray(signs_v, dtype=np.int8)

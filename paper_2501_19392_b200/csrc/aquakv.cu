@@ -26,6 +26,7 @@
 #include "chain_kernel.cuh"
 #include "codec.cuh"
 #include "gemm_pred.cuh"
+#include "grid4.cuh"
 #include "layer_kernel.cuh"
 #include "rope.cuh"
 #include "search_table.h"
@@ -113,9 +114,14 @@ int check_params(const aquakv_params* p) {
     if (!is_pow2(p->scale_group) || p->scale_group < 32 || p->scale_group > p->d_kv) return AQUAKV_ERR_UNSUPPORTED;
     return AQUAKV_OK;
   }
-  if (p->grid_dim != 2) return AQUAKV_ERR_UNSUPPORTED;
+  if (p->grid_dim != 2 && p->grid_dim != 4) return AQUAKV_ERR_UNSUPPORTED;
   if (p->d_kv != 256 && p->d_kv != 512 && p->d_kv != 1024) return AQUAKV_ERR_UNSUPPORTED;
-  if (p->grid_size != 16 && p->grid_size != 64 && p->grid_size != 256) return AQUAKV_ERR_UNSUPPORTED;
+  if (p->grid_dim == 4) {
+    // the four-dimensional grid: 256 points, one byte per four values
+    if (p->grid_size != 256) return AQUAKV_ERR_UNSUPPORTED;
+  } else if (p->grid_size != 16 && p->grid_size != 64 && p->grid_size != 256) {
+    return AQUAKV_ERR_UNSUPPORTED;
+  }
   if (!is_pow2(p->had_block) || p->had_block < 64 || p->had_block > p->d_kv)
     return AQUAKV_ERR_UNSUPPORTED;
   if (!is_pow2(p->scale_group) || p->scale_group < p->had_block || p->scale_group > p->d_kv)
@@ -249,11 +255,57 @@ CodecArgs codec_args(const aquakv_ctx* c, int role, int rows) {
 }
 
 // One phase of Algorithm 2 on `rows` rows: codes/scales = Q(X - P), hat = round16(P + Q^-1(..)).
-inline bool uniform_backbone(const aquakv_ctx* c) { return c->p.grid_dim == 1; }
+// Backbones without a fused layer kernel (the uniform levels, grid_dim 1, and the four-dimensional grid,
+// grid_dim 4): predictor GEMM and a stand-alone row kernel per phase, per-layer entry points only.
+inline bool uniform_backbone(const aquakv_ctx* c) { return c->p.grid_dim != 2; }
+
+// Row kernels of the four-dimensional grid (grid4.cuh): X == nullptr decodes.
+int launch_grid4_rows(aquakv_ctx* c, cudaStream_t st, int role, int rows, const void* X, int64_t ldX, const float* P,
+                      int64_t ldP, uint8_t* codes, uint16_t* scales, void* hat, int64_t ldHat) {
+  Grid4Args ga;
+  UniformArgs& a = ga.u;
+  ga.grid = c->d_grid4;
+  ga.signmask = c->d_signmask[role];
+  ga.log_h = c->log_h;
+  a.X = static_cast<const uint16_t*>(X);
+  a.ldX = ldX;
+  a.P = P;
+  a.ldP = ldP;
+  a.codes = codes;
+  a.scales = scales;
+  a.hat = static_cast<uint16_t*>(hat);
+  a.ldHat = ldHat;
+  a.T = rows;
+  a.d = c->p.d_kv;
+  a.log_g = c->log_g;
+  int64_t blocks = (int64_t(rows) + kUniformWarps - 1) / kUniformWarps;
+  const int64_t cap = int64_t(c->sm_count) * 8;
+  if (blocks > cap) blocks = cap;
+  const int grid = int(blocks), threads = kUniformWarps * 32;
+  const bool enc = X != nullptr;
+  ProfScope prof(c, st, enc ? AQUAKV_KERNEL_ENCODE_ROWS : AQUAKV_KERNEL_DECODE_ROWS);
+#define AQ_GRID4(NCH)                                                                                 \
+  do {                                                                                                \
+    if (enc) {                                                                                        \
+      if (c->bf16) grid4_encode_rows_kernel<true, NCH><<<grid, threads, 0, st>>>(ga);                 \
+      else grid4_encode_rows_kernel<false, NCH><<<grid, threads, 0, st>>>(ga);                        \
+    } else {                                                                                          \
+      if (c->bf16) grid4_decode_rows_kernel<true, NCH><<<grid, threads, 0, st>>>(ga);                 \
+      else grid4_decode_rows_kernel<false, NCH><<<grid, threads, 0, st>>>(ga);                        \
+    }                                                                                                 \
+  } while (0)
+  if (a.d == 256) AQ_GRID4(1);
+  else if (a.d == 512) AQ_GRID4(2);
+  else AQ_GRID4(4);
+#undef AQ_GRID4
+  ++c->launches;
+  return cudaGetLastError() == cudaSuccess ? AQUAKV_OK : AQUAKV_ERR_CUDA;
+}
 
 // Row kernels of the uniform backbone (uniform.cuh): X == nullptr decodes.
 int launch_uniform_rows(aquakv_ctx* c, cudaStream_t st, int role, int rows, const void* X, int64_t ldX, const float* P,
                         int64_t ldP, uint8_t* codes, uint16_t* scales, void* hat, int64_t ldHat) {
+  if (c->p.grid_dim == 4) return launch_grid4_rows(c, st, role, rows, X, ldX, P, ldP, codes, scales, hat, ldHat);
   UniformRotArgs ra;
   UniformArgs& a = ra.u;
   ra.signmask = c->d_signmask[role];
@@ -1100,8 +1152,7 @@ extern "C" {
 int aquakv_code_bytes(const aquakv_params* params) {
   const int rc = check_params(params);
   if (rc) return rc;
-  if (params->grid_dim == 1) return params->d_kv * ilog2(params->grid_size) / 8;
-  return params->d_kv / 2 * ilog2(params->grid_size) / 8;
+  return params->d_kv / params->grid_dim * ilog2(params->grid_size) / 8;
 }
 
 const char* aquakv_status_string(int status) {
@@ -1147,9 +1198,9 @@ int aquakv_create(const aquakv_params* params, const float* grid_host, const int
   const bool rotated = !uniform || params->had_block > 1;   // the signs are read
   if (!uniform && grid_host == nullptr) return AQUAKV_ERR_INVALID_ARG;
   if (rotated && (signs_k_host == nullptr || signs_v_host == nullptr)) return AQUAKV_ERR_INVALID_ARG;
-  const int d = params->d_kv, n = params->grid_size;
+  const int d = params->d_kv, n = params->grid_size, gdim = params->grid_dim;
   if (!uniform)
-    for (int i = 0; i < 2 * n; ++i)
+    for (int i = 0; i < gdim * n; ++i)
       if (!std::isfinite(grid_host[i])) return AQUAKV_ERR_INVALID_ARG;
   if (rotated) {
     for (int i = 0; i < d; ++i) {
@@ -1164,7 +1215,7 @@ int aquakv_create(const aquakv_params* params, const float* grid_host, const int
   c->log_h = ilog2(params->had_block);
   c->log_g = ilog2(params->scale_group);
   c->bits = ilog2(n);
-  c->code_bytes = uniform ? d * c->bits / 8 : d / 2 * c->bits / 8;
+  c->code_bytes = d / gdim * c->bits / 8;
   c->n_groups = d / params->scale_group;
   c->bf16 = params->dtype == AQUAKV_BF16;
   c->attn_block_tokens = 1024;
@@ -1172,7 +1223,10 @@ int aquakv_create(const aquakv_params* params, const float* grid_host, const int
   float4 g4[256];
   std::memset(g4, 0, sizeof(g4));
   std::vector<uint32_t> table(4, 0u);
-  if (!uniform) {
+  if (gdim == 4) {
+    for (int i = 0; i < n; ++i)
+      g4[i] = make_float4(grid_host[4 * i], grid_host[4 * i + 1], grid_host[4 * i + 2], grid_host[4 * i + 3]);
+  } else if (!uniform) {
     for (int i = 0; i < n; ++i) {
       const float gx = grid_host[2 * i], gy = grid_host[2 * i + 1];
       g4[i] = make_float4(gx, gy, 0.0f, 0.0f);
