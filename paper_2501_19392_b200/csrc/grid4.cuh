@@ -10,7 +10,9 @@
 // writes their codes as one 16-bit store.  The search is exhaustive: a 256-point grid in four dimensions
 // has no cheap cell structure like the planar grids' table, and this grid is the paper's slow one.  The
 // points sit in shared memory with half their squared norm, so a candidate costs four FMAs and a
-// compare: argmin |y - g|^2 = argmin (|g|^2 / 2 - y . g).
+// compare: argmin |y - g|^2 = argmin (|g|^2 / 2 - y . g).  A lane's two tuples of a chunk go through the
+// packed two-lane fp32 FMA together (each lane rounds like the scalar instruction), which is why the
+// encoder's copy of the grid holds every coordinate twice.
 #pragma once
 
 #include "uniform.cuh"
@@ -26,16 +28,28 @@ struct Grid4Args {
 
 struct Grid4Smem {
   float4 g[256];
-  float half_norm[256];
+};
+
+// The encoder's search copy: (x, x, y, y), (z, z, w, w) and (|g|^2 / 2, |g|^2 / 2) per point.
+struct Grid4SearchSmem {
+  float4 xy[256];
+  float4 zw[256];
+  float2 half_norm[256];
 };
 
 __device__ __forceinline__ void grid4_load(Grid4Smem& sm, const float4* grid) {
+  for (int k = threadIdx.x; k < 256; k += blockDim.x) sm.g[k] = grid[k];
+  __syncthreads();
+}
+
+__device__ __forceinline__ void grid4_load_search(Grid4SearchSmem& ss, const float4* grid) {
   for (int k = threadIdx.x; k < 256; k += blockDim.x) {
     const float4 p = grid[k];
-    sm.g[k] = p;
-    sm.half_norm[k] = 0.5f * (p.x * p.x + p.y * p.y + p.z * p.z + p.w * p.w);
+    ss.xy[k] = make_float4(p.x, p.x, p.y, p.y);
+    ss.zw[k] = make_float4(p.z, p.z, p.w, p.w);
+    const float hn = 0.5f * (p.x * p.x + p.y * p.y + p.z * p.z + p.w * p.w);
+    ss.half_norm[k] = make_float2(hn, hn);
   }
-  __syncthreads();
 }
 
 // hat = round16(pred + s16 * signs . H(y) / sqrt(h)) for the row's grid points y; sf[c] is the scale of chunk c's group.
@@ -58,6 +72,8 @@ template <bool kBf16, int NCH>
 __global__ void __launch_bounds__(kUniformWarps * 32)
 grid4_encode_rows_kernel(const Grid4Args ga) {
   __shared__ Grid4Smem sm;
+  __shared__ Grid4SearchSmem ss_grid;
+  grid4_load_search(ss_grid, ga.grid);
   grid4_load(sm, ga.grid);
   const UniformArgs& a = ga.u;
   const int lane = threadIdx.x & 31;
@@ -70,16 +86,20 @@ grid4_encode_rows_kernel(const Grid4Args ga) {
   const float rs = rsqrtf(float(1 << ga.log_h));
   const float inv_g = 1.0f / float(1 << a.log_g);
   for (long long t = warp; t < a.T; t += n_warps) {
-    float v[NCH][8], pred[NCH][8];
-    uniform_load_pred_row<NCH>(a, t, lane, pred);
+    float v[NCH][8];
+    {
+      // the prediction is read again for the reconstruction: holding it through the search would cost 32 registers
+      float pred[NCH][8];
+      uniform_load_pred_row<NCH, false>(a, t, lane, pred);
 #pragma unroll
-    for (int c = 0; c < NCH; ++c) {
-      const uint4 raw = __ldcs(reinterpret_cast<const uint4*>(a.X + t * a.ldX + 256 * c + 8 * lane));
-      float lo, hi;
-      unpack2(load16x2<kBf16>(raw.x), lo, hi); v[c][0] = lo - pred[c][0]; v[c][1] = hi - pred[c][1];
-      unpack2(load16x2<kBf16>(raw.y), lo, hi); v[c][2] = lo - pred[c][2]; v[c][3] = hi - pred[c][3];
-      unpack2(load16x2<kBf16>(raw.z), lo, hi); v[c][4] = lo - pred[c][4]; v[c][5] = hi - pred[c][5];
-      unpack2(load16x2<kBf16>(raw.w), lo, hi); v[c][6] = lo - pred[c][6]; v[c][7] = hi - pred[c][7];
+      for (int c = 0; c < NCH; ++c) {
+        const uint4 raw = __ldcs(reinterpret_cast<const uint4*>(a.X + t * a.ldX + 256 * c + 8 * lane));
+        float lo, hi;
+        unpack2(load16x2<kBf16>(raw.x), lo, hi); v[c][0] = lo - pred[c][0]; v[c][1] = hi - pred[c][1];
+        unpack2(load16x2<kBf16>(raw.y), lo, hi); v[c][2] = lo - pred[c][2]; v[c][3] = hi - pred[c][3];
+        unpack2(load16x2<kBf16>(raw.z), lo, hi); v[c][4] = lo - pred[c][4]; v[c][5] = hi - pred[c][5];
+        unpack2(load16x2<kBf16>(raw.w), lo, hi); v[c][6] = lo - pred[c][6]; v[c][7] = hi - pred[c][7];
+      }
     }
     // group scale: root mean square of the residual, rounded to fp16; the rounded value normalises
     float ss[NCH];
@@ -114,27 +134,35 @@ grid4_encode_rows_kernel(const Grid4Args ga) {
     // nearest grid point of every 4-tuple: exhaustive, candidates in ascending order, strict "<" keeps the lowest index
     float best[NCH][2];
     int arg[NCH][2];
+    f32x2_t ny[NCH][4];                  // (-y_j of the first tuple, -y_j of the second) for j = 0 .. 3
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
       best[c][0] = best[c][1] = 3.0e38f;
       arg[c][0] = arg[c][1] = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) ny[c][j] = pack2(-v[c][j], -v[c][4 + j]);
     }
 #pragma unroll 2
     for (int k = 0; k < 256; ++k) {
-      const float4 g = sm.g[k];
-      const float hn = sm.half_norm[k];
+      const float4 gxy = ss_grid.xy[k], gzw = ss_grid.zw[k];
+      const float2 hn = ss_grid.half_norm[k];
+      const f32x2_t gx = pack2(gxy.x, gxy.y), gy = pack2(gxy.z, gxy.w), gz = pack2(gzw.x, gzw.y), gw = pack2(gzw.z, gzw.w);
+      const f32x2_t h2 = pack2(hn.x, hn.y);
 #pragma unroll
       for (int c = 0; c < NCH; ++c) {
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          float s = fmaf(-v[c][4 * u], g.x, hn);
-          s = fmaf(-v[c][4 * u + 1], g.y, s);
-          s = fmaf(-v[c][4 * u + 2], g.z, s);
-          s = fmaf(-v[c][4 * u + 3], g.w, s);
-          if (s < best[c][u]) {
-            best[c][u] = s;
-            arg[c][u] = k;
-          }
+        f32x2_t s2 = fma2(ny[c][0], gx, h2);
+        s2 = fma2(ny[c][1], gy, s2);
+        s2 = fma2(ny[c][2], gz, s2);
+        s2 = fma2(ny[c][3], gw, s2);
+        float s0, s1;
+        unpack2(s2, s0, s1);
+        if (s0 < best[c][0]) {
+          best[c][0] = s0;
+          arg[c][0] = k;
+        }
+        if (s1 < best[c][1]) {
+          best[c][1] = s1;
+          arg[c][1] = k;
         }
       }
     }
@@ -151,7 +179,11 @@ grid4_encode_rows_kernel(const Grid4Args ga) {
         v[c][4 * u + 3] = g.w;
       }
     }
-    if (a.hat != nullptr) grid4_finish<kBf16, NCH>(ga, t, lane, sbits, v, sf, pred);
+    if (a.hat != nullptr) {
+      float pred[NCH][8];
+      uniform_load_pred_row<NCH>(a, t, lane, pred);
+      grid4_finish<kBf16, NCH>(ga, t, lane, sbits, v, sf, pred);
+    }
   }
 }
 

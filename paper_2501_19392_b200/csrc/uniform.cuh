@@ -267,12 +267,20 @@ __device__ __forceinline__ void uniform_scale_all(float (&v)[NCH][8], float f) {
     for (int i = 0; i < 8; ++i) v[c][i] *= f;
 }
 
-template <int NCH>
+// kStream: the last read of the prediction (evict-first); otherwise it stays cached for a second read.
+template <int NCH, bool kStream = true>
 __device__ __forceinline__ void uniform_load_pred_row(const UniformArgs& a, long long t, int lane, float (&pred)[NCH][8]) {
 #pragma unroll
   for (int c = 0; c < NCH; ++c) {
     if (a.P != nullptr) {
-      uniform_load_pred8(a.P + t * a.ldP + 256 * c + 8 * lane, pred[c]);
+      if constexpr (kStream) {
+        uniform_load_pred8(a.P + t * a.ldP + 256 * c + 8 * lane, pred[c]);
+      } else {
+        const float4* p = reinterpret_cast<const float4*>(a.P + t * a.ldP + 256 * c + 8 * lane);
+        const float4 lo = p[0], hi = p[1];
+        pred[c][0] = lo.x; pred[c][1] = lo.y; pred[c][2] = lo.z; pred[c][3] = lo.w;
+        pred[c][4] = hi.x; pred[c][5] = hi.y; pred[c][6] = hi.z; pred[c][7] = hi.w;
+      }
     } else {
 #pragma unroll
       for (int i = 0; i < 8; ++i) pred[c][i] = 0.0f;
