@@ -41,8 +41,8 @@ sys.path.insert(0, ROOT)
 from paper_2501_19392_b200 import synth  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per layer_kernel launch (32768 tokens, d_kv 1024, n 16):
-# mean of the encode (526 MB) and decode + attention (377 MB) launches of profiles/layer_kernel_3layer_32768tok.md
-LAYER_KERNEL_DRAM_BYTES_PER_LAUNCH = 451.5e6
+# mean of the encode (526 MB) and decode (258 MB) launches of profiles/layer_kernel_3layer_32768tok.md
+LAYER_KERNEL_DRAM_BYTES_PER_LAUNCH = 392.0e6
 
 METRIC = "KV tokens/s per layer (encode + decode-attention round trip) at 2 bits/value"
 UNIT = "token-layers/s"
@@ -351,6 +351,14 @@ def ops_by_config(api, chain, peaks, dev, reps=5):
     ms = _time_calls(one, max(2, reps // 2), warm=2)
     out.append(_shape_entry(peaks, shape, "decode_attn", T, ms, _shape_bytes(shape, T, False, write_hat=False),
                             config=5, batch=shape.batch, ctx=ctx_len, n_q_heads=shape.n_q_heads))
+    # the fused form: attention warps inside the decode kernel, decoded rows only in a ring in L2
+    codec.set_attn_mode(api.ATTN_FUSED)
+    ms_f = _time_calls(one, max(2, reps // 2), warm=2)
+    codec.set_attn_mode(api.ATTN_SPLIT)
+    out.append(_shape_entry(peaks, shape, "decode_attn_fused", T, ms_f, _shape_bytes(shape, T, False, write_hat=False),
+                            config=5, batch=shape.batch, ctx=ctx_len, n_q_heads=shape.n_q_heads,
+                            note="aquakv_set_attn_mode(AQUAKV_ATTN_FUSED): one launch of the layer kernel with attention "
+                                 "warps + the merge kernel; the default form is decode kernel, split-KV attention, merge"))
     # the same with the cache policy's uncompressed rows beside the compressed cache: 4 attention sinks and 128
     # recent tokens per sequence (Section 4.1), merged in the same combine kernel
     n16 = 132
@@ -690,7 +698,7 @@ def main():
                 "peak": peaks["tf_sustained"], "unit": "TFLOP/s", "frac": achieved / peaks["tf_sustained"],
                 "frac_burst": achieved / peaks["tf_burst"], "peak_burst": peaks["tf_burst"],
                 "traffic": LAYER_KERNEL_DRAM_BYTES_PER_LAUNCH if (T, d, shape.grid_size) == (32768, 1024, 16) else None,
-                "traffic_unit": "bytes per launch (ncu dram read+write, mean of the encode and decode + attention launches)",
+                "traffic_unit": "bytes per launch (ncu dram read+write, mean of the encode and decode launches)",
                 "algorithmic_bytes_per_launch": 0.5 * (enc_bytes + dec_bytes) * T,
                 "peak_source": peaks["source"] + " (sustained)", "dominant_by_time": dominant,
                 "launches": n_l, "avg_launch_ms": ms_l / max(1, n_l)}

@@ -73,6 +73,10 @@ extern "C" {
 #define AQUAKV_OP_DECODE 1
 #define AQUAKV_OP_DECODE_ATTN 2
 
+/* How aquakv_decode_attn and its variants run (aquakv_set_attn_mode). */
+#define AQUAKV_ATTN_SPLIT 0 /* decode kernel, then a split-KV attention kernel over the fresh rows (default) */
+#define AQUAKV_ATTN_FUSED 1 /* attention warps inside the decode kernel where the shape allows it          */
+
 /* Parameters of the quantizer Q (Section 4.1: group size, p, n) and of the tensors. */
 typedef struct aquakv_params {
   int32_t d_kv;        /* values per token row; supported: 256, 512, 1024                       */
@@ -161,12 +165,13 @@ size_t aquakv_workspace_bytes(const aquakv_ctx* ctx, int64_t n_tokens, int op);
 /*
  * Workspace of aquakv_decode_attn for this problem shape (its attention partials depend on the
  * batch and head counts, which aquakv_workspace_bytes does not see).  0 on invalid arguments.
- * With predictors at d_kv = 1024 (Hadamard block = scale group = d_kv) decode and attention run as
- * one kernel: the workspace holds that kernel's buffers (the prediction ring and, when Khat/Vhat
- * are not requested, rings of three waves of decoded keys and values: about 0.1 GB in all) and one
- * attention partial per 128-token block and query head (about 130 bytes per token at 32 query
- * heads).  In the other cases the cache is decoded in chunks of up to about 147 K tokens into the
- * workspace (4 * d_kv bytes per token of a chunk) and a second kernel attends over each chunk.
+ * The cache is decoded in chunks of up to about 147 K tokens into the workspace (4 * d_kv bytes per
+ * token of a chunk; nothing when Khat/Vhat are given) and a second kernel attends over each chunk.  In
+ * the fused mode (aquakv_set_attn_mode), with predictors at d_kv = 1024 (Hadamard block = scale group =
+ * d_kv), decode and attention run as one kernel: the workspace then holds that kernel's buffers (the
+ * prediction ring and, when Khat/Vhat are not requested, rings of three waves of decoded keys and
+ * values: about 0.1 GB in all) and one attention partial per 128-token block and query head (about 130
+ * bytes per token at 32 query heads).  The returned size covers either mode.
  */
 size_t aquakv_decode_attn_workspace_bytes(const aquakv_ctx* ctx, int32_t batch, int64_t ctx_len,
                                           int32_t n_q_heads, int32_t head_dim);
@@ -339,14 +344,22 @@ int aquakv_decode_noalloc(aquakv_ctx* ctx, int64_t n_tokens,
  * contiguous.  lse: optional fp32 [batch][n_q_heads] log-sum-exp of the scaled scores (NULL =
  * not written).  Khat, Vhat: optional outputs [n_tokens, ld_hat] for the next layer's decode.
  *
- * With predictors at d_kv = 1024 and Hadamard block = scale group = d_kv (the paper's setting) this
- * is ONE kernel: while the tensor cores form the predictions and the row warps reconstruct token
- * rows, attention warps of the same kernel take every 128-token block as soon as its keys and
- * values exist and reduce it to per-block softmax partials; a small second kernel merges the
- * partials of each sequence.  Without Khat/Vhat the decoded rows live only in a ring of three
- * waves of tokens in the workspace.  Without predictors (layer 0) and for the other shapes decode
- * and attention are separate kernels behind this entry point (see the workspace note above).
+ * Two ways to run it (aquakv_set_attn_mode; the results agree to the rounding of the fp32 partial sums):
+ *   AQUAKV_ATTN_SPLIT (default): the layer kernel decodes a chunk of tokens (predictions on the tensor
+ *     cores, row warps reconstruct the rows into Khat/Vhat or the workspace), a split-KV kernel attends
+ *     over the chunk's rows right behind it and a small third kernel merges the partials of each sequence.
+ *   AQUAKV_ATTN_FUSED: with predictors at d_kv = 1024 and Hadamard block = scale group = d_kv (the paper's
+ *     setting) ONE kernel: while the tensor cores form the predictions and the row warps reconstruct
+ *     token rows, attention warps of the same kernel take every 128-token block as soon as its keys and
+ *     values exist and reduce it to per-block softmax partials; the merge kernel follows.  Without
+ *     Khat/Vhat the decoded rows then live only in a ring of three waves of tokens in the workspace and
+ *     never reach HBM.  Other shapes and layer 0 fall back to the split form.
+ * The split form is the default because it is the faster one on B200: the row warps are what bounds the
+ * layer kernel, and the fused kernel has to give four of its ten row-warp slots per CTA to the attention
+ * warps (0.325 ms against 0.251 ms for 32768 tokens, 8.6 ms against 7.6 ms for 32 x 32768 with Khat/Vhat
+ * written in both).
  */
+int aquakv_set_attn_mode(aquakv_ctx* ctx, int mode); /* INVALID_ARG for an unknown mode; takes effect on the next call */
 int aquakv_decode_attn(aquakv_ctx* ctx, int32_t batch, int64_t ctx_len,
                        int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, float softmax_scale,
                        const void* q,

@@ -25,6 +25,7 @@ NOALLOC_MAX_TOKENS = 1024
 KERNEL_PREDICT, KERNEL_ENCODE_ROWS, KERNEL_DECODE_ROWS, KERNEL_ATTN, KERNEL_LAYER, KERNEL_CHAIN = 0, 1, 2, 3, 4, 5
 KERNEL_FIT = 6
 ERR_NUMERIC = -8
+ATTN_SPLIT, ATTN_FUSED = 0, 1
 CHAIN_MAX_TOKENS, CHAIN_MAX_LAYERS = 2048, 128
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -39,6 +40,7 @@ SYMBOLS = [
     "aquakv_fit_workspace_bytes", "aquakv_fit_predictor", "aquakv_gather_rows",
     "aquakv_decode_attn_buffered_workspace_bytes", "aquakv_decode_attn_buffered",
     "aquakv_rope_table", "aquakv_decode_attn_rope_workspace_bytes", "aquakv_decode_attn_rope",
+    "aquakv_set_attn_mode",
 ]
 
 
@@ -106,6 +108,8 @@ def _load():
     L.aquakv_decode_attn_buffered.argtypes = [vp, i32, i64, i32, i32, i32, f32, vp, vp, vp, vp, vp,
                                               vp, vp, i64, vp, vp, vp, vp, vp, vp, i64, i64, vp, vp, vp, vp, i64,
                                               vp, sz, vp]
+    L.aquakv_set_attn_mode.restype = ctypes.c_int
+    L.aquakv_set_attn_mode.argtypes = [vp, ctypes.c_int]
     L.aquakv_rope_table.restype = ctypes.c_int
     L.aquakv_rope_table.argtypes = [vp, i32, ctypes.c_double, i64, vp, vp]
     L.aquakv_decode_attn_rope_workspace_bytes.restype = sz
@@ -383,6 +387,13 @@ class Codec:
         if rc:
             raise AquaKVError(rc, "aquakv_decode_attn_buffered")
         return out, lse
+
+    def set_attn_mode(self, mode: int) -> None:
+        """ATTN_SPLIT (default: decode kernel, then attention over the fresh rows) or ATTN_FUSED (attention
+        warps inside the decode kernel where the shape allows it)."""
+        rc = lib.aquakv_set_attn_mode(self.h, int(mode))
+        if rc:
+            raise AquaKVError(rc, "aquakv_set_attn_mode")
 
     def rope_table(self, head_dim: int, theta_base: float, n_positions: int, device=None):
         """fp32 (cos, sin) pairs [n_positions, head_dim/2, 2] of the rotary angles, evaluated in double."""

@@ -47,6 +47,7 @@ struct aquakv_ctx {
   int sm_count;
   int chunk_tokens;        // tokens per L2-resident chunk
   int attn_block_tokens;   // tokens per split-KV block
+  int attn_mode;           // AQUAKV_ATTN_SPLIT or AQUAKV_ATTN_FUSED (aquakv_set_attn_mode)
   float4* d_grid4;
   uint32_t* d_signmask[2]; // [0] keys, [1] values
   int* d_status;
@@ -597,18 +598,18 @@ struct AttnWs {
 
 bool fused_attn_supported(const aquakv_ctx* c);
 
-// Workspace of aquakv_decode_attn.  With predictors at d_kv = 1024 (Hadamard block = scale group =
-// the row) decode and attention are ONE launch of the layer kernel: the workspace holds that
-// kernel's buffers (prediction ring, rings of three waves of decoded keys / values, counters) and
-// the attention partials, one slot per 128-token block that overlaps a sequence.  Otherwise (no
-// predictor, other shapes) the cache is decoded chunk by chunk, about 32 waves each, into the
+// Workspace of aquakv_decode_attn.  In the fused mode (aquakv_set_attn_mode), with predictors at
+// d_kv = 1024 (Hadamard block = scale group = the row), decode and attention are ONE launch of the
+// layer kernel: the workspace holds that kernel's buffers (prediction ring, rings of three waves of
+// decoded keys / values, counters) and the attention partials, one slot per 128-token block that
+// overlaps a sequence.  Otherwise the cache is decoded chunk by chunk, about 32 waves each, into the
 // workspace (or the caller's Khat/Vhat) and a separate kernel attends over each chunk in blocks of
 // 1024 tokens.
 AttnWs attn_ws(const aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_heads,
                int32_t head_dim, bool has_pred) {
   AttnWs w;
   const size_t d = size_t(c->p.d_kv);
-  w.fused = has_pred && fused_attn_supported(c);
+  w.fused = has_pred && c->attn_mode == AQUAKV_ATTN_FUSED && fused_attn_supported(c);
   if (w.fused) {
     w.n_splits = int((ctx_len + kAttnSubTokens - 2) / kAttnSubTokens) + 1;   // sub-blocks of the flattened token
                                                                              // index a sequence can overlap
@@ -2176,6 +2177,12 @@ int aquakv_decode_attn_buffered(aquakv_ctx* c, int32_t batch, int64_t ctx_len, i
   return decode_attn_impl(c, batch, ctx_len, n_q_heads, n_kv_heads, head_dim, softmax_scale, q, Kcodes, Kscales, Vcodes,
                           Vscales, Khat_prev, Vhat_prev, ld_prev, Wk, Wv, bk, bv, out, lse, Khat, Vhat, ld_hat, K16, V16,
                           n_uncompressed, ld16, nullptr, workspace, workspace_bytes, cuda_stream);
+}
+
+int aquakv_set_attn_mode(aquakv_ctx* c, int mode) {
+  if (c == nullptr || (mode != AQUAKV_ATTN_SPLIT && mode != AQUAKV_ATTN_FUSED)) return AQUAKV_ERR_INVALID_ARG;
+  c->attn_mode = mode;
+  return AQUAKV_OK;
 }
 
 int aquakv_rope_table(aquakv_ctx* c, int32_t head_dim, double theta_base, int64_t n_positions, float* table,

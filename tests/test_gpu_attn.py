@@ -27,8 +27,20 @@ CASES = [
 ]
 
 
-@pytest.mark.parametrize("batch,ctx,n_q,n_kv,hd,dtype,adapters", CASES)
-def test_decode_attn_matches_dequantize_then_attend(batch, ctx, n_q, n_kv, hd, dtype, adapters):
+def _case_modes():
+    """Every case in the default (split) form; the shapes the fused kernel covers (predictors, d_kv = 1024)
+    in the fused form too."""
+    from paper_2501_19392_b200 import api
+    out = []
+    for case in CASES:
+        out.append(case + (api.ATTN_SPLIT,))
+        if case[6] and case[3] * case[4] == 1024:
+            out.append(case + (api.ATTN_FUSED,))
+    return out
+
+
+@pytest.mark.parametrize("batch,ctx,n_q,n_kv,hd,dtype,adapters,mode", _case_modes())
+def test_decode_attn_matches_dequantize_then_attend(batch, ctx, n_q, n_kv, hd, dtype, adapters, mode):
     from paper_2501_19392_b200 import api
     d = n_kv * hd
     T = batch * ctx
@@ -37,6 +49,7 @@ def test_decode_attn_matches_dequantize_then_attend(batch, ctx, n_q, n_kv, hd, d
     grid = synth.lloyd_grid(16, seed=7, n_samples=1 << 14, iters=25)
     sk, sv = synth.hadamard_signs(d, 11), synth.hadamard_signs(d, 12)
     codec = api.Codec(d, d, d, grid, dtype, sk, sv)
+    codec.set_attn_mode(mode)
     ora = oracle.Oracle(d, d, d, grid, dtype, sk, sv)
     cache = synth.random_cache(shape, seed=5001, n_layers=1)
     q = synth.random_16bit((batch, n_q, hd), dtype, seed=5002)
@@ -91,8 +104,13 @@ def test_decode_attn_matches_dequantize_then_attend(batch, ctx, n_q, n_kv, hd, d
     assert np.all((np.abs(o - ref) <= 7e-3 * denom1) | adjacent1)
     assert np.abs(lse.cpu().numpy() - ref_lse).max() <= 5e-4
     # (4) without the optional K_hat/V_hat outputs the result is bit-identical
+    launches = codec.launch_count()
     out_b, lse_b = codec.decode_attn(*args, want_lse=True)
     assert torch.equal(out_b, out) and torch.equal(lse_b, lse)
+    # the fused form is one launch of the layer kernel and the merge; the split form adds the attention kernel
+    # per chunk (and runs two row kernels instead of the layer kernel when there is no predictor)
+    n = codec.launch_count() - launches
+    assert n == 2 if mode == api.ATTN_FUSED else n >= 3
 
 
 def test_decode_attn_at_the_full_llama31_8b_shape():
@@ -141,3 +159,16 @@ def test_decode_attn_at_the_full_llama31_8b_shape():
         denom = np.abs(ref).max(axis=-1, keepdims=True)
         assert np.all((np.abs(o - ref) <= 2e-3 * denom) | adjacent)
         assert np.abs(lse[s:s + 1].cpu().numpy() - ref_lse).max() <= 1e-4
+    # the fused form (attention warps inside the decode kernel) on the same call: the same decoded rows, and
+    # an output that differs only by the order of the fp32 partial sums
+    codec.set_attn_mode(api.ATTN_FUSED)
+    Kh2, Vh2 = torch.empty_like(Kh), torch.empty_like(Vh)
+    out2, lse2 = codec.decode_attn(q, cache.Kcodes[0], cache.Kscales[0], cache.Vcodes[0], cache.Vscales[0], ctx,
+                                   n_kv, scale, pK, pV, ad.Wk[1], ad.Wv[1], Khat=Kh2, Vhat=Vh2, want_lse=True)
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    assert torch.equal(Kh2, Kh) and torch.equal(Vh2, Vh)
+    o1, o2 = out.to(torch.float64).cpu().numpy(), out2.to(torch.float64).cpu().numpy()
+    near = np.abs(gpu_bits(out).astype(np.int64) - gpu_bits(out2).astype(np.int64)) <= 1
+    assert np.all((np.abs(o1 - o2) <= 2e-3 * np.abs(o1).max(axis=-1, keepdims=True)) | near)
+    assert (lse - lse2).abs().max().item() <= 1e-4
