@@ -606,10 +606,10 @@ bool fused_attn_supported(const aquakv_ctx* c);
 // workspace (or the caller's Khat/Vhat) and a separate kernel attends over each chunk in blocks of
 // 1024 tokens.
 AttnWs attn_ws(const aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32_t n_q_heads,
-               int32_t head_dim, bool has_pred) {
+               int32_t head_dim, bool want_fused) {
   AttnWs w;
   const size_t d = size_t(c->p.d_kv);
-  w.fused = has_pred && c->attn_mode == AQUAKV_ATTN_FUSED && fused_attn_supported(c);
+  w.fused = want_fused && fused_attn_supported(c);
   if (w.fused) {
     w.n_splits = int((ctx_len + kAttnSubTokens - 2) / kAttnSubTokens) + 1;   // sub-blocks of the flattened token
                                                                              // index a sequence can overlap
@@ -1314,7 +1314,7 @@ size_t aquakv_decode_attn_workspace_bytes(const aquakv_ctx* c, int32_t batch, in
                                           int32_t n_q_heads, int32_t head_dim) {
   if (c != nullptr && uniform_backbone(c)) return 0;
   if (c == nullptr || batch <= 0 || ctx_len <= 0 || n_q_heads <= 0 || head_dim <= 0) return 0;
-  // the caller may or may not pass predictors: the larger of the two layouts
+  // the caller may or may not pass predictors and may switch the mode: the larger of the two layouts
   const size_t a = attn_ws(c, batch, ctx_len, n_q_heads, head_dim, true).total;
   const size_t b = attn_ws(c, batch, ctx_len, n_q_heads, head_dim, false).total;
   return a > b ? a : b;
@@ -1993,7 +1993,8 @@ static int decode_attn_impl(aquakv_ctx* c, int32_t batch, int64_t ctx_len, int32
                           Vhat == Khat_prev || Vhat == Khat))
     return AQUAKV_ERR_INVALID_ARG;
   // with rotary keys the attention reads a rotated copy of the decoded rows: the two-kernel layout
-  const AttnWs ws = attn_ws(c, batch, ctx_len, n_q_heads, head_dim, has_pred && rope == nullptr);
+  const AttnWs ws = attn_ws(c, batch, ctx_len, n_q_heads, head_dim,
+                            has_pred && rope == nullptr && c->attn_mode == AQUAKV_ATTN_FUSED);
   const AttnExtWs xw = attn_ext_ws(c, ws.total, batch, n16, n_q_heads, head_dim);
   const RopeWs rw = rope_ws(c, n16 > 0 ? xw.total : ws.total,
                             rope != nullptr ? size_t(ws.chunk_blocks) * size_t(c->attn_block_tokens) : 0, batch, n16);
