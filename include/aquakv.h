@@ -89,8 +89,8 @@ typedef struct aquakv_params {
 
 typedef struct aquakv_ctx aquakv_ctx; /* opaque; owns the device copies of grid, signs, status */
 
-/* Bytes of one token's codes for these parameters (d_kv/2 * log2(n) / 8; with grid_dim = 1, see
- * aquakv_create, d_kv * log2(n) / 8), or a negative error. */
+/* Bytes of one token's codes for these parameters: d_kv / grid_dim * log2(grid_size) / 8 (d_kv/2 * log2(n) / 8
+ * for the planar grids; grid_dim 1 and 4: see aquakv_create), or a negative error. */
 int aquakv_code_bytes(const aquakv_params* params);
 
 /*
