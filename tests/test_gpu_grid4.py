@@ -98,6 +98,42 @@ def test_layer0_and_predicted_phases_match_the_oracle(d, h, g, dtype, T):
     assert codec.poll_status() == 0
 
 
+def test_full_size_call_on_sampled_rows():
+    """The benchmark's launch configuration (32768 tokens x d_kv 1024 in one call: four chunks of predictor
+    GEMM + row kernel per phase, the last one short) against the oracle on sampled rows, chunk borders
+    included; rows are independent, so the oracle's result for a row does not depend on the others."""
+    from paper_2501_19392_b200 import api
+    d, T, dtype = 1024, 32768, oracle.BF16
+    codec, ora = make(d, d, d, dtype)
+    shape = dataclasses.replace(synth.CONFIGS[2], n_tokens=T, n_layers=2)
+    kv = synth.kv_chain(shape, seed=6700, device=DEV)
+    ad = synth.random_adapters(shape, seed=6701, device=DEV)
+    prevK, prevV = kv.K[0], kv.V[0]          # any 16-bit rows serve as the previous layer's reconstruction
+    Kc, Ks, Vc, Vs, Kh, Vh = codec.encode(kv.K[1], kv.V[1], prevK, prevV, ad.Wk[1], ad.Wv[1])
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    rng = np.random.default_rng(67)
+    rows = np.unique(np.concatenate([[0, 1, 9471, 9472, 18943, 18944, 28415, 28416, T - 2, T - 1],
+                                     rng.integers(0, T, 120)]))
+    idx = torch.from_numpy(rows).to(DEV)
+    bits = synth.to_bits
+    sel = lambda t: bits(t[idx])
+    sc = lambda t: gpu_bits(t.view(torch.float16))
+    ok_ = ora.encode_phase(sel(kv.K[1]), [sel(prevK)], bits(ad.Wk[1]), role="k")
+    rows_ok, _ = scale_rows_ok(sc(Ks[idx]), ok_["scales"], ok_["scales_exact"])
+    same = check_tuples(Kc[idx].cpu().numpy(), ok_, rows_ok)
+    check_recon(gpu_bits(Kh[idx]), ok_["hat_exact"], ok_["hat"], dtype, same)
+    ov_ = ora.encode_phase(sel(kv.V[1]), [sel(prevV), gpu_bits(Kh[idx])], bits(ad.Wv[1]), role="v")
+    rows_ok, _ = scale_rows_ok(sc(Vs[idx]), ov_["scales"], ov_["scales_exact"])
+    same_v = check_tuples(Vc[idx].cpu().numpy(), ov_, rows_ok)
+    check_recon(gpu_bits(Vh[idx]), ov_["hat_exact"], ov_["hat"], dtype, same_v)
+    # decode of the library's own codes reproduces the encoder's reconstruction bit for bit, all rows
+    Kh2, Vh2 = codec.decode(Kc, Ks, Vc, Vs, prevK, prevV, ad.Wk[1], ad.Wv[1])
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    assert torch.equal(Kh2, Kh) and torch.equal(Vh2, Vh)
+
+
 def test_zero_rows_clamped_scale_and_rows_on_grid_points():
     from paper_2501_19392_b200 import api
     d, h, g = 256, 256, 256

@@ -178,6 +178,43 @@ def test_rotated_variant_spike_row_zero_row_and_clamp_on_the_gpu():
     assert codec.poll_status() == 0
 
 
+@pytest.mark.parametrize("b,g,h", [(2, 64, 1), (2, 1024, 1024)])
+def test_full_size_call_on_sampled_rows(b, g, h):
+    """The benchmark's launch configuration (32768 tokens x d_kv 1024 in one call: four chunks of predictor
+    GEMM + row kernel per phase, the last one short) against the oracle on sampled rows, chunk borders
+    included; rows are independent, so the oracle's result for a row does not depend on the others."""
+    from paper_2501_19392_b200 import api
+    d, T, dtype = 1024, 32768, oracle.BF16
+    codec, ora = make(d, b, g, dtype, h)
+    shape = dataclasses.replace(synth.CONFIGS[2], n_tokens=T, n_layers=2)
+    kv = synth.kv_chain(shape, seed=4700 + h, device=DEV)
+    ad = synth.random_adapters(shape, seed=4701 + h, device=DEV)
+    prevK, prevV = kv.K[0], kv.V[0]          # any 16-bit rows serve as the previous layer's reconstruction
+    Kc, Ks, Vc, Vs, Kh, Vh = codec.encode(kv.K[1], kv.V[1], prevK, prevV, ad.Wk[1], ad.Wv[1])
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    rng = np.random.default_rng(47)
+    rows = np.unique(np.concatenate([[0, 1, 9471, 9472, 18943, 18944, 28415, 28416, T - 2, T - 1],
+                                     rng.integers(0, T, 120)]))
+    idx = torch.from_numpy(rows).to(DEV)
+    bits = synth.to_bits
+    sel = lambda t: bits(t[idx])
+    ok_ = ora.encode_phase(sel(kv.K[1]), [sel(prevK)], bits(ad.Wk[1]), role="k")
+    rows_ok, _ = scale_rows_ok(gpu_bits(Ks[idx].view(torch.float16)), ok_["scales"], ok_["scales_exact"], SCALE_TOL)
+    same = check_levels(Kc[idx].cpu().numpy(), ok_, b, d, rows_ok)
+    check_recon(gpu_bits(Kh[idx]), ok_["hat_exact"], ok_["hat"], dtype, same)
+    ov_ = ora.encode_phase(sel(kv.V[1]), [sel(prevV), gpu_bits(Kh[idx])], bits(ad.Wv[1]), role="v")
+    rows_ok, _ = scale_rows_ok(gpu_bits(Vs[idx].view(torch.float16)), ov_["scales"], ov_["scales_exact"], SCALE_TOL)
+    same_v = check_levels(Vc[idx].cpu().numpy(), ov_, b, d, rows_ok)
+    check_recon(gpu_bits(Vh[idx]), ov_["hat_exact"], ov_["hat"], dtype, same_v)
+    assert same.mean() > 0.8 and same_v.mean() > 0.8
+    # decode of the library's own codes reproduces the encoder's reconstruction bit for bit, all rows
+    Kh2, Vh2 = codec.decode(Kc, Ks, Vc, Vs, prevK, prevV, ad.Wk[1], ad.Wv[1])
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    assert torch.equal(Kh2, Kh) and torch.equal(Vh2, Vh)
+
+
 def test_fitted_predictors_help_this_backbone_too():
     # Section 4.1 evaluates each backbone "with and without learned AQUA-KV predictors"
     from paper_2501_19392_b200 import api, calibrate as gcal
