@@ -148,6 +148,36 @@ def test_batch_of_sequences_shares_the_positions():
         rope_attn_check(out[b:b + 1], lse[b:b + 1], q[b:b + 1], rows_k, rows_v, positions, shape, scale, base)
 
 
+def test_full_context_across_a_chunk_border():
+    """6 sequences x 32768 tokens (196608 cached tokens: two decode chunks, the border inside the fifth
+    sequence), 32 query heads / 8 KV heads x 128, predictors: the oracle attends over the decoded rows of the
+    sequence that straddles the border and of the last one."""
+    from paper_2501_19392_b200 import api
+    B, ctx, pos0, base = 6, 32768, 4, 500000.0
+    shape = dataclasses.replace(synth.CONFIGS[5], n_tokens=B * ctx, n_layers=2, batch=B)
+    codec = make(shape)
+    d, hd, dt = shape.d_kv, shape.head_dim, shape.dtype
+    scale = 1.0 / math.sqrt(hd)
+    q = synth.random_16bit((B, shape.n_q_heads, hd), dt, 1, device=DEV)
+    table = codec.rope_table(hd, base, pos0 + ctx, DEV)
+    rc = synth.random_cache(shape, seed=4, device=DEV, n_layers=1)
+    ad = synth.random_adapters(shape, seed=5, device=DEV)
+    Kp = synth.random_16bit((B * ctx, d), dt, 6, device=DEV)
+    Vp = synth.random_16bit((B * ctx, d), dt, 7, device=DEV)
+    Kh = torch.empty((B * ctx, d), dtype=codec.torch_dtype, device=DEV)
+    Vh = torch.empty_like(Kh)
+    out, lse = codec.decode_attn_rope(q, rc.Kcodes[0], rc.Kscales[0], rc.Vcodes[0], rc.Vscales[0], ctx, shape.n_kv_heads,
+                                      scale, table, pos0, None, None, None, Kp, Vp, ad.Wk[1], ad.Wv[1], Khat=Kh, Vhat=Vh,
+                                      want_lse=True)
+    torch.cuda.synchronize()
+    assert codec.poll_status() == 0
+    positions = pos0 + np.arange(ctx)
+    for b in (4, B - 1):
+        sl = slice(b * ctx, (b + 1) * ctx)
+        rope_attn_check(out[b:b + 1], lse[b:b + 1], q[b:b + 1], gpu_bits(Kh[sl]), gpu_bits(Vh[sl]), positions, shape,
+                        scale, base)
+
+
 def test_error_paths():
     from paper_2501_19392_b200 import api
     shape = dataclasses.replace(synth.CONFIGS[5], n_tokens=256, n_layers=2, batch=1)
