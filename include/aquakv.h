@@ -118,7 +118,9 @@ int aquakv_code_bytes(const aquakv_params* params);
  * Four-dimensional grid (Section 4.1: "one grid without fast GPU support (2-bit precision, d = 4, n = 256)",
  * the paper's d being the grid dimension): grid_dim = 4 with grid_size = 256.  grid_host is then 256 x 4
  * floats; every consecutive 4-tuple of rotated normalised values goes to the nearest of the 256 points
- * (exhaustive search, lowest index on a tie) and takes one byte (d_kv / 4 bytes per token); scale,
+ * (lowest index on a tie; a table of candidate lists per cell of [-4, 4)^4, 16 MB, computed on the device
+ * by this call, with an exhaustive search for what it does not cover) and takes one byte (d_kv / 4 bytes
+ * per token); scale,
  * signs, rotation and reconstruction are those of the planar grids, with the same rules for had_block and
  * scale_group.  It is served like the uniform backbone.
  *

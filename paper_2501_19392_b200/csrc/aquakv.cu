@@ -49,6 +49,7 @@ struct aquakv_ctx {
   int attn_block_tokens;   // tokens per split-KV block
   int attn_mode;           // AQUAKV_ATTN_SPLIT or AQUAKV_ATTN_FUSED (aquakv_set_attn_mode)
   float4* d_grid4;
+  uint4* d_grid4_table;    // candidate lists of the four-dimensional grid's cells (grid_dim 4 only)
   uint32_t* d_signmask[2]; // [0] keys, [1] values
   int* d_status;
   uint32_t* d_search_table;
@@ -266,6 +267,7 @@ int launch_grid4_rows(aquakv_ctx* c, cudaStream_t st, int role, int rows, const 
   Grid4Args ga;
   UniformArgs& a = ga.u;
   ga.grid = c->d_grid4;
+  ga.table = c->d_grid4_table;
   ga.signmask = c->d_signmask[role];
   ga.log_h = c->log_h;
   a.X = static_cast<const uint16_t*>(X);
@@ -1264,6 +1266,15 @@ int aquakv_create(const aquakv_params* params, const float* grid_host, const int
   ok = ok && cudaMemcpy(c->d_signmask[0], masks[0], sizeof(masks[0]), cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(c->d_signmask[1], masks[1], sizeof(masks[1]), cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemset(c->d_status, 0, sizeof(int)) == cudaSuccess;
+  if (ok && gdim == 4) {
+    // the search table of the four-dimensional grid (16 MB) is computed on the device
+    const size_t n_cells = size_t(kGrid4Cells) * kGrid4Cells * kGrid4Cells * kGrid4Cells;
+    ok = cudaMalloc(&c->d_grid4_table, n_cells * sizeof(uint4)) == cudaSuccess;
+    if (ok) {
+      grid4_table_kernel<<<c->sm_count * 8, 256>>>(c->d_grid4, c->d_grid4_table);
+      ok = cudaGetLastError() == cudaSuccess;
+    }
+  }
   ok = ok && cudaFuncSetAttribute(gemm_pred_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   int(kGemmSmemBytes)) == cudaSuccess;
   ok = ok && cudaFuncSetAttribute(gemm_pred_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1285,6 +1296,7 @@ int aquakv_destroy(aquakv_ctx* c) {
   if (c == nullptr) return AQUAKV_OK;
   bool ok = true;
   if (c->d_grid4) ok = cudaFree(c->d_grid4) == cudaSuccess && ok;
+  if (c->d_grid4_table) ok = cudaFree(c->d_grid4_table) == cudaSuccess && ok;
   if (c->d_signmask[0]) ok = cudaFree(c->d_signmask[0]) == cudaSuccess && ok;
   if (c->d_signmask[1]) ok = cudaFree(c->d_signmask[1]) == cudaSuccess && ok;
   if (c->d_status) ok = cudaFree(c->d_status) == cudaSuccess && ok;

@@ -7,12 +7,19 @@
 //
 // One warp per row, the whole row in registers as in the rotated kernels of uniform.cuh: v[c][i] is value
 // 256 c + 8 lane + i, so a lane holds the tuples 64 c + 2 lane and 64 c + 2 lane + 1 of every chunk and
-// writes their codes as one 16-bit store.  The search is exhaustive: a 256-point grid in four dimensions
-// has no cheap cell structure like the planar grids' table, and this grid is the paper's slow one.  The
-// points sit in shared memory with half their squared norm, so a candidate costs four FMAs and a
-// compare: argmin |y - g|^2 = argmin (|g|^2 / 2 - y . g).  A lane's two tuples of a chunk go through the
-// packed two-lane fp32 FMA together (each lane rounds like the scalar instruction), which is why the
-// encoder's copy of the grid holds every coordinate twice.
+// writes their codes as one 16-bit store.  The points sit in shared memory with half their squared norm,
+// so a candidate costs four FMAs and a compare: argmin |y - g|^2 = argmin (|g|^2 / 2 - y . g).
+//
+// Search.  The hypercube [-4, 4)^4 is cut into 32^4 cells of side 1/4.  A table built on the device when
+// the context is created (grid4_table_kernel) lists, for every cell, every point that can be the nearest
+// one somewhere in the cell: with dmin(g) / dmax(g) the smallest / largest squared distance from the
+// (slightly inflated) cell to g and U = min_g dmax(g), the nearest point of any y in the cell has
+// dmin <= U, so the list {g : dmin(g) <= U (1 + 1e-4) + 1e-6} in ascending index order contains every
+// winner and every point tied with it; evaluating it with a strict "<" gives the result of the
+// exhaustive search.  An entry is 16 bytes: up to 15 indices, the last one repeated as padding, and their
+// count (4.8 on average for a Gaussian-optimal grid, where the exhaustive loop visits 256); 255 as the
+// count marks a cell with more candidates.  Tuples in such a cell or outside the hypercube (6e-5 of the
+// coordinates of a normalised row; also every non-finite value) take the exhaustive loop.
 #pragma once
 
 #include "uniform.cuh"
@@ -22,6 +29,7 @@ namespace aquakv {
 struct Grid4Args {
   UniformArgs u;              // X, P, codes, scales, hat, T, d, log_g as for the uniform backbone
   const float4* grid;         // [256] grid points
+  const uint4* table;         // [32^4] candidate lists of the cells (grid4_table_kernel); encode only
   const uint32_t* signmask;   // [32]: lane's word, bit 8 c + i set where the sign of value 256 c + 8 lane + i is -1
   int log_h;                  // 6 .. 10
 };
@@ -30,25 +38,80 @@ struct Grid4Smem {
   float4 g[256];
 };
 
-// The encoder's search copy: (x, x, y, y), (z, z, w, w) and (|g|^2 / 2, |g|^2 / 2) per point.
-struct Grid4SearchSmem {
-  float4 xy[256];
-  float4 zw[256];
-  float2 half_norm[256];
-};
+constexpr int kGrid4Cells = 32;             // per dimension
+constexpr float kGrid4Lo = -4.0f;           // the table covers [-4, 4)^4
+constexpr float kGrid4InvW = 4.0f;          // 1 / cell width
+constexpr unsigned kGrid4Overflow = 255u;   // count byte of a cell with more than 15 candidates
 
 __device__ __forceinline__ void grid4_load(Grid4Smem& sm, const float4* grid) {
   for (int k = threadIdx.x; k < 256; k += blockDim.x) sm.g[k] = grid[k];
   __syncthreads();
 }
 
-__device__ __forceinline__ void grid4_load_search(Grid4SearchSmem& ss, const float4* grid) {
-  for (int k = threadIdx.x; k < 256; k += blockDim.x) {
-    const float4 p = grid[k];
-    ss.xy[k] = make_float4(p.x, p.x, p.y, p.y);
-    ss.zw[k] = make_float4(p.z, p.z, p.w, p.w);
-    const float hn = 0.5f * (p.x * p.x + p.y * p.y + p.z * p.z + p.w * p.w);
-    ss.half_norm[k] = make_float2(hn, hn);
+// |g_k|^2 / 2 - y . g_k: the same instruction sequence wherever a candidate is evaluated.  The half norm
+// is recomputed from the point (five fp32 operations on an idle pipe) rather than looked up: a second
+// shared-memory access at a random index would cost more than it saves.
+__device__ __forceinline__ float grid4_score(const Grid4Smem& sm, int k, float y0, float y1, float y2, float y3) {
+  const float4 g = sm.g[k];
+  const float half_norm = 0.5f * fmaf(g.w, g.w, fmaf(g.z, g.z, fmaf(g.y, g.y, g.x * g.x)));
+  float s = fmaf(-y0, g.x, half_norm);
+  s = fmaf(-y1, g.y, s);
+  s = fmaf(-y2, g.z, s);
+  return fmaf(-y3, g.w, s);
+}
+
+// Candidate lists of all cells: one thread per cell, distances in double.
+__global__ void __launch_bounds__(256) grid4_table_kernel(const float4* __restrict__ grid, uint4* __restrict__ table) {
+  __shared__ float4 g[256];
+  for (int k = threadIdx.x; k < 256; k += blockDim.x) g[k] = grid[k];
+  __syncthreads();
+  constexpr int C = kGrid4Cells;
+  const long long n_cells = (long long)C * C * C * C;
+  for (long long cell = (long long)blockIdx.x * blockDim.x + threadIdx.x; cell < n_cells;
+       cell += (long long)gridDim.x * blockDim.x) {
+    int idx[4] = {int(cell / (C * C * C)), int(cell / (C * C) % C), int(cell / C % C), int(cell % C)};
+    double lo[4], hi[4];
+    for (int k = 0; k < 4; ++k) {
+      // inflated by 1e-5: the kernel finds the cell of a value with one fp32 rounding
+      lo[k] = double(kGrid4Lo) + double(idx[k]) / double(kGrid4InvW) - 1e-5;
+      hi[k] = double(kGrid4Lo) + double(idx[k] + 1) / double(kGrid4InvW) + 1e-5;
+    }
+    auto bounds = [&](int p, double& dmin, double& dmax) {
+      const double c[4] = {double(g[p].x), double(g[p].y), double(g[p].z), double(g[p].w)};
+      dmin = dmax = 0.0;
+      for (int k = 0; k < 4; ++k) {
+        const double below = lo[k] - c[k], above = c[k] - hi[k];
+        const double out = below > 0.0 ? below : (above > 0.0 ? above : 0.0);
+        const double far = fmax(fabs(c[k] - lo[k]), fabs(c[k] - hi[k]));
+        dmin += out * out;
+        dmax += far * far;
+      }
+    };
+    double U = 1.0e300;
+    for (int p = 0; p < 256; ++p) {
+      double dmin, dmax;
+      bounds(p, dmin, dmax);
+      U = fmin(U, dmax);
+    }
+    const double limit = U * (1.0 + 1e-4) + 1e-6;
+    unsigned w[4] = {0u, 0u, 0u, 0u};
+    int n = 0, last = 0;
+    for (int p = 0; p < 256; ++p) {
+      double dmin, dmax;
+      bounds(p, dmin, dmax);
+      if (dmin <= limit) {
+        if (n < 15) w[n >> 2] |= unsigned(p) << (8 * (n & 3));
+        last = p;
+        ++n;
+      }
+    }
+    if (n > 15) {
+      w[3] = (w[3] & 0x00ffffffu) | (kGrid4Overflow << 24);
+    } else {
+      for (int i = n; i < 15; ++i) w[i >> 2] |= unsigned(last) << (8 * (i & 3));
+      w[3] |= unsigned(n) << 24;
+    }
+    table[cell] = make_uint4(w[0], w[1], w[2], w[3]);
   }
 }
 
@@ -72,8 +135,6 @@ template <bool kBf16, int NCH>
 __global__ void __launch_bounds__(kUniformWarps * 32)
 grid4_encode_rows_kernel(const Grid4Args ga) {
   __shared__ Grid4Smem sm;
-  __shared__ Grid4SearchSmem ss_grid;
-  grid4_load_search(ss_grid, ga.grid);
   grid4_load(sm, ga.grid);
   const UniformArgs& a = ga.u;
   const int lane = threadIdx.x & 31;
@@ -131,39 +192,68 @@ grid4_encode_rows_kernel(const Grid4Args ga) {
     uniform_apply_signs<NCH>(v, sbits);
     uniform_hadamard<NCH>(v, ga.log_h, lane);
     uniform_scale_all<NCH>(v, rs);
-    // nearest grid point of every 4-tuple: exhaustive, candidates in ascending order, strict "<" keeps the lowest index
-    float best[NCH][2];
-    int arg[NCH][2];
-    f32x2_t ny[NCH][4];                  // (-y_j of the first tuple, -y_j of the second) for j = 0 .. 3
+    // nearest grid point of every 4-tuple: the candidates of the tuple's cell in ascending order, strict "<"
+    // keeps the lowest index; the exhaustive loop for what the table does not cover
+    uint4 entry[NCH][2];
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
-      best[c][0] = best[c][1] = 3.0e38f;
-      arg[c][0] = arg[c][1] = 0;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) ny[c][j] = pack2(-v[c][j], -v[c][4 + j]);
+      for (int u = 0; u < 2; ++u) {
+        int cell = 0;
+        bool inside = true;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float f = floorf((v[c][4 * u + k] - kGrid4Lo) * kGrid4InvW);
+          inside = inside && f >= 0.0f && f < float(kGrid4Cells);     // false for NaN
+          cell = cell * kGrid4Cells + int(fminf(fmaxf(f, 0.0f), float(kGrid4Cells - 1)));
+        }
+        entry[c][u] = inside ? __ldg(ga.table + cell) : make_uint4(0u, 0u, 0u, kGrid4Overflow << 24);
+      }
     }
-#pragma unroll 2
-    for (int k = 0; k < 256; ++k) {
-      const float4 gxy = ss_grid.xy[k], gzw = ss_grid.zw[k];
-      const float2 hn = ss_grid.half_norm[k];
-      const f32x2_t gx = pack2(gxy.x, gxy.y), gy = pack2(gxy.z, gxy.w), gz = pack2(gzw.x, gzw.y), gw = pack2(gzw.z, gzw.w);
-      const f32x2_t h2 = pack2(hn.x, hn.y);
+    int arg[NCH][2];
 #pragma unroll
-      for (int c = 0; c < NCH; ++c) {
-        f32x2_t s2 = fma2(ny[c][0], gx, h2);
-        s2 = fma2(ny[c][1], gy, s2);
-        s2 = fma2(ny[c][2], gz, s2);
-        s2 = fma2(ny[c][3], gw, s2);
-        float s0, s1;
-        unpack2(s2, s0, s1);
-        if (s0 < best[c][0]) {
-          best[c][0] = s0;
-          arg[c][0] = k;
+    for (int c = 0; c < NCH; ++c) {
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const float y0 = v[c][4 * u], y1 = v[c][4 * u + 1], y2 = v[c][4 * u + 2], y3 = v[c][4 * u + 3];
+        const unsigned n = entry[c][u].w >> 24;
+        const bool listed = n != kGrid4Overflow;
+        const unsigned n_max = __reduce_max_sync(0xffffffffu, listed ? n : 0u);
+        const unsigned words[4] = {entry[c][u].x, entry[c][u].y, entry[c][u].z, entry[c][u].w};
+        float best = 3.0e38f;
+        int best_k = 0;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          if (unsigned(4 * w) < n_max) {         // the same for the whole warp; shorter lists repeat their last index
+            // the four candidates of a word are scored side by side (independent look-ups), then compared in order
+            int k[4];
+            float sc[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              k[j] = int((words[w] >> (8 * j)) & 0xffu);
+              if (4 * w + j < 15) sc[j] = grid4_score(sm, k[j], y0, y1, y2, y3);
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              if (4 * w + j < 15 && sc[j] < best) {
+                best = sc[j];
+                best_k = k[j];
+              }
+            }
+          }
         }
-        if (s1 < best[c][1]) {
-          best[c][1] = s1;
-          arg[c][1] = k;
+        if (!listed) {
+          best = 3.0e38f;
+          best_k = 0;
+          for (int k = 0; k < 256; ++k) {
+            const float sc = grid4_score(sm, k, y0, y1, y2, y3);
+            if (sc < best) {
+              best = sc;
+              best_k = k;
+            }
+          }
         }
+        arg[c][u] = best_k;
       }
     }
 #pragma unroll
