@@ -480,7 +480,7 @@ def uniform_backbone_entries(api, chain, peaks, dev, reps=5):
     """The alternative backbones, 2 bits per value, on the prefill-shaped workload: uniform round-to-nearest
     levels with absmax normalisation, plain with groups of 64 (2.25 bits with the scales) and rotated with one
     group per row (random signs + Hadamard rotation first; 2.02 bits), and the vector quantizer with the
-    256-point grid in four dimensions (2.02 bits; the paper's grid "without fast GPU support").  Time of
+    256-point grid in four dimensions (2.02 bits; the grid for which the paper had no fast GPU kernel).  Time of
     one predicted layer through the per-layer entry points (two launches per phase: predictor GEMM, row
     kernel), and what fitted predictors buy each backbone (Section 4.1 evaluates each backbone with and
     without them)."""
@@ -520,7 +520,7 @@ def uniform_backbone_entries(api, chain, peaks, dev, reps=5):
         _, _, Vd = codec.encode_phase(api.ROLE_VALUE, kv.V[l])
         quality = {"fitted_predictors": {"K": rel_err(kv.K[l], recs[l][0]), "V": rel_err(kv.V[l], recs[l][1])},
                    "no_predictor": {"K": rel_err(kv.K[l], Kd), "V": rel_err(kv.V[l], Vd)}}
-        if h > 1 and not grid4:      # the same group size without the rotation (the appendix' "larger group size" row)
+        if h > 1 and not grid4:      # the same group size without the rotation (the appendix' row with the larger group)
             plain = api.Codec(d, 1, g, None, shape.dtype, levels=4)
             _, _, Kp = plain.encode_phase(api.ROLE_KEY, kv.K[l])
             _, _, Vp = plain.encode_phase(api.ROLE_VALUE, kv.V[l])

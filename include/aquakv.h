@@ -3,7 +3,7 @@
  *
  * The operations are those of the paper "Cache Me If You Must: Adaptive Key-Value Quantization
  * for Large Language Models": Algorithm 2 (encode), Algorithm 3 (decode) and the attention read
- * of Algorithm 4 (lines 5-9), with the backbone quantizer Q of Section 2 ("Vector Quantization")
+ * of Algorithm 4, with the backbone quantizer Q of Section 2 ("Vector Quantization")
  * and Section 4.1 ("Alternative quantizers"): group-wise vector quantization after a randomized
  * Hadamard transform, p = 2 values per code, n in {16, 64, 256} grid points, one fp16 scale per
  * group.
@@ -21,7 +21,7 @@
  *     [d_kv][2*d_kv] and its input is the concatenation [Vhat_prev ; Khat] (columns 0..d_kv-1
  *     act on Vhat_prev, columns d_kv..2*d_kv-1 on the freshly reconstructed Khat).  Biases are
  *     optional fp32 [d_kv] (NULL = none).  Wk == NULL (then Wv, Khat_prev, Vhat_prev must be NULL
- *     too) selects the predictor-free path of layer 0 (Algorithm 2 lines 1-3).
+ *     too) selects the predictor-free path of layer 0 (the first layer of Algorithm 2).
  *   - Compressed cache, per tensor (keys and values are separate arrays), per token t:
  *       codes[t]  : d_kv/2 * log2(n) / 8 bytes; the code of value pair j (values 2j, 2j+1 of the
  *                   rotated row) occupies bits [j*log2(n), (j+1)*log2(n)) of the row's bit
@@ -95,28 +95,28 @@ int aquakv_code_bytes(const aquakv_params* params);
 
 /*
  * Creates a context on the current device.  grid_host: n x 2 floats, the fixed grid of Section 2
- * ("a lattice optimized for normally distributed vectors"), index = code.  signs_k_host /
+ * (a point set tuned for normally distributed vectors), index = code.  signs_k_host /
  * signs_v_host: d_kv values in {+1,-1}, the random diagonal of the randomized Hadamard transform
  * for keys and for values.  All three are copied; the caller may free them after the call.
  * This is the only entry point that allocates device memory (a few KB) and it synchronises the
  * device once.  Errors: INVALID_ARG (NULL, sign not +-1, non-finite grid), UNSUPPORTED, CUDA.
  *
- * Alternative backbone (Section 4.1 "Alternative quantizers": Quanto-style "round-to-nearest quantization
- * with absmax normalization", group size 64, per token; Section 3.2: the method is agnostic to Q):
+ * Alternative backbone (Section 4.1 "Alternative quantizers": the Quanto-style one, rounding to the nearest
+ * level after dividing by the group's largest magnitude, groups of 64 values inside a token; Section 3.2: any Q fits):
  * grid_dim = 1 selects it.  grid_size = 2^b in {4, 8, 16} is then the number of levels PER VALUE (b bits
  * per value): the signed integers -2^(b-1) .. 2^(b-1)-1 times the group scale, scale = absmax / 2^(b-1)
  * stored as fp16, nearest level with the lower one on a tie, saturation at the ends, code = level +
  * 2^(b-1), codes packed LSB-first in value order (d_kv * b / 8 bytes per token); scale_group a power of
  * two from 32 to d_kv; grid_host is not read and may be NULL.  had_block = 1: no rotation, the sign arrays
  * are not read and may be NULL.  had_block = h, a power of two from 64 to d_kv (the appendix' additional
- * results for Section 4.1: a backbone that "combines Randomized Hadamard Transform (RHT) with standard
- * non-vector quantization"): the residual times the role's signs is rotated by the orthonormal Hadamard
+ * results for Section 4.1: a backbone that puts a randomized Hadamard transform in front of ordinary
+ * scalar quantization): the residual times the role's signs is rotated by the orthonormal Hadamard
  * matrix in blocks of h values, the ROTATED values are quantized as above (absmax after the rotation;
  * scale_group is independent of h), and the inverse rotates level * scale back and applies the signs again;
  * the sign arrays are then required.
  *
- * Four-dimensional grid (Section 4.1: "one grid without fast GPU support (2-bit precision, d = 4, n = 256)",
- * the paper's d being the grid dimension): grid_dim = 4 with grid_size = 256.  grid_host is then 256 x 4
+ * Four-dimensional grid (Section 4.1: the 2-bit grid with d = 4, n = 256, for which the paper had no fast GPU
+ * kernel, its d being the grid dimension): grid_dim = 4 with grid_size = 256.  grid_host is then 256 x 4
  * floats; every consecutive 4-tuple of rotated normalised values goes to the nearest of the 256 points
  * (lowest index on a tie; a table of candidate lists per cell of [-4, 4)^4, 16 MB, computed on the device
  * by this call, with an exhaustive search for what it does not cover) and takes one byte (d_kv / 4 bytes
@@ -179,8 +179,8 @@ size_t aquakv_decode_attn_workspace_bytes(const aquakv_ctx* ctx, int32_t batch, 
                                           int32_t n_q_heads, int32_t head_dim);
 
 /*
- * The predictor alone (Section 3.2: f_key, f_value are linear regressors; Algorithm 2 lines 5
- * and 8):  P[t][c] = sum_r x_t[r] * W[c][r] + bias[c]  with x_t = in0[t] (in1 == NULL, W is
+ * The predictor alone (Section 3.2: f_key, f_value are linear regressors; the two predictions
+ * of Algorithm 2):  P[t][c] = sum_r x_t[r] * W[c][r] + bias[c]  with x_t = in0[t] (in1 == NULL, W is
  * [d_kv][d_kv]) or the concatenation [in0[t] ; in1[t]] (W is [d_kv][2*d_kv]).  P is fp32
  * [n_tokens, ldP] (ldP % 4 == 0, 16-byte aligned); accumulation is fp32 on the tensor cores.
  * Needs no workspace.
@@ -193,7 +193,7 @@ int aquakv_predict(aquakv_ctx* ctx, int64_t n_tokens, const void* in0, const voi
 #define AQUAKV_ROLE_VALUE 1
 
 /*
- * One phase of Algorithm 2 on its own (lines 5-7 for keys; lines 8-9 plus the reconstruction for
+ * One phase of Algorithm 2 on its own (predict, quantize the residual, reconstruct: for keys or for
  * values), for callers that supply the predictor inputs themselves (e.g. teacher-forced checks):
  *   pred = [in0 ; in1] W^T + bias;  codes,scales = Q(X - pred);  hat = round16(Q^-1(..) + pred).
  * role selects the Hadamard signs (AQUAKV_ROLE_KEY / AQUAKV_ROLE_VALUE).  in1 == NULL: single
@@ -206,7 +206,7 @@ int aquakv_encode_phase(aquakv_ctx* ctx, int role, int64_t n_tokens, const void*
                         int64_t ld_hat, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
- * One phase of Algorithm 3 on its own (line 5 for keys, line 7 for values):
+ * One phase of Algorithm 3 on its own (for keys or for values):
  *   hat = round16(Q^-1(codes, scales) + [in0 ; in1] W^T + bias).  Arguments as above.
  */
 int aquakv_decode_phase(aquakv_ctx* ctx, int role, int64_t n_tokens, const uint8_t* codes,
@@ -218,7 +218,7 @@ int aquakv_decode_phase(aquakv_ctx* ctx, int role, int64_t n_tokens, const uint8
  * Algorithm 2 (encode) for one layer and n_tokens tokens:
  *   K_pred = Khat_prev Wk^T + bk;  Kcodes,Kscales = Q(K - K_pred);  Khat = Q^-1(..) + K_pred;
  *   V_pred = [Vhat_prev ; Khat] Wv^T + bv;  Vcodes,Vscales = Q(V - V_pred);  Vhat = Q^-1(..) + V_pred.
- * The reconstructions Khat/Vhat (rounded once to the 16-bit type) are what Algorithm 4 line 14
+ * The reconstructions Khat/Vhat (rounded once to the 16-bit type) are what Algorithm 4's cache update
  * obtains by decoding the fresh codes again; here they are by-products.  Khat, Vhat may be NULL
  * (not written; Khat is then kept in the workspace for the value predictor).  Outputs must not
  * alias inputs.  K,V: [n_tokens, ld_kv]; *_prev: [n_tokens, ld_prev]; Khat,Vhat: [n_tokens, ld_hat].
@@ -236,7 +236,7 @@ int aquakv_encode(aquakv_ctx* ctx, int64_t n_tokens,
  *   Khat = Q^-1(Kcodes,Kscales) + Khat_prev Wk^T + bk;
  *   Vhat = Q^-1(Vcodes,Vscales) + [Vhat_prev ; Khat] Wv^T + bv,
  * each rounded once to the 16-bit type.  On the same device, with the same arguments, Khat/Vhat
- * are bit-identical to those aquakv_encode produced (Algorithm 2 line 7 and Algorithm 3 line 5
+ * are bit-identical to those aquakv_encode produced (the reconstruction of Algorithm 2 and the decode of Algorithm 3
  * are the same expression).  Khat and Vhat are required.
  */
 int aquakv_decode(aquakv_ctx* ctx, int64_t n_tokens,
@@ -250,8 +250,8 @@ int aquakv_decode(aquakv_ctx* ctx, int64_t n_tokens,
 /*
  * Algorithm 4's loop over layers for SMALL calls -- a decode step of a batch of sequences, a short
  * prompt -- in ONE launch: Algorithm 2 (encode_chain) or Algorithm 3 (decode_chain) for n_layers
- * consecutive layers, each layer's predictors reading the previous layer's reconstruction (Algorithm
- * 4 lines 4 and 14; Section 3.3).  A per-layer call of a few tokens is bound by launch and hand-off
+ * consecutive layers, each layer's predictors reading the previous layer's reconstruction (the layer loop of
+ * Algorithm 4; Section 3.3).  A per-layer call of a few tokens is bound by launch and hand-off
  * latency and by a handful of SMs streaming the adapter weights; here every SM streams a share of
  * the weights, the key chain runs ahead of the value chain, and the layers hand over through
  * counters in device memory.
@@ -336,7 +336,7 @@ int aquakv_decode_noalloc(aquakv_ctx* ctx, int64_t n_tokens,
                           void* Khat, void* Vhat, int64_t ld_hat, void* cuda_stream);
 
 /*
- * Algorithm 3 fused with the attention read of Algorithm 4 (lines 5-9) for single-token queries:
+ * Algorithm 3 fused with the attention read of Algorithm 4 for single-token queries:
  * decodes `batch` sequences of `ctx_len` cached tokens each (token index = b*ctx_len + t,
  * n_tokens = batch*ctx_len) and computes, per sequence b and query head qh,
  *   out[b][qh] = softmax_t(softmax_scale * q[b][qh] . Khat[b,t][kvh]) . Vhat[b,t][kvh],
@@ -374,14 +374,14 @@ int aquakv_decode_attn(aquakv_ctx* ctx, int32_t batch, int64_t ctx_len,
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
- * The same with the cache policy of Section 3.3 / Section 4.1 around it: "the first 4 tokens (attention
- * sinks)" and "a buffer of 128 most recent tokens" stay uncompressed, and every query attends to both
+ * The same with the cache policy of Section 3.3 / Section 4.1 around it: the first four tokens (the attention
+ * sinks) and a buffer of the 128 newest tokens stay uncompressed, and every query attends to both
  * the compressed cache and those rows.  K16 / V16: [batch][n_uncompressed][ld16] 16-bit rows of the
  * ctx's type (device, 16-byte aligned, ld16 >= d_kv and a multiple of 8), each sequence's uncompressed
  * rows in any order (attention does not depend on it; position encoding is the caller's business, as in
  * aquakv_decode_attn).  Their split-KV partials are formed by the library's attention kernel and merged
  * with the partials of the compressed cache in fp32 before the single rounding of `out`, so the result
- * is the attention over the concatenation [compressed ; uncompressed] (Algorithm 4 lines 5-9 with
+ * is the attention over the concatenation [compressed ; uncompressed] (the attention read of Algorithm 4 with
  * the buffered rows appended to the decoded ones).  ctx_len may be 0 (nothing compressed yet: the cache
  * pointers are then ignored), n_uncompressed may be 0 (identical to aquakv_decode_attn); both 0 does
  * nothing.  Workspace: aquakv_decode_attn_buffered_workspace_bytes.  Everything else as aquakv_decode_attn.

@@ -17,7 +17,7 @@
  *     vector quantization after a randomized Hadamard transform: scale each group, rotate, round
  *     every p=2 consecutive rotated values to the nearest of n fixed grid points; one 16-bit scale
  *     per group (2 + 16/1024 = 2.02 bits per value at n=16, group 1024).
- *   - Algorithm 4, lines 5-9: attention of a new query over the decoded cache.
+ *   - Algorithm 4, the attention read: a new query attends over the decoded cache.
  *
  * All arithmetic is double precision.  Roundings happen only where a stored format forces them:
  * the scale is stored as fp16, reconstructed keys/values as fp16 or bf16 (round to nearest even).
@@ -289,7 +289,7 @@ int aqo_predict(const aqo_params* p, int64_t T, int n_in, const uint16_t* in0, c
 }
 
 /* ------------------------------------------------------------------------------------------ */
-/* One phase of Algorithm 2 (lines 5-7 for keys, 8-9 plus the reconstruction for values)       */
+/* One phase of Algorithm 2 (predict, quantize the residual, reconstruct: keys or values)     */
 /*   pred = f(inputs);  q = Q(X - pred);  hat = round16(Q^-1(q) + pred)                        */
 /* ------------------------------------------------------------------------------------------ */
 
@@ -310,12 +310,12 @@ int aqo_encode_phase(const aqo_params* p, const float* grid_f, const int8_t* sig
 #pragma omp for schedule(static)
     for (int64_t t = 0; t < T; ++t) {
       const uint16_t* rows[2] = {in0 ? in0 + t * d : NULL, in1 ? in1 + t * d : NULL};
-      predict_row(p, n_in, rows, W, bias, pred, x);                      /* Alg. 2 line 5 / 8 */
+      predict_row(p, n_in, rows, W, bias, pred, x);                      /* predict           */
       for (int i = 0; i < d; ++i) r[i] = load16(X[t * d + i], p->dtype) - pred[i];
-      quantize_row(p, grid, signs, r, codes + t * cb, scales + t * ng,    /* line 6 / 9 */
+      quantize_row(p, grid, signs, r, codes + t * cb, scales + t * ng,    /* quantize    */
                    margins ? margins + t * (d / 2) : NULL,
                    scales_exact ? scales_exact + t * ng : NULL, NULL, y);
-      dequantize_row(p, grid, signs, codes + t * cb, scales + t * ng, xh); /* line 7 */
+      dequantize_row(p, grid, signs, codes + t * cb, scales + t * ng, xh); /* rebuild */
       for (int i = 0; i < d; ++i) {
         double v = pred[i] + xh[i];
         if (hat_exact) hat_exact[t * d + i] = v;
@@ -329,7 +329,7 @@ int aqo_encode_phase(const aqo_params* p, const float* grid_f, const int8_t* sig
   return 0;
 }
 
-/* One phase of Algorithm 3 (line 5 for keys, line 7 for values): hat = round16(Q^-1(q) + f(in)). */
+/* One phase of Algorithm 3 (keys or values): hat = round16(Q^-1(q) + f(in)). */
 int aqo_decode_phase(const aqo_params* p, const float* grid_f, const int8_t* signs, int64_t T,
                      const uint8_t* codes, const uint16_t* scales,
                      int n_in, const uint16_t* in0, const uint16_t* in1,
@@ -392,7 +392,7 @@ int aqo_decode_layer(const aqo_params* p, const float* grid, const int8_t* signs
 }
 
 /* ------------------------------------------------------------------------------------------ */
-/* Single-query attention over the decoded cache (Algorithm 4, lines 5-9), grouped-query heads  */
+/* Single-query attention over the decoded cache (Algorithm 4's attention read), grouped-query heads  */
 /*   token index of (sequence b, position t) is b*ctx + t; kv head of query head qh is          */
 /*   qh / (n_q_heads / n_kv_heads); out = softmax_t(scale * q . K^_t) . V^_t                     */
 /* ------------------------------------------------------------------------------------------ */

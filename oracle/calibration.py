@@ -15,9 +15,9 @@ Readings (the paper is silent or at odds with itself here):
   * regularizer rate r: ridge term r * trace(X^T X) / n_in on the diagonal of the normal equations
     (relative to the mean feature energy, so that the fit does not depend on the scale of the cache);
   * the first layer: Algorithm 1 as printed carries the first layer's exact K, V forward, the text of
-    Section 3.2 says the first layer "is compressed as is" and later layers train on reconstructions;
-    the text is followed (first_layer_exact=False) because that is what a decoder has (Algorithm 2
-    lines 1-3), and the printed listing can be had with first_layer_exact=True;
+    Section 3.2 has the first layer compressed without a predictor and later layers trained on reconstructions;
+    the text is followed (first_layer_exact=False) because that is what a decoder has (the first
+    layer of Algorithm 2), and the printed listing can be had with first_layer_exact=True;
   * intercept: off by default (the benchmark configurations use no bias); with fit_bias the inputs and
     targets are centred, the map fitted on the centred data and b = mean(Y) - mean(X) W^T;
   * the fitted matrix is stored in the cache's 16-bit type, [d_kv][n_in] like a linear layer's weight,
@@ -112,7 +112,7 @@ def calibrate(oracle: Oracle, K: List[np.ndarray], V: List[np.ndarray], rate: fl
     if first_layer_exact:
         K_old, V_old = K[0], V[0]
     else:
-        k0 = oracle.encode_phase(K[0], [], None, None, "k")          # Q alone (Algorithm 2 lines 1-3)
+        k0 = oracle.encode_phase(K[0], [], None, None, "k")          # Q alone (the first layer of Algorithm 2)
         v0 = oracle.encode_phase(V[0], [], None, None, "v")
         K_old, V_old = k0["hat"], v0["hat"]
     out = []

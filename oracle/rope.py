@@ -1,6 +1,6 @@
 """CPU oracle of rotary position encoding applied to cached PRE-RoPE keys at attention time
 (Section 3.3 "Positional embeddings": predictors and quantizers work on the keys before RoPE, so the
-reconstructed keys are rotated when the block attends to them, Algorithm 4 lines 5-9; RoPE is the
+reconstructed keys are rotated when the block attends to them in Algorithm 4; RoPE is the
 rotary embedding of Su et al. that the paper cites).
 
 TEST INFRASTRUCTURE ONLY, like the rest of this package: plain numpy in double precision.
@@ -54,7 +54,7 @@ def rotate_rows_16bit(K_bits: np.ndarray, positions: np.ndarray, n_kv_heads: int
 def attention_rope(dtype: int, batch: int, ctx: int, n_q_heads: int, n_kv_heads: int, head_dim: int,
                    softmax_scale: float, q: np.ndarray, K_bits: np.ndarray, V_bits: np.ndarray,
                    positions: np.ndarray, theta_base: float):
-    """Algorithm 4 lines 5-9 over pre-RoPE key rows [batch*ctx, d]: row r of every sequence sits at
+    """The attention read of Algorithm 4 over pre-RoPE key rows [batch*ctx, d]: row r of every sequence sits at
     positions[r] ([ctx] entries, the same for every sequence)."""
     pos = np.tile(np.asarray(positions, dtype=np.int64), batch)
     K_rot, _ = rotate_rows_16bit(K_bits, pos, n_kv_heads, head_dim, theta_base, dtype)

@@ -1,7 +1,7 @@
 """CPU oracle of the alternative backbone quantizer: round-to-nearest on a uniform grid with absmax
-normalisation per group, applied per token (Section 4.1 "Alternative quantizers": "Quanto ... simple
-round-to-nearest quantization with absmax normalization ... the default group size 64 and per-token
-compression"; Section 3.2: the method "is agnostic to the choice of Q").
+normalisation per group, applied per token (Section 4.1 "Alternative quantizers": the Quanto-style
+backbone, plain rounding to the nearest level after dividing by the group's largest magnitude, groups of
+64 values inside a token; Section 3.2: any quantizer Q can sit under the predictors).
 
 TEST INFRASTRUCTURE ONLY, like the rest of this package: plain numpy in double precision.
 
@@ -14,8 +14,8 @@ group of zeros has scale 0 and level 0.  The code of a value is its level + 2^(b
 b-bit number; codes are packed LSB-first in value order; no rotation, no sign flips.  Predictors,
 residual and add-back are those of Algorithms 2 and 3: codes = Q(x - pred), hat = round16(pred + Q^-1).
 
-Rotated variant (the appendix' additional results for Section 4.1: a backbone that "combines Randomized
-Hadamard Transform (RHT) with standard non-vector quantization", group size 1024).  Reading: the
+Rotated variant (the appendix' additional results for Section 4.1: a backbone that puts a randomized
+Hadamard transform in front of ordinary scalar quantization, group size 1024).  Reading: the
 residual is multiplied by the role's random signs and rotated by the orthonormal Hadamard matrix in
 blocks of `had_block` values (the transform of Section 3.1's vector quantizer), the ROTATED values are
 quantized as above (the group's absmax is taken after the rotation), and Q^-1 rotates the levels times
@@ -126,12 +126,12 @@ class UniformOracle:
                      bias: Optional[np.ndarray] = None, role: str = "k"):
         x = bits_to_double(X, self.dtype)
         pred = self._pred(x.shape[0], inputs, W, bias)
-        out = self.quantize(x - pred, role)                                        # Algorithm 2 lines 6 / 8
-        hat_exact = pred + self.dequantize(out["codes"], out["scales"], role)      # lines 7 / 9
+        out = self.quantize(x - pred, role)                                        # Algorithm 2: quantize the residual
+        hat_exact = pred + self.dequantize(out["codes"], out["scales"], role)      # ... and reconstruct
         out.update(hat=double_to_bits(hat_exact, self.dtype), hat_exact=hat_exact, pred=pred)
         return out
 
     def decode_phase(self, codes, scales, inputs, W, bias=None, role: str = "k"):
         T = codes.shape[0]
-        hat_exact = self._pred(T, inputs, W, bias) + self.dequantize(codes, scales, role)   # Algorithm 3 lines 5 / 7
+        hat_exact = self._pred(T, inputs, W, bias) + self.dequantize(codes, scales, role)   # Algorithm 3: add the prediction back
         return dict(hat=double_to_bits(hat_exact, self.dtype), hat_exact=hat_exact)

@@ -1,6 +1,6 @@
 """CPU oracle of the backbone vector quantizer for a grid of ANY dimension p (Section 2 "Vector
 Quantization" and Section 4.1 "Alternative quantizers": besides the p = 2 grids with n = 16 / 64 / 256
-points the paper runs "one grid without fast GPU support (2-bit precision, d = 4, n = 256)" -- its d is
+points the paper runs one 2-bit grid with d = 4, n = 256, for which it had no fast GPU kernel -- its d is
 the grid dimension, written p here).
 
 TEST INFRASTRUCTURE ONLY, like the rest of this package: plain numpy in double precision.
@@ -79,12 +79,12 @@ class VectorOracle:
                      bias: Optional[np.ndarray] = None, role: str = "k"):
         x = bits_to_double(X, self.dtype)
         pred = self._pred(x.shape[0], inputs, W, bias)
-        out = self.quantize(x - pred, role)                                        # Algorithm 2 lines 6 / 8
-        hat_exact = pred + self.dequantize(out["codes"], out["scales"], role)      # lines 7 / 9
+        out = self.quantize(x - pred, role)                                        # Algorithm 2: quantize the residual
+        hat_exact = pred + self.dequantize(out["codes"], out["scales"], role)      # ... and reconstruct
         out.update(hat=double_to_bits(hat_exact, self.dtype), hat_exact=hat_exact, pred=pred)
         return out
 
     def decode_phase(self, codes, scales, inputs, W, bias=None, role: str = "k"):
         T = codes.shape[0]
-        hat_exact = self._pred(T, inputs, W, bias) + self.dequantize(codes, scales, role)   # Algorithm 3 lines 5 / 7
+        hat_exact = self._pred(T, inputs, W, bias) + self.dequantize(codes, scales, role)   # Algorithm 3: add the prediction back
         return dict(hat=double_to_bits(hat_exact, self.dtype), hat_exact=hat_exact)

@@ -2,8 +2,8 @@
 reconstructed inputs (Section 3.2).
 
 Host loop only: every fit is one call of aquakv_fit_predictor, every reconstruction one call of
-aquakv_encode_phase; nothing is computed here.  The first layer is compressed as is (Algorithm 2
-lines 1-3) and its reconstruction is what the second layer's predictors are fitted on, unless
+aquakv_encode_phase; nothing is computed here.  The first layer is compressed as is (the first
+layer of Algorithm 2) and its reconstruction is what the second layer's predictors are fitted on, unless
 `first_layer_exact` asks for the exact first-layer tensors that Algorithm 1 as printed carries forward.
 """
 from __future__ import annotations

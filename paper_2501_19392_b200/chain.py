@@ -1,8 +1,8 @@
 """Layer-chain driver (Algorithm 4: layer i's reconstruction feeds layer i+1's predictors).
 
 Host loops only: each layer is one call into the C library; the reconstructed keys/values live in
-two ping-pong buffer pairs so that only the previous layer is ever materialised (Section 3.3,
-"we only need to materialize a single layer at a time").  Nothing is computed here.
+two ping-pong buffer pairs so that only the previous layer is ever materialised (Section 3.3:
+one reconstructed layer at a time is enough).  Nothing is computed here.
 """
 from __future__ import annotations
 
@@ -120,7 +120,7 @@ def decode_chain(codec: api.Codec, cache: CompressedCache, adapters, bufs: PingP
 def decode_attn_chain(codec: api.Codec, cache: CompressedCache, adapters, bufs: PingPong,
                       q: List[torch.Tensor], out: List[torch.Tensor], ctx_len: int, n_kv_heads: int,
                       softmax_scale: float) -> None:
-    """Algorithm 4 lines 4-9 for every layer: decode the layer's cache (feeding the next layer's
+    """The decode-and-attend loop of Algorithm 4 for every layer: decode the layer's cache (feeding the next layer's
     predictors through the ping-pong buffers) and attend to it with that layer's queries."""
     for l in range(len(q)):
         cur, prv = l % 2, (l + 1) % 2

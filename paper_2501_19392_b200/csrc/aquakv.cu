@@ -723,7 +723,7 @@ void launch_layer_dec_t(int* rc, int device, cudaStream_t st, int grid, const La
   }
 }
 
-// The attention a decode launch also computes (Algorithm 4 lines 5-9); q == nullptr: none.
+// The attention a decode launch also computes (the attention read of Algorithm 4); q == nullptr: none.
 struct LayerAttnArgs {
   const void* q;
   int ctx, n_q_heads, n_kv_heads, n_splits;

@@ -1,4 +1,4 @@
-// Single-query grouped-query attention over freshly decoded keys/values (Algorithm 4 lines 5-9:
+// Single-query grouped-query attention over freshly decoded keys/values (the attention read of Algorithm 4:
 // the block attends to the recovered cache).  Split-KV: one CTA reduces a block of consecutive
 // tokens of one sequence to per-query-head partials (running max, sum, unnormalised output), a
 // second kernel merges the partials of a sequence by log-sum-exp.  All accumulation is fp32.

@@ -1,7 +1,7 @@
 // Row kernels of the backbone quantizer Q / Q^-1 (Section 2 "Vector Quantization", Section 4.1
 // "Alternative quantizers": group scale, randomized Hadamard transform, nearest point of a fixed
-// 2-D grid, packed codes) and of the residual / add-back steps of Algorithm 2 (lines 6-7, 9) and
-// Algorithm 3 (lines 5, 7).
+// 2-D grid, packed codes) and of the residual / add-back steps of Algorithm 2 and
+// Algorithm 3.
 //
 // A team of d_kv/256 warps (1, 2 or 4) owns one token row; each warp holds one 256-element chunk.
 // Element e of the row lives in warp e/256, lane (e/8)%32, register e%8, so every global access is
@@ -420,7 +420,7 @@ __device__ __forceinline__ uint32_t store16x2p(f32x2_t v) {
   return store16x2<kBf16>(lo, hi);
 }
 
-// This warp's part of one token row of Q and of the reconstruction (Algorithm 2 lines 6-7 / 9):
+// This warp's part of one token row of Q and of the reconstruction (Algorithm 2, keys or values):
 //   codes, scales = Q(x - pred);  hat = round16(pred + Q^-1(codes, scales)).
 // All row pointers address the start of the row.  pred_row == nullptr: no predictor.
 // hat_row == nullptr: reconstruction not wanted.  The prediction is read twice (for the residual and
@@ -616,7 +616,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) encode_rows_kernel(const Cod
   }
 }
 
-// This warp's part of one token row of Algorithm 3 line 5 / 7 given the prediction:
+// This warp's part of one token row of Algorithm 3 (keys or values) given the prediction:
 //   hat = round16(pred + Q^-1(codes, scales)).  words = this lane's packed codes per chunk, sf = the
 // scale of each chunk; get_pred(pq) delivers the prediction values of this lane just before they are
 // added, so a caller can fetch them while the rotation runs.

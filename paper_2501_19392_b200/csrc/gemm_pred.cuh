@@ -1,4 +1,4 @@
-// Predictor GEMM (Algorithm 2 lines 5 and 8, Algorithm 3 lines 5 and 7; Section 3.2: the
+// Predictor GEMM (the predictions of Algorithm 2 and Algorithm 3; Section 3.2: the
 // predictors are linear):  P[t][c] = sum_r X[t][r] * W[c][r] (+ bias[c]),  fp32 accumulate.
 //
 // X is the row-wise concatenation of up to two token-major 16-bit tensors (the value predictor

@@ -1,7 +1,7 @@
 // Backbone vector quantizer with the four-dimensional grid (Section 4.1 "Alternative quantizers": besides
-// the p = 2 grids the paper runs "one grid without fast GPU support (2-bit precision, d = 4, n = 256)";
-// its d is the grid dimension).  The steps are those of the p = 2 quantizer (Section 2; Algorithm 2
-// lines 6-7, 9 and Algorithm 3 lines 5, 7) with consecutive 4-tuples in place of pairs: root-mean-square
+// the p = 2 grids the paper runs one 2-bit grid with d = 4, n = 256, for which it had no fast GPU kernel;
+// its d is the grid dimension).  The steps are those of the p = 2 quantizer (Section 2; the residual / add-back
+// steps of Algorithm 2 and Algorithm 3) with consecutive 4-tuples in place of pairs: root-mean-square
 // group scale stored as fp16, normalisation with the rounded scale, random signs, Hadamard rotation in
 // blocks of h values, nearest of the 256 grid points (lowest index on a tie), one byte per tuple.
 //

@@ -1,5 +1,5 @@
 // One persistent kernel per layer call for Algorithm 2 (encode) and Algorithm 3 (decode) with
-// predictors: the predictor GEMMs (Algorithm 2 lines 5 and 8 / Algorithm 3 lines 5 and 7) run on
+// predictors: the predictor GEMMs (the two predictions of Algorithm 2 / Algorithm 3) run on
 // the tensor cores while, on the same SMs, other warps run the row work of the quantizer
 // (Section 2 "Vector Quantization") and of the reconstruction on tokens whose prediction is
 // already complete.  The fp32 prediction is handed from the GEMM warps to the row warps through a
@@ -30,7 +30,7 @@
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = tensor-memory owner + MMA issuer, warps 2..5 =
 // GEMM epilogue (tensor memory -> fp32 rows in the ring), then the row warps and, in the decoder
-// instantiation that also attends (Algorithm 4 lines 5-9), four attention warps: as soon as the value
+// instantiation that also attends (the attention read of Algorithm 4), four attention warps: as soon as the value
 // rows of the CTA's token block are reconstructed they read the block's keys and values back from
 // L2, form the single-query attention partials of the CTA's share of the KV heads for every sequence
 // the block overlaps, and release the block's rows (attn_done), so that decoded rows which the

@@ -1,6 +1,6 @@
 // Rotary position encoding of cached PRE-RoPE keys at attention time (Section 3.3 "Positional
 // embeddings": predictors and quantizers work on the keys before RoPE, so the reconstructed keys are
-// rotated when the block attends to them, Algorithm 4 lines 5-9).
+// rotated when the block attends to them in Algorithm 4).
 //
 // For a head of HD values and a token at position pos, frequency i < HD/2 has the angle
 // pos * theta_base^(-2 i / HD) and rotates the pair (x[i], x[i + HD/2]) (half-split pairing):

@@ -1,6 +1,6 @@
 // Row routines of the backbone quantizer Q / Q^-1 (Section 2 "Vector Quantization", Section 4.1
-// "Alternative quantizers") and of the residual / add-back steps of Algorithm 2 (lines 6-7, 9) and
-// Algorithm 3 (lines 5, 7) for the paper's main setting: d_kv = 1024 with the Hadamard block and the
+// "Alternative quantizers") and of the residual / add-back steps of Algorithm 2 and
+// Algorithm 3 for the paper's main setting: d_kv = 1024 with the Hadamard block and the
 // scale group spanning the whole token row.
 //
 // ONE warp owns a token row; each lane holds 32 of its 1024 values as 16 packed fp32 pairs.  The
@@ -197,7 +197,7 @@ __device__ __forceinline__ void wr_load_x_row(const uint16_t* __restrict__ x_row
   for (int ch = 0; ch < 4; ++ch) xraw[ch] = __ldcs(reinterpret_cast<const uint4*>(x_row + ch * 256 + lane * 8));   // read once
 }
 
-// One token row of Q and of the reconstruction (Algorithm 2 lines 6-7 / 9):
+// One token row of Q and of the reconstruction (Algorithm 2, keys or values):
 //   codes, scale = Q(x - pred);  hat = round16(pred + Q^-1(codes, scale)).
 // Row pointers address the start of the row.  pred_row == nullptr: no predictor.  hat_row == nullptr:
 // reconstruction not wanted.  The prediction is read twice (for the residual and again for the
@@ -357,7 +357,7 @@ __device__ __forceinline__ void wr_encode_row(const WarpRowCtx& rc, const RowSme
   wr_encode_row_x<NPTS, kBf16, false>(rc, rsm, xbuf, xraw, nullptr, pred_row, codes_row, scales_row, hat_row);
 }
 
-// One token row of Algorithm 3 line 5 / 7 given the prediction:
+// One token row of Algorithm 3 (keys or values) given the prediction:
 //   hat = round16(pred + Q^-1(codes, scale)).
 template <int NPTS, bool kBf16, bool kKeep = false, bool kEarly = false>
 __device__ __forceinline__ void wr_decode_row(const WarpRowCtx& rc, const f32x2_t* __restrict__ grid_s,

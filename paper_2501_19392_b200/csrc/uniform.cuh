@@ -1,7 +1,7 @@
-// Alternative backbone quantizer (Section 4.1 "Alternative quantizers": Quanto-style "simple
-// round-to-nearest quantization with absmax normalization", "group size 64 and per-token compression";
-// Section 3.2: the method is agnostic to the choice of Q) for the residual / add-back steps of
-// Algorithm 2 (lines 6-7, 9) and Algorithm 3 (lines 5, 7).
+// Alternative backbone quantizer (Section 4.1 "Alternative quantizers": the Quanto-style
+// one, plain rounding to the nearest level after dividing by the group's largest magnitude, groups of 64
+// values inside a token; Section 3.2: any quantizer Q can sit under the predictors) for the residual / add-back steps of
+// Algorithm 2 and Algorithm 3.
 //
 // For b bits per value the levels are the 2^b signed integers -2^(b-1) .. 2^(b-1)-1 times the group
 // scale; scale = absmax / 2^(b-1), stored as fp16 (clamped to 65504), and the ROUNDED scale normalises;
@@ -9,8 +9,8 @@
 // zeros has scale 0 and level 0.  The code of a value is level + 2^(b-1); codes are packed LSB-first in
 // value order.  No rotation, no sign flips.
 //
-// Rotated variant (the appendix' additional results for Section 4.1: a backbone that "combines Randomized
-// Hadamard Transform (RHT) with standard non-vector quantization", one group per row): had_block = h > 1
+// Rotated variant (the appendix' additional results for Section 4.1: a backbone that puts a randomized
+// Hadamard transform in front of ordinary scalar quantization, one group per row): had_block = h > 1
 // multiplies the residual by the role's random signs, rotates every block of h values by the orthonormal
 // Hadamard matrix, quantizes the ROTATED values as above (absmax after the rotation), and the inverse
 // rotates level * scale back and applies the signs again (kernels uniform_rot_*).

@@ -1,6 +1,6 @@
-"""Cache policy around the codec (Section 3.3; Section 4.1 "Evaluation setup": "we do not quantize the
-first 4 tokens (attention sinks) ... we also keep a buffer of 128 most recent tokens uncompressed";
-"the first layer is quantized at 4 bits"): the first `n_sink` tokens and the most recent tokens stay in
+"""Cache policy around the codec (Section 3.3; Section 4.1 "Evaluation setup": the first four
+tokens, the attention sinks, and a buffer of the 128 newest tokens are left uncompressed, and the first layer
+gets 4 bits per value): the first `n_sink` tokens and the most recent tokens stay in
 16 bits, older tokens are compressed in chunks of `chunk` tokens whenever the recent buffer holds
 `recent + chunk` of them, and every query attends to [compressed | sinks | recent] in one call.
 
@@ -117,7 +117,7 @@ class BufferedKVCache:
 
     def attend(self, q: List[torch.Tensor], n_kv_heads: int, softmax_scale: float,
                rope_table: Optional[torch.Tensor] = None) -> List[torch.Tensor]:
-        """Algorithm 4 lines 4-9 for every layer: q[l] [batch, n_q_heads, head_dim] -> outputs of the same shape.
+        """The decode-and-attend loop of Algorithm 4 for every layer: q[l] [batch, n_q_heads, head_dim] -> outputs of the same shape.
         The decoded compressed rows of layer l feed layer l + 1's predictors and are dropped afterwards.
         rope_table (Codec.rope_table): the cached keys are pre-RoPE and are rotated by their positions; q[l] must
         be rotated by the caller."""

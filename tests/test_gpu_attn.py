@@ -1,5 +1,5 @@
 """Parity of the fused decode + single-query attention entry point against the oracle's
-dequantize-then-attend (Algorithm 3 followed by Algorithm 4 lines 5-9)."""
+dequantize-then-attend (Algorithm 3 followed by the attention read of Algorithm 4)."""
 import dataclasses
 
 import numpy as np

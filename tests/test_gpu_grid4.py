@@ -1,5 +1,5 @@
-"""The backbone quantizer with the four-dimensional 256-point grid (Section 4.1: "one grid without fast
-GPU support (2-bit precision, d = 4, n = 256)") against its oracle: layer 0 (Q alone), teacher-forced key
+"""The backbone quantizer with the four-dimensional 256-point grid (Section 4.1: the 2-bit grid with
+d = 4, n = 256, for which the paper had no fast GPU kernel) against its oracle: layer 0 (Q alone), teacher-forced key
 and value phases with predictors, decode on the oracle's codes, the one-call entry points against the
 phases, edge rows.  Codes (one byte per 4 values) must equal the oracle's for every tuple whose margin
 (relative gap between the two smallest squared distances) exceeds 1e-4; scales and reconstructions follow

@@ -216,7 +216,7 @@ def test_full_size_call_on_sampled_rows(b, g, h):
 
 
 def test_fitted_predictors_help_this_backbone_too():
-    # Section 4.1 evaluates each backbone "with and without learned AQUA-KV predictors"
+    # Section 4.1 evaluates each backbone both with the learned predictors and without them
     from paper_2501_19392_b200 import api, calibrate as gcal
     d, b, g = 256, 2, 64
     codec, ora = make(d, b, g, oracle.BF16)

@@ -1,4 +1,4 @@
-"""Pins for the oracle's single-query attention over the decoded cache (Algorithm 4, lines 5-9):
+"""Pins for the oracle's single-query attention over the decoded cache (the attention read of Algorithm 4):
 scipy's softmax / logsumexp as library references and closed-form special cases."""
 import numpy as np
 import pytest

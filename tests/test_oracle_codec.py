@@ -55,7 +55,7 @@ def test_predictor_sizes_match_paper():
 
 @pytest.mark.parametrize("cfg", [1, 2])
 def test_zero_adapters_reduce_to_plain_rotated_vq(cfg):
-    # Algorithm 2 lines 1-3: layer 0 has no predictor; a zero matrix must give the same bits
+    # Algorithm 2, first layer: layer 0 has no predictor; a zero matrix must give the same bits
     shape, o, kv, ad = setup(cfg)
     K, V = synth.to_bits(kv.K[1]), synth.to_bits(kv.V[1])
     prevK, prevV = synth.to_bits(kv.K[0]), synth.to_bits(kv.V[0])
@@ -88,7 +88,7 @@ def test_identity_adapter_predicts_exactly():
 
 @pytest.mark.parametrize("cfg", [1, 2])
 def test_residual_is_target_minus_prediction(cfg):
-    # sign/ordering of Algorithm 2 line 6: Q acts on K - K_pred (not K_pred - K, not K)
+    # sign/ordering of Algorithm 2's residual: Q acts on K - K_pred (not K_pred - K, not K)
     shape, o, kv, ad = setup(cfg, bias=True)
     K, prevK = synth.to_bits(kv.K[1]), synth.to_bits(kv.K[0])
     Wk, bk = synth.to_bits(ad.Wk[1]), ad.bk[1].numpy()
@@ -106,7 +106,7 @@ def test_residual_is_target_minus_prediction(cfg):
 
 @pytest.mark.parametrize("cfg", [1, 2])
 def test_encode_then_decode_reproduces_encoders_reconstruction(cfg):
-    # Algorithm 2 line 7 and Algorithm 3 line 5 are the same expression
+    # Algorithm 2's reconstruction and Algorithm 3's decode are the same expression
     shape, o, kv, ad = setup(cfg, L=3)
     prevK = prevV = None
     for l in range(shape.n_layers):
