@@ -451,8 +451,8 @@ int aquakv_gather_rows(aquakv_ctx* ctx, int64_t n_rows, const int64_t* idx, int6
                        int64_t ld_src, void* dst, int64_t ld_dst, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
- * Calibration of one predictor (Algorithm 1, the two arg-min lines; Section 3.2: linear regression
- * with "closed-form training"; Appendix A: "closed form solution with regularizer rate 1e-3"):
+ * Calibration of one predictor (Algorithm 1, its two least-squares fits; Section 3.2: linear regressors
+ * trained in closed form; Appendix A: the regularizer rate is 1e-3):
  *
  *   W = argmin_W || [in0 ; in1] W^T (+ b) - target ||^2 + rate * trace(X^T X) / n_in * ||W||^2
  *

@@ -5,8 +5,8 @@ statement per step of the paper's procedure, no blocking.  The CUDA library neve
 
 What it computes.  For one layer the key predictor is the linear map that minimises
 ||f(K_old) - K||^2 over the calibration tokens, the value predictor the one that minimises
-||f([V_old ; K_rec]) - V||^2 (Algorithm 1: "Predict keys from past keys", "Predict values from past
-values and current keys"), both fitted "via closed form solution with regularizer rate 1e-3"
+||f([V_old ; K_rec]) - V||^2 (Algorithm 1: keys from the previous layer's keys, values from the
+previous layer's values and the current keys), both fitted in closed form with the regularizer rate 1e-3
 (Appendix A).  Layers are fitted one after another on RECONSTRUCTED inputs: K_rec = f_key(K_old) +
 Q^-1(Q(K - f_key(K_old))) is produced by the codec oracle itself (Section 3.2: "Each subsequent set
 of predictors is trained using reconstructed cache entries as inputs").

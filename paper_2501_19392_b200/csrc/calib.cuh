@@ -1,5 +1,5 @@
-// Predictor calibration (Algorithm 1, the two arg-min lines; Section 3.2: "simple linear regression
-// ... closed-form training"; Appendix A: "closed form solution with regularizer rate 1e-3"):
+// Predictor calibration (Algorithm 1, its two least-squares fits; Section 3.2: linear regressors that are
+// trained in closed form; Appendix A: the regularizer rate is 1e-3):
 //
 //   W = argmin_W || X W^T (+ b) - Y ||^2 + rate * trace(X^T X) / n_in * ||W||^2
 //
