@@ -67,7 +67,7 @@ def ridge_fit(X: np.ndarray, Y: np.ndarray, rate: float = 1e-3,
     """argmin_W ||X W^T (+ b) - Y||^2 + rate * trace(X^T X)/n_in * ||W||^2 in double precision.
 
     X [T, n_in], Y [T, d_out] float64.  Returns W [d_out, n_in] (a linear layer's weight) and the
-    intercept b [d_out] or None.  (Algorithm 1, the two arg-min lines; Appendix A for the rate.)
+    intercept b [d_out] or None.  (Algorithm 1, its two least-squares fits; Appendix A for the rate.)
     """
     X = np.asarray(X, dtype=np.float64)
     Y = np.asarray(Y, dtype=np.float64)
