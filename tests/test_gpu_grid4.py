@@ -134,6 +134,47 @@ def test_full_size_call_on_sampled_rows():
     assert torch.equal(Kh2, Kh) and torch.equal(Vh2, Vh)
 
 
+def test_tuples_outside_the_search_table_and_many_plain_rows():
+    """The encoder finds a tuple's candidates in a table over [-4, 4)^4 and searches all 256 points for
+    tuples outside it and for cells with more than 15 candidates.  Rows built so that a few percent of their
+    rotated, normalised tuples lie outside the table (coordinates up to +-5), and 2000 plain Gaussian rows (about 40 of
+    their half a million tuples fall into crowded cells, about 80 outside the table), must give the oracle's
+    codes wherever its margin is clear."""
+    from paper_2501_19392_b200 import api
+    from oracle.uniform import rotate_back
+    d, h, g = 1024, 256, 1024
+    codec, ora = make(d, h, g, oracle.BF16)
+    rng = np.random.default_rng(11)
+    Y = rng.standard_normal((64, d))
+    far = rng.random((64, d // 4)) < 0.1
+    Y = Y.reshape(64, d // 4, 4)
+    Y[far] = rng.choice([-1.0, 1.0], size=(int(far.sum()), 4)) * rng.uniform(4.2, 7.0, size=(int(far.sum()), 4)) \
+        * (rng.random((int(far.sum()), 4)) < 0.5) + Y[far] * 0.3
+    Y = Y.reshape(64, d)
+    Y /= np.sqrt((Y ** 2).mean(axis=1, keepdims=True))             # unit root mean square: the scale is then s
+    R = 0.37 * rotate_back(Y, synth.hadamard_signs(d, 1), h)
+    X = torch.from_numpy(R).to(torch.bfloat16)
+    o = ora.encode_phase(synth.to_bits(X), [], None, role="k")
+    outside = (np.abs(o["Y"].reshape(64, d // 4, 4)) >= 4.0).any(axis=2)
+    assert outside.mean() > 0.02                                   # the rows do reach beyond the table
+    Kc, Ks, Kh = codec.encode_phase(api.ROLE_KEY, X.to(DEV))
+    rows_ok, _ = scale_rows_ok(gpu_bits(Ks.view(torch.float16)), o["scales"], o["scales_exact"])
+    clear = (o["margins"] > MARGIN) & rows_ok[:, None]
+    got = Kc.cpu().numpy()
+    assert np.array_equal(got[clear], o["codes"][clear])
+    assert clear[outside].mean() > 0.9 and np.array_equal(got[clear & outside], o["codes"][clear & outside])
+    same = rows_ok & (got == o["codes"]).all(axis=1)
+    check_recon(gpu_bits(Kh), o["hat_exact"], o["hat"], oracle.BF16, same)
+    # many plain rows
+    Xg = synth.random_16bit((2000, d), oracle.BF16, 12)
+    og = ora.encode_phase(synth.to_bits(Xg), [], None, role="v")
+    Vc, Vs, Vh = codec.encode_phase(api.ROLE_VALUE, Xg.to(DEV))
+    rows_ok, _ = scale_rows_ok(gpu_bits(Vs.view(torch.float16)), og["scales"], og["scales_exact"])
+    same = check_tuples(Vc.cpu().numpy(), og, rows_ok)
+    check_recon(gpu_bits(Vh), og["hat_exact"], og["hat"], oracle.BF16, same)
+    assert codec.poll_status() == 0
+
+
 def test_zero_rows_clamped_scale_and_rows_on_grid_points():
     from paper_2501_19392_b200 import api
     d, h, g = 256, 256, 256
