@@ -172,3 +172,17 @@ def test_decode_attn_at_the_full_llama31_8b_shape():
     near = np.abs(gpu_bits(out).astype(np.int64) - gpu_bits(out2).astype(np.int64)) <= 1
     assert np.all((np.abs(o1 - o2) <= 2e-3 * np.abs(o1).max(axis=-1, keepdims=True)) | near)
     assert (lse - lse2).abs().max().item() <= 1e-4
+
+
+def test_attention_mode_switch_rejects_unknown_modes():
+    from paper_2501_19392_b200 import api
+    d = 1024
+    grid = synth.lloyd_grid(16, seed=7, n_samples=1 << 12, iters=5)
+    codec = api.Codec(d, d, d, grid, synth.BF16, synth.hadamard_signs(d, 11), synth.hadamard_signs(d, 12))
+    for bad in (-1, 2, 7):
+        with pytest.raises(api.AquaKVError) as e:
+            codec.set_attn_mode(bad)
+        assert e.value.status == -1
+    codec.set_attn_mode(api.ATTN_FUSED)
+    codec.set_attn_mode(api.ATTN_SPLIT)
+    assert codec.poll_status() == 0
